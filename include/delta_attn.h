@@ -1,0 +1,201 @@
+/*
+ * delta_attn.h -- C ABI of the B200 (sm_100a) delta-attention library.
+ *
+ * The library computes DeltaLLM's hybrid attention (arXiv 2507.19608): the query stream of
+ * every head is turned into a thresholded delta matrix against a carried reference state
+ * (Section II-C, Eq. 2-3; construction strategy (1) of Section III-A), attention scores for
+ * keys outside a context window come from the running sum of sparse delta products (Eq. 4),
+ * scores inside the window are the full q.k (Section III-B), then scale, causal softmax and
+ * the product with V (Eq. 1).  Prefill and single-token decode share one state object
+ * (Section III-C; the decode state of strategy (1) is the reference query and the previous
+ * score row, Section III-A "Decoding Stage Considerations").
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise:
+ *   - pointers named q, k, v, out, *_cache, *_new, workspace are DEVICE pointers to memory the
+ *     caller owns; the library never allocates or frees device memory;
+ *   - `stream` is a cudaStream_t passed as void*; calls only enqueue work on it and return
+ *     (delta_sparsity_stats and the *_host entry point synchronise it);
+ *   - every function returns a delta_status_t; on any error nothing is launched and the state
+ *     is left as it was;
+ *   - tensors are contiguous, row-major, element type from delta_config_t.dtype
+ *     (DELTA_F32: float, DELTA_BF16: bfloat16 bit patterns);
+ *   - query head h reads KV head h / (H / H_kv).
+ */
+#ifndef DELTA_ATTN_H_
+#define DELTA_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(DELTA_BUILDING_LIB) && defined(__GNUC__)
+#define DELTA_API __attribute__((visibility("default")))
+#else
+#define DELTA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Rows per delta tile: per-tile non-zero counters and per-tile reference snapshots use it. */
+#define DELTA_TILE_ROWS 64
+
+typedef enum {
+  DELTA_OK = 0,
+  DELTA_ERR_INVALID_ARG = 1,  /* null pointer, bad size, theta < 0 or not finite, ...          */
+  DELTA_ERR_UNSUPPORTED = 2,  /* a configuration this build has no kernel for                  */
+  DELTA_ERR_WORKSPACE = 3,    /* workspace too small or not 256-byte aligned                   */
+  DELTA_ERR_CAPACITY = 4,     /* sequence would exceed T_max                                   */
+  DELTA_ERR_STATE = 5,        /* call order: prefill on a used state, decode before prefill    */
+  DELTA_ERR_CUDA = 6,         /* a CUDA runtime call failed (delta_last_cuda_error has it)     */
+  DELTA_ERR_TIMEOUT = 7       /* a bounded device-side wait ran out (status word on device)    */
+} delta_status_t;
+
+typedef enum { DELTA_F32 = 0, DELTA_BF16 = 1 } delta_dtype_t;
+
+/* Which operand becomes the delta matrix (Section III-A).  QUERY = strategy (1), top-down
+ * query deltas; KEY = strategy (3), reserved (returns DELTA_ERR_UNSUPPORTED). */
+typedef enum { DELTA_SRC_QUERY = 0, DELTA_SRC_KEY = 1 } delta_source_t;
+
+/* Shape of the exact-attention region in prefill (Section III-B).  BLOCK: squares of side
+ * `window` along the diagonal, anchored at token 0 (pair (i,j) is exact iff i/W == j/W).
+ * SLIDING: the `window` most recent keys of every query (exact iff i - j < W).  window = 0
+ * means no exact score at all; window >= T means dense attention.  Decode always uses
+ * SLIDING (the W_d most recent tokens, the new one included). */
+typedef enum { DELTA_WIN_BLOCK = 0, DELTA_WIN_SLIDING = 1 } delta_window_shape_t;
+
+/* Treatment of row 0 in Eq. 2-3.  BASIS_EXACT: the first vector is the un-thresholded basis
+ * (Delta q(0) = q(0), reference = q(0), all mask bits set).  ZERO_STATE: the reference
+ * starts at 0 and row 0 is thresholded like every other row. */
+typedef enum { DELTA_INIT_BASIS_EXACT = 0, DELTA_INIT_ZERO_STATE = 1 } delta_init_t;
+
+typedef struct {
+  int32_t B;      /* batch elements                                     */
+  int32_t H;      /* query heads                                        */
+  int32_t H_kv;   /* key/value heads, H % H_kv == 0, H / H_kv <= 8      */
+  int32_t d;      /* head dimension, 64 or 128                          */
+  int32_t T_max;  /* capacity in tokens (prefill length + decode steps) */
+  delta_dtype_t dtype;
+  delta_source_t source;
+  delta_window_shape_t prefill_window;
+  delta_init_t init;
+} delta_config_t;
+
+/* Opaque host object; owns no device memory (everything lives in the caller's workspace). */
+typedef struct delta_state delta_state_t;
+
+/* Bytes of device workspace a state with this configuration needs (multiple of 256). */
+DELTA_API delta_status_t delta_state_workspace_bytes(const delta_config_t* cfg, size_t* bytes);
+
+/* delta_state_init -- create a state over a caller-owned device workspace (256-byte aligned,
+ * at least delta_state_workspace_bytes large) and enqueue the zeroing of the reference state
+ * q_hat, the score row R and all counters (Eq. 3: the reference starts at 0).  *out is a host
+ * object the caller releases with delta_state_destroy; the workspace must outlive it. */
+DELTA_API delta_status_t delta_state_init(const delta_config_t* cfg, void* workspace, size_t workspace_bytes,
+                                void* stream, delta_state_t** out);
+
+/* Back to the freshly initialised condition (position 0, counters 0). */
+DELTA_API delta_status_t delta_state_reset(delta_state_t* st, void* stream);
+
+/* Frees the host object only. */
+DELTA_API delta_status_t delta_state_destroy(delta_state_t* st);
+
+/* delta_attn_prefill -- hybrid delta attention over T tokens (Section III, prefilling stage).
+ *   q, out : [B, H, T, d]            k, v : [B, H_kv, T_max, d] (KV-cache layout, rows 0..T-1 read)
+ *   theta  : delta threshold of Eq. 2 (>= 0, finite); |diff| == theta does not fire
+ *   window : W of Section III-B (>= 0), shape from the configuration
+ * Steps enqueued: delta construction over Q (Eq. 2-3: values, bit mask, per-row and per-tile
+ * non-zero counts, compacted channel indices, per-tile reference snapshots), the fused
+ * hybrid-attention kernel (exact q.k inside the window, running delta sums outside (Eq. 4),
+ * scale 1/sqrt(d), causal online softmax, P.V (Eq. 1)), the hand-off of q_hat(T-1) and
+ * R(T-1)[0..T-1] for decode, and the sparsity counters (Eq. 6).
+ * H, H_kv, d must equal the configuration.  Needs a fresh or reset state (else
+ * DELTA_ERR_STATE); 1 <= T <= T_max (else DELTA_ERR_CAPACITY). */
+DELTA_API delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* k, const void* v,
+                                  void* out, int32_t T, int32_t H, int32_t H_kv, int32_t d,
+                                  float theta, int32_t window, void* stream);
+
+/* delta_attn_prefill_host -- the same call for HOST buffers (q, k, v, out are host pointers
+ * with the shapes above; k and v hold T rows per head, i.e. [B, H_kv, T, d]).  `staging` is
+ * a DEVICE buffer of at least delta_prefill_staging_bytes(cfg, T) bytes that receives the
+ * copies.  Copies in, runs the prefill, copies `out` back and synchronises the stream. */
+DELTA_API delta_status_t delta_prefill_staging_bytes(const delta_config_t* cfg, int32_t T, size_t* bytes);
+DELTA_API delta_status_t delta_attn_prefill_host(delta_state_t* st, const void* q_host, const void* k_host,
+                                       const void* v_host, void* out_host, void* staging,
+                                       size_t staging_bytes, int32_t T, float theta,
+                                       int32_t window, void* stream);
+
+/* delta_attn_decode_step -- one decoding step for every (batch, head) (Section III-B/C,
+ * decoding stage, carried state of strategy (1)).
+ *   q_new, out : [B, H, d]     k_new, v_new : [B, H_kv, d]
+ *   k_cache, v_cache : [B, H_kv, T_max, d]; rows 0..n-1 are read, row n is written by the call
+ * With n the tokens seen so far: Delta q = threshold(q_new - q_hat) and q_hat update (Eq. 2-3);
+ * R[j] += Delta q . k_j for every cached key j < n (Eq. 4); R[n] = q_hat . k_new for the key
+ * that arrives now; score j is q_new.k_j if n - j < window else R[j]; softmax over the n + 1
+ * keys; out = P.V; position becomes n + 1.  Needs n >= 1 (else DELTA_ERR_STATE) and
+ * n < T_max (else DELTA_ERR_CAPACITY). */
+DELTA_API delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, const void* k_new,
+                                      const void* v_new, void* k_cache, void* v_cache, void* out,
+                                      float theta, int32_t window, void* stream);
+
+/* Counters of one stage.  S_m = 1 - nnz/elements (sparsity of the delta matrix, Eq. 6);
+ * S_c_eq6 = S_m * (1 - W/n) (Eq. 6); S_c_exact = 1 - macs_done/macs_dense where a causal
+ * pair costs d multiply-adds inside the window and nnz(Delta q_i) outside it, against d for
+ * every causal pair of dense attention. */
+typedef struct {
+  uint64_t nnz, elements, macs_done, macs_dense;
+  double S_m, S_c_eq6, S_c_exact;
+} delta_stage_stats_t;
+
+typedef struct {
+  delta_stage_stats_t prefill, decode, combined;
+  int32_t n;             /* tokens seen so far */
+  uint32_t device_status; /* 0, or the DELTA_ERR_* a kernel recorded in the device status word */
+} delta_stats_t;
+
+/* delta_sparsity_stats -- copy the device counters to the host and finish Eq. 6.
+ * Synchronises `stream`.  host_out is a HOST pointer. */
+DELTA_API delta_status_t delta_sparsity_stats(const delta_state_t* st, delta_stats_t* host_out, void* stream);
+
+/* Eq. 5: W_p,max = min(floor(gamma * n), w_max). */
+DELTA_API int32_t delta_window_from_gamma(int32_t n, float gamma, int32_t w_max);
+
+/* Device views into the state's workspace, for parity checks and checkpointing.
+ * Shapes (T_max rows allocated, rows 0..T-1 valid after a prefill of T tokens):
+ *   DQ        float    [B, H, T_max, d]        Delta q(t), +0.0 where not fired
+ *   MASK      uint32   [B, H, T_max, d/32]     bit (c % 32) of word (c / 32)
+ *   ROW_NNZ   uint16   [B, H, T_max]
+ *   TILE_NNZ  uint32   [B, H, ceil(T_max/64)]
+ *   IDX       uint8    [B, H, T_max, d]        fired channel ids ascending, 0xFF padding
+ *   QHAT_TILE float    [B, H, ceil(T_max/64), d]  reference state before each tile's first row
+ *   QHAT      float    [B, H, d]               current reference state
+ *   R         float    [B, H, T_max]           current score row (un-scaled), entries 0..n-1
+ */
+typedef enum {
+  DELTA_VIEW_DQ = 0, DELTA_VIEW_MASK = 1, DELTA_VIEW_ROW_NNZ = 2, DELTA_VIEW_TILE_NNZ = 3,
+  DELTA_VIEW_IDX = 4, DELTA_VIEW_QHAT_TILE = 5, DELTA_VIEW_QHAT = 6, DELTA_VIEW_R = 7
+} delta_view_t;
+DELTA_API delta_status_t delta_state_view(const delta_state_t* st, int32_t what, const void** dev_ptr,
+                                size_t* bytes);
+
+/* Tokens seen so far (0 after init/reset). */
+DELTA_API int32_t delta_state_position(const delta_state_t* st);
+
+/* Which prefill kernel the next delta_attn_prefill on this state will use:
+ * 0 = generic CUDA-core kernel, 1 = tcgen05/TMA kernel.  delta_state_set_prefill_kernel
+ * forces one (-1 = automatic); forcing a kernel the configuration has none for returns
+ * DELTA_ERR_UNSUPPORTED. */
+DELTA_API int32_t delta_state_prefill_kernel(const delta_state_t* st);
+DELTA_API delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which);
+
+/* Kernels launched by this library in the calling process since it was loaded. */
+DELTA_API uint64_t delta_launch_count(void);
+
+DELTA_API const char* delta_status_string(delta_status_t s);
+/* Text of the last CUDA runtime error seen by this library in the calling thread. */
+DELTA_API const char* delta_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DELTA_ATTN_H_ */

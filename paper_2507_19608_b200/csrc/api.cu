@@ -1,0 +1,345 @@
+// C ABI of the delta-attention library: argument checks, workspace carving, launch order.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "delta_internal.cuh"
+#include "k2_tc.cuh"
+
+namespace delta {
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+static thread_local char g_cuda_err[256] = "";
+static delta_status_t cuda_fail(cudaError_t e) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+  return DELTA_ERR_CUDA;
+}
+}  // namespace delta
+
+using namespace delta;
+
+struct delta_state {
+  delta_config_t cfg;
+  Shape shape;
+  Workspace ws;
+  void* base;
+  size_t bytes;
+  int n;         // tokens seen
+  int qhat_sel;  // which q_hat buffer is current
+  int forced_kernel;  // -1 auto, 0 generic, 1 tensor-core
+  // Eq. 6 bookkeeping that needs no device work: sum of window lengths and sequence lengths
+  double win_sum[2], len_sum[2];
+};
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static delta_status_t check_config(const delta_config_t* c) {
+  if (!c) return DELTA_ERR_INVALID_ARG;
+  if (c->B < 1 || c->H < 1 || c->H_kv < 1 || c->T_max < 1) return DELTA_ERR_INVALID_ARG;
+  if (c->H % c->H_kv != 0) return DELTA_ERR_INVALID_ARG;
+  if (c->dtype != DELTA_F32 && c->dtype != DELTA_BF16) return DELTA_ERR_INVALID_ARG;
+  if (c->prefill_window != DELTA_WIN_BLOCK && c->prefill_window != DELTA_WIN_SLIDING)
+    return DELTA_ERR_INVALID_ARG;
+  if (c->init != DELTA_INIT_BASIS_EXACT && c->init != DELTA_INIT_ZERO_STATE)
+    return DELTA_ERR_INVALID_ARG;
+  if (c->source != DELTA_SRC_QUERY && c->source != DELTA_SRC_KEY) return DELTA_ERR_INVALID_ARG;
+  if (c->source == DELTA_SRC_KEY) return DELTA_ERR_UNSUPPORTED;
+  if (c->d != 64 && c->d != 128) return DELTA_ERR_UNSUPPORTED;
+  const int g = c->H / c->H_kv;
+  if (g != 1 && g != 2 && g != 4 && g != 8) return DELTA_ERR_UNSUPPORTED;
+  if (c->T_max > kMaxDecodeSplits * kDecodeChunkMax) return DELTA_ERR_UNSUPPORTED;
+  if ((long long)c->B * c->H > 65535) return DELTA_ERR_UNSUPPORTED;
+  return DELTA_OK;
+}
+
+// Carve the workspace; base may be null (size query).
+static void carve(const delta_config_t& c, char* base, Workspace* w) {
+  const size_t BH = (size_t)c.B * c.H, BKV = (size_t)c.B * c.H_kv;
+  const size_t nt = (c.T_max + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
+  const size_t g = c.H / c.H_kv;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off += align_up(bytes, 256); return p; };
+  w->dq = (float*)take(BH * c.T_max * c.d * 4);
+  w->mask = (uint32_t*)take(BH * c.T_max * (c.d / 32) * 4);
+  w->row_nnz = (uint16_t*)take(BH * c.T_max * 2);
+  w->tile_nnz = (uint32_t*)take(BH * nt * 4);
+  w->idx = (uint8_t*)take(BH * c.T_max * c.d);
+  w->qhat_tile = (float*)take(BH * nt * c.d * 4);
+  w->qhat[0] = (float*)take(BH * c.d * 4);
+  w->qhat[1] = (float*)take(BH * c.d * 4);
+  w->R = (float*)take(BH * c.T_max * 4);
+  w->counters = (unsigned long long*)take(CNT_SLOTS * 8);
+  w->dec_partial = (float*)take(BKV * kMaxDecodeSplits * g * (c.d + 2) * 4);
+  w->dec_ticket = (uint32_t*)take(BKV * 4);
+  w->qhat_tile_bf16 = (c.dtype == DELTA_BF16) ? (__nv_bfloat16*)take(BH * nt * c.d * 2) : nullptr;
+  w->total_bytes = off;
+}
+
+extern "C" {
+
+delta_status_t delta_state_workspace_bytes(const delta_config_t* cfg, size_t* bytes) {
+  if (!bytes) return DELTA_ERR_INVALID_ARG;
+  delta_status_t s = check_config(cfg);
+  if (s != DELTA_OK) return s;
+  Workspace w;
+  carve(*cfg, nullptr, &w);
+  *bytes = w.total_bytes;
+  return DELTA_OK;
+}
+
+static delta_status_t zero_state(delta_state* st, cudaStream_t stream) {
+  const delta_config_t& c = st->cfg;
+  const size_t BH = (size_t)c.B * c.H;
+  cudaError_t e;
+  if ((e = cudaMemsetAsync(st->ws.qhat[0], 0, BH * c.d * 4, stream)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemsetAsync(st->ws.qhat[1], 0, BH * c.d * 4, stream)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemsetAsync(st->ws.R, 0, BH * c.T_max * 4, stream)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemsetAsync(st->ws.counters, 0, CNT_SLOTS * 8, stream)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemsetAsync(st->ws.dec_ticket, 0, (size_t)c.B * c.H_kv * 4, stream)) != cudaSuccess)
+    return cuda_fail(e);
+  st->n = 0;
+  st->qhat_sel = 0;
+  st->win_sum[0] = st->win_sum[1] = st->len_sum[0] = st->len_sum[1] = 0.0;
+  return DELTA_OK;
+}
+
+delta_status_t delta_state_init(const delta_config_t* cfg, void* workspace, size_t workspace_bytes,
+                                void* stream, delta_state_t** out) {
+  if (!out) return DELTA_ERR_INVALID_ARG;
+  *out = nullptr;
+  delta_status_t s = check_config(cfg);
+  if (s != DELTA_OK) return s;
+  if (!workspace) return DELTA_ERR_INVALID_ARG;
+  if (((uintptr_t)workspace & 255u) != 0) return DELTA_ERR_WORKSPACE;
+  Workspace w;
+  carve(*cfg, (char*)workspace, &w);
+  if (workspace_bytes < w.total_bytes) return DELTA_ERR_WORKSPACE;
+  delta_state* st = new (std::nothrow) delta_state();
+  if (!st) return DELTA_ERR_INVALID_ARG;
+  st->cfg = *cfg;
+  st->shape = Shape{cfg->B, cfg->H, cfg->H_kv, cfg->d, cfg->T_max,
+                    (cfg->T_max + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS};
+  st->ws = w;
+  st->base = workspace;
+  st->bytes = workspace_bytes;
+  st->forced_kernel = -1;
+  s = zero_state(st, (cudaStream_t)stream);
+  if (s != DELTA_OK) { delete st; return s; }
+  *out = st;
+  return DELTA_OK;
+}
+
+delta_status_t delta_state_reset(delta_state_t* st, void* stream) {
+  if (!st) return DELTA_ERR_INVALID_ARG;
+  return zero_state(st, (cudaStream_t)stream);
+}
+
+delta_status_t delta_state_destroy(delta_state_t* st) {
+  if (!st) return DELTA_ERR_INVALID_ARG;
+  delete st;
+  return DELTA_OK;
+}
+
+int32_t delta_state_position(const delta_state_t* st) { return st ? st->n : -1; }
+
+static bool tc_eligible(const delta_state* st) {
+  return st->cfg.dtype == DELTA_BF16 && tc_kernel_available(st->cfg.d);
+}
+
+int32_t delta_state_prefill_kernel(const delta_state_t* st) {
+  if (!st) return -1;
+  if (st->forced_kernel >= 0) return st->forced_kernel;
+  return tc_eligible(st) ? 1 : 0;
+}
+
+delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
+  if (!st || which < -1 || which > 1) return DELTA_ERR_INVALID_ARG;
+  if (which == 1 && !tc_eligible(st)) return DELTA_ERR_UNSUPPORTED;
+  st->forced_kernel = which;
+  return DELTA_OK;
+}
+
+static delta_status_t check_theta_window(float theta, int32_t window) {
+  if (!(theta >= 0.0f) || !std::isfinite(theta)) return DELTA_ERR_INVALID_ARG;
+  if (window < 0) return DELTA_ERR_INVALID_ARG;
+  return DELTA_OK;
+}
+
+delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* k, const void* v,
+                                  void* out, int32_t T, int32_t H, int32_t H_kv, int32_t d,
+                                  float theta, int32_t window, void* stream) {
+  if (!st || !q || !k || !v || !out) return DELTA_ERR_INVALID_ARG;
+  const delta_config_t& c = st->cfg;
+  if (H != c.H || H_kv != c.H_kv || d != c.d) return DELTA_ERR_INVALID_ARG;
+  delta_status_t s = check_theta_window(theta, window);
+  if (s != DELTA_OK) return s;
+  if (T < 1) return DELTA_ERR_INVALID_ARG;
+  if (T > c.T_max) return DELTA_ERR_CAPACITY;
+  if (st->n != 0) return DELTA_ERR_STATE;
+  cudaStream_t cs = (cudaStream_t)stream;
+  cudaError_t e;
+  if ((e = launch_delta_construct(st->shape, st->ws, q, T, theta, c.dtype, c.init, cs)) != cudaSuccess)
+    return cuda_fail(e);
+  if ((e = launch_prefill_stats(st->shape, st->ws, T, window, c.prefill_window, cs)) != cudaSuccess)
+    return cuda_fail(e);
+  if (delta_state_prefill_kernel(st) == 1) {
+    e = launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
+  } else {
+    e = launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window,
+                                   c.dtype, cs);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  if ((e = launch_handoff(st->shape, st->ws, k, T, c.dtype, 0, cs)) != cudaSuccess) return cuda_fail(e);
+  st->n = T;
+  st->qhat_sel = 0;
+  st->win_sum[0] += (double)(window < T ? window : T);
+  st->len_sum[0] += (double)T;
+  return DELTA_OK;
+}
+
+delta_status_t delta_prefill_staging_bytes(const delta_config_t* cfg, int32_t T, size_t* bytes) {
+  if (!bytes) return DELTA_ERR_INVALID_ARG;
+  delta_status_t s = check_config(cfg);
+  if (s != DELTA_OK) return s;
+  if (T < 1 || T > cfg->T_max) return DELTA_ERR_INVALID_ARG;
+  const size_t es = cfg->dtype == DELTA_F32 ? 4 : 2;
+  const size_t qb = align_up((size_t)cfg->B * cfg->H * T * cfg->d * es, 256);
+  const size_t kb = align_up((size_t)cfg->B * cfg->H_kv * cfg->T_max * cfg->d * es, 256);
+  *bytes = 2 * qb + 2 * kb;
+  return DELTA_OK;
+}
+
+delta_status_t delta_attn_prefill_host(delta_state_t* st, const void* q_host, const void* k_host,
+                                       const void* v_host, void* out_host, void* staging,
+                                       size_t staging_bytes, int32_t T, float theta,
+                                       int32_t window, void* stream) {
+  if (!st || !q_host || !k_host || !v_host || !out_host || !staging) return DELTA_ERR_INVALID_ARG;
+  const delta_config_t& c = st->cfg;
+  size_t need = 0;
+  delta_status_t s = delta_prefill_staging_bytes(&c, T, &need);
+  if (s != DELTA_OK) return s;
+  if (staging_bytes < need || ((uintptr_t)staging & 255u)) return DELTA_ERR_WORKSPACE;
+  if (st->n != 0) return DELTA_ERR_STATE;
+  s = check_theta_window(theta, window);
+  if (s != DELTA_OK) return s;
+  const size_t es = c.dtype == DELTA_F32 ? 4 : 2;
+  const size_t q_bytes = (size_t)c.B * c.H * T * c.d * es;
+  const size_t qb = align_up(q_bytes, 256);
+  const size_t kb = align_up((size_t)c.B * c.H_kv * c.T_max * c.d * es, 256);
+  char* dq_ = (char*)staging;
+  char* dout = dq_ + qb;
+  char* dk = dout + qb;
+  char* dv = dk + kb;
+  cudaStream_t cs = (cudaStream_t)stream;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(dq_, q_host, q_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
+  // host K/V hold T rows per head; the device copy uses the cache layout with T_max rows
+  const size_t row = (size_t)c.d * es;
+  if ((e = cudaMemcpy2DAsync(dk, (size_t)c.T_max * row, k_host, (size_t)T * row, (size_t)T * row,
+                             (size_t)c.B * c.H_kv, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpy2DAsync(dv, (size_t)c.T_max * row, v_host, (size_t)T * row, (size_t)T * row,
+                             (size_t)c.B * c.H_kv, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
+  s = delta_attn_prefill(st, dq_, dk, dv, dout, T, c.H, c.H_kv, c.d, theta, window, stream);
+  if (s != DELTA_OK) return s;
+  if ((e = cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, cs)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaStreamSynchronize(cs)) != cudaSuccess) return cuda_fail(e);
+  return DELTA_OK;
+}
+
+delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, const void* k_new,
+                                      const void* v_new, void* k_cache, void* v_cache, void* out,
+                                      float theta, int32_t window, void* stream) {
+  if (!st || !q_new || !k_new || !v_new || !k_cache || !v_cache || !out) return DELTA_ERR_INVALID_ARG;
+  delta_status_t s = check_theta_window(theta, window);
+  if (s != DELTA_OK) return s;
+  if (st->n < 1) return DELTA_ERR_STATE;
+  if (st->n >= st->cfg.T_max) return DELTA_ERR_CAPACITY;
+  cudaError_t e = launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out,
+                                     st->n, theta, window, st->cfg.dtype, st->qhat_sel,
+                                     (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const int L = st->n + 1;
+  st->win_sum[1] += (double)(window < L ? window : L);
+  st->len_sum[1] += (double)L;
+  st->qhat_sel ^= 1;
+  st->n += 1;
+  return DELTA_OK;
+}
+
+static void finish_stage(delta_stage_stats_t* o, const unsigned long long* c, double win, double len) {
+  o->nnz = c[0]; o->elements = c[1]; o->macs_done = c[2]; o->macs_dense = c[3];
+  o->S_m = o->elements ? 1.0 - (double)o->nnz / (double)o->elements : 0.0;
+  o->S_c_eq6 = len > 0.0 ? o->S_m * (1.0 - win / len) : 0.0;
+  o->S_c_exact = o->macs_dense ? 1.0 - (double)o->macs_done / (double)o->macs_dense : 0.0;
+}
+
+delta_status_t delta_sparsity_stats(const delta_state_t* st, delta_stats_t* host_out, void* stream) {
+  if (!st || !host_out) return DELTA_ERR_INVALID_ARG;
+  unsigned long long c[CNT_SLOTS];
+  cudaError_t e = cudaMemcpyAsync(c, st->ws.counters, sizeof(c), cudaMemcpyDeviceToHost,
+                                  (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaStreamSynchronize((cudaStream_t)stream)) != cudaSuccess) return cuda_fail(e);
+  memset(host_out, 0, sizeof(*host_out));
+  finish_stage(&host_out->prefill, c + CNT_PREFILL_NNZ, st->win_sum[0], st->len_sum[0]);
+  finish_stage(&host_out->decode, c + CNT_DECODE_NNZ, st->win_sum[1], st->len_sum[1]);
+  unsigned long long sum[4];
+  for (int i = 0; i < 4; ++i) sum[i] = c[CNT_PREFILL_NNZ + i] + c[CNT_DECODE_NNZ + i];
+  finish_stage(&host_out->combined, sum, 0.0, 0.0);
+  // combined Eq. 6 value: the stages' Eq. 6 values weighted by their dense multiply-adds
+  const double dp = (double)host_out->prefill.macs_dense, dd = (double)host_out->decode.macs_dense;
+  host_out->combined.S_c_eq6 =
+      (dp + dd) > 0.0 ? (host_out->prefill.S_c_eq6 * dp + host_out->decode.S_c_eq6 * dd) / (dp + dd) : 0.0;
+  host_out->n = st->n;
+  host_out->device_status = (uint32_t)c[CNT_STATUS];
+  return host_out->device_status == 0 ? DELTA_OK : (delta_status_t)host_out->device_status;
+}
+
+int32_t delta_window_from_gamma(int32_t n, float gamma, int32_t w_max) {
+  if (n < 0 || !(gamma >= 0.0f)) return 0;
+  const double w = std::floor((double)gamma * (double)n);
+  const double m = w < (double)w_max ? w : (double)w_max;
+  return m < 0.0 ? 0 : (int32_t)m;
+}
+
+delta_status_t delta_state_view(const delta_state_t* st, int32_t what, const void** dev_ptr,
+                                size_t* bytes) {
+  if (!st || !dev_ptr || !bytes) return DELTA_ERR_INVALID_ARG;
+  const delta_config_t& c = st->cfg;
+  const size_t BH = (size_t)c.B * c.H;
+  const size_t nt = st->shape.n_tiles;
+  switch (what) {
+    case DELTA_VIEW_DQ: *dev_ptr = st->ws.dq; *bytes = BH * c.T_max * c.d * 4; break;
+    case DELTA_VIEW_MASK: *dev_ptr = st->ws.mask; *bytes = BH * c.T_max * (c.d / 32) * 4; break;
+    case DELTA_VIEW_ROW_NNZ: *dev_ptr = st->ws.row_nnz; *bytes = BH * c.T_max * 2; break;
+    case DELTA_VIEW_TILE_NNZ: *dev_ptr = st->ws.tile_nnz; *bytes = BH * nt * 4; break;
+    case DELTA_VIEW_IDX: *dev_ptr = st->ws.idx; *bytes = BH * c.T_max * c.d; break;
+    case DELTA_VIEW_QHAT_TILE: *dev_ptr = st->ws.qhat_tile; *bytes = BH * nt * c.d * 4; break;
+    case DELTA_VIEW_QHAT: *dev_ptr = st->ws.qhat[st->qhat_sel]; *bytes = BH * c.d * 4; break;
+    case DELTA_VIEW_R: *dev_ptr = st->ws.R; *bytes = BH * c.T_max * 4; break;
+    default: return DELTA_ERR_INVALID_ARG;
+  }
+  return DELTA_OK;
+}
+
+uint64_t delta_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* delta_status_string(delta_status_t s) {
+  switch (s) {
+    case DELTA_OK: return "ok";
+    case DELTA_ERR_INVALID_ARG: return "invalid argument";
+    case DELTA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case DELTA_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case DELTA_ERR_CAPACITY: return "sequence capacity T_max exceeded";
+    case DELTA_ERR_STATE: return "call order: state not in the required condition";
+    case DELTA_ERR_CUDA: return "CUDA runtime error";
+    case DELTA_ERR_TIMEOUT: return "bounded device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+const char* delta_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

@@ -1,0 +1,84 @@
+// Internal declarations shared by the translation units of the delta-attention library.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/delta_attn.h"
+
+namespace delta {
+
+// Device counters (uint64) in the workspace.
+enum CounterSlot {
+  CNT_PREFILL_NNZ = 0, CNT_PREFILL_ELEMS, CNT_PREFILL_MACS_DONE, CNT_PREFILL_MACS_DENSE,
+  CNT_DECODE_NNZ, CNT_DECODE_ELEMS, CNT_DECODE_MACS_DONE, CNT_DECODE_MACS_DENSE,
+  CNT_STATUS,  // low 32 bits: device status word (0 = ok)
+  CNT_SLOTS = 16
+};
+
+constexpr int kMaxDecodeSplits = 64;   // split-KV partials per (batch, KV head)
+constexpr int kDecodeChunkMax = 1024;  // keys per decode CTA (scores live in shared memory)
+
+// Device pointers carved from the caller's workspace.
+struct Workspace {
+  float* dq;            // [B,H,T_max,d]
+  uint32_t* mask;       // [B,H,T_max,d/32]
+  uint16_t* row_nnz;    // [B,H,T_max]
+  uint32_t* tile_nnz;   // [B,H,n_tiles]
+  uint8_t* idx;         // [B,H,T_max,d]
+  float* qhat_tile;     // [B,H,n_tiles,d]
+  float* qhat[2];       // [B,H,d] ping-pong (decode reads one, writes the other)
+  float* R;             // [B,H,T_max]
+  unsigned long long* counters;  // [CNT_SLOTS]
+  float* dec_partial;   // [B,H_kv,kMaxDecodeSplits,g,(d+2)]
+  uint32_t* dec_ticket; // [B,H_kv]
+  __nv_bfloat16* qhat_tile_bf16;  // [B,H,n_tiles,d] (bf16 configurations only)
+  size_t total_bytes;
+};
+
+struct Shape {
+  int B, H, H_kv, d, T_max, n_tiles;
+  int g() const { return H / H_kv; }
+};
+
+void count_launch(int n = 1);
+
+// K1: delta construction over the query stream (Eq. 2-3).
+cudaError_t launch_delta_construct(const Shape& s, const Workspace& w, const void* q, int T,
+                                   float theta, int dtype, int init, cudaStream_t st);
+// K4: sparsity counters of the prefill stage (Eq. 6 inputs).
+cudaError_t launch_prefill_stats(const Shape& s, const Workspace& w, int T, int window, int shape,
+                                 cudaStream_t st);
+// K2 (generic): fused hybrid attention on CUDA cores, any supported dtype.
+cudaError_t launch_hybrid_attn_generic(const Shape& s, const Workspace& w, const void* q,
+                                       const void* k, const void* v, void* out, int T, int window,
+                                       int shape, int dtype, cudaStream_t st);
+// Hand-off: R(T-1)[j] = q_hat . k_j for j < T.
+cudaError_t launch_handoff(const Shape& s, const Workspace& w, const void* k, int T, int dtype,
+                           int qhat_sel, cudaStream_t st);
+// K3: one decode step.
+cudaError_t launch_decode_step(const Shape& s, const Workspace& w, const void* q_new,
+                               const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                               void* out, int n, float theta, int window, int dtype, int qhat_sel,
+                               cudaStream_t st);
+
+// ---- small device helpers -------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) {
+  return __float2bfloat16_rn(x);
+}
+
+// Is the causal pair (i, j <= i) inside the exact window?  shape: 0 block, 1 sliding.
+__host__ __device__ __forceinline__ bool in_window(int i, int j, int W, int shape) {
+  if (W <= 0) return false;
+  return shape == 0 ? (i / W) == (j / W) : (i - j) < W;
+}
+// Number of in-window keys of query row i.
+__host__ __device__ __forceinline__ int in_window_count(int i, int W, int shape) {
+  if (W <= 0) return 0;
+  return shape == 0 ? (i % W) + 1 : (i + 1 < W ? i + 1 : W);
+}
+
+}  // namespace delta

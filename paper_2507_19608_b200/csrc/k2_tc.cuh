@@ -1,0 +1,11 @@
+// Tensor-core (tcgen05 / TMEM / TMA) hybrid-attention kernel for bf16 inputs: interface.
+#pragma once
+#include "delta_internal.cuh"
+
+namespace delta {
+// Does this build carry a tensor-core prefill kernel for head dimension d?
+bool tc_kernel_available(int d);
+cudaError_t launch_hybrid_attn_tc(const Shape& s, const Workspace& w, const void* q, const void* k,
+                                  const void* v, void* out, int T, int window, int shape,
+                                  cudaStream_t st);
+}  // namespace delta

@@ -1,0 +1,296 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+Bars: masks, counts, indices, delta values and reference states are bit-exact; attention
+outputs agree within max-abs 1e-4 for fp32 inputs and within 2e-2 relative (to the largest
+reference magnitude of the tensor; the normalised RMS error is held to 5e-3 as well) for bf16.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import delta_oracle as O
+from paper_2507_19608_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+
+FP32_ATOL = 1e-4
+BF16_REL = 2e-2
+BF16_NRMS = 5e-3
+
+
+@pytest.fixture(scope="module")
+def B():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2507_19608_b200 import binding
+    return binding
+
+
+def _inputs(Bn, H, Hk, T, d, dtype, seed, rho=0.95, sigma=0.5):
+    w = WL.Workload("t", Bn, H, Hk, T, d, dtype, rho, sigma, 0, (), seed)
+    t = WL.make_qkv(w)
+    return t["q"], t["k"], t["v"]
+
+
+def _check_out(gpu, ref, dtype, what=""):
+    err = np.abs(gpu - ref)
+    if dtype == "f32":
+        assert err.max() <= FP32_ATOL, f"{what}: max abs err {err.max():.3e}"
+    else:
+        scale = np.abs(ref).max()
+        assert err.max() <= BF16_REL * scale, f"{what}: rel err {err.max() / scale:.3e}"
+        nrms = np.sqrt(np.mean(err ** 2)) / np.sqrt(np.mean(ref ** 2))
+        assert nrms <= BF16_NRMS, f"{what}: nrms {nrms:.3e}"
+    assert np.isfinite(gpu).all()
+
+
+def _check_delta_arrays(B, st, q, theta, init, T):
+    Bn, H, _, d = q.shape
+    dq = B.delta_state_view(st, B.DELTA_VIEW_DQ).cpu().numpy()
+    mask = B.delta_state_view(st, B.DELTA_VIEW_MASK).cpu().numpy().view(np.uint32)
+    rnz = B.delta_state_view(st, B.DELTA_VIEW_ROW_NNZ).cpu().numpy().view(np.uint16)
+    tnz = B.delta_state_view(st, B.DELTA_VIEW_TILE_NNZ).cpu().numpy().view(np.uint32)
+    idx = B.delta_state_view(st, B.DELTA_VIEW_IDX).cpu().numpy()
+    qht = B.delta_state_view(st, B.DELTA_VIEW_QHAT_TILE).cpu().numpy()
+    qh = B.delta_state_view(st, B.DELTA_VIEW_QHAT).cpu().numpy()
+    nt = (T + 63) // 64
+    total = 0
+    for b in range(Bn):
+        for h in range(H):
+            r = O.delta_construct(q[b, h], theta, init)
+            assert np.array_equal(dq[b, h, :T].view(np.uint32), r["dq"].view(np.uint32)), (b, h)
+            assert np.array_equal(mask[b, h, :T], r["mask"]), (b, h)
+            assert np.array_equal(rnz[b, h, :T], r["row_nnz"]), (b, h)
+            assert np.array_equal(tnz[b, h, :nt], r["tile_nnz"]), (b, h)
+            assert np.array_equal(idx[b, h, :T], r["idx"]), (b, h)
+            assert np.array_equal(qht[b, h, :nt].view(np.uint32), r["ahat_tile"].view(np.uint32)), (b, h)
+            assert np.array_equal(qh[b, h].view(np.uint32), r["ahat"].view(np.uint32)), (b, h)
+            total += int(r["row_nnz"].astype(np.int64).sum())
+    return total
+
+
+# ------------------------------------------------------------------ delta construction: bit-exact
+@pytest.mark.parametrize("Bn,H,T,d,dtype,theta,init", [
+    (1, 1, 128, 64, "f32", 0.1, "basis_exact"),
+    (2, 3, 200, 128, "bf16", 0.2, "basis_exact"),
+    (1, 2, 1, 64, "bf16", 0.1, "basis_exact"),
+    (1, 2, 64, 64, "f32", 0.3, "zero_state"),
+    (1, 2, 65, 128, "f32", 0.0, "basis_exact"),
+    (1, 4, 1000, 64, "bf16", 0.29, "zero_state"),
+    (1, 2, 17, 64, "bf16", 1e9, "basis_exact"),
+])
+def test_delta_construction_bit_exact(B, Bn, H, T, d, dtype, theta, init):
+    from tests.gpu_helpers import run_prefill
+    q, k, v = _inputs(Bn, H, H, T, d, dtype, seed=7 + T)
+    st, out, _, _ = run_prefill(B, q, k, v, theta, 16, dtype, init=init)
+    total = _check_delta_arrays(B, st, q, theta, init, T)
+    s = B.delta_sparsity_stats(st)
+    assert s["prefill"]["nnz"] == total and s["prefill"]["elements"] == Bn * H * T * d
+
+
+def test_delta_special_values_bit_exact(B):
+    from tests.gpu_helpers import run_prefill
+    T, d = 70, 64
+    q, k, v = _inputs(1, 1, 1, T, d, "f32", seed=3)
+    th = np.float32(0.1)
+    q[0, 0, :6, 0] = [1.0, np.float32(1.0) + th, 1.0, 1.0, 1.0, 1.0]     # |diff| vs theta at rounding level
+    q[0, 0, :6, 1] = [0.0, -0.0, 0.0, 1e-40, 0.0, 0.0]                   # signed zero, subnormal
+    q[0, 0, :6, 2] = [1.0, 1.0 + 0.1, 1.0, 2.0, 2.0, 2.0]
+    q[0, 0, 10:20, 3] = 5.0                                             # constant run: nothing fires inside
+    for theta in (0.1, 0.0):
+        st, out, _, _ = run_prefill(B, q, k, v, theta, 8, "f32")
+        _check_delta_arrays(B, st, q, theta, "basis_exact", T)
+
+
+# ------------------------------------------------------------------ prefill outputs
+CASES = [
+    # Bn, H, Hk, T,   d,  dtype, theta, W,  shape
+    (1, 1, 1, 128, 64, "f32", 0.1, 16, "block"),       # the single-head fp32 configuration
+    (1, 1, 1, 128, 64, "f32", 0.1, 16, "sliding"),
+    (1, 2, 1, 130, 64, "f32", 0.2, 0, "block"),        # no window at all, ragged tail
+    (1, 2, 2, 100, 128, "f32", 0.3, 100, "block"),     # window covers everything: dense
+    (2, 4, 2, 200, 64, "bf16", 0.2, 64, "block"),      # GQA, batch 2, ragged
+    (1, 4, 1, 257, 128, "bf16", 0.29, 50, "block"),    # window not a multiple of the tile
+    (1, 4, 4, 192, 64, "bf16", 0.1, 37, "sliding"),
+    (1, 2, 2, 64, 128, "bf16", 0.0, 5, "sliding"),     # theta = 0
+    (1, 2, 1, 1, 64, "bf16", 0.1, 4, "block"),         # one token
+    (1, 8, 2, 320, 64, "bf16", 1e9, 16, "block"),      # nothing fires after the basis row
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[f"{c[5]}-T{c[3]}-d{c[4]}-W{c[7]}{c[8][0]}-th{c[6]}" for c in CASES])
+@pytest.mark.parametrize("kernel", [0, 1], ids=["generic", "tensorcore"])
+def test_prefill_output_matches_oracle(B, case, kernel):
+    from tests.gpu_helpers import run_prefill, to_host_f64
+    Bn, H, Hk, T, d, dtype, theta, W, shape = case
+    q, k, v = _inputs(Bn, H, Hk, T, d, dtype, seed=100 + T + d)
+    if kernel == 1:
+        cfg = B.make_config(Bn, H, Hk, d, T, dtype)
+        ws = torch.empty(B.delta_state_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+        st0 = B.delta_state_init(cfg, workspace=ws)
+        try:
+            B.delta_state_set_prefill_kernel(st0, 1)
+        except B.DeltaError as e:
+            assert e.status == B.DELTA_ERR_UNSUPPORTED
+            pytest.skip("no tensor-core kernel for this configuration")
+    st, out, _, _ = run_prefill(B, q, k, v, theta, W, dtype, shape=shape, kernel=kernel)
+    ref, heads = O.prefill_mha(q, k, v, theta, W, shape)
+    _check_out(to_host_f64(out), ref, dtype, "prefill out")
+    # hand-off state for decode: reference query and the last score row
+    R = B.delta_state_view(st, B.DELTA_VIEW_R).cpu().numpy()
+    for b in range(Bn):
+        for h in range(H):
+            Rref = heads[(b, h)]["state"]["R"]
+            tol = 1e-4 * max(1.0, np.abs(Rref).max())
+            assert np.abs(R[b, h, :T] - Rref).max() <= tol
+    # counters (Eq. 6 inputs) are integers: exact
+    s = B.delta_sparsity_stats(st)["prefill"]
+    done = dense = nnz = 0
+    for b in range(Bn):
+        for h in range(H):
+            c = O.prefill_stats(heads[(b, h)]["delta"]["row_nnz"], T, d, W, shape)
+            done += c["macs_done"]; dense += c["macs_dense"]; nnz += c["nnz"]
+    assert (s["nnz"], s["macs_done"], s["macs_dense"]) == (nnz, done, dense)
+    one = O.finish_stats(dict(nnz=nnz, elements=Bn * H * T * d, macs_done=done, macs_dense=dense), min(W, T), T)
+    assert s["S_m"] == pytest.approx(one["S_m"], abs=1e-12)
+    assert s["S_c_eq6"] == pytest.approx(one["S_c_eq6"], abs=1e-12)
+    assert s["S_c_exact"] == pytest.approx(one["S_c_exact"], abs=1e-12)
+
+
+def test_theta0_full_window_equals_dense_attention(B):
+    """theta = 0 with W >= T must be plain causal attention (checked against torch SDPA in fp64)."""
+    from tests.gpu_helpers import run_prefill, to_host_f64
+    q, k, v = _inputs(1, 4, 2, 150, 64, "f32", seed=5, sigma=0.0)
+    st, out, _, _ = run_prefill(B, q, k, v, 0.0, 150, "f32")
+    tq = torch.from_numpy(q.astype(np.float64))
+    tk = torch.from_numpy(k.astype(np.float64)).repeat_interleave(2, dim=1)
+    tv = torch.from_numpy(v.astype(np.float64)).repeat_interleave(2, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True).numpy()
+    assert np.abs(to_host_f64(out) - ref).max() <= FP32_ATOL
+
+
+def test_prefill_host_entry_matches_device_entry(B):
+    from tests.gpu_helpers import run_prefill
+    Bn, H, Hk, T, d, dtype = 1, 4, 2, 150, 64, "bf16"
+    q, k, v = _inputs(Bn, H, Hk, T, d, dtype, seed=9)
+    st, out, _, _ = run_prefill(B, q, k, v, 0.2, 32, dtype, T_max=160)
+    cfg = B.make_config(Bn, H, Hk, d, 160, dtype)
+    st2 = B.delta_state_init(cfg)
+    staging = torch.empty(B.delta_prefill_staging_bytes(cfg, T), dtype=torch.uint8, device="cuda")
+    hq = torch.from_numpy(WL.bf16_bits(q).view(np.int16)).pin_memory()
+    hk = torch.from_numpy(WL.bf16_bits(k).view(np.int16)).pin_memory()
+    hv = torch.from_numpy(WL.bf16_bits(v).view(np.int16)).pin_memory()
+    ho = torch.empty_like(hq).pin_memory()
+    B.delta_attn_prefill_host(st2, hq, hk, hv, ho, staging, T, 0.2, 32)
+    assert torch.equal(ho.view(torch.bfloat16), out.cpu())
+
+
+# ------------------------------------------------------------------ decode
+@pytest.mark.parametrize("Bn,H,Hk,T,d,dtype,theta,W,steps", [
+    (1, 2, 1, 100, 64, "f32", 0.2, 8, 6),
+    (2, 4, 2, 130, 64, "bf16", 0.1, 64, 5),
+    (1, 4, 1, 700, 128, "bf16", 0.29, 4, 4),      # several key splits per head group
+    (1, 8, 1, 90, 64, "bf16", 0.1, 0, 3),         # no exact window, group of 8 heads
+    (1, 2, 2, 40, 128, "f32", 0.0, 1000, 3),      # window covers the whole cache
+    (1, 1, 1, 1, 64, "bf16", 0.1, 2, 4),          # decode right after a one-token prefill
+])
+def test_decode_steps_match_oracle(B, Bn, H, Hk, T, d, dtype, theta, W, steps):
+    from tests.gpu_helpers import run_prefill, to_dev, to_host_f64
+    w = WL.Workload("t", Bn, H, Hk, T, d, dtype, 0.95, 0.5, W, (), 77 + T, n_decode=steps)
+    t = WL.make_qkv(w)
+    st, out, kc, vc = run_prefill(B, t["q"], t["k"], t["v"], theta, W, dtype, shape="sliding", T_max=T + steps)
+    ref, heads = O.prefill_mha(t["q"], t["k"], t["v"], theta, W, "sliding")
+    states = {key: r["state"] for key, r in heads.items()}
+    nnz = done = dense = 0
+    for s in range(steps):
+        qn, kn, vn = t["q_dec"][:, :, s], t["k_dec"][:, :, s], t["v_dec"][:, :, s]
+        dqn, dkn, dvn = to_dev(qn, dtype), to_dev(kn, dtype), to_dev(vn, dtype)
+        o = torch.full_like(dqn, float("nan"))
+        B.delta_attn_decode_step(st, dqn, dkn, dvn, kc, vc, o, float(theta), int(W))
+        torch.cuda.synchronize()
+        oref, infos = O.decode_mha(states, qn, kn, vn, theta, W)
+        _check_out(to_host_f64(o), oref, dtype, f"decode step {s}")
+        n = T + s
+        assert B.delta_state_position(st) == n + 1
+        # the cache row was appended
+        assert torch.equal(kc[:, :, n], dkn) and torch.equal(vc[:, :, n], dvn)
+        R = B.delta_state_view(st, B.DELTA_VIEW_R).cpu().numpy()
+        qh = B.delta_state_view(st, B.DELTA_VIEW_QHAT).cpu().numpy()
+        for (b, h), stt in states.items():
+            tol = (1e-4 if dtype == "f32" else 1e-3) * max(1.0, np.abs(stt["R"]).max())
+            assert np.abs(R[b, h, :n + 1] - stt["R"]).max() <= tol
+            assert np.array_equal(qh[b, h].view(np.uint32), stt["qhat"].view(np.uint32))
+            c = O.stage_stats([infos[(b, h)]["row_nnz"]], [n], d, W, "sliding")
+            nnz += c["nnz"]; done += c["macs_done"]; dense += c["macs_dense"]
+    sd = B.delta_sparsity_stats(st)["decode"]
+    assert (sd["nnz"], sd["elements"], sd["macs_done"], sd["macs_dense"]) == (nnz, Bn * H * d * steps, done, dense)
+
+
+# ------------------------------------------------------------------ call-order and capacity errors
+def test_state_errors(B):
+    from tests.gpu_helpers import run_prefill, to_dev
+    q, k, v = _inputs(1, 2, 1, 32, 64, "bf16", seed=1)
+    st, out, kc, vc = run_prefill(B, q, k, v, 0.1, 4, "bf16", T_max=33)
+    with pytest.raises(B.DeltaError) as e:
+        B.delta_attn_prefill(st, out, kc, vc, out, 32, 2, 1, 64, 0.1, 4)
+    assert e.value.status == B.DELTA_ERR_STATE
+    qn, kn = to_dev(q[:, :, 0], "bf16"), to_dev(k[:, :, 0], "bf16")
+    o = torch.empty_like(qn)
+    B.delta_attn_decode_step(st, qn, kn, kn, kc, vc, o, 0.1, 4)
+    with pytest.raises(B.DeltaError) as e:
+        B.delta_attn_decode_step(st, qn, kn, kn, kc, vc, o, 0.1, 4)
+    assert e.value.status == B.DELTA_ERR_CAPACITY
+    B.delta_state_reset(st)
+    with pytest.raises(B.DeltaError) as e:
+        B.delta_attn_decode_step(st, qn, kn, kn, kc, vc, o, 0.1, 4)
+    assert e.value.status == B.DELTA_ERR_STATE
+    for bad in (dict(theta=-1.0), dict(theta=float("nan")), dict(window=-1), dict(T=0), dict(H=3)):
+        a = dict(T=32, H=2, theta=0.1, window=4); a.update(bad)
+        with pytest.raises(B.DeltaError) as e:
+            B.delta_attn_prefill(st, out, kc, vc, out, a["T"], a["H"], 1, 64, a["theta"], a["window"])
+        assert e.value.status == B.DELTA_ERR_INVALID_ARG
+    with pytest.raises(B.DeltaError) as e:
+        B.delta_attn_prefill(st, out, kc, vc, out, 34, 2, 1, 64, 0.1, 4)
+    assert e.value.status == B.DELTA_ERR_CAPACITY
+    # a reset state takes a new prefill and reproduces the first result
+    out2 = torch.empty_like(out)
+    from tests.gpu_helpers import to_dev as td
+    B.delta_attn_prefill(st, td(q, "bf16"), kc, vc, out2, 32, 2, 1, 64, 0.1, 4)
+    torch.cuda.synchronize()
+    assert torch.equal(out2, out)
+    assert B.delta_launch_count() > 0
+
+
+# ------------------------------------------------------------------ full-size configurations
+@pytest.mark.parametrize("name,theta,heads", [
+    ("llama32_1b_prefill", 0.1, (0, 13, 31)),
+    ("llama32_1b_prefill", 0.3, (5, 18)),
+    ("bitnet_2b_prefill", 0.29, (0, 19)),
+])
+def test_full_size_prefill_sampled_heads(B, name, theta, heads):
+    """The benchmark's launch configuration at full size: delta arrays of the sampled heads are
+    bit-exact, outputs of the sampled heads match the oracle, global counters match a recount
+    over all heads."""
+    from tests.gpu_helpers import run_prefill, to_host_f64
+    w = WL.WORKLOADS[name]
+    t = WL.make_qkv(w)
+    st, out, _, _ = run_prefill(B, t["q"], t["k"], t["v"], theta, w.window, w.dtype)
+    g = w.H // w.H_kv
+    dq = B.delta_state_view(st, B.DELTA_VIEW_DQ)
+    mask = B.delta_state_view(st, B.DELTA_VIEW_MASK)
+    idx = B.delta_state_view(st, B.DELTA_VIEW_IDX)
+    rnz = B.delta_state_view(st, B.DELTA_VIEW_ROW_NNZ).cpu().numpy().view(np.uint16)
+    nnz_all = 0
+    for h in range(w.H):
+        r = O.delta_construct(t["q"][0, h], theta)
+        assert np.array_equal(rnz[0, h], r["row_nnz"])
+        assert np.array_equal(mask[0, h].cpu().numpy().view(np.uint32), r["mask"])
+        nnz_all += int(r["row_nnz"].astype(np.int64).sum())
+        if h in heads:
+            assert np.array_equal(dq[0, h].cpu().numpy().view(np.uint32), r["dq"].view(np.uint32))
+            assert np.array_equal(idx[0, h].cpu().numpy(), r["idx"])
+    s = B.delta_sparsity_stats(st)["prefill"]
+    assert s["nnz"] == nnz_all
+    o = to_host_f64(out)
+    for h in heads:
+        ref = O.prefill_head(t["q"][0, h], t["k"][0, h // g], t["v"][0, h // g], theta, w.window, "block")
+        _check_out(o[0, h], ref["out"], w.dtype, f"{name} head {h}")
