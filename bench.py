@@ -1,0 +1,486 @@
+#!/usr/bin/env python
+"""Benchmark of the delta-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one pass of the prefill hot path (delta construction, sparsity counters, fused
+hybrid attention, decode hand-off) over the Llama-3.2-1B attention-layer workload
+(batch 1, 32 query / 8 KV heads, head_dim 64, T = 1024, bf16, block window 64) with the
+threshold that gives about 60 % delta sparsity on the synthetic AR(1) streams.  The decode
+step (cache prefilled to 2048 tokens, 256 steps, batch 1 and 16) is a different workload and
+is timed in its own region of the same run; it is reported under "decode".
+
+Rank 0 prints one JSON line.  With N > 1 every rank runs an independent replica of the
+workload (different seed): the path shards over (batch, KV-head group, layer) with no
+exchange step, so there is no collective on the data path ("scaling": "weak").
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2507_19608_b200 import workloads as WL
+
+HEADLINE_THETA = 0.3          # S_m ~ 0.60 on the Llama-shape AR(1) workload
+FLUSH_BYTES = 256 << 20       # > 126 MB of L2, written between timed iterations
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+                  "sm_max_mhz": 1965.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the hybrid-attention kernel on the
+# headline workload, from the ncu capture summarised under profiles/ (None until captured).
+K2_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, f"/tmp/delta_bench_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()          # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0])); mx.append(float(p[1]))
+                except ValueError:
+                    continue
+                for nme, val in zip(names, p[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(nme)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# --------------------------------------------------------------------------- reference arm
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def oracle_prefill_sample(w, tensors, theta, heads):
+    """The oracle, as it stands, on a few heads of the workload; returns seconds."""
+    from oracle import delta_oracle as O
+    g = w.H // w.H_kv
+    t0 = time.perf_counter()
+    for h in heads:
+        O.prefill_head(tensors["q"][0, h], tensors["k"][0, h // g], tensors["v"][0, h // g], theta,
+                       w.window, "block")
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = WL.WORKLOADS[args.workload]
+    tensors = WL.make_qkv(w, n_decode=0)
+    heads = list(range(0, w.H, max(1, w.H // args.ref_heads)))[:args.ref_heads]
+    for _ in range(args.warmup):
+        oracle_prefill_sample(w, tensors, args.theta, heads[:1])
+    times = [oracle_prefill_sample(w, tensors, args.theta, heads) for _ in range(args.steps)]
+    per_head = statistics.mean(times) / len(heads)
+    step_s = per_head * w.H * w.B           # extrapolated to every head of the layer
+    value = w.B * w.T / step_s
+    cores = blas_threads()
+    sample = (f"{len(heads)} of {w.H} heads per step (heads {heads}), full T={w.T}; "
+              f"layer time extrapolated by head count")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": config_dict(w, args.theta),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+METRIC = "delta-attn prefill tokens/s at Llama-3.2-1B layer shape (decode us/step alongside)"
+
+
+def config_dict(w, theta):
+    return {"workload": w.name, "B": w.B, "H": w.H, "H_kv": w.H_kv, "T": w.T, "d": w.d,
+            "dtype": w.dtype, "theta": theta, "window": w.window, "window_shape": "block",
+            "source": "query", "l2": f"flushed between timed iterations ({FLUSH_BYTES >> 20} MiB write)"}
+
+
+# --------------------------------------------------------------------------- our arm
+def to_dev(x, dtype, torch):
+    if dtype == "bf16":
+        return torch.from_numpy(WL.bf16_bits(x).view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+def flop_model(w, stats, tc_kernel):
+    """Algorithmic flops of one hybrid-attention launch, from the library's own counters."""
+    BH = w.B * w.H
+    N_c = w.T * (w.T + 1) // 2
+    pv = 2.0 * w.d * N_c * BH                                   # P.V over every causal pair
+    qk = 2.0 * stats["macs_done"]                               # exact in-window + fired out-of-window
+    full, rem = divmod(w.T, w.window) if w.window > 0 else (0, 0)
+    n_in = (full * w.window * (w.window + 1) // 2 + rem * (rem + 1) // 2) if w.window > 0 else 0
+    qk_in = 2.0 * w.d * n_in * BH
+    seeds = 2.0 * w.d * (N_c - n_in) * BH / 64.0                # one dense row per 64-row query tile
+    dense_equiv = 4.0 * w.d * N_c * BH
+    alu = (qk - qk_in) + seeds if tc_kernel else qk + seeds + pv
+    return dict(algorithmic=qk + seeds + pv, alu=alu, tensor=(qk_in + pv) if tc_kernel else 0.0,
+                dense_equiv=dense_equiv)
+
+
+def run_ours(args):
+    import torch
+    from paper_2507_19608_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+    props = torch.cuda.get_device_properties(local)
+    n_sm = props.multi_processor_count
+
+    w = WL.WORKLOADS[args.workload]
+    theta = args.theta
+    tens = WL.make_qkv(w, layer=rank, n_decode=0)          # each rank: an independent replica
+    q, k, v = (to_dev(tens[n], w.dtype, torch) for n in ("q", "k", "v"))
+    out = torch.empty_like(q)
+    cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T, w.dtype)
+    st = B.delta_state_init(cfg)
+    if args.kernel >= 0:
+        B.delta_state_set_prefill_kernel(st, args.kernel)
+    tc_kernel = B.delta_state_prefill_kernel(st) == 1
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def step():
+        B.delta_state_reset(st)
+        B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- timed region: K steps, device time by CUDA events, L2 flushed before each step
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = B.delta_launch_count()
+    evs = []
+    barrier()
+    for _ in range(args.steps):
+        flush.zero_()
+        B.delta_state_reset(st)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
+        e1.record()
+        evs.append((e0, e1))
+    barrier()
+    launches = B.delta_launch_count() - launches0
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    total_ms = sum(step_ms)
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    stats = B.delta_sparsity_stats(st)["prefill"]
+
+    # ---- the same steps with per-kernel events (roofline of the dominant kernel)
+    B.delta_state_enable_profiling(st, True)
+    kms = []
+    for _ in range(args.steps):
+        flush.zero_()
+        B.delta_state_reset(st)
+        B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
+        kms.append(B.delta_state_prefill_kernel_ms(st))
+    B.delta_state_enable_profiling(st, False)
+    clocks = sampler.stop() if rank == 0 else None
+    kmean = [statistics.mean(x[i] for x in kms) for i in range(4)]
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    fm = flop_model(w, stats, tc_kernel)
+    sm_max = float(peaks.get("sm_max_mhz", 1965.0))
+    alu_peak = n_sm * 128 * 2 * sm_max * 1e6 / 1e12          # TFLOP/s: SMs x FP32 lanes x FMA x clock
+    k2_s = kmean[2] * 1e-3
+    roofline = {
+        "kernel": "hybrid_attn_tc" if tc_kernel else "hybrid_attn_generic",
+        "bound": "alu", "achieved": fm["alu"] / k2_s / 1e12, "peak": alu_peak, "unit": "TFLOP/s",
+        "frac": fm["alu"] / k2_s / 1e12 / alu_peak, "traffic": K2_DRAM_TRAFFIC_BYTES,
+        "peak_source": f"derived: {n_sm} SMs x 128 FP32 lanes x 2 x {sm_max:.0f} MHz",
+        "kernel_ms": kmean[2], "algorithmic_tflops": fm["algorithmic"] / k2_s / 1e12,
+        "dense_equiv_tflops": fm["dense_equiv"] / k2_s / 1e12,
+        "tensor_tflops": fm["tensor"] / k2_s / 1e12,
+        "tensor_frac_of_" + peaks["_source"]: fm["tensor"] / k2_s / 1e12 / float(peaks["bf16_tflops"]),
+    }
+    # K1 is a streaming pass: report it against the HBM copy bandwidth as well
+    es = 2 if w.dtype == "bf16" else 4
+    k1_bytes = w.B * w.H * w.T * (w.d * (es + 4 + 1) + w.d // 8 + 2)
+    k1 = {"kernel": "delta_construct", "bound": "hbm", "kernel_ms": kmean[0],
+          "achieved": k1_bytes / (kmean[0] * 1e-3) / 1e9, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
+          "frac": k1_bytes / (kmean[0] * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
+          "note": f"{w.B * w.H * w.d} token-sequential chains of {w.T} steps: latency-bound at this size"}
+
+    line = {
+        "metric": METRIC, "value": args.gpus * w.B * w.T / (ms_per_step * 1e-3), "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if w.dtype == "f32" else "bf16 in, f32 accumulate", "data": "synthetic",
+        "config": config_dict(w, theta), "impl": "ours",
+        "prefill_kernel": "tcgen05" if tc_kernel else "generic",
+        "gpu_launches": int(launches),
+        "kernel_ms": {"delta_construct": kmean[0], "prefill_stats": kmean[1], "hybrid_attn": kmean[2],
+                      "handoff": kmean[3]},
+        "sparsity": {"S_m": stats["S_m"], "S_c_eq6": stats["S_c_eq6"], "S_c_exact": stats["S_c_exact"],
+                     "paper_context": "paper: ~60% prefill, ~57% prefill+decode (key deltas, real activations, A100)"},
+        "roofline": roofline, "roofline_delta_construct": k1, "clocks": clocks,
+        "peaks": {k_: peaks[k_] for k_ in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained") if k_ in peaks}
+        | {"source": peaks["_source"]},
+    }
+
+    if not args.quick:
+        line["e2e"] = run_e2e(args, B, torch, w, tens, theta)
+        line["theta_sweep"] = run_sweep(args, B, torch, w, q, k, v, out, st, flush)
+        line["decode"] = run_decode(args, B, torch, peaks)
+        line["cpu_baseline"] = run_cpu_baseline(args, w, tens, theta)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(args, B, torch, w, tens, theta):
+    """Same metric through delta_attn_prefill_host: pinned host buffers in, host buffer out."""
+    cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T, w.dtype)
+    st = B.delta_state_init(cfg)
+    staging = torch.empty(B.delta_prefill_staging_bytes(cfg, w.T), dtype=torch.uint8, device="cuda")
+
+    def host(x):
+        if w.dtype == "bf16":
+            return torch.from_numpy(WL.bf16_bits(x).view(np.int16)).pin_memory()
+        return torch.from_numpy(np.ascontiguousarray(x)).pin_memory()
+    hq, hk, hv = host(tens["q"]), host(tens["k"]), host(tens["v"])
+    ho = torch.empty_like(hq).pin_memory()
+    times = []
+    for i in range(3 + args.steps):
+        B.delta_state_reset(st)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        B.delta_attn_prefill_host(st, hq, hk, hv, ho, staging, w.T, theta, w.window)   # synchronises
+        t1 = time.perf_counter()
+        if i >= 3:
+            times.append(t1 - t0)
+    s = statistics.mean(times)
+    h2d = (hq.numel() + hk.numel() + hv.numel()) * hq.element_size()
+    return {"value": w.B * w.T / s, "unit": "tokens/s", "ms_per_step": s * 1e3,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(ho.numel() * ho.element_size()),
+            "api": "delta_attn_prefill_host (pinned host buffers, wall clock around the synchronous call)"}
+
+
+def run_sweep(args, B, torch, w, q, k, v, out, st, flush):
+    res = []
+    for th in w.thetas:
+        ms = []
+        for i in range(2 + min(args.steps, 10)):
+            flush.zero_()
+            B.delta_state_reset(st)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, th, w.window)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                ms.append(e0.elapsed_time(e1))
+        s = B.delta_sparsity_stats(st)["prefill"]
+        res.append({"theta": th, "ms_per_step": statistics.mean(ms),
+                    "tokens_per_s": w.B * w.T / (statistics.mean(ms) * 1e-3), "S_m": s["S_m"],
+                    "S_c_exact": s["S_c_exact"]})
+    return res
+
+
+def run_decode(args, B, torch, peaks):
+    """Decode leg: cache prefilled to 2048 tokens, then 256 steps; batch 1 and 16."""
+    res = {}
+    for name in ("llama32_1b_decode_b1", "llama32_1b_decode_b16"):
+        w = WL.WORKLOADS[name]
+        theta = w.thetas[0]
+        tens = WL.make_qkv(w)
+        cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T_max, w.dtype, prefill_window=B.DELTA_WIN_SLIDING)
+        st = B.delta_state_init(cfg)
+        q = to_dev(tens["q"], w.dtype, torch)
+
+        def cache(x):
+            full = np.zeros((w.B, w.H_kv, w.T_max, w.d), np.float32)
+            full[:, :, :w.T] = x
+            return to_dev(full, w.dtype, torch)
+        kc, vc = cache(tens["k"]), cache(tens["v"])
+        out_p = torch.empty_like(q)
+        qd = to_dev(np.ascontiguousarray(tens["q_dec"].transpose(2, 0, 1, 3)), w.dtype, torch)
+        kd = to_dev(np.ascontiguousarray(tens["k_dec"].transpose(2, 0, 1, 3)), w.dtype, torch)
+        vd = to_dev(np.ascontiguousarray(tens["v_dec"].transpose(2, 0, 1, 3)), w.dtype, torch)
+        od = torch.empty_like(qd)
+
+        def prefill():
+            B.delta_state_reset(st)
+            B.delta_attn_prefill(st, q, kc, vc, out_p, w.T, w.H, w.H_kv, w.d, theta, w.window)
+
+        def steps():
+            for s in range(w.n_decode):
+                B.delta_attn_decode_step(st, qd[s], kd[s], vd[s], kc, vc, od[s], theta, w.window)
+
+        eager = []
+        for i in range(3):
+            prefill()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); steps(); e1.record()
+            torch.cuda.synchronize()
+            eager.append(e0.elapsed_time(e1) * 1e3 / w.n_decode)
+        od_eager = od.clone()
+        dstats = B.delta_sparsity_stats(st)
+        # the same 256 launches replayed from a CUDA graph (removes the host launch path)
+        graph_us, graph_ok = None, None
+        try:
+            prefill()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                steps()
+            reps = []
+            for i in range(4):
+                prefill()
+                od.zero_()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); g.replay(); e1.record()
+                torch.cuda.synchronize()
+                reps.append(e0.elapsed_time(e1) * 1e3 / w.n_decode)
+            graph_us = statistics.median(reps[1:])
+            graph_ok = bool(torch.equal(od, od_eager))
+        except Exception as ex:  # graph capture is an optimisation of the bench, not of the library
+            graph_ok = f"capture failed: {type(ex).__name__}"
+        es = 2
+        n_avg = w.T + (w.n_decode - 1) / 2.0
+        bytes_step = w.B * (2 * w.H_kv * n_avg * w.d * es + 2 * w.H * n_avg * 4)
+        best = graph_us if graph_us else min(eager)
+        gbs = bytes_step / (best * 1e-6) / 1e9
+        res[f"batch{w.B}"] = {
+            "us_per_step_eager": statistics.median(eager), "us_per_step_graph": graph_us,
+            "graph_matches_eager": graph_ok, "steps": w.n_decode, "cache_tokens": w.T, "theta": theta,
+            "window": w.window, "algorithmic_bytes_per_step": bytes_step,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
+                         "frac": gbs / float(peaks["hbm_gbs"]),
+                         "note": "batch 1 moves ~5 MB per step: launch latency, not bandwidth, sets the time"
+                         if w.B == 1 else ""},
+            "S_m_decode": dstats["decode"]["S_m"], "S_c_exact_decode": dstats["decode"]["S_c_exact"],
+            "S_c_exact_combined": dstats["combined"]["S_c_exact"],
+        }
+        del st, q, kc, vc, qd, kd, vd, od
+        torch.cuda.empty_cache()
+    return res
+
+
+def run_cpu_baseline(args, w, tens, theta):
+    heads = list(range(0, w.H, max(1, w.H // 8)))[:8]
+    oracle_prefill_sample(w, tens, theta, heads[:1])     # warm-up
+    reps, t_used = [], 0.0
+    while t_used < 10.0 and len(reps) < 8:
+        t = oracle_prefill_sample(w, tens, theta, heads)
+        reps.append(t); t_used += t
+    per_head = statistics.mean(reps) / len(heads)
+    value = w.B * w.T / (per_head * w.H * w.B)
+    return {"value": value, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{len(heads)} of {w.H} heads x {len(reps)} repeats, full T={w.T}; extrapolated by head count"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama32_1b_prefill")
+    ap.add_argument("--theta", type=float, default=HEADLINE_THETA)
+    ap.add_argument("--kernel", type=int, default=-1, help="-1 auto, 0 generic, 1 tensor-core")
+    ap.add_argument("--quick", action="store_true", help="prefill timing only (used for ncu launch lists)")
+    ap.add_argument("--ref-heads", type=int, default=4, help="heads per reference step")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

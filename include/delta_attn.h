@@ -188,6 +188,15 @@ DELTA_API int32_t delta_state_position(const delta_state_t* st);
 DELTA_API int32_t delta_state_prefill_kernel(const delta_state_t* st);
 DELTA_API delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which);
 
+/* Per-kernel timing of delta_attn_prefill.  With profiling enabled the call records a CUDA
+ * event in front of and behind each of its kernels on the caller's stream (host-side event
+ * objects; no device memory).  delta_state_prefill_kernel_ms waits for the last event and
+ * returns the elapsed milliseconds of the most recent prefill in ms[0..3]:
+ * [0] delta construction, [1] sparsity counters, [2] hybrid attention, [3] decode hand-off.
+ * DELTA_ERR_STATE if profiling is off or no prefill was recorded. */
+DELTA_API delta_status_t delta_state_enable_profiling(delta_state_t* st, int32_t enable);
+DELTA_API delta_status_t delta_state_prefill_kernel_ms(delta_state_t* st, float* ms);
+
 /* Kernels launched by this library in the calling process since it was loaded. */
 DELTA_API uint64_t delta_launch_count(void);
 

@@ -31,6 +31,7 @@ EXPORTED = [
     "delta_attn_decode_step", "delta_sparsity_stats", "delta_window_from_gamma", "delta_state_view",
     "delta_state_position", "delta_state_prefill_kernel", "delta_state_set_prefill_kernel",
     "delta_launch_count", "delta_status_string", "delta_last_cuda_error",
+    "delta_state_enable_profiling", "delta_state_prefill_kernel_ms",
 ]
 
 
@@ -87,6 +88,8 @@ def _load() -> C.CDLL:
         "delta_state_position": (i32, [vp]),
         "delta_state_prefill_kernel": (i32, [vp]),
         "delta_state_set_prefill_kernel": (C.c_int, [vp, i32]),
+        "delta_state_enable_profiling": (C.c_int, [vp, i32]),
+        "delta_state_prefill_kernel_ms": (C.c_int, [vp, C.POINTER(C.c_float)]),
         "delta_launch_count": (C.c_uint64, []),
         "delta_status_string": (C.c_char_p, [C.c_int]),
         "delta_last_cuda_error": (C.c_char_p, []),
@@ -212,6 +215,16 @@ def delta_state_prefill_kernel(st: DeltaState) -> int:
 
 def delta_state_set_prefill_kernel(st: DeltaState, which: int):
     _check(lib.delta_state_set_prefill_kernel(st.handle, which), "delta_state_set_prefill_kernel")
+
+
+def delta_state_enable_profiling(st: DeltaState, enable: bool):
+    _check(lib.delta_state_enable_profiling(st.handle, int(enable)), "delta_state_enable_profiling")
+
+
+def delta_state_prefill_kernel_ms(st: DeltaState) -> list:
+    ms = (C.c_float * 4)()
+    _check(lib.delta_state_prefill_kernel_ms(st.handle, ms), "delta_state_prefill_kernel_ms")
+    return list(ms)
 
 
 def delta_launch_count() -> int:

@@ -31,6 +31,9 @@ struct delta_state {
   int forced_kernel;  // -1 auto, 0 generic, 1 tensor-core
   // Eq. 6 bookkeeping that needs no device work: sum of window lengths and sequence lengths
   double win_sum[2], len_sum[2];
+  // optional per-kernel timing of prefill (host-side event objects)
+  bool profiling = false, profiled = false;
+  cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -138,7 +141,33 @@ delta_status_t delta_state_reset(delta_state_t* st, void* stream) {
 
 delta_status_t delta_state_destroy(delta_state_t* st) {
   if (!st) return DELTA_ERR_INVALID_ARG;
+  for (auto& ev : st->ev)
+    if (ev) cudaEventDestroy(ev);
   delete st;
+  return DELTA_OK;
+}
+
+delta_status_t delta_state_enable_profiling(delta_state_t* st, int32_t enable) {
+  if (!st) return DELTA_ERR_INVALID_ARG;
+  if (enable) {
+    for (auto& ev : st->ev)
+      if (!ev) {
+        cudaError_t e = cudaEventCreate(&ev);
+        if (e != cudaSuccess) return cuda_fail(e);
+      }
+  }
+  st->profiling = enable != 0;
+  st->profiled = false;
+  return DELTA_OK;
+}
+
+delta_status_t delta_state_prefill_kernel_ms(delta_state_t* st, float* ms) {
+  if (!st || !ms) return DELTA_ERR_INVALID_ARG;
+  if (!st->profiling || !st->profiled) return DELTA_ERR_STATE;
+  cudaError_t e = cudaEventSynchronize(st->ev[4]);
+  if (e != cudaSuccess) return cuda_fail(e);
+  for (int i = 0; i < 4; ++i)
+    if ((e = cudaEventElapsedTime(&ms[i], st->ev[i], st->ev[i + 1])) != cudaSuccess) return cuda_fail(e);
   return DELTA_OK;
 }
 
@@ -180,10 +209,15 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   if (st->n != 0) return DELTA_ERR_STATE;
   cudaStream_t cs = (cudaStream_t)stream;
   cudaError_t e;
+  const bool prof = st->profiling;
+#define MARK(i) do { if (prof && (e = cudaEventRecord(st->ev[i], cs)) != cudaSuccess) return cuda_fail(e); } while (0)
+  MARK(0);
   if ((e = launch_delta_construct(st->shape, st->ws, q, T, theta, c.dtype, c.init, cs)) != cudaSuccess)
     return cuda_fail(e);
+  MARK(1);
   if ((e = launch_prefill_stats(st->shape, st->ws, T, window, c.prefill_window, cs)) != cudaSuccess)
     return cuda_fail(e);
+  MARK(2);
   if (delta_state_prefill_kernel(st) == 1) {
     e = launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
   } else {
@@ -191,7 +225,11 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
                                    c.dtype, cs);
   }
   if (e != cudaSuccess) return cuda_fail(e);
+  MARK(3);
   if ((e = launch_handoff(st->shape, st->ws, k, T, c.dtype, 0, cs)) != cudaSuccess) return cuda_fail(e);
+  MARK(4);
+#undef MARK
+  st->profiled = prof;
   st->n = T;
   st->qhat_sel = 0;
   st->win_sum[0] += (double)(window < T ? window : T);
