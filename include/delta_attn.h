@@ -48,7 +48,8 @@ typedef enum {
   DELTA_ERR_CAPACITY = 4,     /* sequence would exceed T_max                                   */
   DELTA_ERR_STATE = 5,        /* call order: prefill on a used state, decode before prefill    */
   DELTA_ERR_CUDA = 6,         /* a CUDA runtime call failed (delta_last_cuda_error has it)     */
-  DELTA_ERR_TIMEOUT = 7       /* a bounded device-side wait ran out (status word on device)    */
+  DELTA_ERR_TIMEOUT = 7,      /* a bounded device-side wait ran out (status word on device)    */
+  DELTA_ERR_SCRATCH_LIMIT = 8 /* problem larger than the built-in scratch of the no-alloc call */
 } delta_status_t;
 
 typedef enum { DELTA_F32 = 0, DELTA_BF16 = 1 } delta_dtype_t;
@@ -137,6 +138,42 @@ DELTA_API delta_status_t delta_attn_prefill_host(delta_state_t* st, const void* 
 DELTA_API delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, const void* k_new,
                                       const void* v_new, void* k_cache, void* v_cache, void* out,
                                       float theta, int32_t window, void* stream);
+
+/* delta_attn_decode_step_noalloc -- the decode step without any workspace.  (The paper has
+ * no counterpart: this exists only for callers that cannot allocate device memory.)
+ *
+ * Who needs it: code running inside an application whose own memory manager has claimed the
+ * whole GPU, so that cudaMalloc fails or is not allowed; latency-critical loops that must stay
+ * clear of the device-wide synchronisation cudaMalloc/cudaFree imply; plug-ins that are handed
+ * nothing but input and output pointers.  This call allocates and frees nothing, on the host
+ * side of the driver or on the device, and calls no library routine that does.
+ *
+ * It performs exactly the step of delta_attn_decode_step, but stateless: the carried state is
+ * passed in and out by the caller instead of living in a delta_state_t.
+ *   q_new, out       : [B, H, d]        k_new, v_new : [B, H_kv, d]       (element type `dtype`)
+ *   k_cache, v_cache : [B, H_kv, T_max, d]; rows 0..n-1 are read, row n is written
+ *   qhat_in          : [B, H, d] float, reference state before the step (read only)
+ *   qhat_out         : [B, H, d] float, reference state after the step (must differ from qhat_in)
+ *   R                : [B, H, T_max] float, score row; entries 0..n-1 are updated in place,
+ *                      entry n is written
+ *   n                : tokens already in the cache (>= 1, < T_max)
+ * All pointers are DEVICE pointers owned by the caller.  The sparsity counters of the regular
+ * call are not kept.
+ *
+ * Scratch: the split-KV partial results and arrival tickets live in a fixed array of 8 MiB +
+ * 8 KiB inside the library image; every GPU that loads the library holds it until the process
+ * exits.  Limits that follow from its size: B * H_kv <= 1024 and B * H * (d + 2) <= 32768
+ * (for example B = 15 at 32 heads of dimension 64); anything larger returns
+ * DELTA_ERR_SCRATCH_LIMIT and launches nothing.
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call outside of any stream capture.  Every call shares the one
+ * array and finds in it what the previous call left: the parts that must start at zero are
+ * cleared on `stream` at the start of the call.  Calls whose kernels may overlap on one GPU
+ * (different streams or threads) race on the array: serialise them. */
+DELTA_API delta_status_t delta_attn_decode_step_noalloc(
+    const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* out,
+    const float* qhat_in, float* qhat_out, float* R, int32_t n, int32_t B, int32_t H, int32_t H_kv,
+    int32_t d, int32_t T_max, delta_dtype_t dtype, float theta, int32_t window, void* stream);
 
 /* Counters of one stage.  S_m = 1 - nnz/elements (sparsity of the delta matrix, Eq. 6);
  * S_c_eq6 = S_m * (1 - W/n) (Eq. 6); S_c_exact = 1 - macs_done/macs_dense where a causal

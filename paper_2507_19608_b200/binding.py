@@ -17,7 +17,7 @@ DELTA_TILE_ROWS = 64
 # enums (values of include/delta_attn.h)
 DELTA_OK = 0
 DELTA_ERR_INVALID_ARG, DELTA_ERR_UNSUPPORTED, DELTA_ERR_WORKSPACE, DELTA_ERR_CAPACITY = 1, 2, 3, 4
-DELTA_ERR_STATE, DELTA_ERR_CUDA, DELTA_ERR_TIMEOUT = 5, 6, 7
+DELTA_ERR_STATE, DELTA_ERR_CUDA, DELTA_ERR_TIMEOUT, DELTA_ERR_SCRATCH_LIMIT = 5, 6, 7, 8
 DELTA_F32, DELTA_BF16 = 0, 1
 DELTA_SRC_QUERY, DELTA_SRC_KEY = 0, 1
 DELTA_WIN_BLOCK, DELTA_WIN_SLIDING = 0, 1
@@ -32,6 +32,7 @@ EXPORTED = [
     "delta_state_position", "delta_state_prefill_kernel", "delta_state_set_prefill_kernel",
     "delta_launch_count", "delta_status_string", "delta_last_cuda_error",
     "delta_state_enable_profiling", "delta_state_prefill_kernel_ms",
+    "delta_attn_decode_step_noalloc",
 ]
 
 
@@ -90,6 +91,8 @@ def _load() -> C.CDLL:
         "delta_state_set_prefill_kernel": (C.c_int, [vp, i32]),
         "delta_state_enable_profiling": (C.c_int, [vp, i32]),
         "delta_state_prefill_kernel_ms": (C.c_int, [vp, C.POINTER(C.c_float)]),
+        "delta_attn_decode_step_noalloc": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32,
+                                                     i32, i32, C.c_int, f32, i32, vp]),
         "delta_launch_count": (C.c_uint64, []),
         "delta_status_string": (C.c_char_p, [C.c_int]),
         "delta_last_cuda_error": (C.c_char_p, []),
@@ -193,6 +196,17 @@ def delta_attn_decode_step(st: DeltaState, q_new, k_new, v_new, k_cache, v_cache
     _check(lib.delta_attn_decode_step(st.handle, _ptr(q_new), _ptr(k_new), _ptr(v_new),
                                       _ptr(k_cache), _ptr(v_cache), _ptr(out), theta, window,
                                       _stream(stream)), "delta_attn_decode_step")
+
+
+def delta_attn_decode_step_noalloc(q_new, k_new, v_new, k_cache, v_cache, out, qhat_in, qhat_out, R,
+                                   n, B, H, H_kv, d, T_max, dtype, theta, window, stream=None):
+    """Decode step for callers that cannot allocate: the carried state (qhat_in -> qhat_out, R)
+    is passed explicitly and the scratch is a fixed array inside the library.  Allocates nothing."""
+    dt = {"f32": DELTA_F32, "bf16": DELTA_BF16}.get(dtype, dtype)
+    _check(lib.delta_attn_decode_step_noalloc(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
+                                              _ptr(v_cache), _ptr(out), _ptr(qhat_in), _ptr(qhat_out),
+                                              _ptr(R), n, B, H, H_kv, d, T_max, dt, theta, window,
+                                              _stream(stream)), "delta_attn_decode_step_noalloc")
 
 
 def delta_sparsity_stats(st: DeltaState, stream=None) -> dict:

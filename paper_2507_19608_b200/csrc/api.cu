@@ -374,6 +374,8 @@ const char* delta_status_string(delta_status_t s) {
     case DELTA_ERR_STATE: return "call order: state not in the required condition";
     case DELTA_ERR_CUDA: return "CUDA runtime error";
     case DELTA_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case DELTA_ERR_SCRATCH_LIMIT:
+      return "problem larger than the built-in scratch of delta_attn_decode_step_noalloc";
   }
   return "unknown status";
 }
