@@ -1,10 +1,639 @@
-// Tensor-core hybrid-attention kernel (placeholder translation unit until the kernel lands).
+// K2 (tensor-core) -- fused hybrid delta attention for bf16 inputs on sm_100a
+// (Section III-B; Eq. 1, Eq. 4; construction strategy (1) of Section III-A).
+//
+// One CTA of 16 warps owns 128 query rows of one head and walks the 128-key tiles up to the
+// diagonal.  The work is split by what it is:
+//   * dense contractions run on the 5th-generation tensor cores (tcgen05.mma, operands staged
+//     in shared memory by TMA, accumulators in tensor memory): the exact Q.K^T of tiles that
+//     touch the window, and P.V of every tile;
+//   * the out-of-window scores are Eq. 4's running sum of sparse delta products and stay on the
+//     FP32 pipes, because the zeros of a thresholded delta matrix are unstructured.  A warp owns
+//     8 consecutive rows and all 128 keys of the tile (4 keys per lane).  Rows are taken in
+//     blocks of 4: the OR of the 4 rows' mask words says which channels fired anywhere in the
+//     block; channels whose 4x1 delta block is all zero are skipped (find-first-set over the
+//     block mask), every other channel costs one 16-byte key load (channel-major fp32 key tile)
+//     and one 16-byte delta load for a 4x4 register tile of multiply-adds.  Prefix sums over
+//     the rows turn the per-row products into R(i)[j]; the part of the recursion that lies in
+//     front of the warp's rows comes from the other warps' block totals and from the seed
+//     q_hat(i0-1).k_j (the reference in front of the tile telescopes all earlier rows);
+//   * scale, causal mask, hybrid select and the online softmax run in the same key-per-lane
+//     layout; exact scores come out of tensor memory row-per-thread and are transposed through
+//     shared memory; P goes to shared memory as bf16 in the tensor-core operand layout; the
+//     P.V tile product is read back from tensor memory row-per-thread and accumulated in
+//     registers with the softmax rescale.
+//
+// Every wait on an mbarrier is bounded; a wait that runs out records DELTA_ERR_TIMEOUT in the
+// device status word and the CTA leaves through the common exit (which frees its tensor memory).
+#include <cuda.h>
+
 #include "k2_tc.cuh"
 
 namespace delta {
-bool tc_kernel_available(int) { return false; }
-cudaError_t launch_hybrid_attn_tc(const Shape&, const Workspace&, const void*, const void*,
-                                  const void*, void*, int, int, int, cudaStream_t) {
-  return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int BM = 128, BN = 128, NTHR = 512, NWARP = 16;
+constexpr int TC_D = 64;                 // head dimension served by this kernel
+constexpr int DQ_LD = BM + 4;            // leading dimension of the channel-major delta tile
+constexpr uint32_t TMEM_COLS = 256;      // S: columns 0..127, O: columns 128..191
+constexpr uint32_t TMEM_S = 0, TMEM_O = 128;
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr uint32_t SZ_TILE = 128 * 64 * 2;               // one bf16 operand tile, 16 KiB
+constexpr uint32_t OFF_Q = 0;
+constexpr uint32_t OFF_K = OFF_Q + SZ_TILE;
+constexpr uint32_t OFF_V = OFF_K + SZ_TILE;              // two buffers
+constexpr uint32_t OFF_KT = OFF_V + 2 * SZ_TILE;         // fp32 [64 channels][128 keys]
+constexpr uint32_t OFF_P = OFF_KT + 64 * 128 * 4;        // bf16 [2][128 rows][64 keys]
+constexpr uint32_t OFF_SX = OFF_KT;                      // fp32 [128][128] exact scores (KT + P)
+constexpr uint32_t OFF_DQT = OFF_P + 2 * SZ_TILE;        // fp32 [64][DQ_LD]
+constexpr uint32_t OFF_TOT = OFF_DQT + 64 * DQ_LD * 4;   // fp32 [16][128]
+constexpr uint32_t OFF_SEED = OFF_TOT + 16 * 128 * 4;    // fp32 [16][128]
+constexpr uint32_t OFF_ALPHA = OFF_SEED + 16 * 128 * 4;  // fp32 [2][128]
+constexpr uint32_t OFF_M = OFF_ALPHA + 2 * 128 * 4;      // fp32 [128] running max
+constexpr uint32_t OFF_L = OFF_M + 128 * 4;              // fp32 [128] running sum
+constexpr uint32_t OFF_QHAT = OFF_L + 128 * 4;           // fp32 [64]
+constexpr uint32_t OFF_UNION = OFF_QHAT + 64 * 4;        // u64 [32] block masks
+constexpr uint32_t OFF_BAR = OFF_UNION + 32 * 8;         // 8 mbarriers
+constexpr uint32_t OFF_MISC = OFF_BAR + 8 * 8;           // tmem slot, abort flag
+constexpr uint32_t SMEM_USED = OFF_MISC + 16;
+constexpr uint32_t SMEM_BYTES = SMEM_USED + 1024;        // slack for the alignment of the base
+
+enum Bar { BAR_Q = 0, BAR_K, BAR_KT, BAR_V0, BAR_V1, BAR_S, BAR_O };
+
+// ---- PTX wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after about a second of SM clock.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > 2000000000ll) return false;
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
+                                            int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+      "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 operands, fp32 accumulation.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                       uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of the tensor cores: 128-byte swizzle, 16-byte units.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+         ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, given N; b_mn = 1 if B is MN-major.
+__host__ __device__ constexpr uint32_t make_idesc(int n, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(128 >> 4) << 24);
+}
+
+struct TcParams {
+  const float* dq;
+  const uint32_t* mask;
+  const float* qhat_tile;
+  __nv_bfloat16* out;
+  unsigned long long* counters;
+  int T, T_max, n_tiles64, H, g, W, shape;
+  float scale_log2e;
+};
+
+}  // namespace
+
+__global__ void __launch_bounds__(NTHR, 1)
+hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kt,
+                      const TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw);
+
+  float* sKt = reinterpret_cast<float*>(sm + OFF_KT);
+  float* sdQt = reinterpret_cast<float*>(sm + OFF_DQT);
+  float* sTot = reinterpret_cast<float*>(sm + OFF_TOT);
+  float* sSeed = reinterpret_cast<float*>(sm + OFF_SEED);
+  float* sAlpha = reinterpret_cast<float*>(sm + OFF_ALPHA);
+  float* sM = reinterpret_cast<float*>(sm + OFF_M);
+  float* sL = reinterpret_cast<float*>(sm + OFF_L);
+  float* sQhat = reinterpret_cast<float*>(sm + OFF_QHAT);
+  unsigned long long* sUnion = reinterpret_cast<unsigned long long*>(sm + OFF_UNION);
+  volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
+  const uint32_t bar0 = base + OFF_BAR;
+#define BAR(i) (bar0 + 8u * (uint32_t)(i))
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qd = warp & 3, sub = warp >> 2;     // tensor-memory lane quadrant / slot in it
+  const int rg = qd * 4 + sub;                  // row group: rows 8*rg .. 8*rg+7
+  const int my_row = 32 * qd + lane;            // row this thread owns in row-per-thread phases
+  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;  // heaviest query tiles first
+  const int bh = blockIdx.y;
+  const int b = bh / p.H, h = bh - b * p.H;
+  const int bkv = b * (p.H / p.g) + h / p.g;
+  const int i0 = qt * BM;
+  const int T = p.T, W = p.W, shape = p.shape;
+  const int i1 = min(i0 + BM, T) - 1;           // last valid row of the tile
+
+  // ---- set-up: tensor memory, barriers, first loads ---------------------------------------
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     base + OFF_MISC),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    for (int i = 0; i < 8; ++i) mbar_init(BAR(i), 1);
+    sMisc[1] = 0;  // abort flag
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sMisc[0];
+
+  auto tile_needs_exact = [&](int jt) -> bool {
+    if (W <= 0) return false;
+    const int j0 = jt * BN, j1 = min(j0 + BN, T) - 1;
+    if (shape == 0) return (i0 / W <= j1 / W) && (j0 / W <= i1 / W);
+    return max(0, i0 - j1) < W;
+  };
+  auto tile_all_in = [&](int jt) -> bool {
+    if (W <= 0) return false;
+    const int j0 = jt * BN, j1 = min(j0 + BN, T) - 1;
+    if (shape == 0) return (i0 / W == i1 / W) && (j0 / W == j1 / W) && (i0 / W == j0 / W);
+    return (i1 - j0) < W;
+  };
+
+  if (tid == 0) {
+    if (W > 0) {
+      mbar_expect_tx(BAR(BAR_Q), SZ_TILE);
+      tma_load_3d(base + OFF_Q, &tm_q, BAR(BAR_Q), 0, i0, bh);
+    }
+    mbar_expect_tx(BAR(BAR_KT), 64 * 128 * 4);
+    tma_load_3d(base + OFF_KT, &tm_kt, BAR(BAR_KT), 0, 0, bkv);
+    mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
+    tma_load_3d(base + OFF_V, &tm_v, BAR(BAR_V0), 0, 0, bkv);
+    if (tile_needs_exact(0)) {
+      mbar_expect_tx(BAR(BAR_K), SZ_TILE);
+      tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K), 0, 0, bkv);
+    }
+  }
+
+  // ---- stage the query tile's deltas channel-major, the block masks and the seed reference
+  {
+    const float* dqp = p.dq + ((size_t)bh * p.T_max + i0) * TC_D;
+    const int r_sub = lane >> 3, c_sub = lane & 7;
+    for (int it = warp; it < 32 * 8; it += NWARP) {
+      const int rb = it >> 3, cb = it & 7;
+      const int r = rb * 4 + r_sub, c = cb * 8 + c_sub;
+      const float x = (i0 + r < T) ? dqp[(size_t)r * TC_D + c] : 0.0f;
+      sdQt[c * DQ_LD + r] = x;
+    }
+    if (tid < 32) {
+      unsigned long long u = 0;
+      const uint32_t* mp = p.mask + ((size_t)bh * p.T_max + i0) * 2;
+      for (int r = 0; r < 4; ++r) {
+        const int row = tid * 4 + r;
+        if (i0 + row < T) u |= (unsigned long long)mp[row * 2] | ((unsigned long long)mp[row * 2 + 1] << 32);
+      }
+      sUnion[tid] = u;
+    }
+    if (tid < TC_D) sQhat[tid] = p.qhat_tile[((size_t)bh * p.n_tiles64 + 2 * qt) * TC_D + tid];
+    if (tid < BM) { sM[tid] = -INFINITY; sL[tid] = 0.0f; }
+  }
+  float O[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) O[i] = 0.0f;
+  __syncthreads();
+
+  const uint32_t IDESC_QK = make_idesc(BN, 0);
+  const uint32_t IDESC_PV = make_idesc(TC_D, 1);
+  int n_exact = 0;          // exact tiles seen so far (parity of BAR_K / BAR_S)
+  bool aborted = false;
+
+  for (int jt = 0; jt <= qt; ++jt) {
+    const int j0 = jt * BN;
+    const bool need_exact = tile_needs_exact(jt);
+    const bool need_delta = !tile_all_in(jt);
+    const bool diag = (jt == qt);
+
+    // ---- exact Q.K^T of a tile that touches the window: issued first, consumed after the deltas
+    if (need_exact && tid == 0) {
+      bool ok = mbar_wait(BAR(BAR_K), n_exact & 1);
+      if (n_exact == 0) ok = mbar_wait(BAR(BAR_Q), 0) && ok;
+      if (!ok) sMisc[1] = 1;
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < TC_D / 16; ++ks) {
+        const uint64_t da = make_desc(base + OFF_Q + ks * 32, 16, 1024);
+        const uint64_t db = make_desc(base + OFF_K + ks * 32, 16, 1024);
+        tc_mma(tmem + TMEM_S, da, db, IDESC_QK, ks > 0 ? 1u : 0u);
+      }
+      tc_commit(BAR(BAR_S));
+    }
+
+    // ---- Eq. 4 on the FP32 pipes: block-sparse 4x4 register tiles over fired channels
+    float Sl[8][4];
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) Sl[r][k] = 0.0f;
+    if (!mbar_wait(BAR(BAR_KT), jt & 1)) sMisc[1] = 1;
+    if (need_delta) {
+      float run[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      const float* ktp = sKt + 4 * lane;
+#pragma unroll
+      for (int g4 = 0; g4 < 2; ++g4) {
+        float a[4][4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+          for (int k = 0; k < 4; ++k) a[r][k] = 0.0f;
+        unsigned long long m = sUnion[rg * 2 + g4];
+        const float* dqg = sdQt + rg * 8 + g4 * 4;
+        while (m) {
+          const int c = __ffsll((long long)m) - 1;
+          m &= m - 1;
+          const float4 kv = *reinterpret_cast<const float4*>(ktp + c * BN);
+          const float4 dv = *reinterpret_cast<const float4*>(dqg + c * DQ_LD);
+          const float kk[4] = {kv.x, kv.y, kv.z, kv.w};
+          const float dd[4] = {dv.x, dv.y, dv.z, dv.w};
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) a[r][k] = fmaf(dd[r], kk[k], a[r][k]);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            run[k] += a[r][k];
+            Sl[g4 * 4 + r][k] = run[k];
+          }
+      }
+      // this warp's slice of the seed q_hat(i0-1).k_j: channels 4*rg .. 4*rg+3
+      float sd[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        const int c = rg * 4 + cc;
+        const float x = sQhat[c];
+        const float4 kv = *reinterpret_cast<const float4*>(ktp + c * BN);
+        sd[0] = fmaf(x, kv.x, sd[0]); sd[1] = fmaf(x, kv.y, sd[1]);
+        sd[2] = fmaf(x, kv.z, sd[2]); sd[3] = fmaf(x, kv.w, sd[3]);
+      }
+      *reinterpret_cast<float4*>(sTot + rg * BN + 4 * lane) = make_float4(run[0], run[1], run[2], run[3]);
+      *reinterpret_cast<float4*>(sSeed + rg * BN + 4 * lane) = make_float4(sd[0], sd[1], sd[2], sd[3]);
+    }
+    fence_proxy_async();   // generic reads of the key tile are ordered before its next bulk write
+    __syncthreads();       // (A) totals and seed slices visible; channel-major key tile free
+    if (sMisc[1]) { aborted = true; break; }
+
+    const bool more = (jt < qt);
+    if (tid == 0 && more && !need_exact) {
+      mbar_expect_tx(BAR(BAR_KT), 64 * 128 * 4);
+      tma_load_3d(base + OFF_KT, &tm_kt, BAR(BAR_KT), j0 + BN, 0, bkv);
+      if (tile_needs_exact(jt + 1)) {
+        mbar_expect_tx(BAR(BAR_K), SZ_TILE);
+        tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K), 0, j0 + BN, bkv);
+      }
+    }
+
+    // ---- previous tile's P.V: rescale and accumulate (row-per-thread)
+    if (jt > 0) {
+      if (!mbar_wait(BAR(BAR_O), (jt - 1) & 1)) sMisc[1] = 1;
+      tc_fence_after();
+      float v[16];
+      tc_ld16(tmem + TMEM_O + 16 * sub + ((uint32_t)(32 * qd) << 16), v);
+      const float al = sAlpha[((jt - 1) & 1) * BM + my_row];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) O[i] = fmaf(O[i], al, v[i]);
+      tc_fence_before();
+    }
+
+    // ---- exact scores: tensor memory (row per thread) -> shared memory, 16-byte XOR swizzle
+    if (need_exact) {
+      if (!mbar_wait(BAR(BAR_S), n_exact & 1)) sMisc[1] = 1;
+      tc_fence_after();
+      unsigned char* sx_row = sm + OFF_SX + (size_t)my_row * 512;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float v[16];
+        tc_ld16(tmem + TMEM_S + 32 * sub + 16 * half + ((uint32_t)(32 * qd) << 16), v);
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const int chunk = 8 * sub + 4 * half + q4;
+          *reinterpret_cast<float4*>(sx_row + ((chunk ^ lane) << 4)) =
+              make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+        }
+      }
+      tc_fence_before();
+      __syncthreads();     // (B) exact scores visible
+      if (sMisc[1]) { aborted = true; break; }
+    }
+
+    // ---- pass 1: hybrid select (Section III-B): exact inside the window, running sum outside
+    {
+      float bs[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      if (need_delta) {
+        for (int r2 = 0; r2 < NWARP; ++r2) {
+          const float4 s4 = *reinterpret_cast<const float4*>(sSeed + r2 * BN + 4 * lane);
+          bs[0] += s4.x; bs[1] += s4.y; bs[2] += s4.z; bs[3] += s4.w;
+        }
+        for (int r2 = 0; r2 < rg; ++r2) {
+          const float4 t4 = *reinterpret_cast<const float4*>(sTot + r2 * BN + 4 * lane);
+          bs[0] += t4.x; bs[1] += t4.y; bs[2] += t4.z; bs[3] += t4.w;
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        const int row = rg * 8 + r;
+        const int i = i0 + row;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) Sl[r][k] += bs[k];
+        if (need_exact) {
+          int wlo, whi;   // exact keys of row i: wlo <= j < whi
+          if (shape == 0) { wlo = (i / W) * W; whi = wlo + W; }
+          else { wlo = i - W + 1; whi = i + 1; }
+          const float4 e4 = *reinterpret_cast<const float4*>(sm + OFF_SX + (size_t)row * 512 +
+                                                             ((lane ^ (row & 31)) << 4));
+          const float ex[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int j = j0 + 4 * lane + k;
+            if (j >= wlo && j < whi) Sl[r][k] = ex[k];
+          }
+        }
+      }
+    }
+    if (need_exact) {
+      fence_proxy_async();
+      __syncthreads();     // (C) every exact score is in registers; its buffer may be reused
+      if (tid == 0 && more) {
+        mbar_expect_tx(BAR(BAR_KT), 64 * 128 * 4);
+        tma_load_3d(base + OFF_KT, &tm_kt, BAR(BAR_KT), j0 + BN, 0, bkv);
+        if (tile_needs_exact(jt + 1)) {
+          mbar_expect_tx(BAR(BAR_K), SZ_TILE);
+          tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K), 0, j0 + BN, bkv);
+        }
+      }
+      ++n_exact;
+    }
+
+    // ---- pass 2: scale, causal mask, online softmax (Eq. 1); P as bf16 in operand layout
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      const int row = rg * 8 + r;
+      float s[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        s[k] = Sl[r][k] * p.scale_log2e;
+        if (diag && (4 * lane + k > row)) s[k] = -INFINITY;
+      }
+      float mx = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float m_old = sM[row];
+      const float m_new = fmaxf(m_old, mx);
+      float pr[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) pr[k] = exp2f(s[k] - m_new);
+      float sum = (pr[0] + pr[1]) + (pr[2] + pr[3]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(pr[0], pr[1]);
+      const __nv_bfloat162 hi = __floats2bfloat162_rn(pr[2], pr[3]);
+      uint2 pk;
+      pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+      unsigned char* pp = sm + OFF_P + (size_t)(lane >> 4) * SZ_TILE + (size_t)row * 128 +
+                          ((((lane & 15) >> 1) ^ (row & 7)) << 4) + ((lane & 1) << 3);
+      *reinterpret_cast<uint2*>(pp) = pk;
+      __syncwarp();
+      if (lane == 0) {
+        const float al = exp2f(m_old - m_new);
+        sAlpha[(jt & 1) * BM + row] = al;
+        sL[row] = fmaf(sL[row], al, sum);
+        sM[row] = m_new;
+      }
+    }
+    fence_proxy_async();   // P was written through the generic proxy, the tensor cores read it
+    __syncthreads();       // (D)
+    if (sMisc[1]) { aborted = true; break; }
+
+    // ---- P.V on the tensor cores; next value tile into the other buffer
+    if (tid == 0) {
+      if (!mbar_wait(BAR(BAR_V0 + (jt & 1)), (jt >> 1) & 1)) sMisc[1] = 1;
+      tc_fence_after();
+      const uint32_t vbase = base + OFF_V + (jt & 1) * SZ_TILE;
+#pragma unroll
+      for (int ks = 0; ks < BN / 16; ++ks) {
+        const uint64_t da = make_desc(base + OFF_P + (ks >> 2) * SZ_TILE + (ks & 3) * 32, 16, 1024);
+        const uint64_t db = make_desc(vbase + ks * 2048, SZ_TILE, 1024);
+        tc_mma(tmem + TMEM_O, da, db, IDESC_PV, ks > 0 ? 1u : 0u);
+      }
+      tc_commit(BAR(BAR_O));
+      if (more) {
+        const int nb = (jt + 1) & 1;
+        mbar_expect_tx(BAR(BAR_V0 + nb), SZ_TILE);
+        tma_load_3d(base + OFF_V + nb * SZ_TILE, &tm_v, BAR(BAR_V0 + nb), 0, j0 + BN, bkv);
+      }
+    }
+  }
+
+  // ---- last tile's P.V, normalisation, store ---------------------------------------------
+  if (!aborted) {
+    if (!mbar_wait(BAR(BAR_O), qt & 1)) sMisc[1] = 1;
+    tc_fence_after();
+    float v[16];
+    tc_ld16(tmem + TMEM_O + 16 * sub + ((uint32_t)(32 * qd) << 16), v);
+    const float al = sAlpha[(qt & 1) * BM + my_row];
+    const float inv = 1.0f / sL[my_row];
+    if (i0 + my_row < T && !sMisc[1]) {
+      uint32_t w[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const __nv_bfloat162 t2 = __floats2bfloat162_rn(fmaf(O[2 * i], al, v[2 * i]) * inv,
+                                                        fmaf(O[2 * i + 1], al, v[2 * i + 1]) * inv);
+        w[i] = *reinterpret_cast<const uint32_t*>(&t2);
+      }
+      uint4* op = reinterpret_cast<uint4*>(p.out + ((size_t)bh * T + i0 + my_row) * TC_D + 16 * sub);
+      op[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      op[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+    tc_fence_before();
+  } else {
+    // a wait ran out: give copies and tensor-core work already in flight time to land
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (tid == 0 && sMisc[1]) atomicMax(&p.counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS)
+                 : "memory");
+  }
+#undef BAR
+}
+
+// ---------------------------------------------------------------------------------------
+// Channel-major fp32 copy of the keys, kt[b, kv head, c, j] = k[b, kv head, j, c]: the operand
+// layout of the FP32 delta update (a lane reads 4 consecutive keys of one channel).
+__global__ void __launch_bounds__(256) keys_channel_major_kernel(const __nv_bfloat16* __restrict__ k,
+                                                                 float* __restrict__ kt, int T,
+                                                                 int T_max, int ld) {
+  __shared__ float tile[TC_D][65];
+  const int bkv = blockIdx.y;
+  const int j0 = blockIdx.x * 64;
+  const __nv_bfloat16* kp = k + (size_t)bkv * T_max * TC_D;
+  for (int e = threadIdx.x; e < 64 * TC_D; e += 256) {
+    const int j = e / TC_D, c = e - j * TC_D;
+    tile[c][j] = (j0 + j < T) ? __bfloat162float(kp[(size_t)(j0 + j) * TC_D + c]) : 0.0f;
+  }
+  __syncthreads();
+  float* op = kt + (size_t)bkv * TC_D * ld;
+  for (int e = threadIdx.x; e < 64 * TC_D; e += 256) {
+    const int c = e >> 6, j = e & 63;
+    if (j0 + j < ld) op[(size_t)c * ld + j0 + j] = tile[c][j];
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return (EncodeTiledFn)f;
+  }();
+  return fn;
+}
+
+// 3-d map over [outer][rows][inner]; the box is [1][box_rows][box_inner].
+bool encode3(CUtensorMap* m, CUtensorMapDataType dt, size_t es, const void* ptr, uint64_t inner,
+             uint64_t rows, uint64_t outer, uint64_t row_stride_b, uint64_t outer_stride_b,
+             uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle sw) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {inner, rows, outer};
+  const cuuint64_t strides[2] = {row_stride_b, outer_stride_b};
+  const cuuint32_t box[3] = {box_inner, box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  (void)es;
+  return fn(m, dt, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace
+
+bool tc_kernel_shape(int d) { return d == TC_D; }
+bool tc_kernel_available(int d) { return d == TC_D && encode_fn() != nullptr; }
+
+cudaError_t launch_hybrid_attn_tc(const Shape& s, const Workspace& w, const void* q, const void* k,
+                                  const void* v, void* out, int T, int window, int shape,
+                                  cudaStream_t st) {
+  if (s.d != TC_D || !w.kt) return cudaErrorNotSupported;
+  const int ld = (s.T_max + 3) / 4 * 4;
+  const uint64_t BH = (uint64_t)s.B * s.H, BKV = (uint64_t)s.B * s.H_kv;
+  CUtensorMap tq, tk, tv, tkt;
+  const bool ok =
+      encode3(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, q, TC_D, (uint64_t)T, BH, TC_D * 2,
+              (uint64_t)T * TC_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, k, TC_D, (uint64_t)T, BKV, TC_D * 2,
+              (uint64_t)s.T_max * TC_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, v, TC_D, (uint64_t)T, BKV, TC_D * 2,
+              (uint64_t)s.T_max * TC_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tkt, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w.kt, (uint64_t)T, TC_D, BKV, (uint64_t)ld * 4,
+              (uint64_t)ld * TC_D * 4, 128, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
+  if (!ok) return cudaErrorInvalidValue;
+
+  const dim3 gk((T + 63) / 64, (unsigned)BKV);
+  keys_channel_major_kernel<<<gk, 256, 0, st>>>((const __nv_bfloat16*)k, w.kt, T, s.T_max, ld);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  count_launch();
+
+  err = cudaFuncSetAttribute(hybrid_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)SMEM_BYTES);
+  if (err != cudaSuccess) return err;
+  TcParams p;
+  p.dq = w.dq; p.mask = w.mask; p.qhat_tile = w.qhat_tile; p.out = (__nv_bfloat16*)out;
+  p.counters = w.counters;
+  p.T = T; p.T_max = s.T_max; p.n_tiles64 = s.n_tiles; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
+  p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
+  const dim3 grid((T + BM - 1) / BM, (unsigned)BH);
+  hybrid_attn_tc_kernel<<<grid, NTHR, SMEM_BYTES, st>>>(tq, tk, tv, tkt, p);
+  count_launch();
+  return cudaGetLastError();
+}
+
 }  // namespace delta

@@ -5,6 +5,8 @@
 namespace delta {
 // Does this build carry a tensor-core prefill kernel for head dimension d?
 bool tc_kernel_available(int d);
+// Is head dimension d one the tensor-core kernel is written for (no driver query)?
+bool tc_kernel_shape(int d);
 cudaError_t launch_hybrid_attn_tc(const Shape& s, const Workspace& w, const void* q, const void* k,
                                   const void* v, void* out, int T, int window, int shape,
                                   cudaStream_t st);
