@@ -34,30 +34,35 @@ namespace {
 
 constexpr int BM = 128, BN = 128, NTHR = 512, NWARP = 16;
 constexpr int TC_D = 64;                 // head dimension served by this kernel
-constexpr int DQ_LD = BM + 4;            // leading dimension of the channel-major delta tile
 constexpr uint32_t TMEM_COLS = 256;      // S: columns 0..127, O: columns 128..191
 constexpr uint32_t TMEM_S = 0, TMEM_O = 128;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t SZ_TILE = 128 * 64 * 2;               // one bf16 operand tile, 16 KiB
+constexpr uint32_t ROW_B = 128 * 4;                      // one channel row of the fp32 tiles
+constexpr uint32_t PAD_OFF = 64 * ROW_B;                 // row 64 of both fp32 tiles: padding target
 constexpr uint32_t OFF_Q = 0;
 constexpr uint32_t OFF_K = OFF_Q + SZ_TILE;
 constexpr uint32_t OFF_V = OFF_K + SZ_TILE;              // two buffers
-constexpr uint32_t OFF_KT = OFF_V + 2 * SZ_TILE;         // fp32 [64 channels][128 keys]
-constexpr uint32_t OFF_P = OFF_KT + 64 * 128 * 4;        // bf16 [2][128 rows][64 keys]
-constexpr uint32_t OFF_SX = OFF_KT;                      // fp32 [128][128] exact scores (KT + P)
-constexpr uint32_t OFF_DQT = OFF_P + 2 * SZ_TILE;        // fp32 [64][DQ_LD]
-constexpr uint32_t OFF_TOT = OFF_DQT + 64 * DQ_LD * 4;   // fp32 [16][128]
-constexpr uint32_t OFF_SEED = OFF_TOT + 16 * 128 * 4;    // fp32 [16][128]
-constexpr uint32_t OFF_ALPHA = OFF_SEED + 16 * 128 * 4;  // fp32 [2][128]
+constexpr uint32_t OFF_KT = OFF_V + 2 * SZ_TILE;         // fp32 [64 channels + 1][128 keys]
+constexpr uint32_t OFF_P = OFF_KT + 65 * ROW_B + 512;    // bf16 [2][128 rows][64 keys]
+constexpr uint32_t OFF_SX = OFF_KT;                      // fp32 [128][128] exact scores (over KT, P)
+constexpr uint32_t OFF_DQT = OFF_P + 2 * SZ_TILE;        // fp32 [64 channels + 1][128 rows]
+constexpr uint32_t OFF_LIST = OFF_DQT + 65 * ROW_B;      // u32 [32 blocks][64]: fired channel * ROW_B
+constexpr uint32_t OFF_CNT = OFF_LIST + 32 * 64 * 4;     // u32 [32]: list length / 4
+constexpr uint32_t OFF_TOT = OFF_CNT + 32 * 4;           // fp32 [16][128]
+constexpr uint32_t OFF_SEED = OFF_TOT + 16 * 128 * 4;    // fp32 [128]
+constexpr uint32_t OFF_ALPHA = OFF_SEED + 128 * 4;       // fp32 [2][128]
 constexpr uint32_t OFF_M = OFF_ALPHA + 2 * 128 * 4;      // fp32 [128] running max
 constexpr uint32_t OFF_L = OFF_M + 128 * 4;              // fp32 [128] running sum
 constexpr uint32_t OFF_QHAT = OFF_L + 128 * 4;           // fp32 [64]
-constexpr uint32_t OFF_UNION = OFF_QHAT + 64 * 4;        // u64 [32] block masks
-constexpr uint32_t OFF_BAR = OFF_UNION + 32 * 8;         // 8 mbarriers
+constexpr uint32_t OFF_BAR = OFF_QHAT + 64 * 4;          // 8 mbarriers
 constexpr uint32_t OFF_MISC = OFF_BAR + 8 * 8;           // tmem slot, abort flag
 constexpr uint32_t SMEM_USED = OFF_MISC + 16;
 constexpr uint32_t SMEM_BYTES = SMEM_USED + 1024;        // slack for the alignment of the base
+static_assert(OFF_P % 1024 == 0 && OFF_KT % 1024 == 0, "operand tiles need 1024-byte alignment");
+static_assert(OFF_P + 2 * SZ_TILE - OFF_SX >= 128 * 128 * 4, "exact-score buffer must fit");
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 enum Bar { BAR_Q = 0, BAR_K, BAR_KT, BAR_V0, BAR_V1, BAR_S, BAR_O };
 
@@ -172,13 +177,14 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
   float* sKt = reinterpret_cast<float*>(sm + OFF_KT);
   float* sdQt = reinterpret_cast<float*>(sm + OFF_DQT);
+  uint32_t* sList = reinterpret_cast<uint32_t*>(sm + OFF_LIST);
+  uint32_t* sCnt = reinterpret_cast<uint32_t*>(sm + OFF_CNT);
   float* sTot = reinterpret_cast<float*>(sm + OFF_TOT);
   float* sSeed = reinterpret_cast<float*>(sm + OFF_SEED);
   float* sAlpha = reinterpret_cast<float*>(sm + OFF_ALPHA);
   float* sM = reinterpret_cast<float*>(sm + OFF_M);
   float* sL = reinterpret_cast<float*>(sm + OFF_L);
   float* sQhat = reinterpret_cast<float*>(sm + OFF_QHAT);
-  unsigned long long* sUnion = reinterpret_cast<unsigned long long*>(sm + OFF_UNION);
   volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
   const uint32_t bar0 = base + OFF_BAR;
 #define BAR(i) (bar0 + 8u * (uint32_t)(i))
@@ -187,8 +193,8 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const int qd = warp & 3, sub = warp >> 2;     // tensor-memory lane quadrant / slot in it
   const int rg = qd * 4 + sub;                  // row group: rows 8*rg .. 8*rg+7
   const int my_row = 32 * qd + lane;            // row this thread owns in row-per-thread phases
-  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;  // heaviest query tiles first
-  const int bh = blockIdx.y;
+  const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;  // heaviest query tiles of every head first
+  const int bh = blockIdx.x;
   const int b = bh / p.H, h = bh - b * p.H;
   const int bkv = b * (p.H / p.g) + h / p.g;
   const int i0 = qt * BM;
@@ -242,7 +248,9 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     }
   }
 
-  // ---- stage the query tile's deltas channel-major, the block masks and the seed reference
+  // ---- stage the query tile: deltas channel-major, per 4-row block the list of channels that
+  // fired anywhere in the block (ballot of the mask words, popc for the position), the seed
+  // reference, the softmax state
   {
     const float* dqp = p.dq + ((size_t)bh * p.T_max + i0) * TC_D;
     const int r_sub = lane >> 3, c_sub = lane & 7;
@@ -250,16 +258,30 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       const int rb = it >> 3, cb = it & 7;
       const int r = rb * 4 + r_sub, c = cb * 8 + c_sub;
       const float x = (i0 + r < T) ? dqp[(size_t)r * TC_D + c] : 0.0f;
-      sdQt[c * DQ_LD + r] = x;
+      sdQt[c * BM + r] = x;
     }
-    if (tid < 32) {
+    if (tid < 128) {                 // row 64 of both fp32 tiles: where list padding points
+      sdQt[64 * BM + tid] = 0.0f;
+      sKt[64 * BN + tid] = 0.0f;
+    }
+    {
+      const int blk = tid >> 4, sl = tid & 15;       // 16 threads per block of 4 rows
       unsigned long long u = 0;
-      const uint32_t* mp = p.mask + ((size_t)bh * p.T_max + i0) * 2;
-      for (int r = 0; r < 4; ++r) {
-        const int row = tid * 4 + r;
-        if (i0 + row < T) u |= (unsigned long long)mp[row * 2] | ((unsigned long long)mp[row * 2 + 1] << 32);
+      const uint32_t* mp = p.mask + ((size_t)bh * p.T_max + i0 + blk * 4) * 2;
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+        if (i0 + blk * 4 + r < T)
+          u |= (unsigned long long)mp[r * 2] | ((unsigned long long)mp[r * 2 + 1] << 32);
+      const int n = __popcll(u);
+      uint32_t* lp = sList + blk * 64;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int c = sl * 4 + k;
+        if ((u >> c) & 1ull) lp[__popcll(u & ((1ull << c) - 1ull))] = (uint32_t)c * ROW_B;
       }
-      sUnion[tid] = u;
+      const int n4 = (n + 3) >> 2;
+      if (sl < 3 && n + sl < n4 * 4) lp[n + sl] = PAD_OFF;
+      if (sl == 0) sCnt[blk] = (uint32_t)n4;
     }
     if (tid < TC_D) sQhat[tid] = p.qhat_tile[((size_t)bh * p.n_tiles64 + 2 * qt) * TC_D + tid];
     if (tid < BM) { sM[tid] = -INFINITY; sL[tid] = 0.0f; }
@@ -304,7 +326,7 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     if (!mbar_wait(BAR(BAR_KT), jt & 1)) sMisc[1] = 1;
     if (need_delta) {
       float run[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      const float* ktp = sKt + 4 * lane;
+      const unsigned char* ktb = reinterpret_cast<const unsigned char*>(sKt) + 16 * lane;
 #pragma unroll
       for (int g4 = 0; g4 < 2; ++g4) {
         float a[4][4];
@@ -312,19 +334,28 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         for (int r = 0; r < 4; ++r)
 #pragma unroll
           for (int k = 0; k < 4; ++k) a[r][k] = 0.0f;
-        unsigned long long m = sUnion[rg * 2 + g4];
-        const float* dqg = sdQt + rg * 8 + g4 * 4;
-        while (m) {
-          const int c = __ffsll((long long)m) - 1;
-          m &= m - 1;
-          const float4 kv = *reinterpret_cast<const float4*>(ktp + c * BN);
-          const float4 dv = *reinterpret_cast<const float4*>(dqg + c * DQ_LD);
-          const float kk[4] = {kv.x, kv.y, kv.z, kv.w};
-          const float dd[4] = {dv.x, dv.y, dv.z, dv.w};
+        const int blk = rg * 2 + g4;
+        const unsigned char* dqb = reinterpret_cast<const unsigned char*>(sdQt) + 16 * blk;
+        const uint4* lp = reinterpret_cast<const uint4*>(sList + blk * 64);
+        const int n4 = (int)sCnt[blk];
+        for (int q4 = 0; q4 < n4; ++q4) {
+          const uint4 e = lp[q4];
+          const uint32_t off[4] = {e.x, e.y, e.z, e.w};
+          float4 kv[4], dv[4];
 #pragma unroll
-          for (int r = 0; r < 4; ++r)
+          for (int u = 0; u < 4; ++u) {
+            kv[u] = *reinterpret_cast<const float4*>(ktb + off[u]);
+            dv[u] = *reinterpret_cast<const float4*>(dqb + off[u]);
+          }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) a[r][k] = fmaf(dd[r], kk[k], a[r][k]);
+          for (int u = 0; u < 4; ++u) {
+            const float kk[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+            const float dd[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+              for (int k = 0; k < 4; ++k) a[r][k] = fmaf(dd[r], kk[k], a[r][k]);
+          }
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r)
@@ -334,18 +365,20 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             Sl[g4 * 4 + r][k] = run[k];
           }
       }
-      // this warp's slice of the seed q_hat(i0-1).k_j: channels 4*rg .. 4*rg+3
-      float sd[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int c = rg * 4 + cc;
-        const float x = sQhat[c];
-        const float4 kv = *reinterpret_cast<const float4*>(ktp + c * BN);
-        sd[0] = fmaf(x, kv.x, sd[0]); sd[1] = fmaf(x, kv.y, sd[1]);
-        sd[2] = fmaf(x, kv.z, sd[2]); sd[3] = fmaf(x, kv.w, sd[3]);
-      }
       *reinterpret_cast<float4*>(sTot + rg * BN + 4 * lane) = make_float4(run[0], run[1], run[2], run[3]);
-      *reinterpret_cast<float4*>(sSeed + rg * BN + 4 * lane) = make_float4(sd[0], sd[1], sd[2], sd[3]);
+      // seed q_hat(i0-1).k_j: this warp serves keys 8*warp .. 8*warp+7, 16 channels per lane
+      if (qt > 0) {
+        const int kq = lane & 7, cq = lane >> 3;
+        const float* kp = sKt + cq * 16 * BN + 8 * warp + kq;
+        float sd = 0.0f;
+#pragma unroll
+        for (int cc = 0; cc < 16; ++cc) sd = fmaf(sQhat[cq * 16 + cc], kp[cc * BN], sd);
+        sd += __shfl_xor_sync(0xffffffffu, sd, 8);
+        sd += __shfl_xor_sync(0xffffffffu, sd, 16);
+        if (lane < 8) sSeed[8 * warp + lane] = sd;
+      } else if (lane < 8) {
+        sSeed[8 * warp + lane] = 0.0f;
+      }
     }
     fence_proxy_async();   // generic reads of the key tile are ordered before its next bulk write
     __syncthreads();       // (A) totals and seed slices visible; channel-major key tile free
@@ -398,10 +431,8 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     {
       float bs[4] = {0.0f, 0.0f, 0.0f, 0.0f};
       if (need_delta) {
-        for (int r2 = 0; r2 < NWARP; ++r2) {
-          const float4 s4 = *reinterpret_cast<const float4*>(sSeed + r2 * BN + 4 * lane);
-          bs[0] += s4.x; bs[1] += s4.y; bs[2] += s4.z; bs[3] += s4.w;
-        }
+        const float4 s4 = *reinterpret_cast<const float4*>(sSeed + 4 * lane);
+        bs[0] = s4.x; bs[1] = s4.y; bs[2] = s4.z; bs[3] = s4.w;
         for (int r2 = 0; r2 < rg; ++r2) {
           const float4 t4 = *reinterpret_cast<const float4*>(sTot + r2 * BN + 4 * lane);
           bs[0] += t4.x; bs[1] += t4.y; bs[2] += t4.z; bs[3] += t4.w;
@@ -630,7 +661,7 @@ cudaError_t launch_hybrid_attn_tc(const Shape& s, const Workspace& w, const void
   p.counters = w.counters;
   p.T = T; p.T_max = s.T_max; p.n_tiles64 = s.n_tiles; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
   p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
-  const dim3 grid((T + BM - 1) / BM, (unsigned)BH);
+  const dim3 grid((unsigned)BH, (T + BM - 1) / BM);
   hybrid_attn_tc_kernel<<<grid, NTHR, SMEM_BYTES, st>>>(tq, tk, tv, tkt, p);
   count_launch();
   return cudaGetLastError();
