@@ -105,6 +105,7 @@ DELTA_API delta_status_t delta_state_destroy(delta_state_t* st);
  *   q, out : [B, H, T, d]            k, v : [B, H_kv, T_max, d] (KV-cache layout, rows 0..T-1 read)
  *   theta  : delta threshold of Eq. 2 (>= 0, finite); |diff| == theta does not fire
  *   window : W of Section III-B (>= 0), shape from the configuration
+ * q, k, v and out must be 16-byte aligned.
  * Steps enqueued: delta construction over Q (Eq. 2-3: values, bit mask, per-row and per-tile
  * non-zero counts, compacted channel indices, per-tile reference snapshots), the fused
  * hybrid-attention kernel (exact q.k inside the window, running delta sums outside (Eq. 4),
@@ -229,7 +230,8 @@ DELTA_API delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32
  * event in front of and behind each of its kernels on the caller's stream (host-side event
  * objects; no device memory).  delta_state_prefill_kernel_ms waits for the last event and
  * returns the elapsed milliseconds of the most recent prefill in ms[0..3]:
- * [0] delta construction, [1] sparsity counters, [2] hybrid attention, [3] decode hand-off.
+ * [0] delta chain (Eq. 2-3), [1] counts, compacted indices, Eq. 6 counters, decode hand-off and
+ * key re-layout, [2] hybrid attention, [3] reserved (0).
  * DELTA_ERR_STATE if profiling is off or no prefill was recorded. */
 DELTA_API delta_status_t delta_state_enable_profiling(delta_state_t* st, int32_t enable);
 DELTA_API delta_status_t delta_state_prefill_kernel_ms(delta_state_t* st, float* ms);

@@ -202,6 +202,7 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
                                   void* out, int32_t T, int32_t H, int32_t H_kv, int32_t d,
                                   float theta, int32_t window, void* stream) {
   if (!st || !q || !k || !v || !out) return DELTA_ERR_INVALID_ARG;
+  if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return DELTA_ERR_INVALID_ARG;
   const delta_config_t& c = st->cfg;
   if (H != c.H || H_kv != c.H_kv || d != c.d) return DELTA_ERR_INVALID_ARG;
   delta_status_t s = check_theta_window(theta, window);
@@ -213,14 +214,16 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   cudaError_t e;
   const bool prof = st->profiling;
 #define MARK(i) do { if (prof && (e = cudaEventRecord(st->ev[i], cs)) != cudaSuccess) return cuda_fail(e); } while (0)
+  const bool use_tc = delta_state_prefill_kernel(st) == 1;
   MARK(0);
-  if ((e = launch_delta_construct(st->shape, st->ws, q, T, theta, c.dtype, c.init, cs)) != cudaSuccess)
+  if ((e = launch_delta_chain(st->shape, st->ws, q, T, theta, c.dtype, c.init, cs)) != cudaSuccess)
     return cuda_fail(e);
   MARK(1);
-  if ((e = launch_prefill_stats(st->shape, st->ws, T, window, c.prefill_window, cs)) != cudaSuccess)
+  if ((e = launch_delta_finish(st->shape, st->ws, k, T, window, c.prefill_window, c.dtype, use_tc, cs)) !=
+      cudaSuccess)
     return cuda_fail(e);
   MARK(2);
-  if (delta_state_prefill_kernel(st) == 1) {
+  if (use_tc) {
     e = launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
   } else {
     e = launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window,
@@ -228,7 +231,6 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   }
   if (e != cudaSuccess) return cuda_fail(e);
   MARK(3);
-  if ((e = launch_handoff(st->shape, st->ws, k, T, c.dtype, 0, cs)) != cudaSuccess) return cuda_fail(e);
   MARK(4);
 #undef MARK
   st->profiled = prof;

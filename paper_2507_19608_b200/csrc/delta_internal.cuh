@@ -43,19 +43,18 @@ struct Shape {
 
 void count_launch(int n = 1);
 
-// K1: delta construction over the query stream (Eq. 2-3).
-cudaError_t launch_delta_construct(const Shape& s, const Workspace& w, const void* q, int T,
-                                   float theta, int dtype, int init, cudaStream_t st);
-// K4: sparsity counters of the prefill stage (Eq. 6 inputs).
-cudaError_t launch_prefill_stats(const Shape& s, const Workspace& w, int T, int window, int shape,
-                                 cudaStream_t st);
+// K1a: token-sequential delta chain over the query stream (Eq. 2-3): delta values, mask words,
+// per-tile reference snapshots, final reference.
+cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
+                               float theta, int dtype, int init, cudaStream_t st);
+// K1b: row-parallel finish: counts, compacted indices, Eq. 6 counters, the decode hand-off row
+// R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
+cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* k, int T,
+                                int window, int shape, int dtype, bool want_kt, cudaStream_t st);
 // K2 (generic): fused hybrid attention on CUDA cores, any supported dtype.
 cudaError_t launch_hybrid_attn_generic(const Shape& s, const Workspace& w, const void* q,
                                        const void* k, const void* v, void* out, int T, int window,
                                        int shape, int dtype, cudaStream_t st);
-// Hand-off: R(T-1)[j] = q_hat . k_j for j < T.
-cudaError_t launch_handoff(const Shape& s, const Workspace& w, const void* k, int T, int dtype,
-                           int qhat_sel, cudaStream_t st);
 // K3: one decode step.
 cudaError_t launch_decode_step(const Shape& s, const Workspace& w, const void* q_new,
                                const void* k_new, const void* v_new, void* k_cache, void* v_cache,

@@ -1,141 +1,183 @@
 // K1 -- delta construction over the query stream (Section II-C, Eq. 2-3; Section III-A
-// strategy (1)).  One thread owns one channel chain and walks the tokens in order; a warp
-// owns 32 adjacent channels, so every row is one coalesced load and one coalesced store and
-// the row's mask word is a single ballot.  Loads do not depend on the carried state, so they
-// are issued one batch of rows ahead of the compare/select chain.
+// strategy (1)), in two kernels.
 //
-// Outputs per (batch, head): delta values (fp32, +0 where not fired), bit mask, per-row and
-// per-tile non-zero counts, compacted channel indices, the reference state in front of every
-// 64-row tile, and the final reference state.
+// delta_chain_kernel: the token-sequential part.  Eq. 3 makes every channel a chain along the
+// tokens (the reference is the last value that fired), so the only parallelism is across
+// channels: one thread per channel, one warp per 32 channels (= one mask word), one CTA per
+// (batch, head).  The chain itself is three dependent FP32 operations per token; everything
+// else is kept off it: a producer warp streams the head's query rows into a ring of
+// shared-memory stages with bulk asynchronous copies (the rows do not depend on the carried
+// state), delta values leave with one coalesced store per row, the row's mask word is a
+// single ballot parked in the lane whose index is the row number and stored once per 32 rows.
+//
+// delta_finish_kernel: everything that is parallel over rows once the mask exists -- per-row
+// and per-tile non-zero counts, the compacted channel indices, the counters behind Eq. 6 --
+// plus two passes over the keys that prefill needs anyway: the hand-off row
+// R(T-1)[j] = q_hat(T-1).k_j for decode and, for the tensor-core attention kernel, the
+// channel-major fp32 copy of the keys.
 #include "delta_internal.cuh"
 
 namespace delta {
 
-constexpr int kBatchRows = 16;  // rows loaded ahead of the dependent chain
+namespace {
 
-template <typename TIn, int D>
-__global__ void __launch_bounds__(D) delta_construct_kernel(
-    const TIn* __restrict__ q, float* __restrict__ dq, uint32_t* __restrict__ mask,
-    uint16_t* __restrict__ row_nnz, uint32_t* __restrict__ tile_nnz, uint8_t* __restrict__ idx,
-    float* __restrict__ qhat_tile, __nv_bfloat16* __restrict__ qhat_tile_bf16,
-    float* __restrict__ qhat_out, unsigned long long* __restrict__ counters, int T, int T_max,
-    int n_tiles, float theta, int basis_exact) {
-  constexpr int NW = D / 32;
-  const int bh = blockIdx.x;
-  const int c = threadIdx.x;
-  const int lane = c & 31, warp = c >> 5;
-  const TIn* qp = q + (size_t)bh * T * D + c;
-  float* dqp = dq + (size_t)bh * T_max * D + c;
-  uint32_t* maskp = mask + (size_t)bh * T_max * NW;
-  uint16_t* nnzp = row_nnz + (size_t)bh * T_max;
-  uint8_t* idxp = idx + (size_t)bh * T_max * D;
+constexpr int RC = 32;       // rows per ring stage (one mask flush per stage)
+constexpr int NS = 8;        // ring stages
 
-  __shared__ uint32_t smask[DELTA_TILE_ROWS][NW];
-  __shared__ uint32_t s_tile_sum;
-  __shared__ unsigned long long s_total;
-  if (c == 0) { s_tile_sum = 0; s_total = 0; }
-
-  float qh = 0.0f;  // reference state, starts at zero (Eq. 3)
-  float cur[kBatchRows], nxt[kBatchRows];
-  const int n_batches = (T + kBatchRows - 1) / kBatchRows;
-#pragma unroll
-  for (int r = 0; r < kBatchRows; ++r) cur[r] = (r < T) ? to_f32(qp[(size_t)r * D]) : 0.0f;
-
-  for (int b = 0; b < n_batches; ++b) {
-    const int t0 = b * kBatchRows;
-    // rows of the next batch: in flight while this batch's chain runs
-    {
-      const int t1 = t0 + kBatchRows;
-#pragma unroll
-      for (int r = 0; r < kBatchRows; ++r)
-        nxt[r] = (t1 + r < T) ? to_f32(qp[(size_t)(t1 + r) * D]) : 0.0f;
-    }
-    if ((t0 % DELTA_TILE_ROWS) == 0) {
-      const size_t o = ((size_t)bh * n_tiles + t0 / DELTA_TILE_ROWS) * D + c;
-      qhat_tile[o] = qh;
-      if (qhat_tile_bf16) qhat_tile_bf16[o] = __float2bfloat16_rn(qh);
-    }
-#pragma unroll
-    for (int r = 0; r < kBatchRows; ++r) {
-      const int t = t0 + r;
-      if (t < T) {  // uniform across the block
-        const float x = cur[r];
-        bool fire;
-        float delta;
-        if (t == 0 && basis_exact) {
-          fire = true;           // the basis vector is kept whole
-          delta = x;
-        } else {
-          const float diff = __fsub_rn(x, qh);   // one IEEE subtraction
-          fire = fabsf(diff) > theta;            // strict; NaN compares false
-          delta = fire ? diff : 0.0f;
-        }
-        qh = fire ? x : qh;
-        dqp[(size_t)t * D] = delta;
-        const uint32_t m = __ballot_sync(0xffffffffu, fire);
-        if (lane == 0) smask[t % DELTA_TILE_ROWS][warp] = m;
-      }
-    }
-#pragma unroll
-    for (int r = 0; r < kBatchRows; ++r) cur[r] = nxt[r];
-
-    // end of a 64-row tile (or of the stream): emit mask words, counts and compacted indices
-    const int t_end = min(t0 + kBatchRows, T);
-    if ((t_end % DELTA_TILE_ROWS) == 0 || t_end == T) {
-      __syncthreads();
-      const int tile = (t_end - 1) / DELTA_TILE_ROWS;
-      const int tile_t0 = tile * DELTA_TILE_ROWS;
-      const int rows = t_end - tile_t0;
-      uint32_t my_sum = 0;
-      for (int r = warp; r < rows; r += NW) {
-        const int t = tile_t0 + r;
-        uint32_t m[NW];
-        int nnz = 0;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) { m[w] = smask[r][w]; nnz += __popc(m[w]); }
-        int base = 0;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) {
-          if ((m[w] >> lane) & 1u) {
-            const int pos = base + __popc(m[w] & ((1u << lane) - 1u));
-            idxp[(size_t)t * D + pos] = (uint8_t)(w * 32 + lane);
-          }
-          base += __popc(m[w]);
-        }
-#pragma unroll
-        for (int p = lane; p < D; p += 32)
-          if (p >= nnz) idxp[(size_t)t * D + p] = 0xFF;
-        if (lane < NW) maskp[(size_t)t * NW + lane] = smask[r][lane];
-        if (lane == 0) { nnzp[t] = (uint16_t)nnz; my_sum += nnz; }
-      }
-      if (lane == 0 && my_sum) atomicAdd(&s_tile_sum, my_sum);
-      __syncthreads();
-      if (c == 0) {
-        tile_nnz[(size_t)bh * n_tiles + tile] = s_tile_sum;
-        s_total += s_tile_sum;
-        s_tile_sum = 0;
-      }
-      // smask and s_tile_sum are reused by the next tile only after the next __syncthreads
-      // pair above, and lane 0 of each warp writes smask rows of the next tile only after
-      // every warp has passed the second barrier.
-    }
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait (about a second of SM clock); false if it ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > 2000000000ll) return false;
   }
-  qhat_out[(size_t)bh * D + c] = qh;
-  __syncthreads();
-  if (c == 0) {
-    atomicAdd(&counters[CNT_PREFILL_NNZ], s_total);
-    atomicAdd(&counters[CNT_PREFILL_ELEMS], (unsigned long long)T * D);
-  }
+  return true;
 }
 
-cudaError_t launch_delta_construct(const Shape& s, const Workspace& w, const void* q, int T,
-                                   float theta, int dtype, int init, cudaStream_t st) {
+}  // namespace
+
+template <typename TIn, int D>
+__global__ void __launch_bounds__(D + 32) delta_chain_kernel(
+    const TIn* __restrict__ q, float* __restrict__ dq, uint32_t* __restrict__ mask,
+    float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
+    unsigned long long* __restrict__ counters, int T, int T_max, int n_tiles, float theta,
+    int basis_exact) {
+  constexpr int NW = D / 32;                       // chain warps = mask words per row
+  constexpr uint32_t ROW_BYTES = D * sizeof(TIn);
+  constexpr uint32_t STAGE_BYTES = RC * ROW_BYTES;
+  extern __shared__ __align__(128) unsigned char ring[];   // [NS][RC][D] of TIn
+  __shared__ __align__(8) unsigned long long bars[2 * NS];   // full[NS], empty[NS]
+  __shared__ int s_fail;
+
+  const int bh = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[NS]);
+  const int n_chunks = (T + RC - 1) / RC;
+
+  if (tid == 0) {
+    for (int s = 0; s < NS; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * s), "r"(1) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty0 + 8 * s), "r"(NW) : "memory");
+    }
+    s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == NW) {
+    // ---- producer: keeps up to NS stages of query rows in flight
+    if (lane == 0) {
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(q) + (size_t)bh * T * ROW_BYTES;
+      const uint32_t ring0 = smem_u32(ring);
+      for (int i = 0; i < n_chunks; ++i) {
+        const int s = i % NS;
+        if (i >= NS && !mbar_wait(empty0 + 8 * s, ((i / NS) - 1) & 1)) { s_fail = 1; break; }
+        const int rows = min(RC, T - i * RC);
+        const uint32_t bytes = (uint32_t)rows * ROW_BYTES;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full0 + 8 * s),
+                     "r"(bytes)
+                     : "memory");
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                ring0 + s * STAGE_BYTES),
+            "l"(src + (size_t)i * STAGE_BYTES), "r"(bytes), "r"(full0 + 8 * s)
+            : "memory");
+      }
+    }
+  } else {
+    // ---- chain warps: thread c owns channel c
+    const int c = tid;
+    float* dqp = dq + (size_t)bh * T_max * D + c;
+    uint32_t* maskp = mask + (size_t)bh * T_max * NW + warp;
+    float qh = 0.0f;          // reference state, starts at zero (Eq. 3)
+    bool failed = false;
+    for (int i = 0; i < n_chunks; ++i) {
+      const int s = i % NS;
+      const int t0 = i * RC;
+      if ((t0 % DELTA_TILE_ROWS) == 0)
+        qhat_tile[((size_t)bh * n_tiles + t0 / DELTA_TILE_ROWS) * D + c] = qh;
+      if (!mbar_wait(full0 + 8 * s, (i / NS) & 1)) { failed = true; break; }
+      const TIn* rows = reinterpret_cast<const TIn*>(ring + (size_t)s * STAGE_BYTES) + c;
+      const int nrows = min(RC, T - t0);
+      uint32_t mymask = 0;
+      if (nrows == RC && !(t0 == 0 && basis_exact)) {
+        // full stage, no basis row: the loads run ahead of the dependent chain
+#pragma unroll
+        for (int r0 = 0; r0 < RC; r0 += 8) {
+          float x[8];
+#pragma unroll
+          for (int r = 0; r < 8; ++r) x[r] = to_f32(rows[(r0 + r) * D]);
+#pragma unroll
+          for (int r = 0; r < 8; ++r) {
+            const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
+            const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
+            qh = fire ? x[r] : qh;
+            dqp[(size_t)(t0 + r0 + r) * D] = fire ? diff : 0.0f;
+            const uint32_t m = __ballot_sync(0xffffffffu, fire);
+            if (lane == r0 + r) mymask = m;
+          }
+        }
+      } else {
+        for (int r = 0; r < nrows; ++r) {
+          const float x = to_f32(rows[r * D]);
+          bool fire;
+          float delta;
+          if (t0 + r == 0 && basis_exact) {
+            fire = true;                                 // the basis vector is kept whole
+            delta = x;
+          } else {
+            const float diff = __fsub_rn(x, qh);
+            fire = fabsf(diff) > theta;
+            delta = fire ? diff : 0.0f;
+          }
+          qh = fire ? x : qh;
+          dqp[(size_t)(t0 + r) * D] = delta;
+          const uint32_t m = __ballot_sync(0xffffffffu, fire);
+          if (lane == r) mymask = m;
+        }
+      }
+      if (lane < nrows) maskp[(size_t)(t0 + lane) * NW] = mymask;
+      __syncwarp();
+      if (lane == 0)
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * s) : "memory");
+    }
+    if (!failed) qhat_out[(size_t)bh * D + c] = qh;
+    if (failed) s_fail = 1;
+  }
+  __syncthreads();
+  if (tid == 0 && s_fail) atomicMax(&counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
+}
+
+cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
+                               float theta, int dtype, int init, cudaStream_t st) {
   const int grid = s.B * s.H;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
+  cudaError_t err = cudaSuccess;
 #define LAUNCH(TIN, DD)                                                                          \
-  delta_construct_kernel<TIN, DD><<<grid, DD, 0, st>>>(                                          \
-      (const TIN*)q, w.dq, w.mask, w.row_nnz, w.tile_nnz, w.idx, w.qhat_tile, w.qhat_tile_bf16,  \
-      w.qhat[0], w.counters, T, s.T_max, s.n_tiles, theta, basis)
+  do {                                                                                           \
+    auto kern = delta_chain_kernel<TIN, DD>;                                                     \
+    const size_t smem = (size_t)NS * RC * DD * sizeof(TIN);                                      \
+    if (smem > 48 * 1024) {                                                                      \
+      err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+      if (err != cudaSuccess) return err;                                                        \
+    }                                                                                            \
+    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.dq, w.mask, w.qhat_tile, w.qhat[0],       \
+                                      w.counters, T, s.T_max, s.n_tiles, theta, basis);          \
+  } while (0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
   } else {
@@ -147,43 +189,145 @@ cudaError_t launch_delta_construct(const Shape& s, const Workspace& w, const voi
 }
 
 // ---------------------------------------------------------------------------------------
-// K4 -- counters behind Eq. 6 for the prefill stage: multiply-adds actually needed for the
-// score matrix (d per in-window causal pair, nnz(Delta q_i) per out-of-window pair) against
-// d per causal pair of dense attention.
-__global__ void __launch_bounds__(256) prefill_stats_kernel(
-    const uint16_t* __restrict__ row_nnz, unsigned long long* __restrict__ counters, int T,
-    int T_max, int d, int W, int shape, int total_rows) {
-  unsigned long long done = 0, dense = 0;
-  for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < total_rows; r += gridDim.x * blockDim.x) {
-    const int bh = r / T, i = r - bh * T;
-    const unsigned nnz = row_nnz[(size_t)bh * T_max + i];
-    const int n_in = in_window_count(i, W, shape);
-    const int n_out = (i + 1) - n_in;
-    done += (unsigned long long)n_in * d + (unsigned long long)n_out * nnz;
-    dense += (unsigned long long)(i + 1) * d;
+// delta_finish_kernel: block roles by blockIdx.x.
+//   [0, n_idx_blocks): one warp per (batch, head, 64-row tile): row/tile counts, compacted
+//       indices, counters of Eq. 6 (d multiply-adds per in-window causal pair,
+//       nnz(Delta q_i) per out-of-window pair, against d per causal pair of dense attention).
+//   [n_idx_blocks, ...): one block per (batch, KV head, 64 keys): hand-off row
+//       R(T-1)[j] = q_hat(T-1).k_j for the heads of the group, and the channel-major fp32 key
+//       copy when kt != nullptr.
+template <typename TIn, int D>
+__global__ void __launch_bounds__(256) delta_finish_kernel(
+    const uint32_t* __restrict__ mask, uint16_t* __restrict__ row_nnz,
+    uint32_t* __restrict__ tile_nnz, uint8_t* __restrict__ idx,
+    unsigned long long* __restrict__ counters, const TIn* __restrict__ k,
+    const float* __restrict__ qhat, float* __restrict__ R, float* __restrict__ kt, int T,
+    int T_max, int n_tiles, int BH, int H, int g, int W, int shape, int n_idx_blocks, int kt_ld) {
+  constexpr int NW = D / 32;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if ((int)blockIdx.x < n_idx_blocks) {
+    const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
+    const int item = blockIdx.x * 8 + warp;          // (bh, tile)
+    if (item >= BH * tiles_used) return;
+    const int bh = item / tiles_used, tile = item - bh * tiles_used;
+    const int t0 = tile * DELTA_TILE_ROWS;
+    const int rows = min(DELTA_TILE_ROWS, T - t0);
+    // lane l holds the mask words of rows l and l + 32 of the tile
+    uint32_t mw[2][NW];
+#pragma unroll
+    for (int hlf = 0; hlf < 2; ++hlf)
+#pragma unroll
+      for (int w2 = 0; w2 < NW; ++w2) {
+        const int r = hlf * 32 + lane;
+        mw[hlf][w2] = (r < rows) ? mask[((size_t)bh * T_max + t0 + r) * NW + w2] : 0u;
+      }
+    unsigned long long done = 0, dense = 0;
+    uint32_t tile_sum = 0;
+#pragma unroll
+    for (int hlf = 0; hlf < 2; ++hlf) {
+      const int r = hlf * 32 + lane;
+      if (r < rows) {
+        int nnz = 0;
+#pragma unroll
+        for (int w2 = 0; w2 < NW; ++w2) nnz += __popc(mw[hlf][w2]);
+        row_nnz[(size_t)bh * T_max + t0 + r] = (uint16_t)nnz;
+        tile_sum += nnz;
+        const int i = t0 + r;
+        const int n_in = in_window_count(i, W, shape);
+        done += (unsigned long long)n_in * D + (unsigned long long)(i + 1 - n_in) * nnz;
+        dense += (unsigned long long)(i + 1) * D;
+      }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      tile_sum += __shfl_down_sync(0xffffffffu, tile_sum, o);
+      done += __shfl_down_sync(0xffffffffu, done, o);
+      dense += __shfl_down_sync(0xffffffffu, dense, o);
+    }
+    if (lane == 0) {
+      tile_nnz[(size_t)bh * n_tiles + tile] = tile_sum;
+      atomicAdd(&counters[CNT_PREFILL_NNZ], (unsigned long long)tile_sum);
+      atomicAdd(&counters[CNT_PREFILL_ELEMS], (unsigned long long)rows * D);
+      atomicAdd(&counters[CNT_PREFILL_MACS_DONE], done);
+      atomicAdd(&counters[CNT_PREFILL_MACS_DENSE], dense);
+    }
+    // compacted indices: the warp walks the rows, lane = channel within each mask word
+    uint8_t* idxp = idx + ((size_t)bh * T_max + t0) * D;
+    for (int r = 0; r < rows; ++r) {
+      uint32_t m[NW];
+      int nnz = 0;
+#pragma unroll
+      for (int w2 = 0; w2 < NW; ++w2) {
+        m[w2] = __shfl_sync(0xffffffffu, mw[r >> 5][w2], r & 31);
+        nnz += __popc(m[w2]);
+      }
+      int basep = 0;
+#pragma unroll
+      for (int w2 = 0; w2 < NW; ++w2) {
+        if ((m[w2] >> lane) & 1u)
+          idxp[(size_t)r * D + basep + __popc(m[w2] & ((1u << lane) - 1u))] = (uint8_t)(w2 * 32 + lane);
+        basep += __popc(m[w2]);
+      }
+#pragma unroll
+      for (int pp = lane; pp < D; pp += 32)
+        if (pp >= nnz) idxp[(size_t)r * D + pp] = 0xFF;
+    }
+    return;
   }
-  for (int o = 16; o > 0; o >>= 1) {
-    done += __shfl_down_sync(0xffffffffu, done, o);
-    dense += __shfl_down_sync(0xffffffffu, dense, o);
+
+  // ---- key pass: 64 keys of one (batch, KV head)
+  __shared__ float tile[D][65];
+  __shared__ float qh[8][D];
+  const int kblocks = (T + 63) / 64;
+  const int item = (int)blockIdx.x - n_idx_blocks;
+  const int bkv = item / kblocks, j0 = (item - bkv * kblocks) * 64;
+  const int H_kv = H / g;
+  const int b = bkv / H_kv, kvh = bkv - b * H_kv;
+  const TIn* kp = k + (size_t)bkv * T_max * D;
+  for (int e = tid; e < 64 * D; e += 256) {
+    const int j = e / D, c = e - j * D;
+    tile[c][j] = (j0 + j < T) ? to_f32(kp[(size_t)(j0 + j) * D + c]) : 0.0f;
   }
-  __shared__ unsigned long long s_done[8], s_dense[8];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (lane == 0) { s_done[warp] = done; s_dense[warp] = dense; }
+  for (int e = tid; e < g * D; e += 256) {
+    const int hh = e / D, c = e - hh * D;
+    qh[hh][c] = qhat[((size_t)b * H + kvh * g + hh) * D + c];
+  }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int w2 = 1; w2 < 8; ++w2) { done += s_done[w2]; dense += s_dense[w2]; }
-    atomicAdd(&counters[CNT_PREFILL_MACS_DONE], done);
-    atomicAdd(&counters[CNT_PREFILL_MACS_DENSE], dense);
+  if (kt != nullptr) {
+    float* op = kt + (size_t)bkv * D * kt_ld;
+    for (int e = tid; e < 64 * D; e += 256) {
+      const int c = e >> 6, j = e & 63;
+      if (j0 + j < kt_ld) op[(size_t)c * kt_ld + j0 + j] = tile[c][j];
+    }
+  }
+  {
+    const int j = tid & 63;
+    for (int hh = tid >> 6; hh < g; hh += 4) {
+      float acc = 0.0f;
+#pragma unroll 8
+      for (int c = 0; c < D; ++c) acc = fmaf(qh[hh][c], tile[c][j], acc);
+      if (j0 + j < T) R[((size_t)b * H + kvh * g + hh) * T_max + j0 + j] = acc;
+    }
   }
 }
 
-cudaError_t launch_prefill_stats(const Shape& s, const Workspace& w, int T, int window, int shape,
-                                 cudaStream_t st) {
-  const int total = s.B * s.H * T;
-  int grid = (total + 255) / 256;
-  if (grid > 296) grid = 296;
-  prefill_stats_kernel<<<grid, 256, 0, st>>>(w.row_nnz, w.counters, T, s.T_max, s.d, window, shape,
-                                             total);
+cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* k, int T,
+                                int window, int shape, int dtype, bool want_kt, cudaStream_t st) {
+  const int BH = s.B * s.H;
+  const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
+  const int n_idx_blocks = (BH * tiles_used + 7) / 8;
+  const int n_key_blocks = s.B * s.H_kv * ((T + 63) / 64);
+  const int kt_ld = (s.T_max + 3) / 4 * 4;
+  float* kt = (want_kt && w.kt) ? w.kt : nullptr;
+#define LAUNCH(TIN, DD)                                                                          \
+  delta_finish_kernel<TIN, DD><<<n_idx_blocks + n_key_blocks, 256, 0, st>>>(                     \
+      w.mask, w.row_nnz, w.tile_nnz, w.idx, w.counters, (const TIN*)k, w.qhat[0], w.R, kt, T,    \
+      s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld)
+  if (dtype == DELTA_F32) {
+    if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
+  } else {
+    if (s.d == 64) LAUNCH(__nv_bfloat16, 64); else LAUNCH(__nv_bfloat16, 128);
+  }
+#undef LAUNCH
   count_launch();
   return cudaGetLastError();
 }

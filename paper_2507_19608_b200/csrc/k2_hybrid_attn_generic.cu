@@ -287,42 +287,4 @@ cudaError_t launch_hybrid_attn_generic(const Shape& s, const Workspace& w, const
   return cudaGetLastError();
 }
 
-// ---------------------------------------------------------------------------------------
-// Hand-off to decode: the score row that strategy (1) must carry, R(T-1)[j] = sum over all
-// rows of dq . k_j, which telescopes to q_hat(T-1) . k_j.
-template <typename TIn, int D>
-__global__ void __launch_bounds__(256) handoff_kernel(const TIn* __restrict__ k,
-                                                      const float* __restrict__ qhat,
-                                                      float* __restrict__ R, int T, int T_max,
-                                                      int H, int g) {
-  __shared__ float qh[D];
-  const int bh = blockIdx.y;
-  const int b = bh / H, h = bh - b * H;
-  if (threadIdx.x < D) qh[threadIdx.x] = qhat[(size_t)bh * D + threadIdx.x];
-  __syncthreads();
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= T) return;
-  const TIn* kp = k + (((size_t)b * (H / g) + h / g) * T_max + j) * D;
-  float acc = 0.0f;
-#pragma unroll 8
-  for (int c = 0; c < D; ++c) acc = fmaf(qh[c], to_f32(kp[c]), acc);
-  R[(size_t)bh * T_max + j] = acc;
-}
-
-cudaError_t launch_handoff(const Shape& s, const Workspace& w, const void* k, int T, int dtype,
-                           int qhat_sel, cudaStream_t st) {
-  const dim3 grid((T + 255) / 256, s.B * s.H);
-#define LAUNCH(TIN, DD)                                                                       \
-  handoff_kernel<TIN, DD><<<grid, 256, 0, st>>>((const TIN*)k, w.qhat[qhat_sel], w.R, T,      \
-                                                 s.T_max, s.H, s.g())
-  if (dtype == DELTA_F32) {
-    if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
-  } else {
-    if (s.d == 64) LAUNCH(__nv_bfloat16, 64); else LAUNCH(__nv_bfloat16, 128);
-  }
-#undef LAUNCH
-  count_launch();
-  return cudaGetLastError();
-}
-
 }  // namespace delta

@@ -570,28 +570,6 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------
-// Channel-major fp32 copy of the keys, kt[b, kv head, c, j] = k[b, kv head, j, c]: the operand
-// layout of the FP32 delta update (a lane reads 4 consecutive keys of one channel).
-__global__ void __launch_bounds__(256) keys_channel_major_kernel(const __nv_bfloat16* __restrict__ k,
-                                                                 float* __restrict__ kt, int T,
-                                                                 int T_max, int ld) {
-  __shared__ float tile[TC_D][65];
-  const int bkv = blockIdx.y;
-  const int j0 = blockIdx.x * 64;
-  const __nv_bfloat16* kp = k + (size_t)bkv * T_max * TC_D;
-  for (int e = threadIdx.x; e < 64 * TC_D; e += 256) {
-    const int j = e / TC_D, c = e - j * TC_D;
-    tile[c][j] = (j0 + j < T) ? __bfloat162float(kp[(size_t)(j0 + j) * TC_D + c]) : 0.0f;
-  }
-  __syncthreads();
-  float* op = kt + (size_t)bkv * TC_D * ld;
-  for (int e = threadIdx.x; e < 64 * TC_D; e += 256) {
-    const int c = e >> 6, j = e & 63;
-    if (j0 + j < ld) op[(size_t)c * ld + j0 + j] = tile[c][j];
-  }
-}
-
-// ---------------------------------------------------------------------------------------
 namespace {
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -647,12 +625,7 @@ cudaError_t launch_hybrid_attn_tc(const Shape& s, const Workspace& w, const void
               (uint64_t)ld * TC_D * 4, 128, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
   if (!ok) return cudaErrorInvalidValue;
 
-  const dim3 gk((T + 63) / 64, (unsigned)BKV);
-  keys_channel_major_kernel<<<gk, 256, 0, st>>>((const __nv_bfloat16*)k, w.kt, T, s.T_max, ld);
-  cudaError_t err = cudaGetLastError();
-  if (err != cudaSuccess) return err;
-  count_launch();
-
+  cudaError_t err;
   err = cudaFuncSetAttribute(hybrid_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)SMEM_BYTES);
   if (err != cudaSuccess) return err;
