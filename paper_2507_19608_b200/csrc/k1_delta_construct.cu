@@ -7,8 +7,9 @@
 // (batch, head).  The chain itself is three dependent FP32 operations per token; everything
 // else is kept off it: a producer warp streams the head's query rows into a ring of
 // shared-memory stages with bulk asynchronous copies (the rows do not depend on the carried
-// state), delta values leave with one coalesced store per row, the row's mask word is a
-// single ballot parked in the lane whose index is the row number and stored once per 32 rows.
+// state), delta values leave with one coalesced store per row, every thread collects its
+// channel's fire bits of 32 rows in one register and a 32 x 32 bit transpose across the warp
+// (five shuffles) turns them into the 32 rows' mask words.
 //
 // delta_finish_kernel: everything that is parallel over rows once the mask exists -- per-row
 // and per-tile non-zero counts, the compacted channel indices, the counters behind Eq. 6 --
@@ -113,23 +114,21 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
       if (!mbar_wait(full0 + 8 * s, (i / NS) & 1)) { failed = true; break; }
       const TIn* rows = reinterpret_cast<const TIn*>(ring + (size_t)s * STAGE_BYTES) + c;
       const int nrows = min(RC, T - t0);
-      uint32_t mymask = 0;
+      // bit r of `bits`: did this thread's channel fire in row t0 + r
+      uint32_t bits = 0;
       if (nrows == RC && !(t0 == 0 && basis_exact)) {
-        // full stage, no basis row: the loads run ahead of the dependent chain
+        // full stage, no basis row: all loads first, then nothing but the dependent chain,
+        // its store and one bit per row
+        float x[RC];
 #pragma unroll
-        for (int r0 = 0; r0 < RC; r0 += 8) {
-          float x[8];
+        for (int r = 0; r < RC; ++r) x[r] = to_f32(rows[r * D]);
 #pragma unroll
-          for (int r = 0; r < 8; ++r) x[r] = to_f32(rows[(r0 + r) * D]);
-#pragma unroll
-          for (int r = 0; r < 8; ++r) {
-            const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
-            const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
-            qh = fire ? x[r] : qh;
-            dqp[(size_t)(t0 + r0 + r) * D] = fire ? diff : 0.0f;
-            const uint32_t m = __ballot_sync(0xffffffffu, fire);
-            if (lane == r0 + r) mymask = m;
-          }
+        for (int r = 0; r < RC; ++r) {
+          const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
+          const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
+          qh = fire ? x[r] : qh;
+          dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
+          bits |= fire ? (1u << r) : 0u;
         }
       } else {
         for (int r = 0; r < nrows; ++r) {
@@ -146,9 +145,18 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
           }
           qh = fire ? x : qh;
           dqp[(size_t)(t0 + r) * D] = delta;
-          const uint32_t m = __ballot_sync(0xffffffffu, fire);
-          if (lane == r) mymask = m;
+          bits |= fire ? (1u << r) : 0u;
         }
+      }
+      // 32 x 32 bit transpose across the warp: lane r ends up with the mask word of row t0 + r
+      uint32_t mymask = bits;
+#pragma unroll
+      for (int j = 16; j > 0; j >>= 1) {
+        const uint32_t km = (j == 16) ? 0x0000FFFFu : (j == 8) ? 0x00FF00FFu : (j == 4) ? 0x0F0F0F0Fu
+                          : (j == 2) ? 0x33333333u : 0x55555555u;
+        const uint32_t other = __shfl_xor_sync(0xffffffffu, mymask, j);
+        mymask = (lane & j) ? (((other >> j) & km) | (mymask & ~km))
+                            : ((mymask & km) | ((other & km) << j));
       }
       if (lane < nrows) maskp[(size_t)(t0 + lane) * NW] = mymask;
       __syncwarp();
@@ -190,7 +198,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 
 // ---------------------------------------------------------------------------------------
 // delta_finish_kernel: block roles by blockIdx.x.
-//   [0, n_idx_blocks): one warp per (batch, head, 64-row tile): row/tile counts, compacted
+//   [0, n_idx_blocks): one block per (batch, head, 64-row tile): row/tile counts, compacted
 //       indices, counters of Eq. 6 (d multiply-adds per in-window causal pair,
 //       nnz(Delta q_i) per out-of-window pair, against d per causal pair of dense attention).
 //   [n_idx_blocks, ...): one block per (batch, KV head, 64 keys): hand-off row
@@ -206,70 +214,66 @@ __global__ void __launch_bounds__(256) delta_finish_kernel(
   constexpr int NW = D / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if ((int)blockIdx.x < n_idx_blocks) {
+    // ---- one block per (batch, head, 64-row tile); warp w serves rows 8w .. 8w+7
+    __shared__ unsigned long long s_red[3][8];
     const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
-    const int item = blockIdx.x * 8 + warp;          // (bh, tile)
-    if (item >= BH * tiles_used) return;
-    const int bh = item / tiles_used, tile = item - bh * tiles_used;
+    const int bh = blockIdx.x / tiles_used, tile = blockIdx.x - bh * tiles_used;
     const int t0 = tile * DELTA_TILE_ROWS;
     const int rows = min(DELTA_TILE_ROWS, T - t0);
-    // lane l holds the mask words of rows l and l + 32 of the tile
-    uint32_t mw[2][NW];
+    const int r_mine = warp * 8 + (lane & 7);        // lanes 0..7 hold one row each
+    uint32_t mw[NW];
 #pragma unroll
-    for (int hlf = 0; hlf < 2; ++hlf)
+    for (int w2 = 0; w2 < NW; ++w2)
+      mw[w2] = (r_mine < rows) ? mask[((size_t)bh * T_max + t0 + r_mine) * NW + w2] : 0u;
+    unsigned long long done = 0, dense = 0, tsum = 0;
+    if (lane < 8 && r_mine < rows) {
+      int nnz = 0;
 #pragma unroll
-      for (int w2 = 0; w2 < NW; ++w2) {
-        const int r = hlf * 32 + lane;
-        mw[hlf][w2] = (r < rows) ? mask[((size_t)bh * T_max + t0 + r) * NW + w2] : 0u;
-      }
-    unsigned long long done = 0, dense = 0;
-    uint32_t tile_sum = 0;
-#pragma unroll
-    for (int hlf = 0; hlf < 2; ++hlf) {
-      const int r = hlf * 32 + lane;
-      if (r < rows) {
-        int nnz = 0;
-#pragma unroll
-        for (int w2 = 0; w2 < NW; ++w2) nnz += __popc(mw[hlf][w2]);
-        row_nnz[(size_t)bh * T_max + t0 + r] = (uint16_t)nnz;
-        tile_sum += nnz;
-        const int i = t0 + r;
-        const int n_in = in_window_count(i, W, shape);
-        done += (unsigned long long)n_in * D + (unsigned long long)(i + 1 - n_in) * nnz;
-        dense += (unsigned long long)(i + 1) * D;
-      }
+      for (int w2 = 0; w2 < NW; ++w2) nnz += __popc(mw[w2]);
+      row_nnz[(size_t)bh * T_max + t0 + r_mine] = (uint16_t)nnz;
+      tsum = (unsigned long long)nnz;
+      const int i = t0 + r_mine;
+      const int n_in = in_window_count(i, W, shape);
+      done = (unsigned long long)n_in * D + (unsigned long long)(i + 1 - n_in) * nnz;
+      dense = (unsigned long long)(i + 1) * D;
     }
-    for (int o = 16; o > 0; o >>= 1) {
-      tile_sum += __shfl_down_sync(0xffffffffu, tile_sum, o);
+    for (int o = 4; o > 0; o >>= 1) {
+      tsum += __shfl_down_sync(0xffffffffu, tsum, o);
       done += __shfl_down_sync(0xffffffffu, done, o);
       dense += __shfl_down_sync(0xffffffffu, dense, o);
     }
-    if (lane == 0) {
-      tile_nnz[(size_t)bh * n_tiles + tile] = tile_sum;
-      atomicAdd(&counters[CNT_PREFILL_NNZ], (unsigned long long)tile_sum);
-      atomicAdd(&counters[CNT_PREFILL_ELEMS], (unsigned long long)rows * D);
-      atomicAdd(&counters[CNT_PREFILL_MACS_DONE], done);
-      atomicAdd(&counters[CNT_PREFILL_MACS_DENSE], dense);
-    }
-    // compacted indices: the warp walks the rows, lane = channel within each mask word
-    uint8_t* idxp = idx + ((size_t)bh * T_max + t0) * D;
-    for (int r = 0; r < rows; ++r) {
+    if (lane == 0) { s_red[0][warp] = tsum; s_red[1][warp] = done; s_red[2][warp] = dense; }
+    // compacted indices: lane = channel within each mask word
+    uint8_t* idxp = idx + ((size_t)bh * T_max + t0 + warp * 8) * D;
+    const int my_rows = min(8, rows - warp * 8);
+    for (int r = 0; r < my_rows; ++r) {
       uint32_t m[NW];
       int nnz = 0;
 #pragma unroll
       for (int w2 = 0; w2 < NW; ++w2) {
-        m[w2] = __shfl_sync(0xffffffffu, mw[r >> 5][w2], r & 31);
+        m[w2] = __shfl_sync(0xffffffffu, mw[w2], r);
         nnz += __popc(m[w2]);
       }
       int basep = 0;
 #pragma unroll
       for (int w2 = 0; w2 < NW; ++w2) {
         if ((m[w2] >> lane) & 1u)
-          idxp[(size_t)r * D + basep + __popc(m[w2] & ((1u << lane) - 1u))] = (uint8_t)(w2 * 32 + lane);
+          idxp[r * D + basep + __popc(m[w2] & ((1u << lane) - 1u))] = (uint8_t)(w2 * 32 + lane);
         basep += __popc(m[w2]);
       }
 #pragma unroll
       for (int pp = lane; pp < D; pp += 32)
-        if (pp >= nnz) idxp[(size_t)r * D + pp] = 0xFF;
+        if (pp >= nnz) idxp[r * D + pp] = 0xFF;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long a = 0, b2 = 0, c2 = 0;
+      for (int w2 = 0; w2 < 8; ++w2) { a += s_red[0][w2]; b2 += s_red[1][w2]; c2 += s_red[2][w2]; }
+      tile_nnz[(size_t)bh * n_tiles + tile] = (uint32_t)a;
+      atomicAdd(&counters[CNT_PREFILL_NNZ], a);
+      atomicAdd(&counters[CNT_PREFILL_ELEMS], (unsigned long long)rows * D);
+      atomicAdd(&counters[CNT_PREFILL_MACS_DONE], b2);
+      atomicAdd(&counters[CNT_PREFILL_MACS_DENSE], c2);
     }
     return;
   }
@@ -283,9 +287,21 @@ __global__ void __launch_bounds__(256) delta_finish_kernel(
   const int H_kv = H / g;
   const int b = bkv / H_kv, kvh = bkv - b * H_kv;
   const TIn* kp = k + (size_t)bkv * T_max * D;
-  for (int e = tid; e < 64 * D; e += 256) {
-    const int j = e / D, c = e - j * D;
-    tile[c][j] = (j0 + j < T) ? to_f32(kp[(size_t)(j0 + j) * D + c]) : 0.0f;
+  {
+    constexpr int VEC = 16 / sizeof(TIn);            // elements per 16-byte load
+    constexpr int CPR = D / VEC;                     // 16-byte chunks per key row
+    for (int e = tid; e < 64 * CPR; e += 256) {
+      const int j = e / CPR, c = (e - j * CPR) * VEC;
+      TIn vals[VEC];
+      if (j0 + j < T) {
+        *reinterpret_cast<uint4*>(vals) = *reinterpret_cast<const uint4*>(kp + (size_t)(j0 + j) * D + c);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) tile[c + i][j] = to_f32(vals[i]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) tile[c + i][j] = 0.0f;
+      }
+    }
   }
   for (int e = tid; e < g * D; e += 256) {
     const int hh = e / D, c = e - hh * D;
@@ -314,7 +330,7 @@ cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* 
                                 int window, int shape, int dtype, bool want_kt, cudaStream_t st) {
   const int BH = s.B * s.H;
   const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
-  const int n_idx_blocks = (BH * tiles_used + 7) / 8;
+  const int n_idx_blocks = BH * tiles_used;
   const int n_key_blocks = s.B * s.H_kv * ((T + 63) / 64);
   const int kt_ld = (s.T_max + 3) / 4 * 4;
   float* kt = (want_kt && w.kt) ? w.kt : nullptr;
