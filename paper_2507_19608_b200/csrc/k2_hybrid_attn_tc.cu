@@ -1,29 +1,34 @@
 // K2 (tensor-core) -- fused hybrid delta attention for bf16 inputs on sm_100a
 // (Section III-B; Eq. 1, Eq. 4; construction strategy (1) of Section III-A).
 //
-// One CTA of 16 warps owns 128 query rows of one head and walks the 128-key tiles up to the
-// diagonal.  The work is split by what it is:
-//   * dense contractions run on the 5th-generation tensor cores (tcgen05.mma, operands staged
-//     in shared memory by TMA, accumulators in tensor memory): the exact Q.K^T of tiles that
-//     touch the window, and P.V of every tile;
+// One CTA owns 128 query rows of one head and walks the 128-key tiles up to the diagonal.
+// 16 compute warps and one control warp; the work is split by what it is:
+//   * dense contractions run on the 5th-generation tensor cores (tcgen05.mma issued by the
+//     control thread, operands staged in shared memory by TMA, accumulators in tensor memory):
+//     the exact Q.K^T of tiles that touch the window, and P.V of every tile;
 //   * the out-of-window scores are Eq. 4's running sum of sparse delta products and stay on the
-//     FP32 pipes, because the zeros of a thresholded delta matrix are unstructured.  A warp owns
-//     8 consecutive rows and all 128 keys of the tile (4 keys per lane).  Rows are taken in
-//     blocks of 4: the OR of the 4 rows' mask words says which channels fired anywhere in the
-//     block; channels whose 4x1 delta block is all zero are skipped (find-first-set over the
-//     block mask), every other channel costs one 16-byte key load (channel-major fp32 key tile)
-//     and one 16-byte delta load for a 4x4 register tile of multiply-adds.  Prefix sums over
-//     the rows turn the per-row products into R(i)[j]; the part of the recursion that lies in
-//     front of the warp's rows comes from the other warps' block totals and from the seed
-//     q_hat(i0-1).k_j (the reference in front of the tile telescopes all earlier rows);
+//     FP32 pipes, because the zeros of a thresholded delta matrix are unstructured.  A compute
+//     warp owns 8 consecutive rows and all 128 keys of the tile (4 keys per lane).  Rows are
+//     taken in blocks of 4: the OR of the 4 rows' mask words says which channels fired anywhere
+//     in the block (ballot-style mask words, popc for list positions); channels whose 4x1 delta
+//     block is all zero are never touched, every other channel costs one 16-byte key load
+//     (channel-major fp32 key tile) and one 16-byte delta load for a 4x4 register tile of
+//     multiply-adds.  Prefix sums over the rows turn the per-row products into R(i)[j]; the part
+//     of the recursion in front of the warp's rows comes from the other warps' totals and from
+//     the seed q_hat(i0-1).k_j (the reference in front of the tile telescopes all earlier rows);
 //   * scale, causal mask, hybrid select and the online softmax run in the same key-per-lane
-//     layout; exact scores come out of tensor memory row-per-thread and are transposed through
-//     shared memory; P goes to shared memory as bf16 in the tensor-core operand layout; the
-//     P.V tile product is read back from tensor memory row-per-thread and accumulated in
-//     registers with the softmax rescale.
+//     layout (row reductions as an 8-row butterfly); exact scores come out of tensor memory
+//     row-per-thread and are transposed through shared memory; P goes to shared memory as bf16
+//     in the tensor-core operand layout; the P.V tile product is read back from tensor memory
+//     row-per-thread and accumulated in registers with the softmax rescale.
+// Warps are decoupled: the channel-major key tile is double buffered and every hand-over
+// (tile loaded / tile consumed / block totals ready / P ready / P.V done) is an mbarrier, so a
+// warp that has finished its delta update moves on to its softmax while others still
+// multiply.  Only tiles that touch the window synchronise the compute warps with a barrier.
 //
 // Every wait on an mbarrier is bounded; a wait that runs out records DELTA_ERR_TIMEOUT in the
-// device status word and the CTA leaves through the common exit (which frees its tensor memory).
+// device status word, every later wait returns at once, the protocol still runs to its end (so
+// no barrier is left short of arrivals) and the CTA frees its tensor memory and stores nothing.
 #include <cuda.h>
 
 #include "k2_tc.cuh"
@@ -32,7 +37,7 @@ namespace delta {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, NTHR = 512, NWARP = 16;
+constexpr int BM = 128, BN = 128, NCWARP = 16, NCTHR = NCWARP * 32, NTHR = NCTHR + 32;
 constexpr int TC_D = 64;                 // head dimension served by this kernel
 constexpr uint32_t TMEM_COLS = 256;      // S: columns 0..127, O: columns 128..191
 constexpr uint32_t TMEM_S = 0, TMEM_O = 128;
@@ -41,30 +46,39 @@ constexpr uint32_t TMEM_S = 0, TMEM_O = 128;
 constexpr uint32_t SZ_TILE = 128 * 64 * 2;               // one bf16 operand tile, 16 KiB
 constexpr uint32_t ROW_B = 128 * 4;                      // one channel row of the fp32 tiles
 constexpr uint32_t PAD_OFF = 64 * ROW_B;                 // row 64 of both fp32 tiles: padding target
+constexpr uint32_t SZ_KT = 65 * ROW_B + 512;             // one channel-major key buffer (33792)
 constexpr uint32_t OFF_Q = 0;
 constexpr uint32_t OFF_K = OFF_Q + SZ_TILE;
 constexpr uint32_t OFF_V = OFF_K + SZ_TILE;              // two buffers
-constexpr uint32_t OFF_KT = OFF_V + 2 * SZ_TILE;         // fp32 [64 channels + 1][128 keys]
-constexpr uint32_t OFF_P = OFF_KT + 65 * ROW_B + 512;    // bf16 [2][128 rows][64 keys]
-constexpr uint32_t OFF_SX = OFF_KT;                      // fp32 [128][128] exact scores (over KT, P)
-constexpr uint32_t OFF_DQT = OFF_P + 2 * SZ_TILE;        // fp32 [64 channels + 1][128 rows]
+constexpr uint32_t OFF_P = OFF_V + 2 * SZ_TILE;          // bf16 [2][128 rows][64 keys]
+constexpr uint32_t OFF_KT = OFF_P + 2 * SZ_TILE;         // two buffers fp32 [64 channels + 1][128 keys]
+constexpr uint32_t OFF_SX = OFF_KT;                      // fp32 [128][128] exact scores (over both)
+constexpr uint32_t OFF_DQT = OFF_KT + 2 * SZ_KT;         // fp32 [64 channels + 1][128 rows]
 constexpr uint32_t OFF_LIST = OFF_DQT + 65 * ROW_B;      // u32 [32 blocks][64]: fired channel * ROW_B
 constexpr uint32_t OFF_CNT = OFF_LIST + 32 * 64 * 4;     // u32 [32]: list length / 4
-constexpr uint32_t OFF_TOT = OFF_CNT + 32 * 4;           // fp32 [16][128]
-constexpr uint32_t OFF_SEED = OFF_TOT + 16 * 128 * 4;    // fp32 [128]
-constexpr uint32_t OFF_ALPHA = OFF_SEED + 128 * 4;       // fp32 [2][128]
-constexpr uint32_t OFF_M = OFF_ALPHA + 2 * 128 * 4;      // fp32 [128] running max
+constexpr uint32_t OFF_TOT = OFF_CNT + 32 * 4;           // fp32 [2][16][128]
+constexpr uint32_t OFF_SEED = OFF_TOT + 2 * 16 * 128 * 4;  // fp32 [2][128]
+constexpr uint32_t OFF_ALPHA = OFF_SEED + 2 * 128 * 4;   // fp32 [2][128]
+constexpr uint32_t OFF_M = OFF_ALPHA + 2 * 128 * 4;      // fp32 [128] running max (scaled, log2 domain)
 constexpr uint32_t OFF_L = OFF_M + 128 * 4;              // fp32 [128] running sum
 constexpr uint32_t OFF_QHAT = OFF_L + 128 * 4;           // fp32 [64]
-constexpr uint32_t OFF_BAR = OFF_QHAT + 64 * 4;          // 8 mbarriers
-constexpr uint32_t OFF_MISC = OFF_BAR + 8 * 8;           // tmem slot, abort flag
+constexpr uint32_t OFF_BAR = OFF_QHAT + 64 * 4;          // mbarriers
+constexpr uint32_t OFF_MISC = OFF_BAR + 16 * 8;          // tmem slot, abort flag
 constexpr uint32_t SMEM_USED = OFF_MISC + 16;
 constexpr uint32_t SMEM_BYTES = SMEM_USED + 1024;        // slack for the alignment of the base
-static_assert(OFF_P % 1024 == 0 && OFF_KT % 1024 == 0, "operand tiles need 1024-byte alignment");
-static_assert(OFF_P + 2 * SZ_TILE - OFF_SX >= 128 * 128 * 4, "exact-score buffer must fit");
+static_assert(OFF_P % 1024 == 0 && OFF_KT % 1024 == 0 && SZ_KT % 1024 == 0, "1024-byte alignment");
+static_assert(2 * SZ_KT >= 128 * 128 * 4, "exact-score buffer must fit in the two key buffers");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
-enum Bar { BAR_Q = 0, BAR_K, BAR_KT, BAR_V0, BAR_V1, BAR_S, BAR_O };
+enum Bar {
+  BAR_Q = 0, BAR_K, BAR_V0, BAR_V1, BAR_S, BAR_O,     // one arrival (+ bytes) per phase
+  BAR_KT_FULL0, BAR_KT_FULL1,                         // one arrival + bytes
+  BAR_KT_EMPTY0, BAR_KT_EMPTY1,                       // 16 arrivals: every compute warp is done with it
+  BAR_DELTA0, BAR_DELTA1,                             // 16 arrivals: block totals and seed written
+  BAR_P,                                              // 16 arrivals: P tile written
+  BAR_SX,                                             // 16 arrivals: exact scores consumed
+  NUM_BARS
+};
 
 // ---- PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -77,6 +91,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -88,14 +105,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after about a second of SM clock.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: gives up after about a second of SM clock and raises the CTA's abort flag;
+// once the flag is up every wait returns at once.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > 2000000000ll) return false;
+    if (*abort_flag) return;
+    if (clock64() - t0 > 2000000000ll) { *abort_flag = 1; return; }
   }
-  return true;
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
                                             int c0, int c1, int c2) {
@@ -142,6 +160,29 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 16-byte shared-memory accesses by 32-bit shared address
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint4 lds128u(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void compute_barrier() {   // the 16 compute warps only
+  asm volatile("bar.sync 1, %0;" ::"n"(NCTHR) : "memory");
+}
 
 // Shared-memory matrix descriptor of the tensor cores: 128-byte swizzle, 16-byte units.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -152,6 +193,31 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 __host__ __device__ constexpr uint32_t make_idesc(int n, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(128 >> 4) << 24);
+}
+
+// Reduction of 8 per-lane values (one per row of the warp's row group) over the 32 lanes in
+// 9 shuffles: the halves of the value set are exchanged while the lane distance halves.  On
+// return every lane holds the warp-wide result of row (lane >> 2) & 7.
+template <bool IS_MAX>
+__device__ __forceinline__ float reduce8(const float (&v)[8], int lane) {
+  auto op = [](float a, float b) { return IS_MAX ? fmaxf(a, b) : a + b; };
+  float w[4], u[2];
+  const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float send = h16 ? v[i] : v[i + 4], keep = h16 ? v[i + 4] : v[i];
+    w[i] = op(keep, __shfl_xor_sync(0xffffffffu, send, 16));
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const float send = h8 ? w[i] : w[i + 2], keep = h8 ? w[i + 2] : w[i];
+    u[i] = op(keep, __shfl_xor_sync(0xffffffffu, send, 8));
+  }
+  const float send = h4 ? u[0] : u[1], keep = h4 ? u[1] : u[0];
+  float z = op(keep, __shfl_xor_sync(0xffffffffu, send, 4));
+  z = op(z, __shfl_xor_sync(0xffffffffu, z, 2));
+  z = op(z, __shfl_xor_sync(0xffffffffu, z, 1));
+  return z;
 }
 
 struct TcParams {
@@ -175,7 +241,6 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* sm = smem_raw + (base - raw);
 
-  float* sKt = reinterpret_cast<float*>(sm + OFF_KT);
   float* sdQt = reinterpret_cast<float*>(sm + OFF_DQT);
   uint32_t* sList = reinterpret_cast<uint32_t*>(sm + OFF_LIST);
   uint32_t* sCnt = reinterpret_cast<uint32_t*>(sm + OFF_CNT);
@@ -186,13 +251,11 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   float* sL = reinterpret_cast<float*>(sm + OFF_L);
   float* sQhat = reinterpret_cast<float*>(sm + OFF_QHAT);
   volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
+  volatile uint32_t* abort_flag = sMisc + 1;
   const uint32_t bar0 = base + OFF_BAR;
 #define BAR(i) (bar0 + 8u * (uint32_t)(i))
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int qd = warp & 3, sub = warp >> 2;     // tensor-memory lane quadrant / slot in it
-  const int rg = qd * 4 + sub;                  // row group: rows 8*rg .. 8*rg+7
-  const int my_row = 32 * qd + lane;            // row this thread owns in row-per-thread phases
   const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;  // heaviest query tiles of every head first
   const int bh = blockIdx.x;
   const int b = bh / p.H, h = bh - b * p.H;
@@ -201,7 +264,7 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const int T = p.T, W = p.W, shape = p.shape;
   const int i1 = min(i0 + BM, T) - 1;           // last valid row of the tile
 
-  // ---- set-up: tensor memory, barriers, first loads ---------------------------------------
+  // ---- set-up: tensor memory, barriers ----------------------------------------------------
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      base + OFF_MISC),
@@ -210,7 +273,8 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if (tid == 0) {
-    for (int i = 0; i < 8; ++i) mbar_init(BAR(i), 1);
+    for (int i = 0; i < NUM_BARS; ++i)
+      mbar_init(BAR(i), (i >= BAR_KT_EMPTY0) ? (uint32_t)NCWARP : 1u);
     sMisc[1] = 0;  // abort flag
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
@@ -233,316 +297,339 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     return (i1 - j0) < W;
   };
 
-  if (tid == 0) {
-    if (W > 0) {
-      mbar_expect_tx(BAR(BAR_Q), SZ_TILE);
-      tma_load_3d(base + OFF_Q, &tm_q, BAR(BAR_Q), 0, i0, bh);
-    }
-    mbar_expect_tx(BAR(BAR_KT), 64 * 128 * 4);
-    tma_load_3d(base + OFF_KT, &tm_kt, BAR(BAR_KT), 0, 0, bkv);
-    mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
-    tma_load_3d(base + OFF_V, &tm_v, BAR(BAR_V0), 0, 0, bkv);
-    if (tile_needs_exact(0)) {
-      mbar_expect_tx(BAR(BAR_K), SZ_TILE);
-      tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K), 0, 0, bkv);
-    }
-  }
-
-  // ---- stage the query tile: deltas channel-major, per 4-row block the list of channels that
-  // fired anywhere in the block (ballot of the mask words, popc for the position), the seed
-  // reference, the softmax state
-  {
-    const float* dqp = p.dq + ((size_t)bh * p.T_max + i0) * TC_D;
-    const int r_sub = lane >> 3, c_sub = lane & 7;
-    for (int it = warp; it < 32 * 8; it += NWARP) {
-      const int rb = it >> 3, cb = it & 7;
-      const int r = rb * 4 + r_sub, c = cb * 8 + c_sub;
-      const float x = (i0 + r < T) ? dqp[(size_t)r * TC_D + c] : 0.0f;
-      sdQt[c * BM + r] = x;
-    }
-    if (tid < 128) {                 // row 64 of both fp32 tiles: where list padding points
-      sdQt[64 * BM + tid] = 0.0f;
-      sKt[64 * BN + tid] = 0.0f;
-    }
-    {
-      const int blk = tid >> 4, sl = tid & 15;       // 16 threads per block of 4 rows
-      unsigned long long u = 0;
-      const uint32_t* mp = p.mask + ((size_t)bh * p.T_max + i0 + blk * 4) * 2;
-#pragma unroll
-      for (int r = 0; r < 4; ++r)
-        if (i0 + blk * 4 + r < T)
-          u |= (unsigned long long)mp[r * 2] | ((unsigned long long)mp[r * 2 + 1] << 32);
-      const int n = __popcll(u);
-      uint32_t* lp = sList + blk * 64;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int c = sl * 4 + k;
-        if ((u >> c) & 1ull) lp[__popcll(u & ((1ull << c) - 1ull))] = (uint32_t)c * ROW_B;
+  if (warp == NCWARP) {
+    // =========================== control warp: TMA and tensor-core issue =====================
+    if (lane == 0) {
+      const uint32_t IDESC_QK = make_idesc(BN, 0);
+      const uint32_t IDESC_PV = make_idesc(TC_D, 1);
+      if (W > 0) {
+        mbar_expect_tx(BAR(BAR_Q), SZ_TILE);
+        tma_load_3d(base + OFF_Q, &tm_q, BAR(BAR_Q), 0, i0, bh);
       }
-      const int n4 = (n + 3) >> 2;
-      if (sl < 3 && n + sl < n4 * 4) lp[n + sl] = PAD_OFF;
-      if (sl == 0) sCnt[blk] = (uint32_t)n4;
-    }
-    if (tid < TC_D) sQhat[tid] = p.qhat_tile[((size_t)bh * p.n_tiles64 + 2 * qt) * TC_D + tid];
-    if (tid < BM) { sM[tid] = -INFINITY; sL[tid] = 0.0f; }
-  }
-  float O[16];
-#pragma unroll
-  for (int i = 0; i < 16; ++i) O[i] = 0.0f;
-  __syncthreads();
-
-  const uint32_t IDESC_QK = make_idesc(BN, 0);
-  const uint32_t IDESC_PV = make_idesc(TC_D, 1);
-  int n_exact = 0;          // exact tiles seen so far (parity of BAR_K / BAR_S)
-  bool aborted = false;
-
-  for (int jt = 0; jt <= qt; ++jt) {
-    const int j0 = jt * BN;
-    const bool need_exact = tile_needs_exact(jt);
-    const bool need_delta = !tile_all_in(jt);
-    const bool diag = (jt == qt);
-
-    // ---- exact Q.K^T of a tile that touches the window: issued first, consumed after the deltas
-    if (need_exact && tid == 0) {
-      bool ok = mbar_wait(BAR(BAR_K), n_exact & 1);
-      if (n_exact == 0) ok = mbar_wait(BAR(BAR_Q), 0) && ok;
-      if (!ok) sMisc[1] = 1;
-      tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < TC_D / 16; ++ks) {
-        const uint64_t da = make_desc(base + OFF_Q + ks * 32, 16, 1024);
-        const uint64_t db = make_desc(base + OFF_K + ks * 32, 16, 1024);
-        tc_mma(tmem + TMEM_S, da, db, IDESC_QK, ks > 0 ? 1u : 0u);
-      }
-      tc_commit(BAR(BAR_S));
-    }
-
-    // ---- Eq. 4 on the FP32 pipes: block-sparse 4x4 register tiles over fired channels
-    float Sl[8][4];
-#pragma unroll
-    for (int r = 0; r < 8; ++r)
-#pragma unroll
-      for (int k = 0; k < 4; ++k) Sl[r][k] = 0.0f;
-    if (!mbar_wait(BAR(BAR_KT), jt & 1)) sMisc[1] = 1;
-    if (need_delta) {
-      float run[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      const unsigned char* ktb = reinterpret_cast<const unsigned char*>(sKt) + 16 * lane;
-#pragma unroll
-      for (int g4 = 0; g4 < 2; ++g4) {
-        float a[4][4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-#pragma unroll
-          for (int k = 0; k < 4; ++k) a[r][k] = 0.0f;
-        const int blk = rg * 2 + g4;
-        const unsigned char* dqb = reinterpret_cast<const unsigned char*>(sdQt) + 16 * blk;
-        const uint4* lp = reinterpret_cast<const uint4*>(sList + blk * 64);
-        const int n4 = (int)sCnt[blk];
-        for (int q4 = 0; q4 < n4; ++q4) {
-          const uint4 e = lp[q4];
-          const uint32_t off[4] = {e.x, e.y, e.z, e.w};
-          float4 kv[4], dv[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            kv[u] = *reinterpret_cast<const float4*>(ktb + off[u]);
-            dv[u] = *reinterpret_cast<const float4*>(dqb + off[u]);
-          }
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const float kk[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
-            const float dd[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
-#pragma unroll
-            for (int r = 0; r < 4; ++r)
-#pragma unroll
-              for (int k = 0; k < 4; ++k) a[r][k] = fmaf(dd[r], kk[k], a[r][k]);
-          }
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            run[k] += a[r][k];
-            Sl[g4 * 4 + r][k] = run[k];
-          }
-      }
-      *reinterpret_cast<float4*>(sTot + rg * BN + 4 * lane) = make_float4(run[0], run[1], run[2], run[3]);
-      // seed q_hat(i0-1).k_j: this warp serves keys 8*warp .. 8*warp+7, 16 channels per lane
-      if (qt > 0) {
-        const int kq = lane & 7, cq = lane >> 3;
-        const float* kp = sKt + cq * 16 * BN + 8 * warp + kq;
-        float sd = 0.0f;
-#pragma unroll
-        for (int cc = 0; cc < 16; ++cc) sd = fmaf(sQhat[cq * 16 + cc], kp[cc * BN], sd);
-        sd += __shfl_xor_sync(0xffffffffu, sd, 8);
-        sd += __shfl_xor_sync(0xffffffffu, sd, 16);
-        if (lane < 8) sSeed[8 * warp + lane] = sd;
-      } else if (lane < 8) {
-        sSeed[8 * warp + lane] = 0.0f;
-      }
-    }
-    fence_proxy_async();   // generic reads of the key tile are ordered before its next bulk write
-    __syncthreads();       // (A) totals and seed slices visible; channel-major key tile free
-    if (sMisc[1]) { aborted = true; break; }
-
-    const bool more = (jt < qt);
-    if (tid == 0 && more && !need_exact) {
-      mbar_expect_tx(BAR(BAR_KT), 64 * 128 * 4);
-      tma_load_3d(base + OFF_KT, &tm_kt, BAR(BAR_KT), j0 + BN, 0, bkv);
-      if (tile_needs_exact(jt + 1)) {
+      mbar_expect_tx(BAR(BAR_KT_FULL0), 64 * ROW_B);
+      tma_load_3d(base + OFF_KT, &tm_kt, BAR(BAR_KT_FULL0), 0, 0, bkv);
+      mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
+      tma_load_3d(base + OFF_V, &tm_v, BAR(BAR_V0), 0, 0, bkv);
+      if (tile_needs_exact(0)) {
         mbar_expect_tx(BAR(BAR_K), SZ_TILE);
-        tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K), 0, j0 + BN, bkv);
+        tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K), 0, 0, bkv);
       }
-    }
-
-    // ---- previous tile's P.V: rescale and accumulate (row-per-thread)
-    if (jt > 0) {
-      if (!mbar_wait(BAR(BAR_O), (jt - 1) & 1)) sMisc[1] = 1;
-      tc_fence_after();
-      float v[16];
-      tc_ld16(tmem + TMEM_O + 16 * sub + ((uint32_t)(32 * qd) << 16), v);
-      const float al = sAlpha[((jt - 1) & 1) * BM + my_row];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) O[i] = fmaf(O[i], al, v[i]);
-      tc_fence_before();
-    }
-
-    // ---- exact scores: tensor memory (row per thread) -> shared memory, 16-byte XOR swizzle
-    if (need_exact) {
-      if (!mbar_wait(BAR(BAR_S), n_exact & 1)) sMisc[1] = 1;
-      tc_fence_after();
-      unsigned char* sx_row = sm + OFF_SX + (size_t)my_row * 512;
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float v[16];
-        tc_ld16(tmem + TMEM_S + 32 * sub + 16 * half + ((uint32_t)(32 * qd) << 16), v);
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const int chunk = 8 * sub + 4 * half + q4;
-          *reinterpret_cast<float4*>(sx_row + ((chunk ^ lane) << 4)) =
-              make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
-        }
-      }
-      tc_fence_before();
-      __syncthreads();     // (B) exact scores visible
-      if (sMisc[1]) { aborted = true; break; }
-    }
-
-    // ---- pass 1: hybrid select (Section III-B): exact inside the window, running sum outside
-    {
-      float bs[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      if (need_delta) {
-        const float4 s4 = *reinterpret_cast<const float4*>(sSeed + 4 * lane);
-        bs[0] = s4.x; bs[1] = s4.y; bs[2] = s4.z; bs[3] = s4.w;
-        for (int r2 = 0; r2 < rg; ++r2) {
-          const float4 t4 = *reinterpret_cast<const float4*>(sTot + r2 * BN + 4 * lane);
-          bs[0] += t4.x; bs[1] += t4.y; bs[2] += t4.z; bs[3] += t4.w;
-        }
-      }
-#pragma unroll
-      for (int r = 0; r < 8; ++r) {
-        const int row = rg * 8 + r;
-        const int i = i0 + row;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) Sl[r][k] += bs[k];
-        if (need_exact) {
-          int wlo, whi;   // exact keys of row i: wlo <= j < whi
-          if (shape == 0) { wlo = (i / W) * W; whi = wlo + W; }
-          else { wlo = i - W + 1; whi = i + 1; }
-          const float4 e4 = *reinterpret_cast<const float4*>(sm + OFF_SX + (size_t)row * 512 +
-                                                             ((lane ^ (row & 31)) << 4));
-          const float ex[4] = {e4.x, e4.y, e4.z, e4.w};
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const int j = j0 + 4 * lane + k;
-            if (j >= wlo && j < whi) Sl[r][k] = ex[k];
+      int nk = 0;   // exact tiles so far: parity of BAR_K, BAR_S, BAR_SX
+      for (int t = 0; t <= qt; ++t) {
+        const bool exact = tile_needs_exact(t);
+        const bool more = t < qt;
+        const int nb = (t + 1) & 1;
+        auto load_next_keys = [&]() {
+          mbar_expect_tx(BAR(BAR_KT_FULL0 + nb), 64 * ROW_B);
+          tma_load_3d(base + OFF_KT + nb * SZ_KT, &tm_kt, BAR(BAR_KT_FULL0 + nb), (t + 1) * BN, 0, bkv);
+          if (tile_needs_exact(t + 1)) {
+            mbar_expect_tx(BAR(BAR_K), SZ_TILE);
+            tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K), 0, (t + 1) * BN, bkv);
           }
+        };
+        if (exact) {   // exact Q.K^T of a tile that touches the window
+          mbar_wait(BAR(BAR_K), nk & 1, abort_flag);
+          if (nk == 0) mbar_wait(BAR(BAR_Q), 0, abort_flag);
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < TC_D / 16; ++ks) {
+            const uint64_t da = make_desc(base + OFF_Q + ks * 32, 16, 1024);
+            const uint64_t db = make_desc(base + OFF_K + ks * 32, 16, 1024);
+            tc_mma(tmem + TMEM_S, da, db, IDESC_QK, ks > 0 ? 1u : 0u);
+          }
+          tc_commit(BAR(BAR_S));
         }
+        if (t >= 1) mbar_wait(BAR(BAR_O), (t - 1) & 1, abort_flag);   // P.V(t-1) done: its V buffer is free
+        if (more) {
+          mbar_expect_tx(BAR(BAR_V0 + nb), SZ_TILE);
+          tma_load_3d(base + OFF_V + nb * SZ_TILE, &tm_v, BAR(BAR_V0 + nb), 0, (t + 1) * BN, bkv);
+        }
+        if (!exact) {
+          if (more) {
+            if (t >= 1) mbar_wait(BAR(BAR_KT_EMPTY0 + nb), ((t - 1) >> 1) & 1, abort_flag);
+            load_next_keys();
+          }
+        } else {
+          // the exact scores of this tile lie over both key buffers: reload only once consumed
+          mbar_wait(BAR(BAR_SX), nk & 1, abort_flag);
+          if (more) load_next_keys();
+          ++nk;
+        }
+        // P.V on the tensor cores
+        mbar_wait(BAR(BAR_P), t & 1, abort_flag);
+        mbar_wait(BAR(BAR_V0 + (t & 1)), (t >> 1) & 1, abort_flag);
+        tc_fence_after();
+        const uint32_t vbase = base + OFF_V + (t & 1) * SZ_TILE;
+#pragma unroll
+        for (int ks = 0; ks < BN / 16; ++ks) {
+          const uint64_t da = make_desc(base + OFF_P + (ks >> 2) * SZ_TILE + (ks & 3) * 32, 16, 1024);
+          const uint64_t db = make_desc(vbase + ks * 2048, SZ_TILE, 1024);
+          tc_mma(tmem + TMEM_O, da, db, IDESC_PV, ks > 0 ? 1u : 0u);
+        }
+        tc_commit(BAR(BAR_O));
       }
     }
-    if (need_exact) {
-      fence_proxy_async();
-      __syncthreads();     // (C) every exact score is in registers; its buffer may be reused
-      if (tid == 0 && more) {
-        mbar_expect_tx(BAR(BAR_KT), 64 * 128 * 4);
-        tma_load_3d(base + OFF_KT, &tm_kt, BAR(BAR_KT), j0 + BN, 0, bkv);
-        if (tile_needs_exact(jt + 1)) {
-          mbar_expect_tx(BAR(BAR_K), SZ_TILE);
-          tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K), 0, j0 + BN, bkv);
-        }
-      }
-      ++n_exact;
-    }
+    __syncwarp();
+  } else {
+    // =========================== compute warps ===============================================
+    const int qd = warp & 3, sub = warp >> 2;     // tensor-memory lane quadrant / slot in it
+    const int rg = qd * 4 + sub;                  // row group: rows 8*rg .. 8*rg+7
+    const int my_row = 32 * qd + lane;            // row this thread owns in row-per-thread phases
+    const int rho = (lane >> 2) & 7;              // row of the group whose reductions this lane ends up with
 
-    // ---- pass 2: scale, causal mask, online softmax (Eq. 1); P as bf16 in operand layout
-#pragma unroll
-    for (int r = 0; r < 8; ++r) {
-      const int row = rg * 8 + r;
-      float s[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        s[k] = Sl[r][k] * p.scale_log2e;
-        if (diag && (4 * lane + k > row)) s[k] = -INFINITY;
+    // ---- stage the query tile: deltas channel-major, per 4-row block the list of channels that
+    // fired anywhere in the block (OR of the mask words, popc for the position), the seed
+    // reference, the softmax state
+    {
+      const float* dqp = p.dq + ((size_t)bh * p.T_max + i0) * TC_D;
+      const int r_sub = lane >> 3, c_sub = lane & 7;
+      for (int it = warp; it < 32 * 8; it += NCWARP) {
+        const int rb = it >> 3, cb = it & 7;
+        const int r = rb * 4 + r_sub, c = cb * 8 + c_sub;
+        const float x = (i0 + r < T) ? dqp[(size_t)r * TC_D + c] : 0.0f;
+        sdQt[c * BM + r] = x;
       }
-      float mx = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+      if (tid < 128) {               // row 64 of the fp32 tiles: where list padding points
+        sdQt[64 * BM + tid] = 0.0f;
+        reinterpret_cast<float*>(sm + OFF_KT)[64 * BN + tid] = 0.0f;
+        reinterpret_cast<float*>(sm + OFF_KT + SZ_KT)[64 * BN + tid] = 0.0f;
+      }
+      {
+        const int blk = tid >> 4, sl = tid & 15;     // 16 threads per block of 4 rows
+        unsigned long long u = 0;
+        const uint32_t* mp = p.mask + ((size_t)bh * p.T_max + i0 + blk * 4) * 2;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      const float m_old = sM[row];
-      const float m_new = fmaxf(m_old, mx);
-      float pr[4];
+        for (int r = 0; r < 4; ++r)
+          if (i0 + blk * 4 + r < T)
+            u |= (unsigned long long)mp[r * 2] | ((unsigned long long)mp[r * 2 + 1] << 32);
+        const int n = __popcll(u);
+        uint32_t* lp = sList + blk * 64;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) pr[k] = exp2f(s[k] - m_new);
-      float sum = (pr[0] + pr[1]) + (pr[2] + pr[3]);
+        for (int k = 0; k < 4; ++k) {
+          const int c = sl * 4 + k;
+          if ((u >> c) & 1ull) lp[__popcll(u & ((1ull << c) - 1ull))] = (uint32_t)c * ROW_B;
+        }
+        const int n4 = (n + 3) >> 2;
+        if (sl < 3 && n + sl < n4 * 4) lp[n + sl] = PAD_OFF;
+        if (sl == 0) sCnt[blk] = (uint32_t)n4;
+      }
+      if (tid < TC_D) sQhat[tid] = p.qhat_tile[((size_t)bh * p.n_tiles64 + 2 * qt) * TC_D + tid];
+      if (tid < BM) { sM[tid] = -INFINITY; sL[tid] = 0.0f; }
+    }
+    float O[16];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      const __nv_bfloat162 lo = __floats2bfloat162_rn(pr[0], pr[1]);
-      const __nv_bfloat162 hi = __floats2bfloat162_rn(pr[2], pr[3]);
-      uint2 pk;
-      pk.x = *reinterpret_cast<const uint32_t*>(&lo);
-      pk.y = *reinterpret_cast<const uint32_t*>(&hi);
-      unsigned char* pp = sm + OFF_P + (size_t)(lane >> 4) * SZ_TILE + (size_t)row * 128 +
-                          ((((lane & 15) >> 1) ^ (row & 7)) << 4) + ((lane & 1) << 3);
-      *reinterpret_cast<uint2*>(pp) = pk;
+    for (int i = 0; i < 16; ++i) O[i] = 0.0f;
+    compute_barrier();
+
+    const float scale = p.scale_log2e;
+    int n_exact = 0;          // exact tiles seen so far (parity of BAR_S)
+
+    for (int jt = 0; jt <= qt; ++jt) {
+      const int j0 = jt * BN;
+      const int bf = jt & 1;
+      const bool need_exact = tile_needs_exact(jt);
+      const bool need_delta = !tile_all_in(jt);
+      const bool diag = (jt == qt);
+
+      // ---- Eq. 4 on the FP32 pipes: block-sparse 4x4 register tiles over fired channels
+      float Sl[8][4];
+#pragma unroll
+      for (int r = 0; r < 8; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) Sl[r][k] = 0.0f;
+      mbar_wait(BAR(BAR_KT_FULL0 + bf), (jt >> 1) & 1, abort_flag);
+      if (need_delta) {
+        float run[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        const uint32_t ktb = base + OFF_KT + bf * SZ_KT + 16 * lane;
+#pragma unroll
+        for (int g4 = 0; g4 < 2; ++g4) {
+          float a[4][4];
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) a[r][k] = 0.0f;
+          const int blk = rg * 2 + g4;
+          const uint32_t dqb = base + OFF_DQT + 16 * blk;
+          const uint32_t lpa = base + OFF_LIST + blk * 256;
+          const int n4 = (int)sCnt[blk];
+          uint4 e = lds128u(lpa);
+          for (int q4 = 0; q4 < n4; ++q4) {
+            const uint32_t off[4] = {e.x, e.y, e.z, e.w};
+            e = lds128u(lpa + 16 * (q4 + 1));      // next four entries (stays inside the list area)
+            float4 kv[4], dv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              kv[u] = lds128(ktb + off[u]);
+              dv[u] = lds128(dqb + off[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const float kk[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+              const float dd[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+#pragma unroll
+              for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) a[r][k] = fmaf(dd[r], kk[k], a[r][k]);
+            }
+          }
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              run[k] += a[r][k];
+              Sl[g4 * 4 + r][k] = run[k];
+            }
+        }
+        *reinterpret_cast<float4*>(sTot + (bf * 16 + rg) * BN + 4 * lane) =
+            make_float4(run[0], run[1], run[2], run[3]);
+        // seed q_hat(i0-1).k_j: this warp serves keys 8*warp .. 8*warp+7, 16 channels per lane
+        if (qt > 0) {
+          const int kq = lane & 7, cq = lane >> 3;
+          const float* kp = reinterpret_cast<const float*>(sm + OFF_KT + bf * SZ_KT) + cq * 16 * BN + 8 * warp + kq;
+          float sd = 0.0f;
+#pragma unroll
+          for (int cc = 0; cc < 16; ++cc) sd = fmaf(sQhat[cq * 16 + cc], kp[cc * BN], sd);
+          sd += __shfl_xor_sync(0xffffffffu, sd, 8);
+          sd += __shfl_xor_sync(0xffffffffu, sd, 16);
+          if (lane < 8) sSeed[bf * BN + 8 * warp + lane] = sd;
+        } else if (lane < 8) {
+          sSeed[bf * BN + 8 * warp + lane] = 0.0f;
+        }
+      }
+      fence_proxy_async();   // generic reads of the key tile are ordered before its next bulk write
       __syncwarp();
       if (lane == 0) {
-        const float al = exp2f(m_old - m_new);
-        sAlpha[(jt & 1) * BM + row] = al;
-        sL[row] = fmaf(sL[row], al, sum);
-        sM[row] = m_new;
+        mbar_arrive(BAR(BAR_KT_EMPTY0 + bf));
+        mbar_arrive(BAR(BAR_DELTA0 + bf));
       }
-    }
-    fence_proxy_async();   // P was written through the generic proxy, the tensor cores read it
-    __syncthreads();       // (D)
-    if (sMisc[1]) { aborted = true; break; }
 
-    // ---- P.V on the tensor cores; next value tile into the other buffer
-    if (tid == 0) {
-      if (!mbar_wait(BAR(BAR_V0 + (jt & 1)), (jt >> 1) & 1)) sMisc[1] = 1;
-      tc_fence_after();
-      const uint32_t vbase = base + OFF_V + (jt & 1) * SZ_TILE;
+      // ---- previous tile's P.V: rescale and accumulate (row-per-thread)
+      if (jt > 0) {
+        mbar_wait(BAR(BAR_O), (jt - 1) & 1, abort_flag);
+        tc_fence_after();
+        float v[16];
+        tc_ld16(tmem + TMEM_O + 16 * sub + ((uint32_t)(32 * qd) << 16), v);
+        const float al = sAlpha[((jt - 1) & 1) * BM + my_row];
 #pragma unroll
-      for (int ks = 0; ks < BN / 16; ++ks) {
-        const uint64_t da = make_desc(base + OFF_P + (ks >> 2) * SZ_TILE + (ks & 3) * 32, 16, 1024);
-        const uint64_t db = make_desc(vbase + ks * 2048, SZ_TILE, 1024);
-        tc_mma(tmem + TMEM_O, da, db, IDESC_PV, ks > 0 ? 1u : 0u);
+        for (int i = 0; i < 16; ++i) O[i] = fmaf(O[i], al, v[i]);
+        tc_fence_before();
       }
-      tc_commit(BAR(BAR_O));
-      if (more) {
-        const int nb = (jt + 1) & 1;
-        mbar_expect_tx(BAR(BAR_V0 + nb), SZ_TILE);
-        tma_load_3d(base + OFF_V + nb * SZ_TILE, &tm_v, BAR(BAR_V0 + nb), 0, j0 + BN, bkv);
-      }
-    }
-  }
 
-  // ---- last tile's P.V, normalisation, store ---------------------------------------------
-  if (!aborted) {
-    if (!mbar_wait(BAR(BAR_O), qt & 1)) sMisc[1] = 1;
+      // ---- every warp's block totals and seed slice are written
+      mbar_wait(BAR(BAR_DELTA0 + bf), (jt >> 1) & 1, abort_flag);
+
+      // ---- exact scores: tensor memory (row per thread) -> shared memory, 16-byte XOR swizzle
+      if (need_exact) {
+        mbar_wait(BAR(BAR_S), n_exact & 1, abort_flag);
+        tc_fence_after();
+        unsigned char* sx_row = sm + OFF_SX + (size_t)my_row * 512;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          float v[16];
+          tc_ld16(tmem + TMEM_S + 32 * sub + 16 * half + ((uint32_t)(32 * qd) << 16), v);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int chunk = 8 * sub + 4 * half + q4;
+            *reinterpret_cast<float4*>(sx_row + ((chunk ^ lane) << 4)) =
+                make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+          }
+        }
+        tc_fence_before();
+        compute_barrier();     // exact scores visible to the warps that own the rows
+      }
+
+      // ---- pass 1: hybrid select (Section III-B): exact inside the window, running sum outside
+      {
+        float bs[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (need_delta) {
+          const float4 s4 = *reinterpret_cast<const float4*>(sSeed + bf * BN + 4 * lane);
+          bs[0] = s4.x; bs[1] = s4.y; bs[2] = s4.z; bs[3] = s4.w;
+          for (int r2 = 0; r2 < rg; ++r2) {
+            const float4 t4 = *reinterpret_cast<const float4*>(sTot + (bf * 16 + r2) * BN + 4 * lane);
+            bs[0] += t4.x; bs[1] += t4.y; bs[2] += t4.z; bs[3] += t4.w;
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+          const int row = rg * 8 + r;
+          const int i = i0 + row;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) Sl[r][k] += bs[k];
+          if (need_exact) {
+            int wlo, whi;   // exact keys of row i: wlo <= j < whi
+            if (shape == 0) { wlo = (i / W) * W; whi = wlo + W; }
+            else { wlo = i - W + 1; whi = i + 1; }
+            const float4 e4 = *reinterpret_cast<const float4*>(sm + OFF_SX + (size_t)row * 512 +
+                                                               ((lane ^ (row & 31)) << 4));
+            const float ex[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const int j = j0 + 4 * lane + k;
+              if (j >= wlo && j < whi) Sl[r][k] = ex[k];
+            }
+          }
+          if (diag) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (4 * lane + k > row) Sl[r][k] = -INFINITY;   // causal mask on the diagonal tile
+          }
+        }
+      }
+      if (need_exact) {
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(BAR_SX));   // this warp no longer needs the exact-score buffer
+        ++n_exact;
+      }
+
+      // ---- pass 2: scale, online softmax (Eq. 1); P as bf16 in the operand layout
+      {
+        float v8[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) v8[r] = fmaxf(fmaxf(Sl[r][0], Sl[r][1]), fmaxf(Sl[r][2], Sl[r][3]));
+        const float zmax = reduce8<true>(v8, lane);          // raw maximum of row rho
+        const int row_o = rg * 8 + rho;
+        const float m_old = sM[row_o];
+        const float m_new = fmaxf(m_old, zmax * scale);
+        const float al = ex2(m_old - m_new);
+        float mn[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) mn[r] = __shfl_sync(0xffffffffu, m_new, 4 * r);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+          const int row = rg * 8 + r;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) Sl[r][k] = ex2(fmaf(Sl[r][k], scale, -mn[r]));
+          v8[r] = (Sl[r][0] + Sl[r][1]) + (Sl[r][2] + Sl[r][3]);
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(Sl[r][0], Sl[r][1]);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(Sl[r][2], Sl[r][3]);
+          uint2 pk;
+          pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+          unsigned char* pp = sm + OFF_P + (size_t)(lane >> 4) * SZ_TILE + (size_t)row * 128 +
+                              ((((lane & 15) >> 1) ^ (row & 7)) << 4) + ((lane & 1) << 3);
+          *reinterpret_cast<uint2*>(pp) = pk;
+        }
+        const float zsum = reduce8<false>(v8, lane);
+        if ((lane & 3) == 0) {
+          sAlpha[bf * BM + row_o] = al;
+          sL[row_o] = fmaf(sL[row_o], al, zsum);
+          sM[row_o] = m_new;
+        }
+      }
+      fence_proxy_async();   // P was written through the generic proxy, the tensor cores read it
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(BAR_P));
+    }
+
+    // ---- last tile's P.V, normalisation, store -------------------------------------------
+    mbar_wait(BAR(BAR_O), qt & 1, abort_flag);
     tc_fence_after();
     float v[16];
     tc_ld16(tmem + TMEM_O + 16 * sub + ((uint32_t)(32 * qd) << 16), v);
     const float al = sAlpha[(qt & 1) * BM + my_row];
     const float inv = 1.0f / sL[my_row];
-    if (i0 + my_row < T && !sMisc[1]) {
+    if (i0 + my_row < T && !*abort_flag) {
       uint32_t w[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -555,10 +642,8 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       op[1] = make_uint4(w[4], w[5], w[6], w[7]);
     }
     tc_fence_before();
-  } else {
-    // a wait ran out: give copies and tensor-core work already in flight time to land
-    for (int i = 0; i < 64; ++i) __nanosleep(1000);
   }
+
   __syncthreads();
   if (tid == 0 && sMisc[1]) atomicMax(&p.counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
   if (warp == 0) {
