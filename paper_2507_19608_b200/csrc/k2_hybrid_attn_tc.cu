@@ -54,8 +54,9 @@ constexpr uint32_t OFF_P = OFF_V + 2 * SZ_TILE;          // bf16 [2][128 rows][6
 constexpr uint32_t OFF_KT = OFF_P + 2 * SZ_TILE;         // two buffers fp32 [64 channels + 1][128 keys]
 constexpr uint32_t OFF_SX = OFF_KT;                      // fp32 [128][128] exact scores (over both)
 constexpr uint32_t OFF_DQT = OFF_KT + 2 * SZ_KT;         // fp32 [64 channels + 1][128 rows]
-constexpr uint32_t OFF_LIST = OFF_DQT + 65 * ROW_B;      // u32 [32 blocks][64]: fired channel * ROW_B
-constexpr uint32_t OFF_CNT = OFF_LIST + 32 * 64 * 4;     // u32 [32]: list length / 4
+constexpr uint32_t LIST_LD = 68;                         // list entries per block: 64 + one padding quad
+constexpr uint32_t OFF_LIST = OFF_DQT + 65 * ROW_B;      // u32 [32 blocks][LIST_LD]: fired channel * ROW_B
+constexpr uint32_t OFF_CNT = OFF_LIST + 32 * LIST_LD * 4;  // u32 [32]: list length / 4
 constexpr uint32_t OFF_TOT = OFF_CNT + 32 * 4;           // fp32 [2][16][128]
 constexpr uint32_t OFF_SEED = OFF_TOT + 2 * 16 * 128 * 4;  // fp32 [2][128]
 constexpr uint32_t OFF_ALPHA = OFF_SEED + 2 * 128 * 4;   // fp32 [2][128]
@@ -403,14 +404,15 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           if (i0 + blk * 4 + r < T)
             u |= (unsigned long long)mp[r * 2] | ((unsigned long long)mp[r * 2 + 1] << 32);
         const int n = __popcll(u);
-        uint32_t* lp = sList + blk * 64;
+        uint32_t* lp = sList + blk * LIST_LD;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int c = sl * 4 + k;
           if ((u >> c) & 1ull) lp[__popcll(u & ((1ull << c) - 1ull))] = (uint32_t)c * ROW_B;
         }
+        // pad to a multiple of 4 and add one more quad: the loop reads one quad ahead
         const int n4 = (n + 3) >> 2;
-        if (sl < 3 && n + sl < n4 * 4) lp[n + sl] = PAD_OFF;
+        if (sl < 7 && n + sl < n4 * 4 + 4) lp[n + sl] = PAD_OFF;
         if (sl == 0) sCnt[blk] = (uint32_t)n4;
       }
       if (tid < TC_D) sQhat[tid] = p.qhat_tile[((size_t)bh * p.n_tiles64 + 2 * qt) * TC_D + tid];
@@ -450,27 +452,31 @@ hybrid_attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             for (int k = 0; k < 4; ++k) a[r][k] = 0.0f;
           const int blk = rg * 2 + g4;
           const uint32_t dqb = base + OFF_DQT + 16 * blk;
-          const uint32_t lpa = base + OFF_LIST + blk * 256;
+          const uint32_t lpa = base + OFF_LIST + blk * (LIST_LD * 4);
           const int n4 = (int)sCnt[blk];
+          // software pipeline over single entries: the loads of the next entry are in flight
+          // while the current entry's 16 multiply-adds issue
           uint4 e = lds128u(lpa);
+          float4 kvA, dvA, kvB, dvB;
+          auto mac16 = [&](const float4& kv, const float4& dv) {
+            const float kk[4] = {kv.x, kv.y, kv.z, kv.w};
+            const float dd[4] = {dv.x, dv.y, dv.z, dv.w};
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+              for (int k = 0; k < 4; ++k) a[r][k] = fmaf(dd[r], kk[k], a[r][k]);
+          };
+          kvA = lds128(ktb + e.x); dvA = lds128(dqb + e.x);
           for (int q4 = 0; q4 < n4; ++q4) {
-            const uint32_t off[4] = {e.x, e.y, e.z, e.w};
-            e = lds128u(lpa + 16 * (q4 + 1));      // next four entries (stays inside the list area)
-            float4 kv[4], dv[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              kv[u] = lds128(ktb + off[u]);
-              dv[u] = lds128(dqb + off[u]);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const float kk[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
-              const float dd[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
-#pragma unroll
-              for (int r = 0; r < 4; ++r)
-#pragma unroll
-                for (int k = 0; k < 4; ++k) a[r][k] = fmaf(dd[r], kk[k], a[r][k]);
-            }
+            kvB = lds128(ktb + e.y); dvB = lds128(dqb + e.y);
+            mac16(kvA, dvA);
+            kvA = lds128(ktb + e.z); dvA = lds128(dqb + e.z);
+            mac16(kvB, dvB);
+            kvB = lds128(ktb + e.w); dvB = lds128(dqb + e.w);
+            e = lds128u(lpa + 16 * (q4 + 1));      // next quad (the list carries one padding quad)
+            mac16(kvA, dvA);
+            kvA = lds128(ktb + e.x); dvA = lds128(dqb + e.x);
+            mac16(kvB, dvB);
           }
 #pragma unroll
           for (int r = 0; r < 4; ++r)
