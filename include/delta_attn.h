@@ -220,8 +220,13 @@ DELTA_API delta_status_t delta_state_view(const delta_state_t* st, int32_t what,
 DELTA_API int32_t delta_state_position(const delta_state_t* st);
 
 /* Which prefill kernel the next delta_attn_prefill on this state will use:
- * 0 = generic CUDA-core kernel, 1 = tcgen05/TMA kernel.  delta_state_set_prefill_kernel
- * forces one (-1 = automatic); forcing a kernel the configuration has none for returns
+ *   0 = generic CUDA-core kernel (every configuration);
+ *   1 = tcgen05/TMA kernel, out-of-window scores by Eq. 4's running sum of sparse delta
+ *       products on the FP32 pipes, skipping all-zero delta blocks (bf16, d = 64);
+ *   2 = tcgen05/TMA kernel, out-of-window scores by the telescoped form of Eq. 4,
+ *       R(i)[j] = q_hat(i).k_j, as one more tensor-core product (bf16, d = 64).
+ * All three compute the same function.  delta_state_set_prefill_kernel forces one
+ * (-1 = automatic); forcing a kernel the configuration has none for returns
  * DELTA_ERR_UNSUPPORTED. */
 DELTA_API int32_t delta_state_prefill_kernel(const delta_state_t* st);
 DELTA_API delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which);

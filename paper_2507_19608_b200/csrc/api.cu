@@ -79,6 +79,8 @@ static void carve(const delta_config_t& c, char* base, Workspace* w) {
   w->qhat_tile_bf16 = (c.dtype == DELTA_BF16) ? (__nv_bfloat16*)take(BH * nt * c.d * 2) : nullptr;
   w->kt = (c.dtype == DELTA_BF16 && tc_kernel_shape(c.d))
               ? (float*)take(BKV * c.d * (((size_t)c.T_max + 3) / 4 * 4) * 4) : nullptr;
+  w->qhat_rows = (c.dtype == DELTA_BF16 && tc_kernel_shape(c.d))
+                     ? (__nv_bfloat16*)take(BH * c.T_max * c.d * 2) : nullptr;
   w->total_bytes = off;
 }
 
@@ -186,8 +188,8 @@ int32_t delta_state_prefill_kernel(const delta_state_t* st) {
 }
 
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
-  if (!st || which < -1 || which > 1) return DELTA_ERR_INVALID_ARG;
-  if (which == 1 && !tc_eligible(st)) return DELTA_ERR_UNSUPPORTED;
+  if (!st || which < -1 || which > 2) return DELTA_ERR_INVALID_ARG;
+  if (which >= 1 && !tc_eligible(st)) return DELTA_ERR_UNSUPPORTED;
   st->forced_kernel = which;
   return DELTA_OK;
 }
@@ -214,9 +216,10 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   cudaError_t e;
   const bool prof = st->profiling;
 #define MARK(i) do { if (prof && (e = cudaEventRecord(st->ev[i], cs)) != cudaSuccess) return cuda_fail(e); } while (0)
-  const bool use_tc = delta_state_prefill_kernel(st) == 1;
+  const int which = delta_state_prefill_kernel(st);
+  const bool use_tc = which == 1;
   MARK(0);
-  if ((e = launch_delta_chain(st->shape, st->ws, q, T, theta, c.dtype, c.init, cs)) != cudaSuccess)
+  if ((e = launch_delta_chain(st->shape, st->ws, q, T, theta, c.dtype, c.init, which == 2, cs)) != cudaSuccess)
     return cuda_fail(e);
   MARK(1);
   if ((e = launch_delta_finish(st->shape, st->ws, k, T, window, c.prefill_window, c.dtype, use_tc, cs)) !=
@@ -225,6 +228,8 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   MARK(2);
   if (use_tc) {
     e = launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
+  } else if (which == 2) {
+    e = launch_hybrid_attn_tcq(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
   } else {
     e = launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window,
                                    c.dtype, cs);

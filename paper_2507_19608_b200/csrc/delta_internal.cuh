@@ -33,6 +33,7 @@ struct Workspace {
   uint32_t* dec_ticket; // [B,H_kv]
   __nv_bfloat16* qhat_tile_bf16;  // [B,H,n_tiles,d] (bf16 configurations only)
   float* kt;            // [B,H_kv,d,round_up(T_max,4)] channel-major fp32 keys (tensor-core prefill only)
+  __nv_bfloat16* qhat_rows;  // [B,H,T_max,d] reference state after every row (telescoped prefill only)
   size_t total_bytes;
 };
 
@@ -46,7 +47,7 @@ void count_launch(int n = 1);
 // K1a: token-sequential delta chain over the query stream (Eq. 2-3): delta values, mask words,
 // per-tile reference snapshots, final reference.
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
-                               float theta, int dtype, int init, cudaStream_t st);
+                               float theta, int dtype, int init, bool want_qhat_rows, cudaStream_t st);
 // K1b: row-parallel finish: counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* k, int T,

@@ -55,8 +55,8 @@ template <typename TIn, int D>
 __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     const TIn* __restrict__ q, float* __restrict__ dq, uint32_t* __restrict__ mask,
     float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
-    unsigned long long* __restrict__ counters, int T, int T_max, int n_tiles, float theta,
-    int basis_exact) {
+    __nv_bfloat16* __restrict__ qhat_rows, unsigned long long* __restrict__ counters, int T,
+    int T_max, int n_tiles, float theta, int basis_exact) {
   constexpr int NW = D / 32;                       // chain warps = mask words per row
   constexpr uint32_t ROW_BYTES = D * sizeof(TIn);
   constexpr uint32_t STAGE_BYTES = RC * ROW_BYTES;
@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     // ---- chain warps: thread c owns channel c
     const int c = tid;
     float* dqp = dq + (size_t)bh * T_max * D + c;
+    __nv_bfloat16* qrp = qhat_rows ? qhat_rows + (size_t)bh * T_max * D + c : nullptr;
     uint32_t* maskp = mask + (size_t)bh * T_max * NW + warp;
     float qh = 0.0f;          // reference state, starts at zero (Eq. 3)
     bool failed = false;
@@ -128,6 +129,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
           const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
           qh = fire ? x[r] : qh;
           dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
+          if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
           bits |= fire ? (1u << r) : 0u;
         }
       } else {
@@ -145,6 +147,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
           }
           qh = fire ? x : qh;
           dqp[(size_t)(t0 + r) * D] = delta;
+          if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
           bits |= fire ? (1u << r) : 0u;
         }
       }
@@ -171,7 +174,8 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
 }
 
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
-                               float theta, int dtype, int init, cudaStream_t st) {
+                               float theta, int dtype, int init, bool want_qhat_rows, cudaStream_t st) {
+  __nv_bfloat16* qrows = want_qhat_rows ? w.qhat_rows : nullptr;
   const int grid = s.B * s.H;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
   cudaError_t err = cudaSuccess;
@@ -183,7 +187,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
       err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
       if (err != cudaSuccess) return err;                                                        \
     }                                                                                            \
-    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.dq, w.mask, w.qhat_tile, w.qhat[0],       \
+    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.dq, w.mask, w.qhat_tile, w.qhat[0], qrows, \
                                       w.counters, T, s.T_max, s.n_tiles, theta, basis);          \
   } while (0)
   if (dtype == DELTA_F32) {

@@ -1,0 +1,363 @@
+// K2 (tensor-core, telescoped) -- hybrid delta attention for bf16 inputs on sm_100a with every
+// score on the tensor cores (Section III-B; Eq. 1, Eq. 4).
+//
+// Eq. 4's running sum telescopes: R(i)[j] = (sum over rows s <= i of Delta q(s)) . k_j, and by
+// Eq. 3 that sum is the reference state q_hat(i), so the out-of-window score of pair (i, j) is
+// the dense product q_hat(i).k_j.  For bf16 inputs every element of q_hat is a copy of an input
+// element (or 0), hence exactly bf16: the whole out-of-window score matrix is one more
+// Q_hat.K^T on the tensor cores, with the rows of Q_hat written by the delta-construction
+// kernel.  Nothing is skipped (the zeros of the delta matrix are unstructured, and at the
+// sparsity the method reaches a 4-row block of it is nearly dense), but the tensor cores do
+// the dense product far faster than the FP32 pipes do the sparse one.
+//
+// One CTA owns 128 query rows of one head: 16 compute warps and a control warp.  The control
+// thread streams K and V tiles with TMA and issues, per 128-key tile, Q_hat.K^T (and Q.K^T if
+// the tile touches the window) into a double-buffered tensor-memory score region, one tile
+// ahead of the softmax.  Compute threads work row-per-thread straight out of tensor memory:
+// thread (row, quarter) reads 32 score columns of its row, selects exact or telescoped per
+// element, exchanges the row maximum with the three other quarters through shared memory,
+// exponentiates, writes its 32 probabilities as bf16 into the operand layout of the P.V
+// product, and rescales/accumulates its 16 output columns from the previous tile's P.V.
+//
+// Every wait on an mbarrier is bounded (see tc_common.cuh); after a time-out the protocol
+// still runs to its end, nothing is stored and the status word records DELTA_ERR_TIMEOUT.
+#include <cuda.h>
+
+#include "k2_tc.cuh"
+#include "tc_common.cuh"
+
+namespace delta {
+
+using namespace tc;
+
+namespace {
+
+constexpr int BM = 128, BN = 128, NCWARP = 16, NCTHR = NCWARP * 32, NTHR = NCTHR + 32;
+constexpr int TQ_D = 64;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t TMEM_SH = 0;        // telescoped scores, two buffers of 128 columns
+constexpr uint32_t TMEM_SX = 256;      // exact scores, 128 columns
+constexpr uint32_t TMEM_O = 384;       // P.V tile, 64 columns
+
+constexpr uint32_t SZ_TILE = 128 * 64 * 2;
+constexpr uint32_t OFF_Q = 0;
+constexpr uint32_t OFF_QH = OFF_Q + SZ_TILE;
+constexpr uint32_t OFF_K = OFF_QH + SZ_TILE;          // two buffers
+constexpr uint32_t OFF_V = OFF_K + 2 * SZ_TILE;       // two buffers
+constexpr uint32_t OFF_P = OFF_V + 2 * SZ_TILE;       // bf16 [2][128 rows][64 keys]
+constexpr uint32_t OFF_PMAX = OFF_P + 2 * SZ_TILE;    // fp32 [2][128 rows][4 quarters]
+constexpr uint32_t OFF_BAR = OFF_PMAX + 2 * 128 * 4 * 4;
+constexpr uint32_t OFF_MISC = OFF_BAR + 16 * 8;
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;
+
+enum Bar {
+  BAR_Q = 0, BAR_K0, BAR_K1, BAR_V0, BAR_V1, BAR_S0, BAR_S1, BAR_O,   // one arrival (+ bytes)
+  BAR_SFREE0, BAR_SFREE1,                                             // 16 arrivals: scores read
+  BAR_P,                                                              // 16 arrivals: P written
+  NUM_BARS
+};
+
+struct TqParams {
+  __nv_bfloat16* out;
+  unsigned long long* counters;
+  int T, H, g, W, shape;
+  float scale_log2e;
+};
+
+}  // namespace
+
+__global__ void __launch_bounds__(NTHR, 1)
+hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qh,
+                       const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                       const TqParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw);
+  float* sPmax = reinterpret_cast<float*>(sm + OFF_PMAX);
+  volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
+  volatile uint32_t* abort_flag = sMisc + 1;
+  const uint32_t bar0 = base + OFF_BAR;
+#define BAR(i) (bar0 + 8u * (uint32_t)(i))
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;  // heaviest query tiles of every head first
+  const int bh = blockIdx.x;
+  const int b = bh / p.H, h = bh - b * p.H;
+  const int bkv = b * (p.H / p.g) + h / p.g;
+  const int i0 = qt * BM;
+  const int T = p.T, W = p.W, shape = p.shape;
+  const int i1 = min(i0 + BM, T) - 1;
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     base + OFF_MISC),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    for (int i = 0; i < NUM_BARS; ++i) mbar_init(BAR(i), (i >= BAR_SFREE0) ? (uint32_t)NCWARP : 1u);
+    sMisc[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sMisc[0];
+
+  auto tile_needs_exact = [&](int jt) -> bool {
+    if (W <= 0) return false;
+    const int j0 = jt * BN, j1 = min(j0 + BN, T) - 1;
+    if (shape == 0) return (i0 / W <= j1 / W) && (j0 / W <= i1 / W);
+    return max(0, i0 - j1) < W;
+  };
+
+  if (warp == NCWARP) {
+    // =========================== control warp ===============================================
+    if (lane == 0) {
+      const uint32_t IDESC_QK = make_idesc(BN, 0);
+      const uint32_t IDESC_PV = make_idesc(TQ_D, 1);
+      mbar_expect_tx(BAR(BAR_Q), 2 * SZ_TILE);
+      tma_load_3d(base + OFF_Q, &tm_q, BAR(BAR_Q), 0, i0, bh);
+      tma_load_3d(base + OFF_QH, &tm_qh, BAR(BAR_Q), 0, i0, bh);
+      mbar_expect_tx(BAR(BAR_K0), SZ_TILE);
+      tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K0), 0, 0, bkv);
+      mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
+      tma_load_3d(base + OFF_V, &tm_v, BAR(BAR_V0), 0, 0, bkv);
+      if (qt >= 1) {
+        mbar_expect_tx(BAR(BAR_K1), SZ_TILE);
+        tma_load_3d(base + OFF_K + SZ_TILE, &tm_k, BAR(BAR_K1), 0, BN, bkv);
+      }
+      // scores of tile t: Q_hat.K^T into buffer t&1, plus Q.K^T if the tile touches the window
+      auto issue_scores = [&](int t) {
+        const int bf = t & 1;
+        mbar_wait(BAR(BAR_K0 + bf), (t >> 1) & 1, abort_flag);
+        tc_fence_after();
+        const uint32_t kb = base + OFF_K + bf * SZ_TILE;
+#pragma unroll
+        for (int ks = 0; ks < TQ_D / 16; ++ks)
+          tc_mma(tmem + TMEM_SH + bf * 128, make_desc(base + OFF_QH + ks * 32, 16, 1024),
+                 make_desc(kb + ks * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
+        if (tile_needs_exact(t)) {
+#pragma unroll
+          for (int ks = 0; ks < TQ_D / 16; ++ks)
+            tc_mma(tmem + TMEM_SX, make_desc(base + OFF_Q + ks * 32, 16, 1024),
+                   make_desc(kb + ks * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
+        }
+        tc_commit(BAR(BAR_S0 + bf));
+      };
+      mbar_wait(BAR(BAR_Q), 0, abort_flag);
+      issue_scores(0);
+      for (int t = 0; t <= qt; ++t) {
+        const bool more = t < qt;
+        const int nb = (t + 1) & 1;
+        const bool next_exact = more && tile_needs_exact(t + 1);
+        // next tile's scores one tile ahead, unless it needs the single exact-score buffer
+        if (more && !next_exact) {
+          if (t >= 1) mbar_wait(BAR(BAR_SFREE0 + nb), ((t - 1) >> 1) & 1, abort_flag);
+          issue_scores(t + 1);
+        }
+        // key buffer t&1 is free once the scores of tile t are done: stream tile t+2 into it
+        mbar_wait(BAR(BAR_S0 + (t & 1)), (t >> 1) & 1, abort_flag);
+        if (t + 2 <= qt) {
+          mbar_expect_tx(BAR(BAR_K0 + (t & 1)), SZ_TILE);
+          tma_load_3d(base + OFF_K + (t & 1) * SZ_TILE, &tm_k, BAR(BAR_K0 + (t & 1)), 0, (t + 2) * BN, bkv);
+        }
+        if (t >= 1) mbar_wait(BAR(BAR_O), (t - 1) & 1, abort_flag);   // P.V(t-1) done: its V buffer is free
+        if (more) {
+          mbar_expect_tx(BAR(BAR_V0 + nb), SZ_TILE);
+          tma_load_3d(base + OFF_V + nb * SZ_TILE, &tm_v, BAR(BAR_V0 + nb), 0, (t + 1) * BN, bkv);
+        }
+        // P.V of this tile
+        mbar_wait(BAR(BAR_P), t & 1, abort_flag);
+        mbar_wait(BAR(BAR_V0 + (t & 1)), (t >> 1) & 1, abort_flag);
+        tc_fence_after();
+        const uint32_t vbase = base + OFF_V + (t & 1) * SZ_TILE;
+#pragma unroll
+        for (int ks = 0; ks < BN / 16; ++ks)
+          tc_mma(tmem + TMEM_O, make_desc(base + OFF_P + (ks >> 2) * SZ_TILE + (ks & 3) * 32, 16, 1024),
+                 make_desc(vbase + ks * 2048, SZ_TILE, 1024), IDESC_PV, ks > 0 ? 1u : 0u);
+        tc_commit(BAR(BAR_O));
+        if (next_exact) {
+          // every compute warp has read tile t's scores (it wrote P after that)
+          mbar_wait(BAR(BAR_SFREE0 + (t & 1)), (t >> 1) & 1, abort_flag);
+          if (t >= 1) mbar_wait(BAR(BAR_SFREE0 + nb), ((t - 1) >> 1) & 1, abort_flag);
+          issue_scores(t + 1);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // =========================== compute warps: row per thread ==============================
+    const int qd = warp & 3, sub = warp >> 2;     // tensor-memory lane quadrant / column quarter
+    const int row = 32 * qd + lane;
+    const int i = i0 + row;
+    const uint32_t lane_sel = (uint32_t)(32 * qd) << 16;
+    const float scale = p.scale_log2e;
+    float O[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) O[c] = 0.0f;
+    float m_run = -INFINITY, l_part = 0.0f, alpha_prev = 1.0f;
+    int wlo = 0, whi = 0;       // exact keys of row i: wlo <= j < whi
+    if (W > 0) {
+      if (shape == 0) { wlo = (i / W) * W; whi = wlo + W; }
+      else { wlo = i - W + 1; whi = i + 1; }
+    }
+
+    for (int jt = 0; jt <= qt; ++jt) {
+      const int bf = jt & 1;
+      const int jc0 = jt * BN + 32 * sub;      // first key of this thread's 32 columns
+      const bool need_exact = tile_needs_exact(jt);
+      const bool diag = (jt == qt);
+
+      mbar_wait(BAR(BAR_S0 + bf), (jt >> 1) & 1, abort_flag);
+      tc_fence_after();
+      float s[32];
+      {
+        float v[16];
+        tc_ld16(tmem + TMEM_SH + bf * 128 + 32 * sub + lane_sel, v);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) s[c] = v[c];
+        tc_ld16(tmem + TMEM_SH + bf * 128 + 32 * sub + 16 + lane_sel, v);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) s[16 + c] = v[c];
+      }
+      if (need_exact) {
+        // hybrid select (Section III-B): exact score inside the window
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          float v[16];
+          tc_ld16(tmem + TMEM_SX + 32 * sub + 16 * hf + lane_sel, v);
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const int j = jc0 + 16 * hf + c;
+            if (j >= wlo && j < whi) s[16 * hf + c] = v[c];
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(BAR_SFREE0 + bf));
+      if (diag) {
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          if (jc0 + c > i) s[c] = -INFINITY;     // causal mask on the diagonal tile
+      }
+      // row maximum: own 32 columns, then the three other quarters through shared memory
+      float mx = s[0];
+#pragma unroll
+      for (int c = 1; c < 32; ++c) mx = fmaxf(mx, s[c]);
+      sPmax[(bf * BM + row) * 4 + sub] = mx;
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + qd) : "memory");   // the four warps of this quadrant
+      const float4 pm = *reinterpret_cast<const float4*>(sPmax + (bf * BM + row) * 4);
+      mx = fmaxf(fmaxf(pm.x, pm.y), fmaxf(pm.z, pm.w));
+      const float m_new = fmaxf(m_run, mx * scale);
+      const float al = ex2(m_run - m_new);
+      m_run = m_new;
+      float sum = 0.0f;
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        s[c] = ex2(fmaf(s[c], scale, -m_new));
+        sum += s[c];
+      }
+      l_part = fmaf(l_part, al, sum);
+
+      // previous tile's P.V: rescale and accumulate; after it the P buffer may be rewritten
+      if (jt > 0) {
+        mbar_wait(BAR(BAR_O), (jt - 1) & 1, abort_flag);
+        tc_fence_after();
+        float v[16];
+        tc_ld16(tmem + TMEM_O + 16 * sub + lane_sel, v);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) O[c] = fmaf(O[c], alpha_prev, v[c]);
+        tc_fence_before();
+      }
+      alpha_prev = al;
+
+      // P as bf16 in the operand layout: this thread's 32 keys are 4 chunks of 16 bytes
+      {
+        unsigned char* prow = sm + OFF_P + (size_t)(sub >> 1) * SZ_TILE + (size_t)row * 128;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const __nv_bfloat162 t2 = __floats2bfloat162_rn(s[8 * q4 + 2 * e], s[8 * q4 + 2 * e + 1]);
+            w[e] = *reinterpret_cast<const uint32_t*>(&t2);
+          }
+          const int chunk = 4 * (sub & 1) + q4;
+          *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(BAR_P));
+    }
+
+    // ---- last tile's P.V, row sum over the four quarters, normalisation, store
+    mbar_wait(BAR(BAR_O), qt & 1, abort_flag);
+    tc_fence_after();
+    float v[16];
+    tc_ld16(tmem + TMEM_O + 16 * sub + lane_sel, v);
+    sPmax[(((qt + 1) & 1) * BM + row) * 4 + sub] = l_part;
+    asm volatile("bar.sync %0, 128;" ::"r"(1 + qd) : "memory");
+    const float4 lp = *reinterpret_cast<const float4*>(sPmax + (((qt + 1) & 1) * BM + row) * 4);
+    const float inv = 1.0f / ((lp.x + lp.y) + (lp.z + lp.w));
+    if (i < T && !*abort_flag) {
+      uint32_t w[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const __nv_bfloat162 t2 = __floats2bfloat162_rn(fmaf(O[2 * c], alpha_prev, v[2 * c]) * inv,
+                                                        fmaf(O[2 * c + 1], alpha_prev, v[2 * c + 1]) * inv);
+        w[c] = *reinterpret_cast<const uint32_t*>(&t2);
+      }
+      uint4* op = reinterpret_cast<uint4*>(p.out + ((size_t)bh * T + i) * TQ_D + 16 * sub);
+      op[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      op[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+    tc_fence_before();
+  }
+
+  __syncthreads();
+  if (tid == 0 && sMisc[1]) atomicMax(&p.counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS)
+                 : "memory");
+  }
+#undef BAR
+}
+
+cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
+                                   const void* v, void* out, int T, int window, int shape,
+                                   cudaStream_t st) {
+  if (s.d != TQ_D || !w.qhat_rows) return cudaErrorNotSupported;
+  const uint64_t BH = (uint64_t)s.B * s.H, BKV = (uint64_t)s.B * s.H_kv;
+  CUtensorMap tq, tqh, tk, tv;
+  const bool ok =
+      encode3(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, q, TQ_D, (uint64_t)T, BH, TQ_D * 2,
+              (uint64_t)T * TQ_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tqh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, w.qhat_rows, TQ_D, (uint64_t)T, BH, TQ_D * 2,
+              (uint64_t)s.T_max * TQ_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k, TQ_D, (uint64_t)T, BKV, TQ_D * 2,
+              (uint64_t)s.T_max * TQ_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, v, TQ_D, (uint64_t)T, BKV, TQ_D * 2,
+              (uint64_t)s.T_max * TQ_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (!ok) return cudaErrorInvalidValue;
+  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)SMEM_BYTES);
+  if (err != cudaSuccess) return err;
+  TqParams p;
+  p.out = (__nv_bfloat16*)out;
+  p.counters = w.counters;
+  p.T = T; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
+  p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
+  const dim3 grid((unsigned)BH, (T + BM - 1) / BM);
+  hybrid_attn_tcq_kernel<<<grid, NTHR, SMEM_BYTES, st>>>(tq, tqh, tk, tv, p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace delta
