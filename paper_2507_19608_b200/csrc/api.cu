@@ -184,7 +184,7 @@ static bool tc_eligible(const delta_state* st) {
 int32_t delta_state_prefill_kernel(const delta_state_t* st) {
   if (!st) return -1;
   if (st->forced_kernel >= 0) return st->forced_kernel;
-  return tc_eligible(st) ? 1 : 0;
+  return tc_eligible(st) ? 2 : 0;   // the telescoped tensor-core kernel is the fastest where it applies
 }
 
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {

@@ -114,27 +114,35 @@ CASES = [
     (1, 2, 2, 64, 128, "bf16", 0.0, 5, "sliding"),     # theta = 0
     (1, 2, 1, 1, 64, "bf16", 0.1, 4, "block"),         # one token
     (1, 8, 2, 320, 64, "bf16", 1e9, 16, "block"),      # nothing fires after the basis row
+    (1, 4, 2, 700, 64, "bf16", 0.3, 64, "block"),      # six 128-row tiles, ragged last tile
+    (2, 2, 1, 513, 64, "bf16", 0.15, 200, "sliding"),  # window wider than a tile, one row in the last tile
+    (1, 2, 2, 384, 64, "bf16", 0.25, 1000, "sliding"), # every tile exact
+    (1, 2, 1, 300, 64, "bf16", 0.2, 0, "sliding"),     # no exact score at all
+    (1, 2, 2, 260, 64, "bf16", 0.2, 128, "block", "zero_state"),
 ]
 
 
-@pytest.mark.parametrize("case", CASES, ids=[f"{c[5]}-T{c[3]}-d{c[4]}-W{c[7]}{c[8][0]}-th{c[6]}" for c in CASES])
-@pytest.mark.parametrize("kernel", [0, 1], ids=["generic", "tensorcore"])
+@pytest.mark.parametrize("case", CASES, ids=[f"{c[5]}-T{c[3]}-d{c[4]}-W{c[7]}{c[8][0]}-th{c[6]}{'-zs' if len(c) > 9 else ''}" for c in CASES])
+@pytest.mark.parametrize("kernel", [0, 1, 2], ids=["generic", "tc_delta", "tc_telescoped"])
 def test_prefill_output_matches_oracle(B, case, kernel):
     from tests.gpu_helpers import run_prefill, to_host_f64
-    Bn, H, Hk, T, d, dtype, theta, W, shape = case
+    Bn, H, Hk, T, d, dtype, theta, W, shape = case[:9]
+    init = case[9] if len(case) > 9 else "basis_exact"
     q, k, v = _inputs(Bn, H, Hk, T, d, dtype, seed=100 + T + d)
-    if kernel == 1:
+    if kernel >= 1:
         cfg = B.make_config(Bn, H, Hk, d, T, dtype)
         ws = torch.empty(B.delta_state_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
         st0 = B.delta_state_init(cfg, workspace=ws)
         try:
-            B.delta_state_set_prefill_kernel(st0, 1)
+            B.delta_state_set_prefill_kernel(st0, kernel)
         except B.DeltaError as e:
             assert e.status == B.DELTA_ERR_UNSUPPORTED
             pytest.skip("no tensor-core kernel for this configuration")
-    st, out, _, _ = run_prefill(B, q, k, v, theta, W, dtype, shape=shape, kernel=kernel)
-    ref, heads = O.prefill_mha(q, k, v, theta, W, shape)
+    st, out, _, _ = run_prefill(B, q, k, v, theta, W, dtype, shape=shape, init=init, kernel=kernel)
+    assert B.delta_state_prefill_kernel(st) == kernel
+    ref, heads = O.prefill_mha(q, k, v, theta, W, shape, init=init)
     _check_out(to_host_f64(out), ref, dtype, "prefill out")
+    assert B.delta_sparsity_stats(st)["device_status"] == 0
     # hand-off state for decode: reference query and the last score row
     R = B.delta_state_view(st, B.DELTA_VIEW_R).cpu().numpy()
     for b in range(Bn):
@@ -261,19 +269,21 @@ def test_state_errors(B):
 
 
 # ------------------------------------------------------------------ full-size configurations
-@pytest.mark.parametrize("name,theta,heads", [
-    ("llama32_1b_prefill", 0.1, (0, 13, 31)),
-    ("llama32_1b_prefill", 0.3, (5, 18)),
-    ("bitnet_2b_prefill", 0.29, (0, 19)),
+@pytest.mark.parametrize("name,theta,heads,kernel", [
+    ("llama32_1b_prefill", 0.1, (0, 13, 31), 2),
+    ("llama32_1b_prefill", 0.3, (5, 18), 2),
+    ("llama32_1b_prefill", 0.3, (7, 30), 1),
+    ("llama32_1b_prefill", 0.05, (11,), 1),
+    ("bitnet_2b_prefill", 0.29, (0, 19), 0),
 ])
-def test_full_size_prefill_sampled_heads(B, name, theta, heads):
+def test_full_size_prefill_sampled_heads(B, name, theta, heads, kernel):
     """The benchmark's launch configuration at full size: delta arrays of the sampled heads are
     bit-exact, outputs of the sampled heads match the oracle, global counters match a recount
     over all heads."""
     from tests.gpu_helpers import run_prefill, to_host_f64
     w = WL.WORKLOADS[name]
     t = WL.make_qkv(w)
-    st, out, _, _ = run_prefill(B, t["q"], t["k"], t["v"], theta, w.window, w.dtype)
+    st, out, _, _ = run_prefill(B, t["q"], t["k"], t["v"], theta, w.window, w.dtype, kernel=kernel)
     g = w.H // w.H_kv
     dq = B.delta_state_view(st, B.DELTA_VIEW_DQ)
     mask = B.delta_state_view(st, B.DELTA_VIEW_MASK)
