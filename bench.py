@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
                   "sm_max_mhz": 1965.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the hybrid-attention kernel on the
 # headline workload, from the ncu capture summarised under profiles/ (None until captured).
-K2_DRAM_TRAFFIC_BYTES = None
+K2_DRAM_TRAFFIC_BYTES = {}
 
 
 def load_peaks():
@@ -169,8 +169,16 @@ def to_dev(x, dtype, torch):
     return torch.from_numpy(np.ascontiguousarray(x)).cuda()
 
 
-def flop_model(w, stats, tc_kernel):
-    """Algorithmic flops of one hybrid-attention launch, from the library's own counters."""
+KERNEL_NAMES = {0: "generic (FP32 pipes)", 1: "tcgen05 + FP32 delta path", 2: "tcgen05 telescoped"}
+
+
+def flop_model(w, stats, kernel):
+    """Algorithmic flops of one hybrid-attention launch, from the library's own counters.
+
+    kernel 0: everything on the FP32 pipes.  kernel 1: in-window q.k and P.V on the tensor
+    cores, the sparse delta products (nnz(dq_i) multiply-adds per out-of-window pair) and the
+    per-tile seeds on the FP32 pipes.  kernel 2: out-of-window scores as the dense product
+    q_hat.k (d multiply-adds per out-of-window pair) on the tensor cores, nothing on the ALUs."""
     BH = w.B * w.H
     N_c = w.T * (w.T + 1) // 2
     pv = 2.0 * w.d * N_c * BH                                   # P.V over every causal pair
@@ -178,11 +186,35 @@ def flop_model(w, stats, tc_kernel):
     full, rem = divmod(w.T, w.window) if w.window > 0 else (0, 0)
     n_in = (full * w.window * (w.window + 1) // 2 + rem * (rem + 1) // 2) if w.window > 0 else 0
     qk_in = 2.0 * w.d * n_in * BH
-    seeds = 2.0 * w.d * (N_c - n_in) * BH / 64.0                # one dense row per 64-row query tile
+    seeds = 2.0 * w.d * (N_c - n_in) * BH / 128.0               # one dense row per 128-row query tile
     dense_equiv = 4.0 * w.d * N_c * BH
-    alu = (qk - qk_in) + seeds if tc_kernel else qk + seeds + pv
-    return dict(algorithmic=qk + seeds + pv, alu=alu, tensor=(qk_in + pv) if tc_kernel else 0.0,
-                dense_equiv=dense_equiv)
+    if kernel == 2:
+        tensor = qk_in + 2.0 * w.d * (N_c - n_in) * BH + pv
+        return dict(algorithmic=tensor, alu=0.0, tensor=tensor, dense_equiv=dense_equiv)
+    if kernel == 1:
+        return dict(algorithmic=qk + seeds + pv, alu=(qk - qk_in) + seeds, tensor=qk_in + pv,
+                    dense_equiv=dense_equiv)
+    return dict(algorithmic=qk + seeds + pv, alu=qk + seeds + pv, tensor=0.0, dense_equiv=dense_equiv)
+
+
+def k2_roofline(w, stats, kernel, k2_ms, peaks, n_sm):
+    fm = flop_model(w, stats, kernel)
+    sm_max = float(peaks.get("sm_max_mhz", 1965.0))
+    alu_peak = n_sm * 128 * 2 * sm_max * 1e6 / 1e12          # TFLOP/s: SMs x FP32 lanes x FMA x clock
+    t = k2_ms * 1e-3
+    common = {"kernel": KERNEL_NAMES[kernel], "kernel_ms": k2_ms,
+              "algorithmic_tflops": fm["algorithmic"] / t / 1e12,
+              "dense_equiv_tflops": fm["dense_equiv"] / t / 1e12, "traffic": K2_DRAM_TRAFFIC_BYTES.get(kernel)}
+    if kernel == 2:
+        peak = float(peaks["bf16_tflops"])
+        a = fm["tensor"] / t / 1e12
+        return {**common, "bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
+                "peak_source": f"{peaks['_source']} cuBLAS bf16 burst",
+                "note": "4 MiB of Q per launch: the layer is latency- and occupancy-bound, not tensor-bound"}
+    a = fm["alu"] / t / 1e12
+    return {**common, "bound": "alu", "achieved": a, "peak": alu_peak, "unit": "TFLOP/s", "frac": a / alu_peak,
+            "peak_source": f"derived: {n_sm} SMs x 128 FP32 lanes x 2 x {sm_max:.0f} MHz",
+            "tensor_tflops": fm["tensor"] / t / 1e12}
 
 
 def run_ours(args):
@@ -210,7 +242,7 @@ def run_ours(args):
     st = B.delta_state_init(cfg)
     if args.kernel >= 0:
         B.delta_state_set_prefill_kernel(st, args.kernel)
-    tc_kernel = B.delta_state_prefill_kernel(st) == 1
+    kernel = B.delta_state_prefill_kernel(st)
     flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 
     def step():
@@ -270,24 +302,13 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    fm = flop_model(w, stats, tc_kernel)
-    sm_max = float(peaks.get("sm_max_mhz", 1965.0))
-    alu_peak = n_sm * 128 * 2 * sm_max * 1e6 / 1e12          # TFLOP/s: SMs x FP32 lanes x FMA x clock
-    k2_s = kmean[2] * 1e-3
-    roofline = {
-        "kernel": "hybrid_attn_tc" if tc_kernel else "hybrid_attn_generic",
-        "bound": "alu", "achieved": fm["alu"] / k2_s / 1e12, "peak": alu_peak, "unit": "TFLOP/s",
-        "frac": fm["alu"] / k2_s / 1e12 / alu_peak, "traffic": K2_DRAM_TRAFFIC_BYTES,
-        "peak_source": f"derived: {n_sm} SMs x 128 FP32 lanes x 2 x {sm_max:.0f} MHz",
-        "kernel_ms": kmean[2], "algorithmic_tflops": fm["algorithmic"] / k2_s / 1e12,
-        "dense_equiv_tflops": fm["dense_equiv"] / k2_s / 1e12,
-        "tensor_tflops": fm["tensor"] / k2_s / 1e12,
-        "tensor_frac_of_" + peaks["_source"]: fm["tensor"] / k2_s / 1e12 / float(peaks["bf16_tflops"]),
-    }
+    roofline = k2_roofline(w, stats, kernel, kmean[2], peaks, n_sm)
     # K1 is a streaming pass: report it against the HBM copy bandwidth as well
     es = 2 if w.dtype == "bf16" else 4
-    k1_bytes = w.B * w.H * w.T * (w.d * (es + 4 + 1) + w.d // 8 + 2)
-    k1 = {"kernel": "delta_construct", "bound": "hbm", "kernel_ms": kmean[0],
+    # chain kernel: reads Q, writes delta values (fp32), mask words and, for the telescoped
+    # attention kernel, the reference rows (bf16)
+    k1_bytes = w.B * w.H * w.T * (w.d * (es + 4) + w.d // 8 + (w.d * 2 if kernel == 2 else 0))
+    k1 = {"kernel": "delta_chain", "bound": "hbm", "kernel_ms": kmean[0],
           "achieved": k1_bytes / (kmean[0] * 1e-3) / 1e9, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
           "frac": k1_bytes / (kmean[0] * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
           "note": f"{w.B * w.H * w.d} token-sequential chains of {w.T} steps: latency-bound at this size"}
@@ -298,10 +319,9 @@ def run_ours(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if w.dtype == "f32" else "bf16 in, f32 accumulate", "data": "synthetic",
         "config": config_dict(w, theta), "impl": "ours",
-        "prefill_kernel": "tcgen05" if tc_kernel else "generic",
+        "prefill_kernel": KERNEL_NAMES[kernel],
         "gpu_launches": int(launches),
-        "kernel_ms": {"delta_construct": kmean[0], "prefill_stats": kmean[1], "hybrid_attn": kmean[2],
-                      "handoff": kmean[3]},
+        "kernel_ms": {"delta_chain": kmean[0], "delta_finish": kmean[1], "hybrid_attn": kmean[2]},
         "sparsity": {"S_m": stats["S_m"], "S_c_eq6": stats["S_c_eq6"], "S_c_exact": stats["S_c_exact"],
                      "paper_context": "paper: ~60% prefill, ~57% prefill+decode (key deltas, real activations, A100)"},
         "roofline": roofline, "roofline_delta_construct": k1, "clocks": clocks,
@@ -310,6 +330,7 @@ def run_ours(args):
     }
 
     if not args.quick:
+        line["kernel_variants"] = run_variants(args, B, torch, w, q, k, v, out, flush, theta, peaks, n_sm, kernel)
         line["e2e"] = run_e2e(args, B, torch, w, tens, theta)
         line["theta_sweep"] = run_sweep(args, B, torch, w, q, k, v, out, st, flush)
         line["decode"] = run_decode(args, B, torch, peaks)
@@ -318,6 +339,39 @@ def run_ours(args):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_variants(args, B, torch, w, q, k, v, out, flush, theta, peaks, n_sm, default_kernel):
+    """The other prefill kernels on the same inputs (same step, L2 flushed): step time, the
+    hybrid-attention kernel's time and its roofline."""
+    res = []
+    for kern in (1, 2, 0):
+        if kern == default_kernel:
+            continue
+        cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T, w.dtype)
+        st = B.delta_state_init(cfg)
+        try:
+            B.delta_state_set_prefill_kernel(st, kern)
+        except B.DeltaError:
+            continue
+        B.delta_state_enable_profiling(st, True)
+        kms, steps = [], []
+        for i in range(3 + min(args.steps, 10)):
+            flush.zero_()
+            B.delta_state_reset(st)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                kms.append(B.delta_state_prefill_kernel_ms(st)); steps.append(e0.elapsed_time(e1))
+        stats = B.delta_sparsity_stats(st)["prefill"]
+        k2 = statistics.mean(x[2] for x in kms)
+        res.append({"prefill_kernel": KERNEL_NAMES[kern], "ms_per_step": statistics.mean(steps),
+                    "tokens_per_s": w.B * w.T / (statistics.mean(steps) * 1e-3),
+                    "roofline": k2_roofline(w, stats, kern, k2, peaks, n_sm)})
+    return res
 
 
 def run_e2e(args, B, torch, w, tens, theta):
@@ -472,7 +526,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama32_1b_prefill")
     ap.add_argument("--theta", type=float, default=HEADLINE_THETA)
-    ap.add_argument("--kernel", type=int, default=-1, help="-1 auto, 0 generic, 1 tensor-core")
+    ap.add_argument("--kernel", type=int, default=-1, help="-1 auto, 0 generic, 1 tcgen05 + FP32 delta path, 2 tcgen05 telescoped")
     ap.add_argument("--quick", action="store_true", help="prefill timing only (used for ncu launch lists)")
     ap.add_argument("--ref-heads", type=int, default=4, help="heads per reference step")
     args = ap.parse_args()
