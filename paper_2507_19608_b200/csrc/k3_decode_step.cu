@@ -3,21 +3,27 @@
 // pass over the K and V cache plus a read-modify-write of the carried score row R.
 //
 // Grid = (key splits, batch x KV heads).  A CTA serves the G query heads that share one KV
-// head, so every cached key and value row is read once for the group.  It
-//   0. thresholds q_new against the carried reference (Eq. 2-3) for its G heads,
-//   1. streams its slice of the key cache: R[j] += dq . k_j (Eq. 4), exact q_new . k_j for the
-//      W_d most recent keys, and for the key that arrives now R[n] = q_hat . k_new; appends
-//      k_new / v_new to the cache,
-//   2. turns its slice of scores into un-normalised probabilities (slice max, sum),
-//   3. accumulates P.V over its slice of the value cache,
-//   4. stores (max, sum, partial output); the last CTA of a (batch, KV head) to finish merges
-//      the slices and writes the output rows.
+// head, so every cached key and value row is read once for the group, and walks its slice of
+// the cache in tiles of 16 KiB of keys (and as much of values).  Tiles are contiguous in the
+// cache, so one bulk asynchronous copy per tile and tensor brings them into a two-stage ring
+// in shared memory while the previous tile is processed; the R entries of the tile are
+// fetched with coalesced loads ahead of their use.  Per tile:
+//   1. dot products of every key with the G delta vectors (Eq. 4), with the G query vectors
+//      for the W_d most recent keys, and with the new references for the key that arrives now;
+//   2. R[j] += dq.k_j written back coalesced (R[n] = q_hat.k_new for the new key), the
+//      hybrid select, the scale;
+//   3. online softmax over the tile (one warp per head);
+//   4. P.V accumulated in registers.
+// In front of the tiles the CTA thresholds q_new against the carried reference (Eq. 2-3) for
+// its G heads; at the end it stores (max, sum, partial output) and the last CTA of a
+// (batch, KV head) to finish merges the slices and writes the output rows.
 #include "delta_internal.cuh"
 
 namespace delta {
 
 namespace {
 constexpr int DNT = 256, DNW = DNT / 32;
+constexpr int TILE_BYTES = 16384;      // bytes of keys (and of values) per tile
 
 __device__ __forceinline__ void load8(const float* p, float (&x)[8]) {
   const float4 a = *reinterpret_cast<const float4*>(p);
@@ -33,12 +39,34 @@ __device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&x)[8]) {
     x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
   }
 }
-__device__ __forceinline__ void copy8(float* dst, const float* src) {
-  *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(src);
-  *reinterpret_cast<float4*>(dst + 4) = *reinterpret_cast<const float4*>(src + 4);
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ void copy8(__nv_bfloat16* dst, const __nv_bfloat16* src) {
-  *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait (about a second of SM clock); false if it ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > 2000000000ll) return false;
+  }
+  return true;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
 }
 }  // namespace
 
@@ -52,14 +80,22 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
     float theta, int W, float scale_log2e) {
   constexpr int LPK = D / 8;     // lanes per key row (8 elements each)
   constexpr int KPW = 32 / LPK;  // key rows per warp iteration
-  extern __shared__ __align__(16) float dsm[];
-  float* q_s = dsm;              // [G][D]
+  constexpr int ROWB = D * (int)sizeof(TC);
+  constexpr int TK = TILE_BYTES / ROWB;              // keys per tile (128 for bf16 d=64)
+  constexpr int RPT = (G * TK + DNT - 1) / DNT;      // R entries per thread and tile
+  extern __shared__ __align__(128) unsigned char dsm_raw[];
+  TC* sK = reinterpret_cast<TC*>(dsm_raw);                         // [2][TK][D]
+  TC* sV = reinterpret_cast<TC*>(dsm_raw + 2 * TILE_BYTES);        // [2][TK][D]
+  float* q_s = reinterpret_cast<float*>(dsm_raw + 4 * TILE_BYTES); // [G][D]
   float* dq_s = q_s + G * D;     // [G][D]
   float* qh_s = dq_s + G * D;    // [G][D]
   float* red = qh_s + G * D;     // [DNW][G][D]
-  float* ml_s = red + DNW * G * D;  // [2][G]: slice max, slice sum
-  float* sc = ml_s + 2 * 8;      // [G][chunk]
-  __shared__ int s_last;
+  float* spd = red + DNW * G * D;  // [G][TK] delta dot products (new reference . k_new for the new key)
+  float* spq = spd + G * TK;     // [G][TK] exact dot products (window only)
+  float* sc = spq + G * TK;      // [G][TK] scaled scores, then probabilities
+  float* st_s = sc + G * TK;     // [3][8]: running max, running sum, rescale of this tile
+  __shared__ __align__(8) unsigned long long bars[2];
+  __shared__ int s_last, s_fail;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int split = blockIdx.x, bkv = blockIdx.y;
@@ -68,6 +104,36 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
   const int L = n + 1;  // keys after this step
   const int j0 = split * chunk;
   const int len = max(0, min(chunk, L - j0));
+  const int n_tiles = (len + TK - 1) / TK;
+  const TC* kc = k_cache + (size_t)bkv * T_max * D;
+  const TC* vc = v_cache + (size_t)bkv * T_max * D;
+  const uint32_t bar0 = smem_u32(&bars[0]);
+
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0), "r"(1) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8), "r"(1) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
+  }
+  if (tid < 8) { st_s[tid] = -INFINITY; st_s[8 + tid] = 0.0f; st_s[16 + tid] = 1.0f; }
+  __syncthreads();
+
+  // cached rows of tile t (the row that arrives with this step is not in the cache yet)
+  auto tile_cached_rows = [&](int t) { return max(0, min(min(TK, len - t * TK), n - (j0 + t * TK))); };
+  auto issue_tile = [&](int t) {
+    const int rows = tile_cached_rows(t);
+    const uint32_t bar = bar0 + 8 * (t & 1);
+    const uint32_t bytes = (uint32_t)rows * ROWB;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * bytes) : "memory");
+    if (bytes) {
+      bulk_load(smem_u32(sK) + (t & 1) * TILE_BYTES, kc + (size_t)(j0 + t * TK) * D, bytes, bar);
+      bulk_load(smem_u32(sV) + (t & 1) * TILE_BYTES, vc + (size_t)(j0 + t * TK) * D, bytes, bar);
+    }
+  };
+  if (tid == 0) {
+    if (n_tiles > 0) issue_tile(0);
+    if (n_tiles > 1) issue_tile(1);
+  }
 
   // ---- 0. delta of the new query rows against the carried reference (Eq. 2-3)
   int fired_total = 0;
@@ -101,101 +167,150 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
 
   const int sub = lane / LPK;       // which key row of the warp iteration
   const int c0 = (lane % LPK) * 8;  // first of this lane's 8 channels
-  const TC* kc = k_cache + (size_t)bkv * T_max * D;
-  const TC* vc = v_cache + (size_t)bkv * T_max * D;
-
-  // ---- 1. scores of this slice
-  for (int jb = warp * KPW; jb < len; jb += DNW * KPW) {
-    const int jj = jb + sub;
-    const int j = j0 + jj;
-    const bool valid = jj < len;
-    const bool is_new = valid && (j == n);
-    const bool warp_has_new = (j0 + jb <= n) && (n < j0 + jb + KPW);
-    const bool warp_in_win = (n - (j0 + jb + KPW - 1)) < W;  // some row of this iteration is exact
-    float kv[8];
-    if (valid) {
-      const TC* src = is_new ? (k_new + (size_t)bkv * D + c0) : (kc + (size_t)j * D + c0);
-      load8(src, kv);
-      if (is_new) copy8(k_cache + ((size_t)bkv * T_max + n) * D + c0, src);
-    } else {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) kv[e] = 0.0f;
-    }
-#pragma unroll
-    for (int hh = 0; hh < G; ++hh) {
-      float pd = 0.0f, pq = 0.0f, pr = 0.0f;
-      const float* dqh = dq_s + hh * D + c0;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) pd = fmaf(dqh[e], kv[e], pd);
-      if (warp_in_win) {
-        const float* qh = q_s + hh * D + c0;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) pq = fmaf(qh[e], kv[e], pq);
-      }
-      if (warp_has_new) {
-        const float* rh = qh_s + hh * D + c0;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) pr = fmaf(rh[e], kv[e], pr);
-      }
-#pragma unroll
-      for (int o = LPK / 2; o > 0; o >>= 1) {
-        pd += __shfl_xor_sync(0xffffffffu, pd, o);
-        if (warp_in_win) pq += __shfl_xor_sync(0xffffffffu, pq, o);
-        if (warp_has_new) pr += __shfl_xor_sync(0xffffffffu, pr, o);
-      }
-      if (valid && (lane % LPK) == 0) {
-        float* Rp = R + ((size_t)b * H + kvh * G + hh) * T_max + j;
-        const float Rn = is_new ? pr : (*Rp + pd);
-        *Rp = Rn;
-        const float s = (n - j < W) ? pq : Rn;
-        sc[hh * chunk + jj] = s * scale_log2e;
-      }
-    }
-  }
-  __syncthreads();
-
-  // ---- 2. slice max and un-normalised probabilities (warp hh serves head hh)
-  if (warp < G) {
-    float* s = sc + warp * chunk;
-    float mx = -INFINITY;
-    for (int jj = lane; jj < len; jj += 32) mx = fmaxf(mx, s[jj]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float sum = 0.0f;
-    for (int jj = lane; jj < len; jj += 32) {
-      const float p = exp2f(s[jj] - mx);
-      s[jj] = p;
-      sum += p;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (lane == 0) { ml_s[warp] = mx; ml_s[8 + warp] = sum; }
-  }
-  __syncthreads();
-
-  // ---- 3. partial P.V over this slice
   float acc[G][8];
 #pragma unroll
   for (int hh = 0; hh < G; ++hh)
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[hh][e] = 0.0f;
-  for (int jb = warp * KPW; jb < len; jb += DNW * KPW) {
-    const int jj = jb + sub;
-    const int j = j0 + jj;
-    if (jj < len) {
-      const bool is_new = (j == n);
-      const TC* src = is_new ? (v_new + (size_t)bkv * D + c0) : (vc + (size_t)j * D + c0);
-      float vv[8];
-      load8(src, vv);
-      if (is_new) copy8(v_cache + ((size_t)bkv * T_max + n) * D + c0, src);
+  float* Rg = R + ((size_t)b * H + kvh * G) * T_max;   // R rows of the group's heads
+
+  for (int t = 0; t < n_tiles; ++t) {
+    const int tj0 = j0 + t * TK;
+    const int rows = min(TK, len - t * TK);           // keys of this tile, the new one included
+    const TC* kt = sK + (size_t)(t & 1) * TK * D;
+    const TC* vt = sV + (size_t)(t & 1) * TK * D;
+    const bool has_new = (n >= tj0) && (n < tj0 + rows);
+    const bool any_win = (n - (tj0 + rows - 1)) < W;   // some key of the tile is inside the window
+
+    // R entries of the tile: coalesced, in flight while the tile's copies land
+    float r_old[RPT];
+#pragma unroll
+    for (int u = 0; u < RPT; ++u) {
+      const int idx = tid + u * DNT;
+      const int hh = idx / TK, jj = idx - hh * TK;
+      r_old[u] = (hh < G && jj < rows && tj0 + jj < n) ? Rg[(size_t)hh * T_max + tj0 + jj] : 0.0f;
+    }
+    if (!mbar_wait(bar0 + 8 * (t & 1), (t >> 1) & 1)) s_fail = 1;
+    if (has_new) {
+      // the key and value that arrive with this step: into the tile and into the cache
+      const int jn = n - tj0;
+      for (int e = tid; e < D; e += DNT) {
+        const TC kv = k_new[(size_t)bkv * D + e], vv = v_new[(size_t)bkv * D + e];
+        const_cast<TC*>(kt)[jn * D + e] = kv;
+        const_cast<TC*>(vt)[jn * D + e] = vv;
+        k_cache[((size_t)bkv * T_max + n) * D + e] = kv;
+        v_cache[((size_t)bkv * T_max + n) * D + e] = vv;
+      }
+      __syncthreads();
+    }
+
+    // ---- 1. dot products of this tile
+    for (int jb = warp * KPW; jb < rows; jb += DNW * KPW) {
+      const int jj = jb + sub;
+      const bool valid = jj < rows;
+      const bool warp_has_new = has_new && (tj0 + jb <= n) && (n < tj0 + jb + KPW);
+      const bool warp_in_win = any_win && (n - (tj0 + jb + KPW - 1)) < W;
+      float kv[8];
+      if (valid) load8(kt + (size_t)jj * D + c0, kv);
+      else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) kv[e] = 0.0f;
+      }
 #pragma unroll
       for (int hh = 0; hh < G; ++hh) {
-        const float p = sc[hh * chunk + jj];
+        float pd = 0.0f, pq = 0.0f, pr = 0.0f;
+        const float* dqh = dq_s + hh * D + c0;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[hh][e] = fmaf(p, vv[e], acc[hh][e]);
+        for (int e = 0; e < 8; ++e) pd = fmaf(dqh[e], kv[e], pd);
+        if (warp_in_win) {
+          const float* qh = q_s + hh * D + c0;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) pq = fmaf(qh[e], kv[e], pq);
+        }
+        if (warp_has_new) {
+          const float* rh = qh_s + hh * D + c0;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) pr = fmaf(rh[e], kv[e], pr);
+        }
+#pragma unroll
+        for (int o = LPK / 2; o > 0; o >>= 1) {
+          pd += __shfl_xor_sync(0xffffffffu, pd, o);
+          if (warp_in_win) pq += __shfl_xor_sync(0xffffffffu, pq, o);
+          if (warp_has_new) pr += __shfl_xor_sync(0xffffffffu, pr, o);
+        }
+        if (valid && (lane % LPK) == 0) {
+          spd[hh * TK + jj] = (tj0 + jj == n) ? pr : pd;
+          spq[hh * TK + jj] = pq;
+        }
       }
     }
+    __syncthreads();
+
+    // ---- 2. R update (coalesced), hybrid select, scale
+#pragma unroll
+    for (int u = 0; u < RPT; ++u) {
+      const int idx = tid + u * DNT;
+      const int hh = idx / TK, jj = idx - hh * TK;
+      if (hh < G && jj < rows) {
+        const int j = tj0 + jj;
+        const float Rn = r_old[u] + spd[idx];       // r_old is 0 for the key that arrives now
+        Rg[(size_t)hh * T_max + j] = Rn;
+        sc[idx] = ((n - j < W) ? spq[idx] : Rn) * scale_log2e;
+      }
+    }
+    __syncthreads();
+
+    // ---- 3. online softmax over the tile (warp hh serves head hh)
+    if (warp < G) {
+      float* s = sc + warp * TK;
+      float mx = -INFINITY;
+      for (int jj = lane; jj < rows; jj += 32) mx = fmaxf(mx, s[jj]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float m_old = st_s[warp];
+      const float m_new = fmaxf(m_old, mx);
+      float sum = 0.0f;
+      for (int jj = lane; jj < rows; jj += 32) {
+        const float p = exp2f(s[jj] - m_new);
+        s[jj] = p;
+        sum += p;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (lane == 0) {
+        const float al = exp2f(m_old - m_new);
+        st_s[warp] = m_new;
+        st_s[8 + warp] = fmaf(st_s[8 + warp], al, sum);
+        st_s[16 + warp] = al;
+      }
+    }
+    __syncthreads();
+
+    // ---- 4. P.V over the tile
+#pragma unroll
+    for (int hh = 0; hh < G; ++hh) {
+      const float al = st_s[16 + hh];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[hh][e] *= al;
+    }
+    for (int jb = warp * KPW; jb < rows; jb += DNW * KPW) {
+      const int jj = jb + sub;
+      if (jj < rows) {
+        float vv[8];
+        load8(vt + (size_t)jj * D + c0, vv);
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh) {
+          const float p = sc[hh * TK + jj];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[hh][e] = fmaf(p, vv[e], acc[hh][e]);
+        }
+      }
+    }
+    __syncthreads();   // the tile's buffers and score arrays are free
+    if (tid == 0 && t + 2 < n_tiles) issue_tile(t + 2);
   }
+
+  // ---- reduce the partial outputs over key lanes and warps
 #pragma unroll
   for (int hh = 0; hh < G; ++hh)
 #pragma unroll
@@ -213,7 +328,7 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
   }
   __syncthreads();
 
-  // ---- 4. store the slice result; the last slice to arrive merges all of them
+  // ---- store the slice result; the last slice to arrive merges all of them
   float* part = partial + ((size_t)bkv * kMaxDecodeSplits + split) * G * (D + 2);
   for (int e = tid; e < G * D; e += DNT) {
     float x = 0.0f;
@@ -223,14 +338,15 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
     part[hh * (D + 2) + c] = x;
   }
   if (tid < G) {
-    part[tid * (D + 2) + D] = ml_s[tid];
-    part[tid * (D + 2) + D + 1] = ml_s[8 + tid];
+    part[tid * (D + 2) + D] = st_s[tid];
+    part[tid * (D + 2) + D + 1] = st_s[8 + tid];
   }
+  if (tid == 0 && s_fail) atomicMax(&counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
   __threadfence();
   __syncthreads();
   if (tid == 0) {
-    const uint32_t t = atomicAdd(&ticket[bkv], 1u);
-    s_last = (t == (uint32_t)nsplit - 1u);
+    const uint32_t tk = atomicAdd(&ticket[bkv], 1u);
+    s_last = (tk == (uint32_t)nsplit - 1u);
   }
   __syncthreads();
   if (!s_last) return;
@@ -259,31 +375,29 @@ cudaError_t launch_decode_step(const Shape& s, const Workspace& w, const void* q
                                cudaStream_t st) {
   const int L = n + 1;
   const int bkv = s.B * s.H_kv;
-  int nsplit = (296 + bkv - 1) / bkv;
+  const int es = dtype == DELTA_F32 ? 4 : 2;
+  const int TK = TILE_BYTES / (s.d * es);
+  // one wave of two CTAs per SM (the ring holds 64 KiB), no slice shorter than a quarter tile
+  int nsplit = 296 / bkv;
   if (nsplit > kMaxDecodeSplits) nsplit = kMaxDecodeSplits;
-  const int max_by_len = (L + 31) / 32;
+  const int max_by_len = (L + TK / 4 - 1) / (TK / 4);
   if (nsplit > max_by_len) nsplit = max_by_len;
   if (nsplit < 1) nsplit = 1;
   int chunk = (L + nsplit - 1) / nsplit;
   chunk = (chunk + 31) / 32 * 32;
-  if (chunk > kDecodeChunkMax) {
-    chunk = kDecodeChunkMax;
-    nsplit = (L + chunk - 1) / chunk;
-    if (nsplit > kMaxDecodeSplits) return cudaErrorInvalidValue;
-  }
   nsplit = (L + chunk - 1) / chunk;
+  if (nsplit > kMaxDecodeSplits) return cudaErrorInvalidValue;
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const int G = s.g();
   const dim3 grid(nsplit, bkv);
-  const size_t smem = ((size_t)3 * G * s.d + (size_t)DNW * G * s.d + 16 + (size_t)G * chunk) * 4;
+  const size_t smem = (size_t)4 * TILE_BYTES +
+                      ((size_t)3 * G * s.d + (size_t)DNW * G * s.d + (size_t)3 * G * TK + 24) * 4;
   cudaError_t err = cudaSuccess;
 #define LAUNCH(TC, DD, GG)                                                                       \
   do {                                                                                           \
     auto kern = decode_step_kernel<TC, DD, GG>;                                                  \
-    if (smem > 48 * 1024) {                                                                      \
-      err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-      if (err != cudaSuccess) return err;                                                        \
-    }                                                                                            \
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
+    if (err != cudaSuccess) return err;                                                          \
     kern<<<grid, DNT, smem, st>>>((const TC*)q_new, (const TC*)k_new, (const TC*)v_new,          \
                                   (TC*)k_cache, (TC*)v_cache, (TC*)out, w.qhat[qhat_sel],        \
                                   w.qhat[qhat_sel ^ 1], w.R, w.dec_partial, w.dec_ticket,        \
