@@ -167,11 +167,11 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
 
   const int sub = lane / LPK;       // which key row of the warp iteration
   const int c0 = (lane % LPK) * 8;  // first of this lane's 8 channels
-  float acc[G][8];
+  float acc[G][8], dqr[G][8];   // partial outputs; this lane's 8 channels of the G delta vectors
 #pragma unroll
   for (int hh = 0; hh < G; ++hh)
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[hh][e] = 0.0f;
+    for (int e = 0; e < 8; ++e) { acc[hh][e] = 0.0f; dqr[hh][e] = dq_s[hh * D + c0 + e]; }
   float* Rg = R + ((size_t)b * H + kvh * G) * T_max;   // R rows of the group's heads
 
   for (int t = 0; t < n_tiles; ++t) {
@@ -216,31 +216,53 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
 #pragma unroll
         for (int e = 0; e < 8; ++e) kv[e] = 0.0f;
       }
+      float pd[G];
 #pragma unroll
       for (int hh = 0; hh < G; ++hh) {
-        float pd = 0.0f, pq = 0.0f, pr = 0.0f;
-        const float* dqh = dq_s + hh * D + c0;
+        pd[hh] = 0.0f;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) pd = fmaf(dqh[e], kv[e], pd);
-        if (warp_in_win) {
-          const float* qh = q_s + hh * D + c0;
+        for (int e = 0; e < 8; ++e) pd[hh] = fmaf(dqr[hh][e], kv[e], pd[hh]);
+      }
+      if constexpr (G == 4) {
+        // four heads reduced over the key's lanes together: the value set halves as the lane
+        // distance halves; lane (l & 6) of the key group ends with head ((l >> 2) & 1) * 2 + ((l >> 1) & 1)
+        const int kl = lane % LPK;
+        if constexpr (LPK == 16) {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) pq = fmaf(qh[e], kv[e], pq);
+          for (int hh = 0; hh < G; ++hh) pd[hh] += __shfl_xor_sync(0xffffffffu, pd[hh], 8);
         }
-        if (warp_has_new) {
+        const bool h4 = kl & 4, h2 = kl & 2;
+        const float a0 = (h4 ? pd[2] : pd[0]) + __shfl_xor_sync(0xffffffffu, h4 ? pd[0] : pd[2], 4);
+        const float a1 = (h4 ? pd[3] : pd[1]) + __shfl_xor_sync(0xffffffffu, h4 ? pd[1] : pd[3], 4);
+        float z = (h2 ? a1 : a0) + __shfl_xor_sync(0xffffffffu, h2 ? a0 : a1, 2);
+        z += __shfl_xor_sync(0xffffffffu, z, 1);
+        if (valid && (kl & 1) == 0 && kl < 8) spd[((h4 ? 2 : 0) + (h2 ? 1 : 0)) * TK + jj] = z;
+      } else {
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh) {
+#pragma unroll
+          for (int o = LPK / 2; o > 0; o >>= 1) pd[hh] += __shfl_xor_sync(0xffffffffu, pd[hh], o);
+          if (valid && (lane % LPK) == 0) spd[hh * TK + jj] = pd[hh];
+        }
+      }
+      // rare paths: exact scores of the W_d most recent keys, new reference . new key
+      if (warp_in_win || warp_has_new) {
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh) {
+          float pq = 0.0f, pr = 0.0f;
+          const float* qh = q_s + hh * D + c0;
           const float* rh = qh_s + hh * D + c0;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) pr = fmaf(rh[e], kv[e], pr);
-        }
+          for (int e = 0; e < 8; ++e) { pq = fmaf(qh[e], kv[e], pq); pr = fmaf(rh[e], kv[e], pr); }
 #pragma unroll
-        for (int o = LPK / 2; o > 0; o >>= 1) {
-          pd += __shfl_xor_sync(0xffffffffu, pd, o);
-          if (warp_in_win) pq += __shfl_xor_sync(0xffffffffu, pq, o);
-          if (warp_has_new) pr += __shfl_xor_sync(0xffffffffu, pr, o);
-        }
-        if (valid && (lane % LPK) == 0) {
-          spd[hh * TK + jj] = (tj0 + jj == n) ? pr : pd;
-          spq[hh * TK + jj] = pq;
+          for (int o = LPK / 2; o > 0; o >>= 1) {
+            pq += __shfl_xor_sync(0xffffffffu, pq, o);
+            pr += __shfl_xor_sync(0xffffffffu, pr, o);
+          }
+          if (valid && (lane % LPK) == 0) {
+            spq[hh * TK + jj] = pq;
+            if (tj0 + jj == n) spd[hh * TK + jj] = pr;
+          }
         }
       }
     }
@@ -351,20 +373,45 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
   __syncthreads();
   if (!s_last) return;
   __threadfence();
+  // merge: weights of all (head, slice) pairs first (loads in parallel), then the outputs
   const float* pbase = partial + (size_t)bkv * kMaxDecodeSplits * G * (D + 2);
+  float* wgt_s = spd;            // [G][kMaxDecodeSplits] (the score arrays are free by now)
+  float* den_s = st_s;           // [G] (running max / sum are already in the partials)
+  for (int e = tid; e < G * kMaxDecodeSplits; e += DNT) {
+    const int hh = e / kMaxDecodeSplits, s2 = e - hh * kMaxDecodeSplits;
+    wgt_s[e] = (s2 < nsplit) ? __ldcg(pbase + ((size_t)s2 * G + hh) * (D + 2) + D) : -INFINITY;
+  }
+  __syncthreads();
+  if (warp < G) {
+    float m0 = wgt_s[warp * kMaxDecodeSplits + lane], m1 = wgt_s[warp * kMaxDecodeSplits + 32 + lane];
+    float M = fmaxf(m0, m1);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    const float w0 = exp2f(m0 - M), w1 = exp2f(m1 - M);   // slices that do not exist weigh 0
+    float den = 0.0f;
+    if (lane < nsplit) den = w0 * __ldcg(pbase + ((size_t)lane * G + warp) * (D + 2) + D + 1);
+    if (lane + 32 < nsplit) den = fmaf(w1, __ldcg(pbase + ((size_t)(lane + 32) * G + warp) * (D + 2) + D + 1), den);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    wgt_s[warp * kMaxDecodeSplits + lane] = w0;
+    wgt_s[warp * kMaxDecodeSplits + 32 + lane] = w1;
+    if (lane == 0) den_s[warp] = den;
+  }
+  __syncthreads();
   for (int e = tid; e < G * D; e += DNT) {
     const int hh = e / D, c = e - hh * D;
-    float M = -INFINITY;
-    for (int s2 = 0; s2 < nsplit; ++s2)
-      M = fmaxf(M, __ldcg(pbase + ((size_t)s2 * G + hh) * (D + 2) + D));
-    float num = 0.0f, den = 0.0f;
-    for (int s2 = 0; s2 < nsplit; ++s2) {
-      const float* pp = pbase + ((size_t)s2 * G + hh) * (D + 2);
-      const float wgt = exp2f(__ldcg(pp + D) - M);
-      num = fmaf(wgt, __ldcg(pp + c), num);
-      den = fmaf(wgt, __ldcg(pp + D + 1), den);
+    float num = 0.0f;
+    int s2 = 0;
+    for (; s2 + 4 <= nsplit; s2 += 4) {
+      float x[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) x[u] = __ldcg(pbase + ((size_t)(s2 + u) * G + hh) * (D + 2) + c);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) num = fmaf(wgt_s[hh * kMaxDecodeSplits + s2 + u], x[u], num);
     }
-    out[((size_t)b * H + kvh * G + hh) * D + c] = from_f32<TC>(num / den);
+    for (; s2 < nsplit; ++s2)
+      num = fmaf(wgt_s[hh * kMaxDecodeSplits + s2], __ldcg(pbase + ((size_t)s2 * G + hh) * (D + 2) + c), num);
+    out[((size_t)b * H + kvh * G + hh) * D + c] = from_f32<TC>(num / den_s[hh]);
   }
   if (tid == 0) ticket[bkv] = 0;  // ready for the next step
 }
