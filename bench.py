@@ -37,8 +37,9 @@ FLUSH_BYTES = 256 << 20       # > 126 MB of L2, written between timed iterations
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
                   "sm_max_mhz": 1965.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the hybrid-attention kernel on the
-# headline workload, from the ncu capture summarised under profiles/ (None until captured).
-K2_DRAM_TRAFFIC_BYTES = {}
+# headline workload, from the ncu captures summarised under profiles/ (absent = not captured
+# since the kernel last changed).
+K2_DRAM_TRAFFIC_BYTES = {2: 10526208, 1: 17161728}   # per kernel id
 
 
 def load_peaks():
