@@ -224,7 +224,7 @@ DELTA_API int32_t delta_state_position(const delta_state_t* st);
  *   1 = tcgen05/TMA kernel, out-of-window scores by Eq. 4's running sum of sparse delta
  *       products on the FP32 pipes, skipping all-zero delta blocks (bf16, d = 64);
  *   2 = tcgen05/TMA kernel, out-of-window scores by the telescoped form of Eq. 4,
- *       R(i)[j] = q_hat(i).k_j, as one more tensor-core product (bf16, d = 64).
+ *       R(i)[j] = q_hat(i).k_j, as one more tensor-core product (bf16, d = 64 or 128).
  * All three compute the same function.  delta_state_set_prefill_kernel forces one
  * (-1 = automatic); forcing a kernel the configuration has none for returns
  * DELTA_ERR_UNSUPPORTED. */

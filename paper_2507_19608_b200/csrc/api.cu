@@ -79,7 +79,7 @@ static void carve(const delta_config_t& c, char* base, Workspace* w) {
   w->qhat_tile_bf16 = (c.dtype == DELTA_BF16) ? (__nv_bfloat16*)take(BH * nt * c.d * 2) : nullptr;
   w->kt = (c.dtype == DELTA_BF16 && tc_kernel_shape(c.d))
               ? (float*)take(BKV * c.d * (((size_t)c.T_max + 3) / 4 * 4) * 4) : nullptr;
-  w->qhat_rows = (c.dtype == DELTA_BF16 && tc_kernel_shape(c.d))
+  w->qhat_rows = (c.dtype == DELTA_BF16 && tcq_kernel_shape(c.d))
                      ? (__nv_bfloat16*)take(BH * c.T_max * c.d * 2) : nullptr;
   w->total_bytes = off;
 }
@@ -177,19 +177,21 @@ delta_status_t delta_state_prefill_kernel_ms(delta_state_t* st, float* ms) {
 
 int32_t delta_state_position(const delta_state_t* st) { return st ? st->n : -1; }
 
-static bool tc_eligible(const delta_state* st) {
-  return st->cfg.dtype == DELTA_BF16 && tc_kernel_available(st->cfg.d);
+// Can prefill kernel `which` (1 or 2) serve this state?
+static bool tc_eligible(const delta_state* st, int which) {
+  if (st->cfg.dtype != DELTA_BF16 || !tc_kernel_available(64)) return false;
+  return which == 1 ? tc_kernel_shape(st->cfg.d) : tcq_kernel_shape(st->cfg.d);
 }
 
 int32_t delta_state_prefill_kernel(const delta_state_t* st) {
   if (!st) return -1;
   if (st->forced_kernel >= 0) return st->forced_kernel;
-  return tc_eligible(st) ? 2 : 0;   // the telescoped tensor-core kernel is the fastest where it applies
+  return tc_eligible(st, 2) ? 2 : 0;   // the telescoped tensor-core kernel is the fastest where it applies
 }
 
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
   if (!st || which < -1 || which > 2) return DELTA_ERR_INVALID_ARG;
-  if (which >= 1 && !tc_eligible(st)) return DELTA_ERR_UNSUPPORTED;
+  if (which >= 1 && !tc_eligible(st, which)) return DELTA_ERR_UNSUPPORTED;
   st->forced_kernel = which;
   return DELTA_OK;
 }

@@ -19,6 +19,8 @@
 // exponentiates, writes its 32 probabilities as bf16 into the operand layout of the P.V
 // product, and rescales/accumulates its 16 output columns from the previous tile's P.V.
 //
+// Head dimensions 64 and 128 (template parameter).
+//
 // Every wait on an mbarrier is bounded (see tc_common.cuh); after a time-out the protocol
 // still runs to its end, nothing is stored and the status word records DELTA_ERR_TIMEOUT.
 #include <cuda.h>
@@ -33,22 +35,30 @@ using namespace tc;
 namespace {
 
 constexpr int BM = 128, BN = 128, NCWARP = 16, NCTHR = NCWARP * 32, NTHR = NCTHR + 32;
-constexpr int TQ_D = 64;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TMEM_SH = 0;        // telescoped scores, two buffers of 128 columns
 constexpr uint32_t TMEM_SX = 256;      // exact scores, 128 columns
-constexpr uint32_t TMEM_O = 384;       // P.V tile, 64 columns
+constexpr uint32_t TMEM_O = 384;       // P.V tile, d columns (d <= 128)
+constexpr uint32_t SZ_BLK = 128 * 64 * 2;             // one [128 rows][64 elements] bf16 block, 16 KiB
 
-constexpr uint32_t SZ_TILE = 128 * 64 * 2;
-constexpr uint32_t OFF_Q = 0;
-constexpr uint32_t OFF_QH = OFF_Q + SZ_TILE;
-constexpr uint32_t OFF_K = OFF_QH + SZ_TILE;          // two buffers
-constexpr uint32_t OFF_V = OFF_K + 2 * SZ_TILE;       // two buffers
-constexpr uint32_t OFF_P = OFF_V + 2 * SZ_TILE;       // bf16 [2][128 rows][64 keys]
-constexpr uint32_t OFF_PMAX = OFF_P + 2 * SZ_TILE;    // fp32 [2][128 rows][4 quarters]
-constexpr uint32_t OFF_BAR = OFF_PMAX + 2 * 128 * 4 * 4;
-constexpr uint32_t OFF_MISC = OFF_BAR + 16 * 8;
-constexpr uint32_t SMEM_BYTES = OFF_MISC + 16 + 1024;
+// Shared-memory map for head dimension D.  Operand tiles are D/64 blocks of [128][64] bf16 in
+// the 128-byte-swizzle layout.  d = 64: keys double buffered; d = 128: one key buffer (the
+// next tile's keys are fetched as soon as this tile's score products are done).
+template <int D> struct TqSmem {
+  static constexpr uint32_t NKB = D / 64;                 // 64-element blocks per row
+  static constexpr uint32_t SZ_TILE = NKB * SZ_BLK;       // one [128][D] operand tile
+  static constexpr uint32_t NKBUF = (D == 64) ? 2 : 1;
+  static constexpr uint32_t OFF_Q = 0;
+  static constexpr uint32_t OFF_QH = OFF_Q + SZ_TILE;
+  static constexpr uint32_t OFF_K = OFF_QH + SZ_TILE;
+  static constexpr uint32_t OFF_V = OFF_K + NKBUF * SZ_TILE;   // two buffers
+  static constexpr uint32_t OFF_P = OFF_V + 2 * SZ_TILE;       // bf16 [2][128 rows][64 keys]
+  static constexpr uint32_t OFF_PMAX = OFF_P + 2 * SZ_BLK;     // fp32 [2][128 rows][4 quarters]
+  static constexpr uint32_t OFF_BAR = OFF_PMAX + 2 * 128 * 4 * 4;
+  static constexpr uint32_t OFF_MISC = OFF_BAR + 16 * 8;
+  static constexpr uint32_t BYTES = OFF_MISC + 16 + 1024;
+  static_assert(BYTES <= 227 * 1024, "shared memory budget");
+};
 
 enum Bar {
   BAR_Q = 0, BAR_K0, BAR_K1, BAR_V0, BAR_V1, BAR_S0, BAR_S1, BAR_O,   // one arrival (+ bytes)
@@ -66,6 +76,7 @@ struct TqParams {
 
 }  // namespace
 
+template <int D>
 __global__ void __launch_bounds__(NTHR, 1)
 hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qh,
                        const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -74,6 +85,10 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* sm = smem_raw + (base - raw);
+  using SM = TqSmem<D>;
+  constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKBUF = SM::NKBUF;
+  constexpr uint32_t OFF_Q = SM::OFF_Q, OFF_QH = SM::OFF_QH, OFF_K = SM::OFF_K, OFF_V = SM::OFF_V,
+                     OFF_P = SM::OFF_P, OFF_PMAX = SM::OFF_PMAX, OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC;
   float* sPmax = reinterpret_cast<float*>(sm + OFF_PMAX);
   volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
   volatile uint32_t* abort_flag = sMisc + 1;
@@ -118,33 +133,42 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // =========================== control warp ===============================================
     if (lane == 0) {
       const uint32_t IDESC_QK = make_idesc(BN, 0);
-      const uint32_t IDESC_PV = make_idesc(TQ_D, 1);
+      const uint32_t IDESC_PV = make_idesc(D, 1);
+      // one [128][D] tile = NKB boxes of [128][64]
+      auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row0, int outer) {
+#pragma unroll
+        for (uint32_t kb = 0; kb < NKB; ++kb) tma_load_3d(dst + kb * SZ_BLK, tm, bar, 64 * kb, row0, outer);
+      };
       mbar_expect_tx(BAR(BAR_Q), 2 * SZ_TILE);
-      tma_load_3d(base + OFF_Q, &tm_q, BAR(BAR_Q), 0, i0, bh);
-      tma_load_3d(base + OFF_QH, &tm_qh, BAR(BAR_Q), 0, i0, bh);
+      load_tile(base + OFF_Q, &tm_q, BAR(BAR_Q), i0, bh);
+      load_tile(base + OFF_QH, &tm_qh, BAR(BAR_Q), i0, bh);
       mbar_expect_tx(BAR(BAR_K0), SZ_TILE);
-      tma_load_3d(base + OFF_K, &tm_k, BAR(BAR_K0), 0, 0, bkv);
+      load_tile(base + OFF_K, &tm_k, BAR(BAR_K0), 0, bkv);
       mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
-      tma_load_3d(base + OFF_V, &tm_v, BAR(BAR_V0), 0, 0, bkv);
-      if (qt >= 1) {
+      load_tile(base + OFF_V, &tm_v, BAR(BAR_V0), 0, bkv);
+      if (NKBUF == 2 && qt >= 1) {
         mbar_expect_tx(BAR(BAR_K1), SZ_TILE);
-        tma_load_3d(base + OFF_K + SZ_TILE, &tm_k, BAR(BAR_K1), 0, BN, bkv);
+        load_tile(base + OFF_K + SZ_TILE, &tm_k, BAR(BAR_K1), BN, bkv);
       }
+      // key buffer and barrier parity of tile t
+      auto kbuf = [&](int t) { return NKBUF == 2 ? (t & 1) : 0; };
+      auto kpar = [&](int t) { return NKBUF == 2 ? ((t >> 1) & 1) : (t & 1); };
       // scores of tile t: Q_hat.K^T into buffer t&1, plus Q.K^T if the tile touches the window
       auto issue_scores = [&](int t) {
         const int bf = t & 1;
-        mbar_wait(BAR(BAR_K0 + bf), (t >> 1) & 1, abort_flag);
+        mbar_wait(BAR(BAR_K0 + kbuf(t)), kpar(t), abort_flag);
         tc_fence_after();
-        const uint32_t kb = base + OFF_K + bf * SZ_TILE;
+        const uint32_t kb = base + OFF_K + kbuf(t) * SZ_TILE;
 #pragma unroll
-        for (int ks = 0; ks < TQ_D / 16; ++ks)
-          tc_mma(tmem + TMEM_SH + bf * 128, make_desc(base + OFF_QH + ks * 32, 16, 1024),
-                 make_desc(kb + ks * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc_mma(tmem + TMEM_SH + bf * 128,
+                 make_desc(base + OFF_QH + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
+                 make_desc(kb + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
         if (tile_needs_exact(t)) {
 #pragma unroll
-          for (int ks = 0; ks < TQ_D / 16; ++ks)
-            tc_mma(tmem + TMEM_SX, make_desc(base + OFF_Q + ks * 32, 16, 1024),
-                   make_desc(kb + ks * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc_mma(tmem + TMEM_SX, make_desc(base + OFF_Q + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
+                   make_desc(kb + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
         }
         tc_commit(BAR(BAR_S0 + bf));
       };
@@ -154,21 +178,22 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const bool more = t < qt;
         const int nb = (t + 1) & 1;
         const bool next_exact = more && tile_needs_exact(t + 1);
+        // the key buffer of tile t is free once its score products are done: refill it
+        mbar_wait(BAR(BAR_S0 + (t & 1)), (t >> 1) & 1, abort_flag);
+        const int tn = t + (int)NKBUF;         // the tile that takes this buffer next
+        if (tn <= qt) {
+          mbar_expect_tx(BAR(BAR_K0 + kbuf(tn)), SZ_TILE);
+          load_tile(base + OFF_K + kbuf(tn) * SZ_TILE, &tm_k, BAR(BAR_K0 + kbuf(tn)), tn * BN, bkv);
+        }
         // next tile's scores one tile ahead, unless it needs the single exact-score buffer
         if (more && !next_exact) {
           if (t >= 1) mbar_wait(BAR(BAR_SFREE0 + nb), ((t - 1) >> 1) & 1, abort_flag);
           issue_scores(t + 1);
         }
-        // key buffer t&1 is free once the scores of tile t are done: stream tile t+2 into it
-        mbar_wait(BAR(BAR_S0 + (t & 1)), (t >> 1) & 1, abort_flag);
-        if (t + 2 <= qt) {
-          mbar_expect_tx(BAR(BAR_K0 + (t & 1)), SZ_TILE);
-          tma_load_3d(base + OFF_K + (t & 1) * SZ_TILE, &tm_k, BAR(BAR_K0 + (t & 1)), 0, (t + 2) * BN, bkv);
-        }
         if (t >= 1) mbar_wait(BAR(BAR_O), (t - 1) & 1, abort_flag);   // P.V(t-1) done: its V buffer is free
         if (more) {
           mbar_expect_tx(BAR(BAR_V0 + nb), SZ_TILE);
-          tma_load_3d(base + OFF_V + nb * SZ_TILE, &tm_v, BAR(BAR_V0 + nb), 0, (t + 1) * BN, bkv);
+          load_tile(base + OFF_V + nb * SZ_TILE, &tm_v, BAR(BAR_V0 + nb), (t + 1) * BN, bkv);
         }
         // P.V of this tile
         mbar_wait(BAR(BAR_P), t & 1, abort_flag);
@@ -177,8 +202,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const uint32_t vbase = base + OFF_V + (t & 1) * SZ_TILE;
 #pragma unroll
         for (int ks = 0; ks < BN / 16; ++ks)
-          tc_mma(tmem + TMEM_O, make_desc(base + OFF_P + (ks >> 2) * SZ_TILE + (ks & 3) * 32, 16, 1024),
-                 make_desc(vbase + ks * 2048, SZ_TILE, 1024), IDESC_PV, ks > 0 ? 1u : 0u);
+          tc_mma(tmem + TMEM_O, make_desc(base + OFF_P + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
+                 make_desc(vbase + ks * 2048, SZ_BLK, 1024), IDESC_PV, ks > 0 ? 1u : 0u);
         tc_commit(BAR(BAR_O));
         if (next_exact) {
           // every compute warp has read tile t's scores (it wrote P after that)
@@ -196,9 +221,10 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int i = i0 + row;
     const uint32_t lane_sel = (uint32_t)(32 * qd) << 16;
     const float scale = p.scale_log2e;
-    float O[16];
+    constexpr int OC = D / 4;      // output columns per thread (a quarter of the head dimension)
+    float O[OC];
 #pragma unroll
-    for (int c = 0; c < 16; ++c) O[c] = 0.0f;
+    for (int c = 0; c < OC; ++c) O[c] = 0.0f;
     float m_run = -INFINITY, l_part = 0.0f, alpha_prev = 1.0f;
     int wlo = 0, whi = 0;       // exact keys of row i: wlo <= j < whi
     if (W > 0) {
@@ -264,21 +290,12 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
       l_part = fmaf(l_part, al, sum);
 
-      // previous tile's P.V: rescale and accumulate; after it the P buffer may be rewritten
-      if (jt > 0) {
-        mbar_wait(BAR(BAR_O), (jt - 1) & 1, abort_flag);
-        tc_fence_after();
-        float v[16];
-        tc_ld16(tmem + TMEM_O + 16 * sub + lane_sel, v);
-#pragma unroll
-        for (int c = 0; c < 16; ++c) O[c] = fmaf(O[c], alpha_prev, v[c]);
-        tc_fence_before();
-      }
-      alpha_prev = al;
+      // the previous tile's P.V is done: the P buffer may be rewritten
+      if (jt > 0) mbar_wait(BAR(BAR_O), (jt - 1) & 1, abort_flag);
 
       // P as bf16 in the operand layout: this thread's 32 keys are 4 chunks of 16 bytes
       {
-        unsigned char* prow = sm + OFF_P + (size_t)(sub >> 1) * SZ_TILE + (size_t)row * 128;
+        unsigned char* prow = sm + OFF_P + (size_t)(sub >> 1) * SZ_BLK + (size_t)row * 128;
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4) {
           uint32_t w[4];
@@ -291,6 +308,20 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
+      // previous tile's P.V: rescale and accumulate (its tensor-memory tile is rewritten by
+      // this tile's product, which is issued only after every warp has arrived below)
+      if (jt > 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int h16 = 0; h16 < OC / 16; ++h16) {
+          float v[16];
+          tc_ld16(tmem + TMEM_O + OC * sub + 16 * h16 + lane_sel, v);
+#pragma unroll
+          for (int c = 0; c < 16; ++c) O[16 * h16 + c] = fmaf(O[16 * h16 + c], alpha_prev, v[c]);
+        }
+        tc_fence_before();
+      }
+      alpha_prev = al;
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(BAR_P));
@@ -299,23 +330,28 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // ---- last tile's P.V, row sum over the four quarters, normalisation, store
     mbar_wait(BAR(BAR_O), qt & 1, abort_flag);
     tc_fence_after();
-    float v[16];
-    tc_ld16(tmem + TMEM_O + 16 * sub + lane_sel, v);
     sPmax[(((qt + 1) & 1) * BM + row) * 4 + sub] = l_part;
     asm volatile("bar.sync %0, 128;" ::"r"(1 + qd) : "memory");
     const float4 lp = *reinterpret_cast<const float4*>(sPmax + (((qt + 1) & 1) * BM + row) * 4);
     const float inv = 1.0f / ((lp.x + lp.y) + (lp.z + lp.w));
-    if (i < T && !*abort_flag) {
-      uint32_t w[8];
+    const bool store = (i < T) && !*abort_flag;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const __nv_bfloat162 t2 = __floats2bfloat162_rn(fmaf(O[2 * c], alpha_prev, v[2 * c]) * inv,
-                                                        fmaf(O[2 * c + 1], alpha_prev, v[2 * c + 1]) * inv);
-        w[c] = *reinterpret_cast<const uint32_t*>(&t2);
+    for (int h16 = 0; h16 < OC / 16; ++h16) {
+      float v[16];
+      tc_ld16(tmem + TMEM_O + OC * sub + 16 * h16 + lane_sel, v);
+      if (store) {
+        uint32_t w[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const __nv_bfloat162 t2 = __floats2bfloat162_rn(
+              fmaf(O[16 * h16 + 2 * c], alpha_prev, v[2 * c]) * inv,
+              fmaf(O[16 * h16 + 2 * c + 1], alpha_prev, v[2 * c + 1]) * inv);
+          w[c] = *reinterpret_cast<const uint32_t*>(&t2);
+        }
+        uint4* op = reinterpret_cast<uint4*>(p.out + ((size_t)bh * T + i) * D + OC * sub + 16 * h16);
+        op[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        op[1] = make_uint4(w[4], w[5], w[6], w[7]);
       }
-      uint4* op = reinterpret_cast<uint4*>(p.out + ((size_t)bh * T + i) * TQ_D + 16 * sub);
-      op[0] = make_uint4(w[0], w[1], w[2], w[3]);
-      op[1] = make_uint4(w[4], w[5], w[6], w[7]);
     }
     tc_fence_before();
   }
@@ -330,24 +366,23 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #undef BAR
 }
 
-cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
-                                   const void* v, void* out, int T, int window, int shape,
-                                   cudaStream_t st) {
-  if (s.d != TQ_D || !w.qhat_rows) return cudaErrorNotSupported;
+template <int D>
+static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
+                              void* out, int T, int window, int shape, cudaStream_t st) {
   const uint64_t BH = (uint64_t)s.B * s.H, BKV = (uint64_t)s.B * s.H_kv;
   CUtensorMap tq, tqh, tk, tv;
   const bool ok =
-      encode3(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, q, TQ_D, (uint64_t)T, BH, TQ_D * 2,
-              (uint64_t)T * TQ_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
-      encode3(&tqh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, w.qhat_rows, TQ_D, (uint64_t)T, BH, TQ_D * 2,
-              (uint64_t)s.T_max * TQ_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
-      encode3(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k, TQ_D, (uint64_t)T, BKV, TQ_D * 2,
-              (uint64_t)s.T_max * TQ_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
-      encode3(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, v, TQ_D, (uint64_t)T, BKV, TQ_D * 2,
-              (uint64_t)s.T_max * TQ_D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+      encode3(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, q, D, (uint64_t)T, BH, D * 2, (uint64_t)T * D * 2, 64, 128,
+              CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tqh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, w.qhat_rows, D, (uint64_t)T, BH, D * 2,
+              (uint64_t)s.T_max * D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k, D, (uint64_t)T, BKV, D * 2, (uint64_t)s.T_max * D * 2, 64,
+              128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+      encode3(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, v, D, (uint64_t)T, BKV, D * 2, (uint64_t)s.T_max * D * 2, 64,
+              128, CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) return cudaErrorInvalidValue;
-  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)SMEM_BYTES);
+  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)TqSmem<D>::BYTES);
   if (err != cudaSuccess) return err;
   TqParams p;
   p.out = (__nv_bfloat16*)out;
@@ -355,9 +390,20 @@ cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const voi
   p.T = T; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
   p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const dim3 grid((unsigned)BH, (T + BM - 1) / BM);
-  hybrid_attn_tcq_kernel<<<grid, NTHR, SMEM_BYTES, st>>>(tq, tqh, tk, tv, p);
+  hybrid_attn_tcq_kernel<D><<<grid, NTHR, TqSmem<D>::BYTES, st>>>(tq, tqh, tk, tv, p);
   count_launch();
   return cudaGetLastError();
+}
+
+bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
+
+cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
+                                   const void* v, void* out, int T, int window, int shape,
+                                   cudaStream_t st) {
+  if (!w.qhat_rows) return cudaErrorNotSupported;
+  if (s.d == 64) return launch_tcq<64>(s, w, q, k, v, out, T, window, shape, st);
+  if (s.d == 128) return launch_tcq<128>(s, w, q, k, v, out, T, window, shape, st);
+  return cudaErrorNotSupported;
 }
 
 }  // namespace delta

@@ -275,6 +275,7 @@ def test_state_errors(B):
     ("llama32_1b_prefill", 0.3, (7, 30), 1),
     ("llama32_1b_prefill", 0.05, (11,), 1),
     ("bitnet_2b_prefill", 0.29, (0, 19), 0),
+    ("bitnet_2b_prefill", 0.29, (3, 12), 2),
 ])
 def test_full_size_prefill_sampled_heads(B, name, theta, heads, kernel):
     """The benchmark's launch configuration at full size: delta arrays of the sampled heads are
@@ -304,3 +305,21 @@ def test_full_size_prefill_sampled_heads(B, name, theta, heads, kernel):
     for h in heads:
         ref = O.prefill_head(t["q"][0, h], t["k"][0, h // g], t["v"][0, h // g], theta, w.window, "block")
         _check_out(o[0, h], ref["out"], w.dtype, f"{name} head {h}")
+
+
+@pytest.mark.parametrize("kernel,theta", [(2, 0.1), (1, 0.2)])
+def test_stack_layer_sampled_units(B, kernel, theta):
+    """One layer of the 16-layer stack configuration (batch 8, T = 4096, block window 256) at full
+    size: outputs of sampled (batch, head) units against the oracle, masks of the sampled units
+    bit-exact, no device-side time-out."""
+    from tests.gpu_helpers import run_prefill, to_host_f64
+    w = WL.WORKLOADS["llama32_1b_stack_layer"]
+    t = WL.make_qkv(w, layer=3, n_decode=0)
+    st, out, _, _ = run_prefill(B, t["q"], t["k"], t["v"], theta, w.window, w.dtype, kernel=kernel)
+    assert B.delta_sparsity_stats(st)["device_status"] == 0
+    g = w.H // w.H_kv
+    mask = B.delta_state_view(st, B.DELTA_VIEW_MASK)
+    for (b, h) in ((0, 0), (7, 31), (3, 14)):
+        ref = O.prefill_head(t["q"][b, h], t["k"][b, h // g], t["v"][b, h // g], theta, w.window, "block")
+        assert np.array_equal(mask[b, h].cpu().numpy().view(np.uint32), ref["delta"]["mask"])
+        _check_out(to_host_f64(out[b, h]), ref["out"], w.dtype, f"stack layer unit {(b, h)}")
