@@ -73,7 +73,7 @@ static void carve(const delta_config_t& c, char* base, Workspace* w) {
   w->qhat[0] = (float*)take(BH * c.d * 4);
   w->qhat[1] = (float*)take(BH * c.d * 4);
   w->R = (float*)take(BH * c.T_max * 4);
-  w->counters = (unsigned long long*)take(CNT_SLOTS * 8);
+  w->counters = (unsigned long long*)take(CNT_TOTAL * 8);
   w->dec_partial = (float*)take(BKV * kMaxDecodeSplits * g * (c.d + 2) * 4);
   w->dec_ticket = (uint32_t*)take(BKV * 4);
   w->qhat_tile_bf16 = (c.dtype == DELTA_BF16) ? (__nv_bfloat16*)take(BH * nt * c.d * 2) : nullptr;
@@ -103,7 +103,7 @@ static delta_status_t zero_state(delta_state* st, cudaStream_t stream) {
   if ((e = cudaMemsetAsync(st->ws.qhat[0], 0, BH * c.d * 4, stream)) != cudaSuccess) return cuda_fail(e);
   if ((e = cudaMemsetAsync(st->ws.qhat[1], 0, BH * c.d * 4, stream)) != cudaSuccess) return cuda_fail(e);
   if ((e = cudaMemsetAsync(st->ws.R, 0, BH * c.T_max * 4, stream)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaMemsetAsync(st->ws.counters, 0, CNT_SLOTS * 8, stream)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemsetAsync(st->ws.counters, 0, CNT_TOTAL * 8, stream)) != cudaSuccess) return cuda_fail(e);
   if ((e = cudaMemsetAsync(st->ws.dec_ticket, 0, (size_t)c.B * c.H_kv * 4, stream)) != cudaSuccess)
     return cuda_fail(e);
   st->n = 0;
@@ -326,12 +326,14 @@ static void finish_stage(delta_stage_stats_t* o, const unsigned long long* c, do
 
 delta_status_t delta_sparsity_stats(const delta_state_t* st, delta_stats_t* host_out, void* stream) {
   if (!st || !host_out) return DELTA_ERR_INVALID_ARG;
-  unsigned long long c[CNT_SLOTS];
+  unsigned long long c[CNT_TOTAL];
   cudaError_t e = cudaMemcpyAsync(c, st->ws.counters, sizeof(c), cudaMemcpyDeviceToHost,
                                   (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e);
   if ((e = cudaStreamSynchronize((cudaStream_t)stream)) != cudaSuccess) return cuda_fail(e);
   memset(host_out, 0, sizeof(*host_out));
+  for (int sh = 0; sh < CNT_SHARDS; ++sh)          // prefill counters are sharded on the device
+    for (int i = 0; i < 4; ++i) c[CNT_PREFILL_NNZ + i] += c[CNT_SHARD_BASE + 4 * sh + i];
   finish_stage(&host_out->prefill, c + CNT_PREFILL_NNZ, st->win_sum[0], st->len_sum[0]);
   finish_stage(&host_out->decode, c + CNT_DECODE_NNZ, st->win_sum[1], st->len_sum[1]);
   unsigned long long sum[4];

@@ -12,7 +12,12 @@ enum CounterSlot {
   CNT_PREFILL_NNZ = 0, CNT_PREFILL_ELEMS, CNT_PREFILL_MACS_DONE, CNT_PREFILL_MACS_DENSE,
   CNT_DECODE_NNZ, CNT_DECODE_ELEMS, CNT_DECODE_MACS_DONE, CNT_DECODE_MACS_DENSE,
   CNT_STATUS,  // low 32 bits: device status word (0 = ok)
-  CNT_SLOTS = 16
+  CNT_SLOTS = 16,
+  // the prefill counters are kept in CNT_SHARDS shards of 4 (nnz, elements, done, dense) behind
+  // the plain slots, so that thousands of CTAs do not queue on four addresses; the host adds them
+  CNT_SHARDS = 32,
+  CNT_SHARD_BASE = CNT_SLOTS,
+  CNT_TOTAL = CNT_SLOTS + 4 * CNT_SHARDS
 };
 
 constexpr int kMaxDecodeSplits = 64;   // split-KV partials per (batch, KV head)
@@ -28,7 +33,7 @@ struct Workspace {
   float* qhat_tile;     // [B,H,n_tiles,d]
   float* qhat[2];       // [B,H,d] ping-pong (decode reads one, writes the other)
   float* R;             // [B,H,T_max]
-  unsigned long long* counters;  // [CNT_SLOTS]
+  unsigned long long* counters;  // [CNT_TOTAL]
   float* dec_partial;   // [B,H_kv,kMaxDecodeSplits,g,(d+2)]
   uint32_t* dec_ticket; // [B,H_kv]
   __nv_bfloat16* qhat_tile_bf16;  // [B,H,n_tiles,d] (bf16 configurations only)

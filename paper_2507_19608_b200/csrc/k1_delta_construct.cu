@@ -209,7 +209,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 //       R(T-1)[j] = q_hat(T-1).k_j for the heads of the group, and the channel-major fp32 key
 //       copy when kt != nullptr.
 template <typename TIn, int D>
-__global__ void __launch_bounds__(256) delta_finish_kernel(
+__global__ void __launch_bounds__(256, 6) delta_finish_kernel(
     const uint32_t* __restrict__ mask, uint16_t* __restrict__ row_nnz,
     uint32_t* __restrict__ tile_nnz, uint8_t* __restrict__ idx,
     unsigned long long* __restrict__ counters, const TIn* __restrict__ k,
@@ -247,8 +247,10 @@ __global__ void __launch_bounds__(256) delta_finish_kernel(
       dense += __shfl_down_sync(0xffffffffu, dense, o);
     }
     if (lane == 0) { s_red[0][warp] = tsum; s_red[1][warp] = done; s_red[2][warp] = dense; }
-    // compacted indices: lane = channel within each mask word
-    uint8_t* idxp = idx + ((size_t)bh * T_max + t0 + warp * 8) * D;
+    // compacted indices: lane = channel within each mask word; the warp's 8 rows are assembled
+    // in shared memory and leave as 16-byte stores (8 consecutive rows are contiguous)
+    __shared__ __align__(16) uint8_t s_idx[8][8 * D];
+    uint8_t* srow = s_idx[warp];
     const int my_rows = min(8, rows - warp * 8);
     for (int r = 0; r < my_rows; ++r) {
       uint32_t m[NW];
@@ -262,22 +264,29 @@ __global__ void __launch_bounds__(256) delta_finish_kernel(
 #pragma unroll
       for (int w2 = 0; w2 < NW; ++w2) {
         if ((m[w2] >> lane) & 1u)
-          idxp[r * D + basep + __popc(m[w2] & ((1u << lane) - 1u))] = (uint8_t)(w2 * 32 + lane);
+          srow[r * D + basep + __popc(m[w2] & ((1u << lane) - 1u))] = (uint8_t)(w2 * 32 + lane);
         basep += __popc(m[w2]);
       }
 #pragma unroll
       for (int pp = lane; pp < D; pp += 32)
-        if (pp >= nnz) idxp[r * D + pp] = 0xFF;
+        if (pp >= nnz) srow[r * D + pp] = 0xFF;
+    }
+    __syncwarp();
+    {
+      uint4* dst = reinterpret_cast<uint4*>(idx + ((size_t)bh * T_max + t0 + warp * 8) * D);
+      const uint4* src = reinterpret_cast<const uint4*>(srow);
+      for (int e = lane; e < my_rows * D / 16; e += 32) dst[e] = src[e];
     }
     __syncthreads();
     if (tid == 0) {
       unsigned long long a = 0, b2 = 0, c2 = 0;
       for (int w2 = 0; w2 < 8; ++w2) { a += s_red[0][w2]; b2 += s_red[1][w2]; c2 += s_red[2][w2]; }
       tile_nnz[(size_t)bh * n_tiles + tile] = (uint32_t)a;
-      atomicAdd(&counters[CNT_PREFILL_NNZ], a);
-      atomicAdd(&counters[CNT_PREFILL_ELEMS], (unsigned long long)rows * D);
-      atomicAdd(&counters[CNT_PREFILL_MACS_DONE], b2);
-      atomicAdd(&counters[CNT_PREFILL_MACS_DENSE], c2);
+      unsigned long long* cs = counters + CNT_SHARD_BASE + 4 * (blockIdx.x % CNT_SHARDS);
+      atomicAdd(&cs[0], a);
+      atomicAdd(&cs[1], (unsigned long long)rows * D);
+      atomicAdd(&cs[2], b2);
+      atomicAdd(&cs[3], c2);
     }
     return;
   }
