@@ -263,6 +263,20 @@ def stage_stats(row_nnz, rows, d, W, shape):
     return dict(nnz=nnz, elements=elements, macs_done=done, macs_dense=dense)
 
 
+def stage_stats_key(row_nnz, T, d, W, shape, g=1):
+    """Counters of a prefill with key deltas (strategy 3): row_nnz[j] is the fired count of key
+    row j of one KV head, which g query heads read.  A causal pair (i, j) costs d multiply-adds
+    inside the window and row_nnz[j] outside it; nnz / elements count the key delta matrix."""
+    nnz = int(np.sum(np.asarray(row_nnz, np.int64)))
+    done = 0
+    dense = 0
+    for j in range(T):
+        for i in range(j, T):
+            done += d if in_window(i, j, W, shape) else int(row_nnz[j])
+            dense += d
+    return dict(nnz=nnz, elements=T * d, macs_done=g * done, macs_dense=g * dense)
+
+
 def finish_stats(c, win_sum, len_sum):
     """S_m, Eq. 6 and the exact MAC-weighted sparsity from raw counters."""
     S_m = 1.0 - c["nnz"] / c["elements"] if c["elements"] else 0.0

@@ -48,8 +48,10 @@ static delta_status_t check_config(const delta_config_t* c) {
   if (c->init != DELTA_INIT_BASIS_EXACT && c->init != DELTA_INIT_ZERO_STATE)
     return DELTA_ERR_INVALID_ARG;
   if (c->source != DELTA_SRC_QUERY && c->source != DELTA_SRC_KEY) return DELTA_ERR_INVALID_ARG;
-  if (c->source == DELTA_SRC_KEY) return DELTA_ERR_UNSUPPORTED;
   if (c->d != 64 && c->d != 128) return DELTA_ERR_UNSUPPORTED;
+  // key deltas (strategy 3) are served by the telescoped tensor-core kernel only
+  if (c->source == DELTA_SRC_KEY && !(c->dtype == DELTA_BF16 && tcq_kernel_shape(c->d)))
+    return DELTA_ERR_UNSUPPORTED;
   const int g = c->H / c->H_kv;
   if (g != 1 && g != 2 && g != 4 && g != 8) return DELTA_ERR_UNSUPPORTED;
   if (c->T_max > kMaxDecodeSplits * kDecodeChunkMax) return DELTA_ERR_UNSUPPORTED;
@@ -180,6 +182,7 @@ int32_t delta_state_position(const delta_state_t* st) { return st ? st->n : -1; 
 // Can prefill kernel `which` (1 or 2) serve this state?
 static bool tc_eligible(const delta_state* st, int which) {
   if (st->cfg.dtype != DELTA_BF16 || !tc_kernel_available(64)) return false;
+  if (st->cfg.source == DELTA_SRC_KEY && which != 2) return false;
   return which == 1 ? tc_kernel_shape(st->cfg.d) : tcq_kernel_shape(st->cfg.d);
 }
 
@@ -192,6 +195,7 @@ int32_t delta_state_prefill_kernel(const delta_state_t* st) {
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
   if (!st || which < -1 || which > 2) return DELTA_ERR_INVALID_ARG;
   if (which >= 1 && !tc_eligible(st, which)) return DELTA_ERR_UNSUPPORTED;
+  if (which == 0 && st->cfg.source == DELTA_SRC_KEY) return DELTA_ERR_UNSUPPORTED;
   st->forced_kernel = which;
   return DELTA_OK;
 }
@@ -220,18 +224,22 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
 #define MARK(i) do { if (prof && (e = cudaEventRecord(st->ev[i], cs)) != cudaSuccess) return cuda_fail(e); } while (0)
   const int which = delta_state_prefill_kernel(st);
   const bool use_tc = which == 1;
+  const bool key = c.source == DELTA_SRC_KEY;
+  if (key && which != 2) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
   MARK(0);
-  if ((e = launch_delta_chain(st->shape, st->ws, q, T, theta, c.dtype, c.init, which == 2, cs)) != cudaSuccess)
+  // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
+  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, which == 2, key, cs)) !=
+      cudaSuccess)
     return cuda_fail(e);
   MARK(1);
-  if ((e = launch_delta_finish(st->shape, st->ws, k, T, window, c.prefill_window, c.dtype, use_tc, cs)) !=
+  if ((e = launch_delta_finish(st->shape, st->ws, k, T, window, c.prefill_window, c.dtype, use_tc, key, cs)) !=
       cudaSuccess)
     return cuda_fail(e);
   MARK(2);
   if (use_tc) {
     e = launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
   } else if (which == 2) {
-    e = launch_hybrid_attn_tcq(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
+    e = launch_hybrid_attn_tcq(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, key, cs);
   } else {
     e = launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window,
                                    c.dtype, cs);
@@ -305,6 +313,7 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
   if (s != DELTA_OK) return s;
   if (st->n < 1) return DELTA_ERR_STATE;
   if (st->n >= st->cfg.T_max) return DELTA_ERR_CAPACITY;
+  if (st->cfg.source == DELTA_SRC_KEY) return DELTA_ERR_UNSUPPORTED;
   cudaError_t e = launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out,
                                      st->n, theta, window, st->cfg.dtype, st->qhat_sel,
                                      (cudaStream_t)stream);

@@ -51,12 +51,15 @@ void count_launch(int n = 1);
 
 // K1a: token-sequential delta chain over the query stream (Eq. 2-3): delta values, mask words,
 // per-tile reference snapshots, final reference.
+// key_stream: the stream is K in the KV-cache layout, one chain set per KV head (strategy 3).
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
-                               float theta, int dtype, int init, bool want_qhat_rows, cudaStream_t st);
+                               float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
+                               cudaStream_t st);
 // K1b: row-parallel finish: counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* k, int T,
-                                int window, int shape, int dtype, bool want_kt, cudaStream_t st);
+                                int window, int shape, int dtype, bool want_kt, bool key_stream,
+                                cudaStream_t st);
 // K2 (generic): fused hybrid attention on CUDA cores, any supported dtype.
 cudaError_t launch_hybrid_attn_generic(const Shape& s, const Workspace& w, const void* q,
                                        const void* k, const void* v, void* out, int T, int window,
@@ -85,6 +88,13 @@ __host__ __device__ __forceinline__ bool in_window(int i, int j, int W, int shap
 __host__ __device__ __forceinline__ int in_window_count(int i, int W, int shape) {
   if (W <= 0) return 0;
   return shape == 0 ? (i % W) + 1 : (i + 1 < W ? i + 1 : W);
+}
+
+// Number of queries i in [j, T) whose pair (i, j) is inside the exact window (key j's column).
+__host__ __device__ __forceinline__ int in_window_col_count(int j, int T, int W, int shape) {
+  if (W <= 0) return 0;
+  const int last = shape == 0 ? (j / W + 1) * W : j + W;   // first query past the window
+  return (last < T ? last : T) - j;
 }
 
 }  // namespace delta

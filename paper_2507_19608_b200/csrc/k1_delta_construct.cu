@@ -56,7 +56,9 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     const TIn* __restrict__ q, float* __restrict__ dq, uint32_t* __restrict__ mask,
     float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
     __nv_bfloat16* __restrict__ qhat_rows, unsigned long long* __restrict__ counters, int T,
-    int T_max, int n_tiles, float theta, int basis_exact) {
+    int T_max, int n_tiles, float theta, int basis_exact, int src_rows) {
+  // q: the stream that becomes the delta matrix, [heads][src_rows][D] with rows 0..T-1 read
+  // (queries: src_rows = T; keys in the KV-cache layout: src_rows = T_max)
   constexpr int NW = D / 32;                       // chain warps = mask words per row
   constexpr uint32_t ROW_BYTES = D * sizeof(TIn);
   constexpr uint32_t STAGE_BYTES = RC * ROW_BYTES;
@@ -82,7 +84,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
   if (warp == NW) {
     // ---- producer: keeps up to NS stages of query rows in flight
     if (lane == 0) {
-      const unsigned char* src = reinterpret_cast<const unsigned char*>(q) + (size_t)bh * T * ROW_BYTES;
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(q) + (size_t)bh * src_rows * ROW_BYTES;
       const uint32_t ring0 = smem_u32(ring);
       for (int i = 0; i < n_chunks; ++i) {
         const int s = i % NS;
@@ -174,9 +176,11 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
 }
 
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
-                               float theta, int dtype, int init, bool want_qhat_rows, cudaStream_t st) {
+                               float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
+                               cudaStream_t st) {
   __nv_bfloat16* qrows = want_qhat_rows ? w.qhat_rows : nullptr;
-  const int grid = s.B * s.H;
+  const int grid = s.B * (key_stream ? s.H_kv : s.H);
+  const int src_rows = key_stream ? s.T_max : T;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
   cudaError_t err = cudaSuccess;
 #define LAUNCH(TIN, DD)                                                                          \
@@ -188,7 +192,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
       if (err != cudaSuccess) return err;                                                        \
     }                                                                                            \
     kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.dq, w.mask, w.qhat_tile, w.qhat[0], qrows, \
-                                      w.counters, T, s.T_max, s.n_tiles, theta, basis);          \
+                                      w.counters, T, s.T_max, s.n_tiles, theta, basis, src_rows); \
   } while (0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
@@ -214,7 +218,8 @@ __global__ void __launch_bounds__(256, 6) delta_finish_kernel(
     uint32_t* __restrict__ tile_nnz, uint8_t* __restrict__ idx,
     unsigned long long* __restrict__ counters, const TIn* __restrict__ k,
     const float* __restrict__ qhat, float* __restrict__ R, float* __restrict__ kt, int T,
-    int T_max, int n_tiles, int BH, int H, int g, int W, int shape, int n_idx_blocks, int kt_ld) {
+    int T_max, int n_tiles, int BH, int H, int g, int W, int shape, int n_idx_blocks, int kt_ld,
+    int key_stream) {
   constexpr int NW = D / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if ((int)blockIdx.x < n_idx_blocks) {
@@ -237,9 +242,18 @@ __global__ void __launch_bounds__(256, 6) delta_finish_kernel(
       row_nnz[(size_t)bh * T_max + t0 + r_mine] = (uint16_t)nnz;
       tsum = (unsigned long long)nnz;
       const int i = t0 + r_mine;
-      const int n_in = in_window_count(i, W, shape);
-      done = (unsigned long long)n_in * D + (unsigned long long)(i + 1 - n_in) * nnz;
-      dense = (unsigned long long)(i + 1) * D;
+      if (!key_stream) {
+        // query deltas: row i meets i + 1 keys, nnz multiply-adds per out-of-window key
+        const int n_in = in_window_count(i, W, shape);
+        done = (unsigned long long)n_in * D + (unsigned long long)(i + 1 - n_in) * nnz;
+        dense = (unsigned long long)(i + 1) * D;
+      } else {
+        // key deltas: key i meets the T - i queries behind it, for each of the g query heads
+        const int n_q = T - i;
+        const int n_in = in_window_col_count(i, T, W, shape);
+        done = (unsigned long long)g * ((unsigned long long)n_in * D + (unsigned long long)(n_q - n_in) * nnz);
+        dense = (unsigned long long)g * n_q * D;
+      }
     }
     for (int o = 4; o > 0; o >>= 1) {
       tsum += __shfl_down_sync(0xffffffffu, tsum, o);
@@ -340,17 +354,19 @@ __global__ void __launch_bounds__(256, 6) delta_finish_kernel(
 }
 
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* k, int T,
-                                int window, int shape, int dtype, bool want_kt, cudaStream_t st) {
-  const int BH = s.B * s.H;
+                                int window, int shape, int dtype, bool want_kt, bool key_stream,
+                                cudaStream_t st) {
+  // key deltas: the index/counter pass runs over the KV heads and there is no hand-off row
+  const int BH = s.B * (key_stream ? s.H_kv : s.H);
   const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
   const int n_idx_blocks = BH * tiles_used;
-  const int n_key_blocks = s.B * s.H_kv * ((T + 63) / 64);
+  const int n_key_blocks = key_stream ? 0 : s.B * s.H_kv * ((T + 63) / 64);
   const int kt_ld = (s.T_max + 3) / 4 * 4;
   float* kt = (want_kt && w.kt) ? w.kt : nullptr;
 #define LAUNCH(TIN, DD)                                                                          \
   delta_finish_kernel<TIN, DD><<<n_idx_blocks + n_key_blocks, 256, 0, st>>>(                     \
       w.mask, w.row_nnz, w.tile_nnz, w.idx, w.counters, (const TIN*)k, w.qhat[0], w.R, kt, T,    \
-      s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld)
+      s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld, key_stream ? 1 : 0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
   } else {

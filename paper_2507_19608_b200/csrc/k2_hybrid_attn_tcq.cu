@@ -61,7 +61,7 @@ template <int D> struct TqSmem {
 };
 
 enum Bar {
-  BAR_Q = 0, BAR_K0, BAR_K1, BAR_V0, BAR_V1, BAR_S0, BAR_S1, BAR_O,   // one arrival (+ bytes)
+  BAR_Q = 0, BAR_K0, BAR_K1, BAR_V0, BAR_V1, BAR_S0, BAR_S1, BAR_O, BAR_KX,   // one arrival (+ bytes)
   BAR_SFREE0, BAR_SFREE1,                                             // 16 arrivals: scores read
   BAR_P,                                                              // 16 arrivals: P written
   NUM_BARS
@@ -76,7 +76,12 @@ struct TqParams {
 
 }  // namespace
 
-template <int D>
+// KEY = false: query deltas (strategy 1): telescoped scores Q_hat.K^T, tm_qh maps the reference
+// query rows.  KEY = true: key deltas (strategy 3): the column recursion telescopes to
+// S[i][j] = q_i.k_hat(j), so the telescoped scores are Q.K_hat^T; tm_qh maps the reference key
+// rows (per KV head), which take the place of the key tiles in the ring, and the original keys
+// are fetched only for tiles that touch the window.
+template <int D, bool KEY>
 __global__ void __launch_bounds__(NTHR, 1)
 hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qh,
                        const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -139,36 +144,53 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
         for (uint32_t kb = 0; kb < NKB; ++kb) tma_load_3d(dst + kb * SZ_BLK, tm, bar, 64 * kb, row0, outer);
       };
-      mbar_expect_tx(BAR(BAR_Q), 2 * SZ_TILE);
+      const CUtensorMap* tm_ring = KEY ? &tm_qh : &tm_k;   // what streams through the key ring
+      mbar_expect_tx(BAR(BAR_Q), (KEY ? 1 : 2) * SZ_TILE);
       load_tile(base + OFF_Q, &tm_q, BAR(BAR_Q), i0, bh);
-      load_tile(base + OFF_QH, &tm_qh, BAR(BAR_Q), i0, bh);
+      if (!KEY) load_tile(base + OFF_QH, &tm_qh, BAR(BAR_Q), i0, bh);
       mbar_expect_tx(BAR(BAR_K0), SZ_TILE);
-      load_tile(base + OFF_K, &tm_k, BAR(BAR_K0), 0, bkv);
+      load_tile(base + OFF_K, tm_ring, BAR(BAR_K0), 0, bkv);
       mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
       load_tile(base + OFF_V, &tm_v, BAR(BAR_V0), 0, bkv);
       if (NKBUF == 2 && qt >= 1) {
         mbar_expect_tx(BAR(BAR_K1), SZ_TILE);
-        load_tile(base + OFF_K + SZ_TILE, &tm_k, BAR(BAR_K1), BN, bkv);
+        load_tile(base + OFF_K + SZ_TILE, tm_ring, BAR(BAR_K1), BN, bkv);
       }
+      int n_kx = 0;    // exact key tiles fetched so far (key deltas only)
       // key buffer and barrier parity of tile t
       auto kbuf = [&](int t) { return NKBUF == 2 ? (t & 1) : 0; };
       auto kpar = [&](int t) { return NKBUF == 2 ? ((t >> 1) & 1) : (t & 1); };
       // scores of tile t: Q_hat.K^T into buffer t&1, plus Q.K^T if the tile touches the window
       auto issue_scores = [&](int t) {
         const int bf = t & 1;
+        const bool exact = tile_needs_exact(t);
+        if (KEY && exact) {
+          // original keys of a window tile: into the slot the reference queries use otherwise
+          // (its previous reader, the last window tile's product, is done: see the callers)
+          mbar_expect_tx(BAR(BAR_KX), SZ_TILE);
+          load_tile(base + OFF_QH, &tm_k, BAR(BAR_KX), t * BN, bkv);
+        }
         mbar_wait(BAR(BAR_K0 + kbuf(t)), kpar(t), abort_flag);
         tc_fence_after();
         const uint32_t kb = base + OFF_K + kbuf(t) * SZ_TILE;
+        const uint32_t a_tele = base + (KEY ? OFF_Q : OFF_QH);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
           tc_mma(tmem + TMEM_SH + bf * 128,
-                 make_desc(base + OFF_QH + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
+                 make_desc(a_tele + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
                  make_desc(kb + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
-        if (tile_needs_exact(t)) {
+        if (exact) {
+          uint32_t kx = kb;
+          if (KEY) {
+            mbar_wait(BAR(BAR_KX), n_kx & 1, abort_flag);
+            ++n_kx;
+            tc_fence_after();
+            kx = base + OFF_QH;
+          }
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
             tc_mma(tmem + TMEM_SX, make_desc(base + OFF_Q + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
-                   make_desc(kb + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
+                   make_desc(kx + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
         }
         tc_commit(BAR(BAR_S0 + bf));
       };
@@ -183,7 +205,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int tn = t + (int)NKBUF;         // the tile that takes this buffer next
         if (tn <= qt) {
           mbar_expect_tx(BAR(BAR_K0 + kbuf(tn)), SZ_TILE);
-          load_tile(base + OFF_K + kbuf(tn) * SZ_TILE, &tm_k, BAR(BAR_K0 + kbuf(tn)), tn * BN, bkv);
+          load_tile(base + OFF_K + kbuf(tn) * SZ_TILE, tm_ring, BAR(BAR_K0 + kbuf(tn)), tn * BN, bkv);
         }
         // next tile's scores one tile ahead, unless it needs the single exact-score buffer
         if (more && !next_exact) {
@@ -366,22 +388,23 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #undef BAR
 }
 
-template <int D>
+template <int D, bool KEY>
 static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
                               void* out, int T, int window, int shape, cudaStream_t st) {
   const uint64_t BH = (uint64_t)s.B * s.H, BKV = (uint64_t)s.B * s.H_kv;
+  const uint64_t ref_heads = KEY ? BKV : BH;   // the reference rows follow the delta stream
   CUtensorMap tq, tqh, tk, tv;
   const bool ok =
       encode3(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, q, D, (uint64_t)T, BH, D * 2, (uint64_t)T * D * 2, 64, 128,
               CU_TENSOR_MAP_SWIZZLE_128B) &&
-      encode3(&tqh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, w.qhat_rows, D, (uint64_t)T, BH, D * 2,
+      encode3(&tqh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, w.qhat_rows, D, (uint64_t)T, ref_heads, D * 2,
               (uint64_t)s.T_max * D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
       encode3(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k, D, (uint64_t)T, BKV, D * 2, (uint64_t)s.T_max * D * 2, 64,
               128, CU_TENSOR_MAP_SWIZZLE_128B) &&
       encode3(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, v, D, (uint64_t)T, BKV, D * 2, (uint64_t)s.T_max * D * 2, 64,
               128, CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) return cudaErrorInvalidValue;
-  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D, KEY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)TqSmem<D>::BYTES);
   if (err != cudaSuccess) return err;
   TqParams p;
@@ -390,7 +413,7 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
   p.T = T; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
   p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const dim3 grid((unsigned)BH, (T + BM - 1) / BM);
-  hybrid_attn_tcq_kernel<D><<<grid, NTHR, TqSmem<D>::BYTES, st>>>(tq, tqh, tk, tv, p);
+  hybrid_attn_tcq_kernel<D, KEY><<<grid, NTHR, TqSmem<D>::BYTES, st>>>(tq, tqh, tk, tv, p);
   count_launch();
   return cudaGetLastError();
 }
@@ -399,10 +422,14 @@ bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
 
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
                                    const void* v, void* out, int T, int window, int shape,
-                                   cudaStream_t st) {
+                                   bool key_deltas, cudaStream_t st) {
   if (!w.qhat_rows) return cudaErrorNotSupported;
-  if (s.d == 64) return launch_tcq<64>(s, w, q, k, v, out, T, window, shape, st);
-  if (s.d == 128) return launch_tcq<128>(s, w, q, k, v, out, T, window, shape, st);
+  if (s.d == 64)
+    return key_deltas ? launch_tcq<64, true>(s, w, q, k, v, out, T, window, shape, st)
+                      : launch_tcq<64, false>(s, w, q, k, v, out, T, window, shape, st);
+  if (s.d == 128)
+    return key_deltas ? launch_tcq<128, true>(s, w, q, k, v, out, T, window, shape, st)
+                      : launch_tcq<128, false>(s, w, q, k, v, out, T, window, shape, st);
   return cudaErrorNotSupported;
 }
 

@@ -12,8 +12,9 @@ cudaError_t launch_hybrid_attn_tc(const Shape& s, const Workspace& w, const void
                                   cudaStream_t st);
 // Head dimensions the telescoped kernel is written for.
 bool tcq_kernel_shape(int d);
-// Telescoped variant: out-of-window scores as Q_hat.K^T on the tensor cores (needs w.qhat_rows).
+// Telescoped variant: out-of-window scores as Q_hat.K^T (query deltas) or Q.K_hat^T (key deltas)
+// on the tensor cores; w.qhat_rows holds the reference rows of the delta stream.
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
                                    const void* v, void* out, int T, int window, int shape,
-                                   cudaStream_t st);
+                                   bool key_deltas, cudaStream_t st);
 }  // namespace delta

@@ -42,7 +42,8 @@ def test_status_strings():
     (dict(H=6, H_kv=4), B.DELTA_ERR_INVALID_ARG),
     (dict(d=96), B.DELTA_ERR_UNSUPPORTED),
     (dict(H=12, H_kv=4), B.DELTA_ERR_UNSUPPORTED),          # group of 3 query heads
-    (dict(source=B.DELTA_SRC_KEY), B.DELTA_ERR_UNSUPPORTED),
+    (dict(source=B.DELTA_SRC_KEY), B.DELTA_OK),              # key deltas: bf16 only
+    (dict(source=B.DELTA_SRC_KEY, dtype="f32"), B.DELTA_ERR_UNSUPPORTED),
     (dict(T_max=0), B.DELTA_ERR_INVALID_ARG),
     (dict(dtype=7), B.DELTA_ERR_INVALID_ARG),
 ])

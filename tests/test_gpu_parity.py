@@ -323,3 +323,53 @@ def test_stack_layer_sampled_units(B, kernel, theta):
         ref = O.prefill_head(t["q"][b, h], t["k"][b, h // g], t["v"][b, h // g], theta, w.window, "block")
         assert np.array_equal(mask[b, h].cpu().numpy().view(np.uint32), ref["delta"]["mask"])
         _check_out(to_host_f64(out[b, h]), ref["out"], w.dtype, f"stack layer unit {(b, h)}")
+
+
+# ------------------------------------------------------------------ key deltas (strategy 3)
+KEY_CASES = [
+    # Bn, H, Hk, T,  d,  theta, W,  shape
+    (1, 4, 1, 200, 64, 0.2, 64, "block"),
+    (2, 4, 2, 513, 64, 0.15, 100, "sliding"),
+    (1, 2, 2, 300, 64, 0.3, 0, "block"),
+    (1, 8, 2, 384, 128, 0.25, 128, "block"),
+    (1, 2, 1, 130, 64, 0.1, 1000, "block"),        # window covers everything
+    (1, 2, 1, 1, 64, 0.1, 4, "block"),
+]
+
+
+@pytest.mark.parametrize("case", KEY_CASES, ids=[f"T{c[3]}-d{c[4]}-W{c[6]}{c[7][0]}" for c in KEY_CASES])
+def test_key_delta_prefill_matches_oracle(B, case):
+    """Strategy (3): the key stream of every KV head becomes the delta matrix."""
+    from tests.gpu_helpers import to_cache, to_dev, to_host_f64
+    Bn, H, Hk, T, d, theta, W, shape = case
+    q, k, v = _inputs(Bn, H, Hk, T, d, "bf16", seed=300 + T + d)
+    cfg = B.make_config(Bn, H, Hk, d, T, "bf16", source=B.DELTA_SRC_KEY,
+                        prefill_window=B.DELTA_WIN_BLOCK if shape == "block" else B.DELTA_WIN_SLIDING)
+    st = B.delta_state_init(cfg)
+    dq_, kc, vc = to_dev(q, "bf16"), to_cache(k, T, "bf16"), to_cache(v, T, "bf16")
+    out = torch.full_like(dq_, float("nan"))
+    B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, float(theta), int(W))
+    torch.cuda.synchronize()
+    ref, heads = O.prefill_mha(q, k, v, theta, W, shape, source="key")
+    _check_out(to_host_f64(out), ref, "bf16", "key-delta prefill out")
+    # delta arrays are those of the key stream, one set per KV head (the leading H_kv heads of the views)
+    g = H // Hk
+    dk = B.delta_state_view(st, B.DELTA_VIEW_DQ).cpu().numpy()
+    mask = B.delta_state_view(st, B.DELTA_VIEW_MASK).cpu().numpy().view(np.uint32)
+    rnz = B.delta_state_view(st, B.DELTA_VIEW_ROW_NNZ).cpu().numpy().view(np.uint16)
+    idx = B.delta_state_view(st, B.DELTA_VIEW_IDX).cpu().numpy()
+    dk, mask, rnz, idx = (x.reshape(Bn * H, *x.shape[2:]) for x in (dk, mask, rnz, idx))
+    nnz = done = dense = 0
+    for b in range(Bn):
+        for kvh in range(Hk):
+            r = heads[(b, kvh * g)]["delta"]
+            u = b * Hk + kvh
+            assert np.array_equal(dk[u, :T].view(np.uint32), r["dq"].view(np.uint32))
+            assert np.array_equal(mask[u, :T], r["mask"])
+            assert np.array_equal(rnz[u, :T], r["row_nnz"])
+            assert np.array_equal(idx[u, :T], r["idx"])
+            c = O.stage_stats_key(r["row_nnz"], T, d, W, shape, g)
+            nnz += c["nnz"]; done += c["macs_done"]; dense += c["macs_dense"]
+    s = B.delta_sparsity_stats(st)["prefill"]
+    assert (s["nnz"], s["elements"], s["macs_done"], s["macs_dense"]) == (nnz, Bn * Hk * T * d, done, dense)
+    assert B.delta_sparsity_stats(st)["device_status"] == 0

@@ -390,3 +390,17 @@ def test_workload_generator_is_seeded_and_ar1():
     r1 = np.mean([np.corrcoef(x[1:, c], x[:-1, c])[0, 1] for c in range(x.shape[1])])
     assert 0.85 < r1 < 0.99                       # lag-1 autocorrelation near rho = 0.95
     assert np.array_equal(WL.round_to_bf16(t["k"]), t["k"])
+
+
+def test_key_delta_counters_closed_forms():
+    """Key-delta counters: all-dense deltas cost exactly the dense multiply-adds; all-zero deltas
+    outside a block window cost only the in-window pairs (closed form of the block sizes)."""
+    T, d, W = 50, 64, 8
+    full = O.stage_stats_key(np.full(T, d), T, d, W, "block", g=4)
+    assert full["macs_done"] == full["macs_dense"] == 4 * d * T * (T + 1) // 2
+    none = O.stage_stats_key(np.zeros(T, int), T, d, W, "block", g=1)
+    blocks, rem = divmod(T, W)
+    n_in = blocks * W * (W + 1) // 2 + rem * (rem + 1) // 2
+    assert none["macs_done"] == d * n_in and none["nnz"] == 0 and none["elements"] == T * d
+    slid = O.stage_stats_key(np.zeros(T, int), T, d, W, "sliding")
+    assert slid["macs_done"] == d * sum(min(i + 1, W) for i in range(T))
