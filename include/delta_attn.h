@@ -54,8 +54,16 @@ typedef enum {
 
 typedef enum { DELTA_F32 = 0, DELTA_BF16 = 1 } delta_dtype_t;
 
-/* Which operand becomes the delta matrix (Section III-A).  QUERY = strategy (1), top-down
- * query deltas; KEY = strategy (3), reserved (returns DELTA_ERR_UNSUPPORTED). */
+/* Which operand becomes the delta matrix (Section III-A).
+ * QUERY = strategy (1), top-down query deltas: one chain per (query head, channel); the carried
+ *   decode state is the reference query and the score row R.
+ * KEY = strategy (3), the one the paper adopts: the key stream of every KV head is thresholded
+ *   (one chain per (KV head, channel)); the out-of-window score of pair (i, j) is the column
+ *   recursion S[i][j] = S[i][j-1] + q_i.Delta k(j) = q_i.k_hat(j); the carried decode state is
+ *   the reference key, and the library keeps a cache of reference-key rows in its workspace.
+ *   bf16 with d = 64 or 128 only (DELTA_ERR_UNSUPPORTED otherwise).  With KEY the delta arrays
+ *   of delta_state_view hold one set per KV head: read them as [B * H_kv, ...] from the start
+ *   of the view. */
 typedef enum { DELTA_SRC_QUERY = 0, DELTA_SRC_KEY = 1 } delta_source_t;
 
 /* Shape of the exact-attention region in prefill (Section III-B).  BLOCK: squares of side
@@ -135,7 +143,10 @@ DELTA_API delta_status_t delta_attn_prefill_host(delta_state_t* st, const void* 
  * R[j] += Delta q . k_j for every cached key j < n (Eq. 4); R[n] = q_hat . k_new for the key
  * that arrives now; score j is q_new.k_j if n - j < window else R[j]; softmax over the n + 1
  * keys; out = P.V; position becomes n + 1.  Needs n >= 1 (else DELTA_ERR_STATE) and
- * n < T_max (else DELTA_ERR_CAPACITY). */
+ * n < T_max (else DELTA_ERR_CAPACITY).
+ * With DELTA_SRC_KEY the step thresholds k_new against the carried reference key instead
+ * (Eq. 2-3), appends the reference-key row k_hat(n), and scores key j with q_new.k_j if
+ * n - j < window else q_new.k_hat(j). */
 DELTA_API delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, const void* k_new,
                                       const void* v_new, void* k_cache, void* v_cache, void* out,
                                       float theta, int32_t window, void* stream);

@@ -203,6 +203,8 @@ def prefill_head(q, k, v, theta, W, shape="block", init="basis_exact", source="q
     if source == "query" and order == "top_down":
         state = dict(n=T, qhat=delta["ahat"].copy(), R=S_delta[T - 1].copy(),
                      dq_hist=delta["dq"].copy(), k=k.copy(), v=v.copy())
+    elif source == "key":
+        state = dict(n=T, khat=delta["ahat"].copy(), dk_hist=delta["dq"].copy(), k=k.copy(), v=v.copy())
     return dict(out=out, S_star=S_star, S_delta=S_delta, S_exact=S_exact, delta=delta, state=state)
 
 
@@ -240,6 +242,55 @@ def decode_head(state, q_new, k_new, v_new, theta, W_d):
     out = p @ v_all.astype(F64)
     new_state = dict(n=n + 1, qhat=qhat, R=R, dq_hist=dq_hist, k=k_all, v=v_all)
     return out, new_state, dict(row_nnz=int(fire.sum()), dq=dq, fired=fire)
+
+
+def decode_key_step(state, k_new, v_new, theta):
+    """Key side of one decode step of strategy (3) for one KV head: Delta k(n) against the
+    carried reference key (Eq. 2-3); the delta, the key and the value are appended to the
+    cached histories.  Returns (new_state, info with row_nnz / dk / fired)."""
+    theta = F32(theta)
+    k_new = np.asarray(k_new, F32)
+    diff = k_new - state["khat"]
+    fire = np.abs(diff) > theta
+    dk = np.where(fire, diff, F32(0.0)).astype(F32)
+    khat = np.where(fire, k_new, state["khat"]).astype(F32)
+    new_state = dict(n=state["n"] + 1, khat=khat, dk_hist=np.vstack([state["dk_hist"], dk[None, :]]),
+                     k=np.vstack([state["k"], k_new[None, :]]),
+                     v=np.vstack([state["v"], np.asarray(v_new, F32)[None, :]]))
+    return new_state, dict(row_nnz=int(fire.sum()), dk=dk, fired=fire)
+
+
+def decode_key_attend(state, q_new, W_d):
+    """Query side of a strategy-(3) decode step, after decode_key_step appended the new key:
+    the score of key j is q_new.k_j for the W_d most recent keys (the new one included) and the
+    prefix sum of the cached delta products q_new.Delta k(0..j) for the older ones (the column
+    recursion of Section III-A carried into decoding, Section III-C).  Returns out [d] float64."""
+    n = state["n"] - 1                                   # index of the token that just arrived
+    d = q_new.shape[0]
+    q64 = np.asarray(q_new, F32).astype(F64)
+    s_delta = np.cumsum(state["dk_hist"].astype(F64) @ q64)   # S[n][j] = S[n][j-1] + q.Delta k(j)
+    s = np.empty(n + 1, F64)
+    for j in range(n + 1):
+        s[j] = (q64 @ state["k"][j].astype(F64)) if in_window(n, j, W_d, "sliding") else s_delta[j]
+    s *= 1.0 / np.sqrt(F64(d))
+    p = np.exp(s - s.max())
+    p /= p.sum()
+    return p @ state["v"].astype(F64)
+
+
+def decode_mha_key(states, q_new, k_new, v_new, theta, W_d):
+    """states: dict (b, kv head) -> key-delta state.  q_new [B,H,d], k_new,v_new [B,H_kv,d]."""
+    B, H, d = q_new.shape
+    H_kv = k_new.shape[1]
+    g = H // H_kv
+    out = np.zeros((B, H, d), F64)
+    infos = {}
+    for b in range(B):
+        for kvh in range(H_kv):
+            states[(b, kvh)], infos[(b, kvh)] = decode_key_step(states[(b, kvh)], k_new[b, kvh], v_new[b, kvh], theta)
+            for hh in range(g):
+                out[b, kvh * g + hh] = decode_key_attend(states[(b, kvh)], q_new[b, kvh * g + hh], W_d)
+    return out, infos
 
 
 # --------------------------------------------------------------------------- Eq. 6 and exact counts

@@ -313,10 +313,12 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
   if (s != DELTA_OK) return s;
   if (st->n < 1) return DELTA_ERR_STATE;
   if (st->n >= st->cfg.T_max) return DELTA_ERR_CAPACITY;
-  if (st->cfg.source == DELTA_SRC_KEY) return DELTA_ERR_UNSUPPORTED;
-  cudaError_t e = launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out,
-                                     st->n, theta, window, st->cfg.dtype, st->qhat_sel,
-                                     (cudaStream_t)stream);
+  cudaError_t e =
+      st->cfg.source == DELTA_SRC_KEY
+          ? launch_decode_step_key(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n,
+                                   theta, window, st->qhat_sel, (cudaStream_t)stream)
+          : launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n,
+                               theta, window, st->cfg.dtype, st->qhat_sel, (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e);
   const int L = st->n + 1;
   st->win_sum[1] += (double)(window < L ? window : L);

@@ -70,6 +70,12 @@ cudaError_t launch_decode_step(const Shape& s, const Workspace& w, const void* q
                                void* out, int n, float theta, int window, int dtype, int qhat_sel,
                                cudaStream_t st);
 
+// K3 (key deltas): one decode step of strategy (3); bf16 only, needs w.qhat_rows (reference-key cache).
+cudaError_t launch_decode_step_key(const Shape& s, const Workspace& w, const void* q_new,
+                                   const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                   void* out, int n, float theta, int window, int qhat_sel,
+                                   cudaStream_t st);
+
 // ---- small device helpers -------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }

@@ -373,3 +373,54 @@ def test_key_delta_prefill_matches_oracle(B, case):
     s = B.delta_sparsity_stats(st)["prefill"]
     assert (s["nnz"], s["elements"], s["macs_done"], s["macs_dense"]) == (nnz, Bn * Hk * T * d, done, dense)
     assert B.delta_sparsity_stats(st)["device_status"] == 0
+
+
+@pytest.mark.parametrize("Bn,H,Hk,T,d,theta,W,steps", [
+    (1, 4, 1, 100, 64, 0.2, 8, 5),
+    (2, 4, 2, 300, 64, 0.15, 64, 4),
+    (1, 8, 2, 700, 128, 0.29, 4, 4),       # several key slices
+    (1, 2, 1, 90, 64, 0.1, 0, 3),          # no exact window at all
+    (1, 2, 2, 40, 64, 0.0, 1000, 3),       # window covers the whole cache
+    (1, 1, 1, 1, 64, 0.1, 2, 4),
+])
+def test_key_delta_decode_steps_match_oracle(B, Bn, H, Hk, T, d, theta, W, steps):
+    """Strategy (3) carried into decoding: the reference key per KV head is the carried state,
+    old keys are scored through the reference-key rows, the W_d most recent ones exactly."""
+    from tests.gpu_helpers import to_cache, to_dev, to_host_f64
+    w = WL.Workload("t", Bn, H, Hk, T, d, "bf16", 0.95, 0.5, W, (), 500 + T, n_decode=steps)
+    t = WL.make_qkv(w)
+    T_max = T + steps
+    cfg = B.make_config(Bn, H, Hk, d, T_max, "bf16", source=B.DELTA_SRC_KEY, prefill_window=B.DELTA_WIN_SLIDING)
+    st = B.delta_state_init(cfg)
+    dq_, kc, vc = to_dev(t["q"], "bf16"), to_cache(t["k"], T_max, "bf16"), to_cache(t["v"], T_max, "bf16")
+    out = torch.full_like(dq_, float("nan"))
+    B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, float(theta), int(W))
+    ref, heads = O.prefill_mha(t["q"], t["k"], t["v"], theta, W, "sliding", source="key")
+    _check_out(to_host_f64(out), ref, "bf16", "key-delta prefill out")
+    g = H // Hk
+    states = {(b, kvh): heads[(b, kvh * g)]["state"] for b in range(Bn) for kvh in range(Hk)}
+    row_nnz = {key: list(heads[(key[0], key[1] * g)]["delta"]["row_nnz"]) for key in states}
+    nnz = done = dense = 0
+    for s in range(steps):
+        qn, kn, vn = t["q_dec"][:, :, s], t["k_dec"][:, :, s], t["v_dec"][:, :, s]
+        dqn, dkn, dvn = to_dev(qn, "bf16"), to_dev(kn, "bf16"), to_dev(vn, "bf16")
+        o = torch.full_like(dqn, float("nan"))
+        B.delta_attn_decode_step(st, dqn, dkn, dvn, kc, vc, o, float(theta), int(W))
+        torch.cuda.synchronize()
+        oref, infos = O.decode_mha_key(states, qn, kn, vn, theta, W)
+        _check_out(to_host_f64(o), oref, "bf16", f"key-delta decode step {s}")
+        n = T + s
+        assert B.delta_state_position(st) == n + 1
+        assert torch.equal(kc[:, :, n], dkn) and torch.equal(vc[:, :, n], dvn)
+        khat = B.delta_state_view(st, B.DELTA_VIEW_QHAT).cpu().numpy().reshape(Bn * H, d)
+        for (b, kvh), stt in states.items():
+            assert np.array_equal(khat[b * Hk + kvh].view(np.uint32), stt["khat"].view(np.uint32))
+            row_nnz[(b, kvh)].append(infos[(b, kvh)]["row_nnz"])
+            nnz += infos[(b, kvh)]["row_nnz"]
+            for j in range(n + 1):
+                done += g * (d if O.in_window(n, j, W, "sliding") else int(row_nnz[(b, kvh)][j]))
+            dense += g * (n + 1) * d
+    sd = B.delta_sparsity_stats(st)
+    assert sd["device_status"] == 0
+    sd = sd["decode"]
+    assert (sd["nnz"], sd["elements"], sd["macs_done"], sd["macs_dense"]) == (nnz, Bn * Hk * d * steps, done, dense)

@@ -404,3 +404,22 @@ def test_key_delta_counters_closed_forms():
     assert none["macs_done"] == d * n_in and none["nnz"] == 0 and none["elements"] == T * d
     slid = O.stage_stats_key(np.zeros(T, int), T, d, W, "sliding")
     assert slid["macs_done"] == d * sum(min(i + 1, W) for i in range(T))
+
+
+@pytest.mark.parametrize("W", [0, 3, 8, 100])
+def test_key_delta_decode_continues_prefill(W):
+    """Strategy (3): prefill over T + s tokens (sliding window) and prefill over T tokens followed
+    by s decode steps give the same rows (the decode step is the column recursion continued)."""
+    rng = np.random.default_rng(11)
+    T, s_steps, d, theta = 20, 5, 32, 0.4
+    q = rng.standard_normal((T + s_steps, d)).astype(np.float32)
+    k = np.cumsum(0.3 * rng.standard_normal((T + s_steps, d)), axis=0).astype(np.float32)
+    v = rng.standard_normal((T + s_steps, d)).astype(np.float32)
+    full = O.prefill_head(q, k, v, theta, W, "sliding", source="key")
+    st = O.prefill_head(q[:T], k[:T], v[:T], theta, W, "sliding", source="key")["state"]
+    for s in range(s_steps):
+        st, info = O.decode_key_step(st, k[T + s], v[T + s], theta)
+        out = O.decode_key_attend(st, q[T + s], W)
+        assert np.allclose(out, full["out"][T + s], rtol=1e-12, atol=1e-12)
+        assert np.array_equal(info["dk"], full["delta"]["dq"][T + s])
+    assert np.array_equal(st["khat"], full["delta"]["ahat"])
