@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
   constexpr int KPW = 32 / LPK;  // key rows per warp iteration
   constexpr int ROWB = D * (int)sizeof(TC);
   constexpr int TK = TILE_BYTES / ROWB;              // keys per tile (128 for bf16 d=64)
-  constexpr int RPT = (G * TK + DNT - 1) / DNT;      // R entries per thread and tile
+  constexpr int RPT = (TK + 31) / 32;                // R entries per lane and tile (one head per warp)
   extern __shared__ __align__(128) unsigned char dsm_raw[];
   TC* sK = reinterpret_cast<TC*>(dsm_raw);                         // [2][TK][D]
   TC* sV = reinterpret_cast<TC*>(dsm_raw + 2 * TILE_BYTES);        // [2][TK][D]
@@ -133,13 +133,13 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
     const bool has_new = (n >= tj0) && (n < tj0 + rows);
     const bool any_win = (n - (tj0 + rows - 1)) < W;   // some key of the tile is inside the window
 
-    // R entries of the tile: coalesced, in flight while the tile's copies land
+    // R entries of the tile (warp hh < G holds head hh's, lane-strided): coalesced, in flight
+    // while the tile's copies land
     float r_old[RPT];
 #pragma unroll
     for (int u = 0; u < RPT; ++u) {
-      const int idx = tid + u * DNT;
-      const int hh = idx / TK, jj = idx - hh * TK;
-      r_old[u] = (hh < G && jj < rows && tj0 + jj < n) ? Rg[(size_t)hh * T_max + tj0 + jj] : 0.0f;
+      const int jj = lane + 32 * u;
+      r_old[u] = (warp < G && jj < rows && tj0 + jj < n) ? Rg[(size_t)warp * T_max + tj0 + jj] : 0.0f;
     }
     if (!mbar_wait(bar0 + 8 * (t & 1), (t >> 1) & 1)) s_fail = 1;
     if (has_new) {
@@ -219,25 +219,23 @@ __global__ void __launch_bounds__(DNT) decode_step_kernel(
     }
     __syncthreads();
 
-    // ---- 2. R update (coalesced), hybrid select, scale
-#pragma unroll
-    for (int u = 0; u < RPT; ++u) {
-      const int idx = tid + u * DNT;
-      const int hh = idx / TK, jj = idx - hh * TK;
-      if (hh < G && jj < rows) {
-        const int j = tj0 + jj;
-        const float Rn = r_old[u] + spd[idx];       // r_old is 0 for the key that arrives now
-        Rg[(size_t)hh * T_max + j] = Rn;
-        sc[idx] = ((n - j < W) ? spq[idx] : Rn) * scale_log2e;
-      }
-    }
-    __syncthreads();
-
-    // ---- 3. online softmax over the tile (warp hh serves head hh)
+    // ---- 2+3. warp hh serves head hh: R update (coalesced), hybrid select, scale, online softmax
     if (warp < G) {
       float* s = sc + warp * TK;
+      float* Rh = Rg + (size_t)warp * T_max + tj0;
       float mx = -INFINITY;
-      for (int jj = lane; jj < rows; jj += 32) mx = fmaxf(mx, s[jj]);
+#pragma unroll
+      for (int u = 0; u < RPT; ++u) {
+        const int jj = lane + 32 * u;
+        if (jj < rows) {
+          const int j = tj0 + jj;
+          const float Rn = r_old[u] + spd[warp * TK + jj];     // r_old is 0 for the key that arrives now
+          Rh[jj] = Rn;
+          const float v = ((n - j < W) ? spq[warp * TK + jj] : Rn) * scale_log2e;
+          s[jj] = v;
+          mx = fmaxf(mx, v);
+        }
+      }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       const float m_old = st_s[warp];
@@ -296,7 +294,7 @@ cudaError_t launch_decode_step(const Shape& s, const Workspace& w, const void* q
   const int es = dtype == DELTA_F32 ? 4 : 2;
   const int TK = TILE_BYTES / (s.d * es);
   // one wave of two CTAs per SM (the ring holds 64 KiB), no slice shorter than a quarter tile
-  int nsplit = 296 / bkv;
+  int nsplit = kDecodeTargetCtas / bkv;
   if (nsplit > kMaxDecodeSplits) nsplit = kMaxDecodeSplits;
   const int max_by_len = (L + TK / 4 - 1) / (TK / 4);
   if (nsplit > max_by_len) nsplit = max_by_len;

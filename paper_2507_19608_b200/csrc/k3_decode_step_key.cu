@@ -241,7 +241,7 @@ cudaError_t launch_decode_step_key(const Shape& s, const Workspace& w, const voi
   const int L = n + 1;
   const int bkv = s.B * s.H_kv;
   const int TK = TILE_BYTES / (s.d * 2);
-  int nsplit = 296 / bkv;
+  int nsplit = kDecodeTargetCtas / bkv;
   if (nsplit > kMaxDecodeSplits) nsplit = kMaxDecodeSplits;
   const int max_by_len = (L + TK / 4 - 1) / (TK / 4);
   if (nsplit > max_by_len) nsplit = max_by_len;
