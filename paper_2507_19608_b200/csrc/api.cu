@@ -34,6 +34,10 @@ struct delta_state {
   // optional per-kernel timing of prefill (host-side event objects)
   bool profiling = false, profiled = false;
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  // side stream of prefill: the row-parallel finish kernel runs beside the attention kernel when
+  // the latter does not read its outputs (host-side objects, created at the first prefill)
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -149,6 +153,9 @@ delta_status_t delta_state_destroy(delta_state_t* st) {
   if (!st) return DELTA_ERR_INVALID_ARG;
   for (auto& ev : st->ev)
     if (ev) cudaEventDestroy(ev);
+  if (st->ev_fork) cudaEventDestroy(st->ev_fork);
+  if (st->ev_join) cudaEventDestroy(st->ev_join);
+  if (st->side) cudaStreamDestroy(st->side);
   delete st;
   return DELTA_OK;
 }
@@ -231,10 +238,27 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, which == 2, key, cs)) !=
       cudaSuccess)
     return cuda_fail(e);
+  // The telescoped attention kernel reads nothing the finish kernel writes (counts, indices,
+  // counters, hand-off row), so the two run side by side: finish on the state's side stream
+  // between a fork and a join event.  With per-kernel timing on, everything stays in line.
+  const bool fork = (which == 2) && !prof;
+  if (fork && !st->side) {
+    if ((e = cudaStreamCreateWithFlags(&st->side, cudaStreamNonBlocking)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&st->ev_fork, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&st->ev_join, cudaEventDisableTiming)) != cudaSuccess)
+      return cuda_fail(e);
+  }
+  cudaStream_t fs = cs;
+  if (fork) {
+    if ((e = cudaEventRecord(st->ev_fork, cs)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(st->side, st->ev_fork, 0)) != cudaSuccess) return cuda_fail(e);
+    fs = st->side;
+  }
   MARK(1);
-  if ((e = launch_delta_finish(st->shape, st->ws, k, T, window, c.prefill_window, c.dtype, use_tc, key, cs)) !=
+  if ((e = launch_delta_finish(st->shape, st->ws, k, T, window, c.prefill_window, c.dtype, use_tc, key, fs)) !=
       cudaSuccess)
     return cuda_fail(e);
+  if (fork && (e = cudaEventRecord(st->ev_join, st->side)) != cudaSuccess) return cuda_fail(e);
   MARK(2);
   if (use_tc) {
     e = launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
@@ -245,6 +269,7 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
                                    c.dtype, cs);
   }
   if (e != cudaSuccess) return cuda_fail(e);
+  if (fork && (e = cudaStreamWaitEvent(cs, st->ev_join, 0)) != cudaSuccess) return cuda_fail(e);
   MARK(3);
   MARK(4);
 #undef MARK
