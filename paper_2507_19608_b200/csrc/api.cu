@@ -255,7 +255,7 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
     fs = st->side;
   }
   MARK(1);
-  if ((e = launch_delta_finish(st->shape, st->ws, k, T, window, c.prefill_window, c.dtype, use_tc, key, fs)) !=
+  if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, window, c.prefill_window, c.dtype, c.init, use_tc, key, fs)) !=
       cudaSuccess)
     return cuda_fail(e);
   if (fork && (e = cudaEventRecord(st->ev_join, st->side)) != cudaSuccess) return cuda_fail(e);

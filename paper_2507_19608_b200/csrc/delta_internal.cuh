@@ -57,8 +57,8 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
                                cudaStream_t st);
 // K1b: row-parallel finish: counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
-cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* k, int T,
-                                int window, int shape, int dtype, bool want_kt, bool key_stream,
+cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
+                                int window, int shape, int dtype, int init, bool want_kt, bool key_stream,
                                 cudaStream_t st);
 // K2 (generic): fused hybrid attention on CUDA cores, any supported dtype.
 cudaError_t launch_hybrid_attn_generic(const Shape& s, const Workspace& w, const void* q,

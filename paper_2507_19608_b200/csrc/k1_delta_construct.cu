@@ -11,8 +11,9 @@
 // channel's fire bits of 32 rows in one register and a 32 x 32 bit transpose across the warp
 // (five shuffles) turns them into the 32 rows' mask words.
 //
-// delta_finish_kernel: everything that is parallel over rows once the mask exists -- per-row
-// and per-tile non-zero counts, the compacted channel indices, the counters behind Eq. 6 --
+// delta_finish_kernel: everything that is parallel over rows once the mask exists -- the delta
+// values themselves (query deltas), per-row and per-tile non-zero counts, the compacted channel
+// indices, the counters behind Eq. 6 --
 // plus two passes over the keys that prefill needs anyway: the hand-off row
 // R(T-1)[j] = q_hat(T-1).k_j for decode and, for the tensor-core attention kernel, the
 // channel-major fp32 copy of the keys.
@@ -104,7 +105,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
   } else {
     // ---- chain warps: thread c owns channel c
     const int c = tid;
-    float* dqp = dq + (size_t)bh * T_max * D + c;
+    float* dqp = dq ? dq + (size_t)bh * T_max * D + c : nullptr;   // null: values left to the finish kernel
     __nv_bfloat16* qrp = qhat_rows ? qhat_rows + (size_t)bh * T_max * D + c : nullptr;
     uint32_t* maskp = mask + (size_t)bh * T_max * NW + warp;
     float qh = 0.0f;          // reference state, starts at zero (Eq. 3)
@@ -130,7 +131,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
           const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
           const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
           qh = fire ? x[r] : qh;
-          dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
+          if (dqp) dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
           if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
           bits |= fire ? (1u << r) : 0u;
         }
@@ -148,7 +149,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
             delta = fire ? diff : 0.0f;
           }
           qh = fire ? x : qh;
-          dqp[(size_t)(t0 + r) * D] = delta;
+          if (dqp) dqp[(size_t)(t0 + r) * D] = delta;
           if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
           bits |= fire ? (1u << r) : 0u;
         }
@@ -179,6 +180,9 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
                                float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
                                cudaStream_t st) {
   __nv_bfloat16* qrows = want_qhat_rows ? w.qhat_rows : nullptr;
+  // query deltas: the chain leaves mask words and per-tile references only; delta values are
+  // recomputed row-parallel by the finish kernel.  Key deltas: the chain stores them itself.
+  float* dq_out = key_stream ? w.dq : nullptr;
   const int grid = s.B * (key_stream ? s.H_kv : s.H);
   const int src_rows = key_stream ? s.T_max : T;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
@@ -191,7 +195,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
       err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
       if (err != cudaSuccess) return err;                                                        \
     }                                                                                            \
-    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.dq, w.mask, w.qhat_tile, w.qhat[0], qrows, \
+    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, dq_out, w.mask, w.qhat_tile, w.qhat[0], qrows, \
                                       w.counters, T, s.T_max, s.n_tiles, theta, basis, src_rows); \
   } while (0)
   if (dtype == DELTA_F32) {
@@ -213,13 +217,14 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 //       R(T-1)[j] = q_hat(T-1).k_j for the heads of the group, and the channel-major fp32 key
 //       copy when kt != nullptr.
 template <typename TIn, int D>
-__global__ void __launch_bounds__(256, 6) delta_finish_kernel(
+__global__ void __launch_bounds__(256, 4) delta_finish_kernel(
     const uint32_t* __restrict__ mask, uint16_t* __restrict__ row_nnz,
     uint32_t* __restrict__ tile_nnz, uint8_t* __restrict__ idx,
     unsigned long long* __restrict__ counters, const TIn* __restrict__ k,
     const float* __restrict__ qhat, float* __restrict__ R, float* __restrict__ kt, int T,
     int T_max, int n_tiles, int BH, int H, int g, int W, int shape, int n_idx_blocks, int kt_ld,
-    int key_stream) {
+    int key_stream, const TIn* __restrict__ q, float* __restrict__ dq,
+    const float* __restrict__ qhat_tile, int basis_exact) {
   constexpr int NW = D / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if ((int)blockIdx.x < n_idx_blocks) {
@@ -291,6 +296,48 @@ __global__ void __launch_bounds__(256, 6) delta_finish_kernel(
       const uint4* src = reinterpret_cast<const uint4*>(srow);
       for (int e = lane; e < my_rows * D / 16; e += 32) dst[e] = src[e];
     }
+    // delta values of the tile (query deltas; with key deltas the chain kernel stores them).
+    // With the mask known the reference in front of a row is the last fired row below it, so a
+    // 64-row tile splits into row segments: thread (channel, segment) finds its segment's last
+    // fired value, takes the nearest earlier one (or the reference in front of the tile) as
+    // carry-in and walks its rows with one select per row.
+    if (dq != nullptr) {
+      constexpr int NSEG = 256 / D, SEG = DELTA_TILE_ROWS / NSEG;   // 4 x 16 rows (d=64), 2 x 32 (d=128)
+      __shared__ uint32_t s_mask[DELTA_TILE_ROWS][NW];
+      __shared__ float s_lastx[NSEG][D];
+      __shared__ uint8_t s_has[NSEG][D];
+      for (int e = tid; e < DELTA_TILE_ROWS * NW; e += 256) {
+        const int r = e / NW;
+        s_mask[r][e - r * NW] = (r < rows) ? mask[((size_t)bh * T_max + t0 + r) * NW + (e - r * NW)] : 0u;
+      }
+      const int c = tid % D, seg = tid / D;
+      const TIn* qp0 = q + ((size_t)bh * T + t0 + seg * SEG) * D + c;
+      float x[SEG];
+#pragma unroll
+      for (int r = 0; r < SEG; ++r) x[r] = (seg * SEG + r < rows) ? to_f32(qp0[(size_t)r * D]) : 0.0f;
+      __syncthreads();
+      uint32_t bits = 0;      // bit r: channel c fired in row seg*SEG + r
+#pragma unroll
+      for (int r = 0; r < SEG; ++r) bits |= ((s_mask[seg * SEG + r][c >> 5] >> (c & 31)) & 1u) << r;
+      float lastx = 0.0f;
+#pragma unroll
+      for (int r = 0; r < SEG; ++r) lastx = ((bits >> r) & 1u) ? x[r] : lastx;
+      s_lastx[seg][c] = lastx;
+      s_has[seg][c] = bits != 0u;
+      __syncthreads();
+      float ref = qhat_tile[((size_t)bh * n_tiles + tile) * D + c];   // reference in front of the tile
+      for (int s2 = 0; s2 < seg; ++s2) ref = s_has[s2][c] ? s_lastx[s2][c] : ref;
+      float* dqp = dq + ((size_t)bh * T_max + t0 + seg * SEG) * D + c;
+#pragma unroll
+      for (int r = 0; r < SEG; ++r) {
+        if (seg * SEG + r < rows) {
+          const bool fire = (bits >> r) & 1u;
+          const float diff = (t0 + seg * SEG + r == 0 && basis_exact) ? x[r] : __fsub_rn(x[r], ref);
+          dqp[(size_t)r * D] = fire ? diff : 0.0f;
+          ref = fire ? x[r] : ref;
+        }
+      }
+    }
     __syncthreads();
     if (tid == 0) {
       unsigned long long a = 0, b2 = 0, c2 = 0;
@@ -353,8 +400,8 @@ __global__ void __launch_bounds__(256, 6) delta_finish_kernel(
   }
 }
 
-cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* k, int T,
-                                int window, int shape, int dtype, bool want_kt, bool key_stream,
+cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
+                                int window, int shape, int dtype, int init, bool want_kt, bool key_stream,
                                 cudaStream_t st) {
   // key deltas: the index/counter pass runs over the KV heads and there is no hand-off row
   const int BH = s.B * (key_stream ? s.H_kv : s.H);
@@ -366,7 +413,9 @@ cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* 
 #define LAUNCH(TIN, DD)                                                                          \
   delta_finish_kernel<TIN, DD><<<n_idx_blocks + n_key_blocks, 256, 0, st>>>(                     \
       w.mask, w.row_nnz, w.tile_nnz, w.idx, w.counters, (const TIN*)k, w.qhat[0], w.R, kt, T,    \
-      s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld, key_stream ? 1 : 0)
+      s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld, key_stream ? 1 : 0,   \
+      key_stream ? nullptr : (const TIN*)q, key_stream ? nullptr : w.dq, w.qhat_tile,                \
+      init == DELTA_INIT_BASIS_EXACT ? 1 : 0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
   } else {
