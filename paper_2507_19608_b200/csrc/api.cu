@@ -235,7 +235,7 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   if (key && which != 2) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
   MARK(0);
   // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
-  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, which == 2, key, cs)) !=
+  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, key, cs)) !=
       cudaSuccess)
     return cuda_fail(e);
   // The telescoped attention kernel reads nothing the finish kernel writes (counts, indices,

@@ -52,7 +52,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
 
 }  // namespace
 
-template <typename TIn, int D>
+// EMIT: also store the delta values and the reference rows (key deltas); without it the chain
+// leaves mask words and per-tile references only (query deltas: the rest is rebuilt row-parallel).
+template <typename TIn, int D, bool EMIT>
 __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     const TIn* __restrict__ q, float* __restrict__ dq, uint32_t* __restrict__ mask,
     float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
@@ -131,8 +133,10 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
           const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
           const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
           qh = fire ? x[r] : qh;
-          if (dqp) dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
-          if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
+          if (EMIT) {
+            dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
+            if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
+          }
           bits |= fire ? (1u << r) : 0u;
         }
       } else {
@@ -149,8 +153,10 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
             delta = fire ? diff : 0.0f;
           }
           qh = fire ? x : qh;
-          if (dqp) dqp[(size_t)(t0 + r) * D] = delta;
-          if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
+          if (EMIT) {
+            dqp[(size_t)(t0 + r) * D] = delta;
+            if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
+          }
           bits |= fire ? (1u << r) : 0u;
         }
       }
@@ -189,7 +195,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
   cudaError_t err = cudaSuccess;
 #define LAUNCH(TIN, DD)                                                                          \
   do {                                                                                           \
-    auto kern = delta_chain_kernel<TIN, DD>;                                                     \
+    auto kern = key_stream ? delta_chain_kernel<TIN, DD, true> : delta_chain_kernel<TIN, DD, false>; \
     const size_t smem = (size_t)NS * RC * DD * sizeof(TIN);                                      \
     if (smem > 48 * 1024) {                                                                      \
       err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \

@@ -54,7 +54,10 @@ template <int D> struct TqSmem {
   static constexpr uint32_t OFF_V = OFF_K + NKBUF * SZ_TILE;   // two buffers
   static constexpr uint32_t OFF_P = OFF_V + 2 * SZ_TILE;       // bf16 [2][128 rows][64 keys]
   static constexpr uint32_t OFF_PMAX = OFF_P + 2 * SZ_BLK;     // fp32 [2][128 rows][4 quarters]
-  static constexpr uint32_t OFF_BAR = OFF_PMAX + 2 * 128 * 4 * 4;
+  static constexpr uint32_t OFF_MASK = OFF_PMAX + 2 * 128 * 4 * 4;     // u32 [128 rows][D/32]: the tile's mask words
+  static constexpr uint32_t OFF_LASTX = OFF_MASK + 128 * (D / 32) * 4;   // u16 [512 / D segments][D]: last fired value
+  static constexpr uint32_t OFF_HAS = OFF_LASTX + 512 * 2;               // u8  [512 / D segments][D]: segment fired at all
+  static constexpr uint32_t OFF_BAR = OFF_HAS + 512;
   static constexpr uint32_t OFF_MISC = OFF_BAR + 16 * 8;
   static constexpr uint32_t BYTES = OFF_MISC + 16 + 1024;
   static_assert(BYTES <= 227 * 1024, "shared memory budget");
@@ -64,20 +67,25 @@ enum Bar {
   BAR_Q = 0, BAR_K0, BAR_K1, BAR_V0, BAR_V1, BAR_S0, BAR_S1, BAR_O, BAR_KX,   // one arrival (+ bytes)
   BAR_SFREE0, BAR_SFREE1,                                             // 16 arrivals: scores read
   BAR_P,                                                              // 16 arrivals: P written
+  BAR_QH,                                                             // 16 arrivals: reference-query tile built
   NUM_BARS
 };
 
 struct TqParams {
   __nv_bfloat16* out;
   unsigned long long* counters;
-  int T, H, g, W, shape;
+  const uint32_t* mask;        // [B,H,T_max,D/32] mask words of the query deltas (query deltas only)
+  const float* qhat_tile;      // [B,H,n_tiles64,D] reference in front of every 64-row tile
+  int T, T_max, n_tiles64, H, g, W, shape;
   float scale_log2e;
 };
 
 }  // namespace
 
-// KEY = false: query deltas (strategy 1): telescoped scores Q_hat.K^T, tm_qh maps the reference
-// query rows.  KEY = true: key deltas (strategy 3): the column recursion telescopes to
+// KEY = false: query deltas (strategy 1): telescoped scores Q_hat.K^T.  The 128 reference rows
+// of the tile are rebuilt in shared memory from the query tile, the mask words and the reference
+// in front of the tile (the reference after row i is the last fired value at or below i), so
+// the sequential chain kernel does not have to store them and tm_qh is unused.  KEY = true: key deltas (strategy 3): the column recursion telescopes to
 // S[i][j] = q_i.k_hat(j), so the telescoped scores are Q.K_hat^T; tm_qh maps the reference key
 // rows (per KV head), which take the place of the key tiles in the ring, and the original keys
 // are fetched only for tiles that touch the window.
@@ -93,7 +101,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   using SM = TqSmem<D>;
   constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKBUF = SM::NKBUF;
   constexpr uint32_t OFF_Q = SM::OFF_Q, OFF_QH = SM::OFF_QH, OFF_K = SM::OFF_K, OFF_V = SM::OFF_V,
-                     OFF_P = SM::OFF_P, OFF_PMAX = SM::OFF_PMAX, OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC;
+                     OFF_P = SM::OFF_P, OFF_PMAX = SM::OFF_PMAX, OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC,
+                     OFF_MASK = SM::OFF_MASK, OFF_LASTX = SM::OFF_LASTX, OFF_HAS = SM::OFF_HAS;
   float* sPmax = reinterpret_cast<float*>(sm + OFF_PMAX);
   volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
   volatile uint32_t* abort_flag = sMisc + 1;
@@ -145,9 +154,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (uint32_t kb = 0; kb < NKB; ++kb) tma_load_3d(dst + kb * SZ_BLK, tm, bar, 64 * kb, row0, outer);
       };
       const CUtensorMap* tm_ring = KEY ? &tm_qh : &tm_k;   // what streams through the key ring
-      mbar_expect_tx(BAR(BAR_Q), (KEY ? 1 : 2) * SZ_TILE);
+      mbar_expect_tx(BAR(BAR_Q), SZ_TILE);
       load_tile(base + OFF_Q, &tm_q, BAR(BAR_Q), i0, bh);
-      if (!KEY) load_tile(base + OFF_QH, &tm_qh, BAR(BAR_Q), i0, bh);
       mbar_expect_tx(BAR(BAR_K0), SZ_TILE);
       load_tile(base + OFF_K, tm_ring, BAR(BAR_K0), 0, bkv);
       mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
@@ -195,6 +203,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tc_commit(BAR(BAR_S0 + bf));
       };
       mbar_wait(BAR(BAR_Q), 0, abort_flag);
+      if (!KEY) mbar_wait(BAR(BAR_QH), 0, abort_flag);   // the compute warps have built Q_hat
       issue_scores(0);
       for (int t = 0; t <= qt; ++t) {
         const bool more = t < qt;
@@ -252,6 +261,50 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     if (W > 0) {
       if (shape == 0) { wlo = (i / W) * W; whi = wlo + W; }
       else { wlo = i - W + 1; whi = i + 1; }
+    }
+
+    if (!KEY) {
+      // ---- reference-query tile: Q_hat(r)[c] = the last fired q[.][c] at or below row r, or the
+      // reference in front of the tile.  Thread (channel c, row segment) finds the last fired
+      // value of its segment, takes the nearest earlier one as carry-in and walks its rows.
+      constexpr int NW = D / 32, NSEG = NCTHR / D, SEG = BM / NSEG;   // 8 x 16 rows (d=64), 4 x 32 (d=128)
+      uint32_t* s_mask = reinterpret_cast<uint32_t*>(sm + OFF_MASK);
+      uint16_t* s_lastx = reinterpret_cast<uint16_t*>(sm + OFF_LASTX);
+      uint8_t* s_has = sm + OFF_HAS;
+      for (int e = tid; e < BM * NW; e += NCTHR) {
+        const int r = e / NW;
+        s_mask[e] = (i0 + r < T) ? p.mask[((size_t)bh * p.T_max + i0 + r) * NW + (e - r * NW)] : 0u;
+      }
+      const int c = tid % D, seg = tid / D;
+      const float snap = p.qhat_tile[((size_t)bh * p.n_tiles64 + 2 * qt) * D + c];
+      // byte offset of element (r, c) inside a [128][D] operand tile (128-byte swizzle)
+      auto elem_off = [&](int r) -> uint32_t {
+        return (uint32_t)(c >> 6) * SZ_BLK + (uint32_t)r * 128u + ((((uint32_t)(c & 63) >> 3) ^ ((uint32_t)r & 7u)) << 4) +
+               ((uint32_t)c & 7u) * 2u;
+      };
+      mbar_wait(BAR(BAR_Q), 0, abort_flag);      // the query tile has landed
+      asm volatile("bar.sync 5, %0;" ::"n"(NCTHR) : "memory");   // mask words staged
+      uint32_t bits = 0;
+#pragma unroll
+      for (int r = 0; r < SEG; ++r) bits |= ((s_mask[(seg * SEG + r) * NW + (c >> 5)] >> (c & 31)) & 1u) << r;
+      uint16_t lastx = 0;
+      if (bits) lastx = *reinterpret_cast<const uint16_t*>(sm + OFF_Q + elem_off(seg * SEG + 31 - __clz(bits)));
+      s_lastx[seg * D + c] = lastx;
+      s_has[seg * D + c] = bits != 0u;
+      asm volatile("bar.sync 5, %0;" ::"n"(NCTHR) : "memory");
+      const __nv_bfloat16 snap16 = __float2bfloat16_rn(snap);        // exact: a copy of an input element or 0
+      uint16_t cur = *reinterpret_cast<const uint16_t*>(&snap16);
+      for (int s2 = 0; s2 < seg; ++s2) cur = s_has[s2 * D + c] ? s_lastx[s2 * D + c] : cur;
+#pragma unroll
+      for (int r = 0; r < SEG; ++r) {
+        const uint32_t off = elem_off(seg * SEG + r);
+        const uint16_t x = *reinterpret_cast<const uint16_t*>(sm + OFF_Q + off);
+        cur = ((bits >> r) & 1u) ? x : cur;
+        *reinterpret_cast<uint16_t*>(sm + OFF_QH + off) = cur;
+      }
+      fence_proxy_async();      // the tile was written through the generic proxy, the tensor cores read it
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(BAR_QH));
     }
 
     for (int jt = 0; jt <= qt; ++jt) {
@@ -410,6 +463,9 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
   TqParams p;
   p.out = (__nv_bfloat16*)out;
   p.counters = w.counters;
+  p.mask = w.mask;
+  p.qhat_tile = w.qhat_tile;
+  p.T_max = s.T_max; p.n_tiles64 = s.n_tiles;
   p.T = T; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
   p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const dim3 grid((unsigned)BH, (T + BM - 1) / BM);
