@@ -306,9 +306,8 @@ def run_ours(args):
     roofline = k2_roofline(w, stats, kernel, kmean[2], peaks, n_sm)
     # K1 is a streaming pass: report it against the HBM copy bandwidth as well
     es = 2 if w.dtype == "bf16" else 4
-    # chain kernel: reads Q, writes delta values (fp32), mask words and, for the telescoped
-    # attention kernel, the reference rows (bf16)
-    k1_bytes = w.B * w.H * w.T * (w.d * (es + 4) + w.d // 8 + (w.d * 2 if kernel == 2 else 0))
+    # chain kernel (query deltas): reads Q, writes the mask words
+    k1_bytes = w.B * w.H * w.T * (w.d * es + w.d // 8)
     k1 = {"kernel": "delta_chain", "bound": "hbm", "kernel_ms": kmean[0],
           "achieved": k1_bytes / (kmean[0] * 1e-3) / 1e9, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
           "frac": k1_bytes / (kmean[0] * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
@@ -335,6 +334,8 @@ def run_ours(args):
         line["e2e"] = run_e2e(args, B, torch, w, tens, theta)
         line["theta_sweep"] = run_sweep(args, B, torch, w, q, k, v, out, st, flush)
         line["decode"] = run_decode(args, B, torch, peaks)
+        line["key_deltas"] = run_key_deltas(args, B, torch, w, tens, theta, flush, peaks)
+        line["delta_pass_large"] = run_delta_pass_large(B, torch, peaks, flush)
         line["cpu_baseline"] = run_cpu_baseline(args, w, tens, theta)
     print(json.dumps(line))
     if dist is not None:
@@ -424,14 +425,17 @@ def run_sweep(args, B, torch, w, q, k, v, out, st, flush):
     return res
 
 
-def run_decode(args, B, torch, peaks):
-    """Decode leg: cache prefilled to 2048 tokens, then 256 steps; batch 1 and 16."""
+def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_b1", "llama32_1b_decode_b16")):
+    """Decode leg: cache prefilled to 2048 tokens, then 256 steps; batch 1 and 16.
+    source="key": the paper's adopted strategy (3) (key deltas; the carried state is the reference key)."""
     res = {}
-    for name in ("llama32_1b_decode_b1", "llama32_1b_decode_b16"):
+    key = source == "key"
+    for name in names:
         w = WL.WORKLOADS[name]
         theta = w.thetas[0]
         tens = WL.make_qkv(w)
-        cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T_max, w.dtype, prefill_window=B.DELTA_WIN_SLIDING)
+        cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T_max, w.dtype, prefill_window=B.DELTA_WIN_SLIDING,
+                            source=B.DELTA_SRC_KEY if key else B.DELTA_SRC_QUERY)
         st = B.delta_state_init(cfg)
         q = to_dev(tens["q"], w.dtype, torch)
 
@@ -487,7 +491,8 @@ def run_decode(args, B, torch, peaks):
             graph_ok = f"capture failed: {type(ex).__name__}"
         es = 2
         n_avg = w.T + (w.n_decode - 1) / 2.0
-        bytes_step = w.B * (2 * w.H_kv * n_avg * w.d * es + 2 * w.H * n_avg * 4)
+        # K (or reference-key) and V rows once per KV head; query deltas also read and write the score row R
+        bytes_step = w.B * (2 * w.H_kv * n_avg * w.d * es + (0 if key else 2 * w.H * n_avg * 4))
         best = graph_us if graph_us else min(eager)
         gbs = bytes_step / (best * 1e-6) / 1e9
         res[f"batch{w.B}"] = {
@@ -504,6 +509,68 @@ def run_decode(args, B, torch, peaks):
         del st, q, kc, vc, qd, kd, vd, od
         torch.cuda.empty_cache()
     return res
+
+
+def run_key_deltas(args, B, torch, w, tens, theta, flush, peaks):
+    """The paper's adopted strategy (3) on the same inputs: key stream thresholded per KV head."""
+    q, k, v = (to_dev(tens[n], w.dtype, torch) for n in ("q", "k", "v"))
+    out = torch.empty_like(q)
+    st = B.delta_state_init(B.make_config(w.B, w.H, w.H_kv, w.d, w.T, w.dtype, source=B.DELTA_SRC_KEY))
+    ms = []
+    for i in range(3 + min(args.steps, 20)):
+        flush.zero_()
+        B.delta_state_reset(st)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            ms.append(e0.elapsed_time(e1))
+    stt = B.delta_sparsity_stats(st)["prefill"]
+    return {"prefill": {"theta": theta, "ms_per_step": statistics.mean(ms),
+                        "tokens_per_s": w.B * w.T / (statistics.mean(ms) * 1e-3), "S_m": stt["S_m"],
+                        "S_c_exact": stt["S_c_exact"]},
+            "decode": run_decode(args, B, torch, peaks, source="key", names=("llama32_1b_decode_b16",))}
+
+
+def run_delta_pass_large(B, torch, peaks, flush):
+    """Delta construction at the size of one layer of the 16-layer stack configuration
+    (batch 8, T = 4096: 16384 chains per mask word), where the pass is bandwidth- rather than
+    latency-bound: chain and finish kernel times and their algorithmic HBM rates."""
+    w = WL.WORKLOADS["llama32_1b_stack_layer"]
+    theta = 0.2
+    tens = WL.make_qkv(w, n_decode=0)
+    q, k, v = (to_dev(tens[n], w.dtype, torch) for n in ("q", "k", "v"))
+    out = torch.empty_like(q)
+    st = B.delta_state_init(B.make_config(w.B, w.H, w.H_kv, w.d, w.T, w.dtype))
+    B.delta_state_enable_profiling(st, True)
+    kms, steps = [], []
+    for i in range(5):
+        flush.zero_()
+        B.delta_state_reset(st)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            kms.append(B.delta_state_prefill_kernel_ms(st)); steps.append(e0.elapsed_time(e1))
+    stt = B.delta_sparsity_stats(st)["prefill"]
+    n = w.B * w.H * w.T
+    chain_b = n * (w.d * 2 + w.d // 8)                                   # Q read, mask written
+    finish_b = n * (w.d * 2 + w.d // 8 + w.d * 4 + w.d + 2) + 2 * w.B * w.H_kv * w.T * w.d * 2 + n * 4
+    hbm = float(peaks["hbm_gbs"])
+    cm, fm = statistics.mean(x[0] for x in kms), statistics.mean(x[1] for x in kms)
+    am = statistics.mean(x[2] for x in kms)
+    N_c = w.T * (w.T + 1) // 2
+    return {"workload": w.name, "theta": theta, "S_m": stt["S_m"], "ms_per_layer": statistics.mean(steps),
+            "tokens_per_s": w.B * w.T / (statistics.mean(steps) * 1e-3),
+            "delta_chain": {"ms": cm, "bound": "hbm", "achieved": chain_b / (cm * 1e-3) / 1e9, "peak": hbm,
+                            "unit": "GB/s", "frac": chain_b / (cm * 1e-3) / 1e9 / hbm},
+            "delta_finish": {"ms": fm, "bound": "hbm", "achieved": finish_b / (fm * 1e-3) / 1e9, "peak": hbm,
+                             "unit": "GB/s", "frac": finish_b / (fm * 1e-3) / 1e9 / hbm},
+            "hybrid_attn": {"ms": am, "dense_equiv_tflops": 4.0 * w.d * N_c * w.B * w.H / (am * 1e-3) / 1e12}}
 
 
 def run_cpu_baseline(args, w, tens, theta):
