@@ -39,7 +39,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the hybrid-attention kernel on the
 # headline workload, from the ncu captures summarised under profiles/ (absent = not captured
 # since the kernel last changed).
-K2_DRAM_TRAFFIC_BYTES = {2: 10526208, 1: 17161728}   # per kernel id
+K2_DRAM_TRAFFIC_BYTES = {2: 6664448, 1: 17161728}   # per kernel id
 
 
 def load_peaks():
@@ -586,6 +586,20 @@ def run_cpu_baseline(args, w, tens, theta):
             "sample": f"{len(heads)} of {w.H} heads x {len(reps)} repeats, full T={w.T}; extrapolated by head count"}
 
 
+def run_only(args):
+    """One secondary leg alone: the decode leg at one batch size, or one prefill of the stack-layer shape."""
+    import torch
+    from paper_2507_19608_b200 import binding as B
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    if args.only == "stack_layer":
+        flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+        res = run_delta_pass_large(B, torch, peaks, flush)
+    else:
+        res = run_decode(args, B, torch, peaks, names=("llama32_1b_" + args.only,))
+    print(json.dumps({"only": args.only, "result": res}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -596,10 +610,14 @@ def main():
     ap.add_argument("--theta", type=float, default=HEADLINE_THETA)
     ap.add_argument("--kernel", type=int, default=-1, help="-1 auto, 0 generic, 1 tcgen05 + FP32 delta path, 2 tcgen05 telescoped")
     ap.add_argument("--quick", action="store_true", help="prefill timing only (used for ncu launch lists)")
+    ap.add_argument("--only", default="", choices=["", "decode_b1", "decode_b16", "stack_layer"],
+                    help="run one secondary leg alone on one GPU (small ncu captures of its kernels)")
     ap.add_argument("--ref-heads", type=int, default=4, help="heads per reference step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.only:
+        run_only(args)
     else:
         run_ours(args)
 
