@@ -76,6 +76,7 @@ static void carve(const delta_config_t& c, char* base, Workspace* w) {
   w->tile_nnz = (uint32_t*)take(BH * nt * 4);
   w->idx = (uint8_t*)take(BH * c.T_max * c.d);
   w->qhat_tile = (float*)take(BH * nt * c.d * 4);
+  w->ckpt = (float*)take(BH * (((size_t)c.T_max + DELTA_CKPT_ROWS - 1) / DELTA_CKPT_ROWS) * c.d * 4);
   w->qhat[0] = (float*)take(BH * c.d * 4);
   w->qhat[1] = (float*)take(BH * c.d * 4);
   w->R = (float*)take(BH * c.T_max * 4);
@@ -233,14 +234,10 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   const bool use_tc = which == 1;
   const bool key = c.source == DELTA_SRC_KEY;
   if (key && which != 2) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
-  MARK(0);
-  // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
-  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, key, cs)) !=
-      cudaSuccess)
-    return cuda_fail(e);
-  // The telescoped attention kernel reads nothing the finish kernel writes (counts, indices,
-  // counters, hand-off row), so the two run side by side: finish on the state's side stream
-  // between a fork and a join event.  With per-kernel timing on, everything stays in line.
+  // The telescoped attention kernel reads nothing the finish kernel writes (delta values,
+  // counts, indices, counters, hand-off row), so the two run side by side: finish on the
+  // state's side stream between a fork and a join event.  With per-kernel timing on,
+  // everything stays in line on the caller's stream.
   const bool fork = (which == 2) && !prof;
   if (fork && !st->side) {
     if ((e = cudaStreamCreateWithFlags(&st->side, cudaStreamNonBlocking)) != cudaSuccess ||
@@ -248,28 +245,34 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
         (e = cudaEventCreateWithFlags(&st->ev_join, cudaEventDisableTiming)) != cudaSuccess)
       return cuda_fail(e);
   }
-  cudaStream_t fs = cs;
+  MARK(0);
+  // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
+  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, key, cs)) != cudaSuccess)
+    return cuda_fail(e);
+  auto attention = [&]() -> cudaError_t {
+    if (use_tc) return launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
+    if (which == 2)
+      return launch_hybrid_attn_tcq(st->shape, st->ws, q, k, v, out, T, theta, c.init, window, c.prefill_window, key,
+                                    cs);
+    return launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, c.dtype, cs);
+  };
   if (fork) {
     if ((e = cudaEventRecord(st->ev_fork, cs)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(st->side, st->ev_fork, 0)) != cudaSuccess) return cuda_fail(e);
-    fs = st->side;
-  }
-  MARK(1);
-  if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, window, c.prefill_window, c.dtype, c.init, use_tc, key, fs)) !=
-      cudaSuccess)
-    return cuda_fail(e);
-  if (fork && (e = cudaEventRecord(st->ev_join, st->side)) != cudaSuccess) return cuda_fail(e);
-  MARK(2);
-  if (use_tc) {
-    e = launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
-  } else if (which == 2) {
-    e = launch_hybrid_attn_tcq(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, key, cs);
+    if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
+                                 use_tc, key, st->side)) != cudaSuccess)
+      return cuda_fail(e);
+    if ((e = cudaEventRecord(st->ev_join, st->side)) != cudaSuccess) return cuda_fail(e);
+    if ((e = attention()) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(cs, st->ev_join, 0)) != cudaSuccess) return cuda_fail(e);
   } else {
-    e = launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window,
-                                   c.dtype, cs);
+    MARK(1);
+    if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
+                                 use_tc, key, cs)) != cudaSuccess)
+      return cuda_fail(e);
+    MARK(2);
+    if ((e = attention()) != cudaSuccess) return cuda_fail(e);
   }
-  if (e != cudaSuccess) return cuda_fail(e);
-  if (fork && (e = cudaStreamWaitEvent(cs, st->ev_join, 0)) != cudaSuccess) return cuda_fail(e);
   MARK(3);
   MARK(4);
 #undef MARK

@@ -20,6 +20,7 @@ enum CounterSlot {
   CNT_TOTAL = CNT_SLOTS + 4 * CNT_SHARDS
 };
 
+constexpr int DELTA_CKPT_ROWS = 8;     // the chain kernel leaves its reference every 8 rows
 constexpr int kMaxDecodeSplits = 64;   // split-KV partials per (batch, KV head)
 constexpr int kDecodeChunkMax = 1024;  // keys per decode CTA (scores live in shared memory)
 
@@ -31,6 +32,7 @@ struct Workspace {
   uint32_t* tile_nnz;   // [B,H,n_tiles]
   uint8_t* idx;         // [B,H,T_max,d]
   float* qhat_tile;     // [B,H,n_tiles,d]
+  float* ckpt;          // [B,H,ceil(T_max/8),d] reference in front of every 8-row block (query deltas)
   float* qhat[2];       // [B,H,d] ping-pong (decode reads one, writes the other)
   float* R;             // [B,H,T_max]
   unsigned long long* counters;  // [CNT_TOTAL]
@@ -45,21 +47,24 @@ struct Workspace {
 struct Shape {
   int B, H, H_kv, d, T_max, n_tiles;
   int g() const { return H / H_kv; }
+  int n_ckpt() const { return (T_max + DELTA_CKPT_ROWS - 1) / DELTA_CKPT_ROWS; }
 };
 
 void count_launch(int n = 1);
 
-// K1a: token-sequential delta chain over the query stream (Eq. 2-3): delta values, mask words,
-// per-tile reference snapshots, final reference.
+// K1a: token-sequential delta chain (Eq. 2-3).  Query stream: the reference in front of every
+// 8-row block and every 64-row tile, final reference.  Key stream: also delta values, mask
+// words and reference rows.
 // key_stream: the stream is K in the KV-cache layout, one chain set per KV head (strategy 3).
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
                                float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
                                cudaStream_t st);
-// K1b: row-parallel finish: counts, compacted indices, Eq. 6 counters, the decode hand-off row
+// K1b: row-parallel finish: (query stream) delta values and mask words from the 8-row
+// checkpoints; counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
-                                int window, int shape, int dtype, int init, bool want_kt, bool key_stream,
-                                cudaStream_t st);
+                                float theta, int window, int shape, int dtype, int init, bool want_kt,
+                                bool key_stream, cudaStream_t st);
 // K2 (generic): fused hybrid attention on CUDA cores, any supported dtype.
 cudaError_t launch_hybrid_attn_generic(const Shape& s, const Workspace& w, const void* q,
                                        const void* k, const void* v, void* out, int T, int window,

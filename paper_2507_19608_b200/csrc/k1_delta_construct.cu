@@ -1,22 +1,27 @@
-// K1 -- delta construction over the query stream (Section II-C, Eq. 2-3; Section III-A
-// strategy (1)), in two kernels.
+// K1 -- delta construction (Section II-C, Eq. 2-3; Section III-A strategies (1) and (3)), in
+// two kernels.
 //
 // delta_chain_kernel: the token-sequential part.  Eq. 3 makes every channel a chain along the
 // tokens (the reference is the last value that fired), so the only parallelism is across
 // channels: one thread per channel, one warp per 32 channels (= one mask word), one CTA per
-// (batch, head).  The chain itself is three dependent FP32 operations per token; everything
-// else is kept off it: a producer warp streams the head's query rows into a ring of
-// shared-memory stages with bulk asynchronous copies (the rows do not depend on the carried
-// state), delta values leave with one coalesced store per row, every thread collects its
-// channel's fire bits of 32 rows in one register and a 32 x 32 bit transpose across the warp
-// (five shuffles) turns them into the 32 rows' mask words.
+// (batch, head).  The chain itself is three dependent FP32 operations per token and a lone
+// warp issues slowly, so everything else is kept off it: a producer warp streams the head's
+// rows into a ring of shared-memory stages with bulk asynchronous copies (the rows do not
+// depend on the carried state), and for the query stream the chain warps store nothing but
+// the reference in front of every 8-row block (and every 64-row tile, and the final one).
+// Given those checkpoints every 8-row block of Eq. 2-3 is independent of the others: fire
+// bits, delta values, mask words and reference rows are recomputed from them by row-parallel
+// code (the finish kernel below, the attention kernel for its own query tile).
+// For the key stream (strategy 3) the chain kernel still stores delta values, reference rows
+// and mask words itself (fire bits of 32 rows in one register per thread, a 32 x 32 bit
+// transpose across the warp turns them into the rows' mask words).
 //
-// delta_finish_kernel: everything that is parallel over rows once the mask exists -- the delta
-// values themselves (query deltas), per-row and per-tile non-zero counts, the compacted channel
-// indices, the counters behind Eq. 6 --
+// delta_finish_kernel: everything that is parallel over rows -- (query stream) Eq. 2-3 over
+// 8-row blocks from the checkpoints: delta values and mask words; per-row and per-tile
+// non-zero counts, the compacted channel indices, the counters behind Eq. 6 --
 // plus two passes over the keys that prefill needs anyway: the hand-off row
-// R(T-1)[j] = q_hat(T-1).k_j for decode and, for the tensor-core attention kernel, the
-// channel-major fp32 copy of the keys.
+// R(T-1)[j] = q_hat(T-1).k_j for decode and, for the tensor-core attention kernel with the
+// FP32 delta path, the channel-major fp32 copy of the keys.
 #include "delta_internal.cuh"
 
 namespace delta {
@@ -50,6 +55,95 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   return true;
 }
 
+
+
+// One element of the staged rows by shared-memory address, widened to fp32.
+template <typename TIn> __device__ __forceinline__ float lds_elem(uint32_t addr);
+template <> __device__ __forceinline__ float lds_elem<float>(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+template <> __device__ __forceinline__ float lds_elem<__nv_bfloat16>(uint32_t addr) {
+  uint32_t u;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=r"(u) : "r"(addr));
+  return __uint_as_float(u << 16);
+}
+
+// One ring stage of the chain for one thread (= one channel): rows t0 .. t0+nrows-1, the
+// thread's values at rows[r * D]; updates the reference qh.
+// EMIT = false (query deltas): the sequential kernel carries nothing but the reference and,
+// with `write`, leaves it in front of every 8-row block (ckptp); fire bits, delta values and
+// everything derived from them are recomputed from those checkpoints by row-parallel kernels.
+// EMIT = true (key deltas): with `write` stores the stage's mask words, delta values and
+// reference rows itself.
+template <typename TIn, int D, bool EMIT>
+__device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, bool basis_row, bool write,
+                                            float& qh, float theta, int lane, float* dqp,
+                                            __nv_bfloat16* qrp, uint32_t* maskp, float* ckptp) {
+  constexpr int NW = D / 32;
+  // bit r of `bits`: did this thread's channel fire in row t0 + r
+  uint32_t bits = 0;
+  if (nrows == RC && !basis_row) {
+    // full stage, no basis row: all loads first, then nothing but the dependent chain
+    // (volatile loads: the compiler may not sink them into the chain, where their latency
+    // would sit on the dependent path)
+    float x[RC];
+    const uint32_t saddr = smem_u32(rows);
+#pragma unroll
+    for (int r = 0; r < RC; ++r) x[r] = lds_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
+#pragma unroll
+    for (int r = 0; r < RC; ++r) {
+      if (!EMIT && write && (r % DELTA_CKPT_ROWS) == 0) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
+      const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
+      qh = fire ? x[r] : qh;
+      if (EMIT) {
+        if (write) {
+          dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
+          if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
+        }
+        bits |= fire ? (1u << r) : 0u;
+      }
+    }
+  } else {
+    for (int r = 0; r < nrows; ++r) {
+      if (!EMIT && write && ((t0 + r) % DELTA_CKPT_ROWS) == 0) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      const float x = to_f32(rows[r * D]);
+      bool fire;
+      float delta;
+      if (r == 0 && basis_row) {
+        fire = true;                                 // the basis vector is kept whole
+        delta = x;
+      } else {
+        const float diff = __fsub_rn(x, qh);
+        fire = fabsf(diff) > theta;
+        delta = fire ? diff : 0.0f;
+      }
+      qh = fire ? x : qh;
+      if (EMIT) {
+        if (write) {
+          dqp[(size_t)(t0 + r) * D] = delta;
+          if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
+        }
+        bits |= fire ? (1u << r) : 0u;
+      }
+    }
+  }
+  if (!EMIT || !write) return;
+  // 32 x 32 bit transpose across the warp: lane r ends up with the mask word of row t0 + r
+  uint32_t mymask = bits;
+#pragma unroll
+  for (int j = 16; j > 0; j >>= 1) {
+    const uint32_t km = (j == 16) ? 0x0000FFFFu : (j == 8) ? 0x00FF00FFu : (j == 4) ? 0x0F0F0F0Fu
+                      : (j == 2) ? 0x33333333u : 0x55555555u;
+    const uint32_t other = __shfl_xor_sync(0xffffffffu, mymask, j);
+    mymask = (lane & j) ? (((other >> j) & km) | (mymask & ~km))
+                        : ((mymask & km) | ((other & km) << j));
+  }
+  if (lane < nrows) maskp[(size_t)(t0 + lane) * NW] = mymask;
+}
+
 }  // namespace
 
 // EMIT: also store the delta values and the reference rows (key deltas); without it the chain
@@ -58,8 +152,9 @@ template <typename TIn, int D, bool EMIT>
 __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     const TIn* __restrict__ q, float* __restrict__ dq, uint32_t* __restrict__ mask,
     float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
-    __nv_bfloat16* __restrict__ qhat_rows, unsigned long long* __restrict__ counters, int T,
-    int T_max, int n_tiles, float theta, int basis_exact, int src_rows) {
+    __nv_bfloat16* __restrict__ qhat_rows, float* __restrict__ ckpt,
+    unsigned long long* __restrict__ counters, int T, int T_max, int n_tiles, int n_ckpt, float theta,
+    int basis_exact, int src_rows) {
   // q: the stream that becomes the delta matrix, [heads][src_rows][D] with rows 0..T-1 read
   // (queries: src_rows = T; keys in the KV-cache layout: src_rows = T_max)
   constexpr int NW = D / 32;                       // chain warps = mask words per row
@@ -110,77 +205,30 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     float* dqp = dq ? dq + (size_t)bh * T_max * D + c : nullptr;   // null: values left to the finish kernel
     __nv_bfloat16* qrp = qhat_rows ? qhat_rows + (size_t)bh * T_max * D + c : nullptr;
     uint32_t* maskp = mask + (size_t)bh * T_max * NW + warp;
+    float* ckptp = ckpt ? ckpt + (size_t)bh * n_ckpt * D + c : nullptr;
     float qh = 0.0f;          // reference state, starts at zero (Eq. 3)
     bool failed = false;
     for (int i = 0; i < n_chunks; ++i) {
       const int s = i % NS;
       const int t0 = i * RC;
-      if ((t0 % DELTA_TILE_ROWS) == 0)
+      if (qhat_tile && (t0 % DELTA_TILE_ROWS) == 0)
         qhat_tile[((size_t)bh * n_tiles + t0 / DELTA_TILE_ROWS) * D + c] = qh;
       if (!mbar_wait(full0 + 8 * s, (i / NS) & 1)) { failed = true; break; }
       const TIn* rows = reinterpret_cast<const TIn*>(ring + (size_t)s * STAGE_BYTES) + c;
       const int nrows = min(RC, T - t0);
-      // bit r of `bits`: did this thread's channel fire in row t0 + r
-      uint32_t bits = 0;
-      if (nrows == RC && !(t0 == 0 && basis_exact)) {
-        // full stage, no basis row: all loads first, then nothing but the dependent chain,
-        // its store and one bit per row
-        float x[RC];
-#pragma unroll
-        for (int r = 0; r < RC; ++r) x[r] = to_f32(rows[r * D]);
-#pragma unroll
-        for (int r = 0; r < RC; ++r) {
-          const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
-          const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
-          qh = fire ? x[r] : qh;
-          if (EMIT) {
-            dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
-            if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
-          }
-          bits |= fire ? (1u << r) : 0u;
-        }
-      } else {
-        for (int r = 0; r < nrows; ++r) {
-          const float x = to_f32(rows[r * D]);
-          bool fire;
-          float delta;
-          if (t0 + r == 0 && basis_exact) {
-            fire = true;                                 // the basis vector is kept whole
-            delta = x;
-          } else {
-            const float diff = __fsub_rn(x, qh);
-            fire = fabsf(diff) > theta;
-            delta = fire ? diff : 0.0f;
-          }
-          qh = fire ? x : qh;
-          if (EMIT) {
-            dqp[(size_t)(t0 + r) * D] = delta;
-            if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
-          }
-          bits |= fire ? (1u << r) : 0u;
-        }
-      }
-      // 32 x 32 bit transpose across the warp: lane r ends up with the mask word of row t0 + r
-      uint32_t mymask = bits;
-#pragma unroll
-      for (int j = 16; j > 0; j >>= 1) {
-        const uint32_t km = (j == 16) ? 0x0000FFFFu : (j == 8) ? 0x00FF00FFu : (j == 4) ? 0x0F0F0F0Fu
-                          : (j == 2) ? 0x33333333u : 0x55555555u;
-        const uint32_t other = __shfl_xor_sync(0xffffffffu, mymask, j);
-        mymask = (lane & j) ? (((other >> j) & km) | (mymask & ~km))
-                            : ((mymask & km) | ((other & km) << j));
-      }
-      if (lane < nrows) maskp[(size_t)(t0 + lane) * NW] = mymask;
+      chain_stage<TIn, D, EMIT>(rows, t0, nrows, t0 == 0 && basis_exact, true, qh, theta, lane, dqp, qrp, maskp,
+                                ckptp);
       __syncwarp();
       if (lane == 0)
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * s) : "memory");
     }
-    if (!failed) qhat_out[(size_t)bh * D + c] = qh;
+    if (!failed && qhat_out) qhat_out[(size_t)bh * D + c] = qh;
     if (failed) s_fail = 1;
   }
   __syncthreads();
   if (tid == 0 && s_fail) atomicMax(&counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
 }
+
 
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
                                float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
@@ -189,6 +237,9 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
   // query deltas: the chain leaves mask words and per-tile references only; delta values are
   // recomputed row-parallel by the finish kernel.  Key deltas: the chain stores them itself.
   float* dq_out = key_stream ? w.dq : nullptr;
+  float* ckpt_out = key_stream ? nullptr : w.ckpt;
+  float* tile_out = w.qhat_tile;
+  float* fin_out = w.qhat[0];
   const int grid = s.B * (key_stream ? s.H_kv : s.H);
   const int src_rows = key_stream ? s.T_max : T;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
@@ -201,8 +252,9 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
       err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
       if (err != cudaSuccess) return err;                                                        \
     }                                                                                            \
-    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, dq_out, w.mask, w.qhat_tile, w.qhat[0], qrows, \
-                                      w.counters, T, s.T_max, s.n_tiles, theta, basis, src_rows); \
+    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, dq_out, w.mask, tile_out, fin_out, qrows, \
+                                      ckpt_out, w.counters, T, s.T_max, s.n_tiles, s.n_ckpt(), theta, \
+                                      basis, src_rows);                                          \
   } while (0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
@@ -223,14 +275,14 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 //       R(T-1)[j] = q_hat(T-1).k_j for the heads of the group, and the channel-major fp32 key
 //       copy when kt != nullptr.
 template <typename TIn, int D>
-__global__ void __launch_bounds__(256, 4) delta_finish_kernel(
-    const uint32_t* __restrict__ mask, uint16_t* __restrict__ row_nnz,
+__global__ void __launch_bounds__(256, 5) delta_finish_kernel(
+    uint32_t* __restrict__ mask, uint16_t* __restrict__ row_nnz,
     uint32_t* __restrict__ tile_nnz, uint8_t* __restrict__ idx,
     unsigned long long* __restrict__ counters, const TIn* __restrict__ k,
     const float* __restrict__ qhat, float* __restrict__ R, float* __restrict__ kt, int T,
     int T_max, int n_tiles, int BH, int H, int g, int W, int shape, int n_idx_blocks, int kt_ld,
     int key_stream, const TIn* __restrict__ q, float* __restrict__ dq,
-    const float* __restrict__ qhat_tile, int basis_exact) {
+    const float* __restrict__ ckpt, int n_ckpt, float theta, int basis_exact) {
   constexpr int NW = D / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if ((int)blockIdx.x < n_idx_blocks) {
@@ -242,9 +294,51 @@ __global__ void __launch_bounds__(256, 4) delta_finish_kernel(
     const int rows = min(DELTA_TILE_ROWS, T - t0);
     const int r_mine = warp * 8 + (lane & 7);        // lanes 0..7 hold one row each
     uint32_t mw[NW];
+    if (ckpt != nullptr) {
+      // query deltas: the chain kernel left only the reference in front of every 8-row block.
+      // The warp re-runs Eq. 2-3 over its 8 rows (lane = channel of a mask word): delta values,
+      // and one ballot per row for the mask word.
+      const int rbase = t0 + warp * 8;
 #pragma unroll
-    for (int w2 = 0; w2 < NW; ++w2)
-      mw[w2] = (r_mine < rows) ? mask[((size_t)bh * T_max + t0 + r_mine) * NW + w2] : 0u;
+      for (int w2 = 0; w2 < NW; ++w2) {
+        const int c = w2 * 32 + lane;
+        uint32_t word_mine = 0;
+        if (rbase < T) {
+          float ref = ckpt[((size_t)bh * n_ckpt + rbase / DELTA_CKPT_ROWS) * D + c];
+          float x[8];
+#pragma unroll
+          for (int r = 0; r < 8; ++r)
+            x[r] = (rbase + r < T) ? to_f32(q[((size_t)bh * T + rbase + r) * D + c]) : 0.0f;
+#pragma unroll
+          for (int r = 0; r < 8; ++r) {
+            const bool live = rbase + r < T;
+            bool fire;
+            float delta;
+            if (rbase + r == 0 && basis_exact) {
+              fire = true;                               // the basis vector is kept whole
+              delta = x[r];
+            } else {
+              const float diff = __fsub_rn(x[r], ref);
+              fire = fabsf(diff) > theta;
+              delta = fire ? diff : 0.0f;
+            }
+            fire = fire && live;
+            if (live) {
+              dq[((size_t)bh * T_max + rbase + r) * D + c] = delta;
+              ref = fire ? x[r] : ref;
+            }
+            const uint32_t word = __ballot_sync(0xffffffffu, fire);
+            if ((lane & 7) == r) word_mine = word;
+          }
+        }
+        mw[w2] = word_mine;
+        if (lane < 8 && r_mine < rows) mask[((size_t)bh * T_max + t0 + r_mine) * NW + w2] = word_mine;
+      }
+    } else {
+#pragma unroll
+      for (int w2 = 0; w2 < NW; ++w2)
+        mw[w2] = (r_mine < rows) ? mask[((size_t)bh * T_max + t0 + r_mine) * NW + w2] : 0u;
+    }
     unsigned long long done = 0, dense = 0, tsum = 0;
     if (lane < 8 && r_mine < rows) {
       int nnz = 0;
@@ -301,48 +395,6 @@ __global__ void __launch_bounds__(256, 4) delta_finish_kernel(
       uint4* dst = reinterpret_cast<uint4*>(idx + ((size_t)bh * T_max + t0 + warp * 8) * D);
       const uint4* src = reinterpret_cast<const uint4*>(srow);
       for (int e = lane; e < my_rows * D / 16; e += 32) dst[e] = src[e];
-    }
-    // delta values of the tile (query deltas; with key deltas the chain kernel stores them).
-    // With the mask known the reference in front of a row is the last fired row below it, so a
-    // 64-row tile splits into row segments: thread (channel, segment) finds its segment's last
-    // fired value, takes the nearest earlier one (or the reference in front of the tile) as
-    // carry-in and walks its rows with one select per row.
-    if (dq != nullptr) {
-      constexpr int NSEG = 256 / D, SEG = DELTA_TILE_ROWS / NSEG;   // 4 x 16 rows (d=64), 2 x 32 (d=128)
-      __shared__ uint32_t s_mask[DELTA_TILE_ROWS][NW];
-      __shared__ float s_lastx[NSEG][D];
-      __shared__ uint8_t s_has[NSEG][D];
-      for (int e = tid; e < DELTA_TILE_ROWS * NW; e += 256) {
-        const int r = e / NW;
-        s_mask[r][e - r * NW] = (r < rows) ? mask[((size_t)bh * T_max + t0 + r) * NW + (e - r * NW)] : 0u;
-      }
-      const int c = tid % D, seg = tid / D;
-      const TIn* qp0 = q + ((size_t)bh * T + t0 + seg * SEG) * D + c;
-      float x[SEG];
-#pragma unroll
-      for (int r = 0; r < SEG; ++r) x[r] = (seg * SEG + r < rows) ? to_f32(qp0[(size_t)r * D]) : 0.0f;
-      __syncthreads();
-      uint32_t bits = 0;      // bit r: channel c fired in row seg*SEG + r
-#pragma unroll
-      for (int r = 0; r < SEG; ++r) bits |= ((s_mask[seg * SEG + r][c >> 5] >> (c & 31)) & 1u) << r;
-      float lastx = 0.0f;
-#pragma unroll
-      for (int r = 0; r < SEG; ++r) lastx = ((bits >> r) & 1u) ? x[r] : lastx;
-      s_lastx[seg][c] = lastx;
-      s_has[seg][c] = bits != 0u;
-      __syncthreads();
-      float ref = qhat_tile[((size_t)bh * n_tiles + tile) * D + c];   // reference in front of the tile
-      for (int s2 = 0; s2 < seg; ++s2) ref = s_has[s2][c] ? s_lastx[s2][c] : ref;
-      float* dqp = dq + ((size_t)bh * T_max + t0 + seg * SEG) * D + c;
-#pragma unroll
-      for (int r = 0; r < SEG; ++r) {
-        if (seg * SEG + r < rows) {
-          const bool fire = (bits >> r) & 1u;
-          const float diff = (t0 + seg * SEG + r == 0 && basis_exact) ? x[r] : __fsub_rn(x[r], ref);
-          dqp[(size_t)r * D] = fire ? diff : 0.0f;
-          ref = fire ? x[r] : ref;
-        }
-      }
     }
     __syncthreads();
     if (tid == 0) {
@@ -407,8 +459,8 @@ __global__ void __launch_bounds__(256, 4) delta_finish_kernel(
 }
 
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
-                                int window, int shape, int dtype, int init, bool want_kt, bool key_stream,
-                                cudaStream_t st) {
+                                float theta, int window, int shape, int dtype, int init, bool want_kt,
+                                bool key_stream, cudaStream_t st) {
   // key deltas: the index/counter pass runs over the KV heads and there is no hand-off row
   const int BH = s.B * (key_stream ? s.H_kv : s.H);
   const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
@@ -416,11 +468,17 @@ cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* 
   const int n_key_blocks = key_stream ? 0 : s.B * s.H_kv * ((T + 63) / 64);
   const int kt_ld = (s.T_max + 3) / 4 * 4;
   float* kt = (want_kt && w.kt) ? w.kt : nullptr;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(n_idx_blocks + n_key_blocks));
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaError_t err = cudaSuccess;
 #define LAUNCH(TIN, DD)                                                                          \
-  delta_finish_kernel<TIN, DD><<<n_idx_blocks + n_key_blocks, 256, 0, st>>>(                     \
-      w.mask, w.row_nnz, w.tile_nnz, w.idx, w.counters, (const TIN*)k, w.qhat[0], w.R, kt, T,    \
+  err = cudaLaunchKernelEx(&cfg, delta_finish_kernel<TIN, DD>,                                   \
+      w.mask, w.row_nnz, w.tile_nnz, w.idx, w.counters, (const TIN*)k, (const float*)w.qhat[0], w.R, kt, T,    \
       s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld, key_stream ? 1 : 0,   \
-      key_stream ? nullptr : (const TIN*)q, key_stream ? nullptr : w.dq, w.qhat_tile,                \
+      key_stream ? (const TIN*)nullptr : (const TIN*)q, key_stream ? (float*)nullptr : w.dq,      \
+      key_stream ? (const float*)nullptr : (const float*)w.ckpt, s.n_ckpt(), theta,               \
       init == DELTA_INIT_BASIS_EXACT ? 1 : 0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
@@ -429,7 +487,7 @@ cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* 
   }
 #undef LAUNCH
   count_launch();
-  return cudaGetLastError();
+  return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 }  // namespace delta

@@ -54,10 +54,7 @@ template <int D> struct TqSmem {
   static constexpr uint32_t OFF_V = OFF_K + NKBUF * SZ_TILE;   // two buffers
   static constexpr uint32_t OFF_P = OFF_V + 2 * SZ_TILE;       // bf16 [2][128 rows][64 keys]
   static constexpr uint32_t OFF_PMAX = OFF_P + 2 * SZ_BLK;     // fp32 [2][128 rows][4 quarters]
-  static constexpr uint32_t OFF_MASK = OFF_PMAX + 2 * 128 * 4 * 4;     // u32 [128 rows][D/32]: the tile's mask words
-  static constexpr uint32_t OFF_LASTX = OFF_MASK + 128 * (D / 32) * 4;   // u16 [512 / D segments][D]: last fired value
-  static constexpr uint32_t OFF_HAS = OFF_LASTX + 512 * 2;               // u8  [512 / D segments][D]: segment fired at all
-  static constexpr uint32_t OFF_BAR = OFF_HAS + 512;
+  static constexpr uint32_t OFF_BAR = OFF_PMAX + 2 * 128 * 4 * 4;
   static constexpr uint32_t OFF_MISC = OFF_BAR + 16 * 8;
   static constexpr uint32_t BYTES = OFF_MISC + 16 + 1024;
   static_assert(BYTES <= 227 * 1024, "shared memory budget");
@@ -74,18 +71,30 @@ enum Bar {
 struct TqParams {
   __nv_bfloat16* out;
   unsigned long long* counters;
-  const uint32_t* mask;        // [B,H,T_max,D/32] mask words of the query deltas (query deltas only)
-  const float* qhat_tile;      // [B,H,n_tiles64,D] reference in front of every 64-row tile
-  int T, T_max, n_tiles64, H, g, W, shape;
-  float scale_log2e;
+  const float* ckpt;           // [B,H,n_ckpt,D] reference in front of every 8-row block (query deltas only)
+  int T, T_max, n_ckpt, H, g, W, shape, basis_exact;
+  float scale_log2e, theta;
 };
+
+
+// Barrier of the four warps that share a tensor-memory lane quadrant (ids 1..4, 128 threads).
+// Immediate ids: with a register operand the compiler reserves all sixteen hardware barriers
+// for the CTA and no other kernel's CTA can share the SM.
+__device__ __forceinline__ void quad_sync(int qd) {
+  switch (qd) {
+    case 0: asm volatile("bar.sync 1, 128;" ::: "memory"); break;
+    case 1: asm volatile("bar.sync 2, 128;" ::: "memory"); break;
+    case 2: asm volatile("bar.sync 3, 128;" ::: "memory"); break;
+    default: asm volatile("bar.sync 4, 128;" ::: "memory"); break;
+  }
+}
 
 }  // namespace
 
 // KEY = false: query deltas (strategy 1): telescoped scores Q_hat.K^T.  The 128 reference rows
-// of the tile are rebuilt in shared memory from the query tile, the mask words and the reference
-// in front of the tile (the reference after row i is the last fired value at or below i), so
-// the sequential chain kernel does not have to store them and tm_qh is unused.  KEY = true: key deltas (strategy 3): the column recursion telescopes to
+// of the tile are rebuilt in shared memory from the query tile and the references the chain
+// kernel left in front of every 8-row block (Eq. 2-3 re-run over 8 rows, blocks in parallel),
+// so the sequential chain kernel does not have to store them and tm_qh is unused.  KEY = true: key deltas (strategy 3): the column recursion telescopes to
 // S[i][j] = q_i.k_hat(j), so the telescoped scores are Q.K_hat^T; tm_qh maps the reference key
 // rows (per KV head), which take the place of the key tiles in the ring, and the original keys
 // are fetched only for tiles that touch the window.
@@ -101,8 +110,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   using SM = TqSmem<D>;
   constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKBUF = SM::NKBUF;
   constexpr uint32_t OFF_Q = SM::OFF_Q, OFF_QH = SM::OFF_QH, OFF_K = SM::OFF_K, OFF_V = SM::OFF_V,
-                     OFF_P = SM::OFF_P, OFF_PMAX = SM::OFF_PMAX, OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC,
-                     OFF_MASK = SM::OFF_MASK, OFF_LASTX = SM::OFF_LASTX, OFF_HAS = SM::OFF_HAS;
+                     OFF_P = SM::OFF_P, OFF_PMAX = SM::OFF_PMAX, OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC;
   float* sPmax = reinterpret_cast<float*>(sm + OFF_PMAX);
   volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
   volatile uint32_t* abort_flag = sMisc + 1;
@@ -264,43 +272,38 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
 
     if (!KEY) {
-      // ---- reference-query tile: Q_hat(r)[c] = the last fired q[.][c] at or below row r, or the
-      // reference in front of the tile.  Thread (channel c, row segment) finds the last fired
-      // value of its segment, takes the nearest earlier one as carry-in and walks its rows.
-      constexpr int NW = D / 32, NSEG = NCTHR / D, SEG = BM / NSEG;   // 8 x 16 rows (d=64), 4 x 32 (d=128)
-      uint32_t* s_mask = reinterpret_cast<uint32_t*>(sm + OFF_MASK);
-      uint16_t* s_lastx = reinterpret_cast<uint16_t*>(sm + OFF_LASTX);
-      uint8_t* s_has = sm + OFF_HAS;
-      for (int e = tid; e < BM * NW; e += NCTHR) {
-        const int r = e / NW;
-        s_mask[e] = (i0 + r < T) ? p.mask[((size_t)bh * p.T_max + i0 + r) * NW + (e - r * NW)] : 0u;
-      }
+      // ---- reference-query tile.  The chain kernel left the reference in front of every 8-row
+      // block; thread (channel c, row segment) re-runs Eq. 2-3 over its blocks from there (the
+      // reference after row r is the last fired q[.][c] at or below r) and writes the rows of
+      // Q_hat straight into the operand layout.  Blocks are independent of one another.
+      constexpr int NSEG = NCTHR / D, SEG = BM / NSEG;   // 8 x 16 rows (d=64), 4 x 32 (d=128)
       const int c = tid % D, seg = tid / D;
-      const float snap = p.qhat_tile[((size_t)bh * p.n_tiles64 + 2 * qt) * D + c];
       // byte offset of element (r, c) inside a [128][D] operand tile (128-byte swizzle)
       auto elem_off = [&](int r) -> uint32_t {
         return (uint32_t)(c >> 6) * SZ_BLK + (uint32_t)r * 128u + ((((uint32_t)(c & 63) >> 3) ^ ((uint32_t)r & 7u)) << 4) +
                ((uint32_t)c & 7u) * 2u;
       };
+      float ref[SEG / DELTA_CKPT_ROWS];
+#pragma unroll
+      for (int bk = 0; bk < SEG / DELTA_CKPT_ROWS; ++bk) {
+        const int r0 = i0 + seg * SEG + bk * DELTA_CKPT_ROWS;
+        ref[bk] = (r0 < T) ? p.ckpt[((size_t)bh * p.n_ckpt + r0 / DELTA_CKPT_ROWS) * D + c] : 0.0f;
+      }
       mbar_wait(BAR(BAR_Q), 0, abort_flag);      // the query tile has landed
-      asm volatile("bar.sync 5, %0;" ::"n"(NCTHR) : "memory");   // mask words staged
-      uint32_t bits = 0;
 #pragma unroll
-      for (int r = 0; r < SEG; ++r) bits |= ((s_mask[(seg * SEG + r) * NW + (c >> 5)] >> (c & 31)) & 1u) << r;
-      uint16_t lastx = 0;
-      if (bits) lastx = *reinterpret_cast<const uint16_t*>(sm + OFF_Q + elem_off(seg * SEG + 31 - __clz(bits)));
-      s_lastx[seg * D + c] = lastx;
-      s_has[seg * D + c] = bits != 0u;
-      asm volatile("bar.sync 5, %0;" ::"n"(NCTHR) : "memory");
-      const __nv_bfloat16 snap16 = __float2bfloat16_rn(snap);        // exact: a copy of an input element or 0
-      uint16_t cur = *reinterpret_cast<const uint16_t*>(&snap16);
-      for (int s2 = 0; s2 < seg; ++s2) cur = s_has[s2 * D + c] ? s_lastx[s2 * D + c] : cur;
+      for (int bk = 0; bk < SEG / DELTA_CKPT_ROWS; ++bk) {
+        float cur = ref[bk];
 #pragma unroll
-      for (int r = 0; r < SEG; ++r) {
-        const uint32_t off = elem_off(seg * SEG + r);
-        const uint16_t x = *reinterpret_cast<const uint16_t*>(sm + OFF_Q + off);
-        cur = ((bits >> r) & 1u) ? x : cur;
-        *reinterpret_cast<uint16_t*>(sm + OFF_QH + off) = cur;
+        for (int r8 = 0; r8 < DELTA_CKPT_ROWS; ++r8) {
+          const int r = seg * SEG + bk * DELTA_CKPT_ROWS + r8;
+          const uint32_t off = elem_off(r);
+          const uint32_t xb = *reinterpret_cast<const uint16_t*>(sm + OFF_Q + off);
+          const float x = __uint_as_float(xb << 16);
+          const bool fire = (fabsf(__fsub_rn(x, cur)) > p.theta) || (i0 + r == 0 && p.basis_exact);
+          cur = fire ? x : cur;
+          // exact: the reference is a copy of an input element (or the zero it starts from)
+          *reinterpret_cast<uint16_t*>(sm + OFF_QH + off) = (uint16_t)(__float_as_uint(cur) >> 16);
+        }
       }
       fence_proxy_async();      // the tile was written through the generic proxy, the tensor cores read it
       __syncwarp();
@@ -351,7 +354,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
       for (int c = 1; c < 32; ++c) mx = fmaxf(mx, s[c]);
       sPmax[(bf * BM + row) * 4 + sub] = mx;
-      asm volatile("bar.sync %0, 128;" ::"r"(1 + qd) : "memory");   // the four warps of this quadrant
+      quad_sync(qd);   // the four warps of this quadrant
       const float4 pm = *reinterpret_cast<const float4*>(sPmax + (bf * BM + row) * 4);
       mx = fmaxf(fmaxf(pm.x, pm.y), fmaxf(pm.z, pm.w));
       const float m_new = fmaxf(m_run, mx * scale);
@@ -406,7 +409,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     mbar_wait(BAR(BAR_O), qt & 1, abort_flag);
     tc_fence_after();
     sPmax[(((qt + 1) & 1) * BM + row) * 4 + sub] = l_part;
-    asm volatile("bar.sync %0, 128;" ::"r"(1 + qd) : "memory");
+    quad_sync(qd);
     const float4 lp = *reinterpret_cast<const float4*>(sPmax + (((qt + 1) & 1) * BM + row) * 4);
     const float inv = 1.0f / ((lp.x + lp.y) + (lp.z + lp.w));
     const bool store = (i < T) && !*abort_flag;
@@ -443,7 +446,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
 template <int D, bool KEY>
 static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
-                              void* out, int T, int window, int shape, cudaStream_t st) {
+                              void* out, int T, float theta, int init, int window, int shape, cudaStream_t st) {
   const uint64_t BH = (uint64_t)s.B * s.H, BKV = (uint64_t)s.B * s.H_kv;
   const uint64_t ref_heads = KEY ? BKV : BH;   // the reference rows follow the delta stream
   CUtensorMap tq, tqh, tk, tv;
@@ -463,9 +466,9 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
   TqParams p;
   p.out = (__nv_bfloat16*)out;
   p.counters = w.counters;
-  p.mask = w.mask;
-  p.qhat_tile = w.qhat_tile;
-  p.T_max = s.T_max; p.n_tiles64 = s.n_tiles;
+  p.ckpt = w.ckpt;
+  p.T_max = s.T_max; p.n_ckpt = s.n_ckpt();
+  p.theta = theta; p.basis_exact = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
   p.T = T; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
   p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const dim3 grid((unsigned)BH, (T + BM - 1) / BM);
@@ -477,15 +480,15 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
 bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
 
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
-                                   const void* v, void* out, int T, int window, int shape,
-                                   bool key_deltas, cudaStream_t st) {
+                                   const void* v, void* out, int T, float theta, int init, int window,
+                                   int shape, bool key_deltas, cudaStream_t st) {
   if (!w.qhat_rows) return cudaErrorNotSupported;
   if (s.d == 64)
-    return key_deltas ? launch_tcq<64, true>(s, w, q, k, v, out, T, window, shape, st)
-                      : launch_tcq<64, false>(s, w, q, k, v, out, T, window, shape, st);
+    return key_deltas ? launch_tcq<64, true>(s, w, q, k, v, out, T, theta, init, window, shape, st)
+                      : launch_tcq<64, false>(s, w, q, k, v, out, T, theta, init, window, shape, st);
   if (s.d == 128)
-    return key_deltas ? launch_tcq<128, true>(s, w, q, k, v, out, T, window, shape, st)
-                      : launch_tcq<128, false>(s, w, q, k, v, out, T, window, shape, st);
+    return key_deltas ? launch_tcq<128, true>(s, w, q, k, v, out, T, theta, init, window, shape, st)
+                      : launch_tcq<128, false>(s, w, q, k, v, out, T, theta, init, window, shape, st);
   return cudaErrorNotSupported;
 }
 

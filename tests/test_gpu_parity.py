@@ -87,6 +87,53 @@ def test_delta_construction_bit_exact(B, Bn, H, T, d, dtype, theta, init):
     assert s["prefill"]["nnz"] == total and s["prefill"]["elements"] == Bn * H * T * d
 
 
+@pytest.mark.parametrize("T,d,dtype,theta,init", [
+    (1024, 64, "bf16", 0.4, "basis_exact"),
+    (1000, 64, "f32", 0.3, "zero_state"),
+    (777, 128, "bf16", 0.25, "basis_exact"),
+    (2048, 64, "bf16", 0.5, "basis_exact"),
+])
+def test_delta_construction_time_parallel_chain_hard_streams(B, T, d, dtype, theta, init):
+    """Streams on which a chain started late never meets the true one: a steady drift keeps the
+    two references a constant phase apart, so every segment of the time-parallel chain kernel
+    has guessed wrong and the correction has to pass from segment to segment.  Other channels:
+    a constant (nothing ever fires), a staircase, a drift that reverses, noise around a drift,
+    NaN and infinities in the middle of a segment."""
+    from tests.gpu_helpers import run_prefill
+    H = 3
+    q, k, v = _inputs(1, H, H, T, d, dtype, seed=11 + T)
+    t = np.arange(T, dtype=np.float64)
+    rng = np.random.default_rng(5)
+    for h in range(H):
+        for c in range(d):
+            kind = (c + h) % 8
+            slope = theta * (0.011 + 0.0007 * c)
+            if kind == 0:
+                x = slope * t
+            elif kind == 1:
+                x = np.full(T, 0.5 + c)
+            elif kind == 2:
+                x = np.floor(t / 37.0) * theta * 0.75
+            elif kind == 3:
+                x = slope * np.abs(t - T * 0.6)
+            elif kind == 4:
+                x = slope * t + 0.2 * theta * rng.standard_normal(T)
+            elif kind == 5:
+                x = -slope * t * 3.0
+            elif kind == 6:
+                x = theta * 0.9 * np.sin(t / 50.0 + c)
+            else:
+                continue                      # keep the AR(1) stream
+            q[0, h, :, c] = x.astype(np.float32)
+    q[0, 0, T // 2 + 3, 5] = np.nan
+    q[0, 1, T // 3, 9] = np.inf
+    q[0, 1, T // 3 + 40, 9] = -np.inf
+    if dtype == "bf16":
+        q = WL.round_to_bf16(q)
+    st, out, _, _ = run_prefill(B, q, k, v, theta, 64, dtype, init=init)
+    _check_delta_arrays(B, st, q, theta, init, T)
+
+
 def test_delta_special_values_bit_exact(B):
     from tests.gpu_helpers import run_prefill
     T, d = 70, 64
