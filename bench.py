@@ -306,8 +306,8 @@ def run_ours(args):
     roofline = k2_roofline(w, stats, kernel, kmean[2], peaks, n_sm)
     # K1 is a streaming pass: report it against the HBM copy bandwidth as well
     es = 2 if w.dtype == "bf16" else 4
-    # chain kernel (query deltas): reads Q, writes the mask words
-    k1_bytes = w.B * w.H * w.T * (w.d * es + w.d // 8)
+    # chain kernel (query deltas): reads Q, writes the reference in front of every 8-row block
+    k1_bytes = w.B * w.H * w.T * (w.d * es + w.d * 4 // 8)
     k1 = {"kernel": "delta_chain", "bound": "hbm", "kernel_ms": kmean[0],
           "achieved": k1_bytes / (kmean[0] * 1e-3) / 1e9, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
           "frac": k1_bytes / (kmean[0] * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
@@ -558,8 +558,9 @@ def run_delta_pass_large(B, torch, peaks, flush):
             kms.append(B.delta_state_prefill_kernel_ms(st)); steps.append(e0.elapsed_time(e1))
     stt = B.delta_sparsity_stats(st)["prefill"]
     n = w.B * w.H * w.T
-    chain_b = n * (w.d * 2 + w.d // 8)                                   # Q read, mask written
-    finish_b = n * (w.d * 2 + w.d // 8 + w.d * 4 + w.d + 2) + 2 * w.B * w.H_kv * w.T * w.d * 2 + n * 4
+    chain_b = n * (w.d * 2 + w.d * 4 // 8)                               # Q read, 8-row checkpoints written
+    # Q and checkpoints read; delta values, mask words, indices, row counts written; K read, R written
+    finish_b = n * (w.d * 2 + w.d * 4 // 8 + w.d * 4 + w.d // 8 + w.d + 2) + w.B * w.H_kv * w.T * w.d * 2 + n * 4
     hbm = float(peaks["hbm_gbs"])
     cm, fm = statistics.mean(x[0] for x in kms), statistics.mean(x[1] for x in kms)
     am = statistics.mean(x[2] for x in kms)

@@ -28,8 +28,13 @@ namespace delta {
 
 namespace {
 
-constexpr int RC = 32;       // rows per ring stage (one mask flush per stage)
-constexpr int NS = 8;        // ring stages
+// Ring geometry.  Key stream (the chain stores mask words): 32 rows per stage, one mask flush
+// per stage, 8 stages.  Query stream (checkpoints only): 64 rows per stage, 4 stages -- half
+// the per-stage bookkeeping on the chain warps for the same shared memory.
+template <bool EMIT> struct Ring {
+  static constexpr int RC = EMIT ? 32 : 64;   // rows per stage
+  static constexpr int NS = EMIT ? 8 : 4;     // stages
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -82,6 +87,7 @@ __device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, 
                                             float& qh, float theta, int lane, float* dqp,
                                             __nv_bfloat16* qrp, uint32_t* maskp, float* ckptp) {
   constexpr int NW = D / 32;
+  constexpr int RC = Ring<EMIT>::RC;
   // bit r of `bits`: did this thread's channel fire in row t0 + r
   uint32_t bits = 0;
   if (nrows == RC && !basis_row) {
@@ -158,6 +164,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
   // q: the stream that becomes the delta matrix, [heads][src_rows][D] with rows 0..T-1 read
   // (queries: src_rows = T; keys in the KV-cache layout: src_rows = T_max)
   constexpr int NW = D / 32;                       // chain warps = mask words per row
+  constexpr int RC = Ring<EMIT>::RC, NS = Ring<EMIT>::NS;
   constexpr uint32_t ROW_BYTES = D * sizeof(TIn);
   constexpr uint32_t STAGE_BYTES = RC * ROW_BYTES;
   extern __shared__ __align__(128) unsigned char ring[];   // [NS][RC][D] of TIn
@@ -247,7 +254,8 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 #define LAUNCH(TIN, DD)                                                                          \
   do {                                                                                           \
     auto kern = key_stream ? delta_chain_kernel<TIN, DD, true> : delta_chain_kernel<TIN, DD, false>; \
-    const size_t smem = (size_t)NS * RC * DD * sizeof(TIN);                                      \
+    const size_t smem = key_stream ? (size_t)Ring<true>::NS * Ring<true>::RC * DD * sizeof(TIN)  \
+                                   : (size_t)Ring<false>::NS * Ring<false>::RC * DD * sizeof(TIN); \
     if (smem > 48 * 1024) {                                                                      \
       err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
       if (err != cudaSuccess) return err;                                                        \

@@ -93,12 +93,12 @@ def test_delta_construction_bit_exact(B, Bn, H, T, d, dtype, theta, init):
     (777, 128, "bf16", 0.25, "basis_exact"),
     (2048, 64, "bf16", 0.5, "basis_exact"),
 ])
-def test_delta_construction_time_parallel_chain_hard_streams(B, T, d, dtype, theta, init):
-    """Streams on which a chain started late never meets the true one: a steady drift keeps the
-    two references a constant phase apart, so every segment of the time-parallel chain kernel
-    has guessed wrong and the correction has to pass from segment to segment.  Other channels:
-    a constant (nothing ever fires), a staircase, a drift that reverses, noise around a drift,
-    NaN and infinities in the middle of a segment."""
+def test_delta_construction_hard_streams(B, T, d, dtype, theta, init):
+    """Structured streams across several ring stages, checkpoint blocks and tiles: a steady drift
+    (the reference trails the input by a constant phase, so a chain restarted anywhere else
+    would never agree with it again), a constant (nothing ever fires), a staircase, a drift that
+    reverses, noise around a drift, a slow sine below the threshold, NaN and infinities in the
+    middle of a stage."""
     from tests.gpu_helpers import run_prefill
     H = 3
     q, k, v = _inputs(1, H, H, T, d, dtype, seed=11 + T)
