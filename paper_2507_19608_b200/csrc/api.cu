@@ -34,10 +34,6 @@ struct delta_state {
   // optional per-kernel timing of prefill (host-side event objects)
   bool profiling = false, profiled = false;
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
-  // side stream of prefill: the row-parallel finish kernel runs beside the attention kernel when
-  // the latter does not read its outputs (host-side objects, created at the first prefill)
-  cudaStream_t side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -154,9 +150,6 @@ delta_status_t delta_state_destroy(delta_state_t* st) {
   if (!st) return DELTA_ERR_INVALID_ARG;
   for (auto& ev : st->ev)
     if (ev) cudaEventDestroy(ev);
-  if (st->ev_fork) cudaEventDestroy(st->ev_fork);
-  if (st->ev_join) cudaEventDestroy(st->ev_join);
-  if (st->side) cudaStreamDestroy(st->side);
   delete st;
   return DELTA_OK;
 }
@@ -235,16 +228,12 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   const bool key = c.source == DELTA_SRC_KEY;
   if (key && which != 2) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
   // The telescoped attention kernel reads nothing the finish kernel writes (delta values,
-  // counts, indices, counters, hand-off row), so the two run side by side: finish on the
-  // state's side stream between a fork and a join event.  With per-kernel timing on,
-  // everything stays in line on the caller's stream.
-  const bool fork = (which == 2) && !prof;
-  if (fork && !st->side) {
-    if ((e = cudaStreamCreateWithFlags(&st->side, cudaStreamNonBlocking)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&st->ev_fork, cudaEventDisableTiming)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&st->ev_join, cudaEventDisableTiming)) != cudaSuccess)
-      return cuda_fail(e);
-  }
+  // mask words, counts, indices, counters, hand-off row), so it runs directly behind the chain
+  // kernel and the finish kernel comes last.  Both are launched with programmatic stream
+  // serialisation: the attention CTAs are resident and set up by the time the chain ends, and
+  // the finish kernel's launch overlaps the end of the attention kernel.  With per-kernel
+  // timing on, the kernels run in their natural order with events between them.
+  const bool chained = (which == 2) && !prof;
   MARK(0);
   // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
   if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, key, cs)) != cudaSuccess)
@@ -256,19 +245,15 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
                                     cs);
     return launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, c.dtype, cs);
   };
-  if (fork) {
-    if ((e = cudaEventRecord(st->ev_fork, cs)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaStreamWaitEvent(st->side, st->ev_fork, 0)) != cudaSuccess) return cuda_fail(e);
-    if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
-                                 use_tc, key, st->side)) != cudaSuccess)
-      return cuda_fail(e);
-    if ((e = cudaEventRecord(st->ev_join, st->side)) != cudaSuccess) return cuda_fail(e);
+  if (chained) {
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaStreamWaitEvent(cs, st->ev_join, 0)) != cudaSuccess) return cuda_fail(e);
+    if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
+                                 use_tc, key, true, cs)) != cudaSuccess)
+      return cuda_fail(e);
   } else {
     MARK(1);
     if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
-                                 use_tc, key, cs)) != cudaSuccess)
+                                 use_tc, key, false, cs)) != cudaSuccess)
       return cuda_fail(e);
     MARK(2);
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);

@@ -185,6 +185,10 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // a kernel launched behind this one with programmatic stream serialisation may become
+  // resident and run its prologue now; it sees this kernel's results only after its own
+  // grid-dependency wait
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == NW) {
     // ---- producer: keeps up to NS stages of query rows in flight
@@ -293,6 +297,9 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
     const float* __restrict__ ckpt, int n_ckpt, float theta, int basis_exact) {
   constexpr int NW = D / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // launched with programmatic stream serialisation behind the attention kernel: the results
+  // of everything in front are visible from here on (no effect in an ordinary launch)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if ((int)blockIdx.x < n_idx_blocks) {
     // ---- one block per (batch, head, 64-row tile); warp w serves rows 8w .. 8w+7
     __shared__ unsigned long long s_red[3][8];
@@ -468,7 +475,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
 
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
                                 float theta, int window, int shape, int dtype, int init, bool want_kt,
-                                bool key_stream, cudaStream_t st) {
+                                bool key_stream, bool programmatic, cudaStream_t st) {
   // key deltas: the index/counter pass runs over the KV heads and there is no hand-off row
   const int BH = s.B * (key_stream ? s.H_kv : s.H);
   const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
@@ -480,6 +487,11 @@ cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* 
   cfg.gridDim = dim3((unsigned)(n_idx_blocks + n_key_blocks));
   cfg.blockDim = dim3(256);
   cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = programmatic ? 1 : 0;
   cudaError_t err = cudaSuccess;
 #define LAUNCH(TIN, DD)                                                                          \
   err = cudaLaunchKernelEx(&cfg, delta_finish_kernel<TIN, DD>,                                   \

@@ -164,6 +164,9 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const CUtensorMap* tm_ring = KEY ? &tm_qh : &tm_k;   // what streams through the key ring
       mbar_expect_tx(BAR(BAR_Q), SZ_TILE);
       load_tile(base + OFF_Q, &tm_q, BAR(BAR_Q), i0, bh);
+      // everything up to here is independent of the delta-construction kernel in front of
+      // this one (programmatic stream serialisation): wait for its results now
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       mbar_expect_tx(BAR(BAR_K0), SZ_TILE);
       load_tile(base + OFF_K, tm_ring, BAR(BAR_K0), 0, bkv);
       mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
@@ -284,6 +287,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                ((uint32_t)c & 7u) * 2u;
       };
       float ref[SEG / DELTA_CKPT_ROWS];
+      asm volatile("griddepcontrol.wait;" ::: "memory");    // the chain kernel's checkpoints
 #pragma unroll
       for (int bk = 0; bk < SEG / DELTA_CKPT_ROWS; ++bk) {
         const int r0 = i0 + seg * SEG + bk * DELTA_CKPT_ROWS;
@@ -471,10 +475,22 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
   p.theta = theta; p.basis_exact = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
   p.T = T; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
   p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
-  const dim3 grid((unsigned)BH, (T + BM - 1) / BM);
-  hybrid_attn_tcq_kernel<D, KEY><<<grid, NTHR, TqSmem<D>::BYTES, st>>>(tq, tqh, tk, tv, p);
+  // Launched with programmatic stream serialisation: the CTAs become resident and run their
+  // prologue (tensor-memory allocation, barrier setup, query-tile load) while the delta chain
+  // kernel in front is still running; they wait for its results with griddepcontrol.wait.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)BH, (T + BM - 1) / BM);
+  cfg.blockDim = dim3(NTHR);
+  cfg.dynamicSmemBytes = TqSmem<D>::BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  err = cudaLaunchKernelEx(&cfg, hybrid_attn_tcq_kernel<D, KEY>, tq, tqh, tk, tv, p);
   count_launch();
-  return cudaGetLastError();
+  return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
