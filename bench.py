@@ -335,6 +335,7 @@ def run_ours(args):
         line["theta_sweep"] = run_sweep(args, B, torch, w, q, k, v, out, st, flush)
         line["decode"] = run_decode(args, B, torch, peaks)
         line["key_deltas"] = run_key_deltas(args, B, torch, w, tens, theta, flush, peaks)
+        line["strategies"] = run_strategy_errors(B, torch, w, tens, theta)
         line["delta_pass_large"] = run_delta_pass_large(B, torch, peaks, flush)
         line["cpu_baseline"] = run_cpu_baseline(args, w, tens, theta)
     print(json.dumps(line))
@@ -532,6 +533,35 @@ def run_key_deltas(args, B, torch, w, tens, theta, flush, peaks):
                         "tokens_per_s": w.B * w.T / (statistics.mean(ms) * 1e-3), "S_m": stt["S_m"],
                         "S_c_exact": stt["S_c_exact"]},
             "decode": run_decode(args, B, torch, peaks, source="key", names=("llama32_1b_decode_b16",))}
+
+
+
+def run_strategy_errors(B, torch, w, tens, theta):
+    """Section III-A's three construction strategies on the same inputs: output error against
+    dense attention (the library itself with a window that covers the sequence) and the delta
+    sparsity each one reaches.  (1) query deltas top-down, (2) query deltas bottom-up, (3) key
+    deltas; same theta and window for all three."""
+    q, k, v = (to_dev(tens[n], w.dtype, torch) for n in ("q", "k", "v"))
+
+    def run(source, window):
+        st = B.delta_state_init(B.make_config(w.B, w.H, w.H_kv, w.d, w.T, w.dtype, source=source))
+        out = torch.empty_like(q)
+        B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, window)
+        torch.cuda.synchronize()
+        return out.float(), B.delta_sparsity_stats(st)["prefill"]
+    dense, _ = run(B.DELTA_SRC_QUERY, w.T)
+    res = {"theta": theta, "window": w.window, "reference": "dense attention (window = T) by the same library"}
+    for name, src in (("query_top_down", B.DELTA_SRC_QUERY), ("query_bottom_up", B.DELTA_SRC_QUERY_BOTTOM_UP),
+                      ("key", B.DELTA_SRC_KEY)):
+        out, stt = run(src, w.window)
+        err = (out - dense).abs()
+        res[name] = {"mean_abs_err": float(err.mean()), "max_abs_err": float(err.max()),
+                     "rel_rms_err": float((err.pow(2).mean().sqrt() / dense.pow(2).mean().sqrt())),
+                     # rows in the first / last quarter of the sequence: where each strategy's basis row sits
+                     "mean_abs_err_first_quarter": float(err[:, :, : w.T // 4].mean()),
+                     "mean_abs_err_last_quarter": float(err[:, :, -(w.T // 4):].mean()),
+                     "S_m": stt["S_m"], "S_c_exact": stt["S_c_exact"]}
+    return res
 
 
 def run_delta_pass_large(B, torch, peaks, flush):

@@ -63,8 +63,15 @@ typedef enum { DELTA_F32 = 0, DELTA_BF16 = 1 } delta_dtype_t;
  *   the reference key, and the library keeps a cache of reference-key rows in its workspace.
  *   bf16 with d = 64 or 128 only (DELTA_ERR_UNSUPPORTED otherwise).  With KEY the delta arrays
  *   of delta_state_view hold one set per KV head: read them as [B * H_kv, ...] from the start
- *   of the view. */
-typedef enum { DELTA_SRC_QUERY = 0, DELTA_SRC_KEY = 1 } delta_source_t;
+ *   of the view.
+ * QUERY_BOTTOM_UP = strategy (2): query deltas with the rows taken from the last token up to
+ *   the first, so the basis is the last row and the reference of row i is the last value that
+ *   fired among rows i .. T-1.  Prefill only (the method needs the whole sequence before its
+ *   first row): decode on such a state returns DELTA_ERR_UNSUPPORTED.  bf16 with d = 64 or 128
+ *   only.  All delta arrays of delta_state_view stay indexed by token row; the per-tile
+ *   reference snapshot of tile t is the reference before the tile's highest row is processed
+ *   and DELTA_VIEW_QHAT is the reference left after row 0. */
+typedef enum { DELTA_SRC_QUERY = 0, DELTA_SRC_KEY = 1, DELTA_SRC_QUERY_BOTTOM_UP = 2 } delta_source_t;
 
 /* Shape of the exact-attention region in prefill (Section III-B).  BLOCK: squares of side
  * `window` along the diagonal, anchored at token 0 (pair (i,j) is exact iff i/W == j/W).

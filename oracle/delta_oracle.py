@@ -342,7 +342,7 @@ def prefill_stats(row_nnz, T, d, W, shape):
 
 
 # --------------------------------------------------------------------------- multi-head wrappers
-def prefill_mha(q, k, v, theta, W, shape="block", init="basis_exact", source="query"):
+def prefill_mha(q, k, v, theta, W, shape="block", init="basis_exact", source="query", order="top_down"):
     """q [B,H,T,d], k,v [B,H_kv,T,d] -> out [B,H,T,d] float64 plus per-head results.
     Query head h reads KV head h // (H / H_kv)."""
     B, H, T, d = q.shape
@@ -352,7 +352,7 @@ def prefill_mha(q, k, v, theta, W, shape="block", init="basis_exact", source="qu
     heads = {}
     for b in range(B):
         for h in range(H):
-            r = prefill_head(q[b, h], k[b, h // g], v[b, h // g], theta, W, shape, init, source)
+            r = prefill_head(q[b, h], k[b, h // g], v[b, h // g], theta, W, shape, init, source, order)
             out[b, h] = r["out"]
             heads[(b, h)] = r
     return out, heads

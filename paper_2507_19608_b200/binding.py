@@ -19,7 +19,7 @@ DELTA_OK = 0
 DELTA_ERR_INVALID_ARG, DELTA_ERR_UNSUPPORTED, DELTA_ERR_WORKSPACE, DELTA_ERR_CAPACITY = 1, 2, 3, 4
 DELTA_ERR_STATE, DELTA_ERR_CUDA, DELTA_ERR_TIMEOUT, DELTA_ERR_SCRATCH_LIMIT = 5, 6, 7, 8
 DELTA_F32, DELTA_BF16 = 0, 1
-DELTA_SRC_QUERY, DELTA_SRC_KEY = 0, 1
+DELTA_SRC_QUERY, DELTA_SRC_KEY, DELTA_SRC_QUERY_BOTTOM_UP = 0, 1, 2
 DELTA_WIN_BLOCK, DELTA_WIN_SLIDING = 0, 1
 DELTA_INIT_BASIS_EXACT, DELTA_INIT_ZERO_STATE = 0, 1
 (DELTA_VIEW_DQ, DELTA_VIEW_MASK, DELTA_VIEW_ROW_NNZ, DELTA_VIEW_TILE_NNZ, DELTA_VIEW_IDX,

@@ -47,10 +47,12 @@ static delta_status_t check_config(const delta_config_t* c) {
     return DELTA_ERR_INVALID_ARG;
   if (c->init != DELTA_INIT_BASIS_EXACT && c->init != DELTA_INIT_ZERO_STATE)
     return DELTA_ERR_INVALID_ARG;
-  if (c->source != DELTA_SRC_QUERY && c->source != DELTA_SRC_KEY) return DELTA_ERR_INVALID_ARG;
+  if (c->source != DELTA_SRC_QUERY && c->source != DELTA_SRC_KEY && c->source != DELTA_SRC_QUERY_BOTTOM_UP)
+    return DELTA_ERR_INVALID_ARG;
   if (c->d != 64 && c->d != 128) return DELTA_ERR_UNSUPPORTED;
   // key deltas (strategy 3) are served by the telescoped tensor-core kernel only
-  if (c->source == DELTA_SRC_KEY && !(c->dtype == DELTA_BF16 && tcq_kernel_shape(c->d)))
+  // and so are bottom-up query deltas (strategy 2)
+  if (c->source != DELTA_SRC_QUERY && !(c->dtype == DELTA_BF16 && tcq_kernel_shape(c->d)))
     return DELTA_ERR_UNSUPPORTED;
   const int g = c->H / c->H_kv;
   if (g != 1 && g != 2 && g != 4 && g != 8) return DELTA_ERR_UNSUPPORTED;
@@ -183,7 +185,7 @@ int32_t delta_state_position(const delta_state_t* st) { return st ? st->n : -1; 
 // Can prefill kernel `which` (1 or 2) serve this state?
 static bool tc_eligible(const delta_state* st, int which) {
   if (st->cfg.dtype != DELTA_BF16 || !tc_kernel_available(64)) return false;
-  if (st->cfg.source == DELTA_SRC_KEY && which != 2) return false;
+  if (st->cfg.source != DELTA_SRC_QUERY && which != 2) return false;
   return which == 1 ? tc_kernel_shape(st->cfg.d) : tcq_kernel_shape(st->cfg.d);
 }
 
@@ -196,7 +198,7 @@ int32_t delta_state_prefill_kernel(const delta_state_t* st) {
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
   if (!st || which < -1 || which > 2) return DELTA_ERR_INVALID_ARG;
   if (which >= 1 && !tc_eligible(st, which)) return DELTA_ERR_UNSUPPORTED;
-  if (which == 0 && st->cfg.source == DELTA_SRC_KEY) return DELTA_ERR_UNSUPPORTED;
+  if (which == 0 && st->cfg.source != DELTA_SRC_QUERY) return DELTA_ERR_UNSUPPORTED;
   st->forced_kernel = which;
   return DELTA_OK;
 }
@@ -226,7 +228,8 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   const int which = delta_state_prefill_kernel(st);
   const bool use_tc = which == 1;
   const bool key = c.source == DELTA_SRC_KEY;
-  if (key && which != 2) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
+  const bool rev = c.source == DELTA_SRC_QUERY_BOTTOM_UP;
+  if ((key || rev) && which != 2) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
   // The telescoped attention kernel reads nothing the finish kernel writes (delta values,
   // mask words, counts, indices, counters, hand-off row), so it runs directly behind the chain
   // kernel and the finish kernel comes last.  Both are launched with programmatic stream
@@ -236,24 +239,24 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   const bool chained = (which == 2) && !prof;
   MARK(0);
   // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
-  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, key, cs)) != cudaSuccess)
+  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, key, rev, cs)) != cudaSuccess)
     return cuda_fail(e);
   auto attention = [&]() -> cudaError_t {
     if (use_tc) return launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
     if (which == 2)
       return launch_hybrid_attn_tcq(st->shape, st->ws, q, k, v, out, T, theta, c.init, window, c.prefill_window, key,
-                                    cs);
+                                    rev, cs);
     return launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, c.dtype, cs);
   };
   if (chained) {
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
     if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
-                                 use_tc, key, true, cs)) != cudaSuccess)
+                                 use_tc, key, rev, true, cs)) != cudaSuccess)
       return cuda_fail(e);
   } else {
     MARK(1);
     if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
-                                 use_tc, key, false, cs)) != cudaSuccess)
+                                 use_tc, key, rev, false, cs)) != cudaSuccess)
       return cuda_fail(e);
     MARK(2);
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
@@ -324,6 +327,7 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
   if (!st || !q_new || !k_new || !v_new || !k_cache || !v_cache || !out) return DELTA_ERR_INVALID_ARG;
   delta_status_t s = check_theta_window(theta, window);
   if (s != DELTA_OK) return s;
+  if (st->cfg.source == DELTA_SRC_QUERY_BOTTOM_UP) return DELTA_ERR_UNSUPPORTED;   // strategy (2) has no decode
   if (st->n < 1) return DELTA_ERR_STATE;
   if (st->n >= st->cfg.T_max) return DELTA_ERR_CAPACITY;
   cudaError_t e =

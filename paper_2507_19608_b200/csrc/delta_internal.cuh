@@ -56,9 +56,10 @@ void count_launch(int n = 1);
 // 8-row block and every 64-row tile, final reference.  Key stream: also delta values, mask
 // words and reference rows.
 // key_stream: the stream is K in the KV-cache layout, one chain set per KV head (strategy 3).
+// reverse: rows are taken from T-1 down to 0 (strategy 2; query stream only).
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
                                float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
-                               cudaStream_t st);
+                               bool reverse, cudaStream_t st);
 // K1b: row-parallel finish: (query stream) delta values and mask words from the 8-row
 // checkpoints; counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
@@ -66,7 +67,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 // of the kernel in front; the kernel waits for that kernel's completion itself).
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
                                 float theta, int window, int shape, int dtype, int init, bool want_kt,
-                                bool key_stream, bool programmatic, cudaStream_t st);
+                                bool key_stream, bool reverse, bool programmatic, cudaStream_t st);
 // K2 (generic): fused hybrid attention on CUDA cores, any supported dtype.
 cudaError_t launch_hybrid_attn_generic(const Shape& s, const Workspace& w, const void* q,
                                        const void* k, const void* v, void* out, int T, int window,

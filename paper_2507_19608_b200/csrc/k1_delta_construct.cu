@@ -150,6 +150,37 @@ __device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, 
   if (lane < nrows) maskp[(size_t)(t0 + lane) * NW] = mymask;
 }
 
+
+// Strategy (2): the same stage of the query stream taken from its last row down to its first.
+// The checkpoint of an 8-row block is the reference before the block's highest row.
+// basis_last: the stage's last row is row T-1, the un-thresholded basis of this order.
+template <typename TIn, int D>
+__device__ __forceinline__ void chain_stage_rev(const TIn* rows, int t0, int nrows, bool basis_last, float& qh,
+                                                float theta, float* ckptp) {
+  constexpr int RC = Ring<false>::RC;
+  if (nrows == RC && !basis_last) {
+    float x[RC];
+    const uint32_t saddr = smem_u32(rows);
+#pragma unroll
+    for (int r = 0; r < RC; ++r) x[r] = lds_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
+#pragma unroll
+    for (int r = RC - 1; r >= 0; --r) {
+      if ((r % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      const float diff = __fsub_rn(x[r], qh);
+      const bool fire = fabsf(diff) > theta;
+      qh = fire ? x[r] : qh;
+    }
+  } else {
+    for (int r = nrows - 1; r >= 0; --r) {
+      if (((t0 + r) % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 || r == nrows - 1)
+        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      const float x = to_f32(rows[r * D]);
+      const bool fire = (r == nrows - 1 && basis_last) || (fabsf(__fsub_rn(x, qh)) > theta);
+      qh = fire ? x : qh;
+    }
+  }
+}
+
 }  // namespace
 
 // EMIT: also store the delta values and the reference rows (key deltas); without it the chain
@@ -160,7 +191,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
     __nv_bfloat16* __restrict__ qhat_rows, float* __restrict__ ckpt,
     unsigned long long* __restrict__ counters, int T, int T_max, int n_tiles, int n_ckpt, float theta,
-    int basis_exact, int src_rows) {
+    int basis_exact, int src_rows, int reverse) {
   // q: the stream that becomes the delta matrix, [heads][src_rows][D] with rows 0..T-1 read
   // (queries: src_rows = T; keys in the KV-cache layout: src_rows = T_max)
   constexpr int NW = D / 32;                       // chain warps = mask words per row
@@ -198,7 +229,8 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
       for (int i = 0; i < n_chunks; ++i) {
         const int s = i % NS;
         if (i >= NS && !mbar_wait(empty0 + 8 * s, ((i / NS) - 1) & 1)) { s_fail = 1; break; }
-        const int rows = min(RC, T - i * RC);
+        const int ci = reverse ? n_chunks - 1 - i : i;      // stage of the head in token order
+        const int rows = min(RC, T - ci * RC);
         const uint32_t bytes = (uint32_t)rows * ROW_BYTES;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full0 + 8 * s),
                      "r"(bytes)
@@ -206,7 +238,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
         asm volatile(
             "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                 ring0 + s * STAGE_BYTES),
-            "l"(src + (size_t)i * STAGE_BYTES), "r"(bytes), "r"(full0 + 8 * s)
+            "l"(src + (size_t)ci * STAGE_BYTES), "r"(bytes), "r"(full0 + 8 * s)
             : "memory");
       }
     }
@@ -221,14 +253,17 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     bool failed = false;
     for (int i = 0; i < n_chunks; ++i) {
       const int s = i % NS;
-      const int t0 = i * RC;
+      const int t0 = (reverse ? n_chunks - 1 - i : i) * RC;
       if (qhat_tile && (t0 % DELTA_TILE_ROWS) == 0)
         qhat_tile[((size_t)bh * n_tiles + t0 / DELTA_TILE_ROWS) * D + c] = qh;
       if (!mbar_wait(full0 + 8 * s, (i / NS) & 1)) { failed = true; break; }
       const TIn* rows = reinterpret_cast<const TIn*>(ring + (size_t)s * STAGE_BYTES) + c;
       const int nrows = min(RC, T - t0);
-      chain_stage<TIn, D, EMIT>(rows, t0, nrows, t0 == 0 && basis_exact, true, qh, theta, lane, dqp, qrp, maskp,
-                                ckptp);
+      if (!EMIT && reverse)
+        chain_stage_rev<TIn, D>(rows, t0, nrows, t0 + nrows == T && basis_exact, qh, theta, ckptp);
+      else
+        chain_stage<TIn, D, EMIT>(rows, t0, nrows, t0 == 0 && basis_exact, true, qh, theta, lane, dqp, qrp, maskp,
+                                  ckptp);
       __syncwarp();
       if (lane == 0)
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * s) : "memory");
@@ -243,7 +278,8 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
 
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
                                float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
-                               cudaStream_t st) {
+                               bool reverse, cudaStream_t st) {
+  if (key_stream && reverse) return cudaErrorNotSupported;
   __nv_bfloat16* qrows = want_qhat_rows ? w.qhat_rows : nullptr;
   // query deltas: the chain leaves mask words and per-tile references only; delta values are
   // recomputed row-parallel by the finish kernel.  Key deltas: the chain stores them itself.
@@ -266,7 +302,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
     }                                                                                            \
     kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, dq_out, w.mask, tile_out, fin_out, qrows, \
                                       ckpt_out, w.counters, T, s.T_max, s.n_tiles, s.n_ckpt(), theta, \
-                                      basis, src_rows);                                          \
+                                      basis, src_rows, reverse ? 1 : 0);                         \
   } while (0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
@@ -294,7 +330,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
     const float* __restrict__ qhat, float* __restrict__ R, float* __restrict__ kt, int T,
     int T_max, int n_tiles, int BH, int H, int g, int W, int shape, int n_idx_blocks, int kt_ld,
     int key_stream, const TIn* __restrict__ q, float* __restrict__ dq,
-    const float* __restrict__ ckpt, int n_ckpt, float theta, int basis_exact) {
+    const float* __restrict__ ckpt, int n_ckpt, float theta, int basis_exact, int reverse) {
   constexpr int NW = D / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // launched with programmatic stream serialisation behind the attention kernel: the results
@@ -325,11 +361,12 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
           for (int r = 0; r < 8; ++r)
             x[r] = (rbase + r < T) ? to_f32(q[((size_t)bh * T + rbase + r) * D + c]) : 0.0f;
 #pragma unroll
-          for (int r = 0; r < 8; ++r) {
+          for (int rr = 0; rr < 8; ++rr) {
+            const int r = reverse ? 7 - rr : rr;         // strategy (2) takes the rows from the top
             const bool live = rbase + r < T;
             bool fire;
             float delta;
-            if (rbase + r == 0 && basis_exact) {
+            if (rbase + r == (reverse ? T - 1 : 0) && basis_exact) {
               fire = true;                               // the basis vector is kept whole
               delta = x[r];
             } else {
@@ -475,7 +512,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
 
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
                                 float theta, int window, int shape, int dtype, int init, bool want_kt,
-                                bool key_stream, bool programmatic, cudaStream_t st) {
+                                bool key_stream, bool reverse, bool programmatic, cudaStream_t st) {
   // key deltas: the index/counter pass runs over the KV heads and there is no hand-off row
   const int BH = s.B * (key_stream ? s.H_kv : s.H);
   const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
@@ -499,7 +536,7 @@ cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* 
       s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld, key_stream ? 1 : 0,   \
       key_stream ? (const TIN*)nullptr : (const TIN*)q, key_stream ? (float*)nullptr : w.dq,      \
       key_stream ? (const float*)nullptr : (const float*)w.ckpt, s.n_ckpt(), theta,               \
-      init == DELTA_INIT_BASIS_EXACT ? 1 : 0)
+      init == DELTA_INIT_BASIS_EXACT ? 1 : 0, reverse ? 1 : 0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
   } else {

@@ -72,7 +72,9 @@ struct TqParams {
   __nv_bfloat16* out;
   unsigned long long* counters;
   const float* ckpt;           // [B,H,n_ckpt,D] reference in front of every 8-row block (query deltas only)
-  int T, T_max, n_ckpt, H, g, W, shape, basis_exact;
+  int T, T_max, n_ckpt, H, g, W, shape;
+  int reverse;       // strategy (2): Eq. 2-3 runs from row T-1 down to row 0
+  int basis_row;     // the un-thresholded basis row (0, or T-1 in reverse), -1 if there is none
   float scale_log2e, theta;
 };
 
@@ -298,12 +300,14 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       for (int bk = 0; bk < SEG / DELTA_CKPT_ROWS; ++bk) {
         float cur = ref[bk];
 #pragma unroll
-        for (int r8 = 0; r8 < DELTA_CKPT_ROWS; ++r8) {
+        for (int rr = 0; rr < DELTA_CKPT_ROWS; ++rr) {
+          const int r8 = p.reverse ? DELTA_CKPT_ROWS - 1 - rr : rr;   // strategy (2): from the top
           const int r = seg * SEG + bk * DELTA_CKPT_ROWS + r8;
           const uint32_t off = elem_off(r);
           const uint32_t xb = *reinterpret_cast<const uint16_t*>(sm + OFF_Q + off);
           const float x = __uint_as_float(xb << 16);
-          const bool fire = (fabsf(__fsub_rn(x, cur)) > p.theta) || (i0 + r == 0 && p.basis_exact);
+          // rows past the end of the sequence carry no state (in reverse they come first)
+          const bool fire = (i0 + r < T) && ((fabsf(__fsub_rn(x, cur)) > p.theta) || (i0 + r == p.basis_row));
           cur = fire ? x : cur;
           // exact: the reference is a copy of an input element (or the zero it starts from)
           *reinterpret_cast<uint16_t*>(sm + OFF_QH + off) = (uint16_t)(__float_as_uint(cur) >> 16);
@@ -450,7 +454,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
 template <int D, bool KEY>
 static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
-                              void* out, int T, float theta, int init, int window, int shape, cudaStream_t st) {
+                              void* out, int T, float theta, int init, int window, int shape, bool reverse,
+                              cudaStream_t st) {
   const uint64_t BH = (uint64_t)s.B * s.H, BKV = (uint64_t)s.B * s.H_kv;
   const uint64_t ref_heads = KEY ? BKV : BH;   // the reference rows follow the delta stream
   CUtensorMap tq, tqh, tk, tv;
@@ -472,7 +477,8 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
   p.counters = w.counters;
   p.ckpt = w.ckpt;
   p.T_max = s.T_max; p.n_ckpt = s.n_ckpt();
-  p.theta = theta; p.basis_exact = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
+  p.theta = theta; p.reverse = reverse ? 1 : 0;
+  p.basis_row = (init == DELTA_INIT_BASIS_EXACT) ? (reverse ? T - 1 : 0) : -1;
   p.T = T; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
   p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   // Launched with programmatic stream serialisation: the CTAs become resident and run their
@@ -497,14 +503,15 @@ bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
 
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
                                    const void* v, void* out, int T, float theta, int init, int window,
-                                   int shape, bool key_deltas, cudaStream_t st) {
+                                   int shape, bool key_deltas, bool reverse, cudaStream_t st) {
+  if (key_deltas && reverse) return cudaErrorNotSupported;
   if (!w.qhat_rows) return cudaErrorNotSupported;
   if (s.d == 64)
-    return key_deltas ? launch_tcq<64, true>(s, w, q, k, v, out, T, theta, init, window, shape, st)
-                      : launch_tcq<64, false>(s, w, q, k, v, out, T, theta, init, window, shape, st);
+    return key_deltas ? launch_tcq<64, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st)
+                      : launch_tcq<64, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
   if (s.d == 128)
-    return key_deltas ? launch_tcq<128, true>(s, w, q, k, v, out, T, theta, init, window, shape, st)
-                      : launch_tcq<128, false>(s, w, q, k, v, out, T, theta, init, window, shape, st);
+    return key_deltas ? launch_tcq<128, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st)
+                      : launch_tcq<128, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
   return cudaErrorNotSupported;
 }
 

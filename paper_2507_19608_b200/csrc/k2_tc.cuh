@@ -16,5 +16,5 @@ bool tcq_kernel_shape(int d);
 // on the tensor cores; w.qhat_rows holds the reference rows of the delta stream.
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
                                    const void* v, void* out, int T, float theta, int init, int window,
-                                   int shape, bool key_deltas, cudaStream_t st);
+                                   int shape, bool key_deltas, bool reverse, cudaStream_t st);
 }  // namespace delta

@@ -44,6 +44,9 @@ def test_status_strings():
     (dict(H=12, H_kv=4), B.DELTA_ERR_UNSUPPORTED),          # group of 3 query heads
     (dict(source=B.DELTA_SRC_KEY), B.DELTA_OK),              # key deltas: bf16 only
     (dict(source=B.DELTA_SRC_KEY, dtype="f32"), B.DELTA_ERR_UNSUPPORTED),
+    (dict(source=B.DELTA_SRC_QUERY_BOTTOM_UP), B.DELTA_OK),    # strategy (2): bf16 only, prefill only
+    (dict(source=B.DELTA_SRC_QUERY_BOTTOM_UP, dtype="f32"), B.DELTA_ERR_UNSUPPORTED),
+    (dict(source=3), B.DELTA_ERR_INVALID_ARG),
     (dict(T_max=0), B.DELTA_ERR_INVALID_ARG),
     (dict(dtype=7), B.DELTA_ERR_INVALID_ARG),
 ])

@@ -471,3 +471,57 @@ def test_key_delta_decode_steps_match_oracle(B, Bn, H, Hk, T, d, theta, W, steps
     assert sd["device_status"] == 0
     sd = sd["decode"]
     assert (sd["nnz"], sd["elements"], sd["macs_done"], sd["macs_dense"]) == (nnz, Bn * Hk * d * steps, done, dense)
+
+
+# ------------------------------------------------------------------ strategy (2): bottom-up query deltas
+BOTTOM_UP_CASES = [
+    # Bn, H, Hk, T,  d,  theta, W,  shape,    init
+    (1, 4, 2, 200, 64, 0.2, 64, "block", "basis_exact"),       # ragged: the basis row sits inside a block
+    (2, 4, 2, 513, 64, 0.15, 100, "sliding", "basis_exact"),
+    (1, 2, 2, 256, 64, 0.3, 0, "block", "basis_exact"),        # no window: every score from the recursion
+    (1, 8, 2, 384, 128, 0.25, 128, "block", "basis_exact"),
+    (1, 2, 1, 1000, 64, 0.29, 64, "block", "zero_state"),
+    (1, 2, 1, 1, 64, 0.1, 4, "block", "basis_exact"),
+]
+
+
+@pytest.mark.parametrize("case", BOTTOM_UP_CASES, ids=[f"T{c[3]}-d{c[4]}-W{c[6]}{c[7][0]}" for c in BOTTOM_UP_CASES])
+def test_bottom_up_query_delta_prefill_matches_oracle(B, case):
+    """Strategy (2) of Section III-A: Eq. 2-3 and Eq. 4 run from the last row up; the basis is
+    the last row.  Outputs within the bf16 bar; delta arrays (indexed by token row) bit-exact."""
+    from tests.gpu_helpers import to_cache, to_dev, to_host_f64
+    Bn, H, Hk, T, d, theta, W, shape, init = case
+    q, k, v = _inputs(Bn, H, Hk, T, d, "bf16", seed=500 + T + d)
+    cfg = B.make_config(Bn, H, Hk, d, T, "bf16", source=B.DELTA_SRC_QUERY_BOTTOM_UP,
+                        prefill_window=B.DELTA_WIN_BLOCK if shape == "block" else B.DELTA_WIN_SLIDING,
+                        init=B.DELTA_INIT_BASIS_EXACT if init == "basis_exact" else B.DELTA_INIT_ZERO_STATE)
+    st = B.delta_state_init(cfg)
+    dq_, kc, vc = to_dev(q, "bf16"), to_cache(k, T, "bf16"), to_cache(v, T, "bf16")
+    out = torch.full_like(dq_, float("nan"))
+    B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, float(theta), int(W))
+    torch.cuda.synchronize()
+    ref, heads = O.prefill_mha(q, k, v, theta, W, shape, init, source="query", order="bottom_up")
+    _check_out(to_host_f64(out), ref, "bf16", "bottom-up prefill out")
+    dq = B.delta_state_view(st, B.DELTA_VIEW_DQ).cpu().numpy()
+    mask = B.delta_state_view(st, B.DELTA_VIEW_MASK).cpu().numpy().view(np.uint32)
+    rnz = B.delta_state_view(st, B.DELTA_VIEW_ROW_NNZ).cpu().numpy().view(np.uint16)
+    idx = B.delta_state_view(st, B.DELTA_VIEW_IDX).cpu().numpy()
+    qh = B.delta_state_view(st, B.DELTA_VIEW_QHAT).cpu().numpy()
+    nnz = done = dense = 0
+    for b in range(Bn):
+        for h in range(H):
+            r = heads[(b, h)]["delta"]          # the oracle's arrays are in processing order: flip to token rows
+            assert np.array_equal(dq[b, h, :T].view(np.uint32), r["dq"][::-1].view(np.uint32)), (b, h)
+            assert np.array_equal(mask[b, h, :T], r["mask"][::-1]), (b, h)
+            assert np.array_equal(rnz[b, h, :T], r["row_nnz"][::-1]), (b, h)
+            assert np.array_equal(idx[b, h, :T], r["idx"][::-1]), (b, h)
+            assert np.array_equal(qh[b, h].view(np.uint32), r["ahat"].view(np.uint32)), (b, h)
+            c = O.stage_stats(r["row_nnz"][::-1], list(range(T)), d, W, shape)
+            nnz += c["nnz"]; done += c["macs_done"]; dense += c["macs_dense"]
+    s = B.delta_sparsity_stats(st)
+    assert (s["prefill"]["nnz"], s["prefill"]["macs_done"], s["prefill"]["macs_dense"]) == (nnz, done, dense)
+    assert s["device_status"] == 0
+    # the method has no decode stage
+    with pytest.raises(B.DeltaError):
+        B.delta_attn_decode_step(st, dq_[:, :, 0].contiguous(), kc[:, :, 0].contiguous(), vc[:, :, 0].contiguous(),
+                                 kc, vc, out[:, :, 0].contiguous(), float(theta), 4)
