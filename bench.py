@@ -336,6 +336,7 @@ def run_ours(args):
         line["decode"] = run_decode(args, B, torch, peaks)
         line["key_deltas"] = run_key_deltas(args, B, torch, w, tens, theta, flush, peaks)
         line["strategies"] = run_strategy_errors(B, torch, w, tens, theta)
+        line["window_grid"] = run_window_grid(B, torch, flush, theta)
         line["delta_pass_large"] = run_delta_pass_large(B, torch, peaks, flush)
         line["cpu_baseline"] = run_cpu_baseline(args, w, tens, theta)
     print(json.dumps(line))
@@ -562,6 +563,67 @@ def run_strategy_errors(B, torch, w, tens, theta):
                      "mean_abs_err_last_quarter": float(err[:, :, -(w.T // 4):].mean()),
                      "S_m": stt["S_m"], "S_c_exact": stt["S_c_exact"]}
     return res
+
+
+
+def run_window_grid(B, torch, flush, theta):
+    """Eq. 5: the prefill window follows the input length, W = min(floor(gamma n), W_max).  One
+    sequence of every length at the Llama-3.2-1B layer shape, the paper's gamma grid, and its
+    decode window W_d = 4 (64 steps after the longest prefill): delta sparsity, computational
+    sparsity (Eq. 6 and exact) and time per call."""
+    base = WL.WORKLOADS["llama32_1b_prefill"]
+    W_MAX = 256
+    rows = []
+    for n in (128, 256, 512, 1024, 2048, 4096):
+        tens = WL.make_qkv(base, T=n, n_decode=0)
+        q, k, v = (to_dev(tens[x], base.dtype, torch) for x in ("q", "k", "v"))
+        out = torch.empty_like(q)
+        st = B.delta_state_init(B.make_config(base.B, base.H, base.H_kv, base.d, n, base.dtype))
+        for gamma in (0.02, 0.05, 0.1):
+            W = B.delta_window_from_gamma(n, gamma, W_MAX)
+            ms = []
+            for i in range(6):
+                flush.zero_()
+                B.delta_state_reset(st)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                B.delta_attn_prefill(st, q, k, v, out, n, base.H, base.H_kv, base.d, theta, W)
+                e1.record()
+                torch.cuda.synchronize()
+                if i >= 2:
+                    ms.append(e0.elapsed_time(e1))
+            s_ = B.delta_sparsity_stats(st)["prefill"]
+            rows.append({"n": n, "gamma": gamma, "W": W, "ms": statistics.mean(ms), "S_m": s_["S_m"],
+                         "S_c_eq6": s_["S_c_eq6"], "S_c_exact": s_["S_c_exact"]})
+    # decode with the paper's W_d = 4 behind a prefill with gamma = 0.05
+    w = WL.WORKLOADS["llama32_1b_decode_b1"]
+    steps = 64
+    tens = WL.make_qkv(w, n_decode=steps)
+    st = B.delta_state_init(B.make_config(w.B, w.H, w.H_kv, w.d, w.T + steps, w.dtype,
+                                          prefill_window=B.DELTA_WIN_BLOCK))
+    q = to_dev(tens["q"], w.dtype, torch)
+
+    def cache(x):
+        full = np.zeros((w.B, w.H_kv, w.T + steps, w.d), np.float32)
+        full[:, :, :w.T] = x
+        return to_dev(full, w.dtype, torch)
+    kc, vc = cache(tens["k"]), cache(tens["v"])
+    out = torch.empty_like(q)
+    W = B.delta_window_from_gamma(w.T, 0.05, W_MAX)
+    B.delta_attn_prefill(st, q, kc, vc, out, w.T, w.H, w.H_kv, w.d, theta, W)
+    qd, kd, vd = (to_dev(np.ascontiguousarray(tens[x].transpose(2, 0, 1, 3)), w.dtype, torch)
+                  for x in ("q_dec", "k_dec", "v_dec"))
+    od = torch.empty_like(qd)
+    for s in range(steps):
+        B.delta_attn_decode_step(st, qd[s], kd[s], vd[s], kc, vc, od[s], theta, 4)
+    torch.cuda.synchronize()
+    st_all = B.delta_sparsity_stats(st)
+    return {"theta": theta, "W_max": W_MAX, "prefill": rows,
+            "prefill_plus_decode": {"n": w.T, "gamma": 0.05, "W": W, "W_d": 4, "decode_steps": steps,
+                                    "S_c_exact_prefill": st_all["prefill"]["S_c_exact"],
+                                    "S_c_exact_decode": st_all["decode"]["S_c_exact"],
+                                    "S_c_exact_combined": st_all["combined"]["S_c_exact"],
+                                    "S_c_eq6_combined": st_all["combined"]["S_c_eq6"]}}
 
 
 def run_delta_pass_large(B, torch, peaks, flush):

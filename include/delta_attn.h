@@ -213,8 +213,11 @@ typedef struct {
  * Synchronises `stream`.  host_out is a HOST pointer. */
 DELTA_API delta_status_t delta_sparsity_stats(const delta_state_t* st, delta_stats_t* host_out, void* stream);
 
-/* Eq. 5: W_p,max = min(floor(gamma * n), w_max). */
-DELTA_API int32_t delta_window_from_gamma(int32_t n, float gamma, int32_t w_max);
+/* Eq. 5: W_p,max = min(floor(gamma * n), w_max), the product taken in double precision.
+ * gamma is a double so that a decimal scaling factor gives the window the formula gives on
+ * paper (floor(0.02 * 100) = 2; the float nearest to 0.02 lies below it and would give 1).
+ * Returns 0 for n < 0, gamma < 0 or NaN. */
+DELTA_API int32_t delta_window_from_gamma(int32_t n, double gamma, int32_t w_max);
 
 /* Device views into the state's workspace, for parity checks and checkpointing.
  * Shapes (T_max rows allocated, rows 0..T-1 valid after a prefill of T tokens):

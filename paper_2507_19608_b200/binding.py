@@ -84,7 +84,7 @@ def _load() -> C.CDLL:
         "delta_attn_prefill_host": (C.c_int, [vp, vp, vp, vp, vp, vp, sz, i32, f32, i32, vp]),
         "delta_attn_decode_step": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, f32, i32, vp]),
         "delta_sparsity_stats": (C.c_int, [vp, C.POINTER(delta_stats_t), vp]),
-        "delta_window_from_gamma": (i32, [i32, f32, i32]),
+        "delta_window_from_gamma": (i32, [i32, C.c_double, i32]),
         "delta_state_view": (C.c_int, [vp, i32, C.POINTER(vp), C.POINTER(sz)]),
         "delta_state_position": (i32, [vp]),
         "delta_state_prefill_kernel": (i32, [vp]),

@@ -376,9 +376,9 @@ delta_status_t delta_sparsity_stats(const delta_state_t* st, delta_stats_t* host
   return host_out->device_status == 0 ? DELTA_OK : (delta_status_t)host_out->device_status;
 }
 
-int32_t delta_window_from_gamma(int32_t n, float gamma, int32_t w_max) {
-  if (n < 0 || !(gamma >= 0.0f)) return 0;
-  const double w = std::floor((double)gamma * (double)n);
+int32_t delta_window_from_gamma(int32_t n, double gamma, int32_t w_max) {
+  if (n < 0 || !(gamma >= 0.0)) return 0;
+  const double w = std::floor(gamma * (double)n);
   const double m = w < (double)w_max ? w : (double)w_max;
   return m < 0.0 ? 0 : (int32_t)m;
 }

@@ -79,6 +79,13 @@ def test_null_and_misaligned_arguments_are_rejected_before_any_device_work():
 
 
 @pytest.mark.parametrize("n,gamma,wmax", [(1000, 0.05, 64), (1000, 0.1, 64), (10, 0.05, 64),
-                                          (120, 0.25, 1 << 30), (4096, 0.02, 256), (0, 0.5, 8)])
+                                          (120, 0.25, 1 << 30), (4096, 0.02, 256), (0, 0.5, 8),
+                                          (100, 0.02, 48), (257, 0.1, 16), (640, 0.05, 48)])
 def test_window_from_gamma_matches_eq5(n, gamma, wmax):
     assert B.delta_window_from_gamma(n, gamma, wmax) == O.window_from_gamma(n, gamma, wmax)
+
+
+def test_window_from_gamma_out_of_domain_is_zero():
+    assert B.delta_window_from_gamma(-3, 0.5, 8) == 0
+    assert B.delta_window_from_gamma(100, -0.1, 8) == 0
+    assert B.delta_window_from_gamma(100, float("nan"), 8) == 0

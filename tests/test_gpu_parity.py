@@ -525,3 +525,37 @@ def test_bottom_up_query_delta_prefill_matches_oracle(B, case):
     with pytest.raises(B.DeltaError):
         B.delta_attn_decode_step(st, dq_[:, :, 0].contiguous(), kc[:, :, 0].contiguous(), vc[:, :, 0].contiguous(),
                                  kc, vc, out[:, :, 0].contiguous(), float(theta), 4)
+
+
+# ------------------------------------------------------------------ Eq. 5: window from the input length
+@pytest.mark.parametrize("n", [100, 257, 640])
+@pytest.mark.parametrize("gamma", [0.02, 0.05, 0.1])
+def test_eq5_dynamic_window_prefill_and_decode(B, n, gamma):
+    """Section III-B: the prefill window follows the input length, W = min(floor(gamma n), W_max),
+    squares along the diagonal; decode uses the paper's fixed W_d = 4.  Outputs and the Eq. 6
+    statistics of both stages against the oracle."""
+    from tests.gpu_helpers import run_prefill, to_dev, to_host_f64
+    H, Hk, d, theta, W_max, W_d, steps = 4, 2, 64, 0.25, 48, 4, 3
+    W = B.delta_window_from_gamma(n, gamma, W_max)
+    assert W == O.window_from_gamma(n, gamma, W_max)
+    w = WL.Workload("t", 1, H, Hk, n, d, "bf16", 0.95, 0.5, W, (), 900 + n)
+    t = WL.make_qkv(w, n_decode=steps)
+    q, k, v = t["q"], t["k"], t["v"]
+    st, out, kc, vc = run_prefill(B, q, k, v, theta, W, "bf16", T_max=n + steps)
+    ref, heads = O.prefill_mha(q, k, v, theta, W, "block")
+    _check_out(to_host_f64(out), ref, "bf16", f"prefill n={n} gamma={gamma} W={W}")
+    states = {key: h["state"] for key, h in heads.items()}
+    for s_ in range(steps):
+        qn, kn, vn = t["q_dec"][:, :, s_], t["k_dec"][:, :, s_], t["v_dec"][:, :, s_]
+        o = torch.empty_like(to_dev(qn, "bf16"))
+        B.delta_attn_decode_step(st, to_dev(qn, "bf16"), to_dev(kn, "bf16"), to_dev(vn, "bf16"), kc, vc, o,
+                                 float(theta), W_d)
+        ref_o, _ = O.decode_mha(states, qn, kn, vn, theta, W_d)
+        _check_out(to_host_f64(o), ref_o, "bf16", f"decode step {s_}")
+    stats = B.delta_sparsity_stats(st)
+    rn = np.concatenate([heads[(0, h)]["delta"]["row_nnz"] for h in range(H)])
+    want = O.finish_stats(O.stage_stats(rn, [i for _ in range(H) for i in range(n)], d, W, "block"), min(W, n), n)
+    got = stats["prefill"]
+    assert (got["nnz"], got["macs_done"], got["macs_dense"]) == (want["nnz"], want["macs_done"], want["macs_dense"])
+    assert abs(got["S_c_eq6"] - want["S_c_eq6"]) < 1e-6 and abs(got["S_c_exact"] - want["S_c_exact"]) < 1e-9
+    assert stats["device_status"] == 0
