@@ -146,11 +146,17 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   tc_fence_after();
   const uint32_t tmem = sMisc[0];
 
+  // Keys that some row of this query tile scores exactly: ex_lo <= j <= ex_hi (empty if W = 0).
+  // Block window: the window blocks that rows i0..i1 fall into; sliding: i0-W+1 .. i1.
+  // Computed once: the per-tile test below must not divide.
+  int ex_lo = 1, ex_hi = 0;
+  if (W > 0) {
+    if (shape == 0) { ex_lo = (i0 / W) * W; ex_hi = (i1 / W) * W + W - 1; }
+    else { ex_lo = i0 - W + 1; ex_hi = i1; }
+  }
   auto tile_needs_exact = [&](int jt) -> bool {
-    if (W <= 0) return false;
     const int j0 = jt * BN, j1 = min(j0 + BN, T) - 1;
-    if (shape == 0) return (i0 / W <= j1 / W) && (j0 / W <= i1 / W);
-    return max(0, i0 - j1) < W;
+    return j1 >= ex_lo && j0 <= ex_hi;
   };
 
   if (warp == NCWARP) {
