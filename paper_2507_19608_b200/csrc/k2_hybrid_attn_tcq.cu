@@ -364,9 +364,10 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (jc0 + c > i) s[c] = -INFINITY;     // causal mask on the diagonal tile
       }
       // row maximum: own 32 columns, then the three other quarters through shared memory
-      float mx = s[0];
+      float mx = fmax3(s[0], s[1], s[2]);
 #pragma unroll
-      for (int c = 1; c < 32; ++c) mx = fmaxf(mx, s[c]);
+      for (int c = 3; c < 31; c += 2) mx = fmax3(mx, s[c], s[c + 1]);
+      mx = fmaxf(mx, s[31]);
       sPmax[(bf * BM + row) * 4 + sub] = mx;
       quad_sync(qd);   // the four warps of this quadrant
       const float4 pm = *reinterpret_cast<const float4*>(sPmax + (bf * BM + row) * 4);
@@ -374,13 +375,16 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const float m_new = fmaxf(m_run, mx * scale);
       const float al = ex2(m_run - m_new);
       m_run = m_new;
-      float sum = 0.0f;
+      float2 sum2 = make_float2(0.0f, 0.0f);
+      const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-m_new, -m_new);
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        s[c] = ex2(fmaf(s[c], scale, -m_new));
-        sum += s[c];
+      for (int c = 0; c < 32; c += 2) {
+        const float2 t = ffma2(make_float2(s[c], s[c + 1]), sc2, nm2);
+        s[c] = ex2(t.x);
+        s[c + 1] = ex2(t.y);
+        sum2 = fadd2(sum2, make_float2(s[c], s[c + 1]));
       }
-      l_part = fmaf(l_part, al, sum);
+      l_part = fmaf(l_part, al, sum2.x + sum2.y);
 
       // the previous tile's P.V is done: the P buffer may be rewritten
       if (jt > 0) mbar_wait(BAR(BAR_O), (jt - 1) & 1, abort_flag);
@@ -408,8 +412,13 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int h16 = 0; h16 < OC / 16; ++h16) {
           float v[16];
           tc_ld16(tmem + TMEM_O + OC * sub + 16 * h16 + lane_sel, v);
+          const float2 ap2 = make_float2(alpha_prev, alpha_prev);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) O[16 * h16 + c] = fmaf(O[16 * h16 + c], alpha_prev, v[c]);
+          for (int c = 0; c < 16; c += 2) {
+            const float2 o = ffma2(make_float2(O[16 * h16 + c], O[16 * h16 + c + 1]), ap2, make_float2(v[c], v[c + 1]));
+            O[16 * h16 + c] = o.x;
+            O[16 * h16 + c + 1] = o.y;
+          }
         }
         tc_fence_before();
       }
