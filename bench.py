@@ -512,13 +512,16 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
             graph_ok = f"capture failed: {type(ex).__name__}"
         es = 2
         n_avg = w.T + (w.n_decode - 1) / 2.0
-        # K (or reference-key) and V rows once per KV head; query deltas also read and write the score row R
-        bytes_step = w.B * (2 * w.H_kv * n_avg * w.d * es + (0 if key else 2 * w.H * n_avg * 4))
+        # K (or reference-key) and V rows once per KV head; query deltas also write the score row R
+        # (and read it, where the step runs on the FP32 pipes: the tensor-core form recomputes it)
+        r_passes = 0 if key else (1 if B.delta_state_decode_kernel(st) == 1 else 2)
+        bytes_step = w.B * (2 * w.H_kv * n_avg * w.d * es + r_passes * w.H * n_avg * 4)
         best = graph_us if graph_us else min(eager)
         gbs = bytes_step / (best * 1e-6) / 1e9
         res[f"batch{w.B}"] = {
             "us_per_step_eager": statistics.median(eager), "us_per_step_graph": graph_us,
-            "graph_matches_eager": graph_ok, "steps": w.n_decode, "cache_tokens": w.T, "theta": theta,
+            "graph_matches_eager": graph_ok, "steps": w.n_decode,
+            "decode_kernel": "FP32 pipes" if key or B.delta_state_decode_kernel(st) != 1 else "tensor-core scores", "cache_tokens": w.T, "theta": theta,
             "window": w.window, "algorithmic_bytes_per_step": bytes_step,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
                          "frac": gbs / float(peaks["hbm_gbs"]),

@@ -151,6 +151,10 @@ DELTA_API delta_status_t delta_attn_prefill_host(delta_state_t* st, const void* 
  * that arrives now; score j is q_new.k_j if n - j < window else R[j]; softmax over the n + 1
  * keys; out = P.V; position becomes n + 1.  Needs n >= 1 (else DELTA_ERR_STATE) and
  * n < T_max (else DELTA_ERR_CAPACITY).
+ * Eq. 4's sum telescopes to R[j] = q_hat . k_j (exactly, up to the order of the fp32
+ * additions, for bf16 inputs, whose references are copies of input elements); where
+ * delta_state_decode_kernel reports 1 the step computes R[j] in that form on the tensor cores
+ * and writes it back without reading it.  k_cache must then be 16-byte aligned.
  * With DELTA_SRC_KEY the step thresholds k_new against the carried reference key instead
  * (Eq. 2-3), appends the reference-key row k_hat(n), and scores key j with q_new.k_j if
  * n - j < window else q_new.k_hat(j). */
@@ -250,6 +254,12 @@ DELTA_API int32_t delta_state_position(const delta_state_t* st);
  * (-1 = automatic); forcing a kernel the configuration has none for returns
  * DELTA_ERR_UNSUPPORTED. */
 DELTA_API int32_t delta_state_prefill_kernel(const delta_state_t* st);
+
+/* Which kernel the next delta_attn_decode_step of this state would use: 1 = score products
+ * on the tensor cores (bf16, d = 64, query deltas, key slices of at least two 128-key tiles:
+ * the telescoped form of Eq. 4, see delta_attn_decode_step), 0 = the FP32-pipe kernel,
+ * -1 for a null state.  Both compute the same step and keep the same state. */
+DELTA_API int32_t delta_state_decode_kernel(const delta_state_t* st);
 DELTA_API delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which);
 
 /* Per-kernel timing of delta_attn_prefill.  With profiling enabled the call records a CUDA

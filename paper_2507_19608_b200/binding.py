@@ -29,7 +29,8 @@ EXPORTED = [
     "delta_state_workspace_bytes", "delta_state_init", "delta_state_reset", "delta_state_destroy",
     "delta_attn_prefill", "delta_prefill_staging_bytes", "delta_attn_prefill_host",
     "delta_attn_decode_step", "delta_sparsity_stats", "delta_window_from_gamma", "delta_state_view",
-    "delta_state_position", "delta_state_prefill_kernel", "delta_state_set_prefill_kernel",
+    "delta_state_position", "delta_state_prefill_kernel", "delta_state_decode_kernel",
+    "delta_state_set_prefill_kernel",
     "delta_launch_count", "delta_status_string", "delta_last_cuda_error",
     "delta_state_enable_profiling", "delta_state_prefill_kernel_ms",
     "delta_attn_decode_step_noalloc",
@@ -88,6 +89,7 @@ def _load() -> C.CDLL:
         "delta_state_view": (C.c_int, [vp, i32, C.POINTER(vp), C.POINTER(sz)]),
         "delta_state_position": (i32, [vp]),
         "delta_state_prefill_kernel": (i32, [vp]),
+        "delta_state_decode_kernel": (i32, [vp]),
         "delta_state_set_prefill_kernel": (C.c_int, [vp, i32]),
         "delta_state_enable_profiling": (C.c_int, [vp, i32]),
         "delta_state_prefill_kernel_ms": (C.c_int, [vp, C.POINTER(C.c_float)]),
@@ -225,6 +227,10 @@ def delta_state_position(st: DeltaState) -> int:
 
 def delta_state_prefill_kernel(st: DeltaState) -> int:
     return lib.delta_state_prefill_kernel(st.handle)
+
+
+def delta_state_decode_kernel(st: DeltaState) -> int:
+    return lib.delta_state_decode_kernel(st.handle)
 
 
 def delta_state_set_prefill_kernel(st: DeltaState, which: int):

@@ -31,6 +31,7 @@ struct delta_state {
   int forced_kernel;  // -1 auto, 0 generic, 1 tensor-core
   // Eq. 6 bookkeeping that needs no device work: sum of window lengths and sequence lengths
   double win_sum[2], len_sum[2];
+  DecodeTmapCache dec_tmap;   // tensor map of the key cache the decode steps read
   // optional per-kernel timing of prefill (host-side event objects)
   bool profiling = false, profiled = false;
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -195,6 +196,12 @@ int32_t delta_state_prefill_kernel(const delta_state_t* st) {
   return tc_eligible(st, 2) ? 2 : 0;   // the telescoped tensor-core kernel is the fastest where it applies
 }
 
+int32_t delta_state_decode_kernel(const delta_state_t* st) {
+  if (!st) return -1;
+  if (st->cfg.source != DELTA_SRC_QUERY) return 0;
+  return decode_tc_applies(st->shape, st->cfg.dtype, st->n) ? 1 : 0;
+}
+
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
   if (!st || which < -1 || which > 2) return DELTA_ERR_INVALID_ARG;
   if (which >= 1 && !tc_eligible(st, which)) return DELTA_ERR_UNSUPPORTED;
@@ -334,6 +341,9 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
       st->cfg.source == DELTA_SRC_KEY
           ? launch_decode_step_key(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n,
                                    theta, window, st->qhat_sel, (cudaStream_t)stream)
+      : decode_tc_applies(st->shape, st->cfg.dtype, st->n)
+          ? launch_decode_step_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
+                                  window, st->qhat_sel, &st->dec_tmap, (cudaStream_t)stream)
           : launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n,
                                theta, window, st->cfg.dtype, st->qhat_sel, (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e);

@@ -79,6 +79,18 @@ cudaError_t launch_decode_step(const Shape& s, const Workspace& w, const void* q
                                cudaStream_t st);
 
 // K3 (key deltas): one decode step of strategy (3); bf16 only, needs w.qhat_rows (reference-key cache).
+// K3 with the score products on the tensor cores (bf16, d = 64): same step, same state.
+// Host-side cache of the key cache's tensor map (encoded once per cache pointer, not per step).
+struct DecodeTmapCache {
+  const void* ptr = nullptr;
+  alignas(64) unsigned char map[128];
+};
+// Does the step at position n take this kernel?  (bf16, d = 64, and key slices of at least two
+// tiles: with short slices the per-CTA set-up outweighs the saving.)
+bool decode_tc_applies(const Shape& s, int dtype, int n);
+cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
+                                  const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
+                                  int window, int qhat_sel, DecodeTmapCache* cache, cudaStream_t st);
 cudaError_t launch_decode_step_key(const Shape& s, const Workspace& w, const void* q_new,
                                    const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                    void* out, int n, float theta, int window, int qhat_sel,

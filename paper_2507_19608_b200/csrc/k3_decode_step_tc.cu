@@ -1,0 +1,417 @@
+// K3 (tensor-core scores) -- one decode step of strategy (1) for bf16 caches with d = 64
+// (Section III-A "Decoding Stage Considerations", Section III-B "Decoding Stage").
+//
+// Eq. 4's running sum telescopes: R(n)[j] = (sum of all Delta q so far) . k_j = q_hat(n) . k_j,
+// and for bf16 inputs every element of q_hat is a copy of an input element, so the whole score
+// row of a step is two small dense products per cached key: q_hat . k_j (outside the window) and
+// q . k_j (the W_d most recent keys).  Both come from ONE tensor-core product per 128-key tile,
+//   S[128 keys][16] = K_tile[128][64] . Qcat[16][64]^T,
+// where the rows of Qcat are the G new reference vectors, the G new query vectors and zeros.
+// The score row R is no longer read; it is written (R[j] = q_hat . k_j) because it is part of
+// the carried state.  The FP32 pipes keep what is not a contraction of useful shape: the
+// threshold step (Eq. 2-3), the softmax and P.V (G rows of P against the value tile).
+//
+// Grid = (key slices, batch x KV heads); a CTA serves the G query heads of one KV head.
+//   1. threshold q_new against the carried reference, build Qcat in the operand layout;
+//   2. thread 0 streams the slice's key tiles with TMA (128-byte swizzle, two stages) and issues
+//      the products; all score tiles of the slice stay in tensor memory (16 columns per tile);
+//   3. one softmax over the slice: every thread reads its keys' scores (lane = key), hybrid
+//      select, scale, R written; maximum and sum reduced once per slice, not per tile;
+//   4. P.V with the value tiles streamed through a two-stage ring of bulk copies;
+//   5. the slice result is stored and the last CTA of the (batch, KV head) merges the slices.
+// The key and value that arrive with this step are scored on the FP32 pipes by the CTA that
+// owns their slice (their cache row is written by this very kernel).
+// Every wait is bounded; after a time-out the kernel still runs to its end and the status word
+// records DELTA_ERR_TIMEOUT.
+#include <cuda.h>
+
+#include "decode_common.cuh"
+#include "k2_tc.cuh"
+#include "tc_common.cuh"
+
+namespace delta {
+
+namespace {
+
+constexpr int TCD = 64;                // head dimension
+constexpr int TK = 128;                // keys per tile
+constexpr int MAXT = 9;                // tiles per slice at most (1152 keys)
+constexpr int SCOL = 16;               // tensor-memory columns per tile (N of the product)
+constexpr uint32_t DEC_TMEM_COLS = 256;
+
+enum { BAR_K0 = 0, BAR_K1, BAR_KFREE0, BAR_KFREE1, BAR_S, BAR_V0, BAR_V1, DEC_NUM_BARS };
+
+}  // namespace
+
+template <int G>
+__global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
+    const __grid_constant__ CUtensorMap tm_k, const __nv_bfloat16* __restrict__ q_new,
+    const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
+    __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
+    __nv_bfloat16* __restrict__ out, const float* __restrict__ qhat_in, float* __restrict__ qhat_out,
+    float* __restrict__ R, float* __restrict__ partial, uint32_t* __restrict__ ticket,
+    unsigned long long* __restrict__ counters, int n, int T_max, int H, int chunk, int nsplit,
+    float theta, int W, float scale_log2e) {
+  using TC = __nv_bfloat16;
+  constexpr int D = TCD;
+  constexpr int LPK = D / 8, KPW = 32 / LPK;
+  extern __shared__ unsigned char dsm_raw0[];
+  const uint32_t raw = smem_u32(dsm_raw0);
+  const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled operand tiles want 1 KiB alignment
+  unsigned char* sm = dsm_raw0 + (base - raw);
+  constexpr uint32_t OFF_K = 0;                          // [2][128][64] bf16, 128-byte swizzle
+  constexpr uint32_t OFF_V = OFF_K + 2 * TILE_BYTES;     // [2][128][64] bf16, plain rows
+  constexpr uint32_t OFF_QC = OFF_V + 2 * TILE_BYTES;    // Qcat [16][64] bf16, 128-byte swizzle
+  constexpr uint32_t OFF_F = OFF_QC + 2048;              // floats from here on
+  float* q_s = reinterpret_cast<float*>(sm + OFF_F);     // [G][D]
+  float* qh_s = q_s + G * D;                             // [G][D]
+  float* red = qh_s + G * D;                             // [DNW][G][D]
+  float* wgt = red + DNW * G * D;                        // [G * kMaxDecodeSplits] (merge) / [DNW][2G] (reductions)
+  float* p_s = wgt + G * kMaxDecodeSplits;               // [MAXT * TK + 1][G] probabilities
+  float* st_s = p_s + (MAXT * TK + 1) * G;               // [24]
+  __shared__ __align__(8) unsigned long long bars[DEC_NUM_BARS];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_last, s_fail;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int split = blockIdx.x, bkv = blockIdx.y;
+  const int H_kv = H / G;
+  const int b = bkv / H_kv, kvh = bkv - b * H_kv;
+  const int L = n + 1;
+  const int j0 = split * chunk;
+  const int len = max(0, min(chunk, L - j0));            // keys of the slice, the new one included
+  const int cached = max(0, min(len, n - j0));           // of which already in the cache
+  const int n_tiles = (cached + TK - 1) / TK;            // tiles that go through the tensor cores
+  const bool has_new = (n >= j0) && (n < j0 + len);
+  const uint32_t bar0 = smem_u32(&bars[0]);
+#define DBAR(i) (bar0 + 8u * (uint32_t)(i))
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
+                 "r"(DEC_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    for (int i = 0; i < DEC_NUM_BARS; ++i) tc::mbar_init(DBAR(i), 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
+  }
+
+  // ---- 1. delta of the new query rows against the carried reference (Eq. 2-3); Qcat
+  int fired_total = 0;
+  for (int e0 = 0; e0 < G * D; e0 += DNT) {
+    const int e = e0 + tid;
+    bool fire = false;
+    if (e < G * D) {
+      const int hh = e / D, c = e - hh * D;
+      const size_t o = ((size_t)b * H + kvh * G + hh) * D + c;
+      const TC xb = q_new[o];
+      const float x = to_f32(xb);
+      const float old = qhat_in[o];
+      fire = fabsf(__fsub_rn(x, old)) > theta;
+      const float nq = fire ? x : old;
+      q_s[e] = x;
+      qh_s[e] = nq;
+      if (split == 0) qhat_out[o] = nq;
+      // operand rows: hh = new reference (exactly bf16), G + hh = new query
+      auto qc_off = [&](int r) -> uint32_t {
+        return (uint32_t)r * 128u + ((((uint32_t)c >> 3) ^ ((uint32_t)r & 7u)) << 4) + ((uint32_t)c & 7u) * 2u;
+      };
+      *reinterpret_cast<uint16_t*>(sm + OFF_QC + qc_off(hh)) = (uint16_t)(__float_as_uint(nq) >> 16);
+      *reinterpret_cast<TC*>(sm + OFF_QC + qc_off(G + hh)) = xb;
+    }
+    fired_total += __syncthreads_count(fire);
+  }
+  for (int e = tid; e < (16 - 2 * G) * D; e += DNT) {       // unused operand rows: zeros
+    const int r = 2 * G + e / D, c = e % D;
+    *reinterpret_cast<uint16_t*>(sm + OFF_QC + (uint32_t)r * 128u + ((((uint32_t)c >> 3) ^ ((uint32_t)r & 7u)) << 4) +
+                                 ((uint32_t)c & 7u) * 2u) = 0;
+  }
+  if (split == 0 && tid == 0) {
+    const int n_in = min(L, max(W, 0));
+    const int n_out = L - n_in;
+    atomicAdd(&counters[CNT_DECODE_NNZ], (unsigned long long)fired_total);
+    atomicAdd(&counters[CNT_DECODE_ELEMS], (unsigned long long)G * D);
+    atomicAdd(&counters[CNT_DECODE_MACS_DONE],
+              (unsigned long long)n_in * D * G + (unsigned long long)n_out * fired_total);
+    atomicAdd(&counters[CNT_DECODE_MACS_DENSE], (unsigned long long)L * D * G);
+  }
+  if (tid < 8) { st_s[tid] = -INFINITY; st_s[8 + tid] = 0.0f; }
+  tc::fence_proxy_async();           // Qcat was written through the generic proxy
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem = s_tmem;
+
+  const TC* vc = v_cache + (size_t)bkv * T_max * D;
+  auto v_rows = [&](int t) { return min(TK, cached - t * TK); };
+  auto issue_v = [&](int t) {
+    const uint32_t bytes = (uint32_t)v_rows(t) * D * 2u;
+    const uint32_t bar = DBAR(BAR_V0 + (t & 1));
+    tc::mbar_expect_tx(bar, bytes);
+    bulk_load(base + OFF_V + (t & 1) * TILE_BYTES, vc + (size_t)(j0 + t * TK) * D, bytes, bar);
+  };
+
+  // ---- 2. key tiles through the tensor cores (one thread)
+  if (tid == 0 && n_tiles > 0) {
+    const uint32_t IDESC = tc::make_idesc(SCOL, 0);
+    auto issue_k = [&](int t) {
+      tc::mbar_expect_tx(DBAR(BAR_K0 + (t & 1)), TILE_BYTES);
+      tc::tma_load_3d(base + OFF_K + (t & 1) * TILE_BYTES, &tm_k, DBAR(BAR_K0 + (t & 1)), 0, j0 + t * TK, bkv);
+    };
+    issue_k(0);
+    if (n_tiles > 1) issue_k(1);
+    issue_v(0);
+    if (n_tiles > 1) issue_v(1);
+    for (int t = 0; t < n_tiles; ++t) {
+      if (!mbar_wait(DBAR(BAR_K0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
+      tc::tc_fence_after();
+      const uint32_t kb = base + OFF_K + (t & 1) * TILE_BYTES;
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks)
+        tc::tc_mma(tmem + SCOL * t, tc::make_desc(kb + ks * 32, 16, 1024),
+                   tc::make_desc(base + OFF_QC + ks * 32, 16, 1024), IDESC, ks > 0 ? 1u : 0u);
+      if (t + 2 < n_tiles) {
+        // the stage is free once these products are done: then refill it
+        tc::tc_commit(DBAR(BAR_KFREE0 + (t & 1)));
+        if (!mbar_wait(DBAR(BAR_KFREE0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
+        issue_k(t + 2);
+      }
+    }
+    tc::tc_commit(DBAR(BAR_S));
+  }
+
+  // the key and value that arrive with this step: into the cache, scored on the FP32 pipes
+  // (warp 0; results in p_s row MAXT*TK below)
+  float new_s[G];         // scaled hybrid score of the new key, per head (warp 0, all lanes)
+#pragma unroll
+  for (int hh = 0; hh < G; ++hh) new_s[hh] = -INFINITY;
+  if (has_new) {
+    for (int e = tid; e < D; e += DNT) {
+      k_cache[((size_t)bkv * T_max + n) * D + e] = k_new[(size_t)bkv * D + e];
+      v_cache[((size_t)bkv * T_max + n) * D + e] = v_new[(size_t)bkv * D + e];
+    }
+    if (warp == 0) {
+      const float k0 = to_f32(k_new[(size_t)bkv * D + lane]), k1 = to_f32(k_new[(size_t)bkv * D + 32 + lane]);
+#pragma unroll
+      for (int hh = 0; hh < G; ++hh) {
+        float pr = fmaf(qh_s[hh * D + lane], k0, qh_s[hh * D + 32 + lane] * k1);
+        float pq = fmaf(q_s[hh * D + lane], k0, q_s[hh * D + 32 + lane] * k1);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          pr += __shfl_xor_sync(0xffffffffu, pr, o);
+          pq += __shfl_xor_sync(0xffffffffu, pq, o);
+        }
+        if (lane == 0) R[((size_t)b * H + kvh * G + hh) * T_max + n] = pr;     // R[n] = q_hat . k_new
+        new_s[hh] = ((W > 0) ? pq : pr) * scale_log2e;                          // the new key is inside any window
+      }
+    }
+  }
+
+  // ---- 3. one softmax over the slice.  Warp w reads tensor-memory lanes 32 (w % 4) ..; warps
+  // 0..3 take the even tiles, warps 4..7 the odd ones.
+  if (n_tiles > 0) {
+    if (!mbar_wait(DBAR(BAR_S), 0)) s_fail = 1;
+    tc::tc_fence_after();
+  }
+  constexpr int TPW = (MAXT + 1) / 2;     // tiles per warp at most
+  float sv[TPW][G];                       // scaled hybrid scores of this thread's keys
+  float mx[G];
+#pragma unroll
+  for (int hh = 0; hh < G; ++hh) mx[hh] = new_s[hh];
+  const uint32_t lane_sel = (uint32_t)(32 * (warp & 3)) << 16;
+  float* Rg = R + ((size_t)b * H + kvh * G) * T_max;
+#pragma unroll
+  for (int u = 0; u < TPW; ++u) {
+    const int t = 2 * u + (warp >> 2);
+#pragma unroll
+    for (int hh = 0; hh < G; ++hh) sv[u][hh] = -INFINITY;
+    if (t < n_tiles) {                    // warp-uniform
+      float v[16];
+      tc::tc_ld16(tmem + SCOL * t + lane_sel, v);
+      const int jj = t * TK + 32 * (warp & 3) + lane;       // key within the slice
+      const int j = j0 + jj;
+      if (jj < cached) {
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh) {
+          Rg[(size_t)hh * T_max + j] = v[hh];               // R[j] = q_hat . k_j
+          const float s = ((n - j < W) ? v[G + hh] : v[hh]) * scale_log2e;
+          sv[u][hh] = s;
+          mx[hh] = fmaxf(mx[hh], s);
+        }
+      }
+    }
+  }
+  tc::tc_fence_before();
+#pragma unroll
+  for (int hh = 0; hh < G; ++hh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], o));
+    if (lane == 0) wgt[warp * 2 * G + hh] = mx[hh];
+  }
+  __syncthreads();
+  float sum[G];
+#pragma unroll
+  for (int hh = 0; hh < G; ++hh) {
+    float m = wgt[hh];
+#pragma unroll
+    for (int w2 = 1; w2 < DNW; ++w2) m = fmaxf(m, wgt[w2 * 2 * G + hh]);
+    mx[hh] = m;                           // the slice's maximum (never -inf: the slice has a key)
+    sum[hh] = 0.0f;
+  }
+#pragma unroll
+  for (int u = 0; u < TPW; ++u) {
+    const int t = 2 * u + (warp >> 2);
+    if (t < n_tiles) {
+      const int jj = t * TK + 32 * (warp & 3) + lane;
+#pragma unroll
+      for (int hh = 0; hh < G; ++hh) {
+        const float p = exp2f(sv[u][hh] - mx[hh]);          // 0 for keys past the cached rows
+        sum[hh] += p;
+        p_s[(size_t)jj * G + hh] = p;
+      }
+    }
+  }
+  if (warp == 0 && has_new) {
+#pragma unroll
+    for (int hh = 0; hh < G; ++hh) {
+      const float p = exp2f(new_s[hh] - mx[hh]);
+      if (lane == 0) { sum[hh] += p; p_s[(size_t)(MAXT * TK) * G + hh] = p; }
+    }
+  }
+#pragma unroll
+  for (int hh = 0; hh < G; ++hh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum[hh] += __shfl_xor_sync(0xffffffffu, sum[hh], o);
+    if (lane == 0) wgt[warp * 2 * G + G + hh] = sum[hh];
+  }
+  __syncthreads();
+  if (tid < G) {
+    float s = 0.0f;
+    for (int w2 = 0; w2 < DNW; ++w2) s += wgt[w2 * 2 * G + G + tid];
+    st_s[tid] = mx[tid];
+    st_s[8 + tid] = s;
+  }
+
+  // ---- 4. P.V: value tiles through a two-stage ring; lane (l % 8) holds 8 channels, l / 8 the key
+  const int sub = lane / LPK;
+  const int c0 = (lane % LPK) * 8;
+  float acc[G][8];
+#pragma unroll
+  for (int hh = 0; hh < G; ++hh)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[hh][e] = 0.0f;
+  for (int t = 0; t < n_tiles; ++t) {
+    if (!mbar_wait(DBAR(BAR_V0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
+    const TC* vt = reinterpret_cast<const TC*>(sm + OFF_V + (t & 1) * TILE_BYTES);
+    const int rows = v_rows(t);
+    for (int jb = warp * KPW; jb < rows; jb += DNW * KPW) {
+      const int jj = jb + sub;
+      if (jj < rows) {
+        float vv[8];
+        load8(vt + (size_t)jj * D + c0, vv);
+        const float* pp = p_s + (size_t)(t * TK + jj) * G;
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh) {
+          const float p = pp[hh];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[hh][e] = fmaf(p, vv[e], acc[hh][e]);
+        }
+      }
+    }
+    __syncthreads();                      // the stage is free
+    if (tid == 0 && t + 2 < n_tiles) issue_v(t + 2);
+  }
+  if (has_new && warp == 0 && sub == 0) {
+    float vv[8];
+    load8(v_new + (size_t)bkv * D + c0, vv);
+#pragma unroll
+    for (int hh = 0; hh < G; ++hh) {
+      const float p = p_s[(size_t)(MAXT * TK) * G + hh];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[hh][e] = fmaf(p, vv[e], acc[hh][e]);
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    tc::tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(DEC_TMEM_COLS) : "memory");
+  }
+#undef DBAR
+  decode_merge_slices<TC, D, G>(acc, red, wgt, st_s, &s_last, s_fail, partial, ticket, counters, out, split, bkv,
+                                nsplit, b, H, kvh);
+}
+
+// Slice geometry of a step at position n: one wave of two CTAs per SM, no slice shorter than a
+// quarter tile or longer than MAXT tiles.
+static void decode_tc_slices(const Shape& s, int n, int* nsplit_out, int* chunk_out) {
+  const int L = n + 1;
+  const int bkv = s.B * s.H_kv;
+  int nsplit = kDecodeTargetCtas / bkv;
+  if (nsplit > kMaxDecodeSplits) nsplit = kMaxDecodeSplits;
+  const int max_by_len = (L + TK / 4 - 1) / (TK / 4);
+  if (nsplit > max_by_len) nsplit = max_by_len;
+  const int min_by_len = (L + MAXT * TK - 1) / (MAXT * TK);
+  if (nsplit < min_by_len) nsplit = min_by_len;
+  if (nsplit < 1) nsplit = 1;
+  int chunk = (L + nsplit - 1) / nsplit;
+  chunk = (chunk + 31) / 32 * 32;
+  *nsplit_out = (L + chunk - 1) / chunk;
+  *chunk_out = chunk;
+}
+
+bool decode_tc_applies(const Shape& s, int dtype, int n) {
+  if (s.d != TCD || dtype != DELTA_BF16 || tc::encode_fn() == nullptr) return false;
+  int nsplit, chunk;
+  decode_tc_slices(s, n, &nsplit, &chunk);
+  return chunk >= 2 * TK && chunk <= MAXT * TK && nsplit <= kMaxDecodeSplits;
+}
+
+cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
+                                  const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
+                                  int window, int qhat_sel, DecodeTmapCache* cache, cudaStream_t st) {
+  const int bkv = s.B * s.H_kv;
+  int nsplit, chunk;
+  decode_tc_slices(s, n, &nsplit, &chunk);
+  if (nsplit > kMaxDecodeSplits || chunk > MAXT * TK) return cudaErrorInvalidValue;
+  static_assert(sizeof(CUtensorMap) <= sizeof(cache->map), "tensor-map cache");
+  CUtensorMap* tkp = reinterpret_cast<CUtensorMap*>(cache->map);
+  if (cache->ptr != k_cache) {
+    if (!tc::encode3(tkp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k_cache, TCD, (uint64_t)s.T_max, (uint64_t)bkv, TCD * 2,
+                     (uint64_t)s.T_max * TCD * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B))
+      return cudaErrorInvalidValue;
+    cache->ptr = k_cache;
+  }
+  const CUtensorMap& tk = *tkp;
+  const float scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
+  const int G = s.g();
+  const dim3 grid(nsplit, bkv);
+  const size_t smem = 1024 + (size_t)4 * TILE_BYTES + 2048 +
+                      ((size_t)2 * G * TCD + (size_t)DNW * G * TCD + (size_t)G * kMaxDecodeSplits +
+                       (size_t)(MAXT * TK + 1) * G + 24) * 4;
+  cudaError_t err = cudaSuccess;
+  using TC = __nv_bfloat16;
+#define LAUNCH(GG)                                                                               \
+  do {                                                                                           \
+    auto kern = decode_step_tc_kernel<GG>;                                                       \
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
+    if (err != cudaSuccess) return err;                                                          \
+    kern<<<grid, DNT, smem, st>>>(tk, (const TC*)q_new, (const TC*)k_new, (const TC*)v_new, (TC*)k_cache,  \
+                                  (TC*)v_cache, (TC*)out, w.qhat[qhat_sel], w.qhat[qhat_sel ^ 1], w.R,     \
+                                  w.dec_partial, w.dec_ticket, w.counters, n, s.T_max, s.H, chunk, nsplit, \
+                                  theta, window, scale_log2e);                                             \
+  } while (0)
+  switch (G) {
+    case 1: LAUNCH(1); break;
+    case 2: LAUNCH(2); break;
+    case 4: LAUNCH(4); break;
+    case 8: LAUNCH(8); break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef LAUNCH
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace delta
