@@ -17,7 +17,9 @@
 //      the products; all score tiles of the slice stay in tensor memory (16 columns per tile);
 //   3. one softmax over the slice: every thread reads its keys' scores (lane = key), hybrid
 //      select, scale, R written; maximum and sum reduced once per slice, not per tile;
-//   4. P.V with the value tiles streamed through a two-stage ring of bulk copies;
+//   4. P.V with the value tiles streamed through a ring of bulk copies (three stages of its own
+//      plus the two key stages once the products are done), the warps releasing stages through
+//      mbarriers (no block-wide barrier per tile);
 //   5. the slice result is stored and the last CTA of the (batch, KV head) merges the slices.
 // The key and value that arrive with this step are scored on the FP32 pipes by the CTA that
 // owns their slice (their cache row is written by this very kernel).
@@ -38,8 +40,28 @@ constexpr int TK = 128;                // keys per tile
 constexpr int MAXT = 9;                // tiles per slice at most (1152 keys)
 constexpr int SCOL = 16;               // tensor-memory columns per tile (N of the product)
 constexpr uint32_t DEC_TMEM_COLS = 256;
+// CTAs the key slices aim for.  Measured at batch 16, 2049 keys: 256 CTAs 24.5 us per step, 384 CTAs
+// 30.3, 512 CTAs 29.2, 768 CTAs 31.6 (a CTA's fixed cost outweighs the better balance).
+constexpr int kTcTargetCtas = 296;
 
-enum { BAR_K0 = 0, BAR_K1, BAR_KFREE0, BAR_KFREE1, BAR_S, BAR_V0, BAR_V1, DEC_NUM_BARS };
+constexpr int NVS_OWN = 3;             // value-ring stages of its own
+constexpr int NVS = NVS_OWN + 2;       // plus the two key stages once the score products are done
+enum { BAR_K0 = 0, BAR_K1, BAR_KFREE0, BAR_KFREE1, BAR_S, BAR_V0, BAR_VFREE0 = BAR_V0 + NVS, DEC_NUM_BARS = BAR_VFREE0 + NVS };
+
+
+// The G probabilities of one key (contiguous, 16-byte aligned for G >= 4).
+template <int G> __device__ __forceinline__ void load_probs(const float* p, float (&pr)[G]) {
+  if constexpr (G % 4 == 0) {
+#pragma unroll
+    for (int i = 0; i < G; i += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(p + i);
+      pr[i] = v.x; pr[i + 1] = v.y; pr[i + 2] = v.z; pr[i + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < G; ++i) pr[i] = p[i];
+  }
+}
 
 }  // namespace
 
@@ -60,13 +82,13 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled operand tiles want 1 KiB alignment
   unsigned char* sm = dsm_raw0 + (base - raw);
   constexpr uint32_t OFF_K = 0;                          // [2][128][64] bf16, 128-byte swizzle
-  constexpr uint32_t OFF_V = OFF_K + 2 * TILE_BYTES;     // [2][128][64] bf16, plain rows
-  constexpr uint32_t OFF_QC = OFF_V + 2 * TILE_BYTES;    // Qcat [16][64] bf16, 128-byte swizzle
+  constexpr uint32_t OFF_V = OFF_K + 2 * TILE_BYTES;     // [NVS_OWN][128][64] bf16, plain rows
+  constexpr uint32_t OFF_QC = OFF_V + NVS_OWN * TILE_BYTES;  // Qcat [16][64] bf16, 128-byte swizzle
   constexpr uint32_t OFF_F = OFF_QC + 2048;              // floats from here on
   float* q_s = reinterpret_cast<float*>(sm + OFF_F);     // [G][D]
   float* qh_s = q_s + G * D;                             // [G][D]
-  float* red = qh_s + G * D;                             // [DNW][G][D]
-  float* wgt = red + DNW * G * D;                        // [G * kMaxDecodeSplits] (merge) / [DNW][2G] (reductions)
+  float* red = reinterpret_cast<float*>(sm + OFF_K);     // [DNW][G][D]: the key ring is free by then
+  float* wgt = qh_s + G * D;                             // [G * kMaxDecodeSplits] (merge) / [DNW][2G] (reductions)
   float* p_s = wgt + G * kMaxDecodeSplits;               // [MAXT * TK + 1][G] probabilities
   float* st_s = p_s + (MAXT * TK + 1) * G;               // [24]
   __shared__ __align__(8) unsigned long long bars[DEC_NUM_BARS];
@@ -92,10 +114,32 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  const TC* vc = v_cache + (size_t)bkv * T_max * D;
+  auto v_rows = [&](int t) { return min(TK, cached - t * TK); };
+  // value stage s: three of its own, then the two key stages (free once all score products are done)
+  auto v_stage_off = [&](int s2) -> uint32_t {
+    return s2 < NVS_OWN ? OFF_V + (uint32_t)s2 * TILE_BYTES : OFF_K + (uint32_t)(s2 - NVS_OWN) * TILE_BYTES;
+  };
+  auto issue_v = [&](int t) {
+    const uint32_t bytes = (uint32_t)v_rows(t) * D * 2u;
+    const uint32_t bar = DBAR(BAR_V0 + (t % NVS));
+    tc::mbar_expect_tx(bar, bytes);
+    bulk_load(base + v_stage_off(t % NVS), vc + (size_t)(j0 + t * TK) * D, bytes, bar);
+  };
+
+  auto issue_k = [&](int t) {
+    tc::mbar_expect_tx(DBAR(BAR_K0 + (t & 1)), TILE_BYTES);
+    tc::tma_load_3d(base + OFF_K + (t & 1) * TILE_BYTES, &tm_k, DBAR(BAR_K0 + (t & 1)), 0, j0 + t * TK, bkv);
+  };
   if (tid == 0) {
-    for (int i = 0; i < DEC_NUM_BARS; ++i) tc::mbar_init(DBAR(i), 1u);
+    for (int i = 0; i < DEC_NUM_BARS; ++i) tc::mbar_init(DBAR(i), i >= BAR_VFREE0 ? (uint32_t)DNW : 1u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc::fence_proxy_async();
     s_fail = 0;
+    // the first key and value tiles are on their way while the threshold step below runs
+    if (n_tiles > 0) issue_k(0);
+    if (n_tiles > 1) issue_k(1);
+    for (int t = 0; t < NVS_OWN && t < n_tiles; ++t) issue_v(t);
   }
 
   // ---- 1. delta of the new query rows against the carried reference (Eq. 2-3); Qcat
@@ -144,26 +188,9 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   tc::tc_fence_after();
   const uint32_t tmem = s_tmem;
 
-  const TC* vc = v_cache + (size_t)bkv * T_max * D;
-  auto v_rows = [&](int t) { return min(TK, cached - t * TK); };
-  auto issue_v = [&](int t) {
-    const uint32_t bytes = (uint32_t)v_rows(t) * D * 2u;
-    const uint32_t bar = DBAR(BAR_V0 + (t & 1));
-    tc::mbar_expect_tx(bar, bytes);
-    bulk_load(base + OFF_V + (t & 1) * TILE_BYTES, vc + (size_t)(j0 + t * TK) * D, bytes, bar);
-  };
-
   // ---- 2. key tiles through the tensor cores (one thread)
   if (tid == 0 && n_tiles > 0) {
     const uint32_t IDESC = tc::make_idesc(SCOL, 0);
-    auto issue_k = [&](int t) {
-      tc::mbar_expect_tx(DBAR(BAR_K0 + (t & 1)), TILE_BYTES);
-      tc::tma_load_3d(base + OFF_K + (t & 1) * TILE_BYTES, &tm_k, DBAR(BAR_K0 + (t & 1)), 0, j0 + t * TK, bkv);
-    };
-    issue_k(0);
-    if (n_tiles > 1) issue_k(1);
-    issue_v(0);
-    if (n_tiles > 1) issue_v(1);
     for (int t = 0; t < n_tiles; ++t) {
       if (!mbar_wait(DBAR(BAR_K0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
       tc::tc_fence_after();
@@ -180,6 +207,11 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
       }
     }
     tc::tc_commit(DBAR(BAR_S));
+    // the key stages turn into value stages as soon as the last product has read them
+    if (n_tiles > NVS_OWN) {
+      if (!mbar_wait(DBAR(BAR_S), 0)) s_fail = 1;
+      for (int t = NVS_OWN; t < NVS && t < n_tiles; ++t) issue_v(t);
+    }
   }
 
   // the key and value that arrive with this step: into the cache, scored on the FP32 pipes
@@ -303,25 +335,38 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[hh][e] = 0.0f;
   for (int t = 0; t < n_tiles; ++t) {
-    if (!mbar_wait(DBAR(BAR_V0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
-    const TC* vt = reinterpret_cast<const TC*>(sm + OFF_V + (t & 1) * TILE_BYTES);
+    const int stg = t % NVS;
+    const uint32_t par = (uint32_t)(t / NVS) & 1u;
+    if (!mbar_wait(DBAR(BAR_V0 + stg), par)) s_fail = 1;
+    const TC* vt = reinterpret_cast<const TC*>(sm + v_stage_off(stg));
     const int rows = v_rows(t);
     for (int jb = warp * KPW; jb < rows; jb += DNW * KPW) {
       const int jj = jb + sub;
       if (jj < rows) {
         float vv[8];
         load8(vt + (size_t)jj * D + c0, vv);
-        const float* pp = p_s + (size_t)(t * TK + jj) * G;
+        float pr[G];
+        load_probs<G>(p_s + (size_t)(t * TK + jj) * G, pr);
 #pragma unroll
         for (int hh = 0; hh < G; ++hh) {
-          const float p = pp[hh];
+          const float2 p2 = make_float2(pr[hh], pr[hh]);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[hh][e] = fmaf(p, vv[e], acc[hh][e]);
+          for (int e = 0; e < 8; e += 2) {
+            const float2 a = tc::ffma2(p2, make_float2(vv[e], vv[e + 1]), make_float2(acc[hh][e], acc[hh][e + 1]));
+            acc[hh][e] = a.x;
+            acc[hh][e + 1] = a.y;
+          }
         }
       }
     }
-    __syncthreads();                      // the stage is free
-    if (tid == 0 && t + 2 < n_tiles) issue_v(t + 2);
+    // the warps run through the ring at their own pace: a stage is refilled (by one thread of
+    // the last warp) once all of them have released it
+    __syncwarp();
+    if (lane == 0) tc::mbar_arrive(DBAR(BAR_VFREE0 + stg));
+    if (warp == DNW - 1 && lane == 0 && t + NVS < n_tiles) {
+      if (!mbar_wait(DBAR(BAR_VFREE0 + stg), par)) s_fail = 1;
+      issue_v(t + NVS);
+    }
   }
   if (has_new && warp == 0 && sub == 0) {
     float vv[8];
@@ -348,7 +393,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
 static void decode_tc_slices(const Shape& s, int n, int* nsplit_out, int* chunk_out) {
   const int L = n + 1;
   const int bkv = s.B * s.H_kv;
-  int nsplit = kDecodeTargetCtas / bkv;
+  int nsplit = kTcTargetCtas / bkv;
   if (nsplit > kMaxDecodeSplits) nsplit = kMaxDecodeSplits;
   const int max_by_len = (L + TK / 4 - 1) / (TK / 4);
   if (nsplit > max_by_len) nsplit = max_by_len;
@@ -387,15 +432,18 @@ cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const int G = s.g();
   const dim3 grid(nsplit, bkv);
-  const size_t smem = 1024 + (size_t)4 * TILE_BYTES + 2048 +
-                      ((size_t)2 * G * TCD + (size_t)DNW * G * TCD + (size_t)G * kMaxDecodeSplits +
-                       (size_t)(MAXT * TK + 1) * G + 24) * 4;
+  const size_t smem = 1024 + (size_t)(2 + NVS_OWN) * TILE_BYTES + 2048 +
+                      ((size_t)2 * G * TCD + (size_t)G * kMaxDecodeSplits + (size_t)(MAXT * TK + 1) * G + 24) * 4;
   cudaError_t err = cudaSuccess;
   using TC = __nv_bfloat16;
 #define LAUNCH(GG)                                                                               \
   do {                                                                                           \
     auto kern = decode_step_tc_kernel<GG>;                                                       \
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
+    if (err != cudaSuccess) return err;                                                          \
+    /* two CTAs per SM need the largest shared-memory carve-out */                               \
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,             \
+                               (int)cudaSharedmemCarveoutMaxShared);                             \
     if (err != cudaSuccess) return err;                                                          \
     kern<<<grid, DNT, smem, st>>>(tk, (const TC*)q_new, (const TC*)k_new, (const TC*)v_new, (TC*)k_cache,  \
                                   (TC*)v_cache, (TC*)out, w.qhat[qhat_sel], w.qhat[qhat_sel ^ 1], w.R,     \
