@@ -30,6 +30,7 @@ EXPORTED = [
     "delta_attn_prefill", "delta_prefill_staging_bytes", "delta_attn_prefill_host",
     "delta_attn_decode_step", "delta_sparsity_stats", "delta_window_from_gamma", "delta_state_view",
     "delta_state_position", "delta_state_prefill_kernel", "delta_state_decode_kernel",
+    "delta_state_set_decode_kernel",
     "delta_state_set_prefill_kernel",
     "delta_launch_count", "delta_status_string", "delta_last_cuda_error",
     "delta_state_enable_profiling", "delta_state_prefill_kernel_ms",
@@ -90,6 +91,7 @@ def _load() -> C.CDLL:
         "delta_state_position": (i32, [vp]),
         "delta_state_prefill_kernel": (i32, [vp]),
         "delta_state_decode_kernel": (i32, [vp]),
+        "delta_state_set_decode_kernel": (C.c_int, [vp, i32]),
         "delta_state_set_prefill_kernel": (C.c_int, [vp, i32]),
         "delta_state_enable_profiling": (C.c_int, [vp, i32]),
         "delta_state_prefill_kernel_ms": (C.c_int, [vp, C.POINTER(C.c_float)]),
@@ -231,6 +233,10 @@ def delta_state_prefill_kernel(st: DeltaState) -> int:
 
 def delta_state_decode_kernel(st: DeltaState) -> int:
     return lib.delta_state_decode_kernel(st.handle)
+
+
+def delta_state_set_decode_kernel(st: DeltaState, which: int) -> None:
+    _check(lib.delta_state_set_decode_kernel(st.handle, which), "delta_state_set_decode_kernel")
 
 
 def delta_state_set_prefill_kernel(st: DeltaState, which: int):

@@ -32,6 +32,7 @@ struct delta_state {
   // Eq. 6 bookkeeping that needs no device work: sum of window lengths and sequence lengths
   double win_sum[2], len_sum[2];
   DecodeTmapCache dec_tmap;   // tensor map of the key cache the decode steps read
+  int forced_decode_kernel = -1;   // -1: chosen per step
   // optional per-kernel timing of prefill (host-side event objects)
   bool profiling = false, profiled = false;
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -196,10 +197,23 @@ int32_t delta_state_prefill_kernel(const delta_state_t* st) {
   return tc_eligible(st, 2) ? 2 : 0;   // the telescoped tensor-core kernel is the fastest where it applies
 }
 
+// Can the tensor-core decode kernel serve this state at all (whatever the slice length)?
+static bool decode_tc_possible(const delta_state* st) {
+  return st->cfg.source == DELTA_SRC_QUERY && decode_tc_applies(st->shape, st->cfg.dtype, -1);
+}
+
 int32_t delta_state_decode_kernel(const delta_state_t* st) {
   if (!st) return -1;
-  if (st->cfg.source != DELTA_SRC_QUERY) return 0;
+  if (!decode_tc_possible(st)) return 0;
+  if (st->forced_decode_kernel >= 0) return st->forced_decode_kernel;
   return decode_tc_applies(st->shape, st->cfg.dtype, st->n) ? 1 : 0;
+}
+
+delta_status_t delta_state_set_decode_kernel(delta_state_t* st, int32_t which) {
+  if (!st || which < -1 || which > 1) return DELTA_ERR_INVALID_ARG;
+  if (which == 1 && !decode_tc_possible(st)) return DELTA_ERR_UNSUPPORTED;
+  st->forced_decode_kernel = which;
+  return DELTA_OK;
 }
 
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
@@ -341,7 +355,7 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
       st->cfg.source == DELTA_SRC_KEY
           ? launch_decode_step_key(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n,
                                    theta, window, st->qhat_sel, (cudaStream_t)stream)
-      : decode_tc_applies(st->shape, st->cfg.dtype, st->n)
+      : delta_state_decode_kernel(st) == 1
           ? launch_decode_step_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
                                   window, st->qhat_sel, &st->dec_tmap, (cudaStream_t)stream)
           : launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n,

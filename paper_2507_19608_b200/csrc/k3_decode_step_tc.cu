@@ -408,6 +408,7 @@ static void decode_tc_slices(const Shape& s, int n, int* nsplit_out, int* chunk_
 
 bool decode_tc_applies(const Shape& s, int dtype, int n) {
   if (s.d != TCD || dtype != DELTA_BF16 || tc::encode_fn() == nullptr) return false;
+  if (n < 0) return true;      // shape and type only
   int nsplit, chunk;
   decode_tc_slices(s, n, &nsplit, &chunk);
   return chunk >= 2 * TK && chunk <= MAXT * TK && nsplit <= kMaxDecodeSplits;

@@ -247,12 +247,22 @@ def test_prefill_host_entry_matches_device_entry(B):
     (1, 8, 1, 90, 64, "bf16", 0.1, 0, 3),         # no exact window, group of 8 heads
     (1, 2, 2, 40, 128, "f32", 0.0, 1000, 3),      # window covers the whole cache
     (1, 1, 1, 1, 64, "bf16", 0.1, 2, 4),          # decode right after a one-token prefill
+    (1, 4, 1, 700, 64, "bf16", 0.29, 4, 4),       # several key slices, ragged tiles
+    (3, 4, 4, 1500, 64, "bf16", 0.2, 200, 3),     # one head per KV head, window wider than a tile, 12 tiles
+    (2, 4, 2, 255, 64, "bf16", 0.15, 1000, 3),    # window covers the cache; the new key opens a tile at step 2
+    (40, 4, 4, 1100, 64, "bf16", 0.2, 64, 2),     # 160 KV heads: one slice of 9 tiles per head
+    (19, 16, 8, 600, 64, "bf16", 0.25, 16, 2),    # 152 KV heads, groups of 2: one slice of 5 tiles
 ])
-def test_decode_steps_match_oracle(B, Bn, H, Hk, T, d, dtype, theta, W, steps):
+@pytest.mark.parametrize("decode_kernel", [0, 1], ids=["fp32_pipes", "tc_scores"])
+def test_decode_steps_match_oracle(B, Bn, H, Hk, T, d, dtype, theta, W, steps, decode_kernel):
     from tests.gpu_helpers import run_prefill, to_dev, to_host_f64
+    if decode_kernel == 1 and not (dtype == "bf16" and d == 64):
+        pytest.skip("tensor-core decode scores: bf16, d = 64")
     w = WL.Workload("t", Bn, H, Hk, T, d, dtype, 0.95, 0.5, W, (), 77 + T, n_decode=steps)
     t = WL.make_qkv(w)
     st, out, kc, vc = run_prefill(B, t["q"], t["k"], t["v"], theta, W, dtype, shape="sliding", T_max=T + steps)
+    B.delta_state_set_decode_kernel(st, decode_kernel)
+    assert B.delta_state_decode_kernel(st) == decode_kernel
     ref, heads = O.prefill_mha(t["q"], t["k"], t["v"], theta, W, "sliding")
     states = {key: r["state"] for key, r in heads.items()}
     nnz = done = dense = 0
