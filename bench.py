@@ -521,7 +521,7 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
         res[f"batch{w.B}"] = {
             "us_per_step_eager": statistics.median(eager), "us_per_step_graph": graph_us,
             "graph_matches_eager": graph_ok, "steps": w.n_decode,
-            "decode_kernel": "FP32 pipes" if key or B.delta_state_decode_kernel(st) != 1 else "tensor-core scores", "cache_tokens": w.T, "theta": theta,
+            "decode_kernel": "tensor-core scores" if B.delta_state_decode_kernel(st) == 1 else "FP32 pipes", "cache_tokens": w.T, "theta": theta,
             "window": w.window, "algorithmic_bytes_per_step": bytes_step,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
                          "frac": gbs / float(peaks["hbm_gbs"]),

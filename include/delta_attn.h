@@ -256,13 +256,13 @@ DELTA_API int32_t delta_state_position(const delta_state_t* st);
 DELTA_API int32_t delta_state_prefill_kernel(const delta_state_t* st);
 
 /* Which kernel the next delta_attn_decode_step of this state would use: 1 = score products
- * on the tensor cores (bf16, d = 64, query deltas, key slices of at least two 128-key tiles:
+ * on the tensor cores (bf16, d = 64, top-down query deltas or key deltas, key slices of at least two 128-key tiles:
  * the telescoped form of Eq. 4, see delta_attn_decode_step), 0 = the FP32-pipe kernel,
  * -1 for a null state.  Both compute the same step and keep the same state. */
 DELTA_API int32_t delta_state_decode_kernel(const delta_state_t* st);
 
 /* Force the decode kernel of a state: 1 = tensor-core scores whatever the slice length
- * (DELTA_ERR_UNSUPPORTED unless bf16, d = 64, query deltas), 0 = FP32 pipes, -1 = chosen per
+ * (DELTA_ERR_UNSUPPORTED unless bf16, d = 64, top-down query deltas or key deltas), 0 = FP32 pipes, -1 = chosen per
  * step (the default).  Host-side only. */
 DELTA_API delta_status_t delta_state_set_decode_kernel(delta_state_t* st, int32_t which);
 DELTA_API delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which);

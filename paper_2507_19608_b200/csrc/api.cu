@@ -32,6 +32,7 @@ struct delta_state {
   // Eq. 6 bookkeeping that needs no device work: sum of window lengths and sequence lengths
   double win_sum[2], len_sum[2];
   DecodeTmapCache dec_tmap;   // tensor map of the key cache the decode steps read
+  DecodeTmapCache dec_tmap_h; // and of the reference-key cache (key deltas)
   int forced_decode_kernel = -1;   // -1: chosen per step
   // optional per-kernel timing of prefill (host-side event objects)
   bool profiling = false, profiled = false;
@@ -199,7 +200,7 @@ int32_t delta_state_prefill_kernel(const delta_state_t* st) {
 
 // Can the tensor-core decode kernel serve this state at all (whatever the slice length)?
 static bool decode_tc_possible(const delta_state* st) {
-  return st->cfg.source == DELTA_SRC_QUERY && decode_tc_applies(st->shape, st->cfg.dtype, -1);
+  return st->cfg.source != DELTA_SRC_QUERY_BOTTOM_UP && decode_tc_applies(st->shape, st->cfg.dtype, -1);
 }
 
 int32_t delta_state_decode_kernel(const delta_state_t* st) {
@@ -351,15 +352,19 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
   if (st->cfg.source == DELTA_SRC_QUERY_BOTTOM_UP) return DELTA_ERR_UNSUPPORTED;   // strategy (2) has no decode
   if (st->n < 1) return DELTA_ERR_STATE;
   if (st->n >= st->cfg.T_max) return DELTA_ERR_CAPACITY;
-  cudaError_t e =
-      st->cfg.source == DELTA_SRC_KEY
-          ? launch_decode_step_key(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n,
-                                   theta, window, st->qhat_sel, (cudaStream_t)stream)
-      : delta_state_decode_kernel(st) == 1
-          ? launch_decode_step_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
-                                  window, st->qhat_sel, &st->dec_tmap, (cudaStream_t)stream)
-          : launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n,
-                               theta, window, st->cfg.dtype, st->qhat_sel, (cudaStream_t)stream);
+  const bool tcs = delta_state_decode_kernel(st) == 1;
+  cudaStream_t cs = (cudaStream_t)stream;
+  cudaError_t e;
+  if (st->cfg.source == DELTA_SRC_KEY)
+    e = tcs ? launch_decode_step_key_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
+                                        window, st->qhat_sel, &st->dec_tmap, &st->dec_tmap_h, cs)
+            : launch_decode_step_key(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
+                                     window, st->qhat_sel, cs);
+  else
+    e = tcs ? launch_decode_step_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
+                                    window, st->qhat_sel, &st->dec_tmap, cs)
+            : launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
+                                 window, st->cfg.dtype, st->qhat_sel, cs);
   if (e != cudaSuccess) return cuda_fail(e);
   const int L = st->n + 1;
   st->win_sum[1] += (double)(window < L ? window : L);

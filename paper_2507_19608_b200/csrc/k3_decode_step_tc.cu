@@ -25,6 +25,16 @@
 // owns their slice (their cache row is written by this very kernel).
 // Every wait is bounded; after a time-out the kernel still runs to its end and the status word
 // records DELTA_ERR_TIMEOUT.
+//
+// KEY = true is the same step for key deltas (strategy 3): the score of key j is q_new . k_j for
+// the W_d most recent keys and q_new . k_hat(j) for the older ones (the column recursion of
+// Eq. 4, telescoped; k_hat(j) is the reference key after row j, kept in the library's
+// reference-key cache).  Qcat holds the G query rows only, and the tile a product reads is a
+// tile of the reference-key cache (keys older than the window), of the key cache (keys inside
+// it) or -- the one tile the window's edge falls into -- a reference-key tile whose window rows
+// warp 0 replaces in shared memory by the original keys.  The threshold step runs over k_new
+// (one vector per KV head), nothing like R is carried, and the CTA that owns the new key's
+// slice appends k_new, v_new and k_hat(n) to their caches.
 #include <cuda.h>
 
 #include "decode_common.cuh"
@@ -65,11 +75,13 @@ template <int G> __device__ __forceinline__ void load_probs(const float* p, floa
 
 }  // namespace
 
-template <int G>
+template <int G, bool KEY>
 __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
-    const __grid_constant__ CUtensorMap tm_k, const __nv_bfloat16* __restrict__ q_new,
+    const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_h,
+    const __nv_bfloat16* __restrict__ q_new,
     const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
     __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
+    __nv_bfloat16* __restrict__ khat_cache, uint16_t* __restrict__ row_nnz,
     __nv_bfloat16* __restrict__ out, const float* __restrict__ qhat_in, float* __restrict__ qhat_out,
     float* __restrict__ R, float* __restrict__ partial, uint32_t* __restrict__ ticket,
     unsigned long long* __restrict__ counters, int n, int T_max, int H, int chunk, int nsplit,
@@ -105,6 +117,14 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   const int cached = max(0, min(len, n - j0));           // of which already in the cache
   const int n_tiles = (cached + TK - 1) / TK;            // tiles that go through the tensor cores
   const bool has_new = (n >= j0) && (n < j0 + len);
+  const int wl = n - W + 1;                              // first key inside the decode window
+  // key deltas: where tile t's rows come from -- 0 reference-key cache, 1 key cache, 2 mixed
+  auto tile_kind = [&](int t) -> int {
+    const int a0 = j0 + t * TK, a1 = a0 + min(TK, cached - t * TK) - 1;     // cached keys of the tile
+    if (a1 < wl) return 0;
+    if (a0 >= wl) return 1;
+    return 2;
+  };
   const uint32_t bar0 = smem_u32(&bars[0]);
 #define DBAR(i) (bar0 + 8u * (uint32_t)(i))
 
@@ -129,7 +149,8 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
 
   auto issue_k = [&](int t) {
     tc::mbar_expect_tx(DBAR(BAR_K0 + (t & 1)), TILE_BYTES);
-    tc::tma_load_3d(base + OFF_K + (t & 1) * TILE_BYTES, &tm_k, DBAR(BAR_K0 + (t & 1)), 0, j0 + t * TK, bkv);
+    const CUtensorMap* src = (KEY && tile_kind(t) != 1) ? &tm_h : &tm_k;
+    tc::tma_load_3d(base + OFF_K + (t & 1) * TILE_BYTES, src, DBAR(BAR_K0 + (t & 1)), 0, j0 + t * TK, bkv);
   };
   if (tid == 0) {
     for (int i = 0; i < DEC_NUM_BARS; ++i) tc::mbar_init(DBAR(i), i >= BAR_VFREE0 ? (uint32_t)DNW : 1u);
@@ -142,44 +163,85 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     for (int t = 0; t < NVS_OWN && t < n_tiles; ++t) issue_v(t);
   }
 
-  // ---- 1. delta of the new query rows against the carried reference (Eq. 2-3); Qcat
+  // ---- 1. threshold step (Eq. 2-3) and Qcat
+  // operand row r, channel c of Qcat (128-byte swizzle)
+  auto qc_off = [&](int r, int c) -> uint32_t {
+    return (uint32_t)r * 128u + ((((uint32_t)c >> 3) ^ ((uint32_t)r & 7u)) << 4) + ((uint32_t)c & 7u) * 2u;
+  };
+  constexpr int QROWS = KEY ? G : 2 * G;     // operand rows in use
   int fired_total = 0;
-  for (int e0 = 0; e0 < G * D; e0 += DNT) {
-    const int e = e0 + tid;
+  if constexpr (!KEY) {
+    // the new query rows against the carried reference queries
+    for (int e0 = 0; e0 < G * D; e0 += DNT) {
+      const int e = e0 + tid;
+      bool fire = false;
+      if (e < G * D) {
+        const int hh = e / D, c = e - hh * D;
+        const size_t o = ((size_t)b * H + kvh * G + hh) * D + c;
+        const TC xb = q_new[o];
+        const float x = to_f32(xb);
+        const float old = qhat_in[o];
+        fire = fabsf(__fsub_rn(x, old)) > theta;
+        const float nq = fire ? x : old;
+        q_s[e] = x;
+        qh_s[e] = nq;
+        if (split == 0) qhat_out[o] = nq;
+        // operand rows: hh = new reference (exactly bf16), G + hh = new query
+        *reinterpret_cast<uint16_t*>(sm + OFF_QC + qc_off(hh, c)) = (uint16_t)(__float_as_uint(nq) >> 16);
+        *reinterpret_cast<TC*>(sm + OFF_QC + qc_off(G + hh, c)) = xb;
+      }
+      fired_total += __syncthreads_count(fire);
+    }
+    if (split == 0 && tid == 0) {
+      const int n_in = min(L, max(W, 0));
+      const int n_out = L - n_in;
+      atomicAdd(&counters[CNT_DECODE_NNZ], (unsigned long long)fired_total);
+      atomicAdd(&counters[CNT_DECODE_ELEMS], (unsigned long long)G * D);
+      atomicAdd(&counters[CNT_DECODE_MACS_DONE],
+                (unsigned long long)n_in * D * G + (unsigned long long)n_out * fired_total);
+      atomicAdd(&counters[CNT_DECODE_MACS_DENSE], (unsigned long long)L * D * G);
+    }
+  } else {
+    // the new key against the carried reference key (qh_s[0..D) = k_hat(n)); the query rows are
+    // the operand
     bool fire = false;
-    if (e < G * D) {
-      const int hh = e / D, c = e - hh * D;
-      const size_t o = ((size_t)b * H + kvh * G + hh) * D + c;
-      const TC xb = q_new[o];
-      const float x = to_f32(xb);
+    if (tid < D) {
+      const size_t o = (size_t)bkv * D + tid;
+      const float x = to_f32(k_new[o]);
       const float old = qhat_in[o];
       fire = fabsf(__fsub_rn(x, old)) > theta;
-      const float nq = fire ? x : old;
-      q_s[e] = x;
-      qh_s[e] = nq;
-      if (split == 0) qhat_out[o] = nq;
-      // operand rows: hh = new reference (exactly bf16), G + hh = new query
-      auto qc_off = [&](int r) -> uint32_t {
-        return (uint32_t)r * 128u + ((((uint32_t)c >> 3) ^ ((uint32_t)r & 7u)) << 4) + ((uint32_t)c & 7u) * 2u;
-      };
-      *reinterpret_cast<uint16_t*>(sm + OFF_QC + qc_off(hh)) = (uint16_t)(__float_as_uint(nq) >> 16);
-      *reinterpret_cast<TC*>(sm + OFF_QC + qc_off(G + hh)) = xb;
+      const float nk = fire ? x : old;
+      qh_s[tid] = nk;                        // exactly bf16: a copy of an input element (or 0)
+      if (split == 0) qhat_out[o] = nk;
     }
-    fired_total += __syncthreads_count(fire);
+    for (int e = tid; e < G * D; e += DNT) {
+      const int hh = e / D, c = e - hh * D;
+      const TC xb = q_new[((size_t)b * H + kvh * G + hh) * D + c];
+      q_s[e] = to_f32(xb);
+      *reinterpret_cast<TC*>(sm + OFF_QC + qc_off(hh, c)) = xb;
+    }
+    fired_total = __syncthreads_count(fire);
+    // multiply-adds of this step for the slice's keys: d inside the window, nnz(Delta k_j) outside
+    {
+      unsigned long long done = 0;
+      for (int jj = tid; jj < len; jj += DNT) {
+        const int j = j0 + jj;
+        const int nz = (j == n) ? fired_total : (int)row_nnz[(size_t)bkv * T_max + j];
+        done += (n - j < W) ? (unsigned long long)D : (unsigned long long)nz;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) done += __shfl_down_sync(0xffffffffu, done, o);
+      if (lane == 0 && done) atomicAdd(&counters[CNT_DECODE_MACS_DONE], done * G);
+    }
+    if (split == 0 && tid == 0) {
+      atomicAdd(&counters[CNT_DECODE_NNZ], (unsigned long long)fired_total);
+      atomicAdd(&counters[CNT_DECODE_ELEMS], (unsigned long long)D);
+      atomicAdd(&counters[CNT_DECODE_MACS_DENSE], (unsigned long long)L * D * G);
+    }
   }
-  for (int e = tid; e < (16 - 2 * G) * D; e += DNT) {       // unused operand rows: zeros
-    const int r = 2 * G + e / D, c = e % D;
-    *reinterpret_cast<uint16_t*>(sm + OFF_QC + (uint32_t)r * 128u + ((((uint32_t)c >> 3) ^ ((uint32_t)r & 7u)) << 4) +
-                                 ((uint32_t)c & 7u) * 2u) = 0;
-  }
-  if (split == 0 && tid == 0) {
-    const int n_in = min(L, max(W, 0));
-    const int n_out = L - n_in;
-    atomicAdd(&counters[CNT_DECODE_NNZ], (unsigned long long)fired_total);
-    atomicAdd(&counters[CNT_DECODE_ELEMS], (unsigned long long)G * D);
-    atomicAdd(&counters[CNT_DECODE_MACS_DONE],
-              (unsigned long long)n_in * D * G + (unsigned long long)n_out * fired_total);
-    atomicAdd(&counters[CNT_DECODE_MACS_DENSE], (unsigned long long)L * D * G);
+  for (int e = tid; e < (16 - QROWS) * D; e += DNT) {       // unused operand rows: zeros
+    const int r = QROWS + e / D, c = e % D;
+    *reinterpret_cast<uint16_t*>(sm + OFF_QC + qc_off(r, c)) = 0;
   }
   if (tid < 8) { st_s[tid] = -INFINITY; st_s[8 + tid] = 0.0f; }
   tc::fence_proxy_async();           // Qcat was written through the generic proxy
@@ -188,30 +250,49 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   tc::tc_fence_after();
   const uint32_t tmem = s_tmem;
 
-  // ---- 2. key tiles through the tensor cores (one thread)
-  if (tid == 0 && n_tiles > 0) {
+  // ---- 2. key tiles through the tensor cores (warp 0: lane 0 issues the copies and products)
+  if (warp == 0 && n_tiles > 0) {
     const uint32_t IDESC = tc::make_idesc(SCOL, 0);
+    const TC* kc = k_cache + (size_t)bkv * T_max * D;
     for (int t = 0; t < n_tiles; ++t) {
       if (!mbar_wait(DBAR(BAR_K0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
-      tc::tc_fence_after();
       const uint32_t kb = base + OFF_K + (t & 1) * TILE_BYTES;
+      if (KEY && tile_kind(t) == 2) {
+        // the window's edge falls into this tile: its window rows become the original keys
+        const int r0 = wl - (j0 + t * TK), r1 = min(TK, cached - t * TK);
+        for (int e = lane; e < (r1 - r0) * 8; e += 32) {
+          const int r = r0 + (e >> 3), ch = e & 7;
+          *reinterpret_cast<uint4*>(sm + OFF_K + (t & 1) * TILE_BYTES + (uint32_t)r * 128u +
+                                    (((uint32_t)ch ^ ((uint32_t)r & 7u)) << 4)) =
+              *reinterpret_cast<const uint4*>(kc + (size_t)(j0 + t * TK + r) * D + ch * 8);
+        }
+        tc::fence_proxy_async();
+      }
+      __syncwarp();
+      if (lane == 0) {
+        tc::tc_fence_after();
 #pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks)
-        tc::tc_mma(tmem + SCOL * t, tc::make_desc(kb + ks * 32, 16, 1024),
-                   tc::make_desc(base + OFF_QC + ks * 32, 16, 1024), IDESC, ks > 0 ? 1u : 0u);
-      if (t + 2 < n_tiles) {
-        // the stage is free once these products are done: then refill it
-        tc::tc_commit(DBAR(BAR_KFREE0 + (t & 1)));
-        if (!mbar_wait(DBAR(BAR_KFREE0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
-        issue_k(t + 2);
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::tc_mma(tmem + SCOL * t, tc::make_desc(kb + ks * 32, 16, 1024),
+                     tc::make_desc(base + OFF_QC + ks * 32, 16, 1024), IDESC, ks > 0 ? 1u : 0u);
+        if (t + 2 < n_tiles) {
+          // the stage is free once these products are done: then refill it
+          tc::tc_commit(DBAR(BAR_KFREE0 + (t & 1)));
+          if (!mbar_wait(DBAR(BAR_KFREE0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
+          issue_k(t + 2);
+        }
+      }
+      __syncwarp();
+    }
+    if (lane == 0) {
+      tc::tc_commit(DBAR(BAR_S));
+      // the key stages turn into value stages as soon as the last product has read them
+      if (n_tiles > NVS_OWN) {
+        if (!mbar_wait(DBAR(BAR_S), 0)) s_fail = 1;
+        for (int t = NVS_OWN; t < NVS && t < n_tiles; ++t) issue_v(t);
       }
     }
-    tc::tc_commit(DBAR(BAR_S));
-    // the key stages turn into value stages as soon as the last product has read them
-    if (n_tiles > NVS_OWN) {
-      if (!mbar_wait(DBAR(BAR_S), 0)) s_fail = 1;
-      for (int t = NVS_OWN; t < NVS && t < n_tiles; ++t) issue_v(t);
-    }
+    __syncwarp();
   }
 
   // the key and value that arrive with this step: into the cache, scored on the FP32 pipes
@@ -223,20 +304,36 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     for (int e = tid; e < D; e += DNT) {
       k_cache[((size_t)bkv * T_max + n) * D + e] = k_new[(size_t)bkv * D + e];
       v_cache[((size_t)bkv * T_max + n) * D + e] = v_new[(size_t)bkv * D + e];
+      if constexpr (KEY)      // k_hat(n): exactly bf16
+        reinterpret_cast<uint16_t*>(khat_cache)[((size_t)bkv * T_max + n) * D + e] =
+            (uint16_t)(__float_as_uint(qh_s[e]) >> 16);
     }
+    if (KEY && tid == 0) row_nnz[(size_t)bkv * T_max + n] = (uint16_t)fired_total;
     if (warp == 0) {
       const float k0 = to_f32(k_new[(size_t)bkv * D + lane]), k1 = to_f32(k_new[(size_t)bkv * D + 32 + lane]);
+      if constexpr (!KEY) {
 #pragma unroll
-      for (int hh = 0; hh < G; ++hh) {
-        float pr = fmaf(qh_s[hh * D + lane], k0, qh_s[hh * D + 32 + lane] * k1);
-        float pq = fmaf(q_s[hh * D + lane], k0, q_s[hh * D + 32 + lane] * k1);
+        for (int hh = 0; hh < G; ++hh) {
+          float pr = fmaf(qh_s[hh * D + lane], k0, qh_s[hh * D + 32 + lane] * k1);
+          float pq = fmaf(q_s[hh * D + lane], k0, q_s[hh * D + 32 + lane] * k1);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          pr += __shfl_xor_sync(0xffffffffu, pr, o);
-          pq += __shfl_xor_sync(0xffffffffu, pq, o);
+          for (int o = 16; o > 0; o >>= 1) {
+            pr += __shfl_xor_sync(0xffffffffu, pr, o);
+            pq += __shfl_xor_sync(0xffffffffu, pq, o);
+          }
+          if (lane == 0) R[((size_t)b * H + kvh * G + hh) * T_max + n] = pr;     // R[n] = q_hat . k_new
+          new_s[hh] = ((W > 0) ? pq : pr) * scale_log2e;                          // the new key is inside any window
         }
-        if (lane == 0) R[((size_t)b * H + kvh * G + hh) * T_max + n] = pr;     // R[n] = q_hat . k_new
-        new_s[hh] = ((W > 0) ? pq : pr) * scale_log2e;                          // the new key is inside any window
+      } else {
+        // the new key is inside any window W_d >= 1; with W_d = 0 even it is scored by its reference
+        const float r0 = (W > 0) ? k0 : qh_s[lane], r1 = (W > 0) ? k1 : qh_s[32 + lane];
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh) {
+          float pq = fmaf(q_s[hh * D + lane], r0, q_s[hh * D + 32 + lane] * r1);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) pq += __shfl_xor_sync(0xffffffffu, pq, o);
+          new_s[hh] = pq * scale_log2e;
+        }
       }
     }
   }
@@ -253,7 +350,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
 #pragma unroll
   for (int hh = 0; hh < G; ++hh) mx[hh] = new_s[hh];
   const uint32_t lane_sel = (uint32_t)(32 * (warp & 3)) << 16;
-  float* Rg = R + ((size_t)b * H + kvh * G) * T_max;
+  float* Rg = KEY ? nullptr : R + ((size_t)b * H + kvh * G) * T_max;
 #pragma unroll
   for (int u = 0; u < TPW; ++u) {
     const int t = 2 * u + (warp >> 2);
@@ -267,8 +364,13 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
       if (jj < cached) {
 #pragma unroll
         for (int hh = 0; hh < G; ++hh) {
-          Rg[(size_t)hh * T_max + j] = v[hh];               // R[j] = q_hat . k_j
-          const float s = ((n - j < W) ? v[G + hh] : v[hh]) * scale_log2e;
+          float s;
+          if constexpr (KEY) {
+            s = v[hh] * scale_log2e;                          // the tile's rows already are the hybrid keys
+          } else {
+            Rg[(size_t)hh * T_max + j] = v[hh];               // R[j] = q_hat . k_j
+            s = ((n - j < W) ? v[G + hh] : v[hh]) * scale_log2e;
+          }
           sv[u][hh] = s;
           mx[hh] = fmaxf(mx[hh], s);
         }
@@ -414,22 +516,33 @@ bool decode_tc_applies(const Shape& s, int dtype, int n) {
   return chunk >= 2 * TK && chunk <= MAXT * TK && nsplit <= kMaxDecodeSplits;
 }
 
-cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
-                                  const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
-                                  int window, int qhat_sel, DecodeTmapCache* cache, cudaStream_t st) {
+// The tensor map of a [B*H_kv, T_max, 64] bf16 cache, encoded once per cache pointer.
+static const CUtensorMap* cached_map(DecodeTmapCache* cache, const void* ptr, const Shape& s) {
+  static_assert(sizeof(CUtensorMap) <= sizeof(cache->map), "tensor-map cache");
+  CUtensorMap* m = reinterpret_cast<CUtensorMap*>(cache->map);
+  if (cache->ptr != ptr) {
+    if (!tc::encode3(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ptr, TCD, (uint64_t)s.T_max, (uint64_t)s.B * s.H_kv,
+                     TCD * 2, (uint64_t)s.T_max * TCD * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B))
+      return nullptr;
+    cache->ptr = ptr;
+  }
+  return m;
+}
+
+template <bool KEY>
+static cudaError_t launch_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
+                             const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
+                             int window, int qhat_sel, DecodeTmapCache* cache_k, DecodeTmapCache* cache_h,
+                             cudaStream_t st) {
   const int bkv = s.B * s.H_kv;
   int nsplit, chunk;
   decode_tc_slices(s, n, &nsplit, &chunk);
   if (nsplit > kMaxDecodeSplits || chunk > MAXT * TK) return cudaErrorInvalidValue;
-  static_assert(sizeof(CUtensorMap) <= sizeof(cache->map), "tensor-map cache");
-  CUtensorMap* tkp = reinterpret_cast<CUtensorMap*>(cache->map);
-  if (cache->ptr != k_cache) {
-    if (!tc::encode3(tkp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k_cache, TCD, (uint64_t)s.T_max, (uint64_t)bkv, TCD * 2,
-                     (uint64_t)s.T_max * TCD * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B))
-      return cudaErrorInvalidValue;
-    cache->ptr = k_cache;
-  }
+  const CUtensorMap* tkp = cached_map(cache_k, k_cache, s);
+  const CUtensorMap* thp = KEY ? cached_map(cache_h, w.qhat_rows, s) : tkp;
+  if (!tkp || !thp) return cudaErrorInvalidValue;
   const CUtensorMap& tk = *tkp;
+  const CUtensorMap& th = *thp;
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const int G = s.g();
   const dim3 grid(nsplit, bkv);
@@ -439,17 +552,17 @@ cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void
   using TC = __nv_bfloat16;
 #define LAUNCH(GG)                                                                               \
   do {                                                                                           \
-    auto kern = decode_step_tc_kernel<GG>;                                                       \
+    auto kern = decode_step_tc_kernel<GG, KEY>;                                                  \
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
     if (err != cudaSuccess) return err;                                                          \
     /* two CTAs per SM need the largest shared-memory carve-out */                               \
     err = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,             \
                                (int)cudaSharedmemCarveoutMaxShared);                             \
     if (err != cudaSuccess) return err;                                                          \
-    kern<<<grid, DNT, smem, st>>>(tk, (const TC*)q_new, (const TC*)k_new, (const TC*)v_new, (TC*)k_cache,  \
-                                  (TC*)v_cache, (TC*)out, w.qhat[qhat_sel], w.qhat[qhat_sel ^ 1], w.R,     \
-                                  w.dec_partial, w.dec_ticket, w.counters, n, s.T_max, s.H, chunk, nsplit, \
-                                  theta, window, scale_log2e);                                             \
+    kern<<<grid, DNT, smem, st>>>(tk, th, (const TC*)q_new, (const TC*)k_new, (const TC*)v_new, (TC*)k_cache, \
+                                  (TC*)v_cache, w.qhat_rows, w.row_nnz, (TC*)out, w.qhat[qhat_sel],        \
+                                  w.qhat[qhat_sel ^ 1], w.R, w.dec_partial, w.dec_ticket, w.counters, n,   \
+                                  s.T_max, s.H, chunk, nsplit, theta, window, scale_log2e);                \
   } while (0)
   switch (G) {
     case 1: LAUNCH(1); break;
@@ -461,6 +574,22 @@ cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void
 #undef LAUNCH
   count_launch();
   return cudaGetLastError();
+}
+
+cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
+                                  const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
+                                  int window, int qhat_sel, DecodeTmapCache* cache, cudaStream_t st) {
+  return launch_tc<false>(s, w, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window, qhat_sel, cache,
+                          nullptr, st);
+}
+
+cudaError_t launch_decode_step_key_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
+                                      const void* v_new, void* k_cache, void* v_cache, void* out, int n,
+                                      float theta, int window, int qhat_sel, DecodeTmapCache* cache_k,
+                                      DecodeTmapCache* cache_h, cudaStream_t st) {
+  if (!w.qhat_rows) return cudaErrorNotSupported;
+  return launch_tc<true>(s, w, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window, qhat_sel, cache_k,
+                         cache_h, st);
 }
 
 }  // namespace delta

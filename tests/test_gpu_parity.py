@@ -439,8 +439,12 @@ def test_key_delta_prefill_matches_oracle(B, case):
     (1, 2, 1, 90, 64, 0.1, 0, 3),          # no exact window at all
     (1, 2, 2, 40, 64, 0.0, 1000, 3),       # window covers the whole cache
     (1, 1, 1, 1, 64, 0.1, 2, 4),
+    (2, 4, 2, 700, 64, 0.2, 100, 3),       # the window's edge inside a tile, several slices
+    (3, 4, 4, 1500, 64, 0.2, 300, 2),      # window over three tiles: key-cache tiles, one mixed tile
+    (40, 4, 4, 1100, 64, 0.2, 64, 2),      # 160 KV heads: one slice of 9 tiles per head
 ])
-def test_key_delta_decode_steps_match_oracle(B, Bn, H, Hk, T, d, theta, W, steps):
+@pytest.mark.parametrize("decode_kernel", [0, 1], ids=["fp32_pipes", "tc_scores"])
+def test_key_delta_decode_steps_match_oracle(B, Bn, H, Hk, T, d, theta, W, steps, decode_kernel):
     """Strategy (3) carried into decoding: the reference key per KV head is the carried state,
     old keys are scored through the reference-key rows, the W_d most recent ones exactly."""
     from tests.gpu_helpers import to_cache, to_dev, to_host_f64
@@ -449,6 +453,10 @@ def test_key_delta_decode_steps_match_oracle(B, Bn, H, Hk, T, d, theta, W, steps
     T_max = T + steps
     cfg = B.make_config(Bn, H, Hk, d, T_max, "bf16", source=B.DELTA_SRC_KEY, prefill_window=B.DELTA_WIN_SLIDING)
     st = B.delta_state_init(cfg)
+    if decode_kernel == 1 and d != 64:
+        pytest.skip("tensor-core decode scores: d = 64")
+    B.delta_state_set_decode_kernel(st, decode_kernel)
+    assert B.delta_state_decode_kernel(st) == decode_kernel
     dq_, kc, vc = to_dev(t["q"], "bf16"), to_cache(t["k"], T_max, "bf16"), to_cache(t["v"], T_max, "bf16")
     out = torch.full_like(dq_, float("nan"))
     B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, float(theta), int(W))
