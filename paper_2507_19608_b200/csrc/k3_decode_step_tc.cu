@@ -461,13 +461,16 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
         }
       }
     }
-    // the warps run through the ring at their own pace: a stage is refilled (by one thread of
-    // the last warp) once all of them have released it
+    // the warps run through the ring at their own pace: a stage is refilled (by the last warp)
+    // once all of them have released it
     __syncwarp();
     if (lane == 0) tc::mbar_arrive(DBAR(BAR_VFREE0 + stg));
-    if (warp == DNW - 1 && lane == 0 && t + NVS < n_tiles) {
+    if (warp == DNW - 1 && t + NVS < n_tiles) {
+      // the whole warp waits (a lone lane polling beside its working warp would make the warp
+      // run both paths in turns)
       if (!mbar_wait(DBAR(BAR_VFREE0 + stg), par)) s_fail = 1;
-      issue_v(t + NVS);
+      if (lane == 0) issue_v(t + NVS);
+      __syncwarp();
     }
   }
   if (has_new && warp == 0 && sub == 0) {
