@@ -256,7 +256,7 @@ DELTA_API int32_t delta_state_position(const delta_state_t* st);
 DELTA_API int32_t delta_state_prefill_kernel(const delta_state_t* st);
 
 /* Which kernel the next delta_attn_decode_step of this state would use: 1 = score products
- * on the tensor cores (bf16, d = 64, top-down query deltas or key deltas, key slices of at least two 128-key tiles:
+ * on the tensor cores (bf16, d = 64, top-down query deltas or key deltas, at most 73728 keys:
  * the telescoped form of Eq. 4, see delta_attn_decode_step), 0 = the FP32-pipe kernel,
  * -1 for a null state.  Both compute the same step and keep the same state. */
 DELTA_API int32_t delta_state_decode_kernel(const delta_state_t* st);

@@ -85,8 +85,8 @@ struct DecodeTmapCache {
   const void* ptr = nullptr;
   alignas(64) unsigned char map[128];
 };
-// Does the step at position n take this kernel?  (bf16, d = 64, and key slices of at least two
-// tiles: with short slices the per-CTA set-up outweighs the saving.)  n < 0: shape and type only.
+// Does the step at position n take this kernel?  (bf16, d = 64, and a cache short enough for 64
+// slices of nine tiles.)  n < 0: shape and type only.
 bool decode_tc_applies(const Shape& s, int dtype, int n);
 cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
                                   const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
