@@ -84,7 +84,6 @@ static void carve(const delta_config_t& c, char* base, Workspace* w) {
   w->counters = (unsigned long long*)take(CNT_TOTAL * 8);
   w->dec_partial = (float*)take(BKV * kMaxDecodeSplits * g * (c.d + 2) * 4);
   w->dec_ticket = (uint32_t*)take(BKV * 4);
-  w->qhat_tile_bf16 = (c.dtype == DELTA_BF16) ? (__nv_bfloat16*)take(BH * nt * c.d * 2) : nullptr;
   w->kt = (c.dtype == DELTA_BF16 && tc_kernel_shape(c.d))
               ? (float*)take(BKV * c.d * (((size_t)c.T_max + 3) / 4 * 4) * 4) : nullptr;
   w->qhat_rows = (c.dtype == DELTA_BF16 && tcq_kernel_shape(c.d))

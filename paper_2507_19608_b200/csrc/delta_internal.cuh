@@ -38,7 +38,6 @@ struct Workspace {
   unsigned long long* counters;  // [CNT_TOTAL]
   float* dec_partial;   // [B,H_kv,kMaxDecodeSplits,g,(d+2)]
   uint32_t* dec_ticket; // [B,H_kv]
-  __nv_bfloat16* qhat_tile_bf16;  // [B,H,n_tiles,d] (bf16 configurations only)
   float* kt;            // [B,H_kv,d,round_up(T_max,4)] channel-major fp32 keys (tensor-core prefill only)
   __nv_bfloat16* qhat_rows;  // [B,H,T_max,d] reference state after every row (telescoped prefill only)
   size_t total_bytes;

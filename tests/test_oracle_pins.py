@@ -260,6 +260,44 @@ def test_query_deltas_keep_row0_exact_key_deltas_keep_col0_exact():
     assert np.max(np.abs(rb["S_delta"][:T - 1] - exact[:T - 1])) > 1e-2
 
 
+def test_bottom_up_scores_follow_the_reverse_chain_closed_form():
+    """Strategy (2): with the rows taken from the last to the first, the score row of token i is
+    the reference after rows T-1 .. i, dotted with the keys (Eq. 4 telescoped).  The reference is
+    re-derived here by a scalar loop of Eq. 2-3 that shares nothing with the oracle."""
+    T, d, theta = 40, 32, 0.4
+    q, k, v = _qkv(T, d, 83)
+    r = O.prefill_head(q, k, v, theta=theta, W=0, source="query", order="bottom_up")
+    ref = np.zeros(d, np.float32)
+    want = np.zeros((T, T))
+    for i in range(T - 1, -1, -1):
+        for c in range(d):
+            if i == T - 1:
+                ref[c] = q[i, c]                       # the basis row is kept whole
+            else:
+                diff = np.float32(q[i, c]) - ref[c]
+                if abs(diff) > np.float32(theta):
+                    ref[c] = q[i, c]
+        want[i] = ref.astype(np.float64) @ k.astype(np.float64).T
+    assert np.max(np.abs(r["S_delta"] - want)) < 1e-4
+    # a wrong direction would put the exact row at the top
+    assert np.max(np.abs(r["S_delta"][0] - q[0].astype(np.float64) @ k.astype(np.float64).T)) > 1e-2
+
+
+def test_bottom_up_is_top_down_on_the_mirrored_sequence():
+    """Delta construction of strategy (2) over q equals that of strategy (1) over q reversed,
+    row for row (Section III-A describes the two as the same procedure from opposite ends)."""
+    T, d, theta = 70, 32, 0.3
+    q, k, v = _qkv(T, d, 19)
+    rb = O.prefill_head(q, k, v, theta=theta, W=5, source="query", order="bottom_up")
+    rt = O.delta_construct(q[::-1], theta)
+    assert np.array_equal(rb["delta"]["mask"], rt["mask"])
+    assert np.array_equal(rb["delta"]["dq"].view(np.uint32), rt["dq"].view(np.uint32))
+    # and the hybrid output still takes exact scores inside the window
+    exact = q.astype(np.float64) @ k.astype(np.float64).T
+    win = O.window_matrix(T, 5, "block")
+    assert np.array_equal(rb["S_star"][win], exact[win])
+
+
 # ------------------------------------------------------------------ P8: window geometry and Eq. 5-6
 @pytest.mark.parametrize("T,W", [(128, 16), (100, 16), (64, 64), (33, 7), (10, 0), (10, 50)])
 def test_window_pair_counts_closed_form(T, W):
