@@ -338,6 +338,7 @@ def run_ours(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if w.dtype == "f32" else "bf16 in, f32 accumulate", "data": "synthetic",
         "config": config_dict(w, theta), "impl": "ours",
+        "ms_per_step_median": statistics.median(step_ms), "ms_per_step_min": min(step_ms),
         "prefill_kernel": KERNEL_NAMES[kernel],
         "gpu_launches": int(launches),
         "kernel_ms": {"delta_chain": kmean[0], "delta_finish": kmean[1], "hybrid_attn": kmean[2]},
