@@ -260,7 +260,7 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   const bool chained = (which == 2) && !prof;
   MARK(0);
   // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
-  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, key, rev, cs)) != cudaSuccess)
+  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, rev, cs)) != cudaSuccess)
     return cuda_fail(e);
   auto attention = [&]() -> cudaError_t {
     if (use_tc) return launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
@@ -269,11 +269,18 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
                                     rev, cs);
     return launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, c.dtype, cs);
   };
-  if (chained) {
+  if (chained && !key) {
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
     if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
                                  use_tc, key, rev, true, cs)) != cudaSuccess)
       return cuda_fail(e);
+  } else if (chained) {
+    // key deltas: the finish kernel writes the reference-key rows the attention kernel streams,
+    // so it comes first (both programmatically serialised behind the kernel in front)
+    if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
+                                 use_tc, key, rev, true, cs)) != cudaSuccess)
+      return cuda_fail(e);
+    if ((e = attention()) != cudaSuccess) return cuda_fail(e);
   } else {
     MARK(1);
     if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,

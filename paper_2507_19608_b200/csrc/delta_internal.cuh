@@ -51,16 +51,14 @@ struct Shape {
 
 void count_launch(int n = 1);
 
-// K1a: token-sequential delta chain (Eq. 2-3).  Query stream: the reference in front of every
-// 8-row block and every 64-row tile, final reference.  Key stream: also delta values, mask
-// words and reference rows.
+// K1a: token-sequential delta chain (Eq. 2-3): the reference in front of every 8-row block and
+// every 64-row tile, and the final reference.
 // key_stream: the stream is K in the KV-cache layout, one chain set per KV head (strategy 3).
 // reverse: rows are taken from T-1 down to 0 (strategy 2; query stream only).
-cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
-                               float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
-                               bool reverse, cudaStream_t st);
-// K1b: row-parallel finish: (query stream) delta values and mask words from the 8-row
-// checkpoints; counts, compacted indices, Eq. 6 counters, the decode hand-off row
+cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
+                               int init, bool key_stream, bool reverse, cudaStream_t st);
+// K1b: row-parallel finish: delta values, mask words and (key stream) reference rows from the
+// 8-row checkpoints; counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
 // programmatic: launched with programmatic stream serialisation (its launch overlaps the end
 // of the kernel in front; the kernel waits for that kernel's completion itself).

@@ -1,40 +1,32 @@
-// K1 -- delta construction (Section II-C, Eq. 2-3; Section III-A strategies (1) and (3)), in
+// K1 -- delta construction (Section II-C, Eq. 2-3; Section III-A strategies (1), (2), (3)), in
 // two kernels.
 //
 // delta_chain_kernel: the token-sequential part.  Eq. 3 makes every channel a chain along the
 // tokens (the reference is the last value that fired), so the only parallelism is across
-// channels: one thread per channel, one warp per 32 channels (= one mask word), one CTA per
-// (batch, head).  The chain itself is three dependent FP32 operations per token and a lone
-// warp issues slowly, so everything else is kept off it: a producer warp streams the head's
-// rows into a ring of shared-memory stages with bulk asynchronous copies (the rows do not
-// depend on the carried state), and for the query stream the chain warps store nothing but
-// the reference in front of every 8-row block (and every 64-row tile, and the final one).
-// Given those checkpoints every 8-row block of Eq. 2-3 is independent of the others: fire
-// bits, delta values, mask words and reference rows are recomputed from them by row-parallel
-// code (the finish kernel below, the attention kernel for its own query tile).
-// For the key stream (strategy 3) the chain kernel still stores delta values, reference rows
-// and mask words itself (fire bits of 32 rows in one register per thread, a 32 x 32 bit
-// transpose across the warp turns them into the rows' mask words).
+// channels: one thread per channel, one warp per 32 channels, one CTA per (batch, head) of the
+// stream (query heads, or KV heads for key deltas).  The chain itself is three dependent FP32
+// operations per token and a lone warp issues slowly, so everything else is kept off it: a
+// producer warp streams the head's rows into a ring of shared-memory stages with bulk
+// asynchronous copies (the rows do not depend on the carried state), and the chain warps store
+// nothing but the reference in front of every 8-row block (and every 64-row tile, and the final
+// one).  Given those checkpoints every 8-row block of Eq. 2-3 is independent of the others:
+// fire bits, delta values, mask words and reference rows are recomputed from them by
+// row-parallel code (the finish kernel below, the attention kernel for its own query tile).
 //
-// delta_finish_kernel: everything that is parallel over rows -- (query stream) Eq. 2-3 over
-// 8-row blocks from the checkpoints: delta values and mask words; per-row and per-tile
-// non-zero counts, the compacted channel indices, the counters behind Eq. 6 --
-// plus two passes over the keys that prefill needs anyway: the hand-off row
-// R(T-1)[j] = q_hat(T-1).k_j for decode and, for the tensor-core attention kernel with the
-// FP32 delta path, the channel-major fp32 copy of the keys.
+// delta_finish_kernel: everything that is parallel over rows -- Eq. 2-3 over 8-row blocks
+// from the checkpoints: delta values, mask words and (key deltas) the reference-key rows;
+// per-row and per-tile non-zero counts, the compacted channel indices, the counters behind
+// Eq. 6 -- plus, for query deltas, two passes over the keys that prefill needs anyway: the
+// hand-off row R(T-1)[j] = q_hat(T-1).k_j for decode and, for the tensor-core attention kernel
+// with the FP32 delta path, the channel-major fp32 copy of the keys.
 #include "delta_internal.cuh"
 
 namespace delta {
 
 namespace {
 
-// Ring geometry.  Key stream (the chain stores mask words): 32 rows per stage, one mask flush
-// per stage, 8 stages.  Query stream (checkpoints only): 64 rows per stage, 4 stages -- half
-// the per-stage bookkeeping on the chain warps for the same shared memory.
-template <bool EMIT> struct Ring {
-  static constexpr int RC = EMIT ? 32 : 64;   // rows per stage
-  static constexpr int NS = EMIT ? 8 : 4;     // stages
-};
+constexpr int RC = 64;       // rows per ring stage (= one 64-row tile)
+constexpr int NS = 4;        // ring stages
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -76,80 +68,33 @@ template <> __device__ __forceinline__ float lds_elem<__nv_bfloat16>(uint32_t ad
 }
 
 // One ring stage of the chain for one thread (= one channel): rows t0 .. t0+nrows-1, the
-// thread's values at rows[r * D]; updates the reference qh.
-// EMIT = false (query deltas): the sequential kernel carries nothing but the reference and,
-// with `write`, leaves it in front of every 8-row block (ckptp); fire bits, delta values and
-// everything derived from them are recomputed from those checkpoints by row-parallel kernels.
-// EMIT = true (key deltas): with `write` stores the stage's mask words, delta values and
-// reference rows itself.
-template <typename TIn, int D, bool EMIT>
-__device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, bool basis_row, bool write,
-                                            float& qh, float theta, int lane, float* dqp,
-                                            __nv_bfloat16* qrp, uint32_t* maskp, float* ckptp) {
-  constexpr int NW = D / 32;
-  constexpr int RC = Ring<EMIT>::RC;
-  // bit r of `bits`: did this thread's channel fire in row t0 + r
-  uint32_t bits = 0;
+// thread's values at rows[r * D]; updates the reference qh and leaves it in front of every
+// 8-row block (ckptp).  basis_row: the stage's first row is the un-thresholded basis.
+template <typename TIn, int D>
+__device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, bool basis_row, float& qh,
+                                            float theta, float* ckptp) {
   if (nrows == RC && !basis_row) {
-    // full stage, no basis row: all loads first, then nothing but the dependent chain
-    // (volatile loads: the compiler may not sink them into the chain, where their latency
-    // would sit on the dependent path)
+    // full stage, no basis row: nothing but loads, the dependent chain and the checkpoints
     float x[RC];
     const uint32_t saddr = smem_u32(rows);
 #pragma unroll
     for (int r = 0; r < RC; ++r) x[r] = lds_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
 #pragma unroll
     for (int r = 0; r < RC; ++r) {
-      if (!EMIT && write && (r % DELTA_CKPT_ROWS) == 0) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      if ((r % DELTA_CKPT_ROWS) == 0) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
       const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
       const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
       qh = fire ? x[r] : qh;
-      if (EMIT) {
-        if (write) {
-          dqp[(size_t)(t0 + r) * D] = fire ? diff : 0.0f;
-          if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
-        }
-        bits |= fire ? (1u << r) : 0u;
-      }
     }
   } else {
     for (int r = 0; r < nrows; ++r) {
-      if (!EMIT && write && ((t0 + r) % DELTA_CKPT_ROWS) == 0) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      if (((t0 + r) % DELTA_CKPT_ROWS) == 0) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
       const float x = to_f32(rows[r * D]);
-      bool fire;
-      float delta;
-      if (r == 0 && basis_row) {
-        fire = true;                                 // the basis vector is kept whole
-        delta = x;
-      } else {
-        const float diff = __fsub_rn(x, qh);
-        fire = fabsf(diff) > theta;
-        delta = fire ? diff : 0.0f;
-      }
+      const bool fire = (r == 0 && basis_row) || (fabsf(__fsub_rn(x, qh)) > theta);
       qh = fire ? x : qh;
-      if (EMIT) {
-        if (write) {
-          dqp[(size_t)(t0 + r) * D] = delta;
-          if (qrp) qrp[(size_t)(t0 + r) * D] = __float2bfloat16_rn(qh);
-        }
-        bits |= fire ? (1u << r) : 0u;
-      }
     }
   }
-  if (!EMIT || !write) return;
-  // 32 x 32 bit transpose across the warp: lane r ends up with the mask word of row t0 + r
-  uint32_t mymask = bits;
-#pragma unroll
-  for (int j = 16; j > 0; j >>= 1) {
-    const uint32_t km = (j == 16) ? 0x0000FFFFu : (j == 8) ? 0x00FF00FFu : (j == 4) ? 0x0F0F0F0Fu
-                      : (j == 2) ? 0x33333333u : 0x55555555u;
-    const uint32_t other = __shfl_xor_sync(0xffffffffu, mymask, j);
-    mymask = (lane & j) ? (((other >> j) & km) | (mymask & ~km))
-                        : ((mymask & km) | ((other & km) << j));
-  }
-  if (lane < nrows) maskp[(size_t)(t0 + lane) * NW] = mymask;
 }
-
 
 // Strategy (2): the same stage of the query stream taken from its last row down to its first.
 // The checkpoint of an 8-row block is the reference before the block's highest row.
@@ -157,7 +102,6 @@ __device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, 
 template <typename TIn, int D>
 __device__ __forceinline__ void chain_stage_rev(const TIn* rows, int t0, int nrows, bool basis_last, float& qh,
                                                 float theta, float* ckptp) {
-  constexpr int RC = Ring<false>::RC;
   if (nrows == RC && !basis_last) {
     float x[RC];
     const uint32_t saddr = smem_u32(rows);
@@ -183,19 +127,14 @@ __device__ __forceinline__ void chain_stage_rev(const TIn* rows, int t0, int nro
 
 }  // namespace
 
-// EMIT: also store the delta values and the reference rows (key deltas); without it the chain
-// leaves mask words and per-tile references only (query deltas: the rest is rebuilt row-parallel).
-template <typename TIn, int D, bool EMIT>
+template <typename TIn, int D>
 __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
-    const TIn* __restrict__ q, float* __restrict__ dq, uint32_t* __restrict__ mask,
-    float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
-    __nv_bfloat16* __restrict__ qhat_rows, float* __restrict__ ckpt,
-    unsigned long long* __restrict__ counters, int T, int T_max, int n_tiles, int n_ckpt, float theta,
-    int basis_exact, int src_rows, int reverse) {
+    const TIn* __restrict__ q, float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
+    float* __restrict__ ckpt, unsigned long long* __restrict__ counters, int T, int n_tiles, int n_ckpt,
+    float theta, int basis_exact, int src_rows, int reverse) {
   // q: the stream that becomes the delta matrix, [heads][src_rows][D] with rows 0..T-1 read
   // (queries: src_rows = T; keys in the KV-cache layout: src_rows = T_max)
-  constexpr int NW = D / 32;                       // chain warps = mask words per row
-  constexpr int RC = Ring<EMIT>::RC, NS = Ring<EMIT>::NS;
+  constexpr int NW = D / 32;                       // chain warps
   constexpr uint32_t ROW_BYTES = D * sizeof(TIn);
   constexpr uint32_t STAGE_BYTES = RC * ROW_BYTES;
   extern __shared__ __align__(128) unsigned char ring[];   // [NS][RC][D] of TIn
@@ -245,10 +184,7 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
   } else {
     // ---- chain warps: thread c owns channel c
     const int c = tid;
-    float* dqp = dq ? dq + (size_t)bh * T_max * D + c : nullptr;   // null: values left to the finish kernel
-    __nv_bfloat16* qrp = qhat_rows ? qhat_rows + (size_t)bh * T_max * D + c : nullptr;
-    uint32_t* maskp = mask + (size_t)bh * T_max * NW + warp;
-    float* ckptp = ckpt ? ckpt + (size_t)bh * n_ckpt * D + c : nullptr;
+    float* ckptp = ckpt + (size_t)bh * n_ckpt * D + c;
     float qh = 0.0f;          // reference state, starts at zero (Eq. 3)
     bool failed = false;
     for (int i = 0; i < n_chunks; ++i) {
@@ -259,11 +195,10 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
       if (!mbar_wait(full0 + 8 * s, (i / NS) & 1)) { failed = true; break; }
       const TIn* rows = reinterpret_cast<const TIn*>(ring + (size_t)s * STAGE_BYTES) + c;
       const int nrows = min(RC, T - t0);
-      if (!EMIT && reverse)
+      if (reverse)
         chain_stage_rev<TIn, D>(rows, t0, nrows, t0 + nrows == T && basis_exact, qh, theta, ckptp);
       else
-        chain_stage<TIn, D, EMIT>(rows, t0, nrows, t0 == 0 && basis_exact, true, qh, theta, lane, dqp, qrp, maskp,
-                                  ckptp);
+        chain_stage<TIn, D>(rows, t0, nrows, t0 == 0 && basis_exact, qh, theta, ckptp);
       __syncwarp();
       if (lane == 0)
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * s) : "memory");
@@ -276,33 +211,23 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
 }
 
 
-cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T,
-                               float theta, int dtype, int init, bool want_qhat_rows, bool key_stream,
-                               bool reverse, cudaStream_t st) {
+cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
+                               int init, bool key_stream, bool reverse, cudaStream_t st) {
   if (key_stream && reverse) return cudaErrorNotSupported;
-  __nv_bfloat16* qrows = want_qhat_rows ? w.qhat_rows : nullptr;
-  // query deltas: the chain leaves mask words and per-tile references only; delta values are
-  // recomputed row-parallel by the finish kernel.  Key deltas: the chain stores them itself.
-  float* dq_out = key_stream ? w.dq : nullptr;
-  float* ckpt_out = key_stream ? nullptr : w.ckpt;
-  float* tile_out = w.qhat_tile;
-  float* fin_out = w.qhat[0];
   const int grid = s.B * (key_stream ? s.H_kv : s.H);
   const int src_rows = key_stream ? s.T_max : T;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
   cudaError_t err = cudaSuccess;
 #define LAUNCH(TIN, DD)                                                                          \
   do {                                                                                           \
-    auto kern = key_stream ? delta_chain_kernel<TIN, DD, true> : delta_chain_kernel<TIN, DD, false>; \
-    const size_t smem = key_stream ? (size_t)Ring<true>::NS * Ring<true>::RC * DD * sizeof(TIN)  \
-                                   : (size_t)Ring<false>::NS * Ring<false>::RC * DD * sizeof(TIN); \
+    auto kern = delta_chain_kernel<TIN, DD>;                                                     \
+    const size_t smem = (size_t)NS * RC * DD * sizeof(TIN);                                      \
     if (smem > 48 * 1024) {                                                                      \
       err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
       if (err != cudaSuccess) return err;                                                        \
     }                                                                                            \
-    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, dq_out, w.mask, tile_out, fin_out, qrows, \
-                                      ckpt_out, w.counters, T, s.T_max, s.n_tiles, s.n_ckpt(), theta, \
-                                      basis, src_rows, reverse ? 1 : 0);                         \
+    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.qhat_tile, w.qhat[0], w.ckpt, w.counters, T, s.n_tiles, \
+                                      s.n_ckpt(), theta, basis, src_rows, reverse ? 1 : 0);      \
   } while (0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
@@ -311,7 +236,7 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
   }
 #undef LAUNCH
   count_launch();
-  return cudaGetLastError();
+  return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------------------
@@ -329,13 +254,19 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
     unsigned long long* __restrict__ counters, const TIn* __restrict__ k,
     const float* __restrict__ qhat, float* __restrict__ R, float* __restrict__ kt, int T,
     int T_max, int n_tiles, int BH, int H, int g, int W, int shape, int n_idx_blocks, int kt_ld,
-    int key_stream, const TIn* __restrict__ q, float* __restrict__ dq,
-    const float* __restrict__ ckpt, int n_ckpt, float theta, int basis_exact, int reverse) {
+    int key_stream, const TIn* __restrict__ q, int src_rows, float* __restrict__ dq,
+    __nv_bfloat16* __restrict__ ref_rows, const float* __restrict__ ckpt, int n_ckpt, float theta,
+    int basis_exact, int reverse) {
+  // q: the stream the chain kernel ran over, [heads][src_rows][D]; ref_rows (key deltas): the
+  // reference after every row, the cache of reference keys
   constexpr int NW = D / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // launched with programmatic stream serialisation behind the attention kernel: the results
   // of everything in front are visible from here on (no effect in an ordinary launch)
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // key deltas: the attention kernel is serialised programmatically behind this one and may set
+  // itself up meanwhile (it waits for this kernel's results itself)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if ((int)blockIdx.x < n_idx_blocks) {
     // ---- one block per (batch, head, 64-row tile); warp w serves rows 8w .. 8w+7
     __shared__ unsigned long long s_red[3][8];
@@ -345,10 +276,10 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
     const int rows = min(DELTA_TILE_ROWS, T - t0);
     const int r_mine = warp * 8 + (lane & 7);        // lanes 0..7 hold one row each
     uint32_t mw[NW];
-    if (ckpt != nullptr) {
-      // query deltas: the chain kernel left only the reference in front of every 8-row block.
-      // The warp re-runs Eq. 2-3 over its 8 rows (lane = channel of a mask word): delta values,
-      // and one ballot per row for the mask word.
+    {
+      // The chain kernel left only the reference in front of every 8-row block.  The warp
+      // re-runs Eq. 2-3 over its 8 rows (lane = channel of a mask word): delta values, reference
+      // rows (key deltas), and one ballot per row for the mask word.
       const int rbase = t0 + warp * 8;
 #pragma unroll
       for (int w2 = 0; w2 < NW; ++w2) {
@@ -359,7 +290,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
           float x[8];
 #pragma unroll
           for (int r = 0; r < 8; ++r)
-            x[r] = (rbase + r < T) ? to_f32(q[((size_t)bh * T + rbase + r) * D + c]) : 0.0f;
+            x[r] = (rbase + r < T) ? to_f32(q[((size_t)bh * src_rows + rbase + r) * D + c]) : 0.0f;
 #pragma unroll
           for (int rr = 0; rr < 8; ++rr) {
             const int r = reverse ? 7 - rr : rr;         // strategy (2) takes the rows from the top
@@ -378,6 +309,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
             if (live) {
               dq[((size_t)bh * T_max + rbase + r) * D + c] = delta;
               ref = fire ? x[r] : ref;
+              if (ref_rows) ref_rows[((size_t)bh * T_max + rbase + r) * D + c] = __float2bfloat16_rn(ref);
             }
             const uint32_t word = __ballot_sync(0xffffffffu, fire);
             if ((lane & 7) == r) word_mine = word;
@@ -386,10 +318,6 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
         mw[w2] = word_mine;
         if (lane < 8 && r_mine < rows) mask[((size_t)bh * T_max + t0 + r_mine) * NW + w2] = word_mine;
       }
-    } else {
-#pragma unroll
-      for (int w2 = 0; w2 < NW; ++w2)
-        mw[w2] = (r_mine < rows) ? mask[((size_t)bh * T_max + t0 + r_mine) * NW + w2] : 0u;
     }
     unsigned long long done = 0, dense = 0, tsum = 0;
     if (lane < 8 && r_mine < rows) {
@@ -534,8 +462,8 @@ cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* 
   err = cudaLaunchKernelEx(&cfg, delta_finish_kernel<TIN, DD>,                                   \
       w.mask, w.row_nnz, w.tile_nnz, w.idx, w.counters, (const TIN*)k, (const float*)w.qhat[0], w.R, kt, T,    \
       s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld, key_stream ? 1 : 0,   \
-      key_stream ? (const TIN*)nullptr : (const TIN*)q, key_stream ? (float*)nullptr : w.dq,      \
-      key_stream ? (const float*)nullptr : (const float*)w.ckpt, s.n_ckpt(), theta,               \
+      key_stream ? (const TIN*)k : (const TIN*)q, key_stream ? s.T_max : T, w.dq,                 \
+      key_stream ? w.qhat_rows : (__nv_bfloat16*)nullptr, (const float*)w.ckpt, s.n_ckpt(), theta, \
       init == DELTA_INIT_BASIS_EXACT ? 1 : 0, reverse ? 1 : 0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
