@@ -364,6 +364,71 @@ def test_full_size_prefill_sampled_heads(B, name, theta, heads, kernel):
         _check_out(o[0, h], ref["out"], w.dtype, f"{name} head {h}")
 
 
+@pytest.mark.parametrize("name,source,units", [
+    ("llama32_1b_decode_b16", "query", ((0, 0), (9, 5), (15, 7))),
+    ("llama32_1b_decode_b1", "query", ((0, 2), (0, 6))),
+    ("llama32_1b_decode_b16", "key", ((3, 1), (12, 4))),
+])
+def test_full_size_decode_sampled_units(B, name, source, units):
+    """The decode leg as the benchmark runs it (cache prefilled to 2048 tokens through
+    delta_attn_prefill with a sliding window, kernels chosen by the library, then decode steps):
+    outputs, carried references and score rows of sampled (batch, KV head) units against the
+    oracle, step by step."""
+    from tests.gpu_helpers import to_dev, to_host_f64
+    w = WL.WORKLOADS[name]
+    theta, steps = w.thetas[0], 3
+    t = WL.make_qkv(w, n_decode=steps)
+    key = source == "key"
+    cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T_max, w.dtype, prefill_window=B.DELTA_WIN_SLIDING,
+                        source=B.DELTA_SRC_KEY if key else B.DELTA_SRC_QUERY)
+    st = B.delta_state_init(cfg)
+    g = w.H // w.H_kv
+
+    def cache(x):
+        full = np.zeros((w.B, w.H_kv, w.T_max, w.d), np.float32)
+        full[:, :, :w.T] = x
+        return to_dev(full, w.dtype)
+    q, kc, vc = to_dev(t["q"], w.dtype), cache(t["k"]), cache(t["v"])
+    out = torch.empty_like(q)
+    B.delta_attn_prefill(st, q, kc, vc, out, w.T, w.H, w.H_kv, w.d, float(theta), int(w.window))
+    assert B.delta_state_decode_kernel(st) == 1          # the tensor-core score kernel serves this shape
+    o_pre = to_host_f64(out)
+    states = {}
+    for (b, kvh) in units:
+        for hh in range(1 if key else g):
+            h = kvh * g + hh
+            r = O.prefill_head(t["q"][b, h], t["k"][b, kvh], t["v"][b, kvh], theta, w.window, "sliding",
+                               source=source)
+            _check_out(o_pre[b, h], r["out"], w.dtype, f"prefill unit {(b, h)}")
+            states[(b, kvh) if key else (b, h)] = r["state"]
+    for s_ in range(steps):
+        qn, kn, vn = t["q_dec"][:, :, s_], t["k_dec"][:, :, s_], t["v_dec"][:, :, s_]
+        o = torch.empty_like(to_dev(qn, w.dtype))
+        B.delta_attn_decode_step(st, to_dev(qn, w.dtype), to_dev(kn, w.dtype), to_dev(vn, w.dtype), kc, vc, o,
+                                 float(theta), int(w.window))
+        og = to_host_f64(o)
+        n = w.T + s_
+        if key:
+            for (b, kvh) in list(states):
+                stt, _ = O.decode_key_step(states[(b, kvh)], kn[b, kvh], vn[b, kvh], theta)
+                states[(b, kvh)] = stt
+                for hh in range(g):
+                    ref_o = O.decode_key_attend(stt, qn[b, kvh * g + hh], w.window)
+                    _check_out(og[b, kvh * g + hh], np.asarray(ref_o), w.dtype,
+                               f"key decode step {s_} unit {(b, kvh, hh)}")
+        else:
+            R = B.delta_state_view(st, B.DELTA_VIEW_R).cpu().numpy()
+            qh = B.delta_state_view(st, B.DELTA_VIEW_QHAT).cpu().numpy()
+            for (b, h) in list(states):
+                ref_o, stt, _ = O.decode_head(states[(b, h)], qn[b, h], kn[b, h // g], vn[b, h // g], theta, w.window)
+                states[(b, h)] = stt
+                _check_out(og[b, h], np.asarray(ref_o), w.dtype, f"decode step {s_} unit {(b, h)}")
+                assert np.array_equal(qh[b, h].view(np.uint32), stt["qhat"].view(np.uint32))
+                tol = 1e-3 * max(1.0, np.abs(stt["R"]).max())
+                assert np.abs(R[b, h, :n + 1] - stt["R"]).max() <= tol
+    assert B.delta_sparsity_stats(st)["device_status"] == 0
+
+
 @pytest.mark.parametrize("kernel,theta", [(2, 0.1), (1, 0.2)])
 def test_stack_layer_sampled_units(B, kernel, theta):
     """One layer of the 16-layer stack configuration (batch 8, T = 4096, block window 256) at full
