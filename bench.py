@@ -686,7 +686,12 @@ def run_delta_pass_large(B, torch, peaks, flush):
                             "unit": "GB/s", "frac": chain_b / (cm * 1e-3) / 1e9 / hbm},
             "delta_finish": {"ms": fm, "bound": "hbm", "achieved": finish_b / (fm * 1e-3) / 1e9, "peak": hbm,
                              "unit": "GB/s", "frac": finish_b / (fm * 1e-3) / 1e9 / hbm},
-            "hybrid_attn": {"ms": am, "dense_equiv_tflops": 4.0 * w.d * N_c * w.B * w.H / (am * 1e-3) / 1e12}}
+            "hybrid_attn": {"ms": am, "dense_equiv_tflops": 4.0 * w.d * N_c * w.B * w.H / (am * 1e-3) / 1e12,
+                            "bound": "tensor", "peak": float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+                            "unit": "TFLOP/s",
+                            "frac": 4.0 * w.d * N_c * w.B * w.H / (am * 1e-3) / 1e12
+                            / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+                            "note": "dense-equivalent flops (4 d N_c per head) over the sustained cuBLAS bf16 rate"}}
 
 
 def run_cpu_baseline(args, w, tens, theta):
