@@ -32,8 +32,7 @@ struct delta_state {
   // Eq. 6 bookkeeping that needs no device work: sum of window lengths and sequence lengths
   double win_sum[2], len_sum[2];
   DecodeTmapCache dec_tmap;   // tensor map of the key cache the decode steps read
-  DecodeTmapCache dec_tmap_h; // of the reference-key cache (key deltas)
-  DecodeTmapCache dec_tmap_v; // and of the value cache
+  DecodeTmapCache dec_tmap_h; // and of the reference-key cache (key deltas)
   int forced_decode_kernel = -1;   // -1: chosen per step
   // optional per-kernel timing of prefill (host-side event objects)
   bool profiling = false, profiled = false;
@@ -364,12 +363,12 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
   cudaError_t e;
   if (st->cfg.source == DELTA_SRC_KEY)
     e = tcs ? launch_decode_step_key_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
-                                        window, st->qhat_sel, &st->dec_tmap, &st->dec_tmap_h, &st->dec_tmap_v, cs)
+                                        window, st->qhat_sel, &st->dec_tmap, &st->dec_tmap_h, cs)
             : launch_decode_step_key(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
                                      window, st->qhat_sel, cs);
   else
     e = tcs ? launch_decode_step_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
-                                    window, st->qhat_sel, &st->dec_tmap, &st->dec_tmap_v, cs)
+                                    window, st->qhat_sel, &st->dec_tmap, cs)
             : launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
                                  window, st->cfg.dtype, st->qhat_sel, cs);
   if (e != cudaSuccess) return cuda_fail(e);

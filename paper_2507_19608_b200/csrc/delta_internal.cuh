@@ -87,13 +87,12 @@ struct DecodeTmapCache {
 bool decode_tc_applies(const Shape& s, int dtype, int n);
 cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
                                   const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
-                                  int window, int qhat_sel, DecodeTmapCache* cache, DecodeTmapCache* cache_v,
-                                  cudaStream_t st);
+                                  int window, int qhat_sel, DecodeTmapCache* cache, cudaStream_t st);
 // The same for key deltas: tiles come from the reference-key cache or, inside the window, the key cache.
 cudaError_t launch_decode_step_key_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
                                       const void* v_new, void* k_cache, void* v_cache, void* out, int n,
                                       float theta, int window, int qhat_sel, DecodeTmapCache* cache_k,
-                                      DecodeTmapCache* cache_h, DecodeTmapCache* cache_v, cudaStream_t st);
+                                      DecodeTmapCache* cache_h, cudaStream_t st);
 cudaError_t launch_decode_step_key(const Shape& s, const Workspace& w, const void* q_new,
                                    const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                    void* out, int n, float theta, int window, int qhat_sel,

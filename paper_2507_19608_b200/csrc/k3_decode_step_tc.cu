@@ -8,11 +8,8 @@
 //   S[128 keys][16] = K_tile[128][64] . Qcat[16][64]^T,
 // where the rows of Qcat are the G new reference vectors, the G new query vectors and zeros.
 // The score row R is no longer read; it is written (R[j] = q_hat . k_j) because it is part of
-// the carried state.  P.V goes to the tensor cores as well: the G rows of P (bf16, like the
-// prefill kernel's) are the first rows of a 128-row operand whose other rows are whatever
-// shared memory follows -- a row of the product depends on its own operand row only, and the
-// rows past G are never read back.  The FP32 pipes keep the threshold step (Eq. 2-3) and the
-// softmax.
+// the carried state.  The FP32 pipes keep what is not a contraction of useful shape: the
+// threshold step (Eq. 2-3), the softmax and P.V (G rows of P against the value tile).
 //
 // Grid = (key slices, batch x KV heads); a CTA serves the G query heads of one KV head.
 //   1. threshold q_new against the carried reference, build Qcat in the operand layout;
@@ -20,9 +17,9 @@
 //      the products; all score tiles of the slice stay in tensor memory (16 columns per tile);
 //   3. one softmax over the slice: every thread reads its keys' scores (lane = key), hybrid
 //      select, scale, R written; maximum and sum reduced once per slice, not per tile;
-//   4. P.V: warp 4 streams the value tiles with TMA through a ring (three stages of its own plus
-//      the two key stages once the score products are done) and issues one 128 x 64 x 128
-//      product per tile, accumulated in tensor memory over the slice;
+//   4. P.V with the value tiles streamed through a ring of bulk copies (three stages of its own
+//      plus the two key stages once the products are done), the warps releasing stages through
+//      mbarriers (no block-wide barrier per tile);
 //   5. the slice result is stored and the last CTA of the (batch, KV head) merges the slices.
 // The key and value that arrive with this step are scored on the FP32 pipes by the CTA that
 // owns their slice (their cache row is written by this very kernel).
@@ -59,9 +56,7 @@ constexpr int kTcTargetCtas = 296;
 
 constexpr int NVS_OWN = 3;             // value-ring stages of its own
 constexpr int NVS = NVS_OWN + 2;       // plus the two key stages once the score products are done
-enum { BAR_K0 = 0, BAR_K1, BAR_KFREE0, BAR_KFREE1, BAR_S, BAR_O, BAR_V0, BAR_VFREE0 = BAR_V0 + NVS, DEC_NUM_BARS = BAR_VFREE0 + NVS };
-constexpr uint32_t TMEM_OUT = 192;     // P.V accumulator: 64 columns behind the score tiles
-constexpr uint32_t P_TILE = 2048;      // bytes of P per key tile: two 64-key blocks of 8 rows x 128 B
+enum { BAR_K0 = 0, BAR_K1, BAR_KFREE0, BAR_KFREE1, BAR_S, BAR_V0, BAR_VFREE0 = BAR_V0 + NVS, DEC_NUM_BARS = BAR_VFREE0 + NVS };
 
 
 // The G probabilities of one key (contiguous, 16-byte aligned for G >= 4).
@@ -83,7 +78,6 @@ template <int G> __device__ __forceinline__ void load_probs(const float* p, floa
 template <int G, bool KEY>
 __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_h,
-    const __grid_constant__ CUtensorMap tm_v,
     const __nv_bfloat16* __restrict__ q_new,
     const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
     __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
@@ -94,25 +88,21 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     float theta, int W, float scale_log2e) {
   using TC = __nv_bfloat16;
   constexpr int D = TCD;
-  constexpr int LPK = D / 8;
+  constexpr int LPK = D / 8, KPW = 32 / LPK;
   extern __shared__ unsigned char dsm_raw0[];
   const uint32_t raw = smem_u32(dsm_raw0);
   const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled operand tiles want 1 KiB alignment
   unsigned char* sm = dsm_raw0 + (base - raw);
-  // P of every tile of the slice, operand layout (128-byte swizzle): per tile two 64-key blocks,
-  // each one 8-row group (rows = heads).  A product reads 128 rows per block, i.e. up to 16 KiB
-  // past the block's start: the rings below keep that inside the CTA's shared memory.
-  constexpr uint32_t OFF_P = 0;
-  constexpr uint32_t OFF_K = (MAXT * P_TILE + 1023u) & ~1023u;   // [2][128][64] bf16, 128-byte swizzle
-  constexpr uint32_t OFF_V = OFF_K + 2 * TILE_BYTES;     // [NVS_OWN][128][64] bf16, 128-byte swizzle
+  constexpr uint32_t OFF_K = 0;                          // [2][128][64] bf16, 128-byte swizzle
+  constexpr uint32_t OFF_V = OFF_K + 2 * TILE_BYTES;     // [NVS_OWN][128][64] bf16, plain rows
   constexpr uint32_t OFF_QC = OFF_V + NVS_OWN * TILE_BYTES;  // Qcat [16][64] bf16, 128-byte swizzle
   constexpr uint32_t OFF_F = OFF_QC + 2048;              // floats from here on
   float* q_s = reinterpret_cast<float*>(sm + OFF_F);     // [G][D]
   float* qh_s = q_s + G * D;                             // [G][D]
   float* red = reinterpret_cast<float*>(sm + OFF_K);     // [DNW][G][D]: the key ring is free by then
   float* wgt = qh_s + G * D;                             // [G * kMaxDecodeSplits] (merge) / [DNW][2G] (reductions)
-  float* p_s = wgt + G * kMaxDecodeSplits;               // [8]: probabilities of the new key
-  float* st_s = p_s + 8;                                 // [24]
+  float* p_s = wgt + G * kMaxDecodeSplits;               // [MAXT * TK + 1][G] probabilities
+  float* st_s = p_s + (MAXT * TK + 1) * G;               // [24]
   __shared__ __align__(8) unsigned long long bars[DEC_NUM_BARS];
   __shared__ uint32_t s_tmem;
   __shared__ int s_last, s_fail;
@@ -144,15 +134,17 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  const TC* vc = v_cache + (size_t)bkv * T_max * D;
   auto v_rows = [&](int t) { return min(TK, cached - t * TK); };
   // value stage s: three of its own, then the two key stages (free once all score products are done)
   auto v_stage_off = [&](int s2) -> uint32_t {
     return s2 < NVS_OWN ? OFF_V + (uint32_t)s2 * TILE_BYTES : OFF_K + (uint32_t)(s2 - NVS_OWN) * TILE_BYTES;
   };
   auto issue_v = [&](int t) {
+    const uint32_t bytes = (uint32_t)v_rows(t) * D * 2u;
     const uint32_t bar = DBAR(BAR_V0 + (t % NVS));
-    tc::mbar_expect_tx(bar, TILE_BYTES);
-    tc::tma_load_3d(base + v_stage_off(t % NVS), &tm_v, bar, 0, j0 + t * TK, bkv);
+    tc::mbar_expect_tx(bar, bytes);
+    bulk_load(base + v_stage_off(t % NVS), vc + (size_t)(j0 + t * TK) * D, bytes, bar);
   };
 
   auto issue_k = [&](int t) {
@@ -161,7 +153,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     tc::tma_load_3d(base + OFF_K + (t & 1) * TILE_BYTES, src, DBAR(BAR_K0 + (t & 1)), 0, j0 + t * TK, bkv);
   };
   if (tid == 0) {
-    for (int i = 0; i < DEC_NUM_BARS; ++i) tc::mbar_init(DBAR(i), 1u);
+    for (int i = 0; i < DEC_NUM_BARS; ++i) tc::mbar_init(DBAR(i), i >= BAR_VFREE0 ? (uint32_t)DNW : 1u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     tc::fence_proxy_async();
     s_fail = 0;
@@ -406,15 +398,12 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   for (int u = 0; u < TPW; ++u) {
     const int t = 2 * u + (warp >> 2);
     if (t < n_tiles) {
+      const int jj = t * TK + 32 * (warp & 3) + lane;
 #pragma unroll
       for (int hh = 0; hh < G; ++hh) {
         const float p = exp2f(sv[u][hh] - mx[hh]);          // 0 for keys past the cached rows
         sum[hh] += p;
-        // row hh, key kk of the tile's P operand
-        const int kk = 32 * (warp & 3) + lane;
-        *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + (uint32_t)t * P_TILE + (uint32_t)(kk >> 6) * 1024u +
-                                          (uint32_t)hh * 128u + (((((uint32_t)kk & 63u) >> 3) ^ (uint32_t)hh) << 4) +
-                                          ((uint32_t)kk & 7u) * 2u) = __float2bfloat16_rn(p);
+        p_s[(size_t)jj * G + hh] = p;
       }
     }
   }
@@ -422,7 +411,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
 #pragma unroll
     for (int hh = 0; hh < G; ++hh) {
       const float p = exp2f(new_s[hh] - mx[hh]);
-      if (lane == 0) { sum[hh] += p; p_s[hh] = p; }
+      if (lane == 0) { sum[hh] += p; p_s[(size_t)(MAXT * TK) * G + hh] = p; }
     }
   }
 #pragma unroll
@@ -431,7 +420,6 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     for (int o = 16; o > 0; o >>= 1) sum[hh] += __shfl_xor_sync(0xffffffffu, sum[hh], o);
     if (lane == 0) wgt[warp * 2 * G + G + hh] = sum[hh];
   }
-  tc::fence_proxy_async();           // P was written through the generic proxy
   __syncthreads();
   if (tid < G) {
     float s = 0.0f;
@@ -440,44 +428,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     st_s[8 + tid] = s;
   }
 
-  // ---- 4. P.V on the tensor cores (warp 4: lane 0 issues, the warp stays converged)
-  if (warp == 4 && n_tiles > 0) {
-    const uint32_t IDESC_PV = tc::make_idesc(D, 1);
-    for (int t = 0; t < n_tiles; ++t) {
-      const int stg = t % NVS;
-      const uint32_t par = (uint32_t)(t / NVS) & 1u;
-      if (!mbar_wait(DBAR(BAR_V0 + stg), par)) s_fail = 1;
-      const int rows = v_rows(t);
-      if (rows < TK) {
-        // value rows past the cached keys are not the slice's (they may hold anything, and
-        // 0 x NaN would spoil the product): zero them
-        for (int e = lane; e < (TK - rows) * 8; e += 32)
-          *reinterpret_cast<uint4*>(sm + v_stage_off(stg) + (uint32_t)(rows + (e >> 3)) * 128u + (uint32_t)(e & 7) * 16u) =
-              make_uint4(0u, 0u, 0u, 0u);
-        tc::fence_proxy_async();
-      }
-      __syncwarp();
-      if (lane == 0) {
-        tc::tc_fence_after();
-        const uint32_t vb = base + v_stage_off(stg);
-        const uint32_t pb = base + OFF_P + (uint32_t)t * P_TILE;
-#pragma unroll
-        for (int ks = 0; ks < TK / 16; ++ks)
-          tc::tc_mma(tmem + TMEM_OUT, tc::make_desc(pb + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 1024),
-                     tc::make_desc(vb + ks * 2048, TILE_BYTES, 1024), IDESC_PV, (t > 0 || ks > 0) ? 1u : 0u);
-        if (t + NVS < n_tiles) {
-          tc::tc_commit(DBAR(BAR_VFREE0 + stg));
-          if (!mbar_wait(DBAR(BAR_VFREE0 + stg), par)) s_fail = 1;
-          issue_v(t + NVS);
-        }
-      }
-      __syncwarp();
-    }
-    if (lane == 0) tc::tc_commit(DBAR(BAR_O));
-    __syncwarp();
-  }
-  // the slice's output rows: tensor-memory lanes 0 .. G-1, 64 columns; through shared memory
-  // into the register layout the slice merge expects (warp 0, lanes 0..7: 8 channels each)
+  // ---- 4. P.V: value tiles through a two-stage ring; lane (l % 8) holds 8 channels, l / 8 the key
   const int sub = lane / LPK;
   const int c0 = (lane % LPK) * 8;
   float acc[G][8];
@@ -485,35 +436,51 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   for (int hh = 0; hh < G; ++hh)
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[hh][e] = 0.0f;
-  if (warp == 0) {
-    float* o_s = wgt;                 // [G][D] (the reductions above are done with it)
-    __syncwarp();
-    if (n_tiles > 0) {
-      if (!mbar_wait(DBAR(BAR_O), 0)) s_fail = 1;
-      tc::tc_fence_after();
+  for (int t = 0; t < n_tiles; ++t) {
+    const int stg = t % NVS;
+    const uint32_t par = (uint32_t)(t / NVS) & 1u;
+    if (!mbar_wait(DBAR(BAR_V0 + stg), par)) s_fail = 1;
+    const TC* vt = reinterpret_cast<const TC*>(sm + v_stage_off(stg));
+    const int rows = v_rows(t);
+    for (int jb = warp * KPW; jb < rows; jb += DNW * KPW) {
+      const int jj = jb + sub;
+      if (jj < rows) {
+        float vv[8];
+        load8(vt + (size_t)jj * D + c0, vv);
+        float pr[G];
+        load_probs<G>(p_s + (size_t)(t * TK + jj) * G, pr);
 #pragma unroll
-      for (int q4 = 0; q4 < D / 16; ++q4) {
-        float v[16];
-        tc::tc_ld16(tmem + TMEM_OUT + 16 * q4, v);
-        if (lane < G) {
+        for (int hh = 0; hh < G; ++hh) {
+          const float2 p2 = make_float2(pr[hh], pr[hh]);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) o_s[lane * D + 16 * q4 + c] = v[c];
+          for (int e = 0; e < 8; e += 2) {
+            const float2 a = tc::ffma2(p2, make_float2(vv[e], vv[e + 1]), make_float2(acc[hh][e], acc[hh][e + 1]));
+            acc[hh][e] = a.x;
+            acc[hh][e + 1] = a.y;
+          }
         }
       }
-      tc::tc_fence_before();
-    } else {
-      for (int e = lane; e < G * D; e += 32) o_s[e] = 0.0f;
     }
+    // the warps run through the ring at their own pace: a stage is refilled (by the last warp)
+    // once all of them have released it
     __syncwarp();
-    if (sub == 0) {
-      float vv[8];
-      if (has_new) load8(v_new + (size_t)bkv * D + c0, vv);
+    if (lane == 0) tc::mbar_arrive(DBAR(BAR_VFREE0 + stg));
+    if (warp == DNW - 1 && t + NVS < n_tiles) {
+      // the whole warp waits (a lone lane polling beside its working warp would make the warp
+      // run both paths in turns)
+      if (!mbar_wait(DBAR(BAR_VFREE0 + stg), par)) s_fail = 1;
+      if (lane == 0) issue_v(t + NVS);
+      __syncwarp();
+    }
+  }
+  if (has_new && warp == 0 && sub == 0) {
+    float vv[8];
+    load8(v_new + (size_t)bkv * D + c0, vv);
 #pragma unroll
-      for (int hh = 0; hh < G; ++hh) {
-        const float pn = has_new ? p_s[hh] : 0.0f;
+    for (int hh = 0; hh < G; ++hh) {
+      const float p = p_s[(size_t)(MAXT * TK) * G + hh];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[hh][e] = o_s[hh * D + c0 + e] + (has_new ? pn * vv[e] : 0.0f);
-      }
+      for (int e = 0; e < 8; ++e) acc[hh][e] = fmaf(p, vv[e], acc[hh][e]);
     }
   }
   __syncthreads();
@@ -570,23 +537,21 @@ template <bool KEY>
 static cudaError_t launch_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
                              const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
                              int window, int qhat_sel, DecodeTmapCache* cache_k, DecodeTmapCache* cache_h,
-                             DecodeTmapCache* cache_v, cudaStream_t st) {
+                             cudaStream_t st) {
   const int bkv = s.B * s.H_kv;
   int nsplit, chunk;
   decode_tc_slices(s, n, &nsplit, &chunk);
   if (nsplit > kMaxDecodeSplits || chunk > MAXT * TK) return cudaErrorInvalidValue;
   const CUtensorMap* tkp = cached_map(cache_k, k_cache, s);
   const CUtensorMap* thp = KEY ? cached_map(cache_h, w.qhat_rows, s) : tkp;
-  const CUtensorMap* tvp = cached_map(cache_v, v_cache, s);
-  if (!tkp || !thp || !tvp) return cudaErrorInvalidValue;
+  if (!tkp || !thp) return cudaErrorInvalidValue;
   const CUtensorMap& tk = *tkp;
   const CUtensorMap& th = *thp;
-  const CUtensorMap& tv = *tvp;
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const int G = s.g();
   const dim3 grid(nsplit, bkv);
-  const size_t smem = 1024 + (((size_t)MAXT * P_TILE + 1023) & ~(size_t)1023) + (size_t)(2 + NVS_OWN) * TILE_BYTES +
-                      2048 + ((size_t)2 * G * TCD + (size_t)G * kMaxDecodeSplits + 8 + 24) * 4;
+  const size_t smem = 1024 + (size_t)(2 + NVS_OWN) * TILE_BYTES + 2048 +
+                      ((size_t)2 * G * TCD + (size_t)G * kMaxDecodeSplits + (size_t)(MAXT * TK + 1) * G + 24) * 4;
   cudaError_t err = cudaSuccess;
   using TC = __nv_bfloat16;
 #define LAUNCH(GG)                                                                               \
@@ -598,7 +563,7 @@ static cudaError_t launch_tc(const Shape& s, const Workspace& w, const void* q_n
     err = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,             \
                                (int)cudaSharedmemCarveoutMaxShared);                             \
     if (err != cudaSuccess) return err;                                                          \
-    kern<<<grid, DNT, smem, st>>>(tk, th, tv, (const TC*)q_new, (const TC*)k_new, (const TC*)v_new, (TC*)k_cache, \
+    kern<<<grid, DNT, smem, st>>>(tk, th, (const TC*)q_new, (const TC*)k_new, (const TC*)v_new, (TC*)k_cache, \
                                   (TC*)v_cache, w.qhat_rows, w.row_nnz, (TC*)out, w.qhat[qhat_sel],        \
                                   w.qhat[qhat_sel ^ 1], w.R, w.dec_partial, w.dec_ticket, w.counters, n,   \
                                   s.T_max, s.H, chunk, nsplit, theta, window, scale_log2e);                \
@@ -617,19 +582,18 @@ static cudaError_t launch_tc(const Shape& s, const Workspace& w, const void* q_n
 
 cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
                                   const void* v_new, void* k_cache, void* v_cache, void* out, int n, float theta,
-                                  int window, int qhat_sel, DecodeTmapCache* cache, DecodeTmapCache* cache_v,
-                                  cudaStream_t st) {
+                                  int window, int qhat_sel, DecodeTmapCache* cache, cudaStream_t st) {
   return launch_tc<false>(s, w, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window, qhat_sel, cache,
-                          nullptr, cache_v, st);
+                          nullptr, st);
 }
 
 cudaError_t launch_decode_step_key_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
                                       const void* v_new, void* k_cache, void* v_cache, void* out, int n,
                                       float theta, int window, int qhat_sel, DecodeTmapCache* cache_k,
-                                      DecodeTmapCache* cache_h, DecodeTmapCache* cache_v, cudaStream_t st) {
+                                      DecodeTmapCache* cache_h, cudaStream_t st) {
   if (!w.qhat_rows) return cudaErrorNotSupported;
   return launch_tc<true>(s, w, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window, qhat_sel, cache_k,
-                         cache_h, cache_v, st);
+                         cache_h, st);
 }
 
 }  // namespace delta
