@@ -128,6 +128,10 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   const uint32_t bar0 = smem_u32(&bars[0]);
 #define DBAR(i) (bar0 + 8u * (uint32_t)(i))
 
+  // Decode steps follow one another in a stream: launched with programmatic stream
+  // serialisation, the next step's CTAs may become resident as soon as all of this step's have
+  // started; whatever touches global memory waits for the step in front below.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
                  "r"(DEC_TMEM_COLS)
@@ -152,6 +156,9 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     const CUtensorMap* src = (KEY && tile_kind(t) != 1) ? &tm_h : &tm_k;
     tc::tma_load_3d(base + OFF_K + (t & 1) * TILE_BYTES, src, DBAR(BAR_K0 + (t & 1)), 0, j0 + t * TK, bkv);
   };
+  // the step in front (or the prefill) has written the carried reference, the cache rows and
+  // the slice tickets this step reads
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tid == 0) {
     for (int i = 0; i < DEC_NUM_BARS; ++i) tc::mbar_init(DBAR(i), i >= BAR_VFREE0 ? (uint32_t)DNW : 1u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -554,6 +561,16 @@ static cudaError_t launch_tc(const Shape& s, const Workspace& w, const void* q_n
                       ((size_t)2 * G * TCD + (size_t)G * kMaxDecodeSplits + (size_t)(MAXT * TK + 1) * G + 24) * 4;
   cudaError_t err = cudaSuccess;
   using TC = __nv_bfloat16;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(DNT);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
 #define LAUNCH(GG)                                                                               \
   do {                                                                                           \
     auto kern = decode_step_tc_kernel<GG, KEY>;                                                  \
@@ -563,10 +580,11 @@ static cudaError_t launch_tc(const Shape& s, const Workspace& w, const void* q_n
     err = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,             \
                                (int)cudaSharedmemCarveoutMaxShared);                             \
     if (err != cudaSuccess) return err;                                                          \
-    kern<<<grid, DNT, smem, st>>>(tk, th, (const TC*)q_new, (const TC*)k_new, (const TC*)v_new, (TC*)k_cache, \
-                                  (TC*)v_cache, w.qhat_rows, w.row_nnz, (TC*)out, w.qhat[qhat_sel],        \
-                                  w.qhat[qhat_sel ^ 1], w.R, w.dec_partial, w.dec_ticket, w.counters, n,   \
-                                  s.T_max, s.H, chunk, nsplit, theta, window, scale_log2e);                \
+    err = cudaLaunchKernelEx(&cfg, kern, tk, th, (const TC*)q_new, (const TC*)k_new, (const TC*)v_new,     \
+                             (TC*)k_cache, (TC*)v_cache, w.qhat_rows, w.row_nnz, (TC*)out,                 \
+                             (const float*)w.qhat[qhat_sel], w.qhat[qhat_sel ^ 1], w.R, w.dec_partial,     \
+                             w.dec_ticket, w.counters, n, s.T_max, s.H, chunk, nsplit, theta, window,      \
+                             scale_log2e);                                                                 \
   } while (0)
   switch (G) {
     case 1: LAUNCH(1); break;
@@ -577,7 +595,7 @@ static cudaError_t launch_tc(const Shape& s, const Workspace& w, const void* q_n
   }
 #undef LAUNCH
   count_launch();
-  return cudaGetLastError();
+  return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 cudaError_t launch_decode_step_tc(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
