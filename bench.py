@@ -527,7 +527,8 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
                          "frac": gbs / float(peaks["hbm_gbs"]),
                          "note": "batch 1 moves ~5 MB per step: launch latency, not bandwidth, sets the time"
-                         if w.B == 1 else ""},
+                         if w.B == 1 else "the step re-reads the same cache every step and 71 MB fit the 126 MB L2: "
+                         "the fraction compares with the HBM copy rate, the data comes largely from L2"},
             "S_m_decode": dstats["decode"]["S_m"], "S_c_exact_decode": dstats["decode"]["S_c_exact"],
             "S_c_exact_combined": dstats["combined"]["S_c_exact"],
         }
