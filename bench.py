@@ -517,10 +517,32 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
         # (and read it, where the step runs on the FP32 pipes: the tensor-core form recomputes it)
         r_passes = 0 if key else (1 if B.delta_state_decode_kernel(st) == 1 else 2)
         bytes_step = w.B * (2 * w.H_kv * n_avg * w.d * es + r_passes * w.H * n_avg * 4)
+        # the same steps with L2 flushed before each one (in a model every layer's cache passes
+        # through L2 between two steps of the same layer, so a step finds its cache in HBM):
+        # device time of each step alone, by events
+        flushed_us = None
+        try:
+            flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+            prefill()
+            evs = []
+            for s in range(min(w.n_decode, 64)):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                B.delta_attn_decode_step(st, qd[s], kd[s], vd[s], kc, vc, od[s], theta, w.window)
+                e1.record()
+                evs.append((e0, e1))
+            torch.cuda.synchronize()
+            flushed_us = statistics.mean(a.elapsed_time(b) * 1e3 for a, b in evs[4:])
+            del flush
+        except Exception as ex:
+            flushed_us = None
         best = graph_us if graph_us else min(eager)
         gbs = bytes_step / (best * 1e-6) / 1e9
+        gbs_flushed = bytes_step / (flushed_us * 1e-6) / 1e9 if flushed_us else None
         res[f"batch{w.B}"] = {
             "us_per_step_eager": statistics.median(eager), "us_per_step_graph": graph_us,
+            "us_per_step_l2_flushed": flushed_us,
             "graph_matches_eager": graph_ok, "steps": w.n_decode,
             "decode_kernel": "tensor-core scores" if B.delta_state_decode_kernel(st) == 1 else "FP32 pipes", "cache_tokens": w.T, "theta": theta,
             "window": w.window, "algorithmic_bytes_per_step": bytes_step,
@@ -529,6 +551,9 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
                          "note": "batch 1 moves ~5 MB per step: launch latency, not bandwidth, sets the time"
                          if w.B == 1 else "the step re-reads the same cache every step and 71 MB fit the 126 MB L2: "
                          "the fraction compares with the HBM copy rate, the data comes largely from L2"},
+            "roofline_l2_flushed": ({"bound": "hbm", "achieved": gbs_flushed, "peak": float(peaks["hbm_gbs"]),
+                                     "unit": "GB/s", "frac": gbs_flushed / float(peaks["hbm_gbs"])}
+                                    if gbs_flushed else None),
             "S_m_decode": dstats["decode"]["S_m"], "S_c_exact_decode": dstats["decode"]["S_c_exact"],
             "S_c_exact_combined": dstats["combined"]["S_c_exact"],
         }
