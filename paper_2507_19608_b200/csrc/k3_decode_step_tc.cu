@@ -13,13 +13,13 @@
 //
 // Grid = (key slices, batch x KV heads); a CTA serves the G query heads of one KV head.
 //   1. threshold q_new against the carried reference, build Qcat in the operand layout;
-//   2. thread 0 streams the slice's key tiles with TMA (128-byte swizzle, two stages) and issues
+//   2. warp 0 streams the slice's key tiles with TMA (128-byte swizzle, five stages) and issues
 //      the products; all score tiles of the slice stay in tensor memory (16 columns per tile);
 //   3. one softmax over the slice: every thread reads its keys' scores (lane = key), hybrid
 //      select, scale, R written; maximum and sum reduced once per slice, not per tile;
-//   4. P.V with the value tiles streamed through a ring of bulk copies (three stages of its own
-//      plus the two key stages once the products are done), the warps releasing stages through
-//      mbarriers (no block-wide barrier per tile);
+//   4. P.V with the value tiles streamed by bulk copies through the same five stages once the
+//      products are done, the warps releasing stages through mbarriers (no block-wide barrier
+//      per tile);
 //   5. the slice result is stored and the last CTA of the (batch, KV head) merges the slices.
 // The key and value that arrive with this step are scored on the FP32 pipes by the CTA that
 // owns their slice (their cache row is written by this very kernel).
@@ -54,9 +54,14 @@ constexpr uint32_t DEC_TMEM_COLS = 256;
 // 30.3, 512 CTAs 29.2, 768 CTAs 31.6 (a CTA's fixed cost outweighs the better balance).
 constexpr int kTcTargetCtas = 296;
 
-constexpr int NVS_OWN = 3;             // value-ring stages of its own
-constexpr int NVS = NVS_OWN + 2;       // plus the two key stages once the score products are done
-enum { BAR_K0 = 0, BAR_K1, BAR_KFREE0, BAR_KFREE1, BAR_S, BAR_V0, BAR_VFREE0 = BAR_V0 + NVS, DEC_NUM_BARS = BAR_VFREE0 + NVS };
+// One ring of five 16 KiB stages serves both streams: all five carry key tiles while the score
+// products run and value tiles afterwards.  Measured at batch 16 (warm L2 / L2 flushed before every
+// step, us per step): 2 key + 3 value stages 19.0 / 30.9, 3 + 2: 18.6 / 29.8, 4 + 1: 18.4 / 29.2,
+// all five shared: 18.3 / 28.8.
+constexpr int NKS = 5;                 // key-ring stages
+constexpr int NVS_OWN = 0;             // value-ring stages of its own
+constexpr int NVS = NVS_OWN + NKS;     // plus the key stages once the score products are done
+enum { BAR_K0 = 0, BAR_KFREE0 = BAR_K0 + NKS, BAR_S = BAR_KFREE0 + NKS, BAR_V0, BAR_VFREE0 = BAR_V0 + NVS, DEC_NUM_BARS = BAR_VFREE0 + NVS };
 
 
 // The G probabilities of one key (contiguous, 16-byte aligned for G >= 4).
@@ -94,7 +99,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled operand tiles want 1 KiB alignment
   unsigned char* sm = dsm_raw0 + (base - raw);
   constexpr uint32_t OFF_K = 0;                          // [2][128][64] bf16, 128-byte swizzle
-  constexpr uint32_t OFF_V = OFF_K + 2 * TILE_BYTES;     // [NVS_OWN][128][64] bf16, plain rows
+  constexpr uint32_t OFF_V = OFF_K + NKS * TILE_BYTES;     // [NVS_OWN][128][64] bf16, plain rows
   constexpr uint32_t OFF_QC = OFF_V + NVS_OWN * TILE_BYTES;  // Qcat [16][64] bf16, 128-byte swizzle
   constexpr uint32_t OFF_F = OFF_QC + 2048;              // floats from here on
   float* q_s = reinterpret_cast<float*>(sm + OFF_F);     // [G][D]
@@ -152,9 +157,9 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   };
 
   auto issue_k = [&](int t) {
-    tc::mbar_expect_tx(DBAR(BAR_K0 + (t & 1)), TILE_BYTES);
+    tc::mbar_expect_tx(DBAR(BAR_K0 + (t % NKS)), TILE_BYTES);
     const CUtensorMap* src = (KEY && tile_kind(t) != 1) ? &tm_h : &tm_k;
-    tc::tma_load_3d(base + OFF_K + (t & 1) * TILE_BYTES, src, DBAR(BAR_K0 + (t & 1)), 0, j0 + t * TK, bkv);
+    tc::tma_load_3d(base + OFF_K + (t % NKS) * TILE_BYTES, src, DBAR(BAR_K0 + (t % NKS)), 0, j0 + t * TK, bkv);
   };
   // the step in front (or the prefill) has written the carried reference, the cache rows and
   // the slice tickets this step reads
@@ -166,7 +171,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     s_fail = 0;
     // the first key and value tiles are on their way while the threshold step below runs
     if (n_tiles > 0) issue_k(0);
-    if (n_tiles > 1) issue_k(1);
+    for (int t = 1; t < NKS && t < n_tiles; ++t) issue_k(t);
     for (int t = 0; t < NVS_OWN && t < n_tiles; ++t) issue_v(t);
   }
 
@@ -262,14 +267,14 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
     const uint32_t IDESC = tc::make_idesc(SCOL, 0);
     const TC* kc = k_cache + (size_t)bkv * T_max * D;
     for (int t = 0; t < n_tiles; ++t) {
-      if (!mbar_wait(DBAR(BAR_K0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
-      const uint32_t kb = base + OFF_K + (t & 1) * TILE_BYTES;
+      if (!mbar_wait(DBAR(BAR_K0 + (t % NKS)), (t / NKS) & 1)) s_fail = 1;
+      const uint32_t kb = base + OFF_K + (t % NKS) * TILE_BYTES;
       if (KEY && tile_kind(t) == 2) {
         // the window's edge falls into this tile: its window rows become the original keys
         const int r0 = wl - (j0 + t * TK), r1 = min(TK, cached - t * TK);
         for (int e = lane; e < (r1 - r0) * 8; e += 32) {
           const int r = r0 + (e >> 3), ch = e & 7;
-          *reinterpret_cast<uint4*>(sm + OFF_K + (t & 1) * TILE_BYTES + (uint32_t)r * 128u +
+          *reinterpret_cast<uint4*>(sm + OFF_K + (t % NKS) * TILE_BYTES + (uint32_t)r * 128u +
                                     (((uint32_t)ch ^ ((uint32_t)r & 7u)) << 4)) =
               *reinterpret_cast<const uint4*>(kc + (size_t)(j0 + t * TK + r) * D + ch * 8);
         }
@@ -282,11 +287,11 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
         for (int ks = 0; ks < D / 16; ++ks)
           tc::tc_mma(tmem + SCOL * t, tc::make_desc(kb + ks * 32, 16, 1024),
                      tc::make_desc(base + OFF_QC + ks * 32, 16, 1024), IDESC, ks > 0 ? 1u : 0u);
-        if (t + 2 < n_tiles) {
+        if (t + NKS < n_tiles) {
           // the stage is free once these products are done: then refill it
-          tc::tc_commit(DBAR(BAR_KFREE0 + (t & 1)));
-          if (!mbar_wait(DBAR(BAR_KFREE0 + (t & 1)), (t >> 1) & 1)) s_fail = 1;
-          issue_k(t + 2);
+          tc::tc_commit(DBAR(BAR_KFREE0 + (t % NKS)));
+          if (!mbar_wait(DBAR(BAR_KFREE0 + (t % NKS)), (t / NKS) & 1)) s_fail = 1;
+          issue_k(t + NKS);
         }
       }
       __syncwarp();
@@ -557,7 +562,7 @@ static cudaError_t launch_tc(const Shape& s, const Workspace& w, const void* q_n
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   const int G = s.g();
   const dim3 grid(nsplit, bkv);
-  const size_t smem = 1024 + (size_t)(2 + NVS_OWN) * TILE_BYTES + 2048 +
+  const size_t smem = 1024 + (size_t)(NKS + NVS_OWN) * TILE_BYTES + 2048 +
                       ((size_t)2 * G * TCD + (size_t)G * kMaxDecodeSplits + (size_t)(MAXT * TK + 1) * G + 24) * 4;
   cudaError_t err = cudaSuccess;
   using TC = __nv_bfloat16;
