@@ -520,29 +520,40 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
         # the same steps with L2 flushed before each one (in a model every layer's cache passes
         # through L2 between two steps of the same layer, so a step finds its cache in HBM):
         # device time of each step alone, by events
-        flushed_us = None
+        # two ways of emptying L2: overwriting a 256 MiB buffer leaves L2 full of dirty lines, whose
+        # write-back then shares HBM with the step's reads; reading the buffer leaves clean lines
+        # (what a preceding weight-streaming GEMM leaves behind)
+        flushed_us = flushed_read_us = None
         try:
             flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
-            prefill()
-            evs = []
-            for s in range(min(w.n_decode, 64)):
-                flush.zero_()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                B.delta_attn_decode_step(st, qd[s], kd[s], vd[s], kc, vc, od[s], theta, w.window)
-                e1.record()
-                evs.append((e0, e1))
-            torch.cuda.synchronize()
-            flushed_us = statistics.mean(a.elapsed_time(b) * 1e3 for a, b in evs[4:])
-            del flush
+            flush.zero_()
+            flush64 = flush.view(torch.int64)
+            sink = torch.zeros((), dtype=torch.int64, device="cuda")
+
+            def flushed(evict):
+                prefill()
+                evs = []
+                for s in range(min(w.n_decode, 64)):
+                    evict()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    B.delta_attn_decode_step(st, qd[s], kd[s], vd[s], kc, vc, od[s], theta, w.window)
+                    e1.record()
+                    evs.append((e0, e1))
+                torch.cuda.synchronize()
+                return statistics.mean(a.elapsed_time(b) * 1e3 for a, b in evs[4:])
+
+            flushed_us = flushed(lambda: flush.zero_())
+            flushed_read_us = flushed(lambda: sink.copy_(flush64.sum()))
+            del flush, flush64, sink
         except Exception as ex:
-            flushed_us = None
+            pass
         best = graph_us if graph_us else min(eager)
         gbs = bytes_step / (best * 1e-6) / 1e9
         gbs_flushed = bytes_step / (flushed_us * 1e-6) / 1e9 if flushed_us else None
         res[f"batch{w.B}"] = {
             "us_per_step_eager": statistics.median(eager), "us_per_step_graph": graph_us,
-            "us_per_step_l2_flushed": flushed_us,
+            "us_per_step_l2_flushed": flushed_us, "us_per_step_l2_flushed_by_read": flushed_read_us,
             "graph_matches_eager": graph_ok, "steps": w.n_decode,
             "decode_kernel": "tensor-core scores" if B.delta_state_decode_kernel(st) == 1 else "FP32 pipes", "cache_tokens": w.T, "theta": theta,
             "window": w.window, "algorithmic_bytes_per_step": bytes_step,
