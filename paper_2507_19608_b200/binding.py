@@ -157,7 +157,7 @@ class DeltaState:
 
     def __del__(self):
         h, self.handle = getattr(self, "handle", None), None
-        if h:
+        if h and lib is not None:      # module globals are gone while the interpreter shuts down
             lib.delta_state_destroy(h)
 
 
