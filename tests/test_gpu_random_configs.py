@@ -113,9 +113,9 @@ def _run(B, c):
 
 
 @pytest.mark.parametrize("mode,large,count,seed", [
-    ("query", False, 60, 11), ("query", True, 12, 12),
-    ("key", False, 40, 21), ("key", True, 10, 22),
-    ("bottom_up", False, 40, 31), ("bottom_up", True, 10, 32),
+    ("query", False, 200, 11), ("query", True, 40, 12),
+    ("key", False, 120, 21), ("key", True, 30, 22),
+    ("bottom_up", False, 120, 31), ("bottom_up", True, 30, 32),
 ])
 def test_random_configurations_match_oracle(B, mode, large, count, seed):
     rng = np.random.default_rng(seed)
