@@ -338,10 +338,16 @@ delta_status_t delta_attn_prefill_host(delta_state_t* st, const void* q_host, co
   if ((e = cudaMemcpyAsync(dq_, q_host, q_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
   // host K/V hold T rows per head; the device copy uses the cache layout with T_max rows
   const size_t row = (size_t)c.d * es;
-  if ((e = cudaMemcpy2DAsync(dk, (size_t)c.T_max * row, k_host, (size_t)T * row, (size_t)T * row,
-                             (size_t)c.B * c.H_kv, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaMemcpy2DAsync(dv, (size_t)c.T_max * row, v_host, (size_t)T * row, (size_t)T * row,
-                             (size_t)c.B * c.H_kv, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
+  const size_t units = (size_t)c.B * c.H_kv;
+  if (T == c.T_max) {      // the two layouts coincide: one contiguous copy each
+    if ((e = cudaMemcpyAsync(dk, k_host, units * T * row, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(dv, v_host, units * T * row, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
+  } else {
+    if ((e = cudaMemcpy2DAsync(dk, (size_t)c.T_max * row, k_host, (size_t)T * row, (size_t)T * row, units,
+                               cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpy2DAsync(dv, (size_t)c.T_max * row, v_host, (size_t)T * row, (size_t)T * row, units,
+                               cudaMemcpyHostToDevice, cs)) != cudaSuccess) return cuda_fail(e);
+  }
   s = delta_attn_prefill(st, dq_, dk, dv, dout, T, c.H, c.H_kv, c.d, theta, window, stream);
   if (s != DELTA_OK) return s;
   if ((e = cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, cs)) != cudaSuccess) return cuda_fail(e);

@@ -223,12 +223,13 @@ def test_theta0_full_window_equals_dense_attention(B):
     assert np.abs(to_host_f64(out) - ref).max() <= FP32_ATOL
 
 
-def test_prefill_host_entry_matches_device_entry(B):
+@pytest.mark.parametrize("T_max", [160, 150], ids=["cache_longer_than_prompt", "cache_full"])
+def test_prefill_host_entry_matches_device_entry(B, T_max):
     from tests.gpu_helpers import run_prefill
     Bn, H, Hk, T, d, dtype = 1, 4, 2, 150, 64, "bf16"
     q, k, v = _inputs(Bn, H, Hk, T, d, dtype, seed=9)
-    st, out, _, _ = run_prefill(B, q, k, v, 0.2, 32, dtype, T_max=160)
-    cfg = B.make_config(Bn, H, Hk, d, 160, dtype)
+    st, out, _, _ = run_prefill(B, q, k, v, 0.2, 32, dtype, T_max=T_max)
+    cfg = B.make_config(Bn, H, Hk, d, T_max, dtype)
     st2 = B.delta_state_init(cfg)
     staging = torch.empty(B.delta_prefill_staging_bytes(cfg, T), dtype=torch.uint8, device="cuda")
     hq = torch.from_numpy(WL.bf16_bits(q).view(np.int16)).pin_memory()
