@@ -643,3 +643,66 @@ def test_eq5_dynamic_window_prefill_and_decode(B, n, gamma):
     assert (got["nnz"], got["macs_done"], got["macs_dense"]) == (want["nnz"], want["macs_done"], want["macs_dense"])
     assert abs(got["S_c_eq6"] - want["S_c_eq6"]) < 1e-6 and abs(got["S_c_exact"] - want["S_c_exact"]) < 1e-9
     assert stats["device_status"] == 0
+
+
+# ------------------------------------------------------------------ streams
+def test_two_states_on_two_streams_match_the_default_stream(B):
+    """The library works on the stream it is given: two independent states, each driven on a
+    stream of its own with their calls interleaved, give bit for bit what one state gives on
+    the default stream (outputs, cache rows, reference state, counters)."""
+    from tests.gpu_helpers import to_cache, to_dev
+    Bn, H, Hk, T, d, dtype, theta, W, steps = 2, 8, 2, 700, 64, "bf16", 0.2, 64, 4
+    sets = []
+    for seed in (41, 42):
+        w = WL.Workload("t", Bn, H, Hk, T, d, dtype, 0.95, 0.5, W, (), seed, n_decode=steps)
+        sets.append(WL.make_qkv(w))
+
+    def run(t, stream_ctx, other=None):
+        """Generator: yields after every call so that two runs can be interleaved."""
+        with stream_ctx():
+            cfg = B.make_config(Bn, H, Hk, d, T + steps, dtype, prefill_window=B.DELTA_WIN_SLIDING)
+            st = B.delta_state_init(cfg)
+            dq_, kc, vc = to_dev(t["q"], dtype), to_cache(t["k"], T + steps, dtype), to_cache(t["v"], T + steps, dtype)
+            out = torch.full_like(dq_, float("nan"))
+            outs = []
+        yield
+        with stream_ctx():
+            B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, theta, W)
+        yield
+        for s in range(steps):
+            with stream_ctx():
+                dqn, dkn, dvn = (to_dev(t[n][:, :, s], dtype) for n in ("q_dec", "k_dec", "v_dec"))
+                o = torch.full_like(dqn, float("nan"))
+                B.delta_attn_decode_step(st, dqn, dkn, dvn, kc, vc, o, theta, W)
+                outs.append(o)
+            yield
+        with stream_ctx():
+            stats = B.delta_sparsity_stats(st)
+            qh = B.delta_state_view(st, B.DELTA_VIEW_QHAT).clone()
+        torch.cuda.synchronize()
+        res.append((out, outs, kc, vc, qh, stats))
+        yield
+
+    import contextlib
+    res = []
+    for t in sets:                                  # one after the other on the default stream
+        for _ in run(t, contextlib.nullcontext):
+            pass
+    want = list(res)
+    res.clear()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    g1 = run(sets[0], lambda: torch.cuda.stream(s1))
+    g2 = run(sets[1], lambda: torch.cuda.stream(s2))
+    for _ in zip(g1, g2):                           # interleaved, each on its own stream
+        pass
+    torch.cuda.synchronize()
+    assert len(res) == 2
+    for got, ref in zip(res, want):
+        assert torch.equal(got[0], ref[0])
+        for a, b in zip(got[1], ref[1]):
+            assert torch.equal(a, b)
+        assert torch.equal(got[2][:, :, :T + steps], ref[2][:, :, :T + steps])
+        assert torch.equal(got[3][:, :, :T + steps], ref[3][:, :, :T + steps])
+        assert torch.equal(got[4], ref[4])
+        assert got[5] == ref[5] and got[5]["device_status"] == 0
