@@ -706,3 +706,59 @@ def test_two_states_on_two_streams_match_the_default_stream(B):
         assert torch.equal(got[3][:, :, :T + steps], ref[3][:, :, :T + steps])
         assert torch.equal(got[4], ref[4])
         assert got[5] == ref[5] and got[5]["device_status"] == 0
+
+
+# ------------------------------------------------------------------ long decode runs
+@pytest.mark.parametrize("source", ["query", "key"])
+@pytest.mark.parametrize("decode_kernel", [0, 1], ids=["fp32_pipes", "tc_scores"])
+def test_long_decode_run_crosses_tile_and_slice_boundaries(B, source, decode_kernel):
+    """300 decode steps from a 100-token prompt: the cache grows across three 128-key tile
+    boundaries and the number of key slices per head changes on the way; every step's output is
+    held to the oracle's, the carried reference state bit for bit."""
+    from tests.gpu_helpers import to_cache, to_dev, to_host_f64
+    Bn, H, Hk, T, d, dtype, theta, W, W_d, steps = 1, 4, 2, 100, 64, "bf16", 0.2, 32, 4, 300
+    g = H // Hk
+    w = WL.Workload("t", Bn, H, Hk, T, d, dtype, 0.95, 0.5, W, (), 900, n_decode=steps)
+    t = WL.make_qkv(w)
+    T_max = T + steps
+    cfg = B.make_config(Bn, H, Hk, d, T_max, dtype, prefill_window=B.DELTA_WIN_SLIDING,
+                        source=B.DELTA_SRC_KEY if source == "key" else B.DELTA_SRC_QUERY)
+    st = B.delta_state_init(cfg)
+    B.delta_state_set_decode_kernel(st, decode_kernel)
+    dq_, kc, vc = to_dev(t["q"], dtype), to_cache(t["k"], T_max, dtype), to_cache(t["v"], T_max, dtype)
+    out = torch.full_like(dq_, float("nan"))
+    B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, theta, W)
+    ref, heads = O.prefill_mha(t["q"], t["k"], t["v"], theta, W, "sliding", source=source)
+    if source == "key":
+        states = {(b, kvh): heads[(b, kvh * g)]["state"] for b in range(Bn) for kvh in range(Hk)}
+    else:
+        states = {key: r["state"] for key, r in heads.items()}
+    qd, kd, vd = (to_dev(np.ascontiguousarray(t[n].transpose(2, 0, 1, 3)), dtype) for n in ("q_dec", "k_dec", "v_dec"))
+    od = torch.full_like(qd, float("nan"))
+    for s in range(steps):
+        B.delta_attn_decode_step(st, qd[s], kd[s], vd[s], kc, vc, od[s], theta, W_d)
+    torch.cuda.synchronize()
+    got = to_host_f64(od)
+    for s in range(steps):
+        qn, kn, vn = t["q_dec"][:, :, s], t["k_dec"][:, :, s], t["v_dec"][:, :, s]
+        if source == "key":
+            oref, _ = O.decode_mha_key(states, qn, kn, vn, theta, W_d)
+        else:
+            oref, _ = O.decode_mha(states, qn, kn, vn, theta, W_d)
+        _check_out(got[s], oref, dtype, f"decode step {s}")
+    assert B.delta_state_position(st) == T_max
+    ref_state = B.delta_state_view(st, B.DELTA_VIEW_QHAT).cpu().numpy()
+    if source == "key":
+        kh = ref_state.reshape(Bn * H, d)
+        for (b, kvh), stt in states.items():
+            assert np.array_equal(kh[b * Hk + kvh].view(np.uint32), stt["khat"].view(np.uint32))
+    else:
+        R = B.delta_state_view(st, B.DELTA_VIEW_R).cpu().numpy()
+        for (b, h), stt in states.items():
+            assert np.array_equal(ref_state[b, h].view(np.uint32), stt["qhat"].view(np.uint32))
+            assert np.abs(R[b, h, :T_max] - stt["R"]).max() <= 1e-3 * max(1.0, np.abs(stt["R"]).max())
+    assert B.delta_sparsity_stats(st)["device_status"] == 0
+    # the cache is full now
+    with pytest.raises(B.DeltaError) as e:
+        B.delta_attn_decode_step(st, qd[0], kd[0], vd[0], kc, vc, od[0], theta, W_d)
+    assert e.value.status == B.DELTA_ERR_CAPACITY
