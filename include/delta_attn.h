@@ -15,8 +15,11 @@
  *     caller owns; the library never allocates or frees device memory;
  *   - `stream` is a cudaStream_t passed as void*; calls only enqueue work on it and return
  *     (delta_sparsity_stats and the *_host entry point synchronise it);
- *   - every function returns a delta_status_t; on any error nothing is launched and the state
- *     is left as it was;
+ *   - every function returns a delta_status_t; an argument, capacity or call-order error is
+ *     found before anything is launched and leaves the state as it was.  DELTA_ERR_CUDA (a
+ *     launch or copy the runtime refused) can come after earlier kernels of the same call were
+ *     enqueued: the state's position is left unchanged, but workspace and output buffers may
+ *     be partly written, so reset the state before using it again;
  *   - tensors are contiguous, row-major, element type from delta_config_t.dtype
  *     (DELTA_F32: float, DELTA_BF16: bfloat16 bit patterns);
  *   - query head h reads KV head h / (H / H_kv).
@@ -154,7 +157,9 @@ DELTA_API delta_status_t delta_attn_prefill_host(delta_state_t* st, const void* 
  * Eq. 4's sum telescopes to R[j] = q_hat . k_j (exactly, up to the order of the fp32
  * additions, for bf16 inputs, whose references are copies of input elements); where
  * delta_state_decode_kernel reports 1 the step computes R[j] in that form on the tensor cores
- * and writes it back without reading it.  k_cache must then be 16-byte aligned.
+ * and writes it back without reading it.
+ * All six tensor pointers must be 16-byte aligned (the kernels stage cache tiles with bulk
+ * copies and read rows as 16-byte vectors): DELTA_ERR_INVALID_ARG otherwise, nothing launched.
  * With DELTA_SRC_KEY the step thresholds k_new against the carried reference key instead
  * (Eq. 2-3), appends the reference-key row k_hat(n), and scores key j with q_new.k_j if
  * n - j < window else q_new.k_hat(j). */
@@ -192,11 +197,22 @@ DELTA_API delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q
  * current); make that first call outside of any stream capture.  Every call shares the one
  * array and finds in it what the previous call left: the parts that must start at zero are
  * cleared on `stream` at the start of the call.  Calls whose kernels may overlap on one GPU
- * (different streams or threads) race on the array: serialise them. */
+ * (different streams or threads) race on the array: serialise them.
+ * All nine pointers must be 16-byte aligned (DELTA_ERR_INVALID_ARG otherwise).
+ * The call itself never returns DELTA_ERR_TIMEOUT: a bounded device-side wait that ran out
+ * leaves its mark in a status word inside the scratch array, which stays set across later
+ * calls until delta_noalloc_device_status reads it. */
 DELTA_API delta_status_t delta_attn_decode_step_noalloc(
     const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* out,
     const float* qhat_in, float* qhat_out, float* R, int32_t n, int32_t B, int32_t H, int32_t H_kv,
     int32_t d, int32_t T_max, delta_dtype_t dtype, float theta, int32_t window, void* stream);
+
+/* delta_noalloc_device_status -- the device status word of delta_attn_decode_step_noalloc on the
+ * current device (the paper has no counterpart): copies it to *host_status (HOST pointer),
+ * clears it and synchronises `stream`.  0 means every no-alloc step enqueued on `stream` so far
+ * ran to its end; DELTA_ERR_TIMEOUT means one of them gave up a bounded wait and its outputs
+ * are not valid.  The return value is DELTA_OK or that status.  Allocates nothing. */
+DELTA_API delta_status_t delta_noalloc_device_status(uint32_t* host_status, void* stream);
 
 /* Counters of one stage.  S_m = 1 - nnz/elements (sparsity of the delta matrix, Eq. 6);
  * S_c_eq6 = S_m * (1 - W/n) (Eq. 6); S_c_exact = 1 - macs_done/macs_dense where a causal

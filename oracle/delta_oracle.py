@@ -15,10 +15,10 @@ Delta a(t) delta vector, theta threshold (Eq. 2-3); R(t) recursive product
 Readings of points the paper leaves open (each one is a named argument so the
 tests can exercise the alternatives):
   * init="basis_exact": row 0 is the un-thresholded basis vector, Delta a(0) =
-    a(0) and a_hat(0) = a(0) ("stacking the basis vector a(0) with these delta
-    vectors", Section II-C; "dense first row", Section III-A strategy 1).
-    init="zero_state": a_hat(-1) = 0 and Eq. 2-3 are applied at t = 0 as well
-    (the literal "a_hat(0) is initialized to 0" sentence).
+    a(0) and a_hat(0) = a(0) (the delta matrix of Section II-C has the basis
+    vector as its first row; strategy 1 of Section III-A keeps the first
+    attention row dense).  init="zero_state": the reference starts at zero, as
+    the sentence after Eq. 3 has it, and Eq. 2-3 are applied at t = 0 as well.
   * the threshold is per element; |diff| == theta does not fire (Eq. 2 uses >).
   * window shape "block": squares of side W along the diagonal anchored at
     token 0 (Section III-B, prefill); "sliding": the most recent W tokens
@@ -339,6 +339,26 @@ def finish_stats(c, win_sum, len_sum):
 def prefill_stats(row_nnz, T, d, W, shape):
     c = stage_stats(row_nnz, list(range(T)), d, W, shape)
     return finish_stats(c, min(W, T), T)
+
+
+def decode_stage_stats(counters, windows, lengths):
+    """Decode stage of Eq. 6: the stage is a run of steps, step s attends lengths[s] keys (the
+    new one included) with window windows[s]; Eq. 6's W/n becomes sum(min(W_s, n_s)) / sum(n_s)
+    over the steps.  counters: the summed raw counters of the steps."""
+    win_sum = sum(min(int(w), int(n)) for w, n in zip(windows, lengths))
+    return finish_stats(counters, win_sum, sum(int(n) for n in lengths))
+
+
+def combined_stats(prefill, decode):
+    """Prefill and decode taken together (the paper's "both stages" figure): the raw counters add,
+    S_m and the exact multiply-add sparsity follow from the sums, and the Eq. 6 value is the mean
+    of the two stages' Eq. 6 values weighted by their dense multiply-adds."""
+    c = {key: prefill[key] + decode[key] for key in ("nnz", "elements", "macs_done", "macs_dense")}
+    out = finish_stats(c, 0, 0)
+    dense = c["macs_dense"]
+    out["S_c_eq6"] = ((prefill["S_c_eq6"] * prefill["macs_dense"] + decode["S_c_eq6"] * decode["macs_dense"]) / dense
+                      if dense else 0.0)
+    return out
 
 
 # --------------------------------------------------------------------------- multi-head wrappers

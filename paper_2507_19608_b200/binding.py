@@ -34,7 +34,7 @@ EXPORTED = [
     "delta_state_set_prefill_kernel",
     "delta_launch_count", "delta_status_string", "delta_last_cuda_error",
     "delta_state_enable_profiling", "delta_state_prefill_kernel_ms",
-    "delta_attn_decode_step_noalloc",
+    "delta_attn_decode_step_noalloc", "delta_noalloc_device_status",
 ]
 
 
@@ -97,6 +97,7 @@ def _load() -> C.CDLL:
         "delta_state_prefill_kernel_ms": (C.c_int, [vp, C.POINTER(C.c_float)]),
         "delta_attn_decode_step_noalloc": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32,
                                                      i32, i32, C.c_int, f32, i32, vp]),
+        "delta_noalloc_device_status": (C.c_int, [C.POINTER(C.c_uint32), vp]),
         "delta_launch_count": (C.c_uint64, []),
         "delta_status_string": (C.c_char_p, [C.c_int]),
         "delta_last_cuda_error": (C.c_char_p, []),
@@ -211,6 +212,13 @@ def delta_attn_decode_step_noalloc(q_new, k_new, v_new, k_cache, v_cache, out, q
                                               _ptr(v_cache), _ptr(out), _ptr(qhat_in), _ptr(qhat_out),
                                               _ptr(R), n, B, H, H_kv, d, T_max, dt, theta, window,
                                               _stream(stream)), "delta_attn_decode_step_noalloc")
+
+
+def delta_noalloc_device_status(stream=None) -> int:
+    """Reads and clears the status word of the no-alloc decode step on the current device."""
+    v = C.c_uint32(0)
+    lib.delta_noalloc_device_status(C.byref(v), _stream(stream))
+    return v.value
 
 
 def delta_sparsity_stats(st: DeltaState, stream=None) -> dict:

@@ -12,7 +12,7 @@ namespace delta {
 static std::atomic<unsigned long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 static thread_local char g_cuda_err[256] = "";
-static delta_status_t cuda_fail(cudaError_t e) {
+delta_status_t cuda_fail(cudaError_t e) {
   snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
   return DELTA_ERR_CUDA;
 }
@@ -359,6 +359,10 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
                                       const void* v_new, void* k_cache, void* v_cache, void* out,
                                       float theta, int32_t window, void* stream) {
   if (!st || !q_new || !k_new || !v_new || !k_cache || !v_cache || !out) return DELTA_ERR_INVALID_ARG;
+  // every decode kernel stages cache tiles with bulk copies and reads rows as 16-byte vectors
+  if ((((uintptr_t)q_new | (uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache |
+        (uintptr_t)out) & 15u) != 0)
+    return DELTA_ERR_INVALID_ARG;
   delta_status_t s = check_theta_window(theta, window);
   if (s != DELTA_OK) return s;
   if (st->cfg.source == DELTA_SRC_QUERY_BOTTOM_UP) return DELTA_ERR_UNSUPPORTED;   // strategy (2) has no decode

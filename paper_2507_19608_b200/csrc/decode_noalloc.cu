@@ -64,6 +64,10 @@ extern "C" delta_status_t delta_attn_decode_step_noalloc(
   if (!q_new || !k_new || !v_new || !k_cache || !v_cache || !out || !qhat_in || !qhat_out || !R)
     return DELTA_ERR_INVALID_ARG;
   if (qhat_in == qhat_out) return DELTA_ERR_INVALID_ARG;   // other CTAs still read the old reference
+  // cache tiles are staged with bulk copies and rows are read as 16-byte vectors
+  if ((((uintptr_t)q_new | (uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache |
+        (uintptr_t)out | (uintptr_t)qhat_in | (uintptr_t)qhat_out | (uintptr_t)R) & 15u) != 0)
+    return DELTA_ERR_INVALID_ARG;
   if (B < 1 || H < 1 || H_kv < 1 || T_max < 1 || H % H_kv != 0) return DELTA_ERR_INVALID_ARG;
   if (dtype != DELTA_F32 && dtype != DELTA_BF16) return DELTA_ERR_INVALID_ARG;
   if (!(theta >= 0.0f) || !(theta <= 3.0e38f) || window < 0) return DELTA_ERR_INVALID_ARG;
@@ -81,11 +85,13 @@ extern "C" delta_status_t delta_attn_decode_step_noalloc(
 
   unsigned char* base = nullptr;
   cudaError_t e = scratch_on_current_device(&base);
-  if (e != cudaSuccess) return DELTA_ERR_CUDA;
+  if (e != cudaSuccess) return cuda_fail(e);
   cudaStream_t cs = (cudaStream_t)stream;
-  // tickets and counters must start at zero; the partial results are fully rewritten
-  if ((e = cudaMemsetAsync(base, 0, kTicketBytes + kCounterBytes, cs)) != cudaSuccess)
-    return DELTA_ERR_CUDA;
+  // tickets and the counters in front of the status word must start at zero; the partial
+  // results are fully rewritten.  The status word (counter slot CNT_STATUS) is left alone: a
+  // time-out recorded by an earlier step stays there until delta_noalloc_device_status reads it.
+  if ((e = cudaMemsetAsync(base, 0, kTicketBytes + CNT_STATUS * sizeof(unsigned long long), cs)) != cudaSuccess)
+    return cuda_fail(e);
 
   Workspace w{};
   w.qhat[0] = const_cast<float*>(qhat_in);
@@ -97,5 +103,20 @@ extern "C" delta_status_t delta_attn_decode_step_noalloc(
   const Shape s{B, H, H_kv, d, T_max, (T_max + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS};
   e = launch_decode_step(s, w, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window,
                          (int)dtype, /*qhat_sel=*/0, cs);
-  return e == cudaSuccess ? DELTA_OK : DELTA_ERR_CUDA;
+  return e == cudaSuccess ? DELTA_OK : cuda_fail(e);
+}
+
+extern "C" delta_status_t delta_noalloc_device_status(uint32_t* host_status, void* stream) {
+  if (!host_status) return DELTA_ERR_INVALID_ARG;
+  unsigned char* base = nullptr;
+  cudaError_t e = scratch_on_current_device(&base);
+  if (e != cudaSuccess) return cuda_fail(e);
+  cudaStream_t cs = (cudaStream_t)stream;
+  unsigned long long* word = reinterpret_cast<unsigned long long*>(base + kTicketBytes) + CNT_STATUS;
+  unsigned long long v = 0;
+  if ((e = cudaMemcpyAsync(&v, word, sizeof(v), cudaMemcpyDeviceToHost, cs)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemsetAsync(word, 0, sizeof(v), cs)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaStreamSynchronize(cs)) != cudaSuccess) return cuda_fail(e);
+  *host_status = (uint32_t)v;
+  return v == 0 ? DELTA_OK : (delta_status_t)(uint32_t)v;
 }

@@ -50,6 +50,8 @@ struct Shape {
 };
 
 void count_launch(int n = 1);
+// Records the text of a failed CUDA runtime call for delta_last_cuda_error; returns DELTA_ERR_CUDA.
+delta_status_t cuda_fail(cudaError_t e);
 
 // K1a: token-sequential delta chain (Eq. 2-3): the reference in front of every 8-row block and
 // every 64-row tile, and the final reference.

@@ -20,6 +20,7 @@
 // hand-off row R(T-1)[j] = q_hat(T-1).k_j for decode and, for the tensor-core attention kernel
 // with the FP32 delta path, the channel-major fp32 copy of the keys.
 #include "delta_internal.cuh"
+#include "mbar.cuh"
 
 namespace delta {
 
@@ -27,32 +28,6 @@ namespace {
 
 constexpr int RC = 64;       // rows per ring stage (= one 64-row tile)
 constexpr int NS = 4;        // ring stages
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait (about a second of SM clock); false if it ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > 2000000000ll) return false;
-  }
-  return true;
-}
-
-
 
 // One element of the staged rows by shared-memory address, widened to fp32.
 template <typename TIn> __device__ __forceinline__ float lds_elem(uint32_t addr);

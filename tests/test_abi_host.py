@@ -75,6 +75,15 @@ def test_null_and_misaligned_arguments_are_rejected_before_any_device_work():
     assert B.lib.delta_attn_prefill(None, 1, 1, 1, 1, 8, 8, 2, 64, 0.1, 4, None) == B.DELTA_ERR_INVALID_ARG
     assert B.lib.delta_attn_decode_step(None, 1, 1, 1, 1, 1, 1, 0.1, 4, None) == B.DELTA_ERR_INVALID_ARG
     assert B.lib.delta_sparsity_stats(None, None, None) == B.DELTA_ERR_INVALID_ARG
+    # decode pointers off the 16-byte grid: rejected on the host (the argument check comes before
+    # anything looks at the state, so a dummy handle is enough here and nothing is launched)
+    ok = 0x1000
+    for bad in range(6):
+        ptrs = [ok + (4 if i == bad else 0) for i in range(6)]
+        assert B.lib.delta_attn_decode_step(0x10, *ptrs, 0.1, 4, None) == B.DELTA_ERR_INVALID_ARG
+        assert B.lib.delta_attn_decode_step_noalloc(*ptrs, ok, ok + 64, ok, 10, 1, 8, 2, 64, 128, B.DELTA_BF16,
+                                                    0.1, 4, None) == B.DELTA_ERR_INVALID_ARG
+    assert B.lib.delta_noalloc_device_status(None, None) == B.DELTA_ERR_INVALID_ARG
     assert B.lib.delta_state_position(None) == -1
 
 

@@ -1,8 +1,9 @@
 """GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
 
 Bars: masks, counts, indices, delta values and reference states are bit-exact; attention
-outputs agree within max-abs 1e-4 for fp32 inputs and within 2e-2 relative (to the largest
-reference magnitude of the tensor; the normalised RMS error is held to 5e-3 as well) for bf16.
+outputs agree within max-abs 1e-4 for fp32 inputs and within 2e-2 relative for bf16 (per output
+row: its largest error against its own largest reference magnitude; the normalised RMS error of
+the whole tensor is held to 5e-3 as well).
 """
 import numpy as np
 import pytest
@@ -36,8 +37,11 @@ def _check_out(gpu, ref, dtype, what=""):
     if dtype == "f32":
         assert err.max() <= FP32_ATOL, f"{what}: max abs err {err.max():.3e}"
     else:
-        scale = np.abs(ref).max()
-        assert err.max() <= BF16_REL * scale, f"{what}: rel err {err.max() / scale:.3e}"
+        # relative 2e-2, taken row by row: the largest error of an output row against the largest
+        # reference magnitude of that same row (a small row cannot hide behind a large one)
+        row_scale = np.abs(ref).max(axis=-1, keepdims=True)
+        rel = err.max(axis=-1, keepdims=True) / np.maximum(row_scale, 1e-30)
+        assert rel.max() <= BF16_REL, f"{what}: worst row rel err {rel.max():.3e}"
         nrms = np.sqrt(np.mean(err ** 2)) / np.sqrt(np.mean(ref ** 2))
         assert nrms <= BF16_NRMS, f"{what}: nrms {nrms:.3e}"
     assert np.isfinite(gpu).all()
@@ -287,8 +291,21 @@ def test_decode_steps_match_oracle(B, Bn, H, Hk, T, d, dtype, theta, W, steps, d
             assert np.array_equal(qh[b, h].view(np.uint32), stt["qhat"].view(np.uint32))
             c = O.stage_stats([infos[(b, h)]["row_nnz"]], [n], d, W, "sliding")
             nnz += c["nnz"]; done += c["macs_done"]; dense += c["macs_dense"]
-    sd = B.delta_sparsity_stats(st)["decode"]
+    stats = B.delta_sparsity_stats(st)
+    sd = stats["decode"]
     assert (sd["nnz"], sd["elements"], sd["macs_done"], sd["macs_dense"]) == (nnz, Bn * H * d * steps, done, dense)
+    # Eq. 6 per stage and over both stages against the oracle's aggregates
+    want_dec = O.decode_stage_stats(dict(nnz=nnz, elements=Bn * H * d * steps, macs_done=done, macs_dense=dense),
+                                    [W] * steps, [T + s + 1 for s in range(steps)])
+    pre = [O.prefill_stats(r["delta"]["row_nnz"], T, d, W, "sliding") for r in heads.values()]
+    want_pre = O.finish_stats({key: sum(c[key] for c in pre) for key in ("nnz", "elements", "macs_done", "macs_dense")},
+                              min(W, T), T)
+    want_all = O.combined_stats(want_pre, want_dec)
+    for name, want in (("prefill", want_pre), ("decode", want_dec), ("combined", want_all)):
+        for key in ("nnz", "elements", "macs_done", "macs_dense"):
+            assert stats[name][key] == want[key], (name, key)
+        for key in ("S_m", "S_c_eq6", "S_c_exact"):
+            assert stats[name][key] == pytest.approx(want[key], abs=1e-12), (name, key)
 
 
 # ------------------------------------------------------------------ call-order and capacity errors

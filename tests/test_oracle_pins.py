@@ -461,3 +461,99 @@ def test_key_delta_decode_continues_prefill(W):
         assert np.allclose(out, full["out"][T + s], rtol=1e-12, atol=1e-12)
         assert np.array_equal(info["dk"], full["delta"]["dq"][T + s])
     assert np.array_equal(st["khat"], full["delta"]["ahat"])
+
+
+# ------------------------------------------------------------------ key-delta counters, non-uniform counts
+@pytest.mark.parametrize("shape,W,g", [("block", 5, 1), ("block", 8, 4), ("sliding", 3, 2), ("sliding", 7, 1)])
+def test_key_delta_counters_recounted_with_uneven_rows(shape, W, g):
+    """stage_stats_key against a recount written out here: the cost of an out-of-window pair
+    (i, j) is the fired count of KEY row j (its column), not of the query row i.  The fired
+    counts differ from row to row, so taking the wrong index changes the total."""
+    T, d = 23, 32
+    k = np.cumsum(0.25 * np.random.default_rng(17).standard_normal((T, d)), axis=0).astype(np.float32)
+    dl = O.delta_construct(k, 0.35)
+    rn = dl["row_nnz"].astype(int)
+    assert len(set(rn.tolist())) > 5                      # really uneven
+    done = dense = 0
+    for i in range(T):                                    # query row
+        for j in range(i + 1):                            # key column
+            inside = W > 0 and ((i // W == j // W) if shape == "block" else (i - j < W))
+            nz_key_j = d if j == 0 else int(np.count_nonzero(dl["dq"][j]))
+            done += d if inside else nz_key_j
+            dense += d
+    got = O.stage_stats_key(dl["row_nnz"], T, d, W, shape, g)
+    assert got["macs_done"] == g * done and got["macs_dense"] == g * dense
+    assert got["nnz"] == int(rn.sum()) and got["elements"] == T * d
+    # the transposed reading (query row's count) gives another total on this input
+    wrong = sum((d if (W > 0 and ((i // W == j // W) if shape == "block" else (i - j < W))) else rn[i])
+                for i in range(T) for j in range(i + 1))
+    assert wrong != done
+
+
+# ------------------------------------------------------------------ GQA mapping of the decode wrappers
+def _sdpa_last_row_gqa(q_new, k_all, v_all):
+    """fp64 attention of one new query per head over all keys, KV heads repeated per group."""
+    H, Hkv = q_new.shape[1], k_all.shape[1]
+    tq = torch.from_numpy(q_new.astype(np.float64))[:, :, None, :]
+    tk = torch.from_numpy(k_all.astype(np.float64)).repeat_interleave(H // Hkv, dim=1)
+    tv = torch.from_numpy(v_all.astype(np.float64)).repeat_interleave(H // Hkv, dim=1)
+    return torch.nn.functional.scaled_dot_product_attention(tq, tk, tv)[:, :, 0].numpy()
+
+
+def test_decode_wrappers_gqa_head_mapping_against_sdpa():
+    """decode_mha and decode_mha_key with theta = 0 and a window over the whole cache are plain
+    attention of the new query: query head h must read KV head h // (H / H_kv) -- checked against
+    torch SDPA in fp64 with the KV heads repeated per group, on heads that all differ."""
+    B, H, Hkv, T, d, steps = 2, 4, 2, 9, 32, 2
+    rng = np.random.default_rng(23)
+    q = rng.standard_normal((B, H, T + steps, d)).astype(np.float32)
+    k = rng.standard_normal((B, Hkv, T + steps, d)).astype(np.float32)
+    v = rng.standard_normal((B, Hkv, T + steps, d)).astype(np.float32)
+    W = T + steps + 1
+    _, heads_q = O.prefill_mha(q[:, :, :T], k[:, :, :T], v[:, :, :T], 0.0, W, "sliding")
+    _, heads_k = O.prefill_mha(q[:, :, :T], k[:, :, :T], v[:, :, :T], 0.0, W, "sliding", source="key")
+    st_q = {key: r["state"] for key, r in heads_q.items()}
+    st_k = {(b, kvh): heads_k[(b, kvh * (H // Hkv))]["state"] for b in range(B) for kvh in range(Hkv)}
+    for s in range(steps):
+        n = T + s
+        ref = _sdpa_last_row_gqa(q[:, :, n], k[:, :, :n + 1], v[:, :, :n + 1])
+        out_q, _ = O.decode_mha(st_q, q[:, :, n], k[:, :, n], v[:, :, n], 0.0, W)
+        out_k, _ = O.decode_mha_key(st_k, q[:, :, n], k[:, :, n], v[:, :, n], 0.0, W)
+        assert np.max(np.abs(out_q - ref)) < 1e-12
+        assert np.max(np.abs(out_k - ref)) < 1e-12
+    # the other mapping (h % H_kv) is a different function on this input
+    wrong_k = np.stack([k[:, h % Hkv] for h in range(H)], axis=1)
+    wrong_v = np.stack([v[:, h % Hkv] for h in range(H)], axis=1)
+    wrong = _sdpa_last_row_gqa(q[:, :, T], wrong_k[:, :, :T + 1], wrong_v[:, :, :T + 1])
+    assert np.max(np.abs(wrong - _sdpa_last_row_gqa(q[:, :, T], k[:, :, :T + 1], v[:, :, :T + 1]))) > 1e-3
+
+
+# ------------------------------------------------------------------ Eq. 6 over stages (hand-worked fixture)
+def _read_eq6_fixture():
+    rows = {}
+    with open(os.path.join(GOLDEN, "eq6_two_stage.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            name, *vals = [x.strip() for x in line.split("|")]
+            rows[name] = dict(nnz=int(vals[0]), elements=int(vals[1]), macs_done=int(vals[2]), macs_dense=int(vals[3]),
+                              S_m=float(vals[4]), S_c_eq6=float(vals[5]), S_c_exact=float(vals[6]))
+    return rows
+
+
+def test_eq6_stage_aggregates_match_hand_worked_example():
+    want = _read_eq6_fixture()
+    d = 2
+    pre = O.prefill_stats([2, 1], 2, d, 1, "block")
+    steps = [O.stage_stats([0], [2], d, 1, "sliding"), O.stage_stats([2], [3], d, 1, "sliding")]
+    raw = {key: sum(s[key] for s in steps) for key in ("nnz", "elements", "macs_done", "macs_dense")}
+    dec = O.decode_stage_stats(raw, windows=[1, 1], lengths=[3, 4])
+    both = O.combined_stats(pre, dec)
+    for name, got in (("prefill", pre), ("decode", dec), ("combined", both)):
+        for key in ("nnz", "elements", "macs_done", "macs_dense"):
+            assert got[key] == want[name][key], (name, key)
+        for key in ("S_m", "S_c_eq6", "S_c_exact"):
+            assert got[key] == pytest.approx(want[name][key], abs=1e-15), (name, key)
+    # a window longer than a step's sequence counts as the sequence length
+    assert O.decode_stage_stats(raw, [10, 10], [3, 4])["S_c_eq6"] == 0.0
