@@ -108,12 +108,15 @@ DELTA_API delta_status_t delta_state_workspace_bytes(const delta_config_t* cfg, 
 
 /* delta_state_init -- create a state over a caller-owned device workspace (256-byte aligned,
  * at least delta_state_workspace_bytes large) and enqueue the zeroing of the reference state
- * q_hat, the score row R and all counters (Eq. 3: the reference starts at 0).  *out is a host
- * object the caller releases with delta_state_destroy; the workspace must outlive it. */
+ * q_hat and all counters (Eq. 3: the reference starts at 0; one small memset).  The score row R
+ * is not cleared: prefill writes its entries 0..T-1 and a decode step reads only entries below
+ * its position.  *out is a host object the caller releases with delta_state_destroy; the
+ * workspace must outlive it. */
 DELTA_API delta_status_t delta_state_init(const delta_config_t* cfg, void* workspace, size_t workspace_bytes,
                                 void* stream, delta_state_t** out);
 
-/* Back to the freshly initialised condition (position 0, counters 0). */
+/* Back to the freshly initialised condition (position 0, reference 0, counters 0): the same
+ * one small memset on `stream`. */
 DELTA_API delta_status_t delta_state_reset(delta_state_t* st, void* stream);
 
 /* Frees the host object only. */

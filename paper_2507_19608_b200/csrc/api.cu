@@ -71,6 +71,15 @@ static void carve(const delta_config_t& c, char* base, Workspace* w) {
   const size_t g = c.H / c.H_kv;
   size_t off = 0;
   auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off += align_up(bytes, 256); return p; };
+  // what a reset has to zero comes first, as one contiguous span: the two reference buffers
+  // (Eq. 3: the reference starts at 0), the counters and the decode tickets.  The score row R
+  // needs no zeroing: prefill writes entries 0..T-1 and a decode step reads only entries below
+  // its position.
+  w->qhat[0] = (float*)take(BH * c.d * 4);
+  w->qhat[1] = (float*)take(BH * c.d * 4);
+  w->counters = (unsigned long long*)take(CNT_TOTAL * 8);
+  w->dec_ticket = (uint32_t*)take(BKV * 4);
+  w->zero_bytes = off;
   w->dq = (float*)take(BH * c.T_max * c.d * 4);
   w->mask = (uint32_t*)take(BH * c.T_max * (c.d / 32) * 4);
   w->row_nnz = (uint16_t*)take(BH * c.T_max * 2);
@@ -78,12 +87,8 @@ static void carve(const delta_config_t& c, char* base, Workspace* w) {
   w->idx = (uint8_t*)take(BH * c.T_max * c.d);
   w->qhat_tile = (float*)take(BH * nt * c.d * 4);
   w->ckpt = (float*)take(BH * (((size_t)c.T_max + DELTA_CKPT_ROWS - 1) / DELTA_CKPT_ROWS) * c.d * 4);
-  w->qhat[0] = (float*)take(BH * c.d * 4);
-  w->qhat[1] = (float*)take(BH * c.d * 4);
   w->R = (float*)take(BH * c.T_max * 4);
-  w->counters = (unsigned long long*)take(CNT_TOTAL * 8);
   w->dec_partial = (float*)take(BKV * kMaxDecodeSplits * g * (c.d + 2) * 4);
-  w->dec_ticket = (uint32_t*)take(BKV * 4);
   w->kt = (c.dtype == DELTA_BF16 && tc_kernel_shape(c.d))
               ? (float*)take(BKV * c.d * (((size_t)c.T_max + 3) / 4 * 4) * 4) : nullptr;
   w->qhat_rows = (c.dtype == DELTA_BF16 && tcq_kernel_shape(c.d))
@@ -104,15 +109,9 @@ delta_status_t delta_state_workspace_bytes(const delta_config_t* cfg, size_t* by
 }
 
 static delta_status_t zero_state(delta_state* st, cudaStream_t stream) {
-  const delta_config_t& c = st->cfg;
-  const size_t BH = (size_t)c.B * c.H;
-  cudaError_t e;
-  if ((e = cudaMemsetAsync(st->ws.qhat[0], 0, BH * c.d * 4, stream)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaMemsetAsync(st->ws.qhat[1], 0, BH * c.d * 4, stream)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaMemsetAsync(st->ws.R, 0, BH * c.T_max * 4, stream)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaMemsetAsync(st->ws.counters, 0, CNT_TOTAL * 8, stream)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaMemsetAsync(st->ws.dec_ticket, 0, (size_t)c.B * c.H_kv * 4, stream)) != cudaSuccess)
-    return cuda_fail(e);
+  // one memset: the span carve() put at the front of the workspace
+  cudaError_t e = cudaMemsetAsync(st->base, 0, st->ws.zero_bytes, stream);
+  if (e != cudaSuccess) return cuda_fail(e);
   st->n = 0;
   st->qhat_sel = 0;
   st->win_sum[0] = st->win_sum[1] = st->len_sum[0] = st->len_sum[1] = 0.0;

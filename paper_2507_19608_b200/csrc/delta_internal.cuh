@@ -40,6 +40,7 @@ struct Workspace {
   uint32_t* dec_ticket; // [B,H_kv]
   float* kt;            // [B,H_kv,d,round_up(T_max,4)] channel-major fp32 keys (tensor-core prefill only)
   __nv_bfloat16* qhat_rows;  // [B,H,T_max,d] reference state after every row (telescoped prefill only)
+  size_t zero_bytes;    // leading span of the workspace that a reset clears (q_hat, counters, tickets)
   size_t total_bytes;
 };
 

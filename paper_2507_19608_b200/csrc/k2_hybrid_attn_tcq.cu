@@ -5,24 +5,33 @@
 // Eq. 3 that sum is the reference state q_hat(i), so the out-of-window score of pair (i, j) is
 // the dense product q_hat(i).k_j.  For bf16 inputs every element of q_hat is a copy of an input
 // element (or 0), hence exactly bf16: the whole out-of-window score matrix is one more
-// Q_hat.K^T on the tensor cores, with the rows of Q_hat written by the delta-construction
-// kernel.  Nothing is skipped (the zeros of the delta matrix are unstructured, and at the
-// sparsity the method reaches a 4-row block of it is nearly dense), but the tensor cores do
-// the dense product far faster than the FP32 pipes do the sparse one.
+// Q_hat.K^T on the tensor cores.  Nothing is skipped (the zeros of the delta matrix are
+// unstructured, and at the sparsity the method reaches a 4-row block of it is nearly dense),
+// but the tensor cores do the dense product far faster than the FP32 pipes do the sparse one.
 //
-// One CTA owns 128 query rows of one head: 16 compute warps and a control warp.  The control
-// thread streams K and V tiles with TMA and issues, per 128-key tile, Q_hat.K^T (and Q.K^T if
-// the tile touches the window) into a double-buffered tensor-memory score region, one tile
-// ahead of the softmax.  Compute threads work row-per-thread straight out of tensor memory:
-// thread (row, quarter) reads 32 score columns of its row, selects exact or telescoped per
-// element, exchanges the row maximum with the three other quarters through shared memory,
-// exponentiates, writes its 32 probabilities as bf16 into the operand layout of the P.V
-// product, and rescales/accumulates its 16 output columns from the previous tile's P.V.
+// Organisation.  One CTA owns TWO 128-row query tiles of one head, a short one (tile p) and a
+// long one (tile n-1-p), so that every CTA of a head walks the same number of key tiles in
+// total; both read the same key and value tiles out of one shared-memory ring.  Ten warps:
+//   warps 0-3  softmax of query tile A, warps 4-7 softmax of query tile B: ONE THREAD PER SCORE
+//              ROW.  A thread reads its 128 scores of a key tile out of tensor memory, takes the
+//              row maximum and the exponentials without talking to any other thread, and writes
+//              the probabilities back into tensor memory as bf16, over the scores it has read;
+//   warp 8     one thread issues every tcgen05.mma: scores S = Q_hat.K^T (A and B operands in
+//              shared memory) and O += P.V with P read from tensor memory;
+//   warp 9     one thread streams key and value tiles by TMA.
+// The output tile stays in tensor memory for the whole key loop (the products accumulate);
+// a row is rescaled only when its running maximum has grown by more than 2^8 since the scale
+// it is stored at, by the softmax thread that owns the row.  While one group of softmax warps
+// exponentiates, the tensor cores work on the other group's products.
+//
+// A key tile that some row of the query tile scores exactly (Section III-B window) takes two
+// passes through the same score buffer: the telescoped product first, which the threads read
+// into registers, then Q.K^T, from which they take the in-window elements.
 //
 // Head dimensions 64 and 128 (template parameter).
 //
-// Every wait on an mbarrier is bounded (see tc_common.cuh); after a time-out the protocol
-// still runs to its end, nothing is stored and the status word records DELTA_ERR_TIMEOUT.
+// Every wait on an mbarrier is bounded; after a time-out the protocol still runs to its end,
+// nothing is stored and the status word records DELTA_ERR_TIMEOUT.
 #include <cuda.h>
 
 #include "k2_tc.cuh"
@@ -34,37 +43,44 @@ using namespace tc;
 
 namespace {
 
-constexpr int BM = 128, BN = 128, NCWARP = 16, NCTHR = NCWARP * 32, NTHR = NCTHR + 32;
+constexpr int BM = 128, BN = 128;
+constexpr int NSW = 8;                     // softmax warps: 4 per query tile
+constexpr int WARP_MMA = 8, WARP_TMA = 9;
+constexpr int NTHR = 320;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t TMEM_SH = 0;        // telescoped scores, two buffers of 128 columns
-constexpr uint32_t TMEM_SX = 256;      // exact scores, 128 columns
-constexpr uint32_t TMEM_O = 384;       // P.V tile, d columns (d <= 128)
-constexpr uint32_t SZ_BLK = 128 * 64 * 2;             // one [128 rows][64 elements] bf16 block, 16 KiB
+constexpr uint32_t TMEM_S = 0;             // scores of tile A at column 0, of tile B at column 128
+constexpr uint32_t TMEM_O = 256;           // output tile of A at 256, of B at 256 + D
+constexpr uint32_t SZ_BLK = 128 * 64 * 2;  // one [128 rows][64 elements] bf16 block, 16 KiB
+constexpr float RESCALE_LOG2 = 8.0f;       // a row is rescaled when its maximum grew by more than 2^8
 
 // Shared-memory map for head dimension D.  Operand tiles are D/64 blocks of [128][64] bf16 in
-// the 128-byte-swizzle layout.  d = 64: keys double buffered; d = 128: one key buffer (the
-// next tile's keys are fetched as soon as this tile's score products are done).
-template <int D> struct TqSmem {
+// the 128-byte-swizzle layout.  Query deltas: the two query tiles and their reference tiles;
+// key deltas: the two query tiles and one tile of original keys for window tiles.
+template <int D, bool KEY> struct TqSmem {
   static constexpr uint32_t NKB = D / 64;                 // 64-element blocks per row
   static constexpr uint32_t SZ_TILE = NKB * SZ_BLK;       // one [128][D] operand tile
-  static constexpr uint32_t NKBUF = (D == 64) ? 2 : 1;
-  static constexpr uint32_t OFF_Q = 0;
-  static constexpr uint32_t OFF_QH = OFF_Q + SZ_TILE;
-  static constexpr uint32_t OFF_K = OFF_QH + SZ_TILE;
-  static constexpr uint32_t OFF_V = OFF_K + NKBUF * SZ_TILE;   // two buffers
-  static constexpr uint32_t OFF_P = OFF_V + 2 * SZ_TILE;       // bf16 [2][128 rows][64 keys]
-  static constexpr uint32_t OFF_PMAX = OFF_P + 2 * SZ_BLK;     // fp32 [2][128 rows][4 quarters]
-  static constexpr uint32_t OFF_BAR = OFF_PMAX + 2 * 128 * 4 * 4;
-  static constexpr uint32_t OFF_MISC = OFF_BAR + 16 * 8;
+  static constexpr uint32_t NKS = 2;                      // key ring stages
+  static constexpr uint32_t NVS = (D == 64 || KEY) ? 2 : 1;   // value ring stages
+  static constexpr uint32_t OFF_Q = 0;                    // query tiles A, B
+  static constexpr uint32_t OFF_QH = OFF_Q + 2 * SZ_TILE; // reference tiles A, B (query deltas) / key tile (key deltas)
+  static constexpr uint32_t OFF_K = OFF_QH + (KEY ? 1 : 2) * SZ_TILE;
+  static constexpr uint32_t OFF_V = OFF_K + NKS * SZ_TILE;
+  static constexpr uint32_t OFF_BAR = OFF_V + NVS * SZ_TILE;
+  static constexpr uint32_t OFF_MISC = OFF_BAR + 32 * 8;
   static constexpr uint32_t BYTES = OFF_MISC + 16 + 1024;
   static_assert(BYTES <= 227 * 1024, "shared memory budget");
 };
 
 enum Bar {
-  BAR_Q = 0, BAR_K0, BAR_K1, BAR_V0, BAR_V1, BAR_S0, BAR_S1, BAR_O, BAR_KX,   // one arrival (+ bytes)
-  BAR_SFREE0, BAR_SFREE1,                                             // 16 arrivals: scores read
-  BAR_P,                                                              // 16 arrivals: P written
-  BAR_QH,                                                             // 16 arrivals: reference-query tile built
+  BAR_Q = 0,                 // both query tiles landed (one arrival + bytes)
+  BAR_QH,                    // reference-query tiles built (8 warps)
+  BAR_KFULL0, BAR_KFULL1, BAR_KFREE0, BAR_KFREE1,
+  BAR_VFULL0, BAR_VFULL1, BAR_VFREE0, BAR_VFREE1,
+  BAR_KXFULL, BAR_KXFREE,    // original keys of a window tile (key deltas)
+  BAR_SFULL_A, BAR_SFULL_B,  // a score product is complete (tcgen05.commit)
+  BAR_PRDY_A, BAR_PRDY_B,    // probabilities written (4 warps)
+  BAR_SXREQ_A, BAR_SXREQ_B,  // telescoped scores read, exact pass may overwrite them (4 warps)
+  BAR_ODONE_A, BAR_ODONE_B,  // last P.V complete
   NUM_BARS
 };
 
@@ -78,28 +94,27 @@ struct TqParams {
   float scale_log2e, theta;
 };
 
-
-// Barrier of the four warps that share a tensor-memory lane quadrant (ids 1..4, 128 threads).
-// Immediate ids: with a register operand the compiler reserves all sixteen hardware barriers
-// for the CTA and no other kernel's CTA can share the SM.
-__device__ __forceinline__ void quad_sync(int qd) {
-  switch (qd) {
-    case 0: asm volatile("bar.sync 1, 128;" ::: "memory"); break;
-    case 1: asm volatile("bar.sync 2, 128;" ::: "memory"); break;
-    case 2: asm volatile("bar.sync 3, 128;" ::: "memory"); break;
-    default: asm volatile("bar.sync 4, 128;" ::: "memory"); break;
+// Keys that some row of the query tile [i0, i1] scores exactly: lo <= j <= hi (empty if W = 0).
+// Block window: the window blocks that rows i0..i1 fall into; sliding: i0-W+1 .. i1.
+struct ExactRange { int lo, hi; };
+__device__ __forceinline__ ExactRange exact_range(int i0, int i1, int W, int shape) {
+  ExactRange r{1, 0};
+  if (W > 0) {
+    if (shape == 0) { r.lo = (i0 / W) * W; r.hi = (i1 / W) * W + W - 1; }
+    else { r.lo = i0 - W + 1; r.hi = i1; }
   }
+  return r;
 }
 
 }  // namespace
 
-// KEY = false: query deltas (strategy 1): telescoped scores Q_hat.K^T.  The 128 reference rows
-// of the tile are rebuilt in shared memory from the query tile and the references the chain
-// kernel left in front of every 8-row block (Eq. 2-3 re-run over 8 rows, blocks in parallel),
-// so the sequential chain kernel does not have to store them and tm_qh is unused.  KEY = true: key deltas (strategy 3): the column recursion telescopes to
-// S[i][j] = q_i.k_hat(j), so the telescoped scores are Q.K_hat^T; tm_qh maps the reference key
-// rows (per KV head), which take the place of the key tiles in the ring, and the original keys
-// are fetched only for tiles that touch the window.
+// KEY = false: query deltas (strategy 1, or 2 with p.reverse): telescoped scores Q_hat.K^T.  The
+// reference rows of both query tiles are rebuilt in shared memory from the query tiles and the
+// references the chain kernel left in front of every 8-row block (Eq. 2-3 re-run over 8 rows,
+// blocks in parallel); tm_qh is unused.  KEY = true: key deltas (strategy 3): the column
+// recursion telescopes to S[i][j] = q_i.k_hat(j), so the telescoped scores are Q.K_hat^T; tm_qh
+// maps the reference-key rows (per KV head), which take the place of the key tiles in the ring,
+// and the original keys are fetched only for tiles that touch the window.
 template <int D, bool KEY>
 __global__ void __launch_bounds__(NTHR, 1)
 hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qh,
@@ -109,24 +124,26 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* sm = smem_raw + (base - raw);
-  using SM = TqSmem<D>;
-  constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKBUF = SM::NKBUF;
+  using SM = TqSmem<D, KEY>;
+  constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKS = SM::NKS, NVS = SM::NVS;
   constexpr uint32_t OFF_Q = SM::OFF_Q, OFF_QH = SM::OFF_QH, OFF_K = SM::OFF_K, OFF_V = SM::OFF_V,
-                     OFF_P = SM::OFF_P, OFF_PMAX = SM::OFF_PMAX, OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC;
-  float* sPmax = reinterpret_cast<float*>(sm + OFF_PMAX);
+                     OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC;
   volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
   volatile uint32_t* abort_flag = sMisc + 1;
   const uint32_t bar0 = base + OFF_BAR;
 #define BAR(i) (bar0 + 8u * (uint32_t)(i))
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;  // heaviest query tiles of every head first
   const int bh = blockIdx.x;
   const int b = bh / p.H, h = bh - b * p.H;
   const int bkv = b * (p.H / p.g) + h / p.g;
-  const int i0 = qt * BM;
   const int T = p.T, W = p.W, shape = p.shape;
-  const int i1 = min(i0 + BM, T) - 1;
+  const int n_qt = (T + BM - 1) / BM;
+  // the CTA's two query tiles: X = 0 (A, the short one) and X = 1 (B, the long one)
+  const int qt_of[2] = {(int)blockIdx.y, n_qt - 1 - (int)blockIdx.y};
+  const bool has_b = qt_of[1] > qt_of[0];
+  const int n_of[2] = {qt_of[0] + 1, has_b ? qt_of[1] + 1 : 0};     // key tiles each one walks
+  const int n_max = has_b ? n_of[1] : n_of[0];
 
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -136,7 +153,12 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if (tid == 0) {
-    for (int i = 0; i < NUM_BARS; ++i) mbar_init(BAR(i), (i >= BAR_SFREE0) ? (uint32_t)NCWARP : 1u);
+    for (int i = 0; i < NUM_BARS; ++i) {
+      uint32_t cnt = 1;
+      if (i == BAR_QH) cnt = NSW;
+      if (i == BAR_PRDY_A || i == BAR_PRDY_B || i == BAR_SXREQ_A || i == BAR_SXREQ_B) cnt = 4;
+      mbar_init(BAR(i), cnt);
+    }
     sMisc[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
@@ -146,315 +168,299 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   tc_fence_after();
   const uint32_t tmem = sMisc[0];
 
-  // Keys that some row of this query tile scores exactly: ex_lo <= j <= ex_hi (empty if W = 0).
-  // Block window: the window blocks that rows i0..i1 fall into; sliding: i0-W+1 .. i1.
-  // Computed once: the per-tile test below must not divide.
-  int ex_lo = 1, ex_hi = 0;
-  if (W > 0) {
-    if (shape == 0) { ex_lo = (i0 / W) * W; ex_hi = (i1 / W) * W + W - 1; }
-    else { ex_lo = i0 - W + 1; ex_hi = i1; }
+  // does key tile t hold a key that some row of query tile X scores exactly?
+  ExactRange ex[2];
+#pragma unroll
+  for (int X = 0; X < 2; ++X) {
+    const int i0 = qt_of[X] * BM;
+    ex[X] = exact_range(i0, min(i0 + BM, T) - 1, W, shape);
   }
-  auto tile_needs_exact = [&](int jt) -> bool {
-    const int j0 = jt * BN, j1 = min(j0 + BN, T) - 1;
-    return j1 >= ex_lo && j0 <= ex_hi;
+  auto needs_exact = [&](int X, int t) -> bool {
+    const int j0 = t * BN, j1 = min(j0 + BN, T) - 1;
+    return j1 >= ex[X].lo && j0 <= ex[X].hi;
   };
 
-  if (warp == NCWARP) {
-    // =========================== control warp ===============================================
+  if (warp == WARP_TMA) {
+    // =========================== loader ====================================================
     if (lane == 0) {
-      const uint32_t IDESC_QK = make_idesc(BN, 0);
-      const uint32_t IDESC_PV = make_idesc(D, 1);
-      // one [128][D] tile = NKB boxes of [128][64]
       auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row0, int outer) {
 #pragma unroll
         for (uint32_t kb = 0; kb < NKB; ++kb) tma_load_3d(dst + kb * SZ_BLK, tm, bar, 64 * kb, row0, outer);
       };
-      const CUtensorMap* tm_ring = KEY ? &tm_qh : &tm_k;   // what streams through the key ring
-      mbar_expect_tx(BAR(BAR_Q), SZ_TILE);
-      load_tile(base + OFF_Q, &tm_q, BAR(BAR_Q), i0, bh);
-      // everything up to here is independent of the delta-construction kernel in front of
-      // this one (programmatic stream serialisation): wait for its results now
-      asm volatile("griddepcontrol.wait;" ::: "memory");
-      mbar_expect_tx(BAR(BAR_K0), SZ_TILE);
-      load_tile(base + OFF_K, tm_ring, BAR(BAR_K0), 0, bkv);
-      mbar_expect_tx(BAR(BAR_V0), SZ_TILE);
-      load_tile(base + OFF_V, &tm_v, BAR(BAR_V0), 0, bkv);
-      if (NKBUF == 2 && qt >= 1) {
-        mbar_expect_tx(BAR(BAR_K1), SZ_TILE);
-        load_tile(base + OFF_K + SZ_TILE, tm_ring, BAR(BAR_K1), BN, bkv);
-      }
-      int n_kx = 0;    // exact key tiles fetched so far (key deltas only)
-      // key buffer and barrier parity of tile t
-      auto kbuf = [&](int t) { return NKBUF == 2 ? (t & 1) : 0; };
-      auto kpar = [&](int t) { return NKBUF == 2 ? ((t >> 1) & 1) : (t & 1); };
-      // scores of tile t: Q_hat.K^T into buffer t&1, plus Q.K^T if the tile touches the window
-      auto issue_scores = [&](int t) {
-        const int bf = t & 1;
-        const bool exact = tile_needs_exact(t);
-        if (KEY && exact) {
-          // original keys of a window tile: into the slot the reference queries use otherwise
-          // (its previous reader, the last window tile's product, is done: see the callers)
-          mbar_expect_tx(BAR(BAR_KX), SZ_TILE);
-          load_tile(base + OFF_QH, &tm_k, BAR(BAR_KX), t * BN, bkv);
+      mbar_expect_tx(BAR(BAR_Q), (has_b ? 2u : 1u) * SZ_TILE);
+      load_tile(base + OFF_Q, &tm_q, BAR(BAR_Q), qt_of[0] * BM, bh);
+      if (has_b) load_tile(base + OFF_Q + SZ_TILE, &tm_q, BAR(BAR_Q), qt_of[1] * BM, bh);
+      // key deltas: the ring streams reference-key rows, which the finish kernel in front of
+      // this one writes (programmatic stream serialisation): wait for them.  Keys and values
+      // themselves are inputs.
+      if (KEY) asm volatile("griddepcontrol.wait;" ::: "memory");
+      const CUtensorMap* tm_ring = KEY ? &tm_qh : &tm_k;
+      int n_kx = 0;
+      for (int t = 0; t < n_max; ++t) {
+        const uint32_t ks = (uint32_t)t % NKS, vs = (uint32_t)t % NVS;
+        if (t >= (int)NKS) mbar_wait(BAR(BAR_KFREE0 + ks), ((t / NKS) - 1) & 1, abort_flag);
+        mbar_expect_tx(BAR(BAR_KFULL0 + ks), SZ_TILE);
+        load_tile(base + OFF_K + ks * SZ_TILE, tm_ring, BAR(BAR_KFULL0 + ks), t * BN, bkv);
+        if (KEY && ((t < n_of[0] && needs_exact(0, t)) || (t < n_of[1] && needs_exact(1, t)))) {
+          if (n_kx > 0) mbar_wait(BAR(BAR_KXFREE), (n_kx - 1) & 1, abort_flag);
+          mbar_expect_tx(BAR(BAR_KXFULL), SZ_TILE);
+          load_tile(base + OFF_QH, &tm_k, BAR(BAR_KXFULL), t * BN, bkv);
+          ++n_kx;
         }
-        mbar_wait(BAR(BAR_K0 + kbuf(t)), kpar(t), abort_flag);
-        tc_fence_after();
-        const uint32_t kb = base + OFF_K + kbuf(t) * SZ_TILE;
-        const uint32_t a_tele = base + (KEY ? OFF_Q : OFF_QH);
+        if (t >= (int)NVS) mbar_wait(BAR(BAR_VFREE0 + vs), ((t / NVS) - 1) & 1, abort_flag);
+        mbar_expect_tx(BAR(BAR_VFULL0 + vs), SZ_TILE);
+        load_tile(base + OFF_V + vs * SZ_TILE, &tm_v, BAR(BAR_VFULL0 + vs), t * BN, bkv);
+      }
+    }
+    __syncwarp();
+  } else if (warp == WARP_MMA) {
+    // =========================== tensor-core issue ==========================================
+    if (lane == 0) {
+      const uint32_t IDESC_QK = make_idesc(BN, 0);
+      const uint32_t IDESC_PV = make_idesc(D, 1);
+      int k_seen = -1, v_seen = -1;        // highest tile whose keys / values were waited for
+      auto wait_k = [&](int t) {
+        if (t > k_seen) { mbar_wait(BAR(BAR_KFULL0 + (uint32_t)t % NKS), (t / NKS) & 1, abort_flag); k_seen = t; tc_fence_after(); }
+      };
+      auto wait_v = [&](int t) {
+        if (t > v_seen) { mbar_wait(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag); v_seen = t; tc_fence_after(); }
+      };
+      // S_X = A . B^T into the score buffer of tile X
+      auto scores = [&](int X, uint32_t a, uint32_t bq) {
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
-          tc_mma(tmem + TMEM_SH + bf * 128,
-                 make_desc(a_tele + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
-                 make_desc(kb + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
-        if (exact) {
-          uint32_t kx = kb;
-          if (KEY) {
-            mbar_wait(BAR(BAR_KX), n_kx & 1, abort_flag);
-            ++n_kx;
-            tc_fence_after();
-            kx = base + OFF_QH;
-          }
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks)
-            tc_mma(tmem + TMEM_SX, make_desc(base + OFF_Q + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
-                   make_desc(kx + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
-        }
-        tc_commit(BAR(BAR_S0 + bf));
+          tc_mma(tmem + TMEM_S + 128u * X, make_desc(a + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
+                 make_desc(bq + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
+        tc_commit(BAR(BAR_SFULL_A + X));
+      };
+      auto tele = [&](int X, int t) {     // telescoped scores of key tile t
+        wait_k(t);
+        scores(X, base + (KEY ? OFF_Q : OFF_QH) + (uint32_t)X * SZ_TILE, base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE);
       };
       mbar_wait(BAR(BAR_Q), 0, abort_flag);
-      if (!KEY) mbar_wait(BAR(BAR_QH), 0, abort_flag);   // the compute warps have built Q_hat
-      issue_scores(0);
-      for (int t = 0; t <= qt; ++t) {
-        const bool more = t < qt;
-        const int nb = (t + 1) & 1;
-        const bool next_exact = more && tile_needs_exact(t + 1);
-        // the key buffer of tile t is free once its score products are done: refill it
-        mbar_wait(BAR(BAR_S0 + (t & 1)), (t >> 1) & 1, abort_flag);
-        const int tn = t + (int)NKBUF;         // the tile that takes this buffer next
-        if (tn <= qt) {
-          mbar_expect_tx(BAR(BAR_K0 + kbuf(tn)), SZ_TILE);
-          load_tile(base + OFF_K + kbuf(tn) * SZ_TILE, tm_ring, BAR(BAR_K0 + kbuf(tn)), tn * BN, bkv);
-        }
-        // next tile's scores one tile ahead, unless it needs the single exact-score buffer
-        if (more && !next_exact) {
-          if (t >= 1) mbar_wait(BAR(BAR_SFREE0 + nb), ((t - 1) >> 1) & 1, abort_flag);
-          issue_scores(t + 1);
-        }
-        if (t >= 1) mbar_wait(BAR(BAR_O), (t - 1) & 1, abort_flag);   // P.V(t-1) done: its V buffer is free
-        if (more) {
-          mbar_expect_tx(BAR(BAR_V0 + nb), SZ_TILE);
-          load_tile(base + OFF_V + nb * SZ_TILE, &tm_v, BAR(BAR_V0 + nb), (t + 1) * BN, bkv);
-        }
-        // P.V of this tile
-        mbar_wait(BAR(BAR_P), t & 1, abort_flag);
-        mbar_wait(BAR(BAR_V0 + (t & 1)), (t >> 1) & 1, abort_flag);
-        tc_fence_after();
-        const uint32_t vbase = base + OFF_V + (t & 1) * SZ_TILE;
+      if (!KEY) mbar_wait(BAR(BAR_QH), 0, abort_flag);   // the softmax warps have built Q_hat
+      tc_fence_after();
+      tele(0, 0);
+      if (has_b) tele(1, 0);
+      int n_kx = 0, n_sx[2] = {0, 0};
+      for (int t = 0; t < n_max; ++t) {
+        // ---- exact passes of window tiles (rare: the last tiles of a query tile)
+        bool any_x = false;
 #pragma unroll
-        for (int ks = 0; ks < BN / 16; ++ks)
-          tc_mma(tmem + TMEM_O, make_desc(base + OFF_P + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
-                 make_desc(vbase + ks * 2048, SZ_BLK, 1024), IDESC_PV, ks > 0 ? 1u : 0u);
-        tc_commit(BAR(BAR_O));
-        if (next_exact) {
-          // every compute warp has read tile t's scores (it wrote P after that)
-          mbar_wait(BAR(BAR_SFREE0 + (t & 1)), (t >> 1) & 1, abort_flag);
-          if (t >= 1) mbar_wait(BAR(BAR_SFREE0 + nb), ((t - 1) >> 1) & 1, abort_flag);
-          issue_scores(t + 1);
+        for (int X = 0; X < 2; ++X) {
+          if (t < n_of[X] && needs_exact(X, t)) {
+            if (KEY && !any_x) { mbar_wait(BAR(BAR_KXFULL), n_kx & 1, abort_flag); }
+            any_x = true;
+            mbar_wait(BAR(BAR_SXREQ_A + X), n_sx[X] & 1, abort_flag);     // telescoped scores are in registers
+            ++n_sx[X];
+            tc_fence_after();
+            scores(X, base + OFF_Q + (uint32_t)X * SZ_TILE,
+                   KEY ? base + OFF_QH : base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE);
+          }
         }
+        if (KEY && any_x) { tc_commit(BAR(BAR_KXFREE)); ++n_kx; }
+        tc_commit(BAR(BAR_KFREE0 + (uint32_t)t % NKS));   // every product that reads this key stage is issued
+        // ---- P.V of this tile, then the next tile's scores of the same query tile at once
+#pragma unroll
+        for (int X = 0; X < 2; ++X) {
+          if (t >= n_of[X]) continue;
+          mbar_wait(BAR(BAR_PRDY_A + X), t & 1, abort_flag);
+          tc_fence_after();
+          wait_v(t);
+          const uint32_t vb = base + OFF_V + ((uint32_t)t % NVS) * SZ_TILE;
+#pragma unroll
+          for (int ks = 0; ks < BN / 16; ++ks)
+            tc_mma_ts(tmem + TMEM_O + (uint32_t)(D * X), tmem + TMEM_S + 128u * X + 8u * ks,
+                      make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (t > 0 || ks > 0) ? 1u : 0u);
+          if (t == n_of[X] - 1) tc_commit(BAR(BAR_ODONE_A + X));
+          if (t + 1 < n_of[X]) tele(X, t + 1);
+        }
+        tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
       }
     }
     __syncwarp();
   } else {
-    // =========================== compute warps: row per thread ==============================
-    const int qd = warp & 3, sub = warp >> 2;     // tensor-memory lane quadrant / column quarter
-    const int row = 32 * qd + lane;
-    const int i = i0 + row;
-    const uint32_t lane_sel = (uint32_t)(32 * qd) << 16;
+    // =========================== softmax warps: one thread per score row ====================
+    const int X = warp >> 2;                       // query tile of this warp group
+    const int row = 32 * (warp & 3) + lane;        // tensor-memory lane = row of the tile
+    const int qt = qt_of[X];
+    const int i0 = qt * BM, i = i0 + row;
+    const uint32_t lane_sel = (uint32_t)(32 * (warp & 3)) << 16;
+    const uint32_t t_s = tmem + TMEM_S + 128u * X + lane_sel;
+    const uint32_t t_o = tmem + TMEM_O + (uint32_t)(D * X) + lane_sel;
     const float scale = p.scale_log2e;
-    constexpr int OC = D / 4;      // output columns per thread (a quarter of the head dimension)
-    float O[OC];
-#pragma unroll
-    for (int c = 0; c < OC; ++c) O[c] = 0.0f;
-    float m_run = -INFINITY, l_part = 0.0f, alpha_prev = 1.0f;
-    int wlo = 0, whi = 0;       // exact keys of row i: wlo <= j < whi
-    if (W > 0) {
-      if (shape == 0) { wlo = (i / W) * W; whi = wlo + W; }
-      else { wlo = i - W + 1; whi = i + 1; }
-    }
+    const int n_tiles = n_of[X];
 
     if (!KEY) {
-      // ---- reference-query tile.  The chain kernel left the reference in front of every 8-row
+      // ---- reference-query tiles.  The chain kernel left the reference in front of every 8-row
       // block; thread (channel c, row segment) re-runs Eq. 2-3 over its blocks from there (the
       // reference after row r is the last fired q[.][c] at or below r) and writes the rows of
       // Q_hat straight into the operand layout.  Blocks are independent of one another.
-      constexpr int NSEG = NCTHR / D, SEG = BM / NSEG;   // 8 x 16 rows (d=64), 4 x 32 (d=128)
+      constexpr int SEG = 2 * BM / ((NSW * 32) / D);     // rows per thread: 64 (d = 64), 128 (d = 128)
+      constexpr int NBK = SEG / DELTA_CKPT_ROWS;
       const int c = tid % D, seg = tid / D;
-      // byte offset of element (r, c) inside a [128][D] operand tile (128-byte swizzle)
-      auto elem_off = [&](int r) -> uint32_t {
+      const int Xs = (seg * SEG) / BM;                   // which query tile the segment lies in
+      const int r_seg = (seg * SEG) % BM;                // its first row inside that tile
+      const int i0s = qt_of[Xs] * BM;
+      const bool live = (Xs == 0) || has_b;
+      auto elem_off = [&](int r) -> uint32_t {   // byte offset of (r, c) in a [128][D] tile, 128-byte swizzle
         return (uint32_t)(c >> 6) * SZ_BLK + (uint32_t)r * 128u + ((((uint32_t)(c & 63) >> 3) ^ ((uint32_t)r & 7u)) << 4) +
                ((uint32_t)c & 7u) * 2u;
       };
-      float ref[SEG / DELTA_CKPT_ROWS];
+      float ref[NBK];
       asm volatile("griddepcontrol.wait;" ::: "memory");    // the chain kernel's checkpoints
+      if (live) {
 #pragma unroll
-      for (int bk = 0; bk < SEG / DELTA_CKPT_ROWS; ++bk) {
-        const int r0 = i0 + seg * SEG + bk * DELTA_CKPT_ROWS;
-        ref[bk] = (r0 < T) ? p.ckpt[((size_t)bh * p.n_ckpt + r0 / DELTA_CKPT_ROWS) * D + c] : 0.0f;
-      }
-      mbar_wait(BAR(BAR_Q), 0, abort_flag);      // the query tile has landed
-#pragma unroll
-      for (int bk = 0; bk < SEG / DELTA_CKPT_ROWS; ++bk) {
-        float cur = ref[bk];
-#pragma unroll
-        for (int rr = 0; rr < DELTA_CKPT_ROWS; ++rr) {
-          const int r8 = p.reverse ? DELTA_CKPT_ROWS - 1 - rr : rr;   // strategy (2): from the top
-          const int r = seg * SEG + bk * DELTA_CKPT_ROWS + r8;
-          const uint32_t off = elem_off(r);
-          const uint32_t xb = *reinterpret_cast<const uint16_t*>(sm + OFF_Q + off);
-          const float x = __uint_as_float(xb << 16);
-          // rows past the end of the sequence carry no state (in reverse they come first)
-          const bool fire = (i0 + r < T) && ((fabsf(__fsub_rn(x, cur)) > p.theta) || (i0 + r == p.basis_row));
-          cur = fire ? x : cur;
-          // exact: the reference is a copy of an input element (or the zero it starts from)
-          *reinterpret_cast<uint16_t*>(sm + OFF_QH + off) = (uint16_t)(__float_as_uint(cur) >> 16);
+        for (int bk = 0; bk < NBK; ++bk) {
+          const int r0 = i0s + r_seg + bk * DELTA_CKPT_ROWS;
+          ref[bk] = (r0 < T) ? p.ckpt[((size_t)bh * p.n_ckpt + r0 / DELTA_CKPT_ROWS) * D + c] : 0.0f;
         }
       }
-      fence_proxy_async();      // the tile was written through the generic proxy, the tensor cores read it
+      mbar_wait(BAR(BAR_Q), 0, abort_flag);      // the query tiles have landed
+      if (live) {
+        const unsigned char* qs = sm + OFF_Q + (size_t)Xs * SZ_TILE;
+        unsigned char* qh = sm + OFF_QH + (size_t)Xs * SZ_TILE;
+#pragma unroll
+        for (int bk = 0; bk < NBK; ++bk) {
+          float cur = ref[bk];
+#pragma unroll
+          for (int rr = 0; rr < DELTA_CKPT_ROWS; ++rr) {
+            const int r8 = p.reverse ? DELTA_CKPT_ROWS - 1 - rr : rr;   // strategy (2): from the top
+            const int r = r_seg + bk * DELTA_CKPT_ROWS + r8;
+            const uint32_t off = elem_off(r);
+            const uint32_t xb = *reinterpret_cast<const uint16_t*>(qs + off);
+            const float x = __uint_as_float(xb << 16);
+            // rows past the end of the sequence carry no state (in reverse they come first)
+            const bool fire = (i0s + r < T) && ((fabsf(__fsub_rn(x, cur)) > p.theta) || (i0s + r == p.basis_row));
+            cur = fire ? x : cur;
+            // exact: the reference is a copy of an input element (or the zero it starts from)
+            *reinterpret_cast<uint16_t*>(qh + off) = (uint16_t)(__float_as_uint(cur) >> 16);
+          }
+        }
+      }
+      fence_proxy_async();      // written through the generic proxy, read by the tensor cores
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(BAR_QH));
     }
 
-    for (int jt = 0; jt <= qt; ++jt) {
-      const int bf = jt & 1;
-      const int jc0 = jt * BN + 32 * sub;      // first key of this thread's 32 columns
-      const bool need_exact = tile_needs_exact(jt);
-      const bool diag = (jt == qt);
-
-      mbar_wait(BAR(BAR_S0 + bf), (jt >> 1) & 1, abort_flag);
-      tc_fence_after();
-      float s[32];
-      {
-        float v[16];
-        tc_ld16(tmem + TMEM_SH + bf * 128 + 32 * sub + lane_sel, v);
-#pragma unroll
-        for (int c = 0; c < 16; ++c) s[c] = v[c];
-        tc_ld16(tmem + TMEM_SH + bf * 128 + 32 * sub + 16 + lane_sel, v);
-#pragma unroll
-        for (int c = 0; c < 16; ++c) s[16 + c] = v[c];
+    if (n_tiles > 0) {
+      int wlo = 0, whi = 0;       // exact keys of row i: wlo <= j < whi
+      if (W > 0) {
+        if (shape == 0) { wlo = (i / W) * W; whi = wlo + W; }
+        else { wlo = i - W + 1; whi = i + 1; }
       }
-      if (need_exact) {
-        // hybrid select (Section III-B): exact score inside the window
+      float m_used = -INFINITY;   // the scale (log2 domain) the row's P and O are stored at
+      float l_sum = 0.0f;
+      int s_phase = 0;
+      for (int t = 0; t < n_tiles; ++t) {
+        mbar_wait(BAR(BAR_SFULL_A + X), s_phase & 1, abort_flag);
+        ++s_phase;
+        tc_fence_after();
+        float s[128];
+        {
+          uint32_t u[128];
+          tc_ld128(t_s, u);
+#pragma unroll
+          for (int c = 0; c < 128; ++c) s[c] = __uint_as_float(u[c]);
+        }
+        if (needs_exact(X, t)) {
+          // hybrid select (Section III-B): hand the buffer back for the exact product, then take
+          // the in-window elements from it
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(BAR(BAR_SXREQ_A + X));
+          mbar_wait(BAR(BAR_SFULL_A + X), s_phase & 1, abort_flag);
+          ++s_phase;
+          tc_fence_after();
+          const int j0 = t * BN;
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t u[32];
+            tc_ld32(t_s + 32u * ch, u);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int j = j0 + 32 * ch + c;
+              if (j >= wlo && j < whi) s[32 * ch + c] = __uint_as_float(u[c]);
+            }
+          }
+        }
+        if (t == qt) {
+          const int j0 = t * BN;
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (j0 + c > i) s[c] = -INFINITY;     // causal mask on the diagonal tile
+        }
+        float mx = fmax3(s[0], s[1], s[2]);
+#pragma unroll
+        for (int c = 3; c < 127; c += 2) mx = fmax3(mx, s[c], s[c + 1]);
+        mx = fmaxf(mx, s[127]);
+        const float m_new = fmaxf(m_used, mx * scale);
+        if (t == 0) {
+          m_used = m_new;                          // nothing accumulated yet
+        } else {
+          // S_full of this tile was committed behind P.V of the previous one, so the output tile
+          // holds every product up to tile t-1.  Rescale the rows whose maximum ran away.
+          const bool grow = (m_new - m_used) > RESCALE_LOG2;
+          if (__any_sync(0xffffffffu, grow)) {
+            const float al = grow ? ex2(m_used - m_new) : 1.0f;
+            if (grow) { l_sum *= al; m_used = m_new; }
+#pragma unroll
+            for (int ch = 0; ch < D / 32; ++ch) {
+              uint32_t u[32];
+              tc_ld32(t_o + 32u * ch, u);
+#pragma unroll
+              for (int c = 0; c < 32; ++c) u[c] = __float_as_uint(__uint_as_float(u[c]) * al);
+              tc_st32(t_o + 32u * ch, u);
+            }
+            tc_wait_st();
+          }
+        }
+        // probabilities, row sum, bf16 pairs back into tensor memory over the scores
+        const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-m_used, -m_used);
+        float2 sum2 = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
-          float v[16];
-          tc_ld16(tmem + TMEM_SX + 32 * sub + 16 * hf + lane_sel, v);
+          uint32_t w[32];
+#pragma unroll
+          for (int c = 0; c < 64; c += 2) {
+            const float2 e = ffma2(make_float2(s[64 * hf + c], s[64 * hf + c + 1]), sc2, nm2);
+            const float p0 = ex2(e.x), p1 = ex2(e.y);
+            sum2 = fadd2(sum2, make_float2(p0, p1));
+            const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+            w[c >> 1] = *reinterpret_cast<const uint32_t*>(&pk);
+          }
+          tc_st32(t_s + 32u * hf, w);
+        }
+        l_sum += sum2.x + sum2.y;
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(BAR_PRDY_A + X));
+      }
+
+      // ---- normalise and store the row
+      mbar_wait(BAR(BAR_ODONE_A + X), 0, abort_flag);
+      tc_fence_after();
+      const float inv = 1.0f / l_sum;
+      const bool store = (i < T) && !*abort_flag;
+#pragma unroll
+      for (int ch = 0; ch < D / 32; ++ch) {
+        uint32_t u[32];
+        tc_ld32(t_o + 32u * ch, u);
+        if (store) {
+          uint32_t w[16];
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
-            const int j = jc0 + 16 * hf + c;
-            if (j >= wlo && j < whi) s[16 * hf + c] = v[c];
+            const __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(u[2 * c]) * inv, __uint_as_float(u[2 * c + 1]) * inv);
+            w[c] = *reinterpret_cast<const uint32_t*>(&t2);
           }
+          uint4* op = reinterpret_cast<uint4*>(p.out + ((size_t)bh * T + i) * D + 32 * ch);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) op[q4] = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
         }
       }
       tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(BAR_SFREE0 + bf));
-      if (diag) {
-#pragma unroll
-        for (int c = 0; c < 32; ++c)
-          if (jc0 + c > i) s[c] = -INFINITY;     // causal mask on the diagonal tile
-      }
-      // row maximum: own 32 columns, then the three other quarters through shared memory
-      float mx = fmax3(s[0], s[1], s[2]);
-#pragma unroll
-      for (int c = 3; c < 31; c += 2) mx = fmax3(mx, s[c], s[c + 1]);
-      mx = fmaxf(mx, s[31]);
-      sPmax[(bf * BM + row) * 4 + sub] = mx;
-      quad_sync(qd);   // the four warps of this quadrant
-      const float4 pm = *reinterpret_cast<const float4*>(sPmax + (bf * BM + row) * 4);
-      mx = fmaxf(fmaxf(pm.x, pm.y), fmaxf(pm.z, pm.w));
-      const float m_new = fmaxf(m_run, mx * scale);
-      const float al = ex2(m_run - m_new);
-      m_run = m_new;
-      float2 sum2 = make_float2(0.0f, 0.0f);
-      const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-m_new, -m_new);
-#pragma unroll
-      for (int c = 0; c < 32; c += 2) {
-        const float2 t = ffma2(make_float2(s[c], s[c + 1]), sc2, nm2);
-        s[c] = ex2(t.x);
-        s[c + 1] = ex2(t.y);
-        sum2 = fadd2(sum2, make_float2(s[c], s[c + 1]));
-      }
-      l_part = fmaf(l_part, al, sum2.x + sum2.y);
-
-      // the previous tile's P.V is done: the P buffer may be rewritten
-      if (jt > 0) mbar_wait(BAR(BAR_O), (jt - 1) & 1, abort_flag);
-
-      // P as bf16 in the operand layout: this thread's 32 keys are 4 chunks of 16 bytes
-      {
-        unsigned char* prow = sm + OFF_P + (size_t)(sub >> 1) * SZ_BLK + (size_t)row * 128;
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const __nv_bfloat162 t2 = __floats2bfloat162_rn(s[8 * q4 + 2 * e], s[8 * q4 + 2 * e + 1]);
-            w[e] = *reinterpret_cast<const uint32_t*>(&t2);
-          }
-          const int chunk = 4 * (sub & 1) + q4;
-          *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-      }
-      // previous tile's P.V: rescale and accumulate (its tensor-memory tile is rewritten by
-      // this tile's product, which is issued only after every warp has arrived below)
-      if (jt > 0) {
-        tc_fence_after();
-#pragma unroll
-        for (int h16 = 0; h16 < OC / 16; ++h16) {
-          float v[16];
-          tc_ld16(tmem + TMEM_O + OC * sub + 16 * h16 + lane_sel, v);
-          const float2 ap2 = make_float2(alpha_prev, alpha_prev);
-#pragma unroll
-          for (int c = 0; c < 16; c += 2) {
-            const float2 o = ffma2(make_float2(O[16 * h16 + c], O[16 * h16 + c + 1]), ap2, make_float2(v[c], v[c + 1]));
-            O[16 * h16 + c] = o.x;
-            O[16 * h16 + c + 1] = o.y;
-          }
-        }
-        tc_fence_before();
-      }
-      alpha_prev = al;
-      fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(BAR_P));
     }
-
-    // ---- last tile's P.V, row sum over the four quarters, normalisation, store
-    mbar_wait(BAR(BAR_O), qt & 1, abort_flag);
-    tc_fence_after();
-    sPmax[(((qt + 1) & 1) * BM + row) * 4 + sub] = l_part;
-    quad_sync(qd);
-    const float4 lp = *reinterpret_cast<const float4*>(sPmax + (((qt + 1) & 1) * BM + row) * 4);
-    const float inv = 1.0f / ((lp.x + lp.y) + (lp.z + lp.w));
-    const bool store = (i < T) && !*abort_flag;
-#pragma unroll
-    for (int h16 = 0; h16 < OC / 16; ++h16) {
-      float v[16];
-      tc_ld16(tmem + TMEM_O + OC * sub + 16 * h16 + lane_sel, v);
-      if (store) {
-        uint32_t w[8];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const __nv_bfloat162 t2 = __floats2bfloat162_rn(
-              fmaf(O[16 * h16 + 2 * c], alpha_prev, v[2 * c]) * inv,
-              fmaf(O[16 * h16 + 2 * c + 1], alpha_prev, v[2 * c + 1]) * inv);
-          w[c] = *reinterpret_cast<const uint32_t*>(&t2);
-        }
-        uint4* op = reinterpret_cast<uint4*>(p.out + ((size_t)bh * T + i) * D + OC * sub + 16 * h16);
-        op[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        op[1] = make_uint4(w[4], w[5], w[6], w[7]);
-      }
-    }
-    tc_fence_before();
   }
 
   __syncthreads();
@@ -485,7 +491,7 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
               128, CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) return cudaErrorInvalidValue;
   cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D, KEY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)TqSmem<D>::BYTES);
+                                         (int)TqSmem<D, KEY>::BYTES);
   if (err != cudaSuccess) return err;
   TqParams p;
   p.out = (__nv_bfloat16*)out;
@@ -497,12 +503,14 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
   p.T = T; p.H = s.H; p.g = s.g(); p.W = window; p.shape = shape;
   p.scale_log2e = 1.4426950408889634f / sqrtf((float)s.d);
   // Launched with programmatic stream serialisation: the CTAs become resident and run their
-  // prologue (tensor-memory allocation, barrier setup, query-tile load) while the delta chain
-  // kernel in front is still running; they wait for its results with griddepcontrol.wait.
+  // prologue (tensor-memory allocation, barrier setup, query, key and value loads) while the
+  // delta chain kernel in front is still running; they wait for its results with
+  // griddepcontrol.wait.
+  const int n_qt = (T + BM - 1) / BM;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)BH, (T + BM - 1) / BM);
+  cfg.gridDim = dim3((unsigned)BH, (unsigned)((n_qt + 1) / 2));
   cfg.blockDim = dim3(NTHR);
-  cfg.dynamicSmemBytes = TqSmem<D>::BYTES;
+  cfg.dynamicSmemBytes = TqSmem<D, KEY>::BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
