@@ -47,11 +47,12 @@ namespace {
 
 constexpr int BM = 128, BN = 128;
 constexpr int NSW = 8;                     // softmax warps: two groups of 4
-constexpr int WARP_MMA = 8, WARP_TMA = 9;
-constexpr int NTHR = 320;
+constexpr int WARP_QK = 8, WARP_PV = 9, WARP_TMA = 10;
+constexpr int NTHR = 352;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TMEM_S = 0;             // score buffer of group 0 at column 0, of group 1 at column 128
 constexpr uint32_t TMEM_O = 256;           // output tile of group 0 at 256, of group 1 at 256 + D
+constexpr uint32_t TMEM_P64 = 384;         // d = 64: probabilities of group 0 at 384, of group 1 at 448
 constexpr uint32_t SZ_BLK = 128 * 64 * 2;  // one [128 rows][64 elements] bf16 block, 16 KiB
 constexpr float RESCALE_LOG2 = 8.0f;       // a row is rescaled when its maximum grew by more than 2^8
 
@@ -69,7 +70,7 @@ template <int D> struct TqSmem {
   static constexpr uint32_t OFF_K = OFF_QH + SZ_TILE;
   static constexpr uint32_t OFF_V = OFF_K + NKS * SZ_TILE;
   static constexpr uint32_t OFF_BAR = OFF_V + NVS * SZ_TILE;
-  static constexpr uint32_t OFF_MISC = OFF_BAR + 32 * 8;
+  static constexpr uint32_t OFF_MISC = OFF_BAR + 40 * 8;
   static constexpr uint32_t BYTES = OFF_MISC + 16 + 1024;
   static constexpr uint32_t XCH_FLOATS = 2 * 128 * (D / 2 + 2);   // merge exchange: [group][column][row]
   static_assert(XCH_FLOATS * 4 <= (NKS + NVS) * SZ_TILE, "the exchange buffer fits the ring space");
@@ -88,9 +89,11 @@ enum Bar {
   BAR_PRDY0, BAR_PRDY1,      // probabilities written (4 warps)
   BAR_SXREQ0, BAR_SXREQ1,    // telescoped scores read, the exact pass may overwrite them (4 warps)
   BAR_ODONE0, BAR_ODONE1,    // the group's last P.V is complete
+  BAR_SCONS0, BAR_SCONS1,    // scores read, the next product may overwrite the buffer (4 warps; d = 64)
+  BAR_PFREE0, BAR_PFREE1,    // a P.V is complete, the probabilities may be overwritten (d = 64)
   NUM_BARS
 };
-static_assert(NUM_BARS <= 32, "barrier space");
+static_assert(NUM_BARS <= 40, "barrier space");
 
 struct TqParams {
   __nv_bfloat16* out;
@@ -142,6 +145,12 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int i0 = qt * BM;
   const int i1 = min(i0 + BM, T) - 1;
   const int n = qt + 1;                                 // key tiles up to the diagonal
+  // d = 128 fills tensor memory with two score buffers and two output tiles: the probabilities
+  // overwrite the scores they come from and a group's next score product has to follow its
+  // P.V (one issuing thread does both).  d = 64 leaves room for the probabilities beside the
+  // scores: the next score product is issued as soon as the group has read the buffer, by a
+  // thread of its own, while another thread issues the P.V products.
+  constexpr bool ALIAS = (D == 128);
 
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -154,7 +163,9 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     for (int i = 0; i < NUM_BARS; ++i) {
       uint32_t cnt = 1;
       if (i == BAR_QH) cnt = NSW;
-      if (i == BAR_PRDY0 || i == BAR_PRDY1 || i == BAR_SXREQ0 || i == BAR_SXREQ1) cnt = 4;
+      if (i == BAR_PRDY0 || i == BAR_PRDY1 || i == BAR_SXREQ0 || i == BAR_SXREQ1 || i == BAR_SCONS0 ||
+          i == BAR_SCONS1)
+        cnt = 4;
       mbar_init(BAR(i), cnt);
     }
     sMisc[1] = 0;
@@ -211,8 +222,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
     }
     __syncwarp();
-  } else if (warp == WARP_MMA) {
-    // =========================== tensor-core issue ==========================================
+  } else if (warp == WARP_QK) {
+    // =========================== tensor-core issue: scores (d = 128: and P.V) ================
     if (lane == 0) {
       const uint32_t IDESC_QK = make_idesc(BN, 0);
       const uint32_t IDESC_PV = make_idesc(D, 1);
@@ -248,18 +259,46 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (KEY) { tc_commit(BAR(BAR_KXFREE)); ++n_kx; }
         }
         tc_commit(BAR(BAR_KFREE0 + (uint32_t)t % NKS));   // every product that reads this key stage is issued
-        // P.V of this tile into the group's output tile
-        mbar_wait(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
+        if (ALIAS) {
+          // P.V of this tile into the group's output tile, then the group's next scores at once
+          mbar_wait(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
+          mbar_wait(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
+          tc_fence_after();
+          const uint32_t vb = base + OFF_V + ((uint32_t)t % NVS) * SZ_TILE;
+#pragma unroll
+          for (int ks = 0; ks < BN / 16; ++ks)
+            tc_mma_ts(tmem + TMEM_O + (uint32_t)D * X, tmem + TMEM_S + 128u * X + 8u * ks,
+                      make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (t >= 2 || ks > 0) ? 1u : 0u);
+          tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
+          if (t + 2 >= n) tc_commit(BAR(BAR_ODONE0 + X));   // the group's last product
+          else tele(t + 2);
+        } else if (t + 2 < n) {
+          // the group's next scores as soon as it has read this tile's
+          mbar_wait(BAR(BAR_KFULL0 + (uint32_t)(t + 2) % NKS), ((t + 2) / NKS) & 1, abort_flag);
+          mbar_wait(BAR(BAR_SCONS0 + X), (t >> 1) & 1, abort_flag);
+          tc_fence_after();
+          scores(X, base + (KEY ? OFF_Q : OFF_QH), base + OFF_K + ((uint32_t)(t + 2) % NKS) * SZ_TILE);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == WARP_PV) {
+    // =========================== tensor-core issue: P.V (d = 64) ============================
+    if (!ALIAS && lane == 0) {
+      const uint32_t IDESC_PV = make_idesc(D, 1);
+      for (int t = 0; t < n; ++t) {
+        const uint32_t X = (uint32_t)t & 1u;
         mbar_wait(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
+        mbar_wait(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
         tc_fence_after();
         const uint32_t vb = base + OFF_V + ((uint32_t)t % NVS) * SZ_TILE;
 #pragma unroll
         for (int ks = 0; ks < BN / 16; ++ks)
-          tc_mma_ts(tmem + TMEM_O + (uint32_t)D * X, tmem + TMEM_S + 128u * X + 8u * ks,
+          tc_mma_ts(tmem + TMEM_O + (uint32_t)D * X, tmem + TMEM_P64 + 64u * X + 8u * ks,
                     make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (t >= 2 || ks > 0) ? 1u : 0u);
         tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
         if (t + 2 >= n) tc_commit(BAR(BAR_ODONE0 + X));   // the group's last product
-        else tele(t + 2);                                 // the group's next scores at once
+        else tc_commit(BAR(BAR_PFREE0 + X));              // the group may write its next probabilities
       }
     }
     __syncwarp();
@@ -271,6 +310,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const uint32_t lane_sel = (uint32_t)(32 * (warp & 3)) << 16;
     const uint32_t t_s = tmem + TMEM_S + 128u * X + lane_sel;
     const uint32_t t_o = tmem + TMEM_O + (uint32_t)D * X + lane_sel;
+    const uint32_t t_p = ALIAS ? t_s : tmem + TMEM_P64 + 64u * X + lane_sel;   // bf16 probabilities
     const float scale = p.scale_log2e;
 
     if (!KEY) {
@@ -323,10 +363,11 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     float m_used = -INFINITY;   // the scale (log2 domain) the row's P and O are stored at
     float l_sum = 0.0f;
     uint32_t s_phase = 0;
-    // Rescale of the group's output tile: S_full of a tile is committed behind the group's
-    // previous P.V, so the output tile holds every product so far; the rows whose maximum ran
-    // away since the scale they are stored at are brought to the new one (whole warp together:
-    // the tensor-memory accesses are warp-wide).
+    // Rescale of the group's output tile.  The group's previous P.V is complete (d = 128: S_full
+    // of this tile was committed behind it by the same thread; d = 64: p_free has waited for it),
+    // so the output tile holds every product so far; the rows whose maximum ran away since the
+    // scale they are stored at are brought to the new one (whole warp together: the
+    // tensor-memory accesses are warp-wide).
     auto settle_scale = [&](int t, float mx) {
       const float m_new = fmaxf(m_used, mx * scale);
       if (t < 2) { m_used = m_new; return; }     // the group's first tile: nothing accumulated yet
@@ -362,8 +403,23 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         w[c >> 1] = *reinterpret_cast<const uint32_t*>(&pk0);
         w[(c >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&pk1);
       }
-      tc_st32(t_s + 32u * hf, w);
+      tc_st32(t_p + 32u * hf, w);
       l_sum += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
+    };
+    // d = 64: the score buffer has been read (the next product may overwrite it) / the
+    // previous P.V of the group is complete (the probabilities may be overwritten)
+    auto s_consumed = [&]() {
+      if (!ALIAS) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(BAR_SCONS0 + X));
+      }
+    };
+    auto p_free = [&](int t) {
+      if (!ALIAS && t >= 2) {
+        mbar_wait(BAR(BAR_PFREE0 + X), ((t >> 1) - 1) & 1, abort_flag);
+        tc_fence_after();
+      }
     };
     auto max64 = [&](const float (&v)[64]) -> float {
       float mx0 = fmax3(v[0], v[1], v[2]), mx1 = fmax3(v[3], v[4], v[5]);
@@ -403,6 +459,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           }
           mx = fmaxf(mx, max64(v));
         }
+        p_free(t);            // (also: the output tile holds every earlier product of the group)
         settle_scale(t, mx);
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
@@ -413,6 +470,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
             for (int c = 0; c < 64; ++c) v[c] = __uint_as_float(u[c]);
           }
+          if (hf == 1) s_consumed();
           if (diag) {
 #pragma unroll
             for (int c = 0; c < 64; ++c)
@@ -460,6 +518,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (j0 + 64 + c > i) hi[c] = -INFINITY;
           }
         }
+        s_consumed();
+        p_free(t);
         settle_scale(t, fmaxf(max64(lo), max64(hi)));
         exp_store(lo, 0);
         exp_store(hi, 1);
