@@ -17,18 +17,22 @@
 //              ROW.  A thread reads its 128 scores of a key tile out of tensor memory, takes the
 //              row maximum and the exponentials without talking to any other thread, and writes
 //              the probabilities back into tensor memory as bf16, over the scores it has read;
-//   warp 8     one thread issues every tcgen05.mma: scores S = Q_hat.K^T (A and B operands in
-//              shared memory) and O += P.V with P read from tensor memory;
-//   warp 9     one thread streams key and value tiles by TMA through a ring of stages.
+//   warp 8     one thread issues the score products S = Q_hat.K^T (A and B operands in shared
+//              memory); warp 9: one thread issues O += P.V with P read from tensor memory (for
+//              d = 128, where P lies over S, warp 8 issues both in turn);
+//   warp 10    one thread streams key and value tiles by TMA through a ring of stages.
+
 // The output tiles stay in tensor memory for the whole key loop (the products accumulate);
 // a row is rescaled only when its running maximum has grown by more than 2^8 since the scale
 // it is stored at, by the softmax thread that owns the row.  While one group exponentiates,
 // the tensor cores work on the other group's products, also for a query tile that is alone
 // on its SM.
 //
-// A key tile that some row of the query tile scores exactly (Section III-B window) takes two
-// passes through the same score buffer: the telescoped product first, which the threads read
-// into registers, then Q.K^T, from which they take the in-window elements.
+// Key tiles and the window (Section III-B).  A tile none of whose pairs is inside the window is
+// scored by the telescoped product alone; a tile all of whose causal pairs are inside it by
+// Q.K^T alone; a mixed tile takes the telescoped product first and then, one half of 64 keys
+// at a time, hands the half the threads have read into registers back for Q.K^T, from which
+// they take the in-window elements.
 //
 // Head dimensions 64 and 128 (template parameter).
 //
@@ -185,9 +189,18 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     if (shape == 0) { ex_lo = (i0 / W) * W; ex_hi = (i1 / W) * W + W - 1; }
     else { ex_lo = i0 - W + 1; ex_hi = i1; }
   }
-  auto needs_exact = [&](int t) -> bool {
+  // Keys j with full_lo <= j <= full_hi are inside the window of EVERY row of the tile (block
+  // window: the rows lie in one block; sliding: the keys within W of the first row).
+  int full_lo = 1, full_hi = 0;
+  if (W > 0) {
+    if (shape == 0) { if (i1 < ex_lo + W) { full_lo = ex_lo; full_hi = ex_lo + W - 1; } }
+    else { full_lo = i1 - W + 1; full_hi = i1; }
+  }
+  // 0: telescoped scores only, 1: mixed, 2: exact scores only
+  auto tile_class = [&](int t) -> int {
     const int j0 = t * BN, j1 = min(j0 + BN, T) - 1;
-    return j1 >= ex_lo && j0 <= ex_hi;
+    if (!(j1 >= ex_lo && j0 <= ex_hi)) return 0;
+    return (j0 >= full_lo && j1 <= full_hi) ? 2 : 1;
   };
 
   if (warp == WARP_TMA) {
@@ -209,8 +222,10 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const uint32_t ks = (uint32_t)t % NKS, vs = (uint32_t)t % NVS;
         if (t >= (int)NKS) mbar_wait(BAR(BAR_KFREE0 + ks), ((t / NKS) - 1) & 1, abort_flag);
         mbar_expect_tx(BAR(BAR_KFULL0 + ks), SZ_TILE);
-        load_tile(base + OFF_K + ks * SZ_TILE, tm_ring, BAR(BAR_KFULL0 + ks), t * BN, bkv);
-        if (KEY && needs_exact(t)) {
+        // (key deltas: a tile scored exactly throughout needs the original keys, not the reference keys)
+        const int cls = tile_class(t);
+        load_tile(base + OFF_K + ks * SZ_TILE, (KEY && cls == 2) ? &tm_k : tm_ring, BAR(BAR_KFULL0 + ks), t * BN, bkv);
+        if (KEY && cls == 1) {
           if (n_kx > 0) mbar_wait(BAR(BAR_KXFREE), (n_kx - 1) & 1, abort_flag);
           mbar_expect_tx(BAR(BAR_KXFULL), SZ_TILE);
           load_tile(base + OFF_QH, &tm_k, BAR(BAR_KXFULL), t * BN, bkv);
@@ -235,34 +250,51 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                  make_desc(bq + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK, ks > 0 ? 1u : 0u);
         tc_commit(BAR(BAR_SFULL0 + X));
       };
-      auto tele = [&](int t) {     // telescoped scores of key tile t, for group t & 1
-        mbar_wait(BAR(BAR_KFULL0 + (uint32_t)t % NKS), (t / NKS) & 1, abort_flag);
-        tc_fence_after();
-        scores((uint32_t)t & 1u, base + (KEY ? OFF_Q : OFF_QH), base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE);
-      };
-      mbar_wait(BAR(BAR_Q), 0, abort_flag);
-      if (!KEY) mbar_wait(BAR(BAR_QH), 0, abort_flag);   // the softmax warps have built Q_hat
-      tc_fence_after();
-      tele(0);
-      if (n > 1) tele(1);
+      const uint32_t IDESC_QK64 = make_idesc(64, 0);
       int n_kx = 0, n_sx0 = 0, n_sx1 = 0;
+      // first scores of key tile t, for group t & 1: telescoped, or exact where the whole tile
+      // lies inside the window
+      auto first_scores = [&](int t) {
+        mbar_poll(BAR(BAR_KFULL0 + (uint32_t)t % NKS), (t / NKS) & 1, abort_flag);
+        tc_fence_after();
+        // query deltas: Q for an exact tile, Q_hat otherwise, against the keys; key deltas: Q
+        // against what the loader put into the stage (original keys for an exact tile)
+        const bool q_exact = KEY || tile_class(t) == 2;
+        scores((uint32_t)t & 1u, base + (q_exact ? OFF_Q : OFF_QH), base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE);
+      };
+      mbar_poll(BAR(BAR_Q), 0, abort_flag);
+      if (!KEY) mbar_poll(BAR(BAR_QH), 0, abort_flag);   // the softmax warps have built Q_hat
+      tc_fence_after();
+      first_scores(0);
+      if (n > 1) first_scores(1);
       for (int t = 0; t < n; ++t) {
         const uint32_t X = (uint32_t)t & 1u;
-        if (needs_exact(t)) {
-          // exact pass of a window tile: once the group has the telescoped scores in registers
-          if (KEY) mbar_wait(BAR(BAR_KXFULL), n_kx & 1, abort_flag);
+        if (tile_class(t) == 1) {
+          // mixed tile: Q.K^T over each half of 64 keys once the group has that half's
+          // telescoped scores in registers
+          if (KEY) mbar_poll(BAR(BAR_KXFULL), n_kx & 1, abort_flag);
           int& n_sx = X ? n_sx1 : n_sx0;
-          mbar_wait(BAR(BAR_SXREQ0 + X), n_sx & 1, abort_flag);
-          ++n_sx;
-          tc_fence_after();
-          scores(X, base + OFF_Q, KEY ? base + OFF_QH : base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE);
+          const uint32_t kx = KEY ? base + OFF_QH : base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE;
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            mbar_poll(BAR(BAR_SXREQ0 + X), n_sx & 1, abort_flag);
+            ++n_sx;
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+              tc_mma(tmem + TMEM_S + 128u * X + 64u * hf,
+                     make_desc(base + OFF_Q + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
+                     make_desc(kx + 8192u * hf + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK64,
+                     ks > 0 ? 1u : 0u);
+            tc_commit(BAR(BAR_SFULL0 + X));
+          }
           if (KEY) { tc_commit(BAR(BAR_KXFREE)); ++n_kx; }
         }
         tc_commit(BAR(BAR_KFREE0 + (uint32_t)t % NKS));   // every product that reads this key stage is issued
         if (ALIAS) {
           // P.V of this tile into the group's output tile, then the group's next scores at once
-          mbar_wait(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
-          mbar_wait(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
+          mbar_poll(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
+          mbar_poll(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
           tc_fence_after();
           const uint32_t vb = base + OFF_V + ((uint32_t)t % NVS) * SZ_TILE;
 #pragma unroll
@@ -271,13 +303,11 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                       make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (t >= 2 || ks > 0) ? 1u : 0u);
           tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
           if (t + 2 >= n) tc_commit(BAR(BAR_ODONE0 + X));   // the group's last product
-          else tele(t + 2);
+          else first_scores(t + 2);
         } else if (t + 2 < n) {
           // the group's next scores as soon as it has read this tile's
-          mbar_wait(BAR(BAR_KFULL0 + (uint32_t)(t + 2) % NKS), ((t + 2) / NKS) & 1, abort_flag);
-          mbar_wait(BAR(BAR_SCONS0 + X), (t >> 1) & 1, abort_flag);
-          tc_fence_after();
-          scores(X, base + (KEY ? OFF_Q : OFF_QH), base + OFF_K + ((uint32_t)(t + 2) % NKS) * SZ_TILE);
+          mbar_poll(BAR(BAR_SCONS0 + X), (t >> 1) & 1, abort_flag);
+          first_scores(t + 2);
         }
       }
     }
@@ -288,8 +318,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const uint32_t IDESC_PV = make_idesc(D, 1);
       for (int t = 0; t < n; ++t) {
         const uint32_t X = (uint32_t)t & 1u;
-        mbar_wait(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
-        mbar_wait(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
+        mbar_poll(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
+        mbar_poll(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
         tc_fence_after();
         const uint32_t vb = base + OFF_V + ((uint32_t)t % NVS) * SZ_TILE;
 #pragma unroll
@@ -363,32 +393,67 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     float m_used = -INFINITY;   // the scale (log2 domain) the row's P and O are stored at
     float l_sum = 0.0f;
     uint32_t s_phase = 0;
+    // d = 64: the score buffer has been read (the next product may overwrite it) / the
+    // previous P.V of the group is complete (the probabilities may be overwritten and the
+    // output tile holds every earlier product of the group; waited for once per tile, as late
+    // as the tile allows)
+    auto s_consumed = [&]() {
+      if (!ALIAS) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(BAR_SCONS0 + X));
+      }
+    };
+    bool pv_waited = false;
+    auto p_free = [&](int t) {
+      if (!ALIAS && t >= 2 && !pv_waited) {
+        mbar_wait(BAR(BAR_PFREE0 + X), ((t >> 1) - 1) & 1, abort_flag);
+        tc_fence_after();
+        pv_waited = true;
+      }
+    };
     // Rescale of the group's output tile.  The group's previous P.V is complete (d = 128: S_full
-    // of this tile was committed behind it by the same thread; d = 64: p_free has waited for it),
+    // of this tile was committed behind it by the same thread; d = 64: p_free waits for it),
     // so the output tile holds every product so far; the rows whose maximum ran away since the
     // scale they are stored at are brought to the new one (whole warp together: the
     // tensor-memory accesses are warp-wide).
-    auto settle_scale = [&](int t, float mx) {
+    // has_o: the output tile holds earlier products of the group; has_p0: the first half of this
+    // tile's probabilities is already stored (second half of a mixed tile)
+    auto settle_scale = [&](int t, float mx, bool has_o, bool has_p0) {
       const float m_new = fmaxf(m_used, mx * scale);
-      if (t < 2) { m_used = m_new; return; }     // the group's first tile: nothing accumulated yet
+      if (!has_o && !has_p0) { m_used = m_new; return; }     // nothing stored at the old scale yet
       const bool grow = (m_new - m_used) > RESCALE_LOG2;
       if (__any_sync(0xffffffffu, grow)) {
         const float al = grow ? ex2(m_used - m_new) : 1.0f;
         if (grow) { l_sum *= al; m_used = m_new; }
+        if (has_o) {
+          p_free(t);
 #pragma unroll
-        for (int ch = 0; ch < D / 32; ++ch) {
+          for (int ch = 0; ch < D / 32; ++ch) {
+            uint32_t u[32];
+            tc_ld32(t_o + 32u * ch, u);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) u[c] = __float_as_uint(__uint_as_float(u[c]) * al);
+            tc_st32(t_o + 32u * ch, u);
+          }
+        }
+        if (has_p0) {
           uint32_t u[32];
-          tc_ld32(t_o + 32u * ch, u);
+          tc_ld32(t_p, u);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) u[c] = __float_as_uint(__uint_as_float(u[c]) * al);
-          tc_st32(t_o + 32u * ch, u);
+          for (int c = 0; c < 32; ++c) {
+            const float lo_ = __uint_as_float(u[c] << 16) * al, hi_ = __uint_as_float(u[c] & 0xffff0000u) * al;
+            const __nv_bfloat162 pk = __floats2bfloat162_rn(lo_, hi_);
+            u[c] = *reinterpret_cast<const uint32_t*>(&pk);
+          }
+          tc_st32(t_p, u);
         }
         tc_wait_st();
       }
     };
     // 64 scores -> probabilities at the row's scale, bf16 pairs into tensor-memory columns
-    // [32 hf, 32 hf + 32) of the score buffer (over scores that have been read), row sum
-    auto exp_store = [&](const float (&v)[64], int hf) {
+    // [32 hf, 32 hf + 32) of the probability buffer, row sum
+    auto exp_store = [&](const float (&v)[64], int hf, int t) {
       const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-m_used, -m_used);
       float2 sum_a = make_float2(0.0f, 0.0f), sum_b = make_float2(0.0f, 0.0f);
       uint32_t w[32];
@@ -403,23 +468,9 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         w[c >> 1] = *reinterpret_cast<const uint32_t*>(&pk0);
         w[(c >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&pk1);
       }
+      p_free(t);      // the group's previous P.V has read the probabilities
       tc_st32(t_p + 32u * hf, w);
       l_sum += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
-    };
-    // d = 64: the score buffer has been read (the next product may overwrite it) / the
-    // previous P.V of the group is complete (the probabilities may be overwritten)
-    auto s_consumed = [&]() {
-      if (!ALIAS) {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(BAR_SCONS0 + X));
-      }
-    };
-    auto p_free = [&](int t) {
-      if (!ALIAS && t >= 2) {
-        mbar_wait(BAR(BAR_PFREE0 + X), ((t >> 1) - 1) & 1, abort_flag);
-        tc_fence_after();
-      }
     };
     auto max64 = [&](const float (&v)[64]) -> float {
       float mx0 = fmax3(v[0], v[1], v[2]), mx1 = fmax3(v[3], v[4], v[5]);
@@ -439,28 +490,35 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       tc_fence_after();
       const int j0 = t * BN;
       const bool diag = (t == qt);
-      if (!needs_exact(t)) {
-        // ---- the common tile: two passes over the score buffer in halves of 64 columns (a
-        // thread never holds more than half a row), maximum first, then the exponentials
-        float mx = -INFINITY;
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          float v[64];
-          {
-            uint32_t u[64];
-            tc_ld64(t_s + 64u * hf, u);
-#pragma unroll
-            for (int c = 0; c < 64; ++c) v[c] = __uint_as_float(u[c]);
-          }
+      pv_waited = false;
+      if (tile_class(t) != 1) {
+        // ---- the common tile: two passes over the score buffer, the row maximum first, then the
+        // exponentials in halves of 64 columns
+        float mx;
+        {
+          uint32_t u[128];
+          tc_ld128(t_s, u);
           if (diag) {
 #pragma unroll
-            for (int c = 0; c < 64; ++c)
-              if (j0 + 64 * hf + c > i) v[c] = -INFINITY;     // causal mask on the diagonal tile
+            for (int c = 0; c < 128; ++c)
+              if (j0 + c > i) u[c] = 0xff800000u;     // causal mask on the diagonal tile (-inf)
           }
-          mx = fmaxf(mx, max64(v));
+          float m0 = fmax3(__uint_as_float(u[0]), __uint_as_float(u[1]), __uint_as_float(u[2]));
+          float m1 = fmax3(__uint_as_float(u[3]), __uint_as_float(u[4]), __uint_as_float(u[5]));
+          float m2 = fmax3(__uint_as_float(u[6]), __uint_as_float(u[7]), __uint_as_float(u[8]));
+          float m3 = fmax3(__uint_as_float(u[9]), __uint_as_float(u[10]), __uint_as_float(u[11]));
+#pragma unroll
+          for (int c = 12; c < 124; c += 8) {
+            m0 = fmax3(m0, __uint_as_float(u[c]), __uint_as_float(u[c + 1]));
+            m1 = fmax3(m1, __uint_as_float(u[c + 2]), __uint_as_float(u[c + 3]));
+            m2 = fmax3(m2, __uint_as_float(u[c + 4]), __uint_as_float(u[c + 5]));
+            m3 = fmax3(m3, __uint_as_float(u[c + 6]), __uint_as_float(u[c + 7]));
+          }
+          m0 = fmax3(m0, __uint_as_float(u[124]), __uint_as_float(u[125]));
+          m1 = fmax3(m1, __uint_as_float(u[126]), __uint_as_float(u[127]));
+          mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         }
-        p_free(t);            // (also: the output tile holds every earlier product of the group)
-        settle_scale(t, mx);
+        settle_scale(t, mx, t >= 2, false);
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
           float v[64];
@@ -476,53 +534,46 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int c = 0; c < 64; ++c)
               if (j0 + 64 * hf + c > i) v[c] = -INFINITY;
           }
-          exp_store(v, hf);
+          exp_store(v, hf, t);
         }
       } else {
-        // ---- a window tile (Section III-B hybrid select): the telescoped scores go to
-        // registers, the buffer goes back for the exact product, the in-window elements are
-        // taken from that
-        float lo[64], hi[64];
-        {
-          uint32_t u[64];
-          tc_ld64(t_s, u);
+        // ---- a mixed tile (Section III-B hybrid select), one half of 64 keys at a time: the
+        // half's telescoped scores go to registers, its columns go back for the exact product,
+        // the in-window elements are taken from that
 #pragma unroll
-          for (int c = 0; c < 64; ++c) lo[c] = __uint_as_float(u[c]);
-          tc_ld64(t_s + 64u, u);
+        for (int hf = 0; hf < 2; ++hf) {
+          float v[64];
+          {
+            uint32_t u[64];
+            tc_ld64(t_s + 64u * hf, u);
 #pragma unroll
-          for (int c = 0; c < 64; ++c) hi[c] = __uint_as_float(u[c]);
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(BAR_SXREQ0 + X));
-        mbar_wait(BAR(BAR_SFULL0 + X), s_phase & 1u, abort_flag);
-        ++s_phase;
-        tc_fence_after();
+            for (int c = 0; c < 64; ++c) v[c] = __uint_as_float(u[c]);
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(BAR(BAR_SXREQ0 + X));
+          mbar_wait(BAR(BAR_SFULL0 + X), s_phase & 1u, abort_flag);
+          ++s_phase;
+          tc_fence_after();
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t u[32];
-          tc_ld32(t_s + 32u * ch, u);
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t u[32];
+            tc_ld32(t_s + 64u * hf + 32u * ch, u);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const int j = j0 + 32 * ch + c;
-            if (j >= wlo && j < whi) {
-              if (ch < 2) lo[32 * ch + c] = __uint_as_float(u[c]);
-              else hi[32 * (ch - 2) + c] = __uint_as_float(u[c]);
+            for (int c = 0; c < 32; ++c) {
+              const int j = j0 + 64 * hf + 32 * ch + c;
+              if (j >= wlo && j < whi) v[32 * ch + c] = __uint_as_float(u[c]);
             }
           }
-        }
-        if (diag) {
+          if (hf == 1) s_consumed();
+          if (diag) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {
-            if (j0 + c > i) lo[c] = -INFINITY;
-            if (j0 + 64 + c > i) hi[c] = -INFINITY;
+            for (int c = 0; c < 64; ++c)
+              if (j0 + 64 * hf + c > i) v[c] = -INFINITY;
           }
+          settle_scale(t, max64(v), t >= 2, hf == 1);
+          exp_store(v, hf, t);
         }
-        s_consumed();
-        p_free(t);
-        settle_scale(t, fmaxf(max64(lo), max64(hi)));
-        exp_store(lo, 0);
-        exp_store(hi, 1);
       }
       tc_wait_st();
       tc_fence_before();

@@ -41,4 +41,30 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// The same bounded wait as a tight poll (mbarrier.test_wait returns at once where try_wait may
+// suspend the thread for a while): for the single threads that issue tensor-core work, whose
+// reaction time is on the critical path of every tile.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void mbar_poll(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_test_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  unsigned spins = 0;
+  while (!mbar_test_wait(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (*abort_flag) return;
+      if (clock64() - t0 > kWaitBudgetClocks) { *abort_flag = 1; return; }
+    }
+  }
+}
+
 }  // namespace delta
