@@ -71,7 +71,11 @@ template <int D> struct TqSmem {
   static constexpr uint32_t NVS = (D == 64) ? 4 : 2;      // value ring stages
   static constexpr uint32_t OFF_Q = 0;
   static constexpr uint32_t OFF_QH = OFF_Q + SZ_TILE;
-  static constexpr uint32_t OFF_K = OFF_QH + SZ_TILE;
+  // d = 64, query deltas: two operand tiles mixed by row halves, [Q rows 0-63; Q_hat rows
+  // 64-127] and [Q_hat rows 0-63; Q rows 64-127] (mixed tiles of block windows whose edges
+  // fall on multiples of 64)
+  static constexpr uint32_t OFF_QM = OFF_QH + SZ_TILE;
+  static constexpr uint32_t OFF_K = OFF_QM + ((D == 64) ? 2 * SZ_TILE : 0);
   static constexpr uint32_t OFF_V = OFF_K + NKS * SZ_TILE;
   static constexpr uint32_t OFF_BAR = OFF_V + NVS * SZ_TILE;
   static constexpr uint32_t OFF_MISC = OFF_BAR + 40 * 8;
@@ -134,7 +138,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   using SM = TqSmem<D>;
   constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKS = SM::NKS, NVS = SM::NVS;
   constexpr uint32_t OFF_Q = SM::OFF_Q, OFF_QH = SM::OFF_QH, OFF_K = SM::OFF_K, OFF_V = SM::OFF_V,
-                     OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC;
+                     OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC, OFF_QM = SM::OFF_QM;
   volatile uint32_t* sMisc = reinterpret_cast<volatile uint32_t*>(sm + OFF_MISC);
   volatile uint32_t* abort_flag = sMisc + 1;
   const uint32_t bar0 = base + OFF_BAR;
@@ -196,11 +200,16 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     if (shape == 0) { if (i1 < ex_lo + W) { full_lo = ex_lo; full_hi = ex_lo + W - 1; } }
     else { full_lo = i1 - W + 1; full_hi = i1; }
   }
-  // 0: telescoped scores only, 1: mixed, 2: exact scores only
+  // A block window whose edges fall on multiples of 64 splits a mixed tile into quarters (row
+  // half x key half) that are each wholly inside or outside the window: with the row-mixed
+  // operand tiles such a tile needs no second pass (d = 64, query deltas).
+  const bool quarters = (D == 64) && !KEY && shape == 0 && W > 0 && (W % 64) == 0;
+  // 0: telescoped scores only, 1: mixed, 2: exact scores only, 3: mixed by quarters
   auto tile_class = [&](int t) -> int {
     const int j0 = t * BN, j1 = min(j0 + BN, T) - 1;
     if (!(j1 >= ex_lo && j0 <= ex_hi)) return 0;
-    return (j0 >= full_lo && j1 <= full_hi) ? 2 : 1;
+    if (j0 >= full_lo && j1 <= full_hi) return 2;
+    return quarters ? 3 : 1;
   };
 
   if (warp == WARP_TMA) {
@@ -259,8 +268,29 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tc_fence_after();
         // query deltas: Q for an exact tile, Q_hat otherwise, against the keys; key deltas: Q
         // against what the loader put into the stage (original keys for an exact tile)
-        const bool q_exact = KEY || tile_class(t) == 2;
-        scores((uint32_t)t & 1u, base + (q_exact ? OFF_Q : OFF_QH), base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE);
+        const int cls = tile_class(t);
+        const uint32_t ring = base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE;
+        if (cls == 3) {
+          // each half of 64 keys against the operand tile whose row halves are Q where the
+          // quarter lies inside the window and Q_hat where it does not
+          const uint32_t X = (uint32_t)t & 1u;
+          const int rb0 = i0 / W, rb1 = (i0 + 64) / W;
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            const int jb = (t * BN + 64 * hf) / W;
+            const bool in0 = rb0 == jb, in1 = rb1 == jb;
+            const uint32_t a = base + (in0 ? (in1 ? OFF_Q : OFF_QM) : (in1 ? OFF_QM + SZ_TILE : OFF_QH));
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+              tc_mma(tmem + TMEM_S + 128u * X + 64u * hf, make_desc(a + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
+                     make_desc(ring + 8192u * hf + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK64,
+                     ks > 0 ? 1u : 0u);
+          }
+          tc_commit(BAR(BAR_SFULL0 + X));
+          return;
+        }
+        const bool q_exact = KEY || cls == 2;
+        scores((uint32_t)t & 1u, base + (q_exact ? OFF_Q : OFF_QH), ring);
       };
       mbar_poll(BAR(BAR_Q), 0, abort_flag);
       if (!KEY) mbar_poll(BAR(BAR_QH), 0, abort_flag);   // the softmax warps have built Q_hat
@@ -377,7 +407,12 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           const bool fire = (i0 + r < T) && ((fabsf(__fsub_rn(x, cur)) > p.theta) || (i0 + r == p.basis_row));
           cur = fire ? x : cur;
           // exact: the reference is a copy of an input element (or the zero it starts from)
-          *reinterpret_cast<uint16_t*>(sm + OFF_QH + off) = (uint16_t)(__float_as_uint(cur) >> 16);
+          const uint16_t hb = (uint16_t)(__float_as_uint(cur) >> 16);
+          *reinterpret_cast<uint16_t*>(sm + OFF_QH + off) = hb;
+          if (quarters) {
+            *reinterpret_cast<uint16_t*>(sm + OFF_QM + off) = (r < 64) ? (uint16_t)xb : hb;
+            *reinterpret_cast<uint16_t*>(sm + OFF_QM + SZ_TILE + off) = (r < 64) ? hb : (uint16_t)xb;
+          }
         }
       }
       fence_proxy_async();      // written through the generic proxy, read by the tensor cores
