@@ -36,10 +36,29 @@ HEADLINE_THETA = 0.3          # S_m ~ 0.60 on the Llama-shape AR(1) workload
 FLUSH_BYTES = 256 << 20       # > 126 MB of L2, written between timed iterations
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
                   "sm_max_mhz": 1965.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the hybrid-attention kernel on the
-# headline workload, from the ncu captures summarised under profiles/ (absent = not captured
-# since the kernel last changed).
-K2_DRAM_TRAFFIC_BYTES = {2: 7386368, 1: 17161728}   # per kernel id
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "hybrid_attn_dram_traffic.txt")
+KERNEL_SOURCES = {2: "k2_hybrid_attn_tcq.cu", 1: "k2_hybrid_attn_tc.cu", 0: "k2_hybrid_attn_generic.cu"}
+
+
+def kernel_source_digest(kernel: int) -> str:
+    import hashlib
+    path = os.path.join(ROOT, "paper_2507_19608_b200", "csrc", KERNEL_SOURCES[kernel])
+    with open(path, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def measured_traffic(kernel: int, workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the hybrid-attention kernel, as the
+    ncu capture summarised under profiles/ recorded it: lines `kernel workload source-digest bytes`.
+    None when there is no capture of this workload, or the kernel source has changed since."""
+    try:
+        for line in open(TRAFFIC_FILE):
+            f = line.split()
+            if len(f) == 4 and not line.startswith("#") and int(f[0]) == kernel and f[1] == workload:
+                return int(f[3]) if f[2] == kernel_source_digest(kernel) else None
+    except (OSError, ValueError):
+        pass
+    return None
 
 
 def load_peaks():
@@ -107,13 +126,42 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- reference arm
+def host_cores() -> int:
+    """Cores this process may run on (the scheduler's affinity mask, not the machine's count)."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
         n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
-        return max(n) if n else 1
+        return min(max(n) if n else 1, host_cores())
     except Exception:
         return 1
+
+
+class blas_limit:
+    """Pins the BLAS pool the oracle's matrix products use to n threads (its Python loops are
+    single-threaded whatever the pool is)."""
+
+    def __init__(self, n):
+        self.n, self.ctx = n, None
+
+    def __enter__(self):
+        try:
+            from threadpoolctl import threadpool_limits
+            self.ctx = threadpool_limits(limits=self.n, user_api="blas")
+            self.ctx.__enter__()
+        except Exception:
+            self.ctx = None
+        return self
+
+    def __exit__(self, *a):
+        if self.ctx is not None:
+            self.ctx.__exit__(*a)
 
 
 def oracle_prefill_sample(w, tensors, theta, heads):
@@ -142,7 +190,8 @@ def run_reference(args):
     value = w.B * w.T / step_s
     cores = blas_threads()
     sample = (f"{len(heads)} of {w.H} heads per step (heads {heads}), full T={w.T}; "
-              f"layer time extrapolated by head count")
+              f"layer time extrapolated by head count; BLAS pool of {cores} threads on {host_cores()} "
+              f"available cores, the oracle's row loops are single-threaded")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
@@ -174,12 +223,16 @@ KERNEL_NAMES = {0: "generic (FP32 pipes)", 1: "tcgen05 + FP32 delta path", 2: "t
 
 
 def flop_model(w, stats, kernel):
-    """Algorithmic flops of one hybrid-attention launch, from the library's own counters.
+    """Flops of one hybrid-attention launch, from the library's own counters.
 
-    kernel 0: everything on the FP32 pipes.  kernel 1: in-window q.k and P.V on the tensor
-    cores, the sparse delta products (nnz(dq_i) multiply-adds per out-of-window pair) and the
-    per-tile seeds on the FP32 pipes.  kernel 2: out-of-window scores as the dense product
-    q_hat.k (d multiply-adds per out-of-window pair) on the tensor cores, nothing on the ALUs."""
+    method: what the method itself has to do (Eq. 4 + Eq. 1): 2 x the executed multiply-adds of the
+      score stage (d per in-window pair, nnz(dq_i) per out-of-window pair: the library's macs_done)
+      plus 2 d per causal pair for P.V.  This is the figure the roofline fraction is taken from.
+    executed: what the selected kernel really runs.  Kernel 2 (telescoped) multiplies q_hat.k
+      densely, d multiply-adds for every pair, on the tensor cores and skips nothing; kernel 1
+      runs the sparse products (plus one dense seed row per 128-row query tile) on the FP32 pipes;
+      kernel 0 runs everything on the FP32 pipes.
+    dense_equiv: 4 d per causal pair, what dense attention would be credited with."""
     BH = w.B * w.H
     N_c = w.T * (w.T + 1) // 2
     pv = 2.0 * w.d * N_c * BH                                   # P.V over every causal pair
@@ -189,29 +242,36 @@ def flop_model(w, stats, kernel):
     qk_in = 2.0 * w.d * n_in * BH
     seeds = 2.0 * w.d * (N_c - n_in) * BH / 128.0               # one dense row per 128-row query tile
     dense_equiv = 4.0 * w.d * N_c * BH
+    method = qk + pv
     if kernel == 2:
-        tensor = qk_in + 2.0 * w.d * (N_c - n_in) * BH + pv
-        return dict(algorithmic=tensor, alu=0.0, tensor=tensor, dense_equiv=dense_equiv)
+        return dict(method=method, executed=dense_equiv, alu=0.0, tensor=dense_equiv, dense_equiv=dense_equiv)
     if kernel == 1:
-        return dict(algorithmic=qk + seeds + pv, alu=(qk - qk_in) + seeds, tensor=qk_in + pv,
+        return dict(method=method, executed=qk + seeds + pv, alu=(qk - qk_in) + seeds, tensor=qk_in + pv,
                     dense_equiv=dense_equiv)
-    return dict(algorithmic=qk + seeds + pv, alu=qk + seeds + pv, tensor=0.0, dense_equiv=dense_equiv)
+    return dict(method=method, executed=qk + seeds + pv, alu=qk + seeds + pv, tensor=0.0, dense_equiv=dense_equiv)
 
 
-def k2_roofline(w, stats, kernel, k2_ms, peaks, n_sm):
+def k2_roofline(w, stats, kernel, k2_ms, peaks, n_sm, sustained=False):
+    """Roofline of the hybrid-attention kernel.  `achieved` and `frac` count the method's own flops
+    (2 x executed multiply-adds of the score stage + 2 d N_c for P.V); the flops the kernel really
+    executed and the dense-equivalent figure stand beside them under their own keys."""
     fm = flop_model(w, stats, kernel)
     sm_max = float(peaks.get("sm_max_mhz", 1965.0))
     alu_peak = n_sm * 128 * 2 * sm_max * 1e6 / 1e12          # TFLOP/s: SMs x FP32 lanes x FMA x clock
     t = k2_ms * 1e-3
     common = {"kernel": KERNEL_NAMES[kernel], "kernel_ms": k2_ms,
-              "algorithmic_tflops": fm["algorithmic"] / t / 1e12,
-              "dense_equiv_tflops": fm["dense_equiv"] / t / 1e12, "traffic": K2_DRAM_TRAFFIC_BYTES.get(kernel)}
+              "method_gflop_per_launch": fm["method"] / 1e9, "executed_gflop_per_launch": fm["executed"] / 1e9,
+              "method_tflops": fm["method"] / t / 1e12, "executed_tflops": fm["executed"] / t / 1e12,
+              "dense_equiv_tflops": fm["dense_equiv"] / t / 1e12, "traffic": measured_traffic(kernel, w.name)}
     if kernel == 2:
-        peak = float(peaks["bf16_tflops"])
-        a = fm["tensor"] / t / 1e12
+        key = "bf16_tflops_sustained" if sustained and "bf16_tflops_sustained" in peaks else "bf16_tflops"
+        peak = float(peaks[key])
+        a = fm["method"] / t / 1e12
         return {**common, "bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
-                "peak_source": f"{peaks['_source']} cuBLAS bf16 burst",
-                "note": "4 MiB of Q per launch: the layer is latency- and occupancy-bound, not tensor-bound"}
+                "executed_frac": fm["executed"] / t / 1e12 / peak,
+                "peak_source": f"{peaks['_source']} cuBLAS bf16 {'sustained' if key.endswith('sustained') else 'burst'}",
+                "note": "achieved = the method's flops (the kernel multiplies q_hat.k densely and skips nothing: "
+                        "executed_tflops = dense_equiv_tflops)"}
     a = fm["alu"] / t / 1e12
     return {**common, "bound": "alu", "achieved": a, "peak": alu_peak, "unit": "TFLOP/s", "frac": a / alu_peak,
             "peak_source": f"derived: {n_sm} SMs x 128 FP32 lanes x 2 x {sm_max:.0f} MHz",
@@ -291,9 +351,9 @@ def run_ours(args):
     barrier()
     for _ in range(args.steps):
         flush.zero_()
-        B.delta_state_reset(st)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
+        B.delta_state_reset(st)                 # the memset a fresh sequence needs is part of the step
         B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
         e1.record()
         evs.append((e0, e1))
@@ -357,12 +417,44 @@ def run_ours(args):
         line["key_deltas"] = run_key_deltas(args, B, torch, w, tens, theta, flush, peaks)
         line["strategies"] = run_strategy_errors(B, torch, w, tens, theta)
         line["window_grid"] = run_window_grid(B, torch, flush, theta)
-        line["delta_pass_large"] = run_delta_pass_large(B, torch, peaks, flush)
+        line["delta_pass_large"] = run_delta_pass_large(B, torch, peaks, flush, n_sm)
+        line["configs"] = {
+            "single_head_fp32": run_config_leg(args, B, torch, "single_head_fp32", (0.1,), flush, peaks, n_sm),
+            "bitnet_2b_prefill": run_config_leg(args, B, torch, "bitnet_2b_prefill",
+                                                WL.WORKLOADS["bitnet_2b_prefill"].thetas, flush, peaks, n_sm),
+            "llama32_1b_stack": run_stack_layer(args, B, torch, peaks, flush, n_sm),
+        }
+        d16 = line["decode"].get("batch16") or {}
+        if d16.get("roofline_l2_flushed"):
+            line["roofline_decode"] = {**d16["roofline_l2_flushed"], "workload": "llama32_1b_decode_b16",
+                                       "us_per_step": d16["us_per_step_l2_flushed"],
+                                       "us_per_step_l2_flushed_by_read": d16["us_per_step_l2_flushed_by_read"],
+                                       "us_per_step_graph_l2_warm": d16["us_per_step_graph"],
+                                       "algorithmic_bytes_per_step": d16["algorithmic_bytes_per_step"],
+                                       "note": "L2 flushed (256 MiB write) before every step, each step timed alone by events"}
         line["cpu_baseline"] = run_cpu_baseline(args, w, tens, theta)
     print(json.dumps(line))
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def time_prefill(B, torch, st, q, k, v, out, w, theta, window, flush, iters, warm=2, T=None):
+    """Device time of `iters` prefill steps (state reset + delta_attn_prefill, both inside the
+    events; L2 flushed before each step); returns the list of milliseconds."""
+    T = w.T if T is None else T
+    ms = []
+    for i in range(warm + iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.delta_state_reset(st)
+        B.delta_attn_prefill(st, q, k, v, out, T, w.H, w.H_kv, w.d, theta, window)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= warm:
+            ms.append(e0.elapsed_time(e1))
+    return ms
 
 
 def run_variants(args, B, torch, w, q, k, v, out, flush, theta, peaks, n_sm, default_kernel):
@@ -382,9 +474,9 @@ def run_variants(args, B, torch, w, q, k, v, out, flush, theta, peaks, n_sm, def
         kms, steps = [], []
         for i in range(3 + min(args.steps, 10)):
             flush.zero_()
-            B.delta_state_reset(st)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
+            B.delta_state_reset(st)
             B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
             e1.record()
             torch.cuda.synchronize()
@@ -429,17 +521,7 @@ def run_e2e(args, B, torch, w, tens, theta):
 def run_sweep(args, B, torch, w, q, k, v, out, st, flush):
     res = []
     for th in w.thetas:
-        ms = []
-        for i in range(2 + min(args.steps, 10)):
-            flush.zero_()
-            B.delta_state_reset(st)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, th, w.window)
-            e1.record()
-            torch.cuda.synchronize()
-            if i >= 2:
-                ms.append(e0.elapsed_time(e1))
+        ms = time_prefill(B, torch, st, q, k, v, out, w, th, w.window, flush, min(args.steps, 10))
         s = B.delta_sparsity_stats(st)["prefill"]
         res.append({"theta": th, "ms_per_step": statistics.mean(ms),
                     "tokens_per_s": w.B * w.T / (statistics.mean(ms) * 1e-3), "S_m": s["S_m"],
@@ -578,17 +660,7 @@ def run_key_deltas(args, B, torch, w, tens, theta, flush, peaks):
     q, k, v = (to_dev(tens[n], w.dtype, torch) for n in ("q", "k", "v"))
     out = torch.empty_like(q)
     st = B.delta_state_init(B.make_config(w.B, w.H, w.H_kv, w.d, w.T, w.dtype, source=B.DELTA_SRC_KEY))
-    ms = []
-    for i in range(3 + min(args.steps, 20)):
-        flush.zero_()
-        B.delta_state_reset(st)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
-        e1.record()
-        torch.cuda.synchronize()
-        if i >= 3:
-            ms.append(e0.elapsed_time(e1))
+    ms = time_prefill(B, torch, st, q, k, v, out, w, theta, w.window, flush, min(args.steps, 20), warm=3)
     stt = B.delta_sparsity_stats(st)["prefill"]
     return {"prefill": {"theta": theta, "ms_per_step": statistics.mean(ms),
                         "tokens_per_s": w.B * w.T / (statistics.mean(ms) * 1e-3), "S_m": stt["S_m"],
@@ -641,17 +713,7 @@ def run_window_grid(B, torch, flush, theta):
         st = B.delta_state_init(B.make_config(base.B, base.H, base.H_kv, base.d, n, base.dtype))
         for gamma in (0.02, 0.05, 0.1):
             W = B.delta_window_from_gamma(n, gamma, W_MAX)
-            ms = []
-            for i in range(6):
-                flush.zero_()
-                B.delta_state_reset(st)
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                B.delta_attn_prefill(st, q, k, v, out, n, base.H, base.H_kv, base.d, theta, W)
-                e1.record()
-                torch.cuda.synchronize()
-                if i >= 2:
-                    ms.append(e0.elapsed_time(e1))
+            ms = time_prefill(B, torch, st, q, k, v, out, base, theta, W, flush, 4, T=n)
             s_ = B.delta_sparsity_stats(st)["prefill"]
             rows.append({"n": n, "gamma": gamma, "W": W, "ms": statistics.mean(ms), "S_m": s_["S_m"],
                          "S_c_eq6": s_["S_c_eq6"], "S_c_exact": s_["S_c_exact"]})
@@ -686,7 +748,7 @@ def run_window_grid(B, torch, flush, theta):
                                     "S_c_eq6_combined": st_all["combined"]["S_c_eq6"]}}
 
 
-def run_delta_pass_large(B, torch, peaks, flush):
+def run_delta_pass_large(B, torch, peaks, flush, n_sm=148):
     """Delta construction at the size of one layer of the 16-layer stack configuration
     (batch 8, T = 4096: 16384 chains per mask word), where the pass is bandwidth- rather than
     latency-bound: chain and finish kernel times and their algorithmic HBM rates."""
@@ -700,9 +762,9 @@ def run_delta_pass_large(B, torch, peaks, flush):
     kms, steps = [], []
     for i in range(5):
         flush.zero_()
-        B.delta_state_reset(st)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
+        B.delta_state_reset(st)
         B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, theta, w.window)
         e1.record()
         torch.cuda.synchronize()
@@ -723,25 +785,125 @@ def run_delta_pass_large(B, torch, peaks, flush):
                             "unit": "GB/s", "frac": chain_b / (cm * 1e-3) / 1e9 / hbm},
             "delta_finish": {"ms": fm, "bound": "hbm", "achieved": finish_b / (fm * 1e-3) / 1e9, "peak": hbm,
                              "unit": "GB/s", "frac": finish_b / (fm * 1e-3) / 1e9 / hbm},
-            "hybrid_attn": {"ms": am, "dense_equiv_tflops": 4.0 * w.d * N_c * w.B * w.H / (am * 1e-3) / 1e12,
-                            "bound": "tensor", "peak": float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
-                            "unit": "TFLOP/s",
-                            "frac": 4.0 * w.d * N_c * w.B * w.H / (am * 1e-3) / 1e12
-                            / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
-                            "note": "dense-equivalent flops (4 d N_c per head) over the sustained cuBLAS bf16 rate"}}
+            "hybrid_attn": k2_roofline(w, stt, B.delta_state_prefill_kernel(st), am, peaks, n_sm, sustained=True)}
 
 
 def run_cpu_baseline(args, w, tens, theta):
+    """The oracle, as it stands, on a bounded head sample: once with the BLAS pool pinned to one
+    thread, once with the pool it gets by default on the cores this process may use."""
     heads = list(range(0, w.H, max(1, w.H // 8)))[:8]
     oracle_prefill_sample(w, tens, theta, heads[:1])     # warm-up
-    reps, t_used = [], 0.0
-    while t_used < 10.0 and len(reps) < 8:
-        t = oracle_prefill_sample(w, tens, theta, heads)
-        reps.append(t); t_used += t
-    per_head = statistics.mean(reps) / len(heads)
-    value = w.B * w.T / (per_head * w.H * w.B)
-    return {"value": value, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
-            "sample": f"{len(heads)} of {w.H} heads x {len(reps)} repeats, full T={w.T}; extrapolated by head count"}
+
+    def timed(budget_s):
+        reps, t_used = [], 0.0
+        while t_used < budget_s and len(reps) < 6:
+            t = oracle_prefill_sample(w, tens, theta, heads)
+            reps.append(t); t_used += t
+        per_head = statistics.mean(reps) / len(heads)
+        return w.B * w.T / (per_head * w.H * w.B), len(reps)
+    with blas_limit(1):
+        v1, n1 = timed(6.0)
+    vall, nall = timed(6.0)
+    pool = blas_threads()
+    best, cores = (vall, pool) if vall >= v1 else (v1, 1)
+    return {"value": best, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "single_thread": {"value": v1, "cores": 1}, "all_cores": {"value": vall, "cores": pool},
+            "available_cores": host_cores(),
+            "sample": f"{len(heads)} of {w.H} heads x {n1}+{nall} repeats, full T={w.T}; extrapolated by head "
+                      f"count; the oracle's row loops are single-threaded, only its matrix products use the BLAS pool"}
+
+
+def run_config_leg(args, B, torch, name, thetas, flush, peaks, n_sm, iters=10):
+    """One BASELINE configuration that is not the headline: step time (reset + prefill, L2
+    flushed), tokens/s, per-kernel times and the hybrid-attention roofline, per theta."""
+    w = WL.WORKLOADS[name]
+    tens = WL.make_qkv(w, n_decode=0)
+    q, k, v = (to_dev(tens[n], w.dtype, torch) for n in ("q", "k", "v"))
+    out = torch.empty_like(q)
+    st = B.delta_state_init(B.make_config(w.B, w.H, w.H_kv, w.d, w.T, w.dtype))
+    kernel = B.delta_state_prefill_kernel(st)
+    rows = []
+    for th in thetas:
+        ms = time_prefill(B, torch, st, q, k, v, out, w, th, w.window, flush, iters)
+        B.delta_state_enable_profiling(st, True)
+        kms = []
+        for i in range(4):
+            flush.zero_()
+            B.delta_state_reset(st)
+            B.delta_attn_prefill(st, q, k, v, out, w.T, w.H, w.H_kv, w.d, th, w.window)
+            if i >= 1:
+                kms.append(B.delta_state_prefill_kernel_ms(st))
+        B.delta_state_enable_profiling(st, False)
+        stt = B.delta_sparsity_stats(st)["prefill"]
+        km = [statistics.mean(x[i] for x in kms) for i in range(3)]
+        rows.append({"theta": th, "ms_per_step": statistics.mean(ms), "ms_per_step_min": min(ms),
+                     "tokens_per_s": w.B * w.T / (statistics.mean(ms) * 1e-3), "S_m": stt["S_m"],
+                     "S_c_exact": stt["S_c_exact"],
+                     "kernel_ms": {"delta_chain": km[0], "delta_finish": km[1], "hybrid_attn": km[2]},
+                     "roofline": k2_roofline(w, stt, kernel, km[2], peaks, n_sm)})
+    return {"workload": name, "config": config_dict(w, list(thetas)), "prefill_kernel": KERNEL_NAMES[kernel], "runs": rows}
+
+
+def run_stack_layer(args, B, torch, peaks, flush, n_sm):
+    """One layer of the 16-layer stack configuration (batch 8, T = 4096, window 256): prefill at
+    each theta of the sweep, then the 128 decode steps (n = 4096 .. 4223) with L2 flushed before
+    every step.  The layers are independent draws of the same shape, so the 16-layer figures are
+    16 x one layer."""
+    w = WL.WORKLOADS["llama32_1b_stack_layer"]
+    tens = WL.make_qkv(w)
+    cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T_max, w.dtype)
+    st = B.delta_state_init(cfg)
+    q = to_dev(tens["q"], w.dtype, torch)
+
+    def cache(x):
+        full = np.zeros((w.B, w.H_kv, w.T_max, w.d), np.float32)
+        full[:, :, :w.T] = x
+        return to_dev(full, w.dtype, torch)
+    kc, vc = cache(tens["k"]), cache(tens["v"])
+    out = torch.empty_like(q)
+    kernel = B.delta_state_prefill_kernel(st)
+    pre = []
+    for th in w.thetas:
+        ms = time_prefill(B, torch, st, q, kc, vc, out, w, th, w.window, flush, 3, warm=1)
+        B.delta_state_enable_profiling(st, True)
+        flush.zero_()
+        B.delta_state_reset(st)
+        B.delta_attn_prefill(st, q, kc, vc, out, w.T, w.H, w.H_kv, w.d, th, w.window)
+        km = B.delta_state_prefill_kernel_ms(st)
+        B.delta_state_enable_profiling(st, False)
+        stt = B.delta_sparsity_stats(st)["prefill"]
+        pre.append({"theta": th, "ms_per_layer": statistics.mean(ms), "ms_16_layers": 16 * statistics.mean(ms),
+                    "tokens_per_s": w.B * w.T / (statistics.mean(ms) * 1e-3), "S_m": stt["S_m"],
+                    "S_c_exact": stt["S_c_exact"],
+                    "kernel_ms": {"delta_chain": km[0], "delta_finish": km[1], "hybrid_attn": km[2]},
+                    "roofline": k2_roofline(w, stt, kernel, km[2], peaks, n_sm, sustained=True)})
+    # decode: the state the last prefill left (theta = the sweep's last value), 128 steps
+    theta = w.thetas[-1]
+    qd, kd, vd = (to_dev(np.ascontiguousarray(tens[x].transpose(2, 0, 1, 3)), w.dtype, torch)
+                  for x in ("q_dec", "k_dec", "v_dec"))
+    od = torch.empty_like(qd)
+    evs = []
+    for s_ in range(w.n_decode):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.delta_attn_decode_step(st, qd[s_], kd[s_], vd[s_], kc, vc, od[s_], theta, w.window)
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    us = [a.elapsed_time(b) * 1e3 for a, b in evs[4:]]
+    n_avg = w.T + (w.n_decode - 1) / 2.0
+    r_passes = 1 if B.delta_state_decode_kernel(st) == 1 else 2
+    bytes_step = w.B * (2 * w.H_kv * n_avg * w.d * 2 + r_passes * w.H * n_avg * 4)
+    gbs = bytes_step / (statistics.mean(us) * 1e-6) / 1e9
+    dec = {"theta": theta, "steps": w.n_decode, "us_per_step_l2_flushed": statistics.mean(us),
+           "us_per_step_16_layers": 16 * statistics.mean(us), "algorithmic_bytes_per_step": bytes_step,
+           "roofline": {"bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
+                        "frac": gbs / float(peaks["hbm_gbs"])},
+           "S_c_exact_combined": B.delta_sparsity_stats(st)["combined"]["S_c_exact"]}
+    return {"workload": w.name, "config": config_dict(w, list(w.thetas)), "layers": 16,
+            "note": "one layer measured; layers are independent draws of one shape: 16-layer figures = 16 x one layer",
+            "prefill": pre, "decode": dec}
 
 
 def run_only(args):
@@ -750,9 +912,15 @@ def run_only(args):
     from paper_2507_19608_b200 import binding as B
     torch.cuda.set_device(0)
     peaks = load_peaks()
-    if args.only == "stack_layer":
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    if args.only in ("stack", "bitnet"):
         flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
-        res = run_delta_pass_large(B, torch, peaks, flush)
+        res = (run_stack_layer(args, B, torch, peaks, flush, n_sm) if args.only == "stack" else
+               run_config_leg(args, B, torch, "bitnet_2b_prefill", WL.WORKLOADS["bitnet_2b_prefill"].thetas, flush,
+                              peaks, n_sm))
+    elif args.only == "stack_layer":
+        flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+        res = run_delta_pass_large(B, torch, peaks, flush, torch.cuda.get_device_properties(0).multi_processor_count)
     else:
         res = run_decode(args, B, torch, peaks, names=("llama32_1b_" + args.only,))
     print(json.dumps({"only": args.only, "result": res}))
@@ -768,7 +936,7 @@ def main():
     ap.add_argument("--theta", type=float, default=HEADLINE_THETA)
     ap.add_argument("--kernel", type=int, default=-1, help="-1 auto, 0 generic, 1 tcgen05 + FP32 delta path, 2 tcgen05 telescoped")
     ap.add_argument("--quick", action="store_true", help="prefill timing only (used for ncu launch lists)")
-    ap.add_argument("--only", default="", choices=["", "decode_b1", "decode_b16", "stack_layer"],
+    ap.add_argument("--only", default="", choices=["", "decode_b1", "decode_b16", "stack_layer", "stack", "bitnet"],
                     help="run one secondary leg alone on one GPU (small ncu captures of its kernels)")
     ap.add_argument("--ref-heads", type=int, default=4, help="heads per reference step")
     args = ap.parse_args()
