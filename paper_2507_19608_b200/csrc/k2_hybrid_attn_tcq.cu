@@ -167,16 +167,15 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (tid == 0) {
-    for (int i = 0; i < NUM_BARS; ++i) {
-      uint32_t cnt = 1;
-      if (i == BAR_QH) cnt = NSW;
-      if (i == BAR_PRDY0 || i == BAR_PRDY1 || i == BAR_SXREQ0 || i == BAR_SXREQ1 || i == BAR_SCONS0 ||
-          i == BAR_SCONS1)
-        cnt = 4;
-      mbar_init(BAR(i), cnt);
-    }
-    sMisc[1] = 0;
+  if (tid >= 32 && tid < 32 + NUM_BARS) {       // one barrier per thread of warp 1 (and 2)
+    const int i = tid - 32;
+    uint32_t cnt = 1;
+    if (i == BAR_QH) cnt = NSW;
+    if (i == BAR_PRDY0 || i == BAR_PRDY1 || i == BAR_SXREQ0 || i == BAR_SXREQ1 || i == BAR_SCONS0 ||
+        i == BAR_SCONS1)
+      cnt = 4;
+    mbar_init(BAR(i), cnt);
+    if (i == 0) sMisc[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
   }
