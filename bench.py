@@ -717,6 +717,39 @@ def run_window_grid(B, torch, flush, theta):
             s_ = B.delta_sparsity_stats(st)["prefill"]
             rows.append({"n": n, "gamma": gamma, "W": W, "ms": statistics.mean(ms), "S_m": s_["S_m"],
                          "S_c_eq6": s_["S_c_eq6"], "S_c_exact": s_["S_c_exact"]})
+    # the same lengths as ONE ragged batch per gamma (delta_attn_prefill_varlen): every sequence
+    # with its own window, Eq. 6 aggregated over the batch
+    lengths = (128, 256, 512, 1024, 2048, 4096)
+    seqs = [WL.make_qkv(base, layer=7 + i, T=n, n_decode=0) for i, n in enumerate(lengths)]
+    T_max = max(lengths)
+    st = B.delta_state_init(B.make_config(len(lengths), base.H, base.H_kv, base.d, T_max, base.dtype))
+    qp = to_dev(np.concatenate([x["q"][0].reshape(-1) for x in seqs]), base.dtype, torch)
+    kc = np.zeros((len(lengths), base.H_kv, T_max, base.d), np.float32)
+    vc = np.zeros_like(kc)
+    for b_, (x, n) in enumerate(zip(seqs, lengths)):
+        kc[b_, :, :n] = x["k"][0]
+        vc[b_, :, :n] = x["v"][0]
+    kcd, vcd = to_dev(kc, base.dtype, torch), to_dev(vc, base.dtype, torch)
+    outp = torch.empty_like(qp)
+    ragged = []
+    for gamma in (0.02, 0.05, 0.1):
+        wins = [B.delta_window_from_gamma(n, gamma, W_MAX) for n in lengths]
+        ms = []
+        for i in range(5):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.delta_state_reset(st)
+            B.delta_attn_prefill_varlen(st, qp, kcd, vcd, outp, lengths, wins, theta)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                ms.append(e0.elapsed_time(e1))
+        s_ = B.delta_sparsity_stats(st)["prefill"]
+        ragged.append({"gamma": gamma, "lengths": list(lengths), "windows": wins, "ms_per_call": statistics.mean(ms),
+                       "tokens_per_s": sum(lengths) / (statistics.mean(ms) * 1e-3), "S_m": s_["S_m"],
+                       "S_c_eq6": s_["S_c_eq6"], "S_c_exact": s_["S_c_exact"]})
+    del st, qp, kcd, vcd, outp
     # decode with the paper's W_d = 4 behind a prefill with gamma = 0.05
     w = WL.WORKLOADS["llama32_1b_decode_b1"]
     steps = 64
@@ -740,7 +773,7 @@ def run_window_grid(B, torch, flush, theta):
         B.delta_attn_decode_step(st, qd[s], kd[s], vd[s], kc, vc, od[s], theta, 4)
     torch.cuda.synchronize()
     st_all = B.delta_sparsity_stats(st)
-    return {"theta": theta, "W_max": W_MAX, "prefill": rows,
+    return {"theta": theta, "W_max": W_MAX, "prefill": rows, "ragged_batch": ragged,
             "prefill_plus_decode": {"n": w.T, "gamma": 0.05, "W": W, "W_d": 4, "decode_steps": steps,
                                     "S_c_exact_prefill": st_all["prefill"]["S_c_exact"],
                                     "S_c_exact_decode": st_all["decode"]["S_c_exact"],

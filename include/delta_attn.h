@@ -138,6 +138,25 @@ DELTA_API delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, co
                                   void* out, int32_t T, int32_t H, int32_t H_kv, int32_t d,
                                   float theta, int32_t window, void* stream);
 
+/* delta_attn_prefill_varlen -- one prefill over a batch of sequences of different lengths, each
+ * with its own window (Section III-B, Eq. 5: the prefill window follows the input length,
+ * W = min(floor(gamma n), W_max); delta_window_from_gamma gives it).
+ *   seq_lens : HOST array [B], tokens of every sequence (1 .. T_max)
+ *   windows  : HOST array [B], W of every sequence (>= 0), shape from the configuration
+ *   q, out   : packed: sequence b occupies [H, seq_lens[b], d] elements, the sequences one behind
+ *              the other in batch order (sequence b starts H * d * (seq_lens[0] + .. + seq_lens[b-1])
+ *              elements into the array)
+ *   k, v     : [B, H_kv, T_max, d] (KV-cache layout; rows 0 .. seq_lens[b]-1 of element b are read)
+ * Every sequence is what delta_attn_prefill computes for a batch of one: its own delta chains,
+ * window, counters (Eq. 6 sums over the sequences: S_c_eq6 uses sum min(W_b, n_b) / sum n_b) and
+ * decode hand-off.  Afterwards the batch elements stand at different positions:
+ * delta_state_sequence_position reports each, delta_state_position the longest, and
+ * delta_attn_decode_step advances every sequence by one token from where it stands (one kernel
+ * launch per batch element while the positions differ).  Needs a fresh or reset state. */
+DELTA_API delta_status_t delta_attn_prefill_varlen(delta_state_t* st, const void* q, const void* k, const void* v,
+                                         void* out, const int32_t* seq_lens, const int32_t* windows,
+                                         float theta, void* stream);
+
 /* delta_attn_prefill_host -- the same call for HOST buffers (q, k, v, out are host pointers
  * with the shapes above; k and v hold T rows per head, i.e. [B, H_kv, T, d]).  `staging` is
  * a DEVICE buffer of at least delta_prefill_staging_bytes(cfg, T) bytes that receives the
@@ -260,8 +279,10 @@ typedef enum {
 DELTA_API delta_status_t delta_state_view(const delta_state_t* st, int32_t what, const void** dev_ptr,
                                 size_t* bytes);
 
-/* Tokens seen so far (0 after init/reset). */
+/* Tokens seen so far (0 after init/reset); after delta_attn_prefill_varlen, of the longest sequence. */
 DELTA_API int32_t delta_state_position(const delta_state_t* st);
+/* Tokens seen so far by batch element b (-1 for a bad argument). */
+DELTA_API int32_t delta_state_sequence_position(const delta_state_t* st, int32_t b);
 
 /* Which prefill kernel the next delta_attn_prefill on this state will use:
  *   0 = generic CUDA-core kernel (every configuration);

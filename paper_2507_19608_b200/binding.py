@@ -27,7 +27,8 @@ DELTA_INIT_BASIS_EXACT, DELTA_INIT_ZERO_STATE = 0, 1
 
 EXPORTED = [
     "delta_state_workspace_bytes", "delta_state_init", "delta_state_reset", "delta_state_destroy",
-    "delta_attn_prefill", "delta_prefill_staging_bytes", "delta_attn_prefill_host",
+    "delta_attn_prefill", "delta_prefill_staging_bytes", "delta_attn_prefill_host", "delta_attn_prefill_varlen",
+    "delta_state_sequence_position",
     "delta_attn_decode_step", "delta_sparsity_stats", "delta_window_from_gamma", "delta_state_view",
     "delta_state_position", "delta_state_prefill_kernel", "delta_state_decode_kernel",
     "delta_state_set_decode_kernel",
@@ -83,6 +84,8 @@ def _load() -> C.CDLL:
         "delta_state_destroy": (C.c_int, [vp]),
         "delta_attn_prefill": (C.c_int, [vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp]),
         "delta_prefill_staging_bytes": (C.c_int, [cfgp, i32, C.POINTER(sz)]),
+        "delta_attn_prefill_varlen": (C.c_int, [vp, vp, vp, vp, vp, C.POINTER(i32), C.POINTER(i32), f32, vp]),
+        "delta_state_sequence_position": (i32, [vp, i32]),
         "delta_attn_prefill_host": (C.c_int, [vp, vp, vp, vp, vp, vp, sz, i32, f32, i32, vp]),
         "delta_attn_decode_step": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, f32, i32, vp]),
         "delta_sparsity_stats": (C.c_int, [vp, C.POINTER(delta_stats_t), vp]),
@@ -181,6 +184,20 @@ def delta_state_reset(st: DeltaState, stream=None):
 def delta_attn_prefill(st: DeltaState, q, k, v, out, T, H, H_kv, d, theta, window, stream=None):
     _check(lib.delta_attn_prefill(st.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), T, H, H_kv, d,
                                   theta, window, _stream(stream)), "delta_attn_prefill")
+
+
+def delta_attn_prefill_varlen(st: DeltaState, q, k, v, out, seq_lens, windows, theta, stream=None):
+    """q, out packed per sequence ([H, seq_lens[b], d] one behind the other); seq_lens and windows are
+    host integer sequences of length B."""
+    n = st.cfg.B
+    lens = (C.c_int32 * n)(*[int(x) for x in seq_lens])
+    wins = (C.c_int32 * n)(*[int(x) for x in windows])
+    _check(lib.delta_attn_prefill_varlen(st.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), lens, wins, theta,
+                                         _stream(stream)), "delta_attn_prefill_varlen")
+
+
+def delta_state_sequence_position(st: DeltaState, b: int) -> int:
+    return lib.delta_state_sequence_position(st.handle, b)
 
 
 def delta_prefill_staging_bytes(cfg: delta_config_t, T: int) -> int:

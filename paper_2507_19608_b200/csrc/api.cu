@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "delta_internal.cuh"
 #include "k2_tc.cuh"
@@ -26,7 +27,10 @@ struct delta_state {
   Workspace ws;
   void* base;
   size_t bytes;
-  int n;         // tokens seen
+  int n;         // tokens seen (of the longest sequence, after a prefill over sequences of different lengths)
+  std::vector<int> n_b;   // tokens seen per batch element
+  bool ragged = false;    // the batch elements stand at different positions
+  std::vector<DecodeTmapCache> dec_tmap_b, dec_tmap_h_b;   // per batch element, for ragged decoding
   int qhat_sel;  // which q_hat buffer is current
   int forced_kernel;  // -1 auto, 0 generic, 1 tensor-core
   // Eq. 6 bookkeeping that needs no device work: sum of window lengths and sequence lengths
@@ -113,6 +117,8 @@ static delta_status_t zero_state(delta_state* st, cudaStream_t stream) {
   cudaError_t e = cudaMemsetAsync(st->base, 0, st->ws.zero_bytes, stream);
   if (e != cudaSuccess) return cuda_fail(e);
   st->n = 0;
+  st->n_b.assign((size_t)st->cfg.B, 0);
+  st->ragged = false;
   st->qhat_sel = 0;
   st->win_sum[0] = st->win_sum[1] = st->len_sum[0] = st->len_sum[1] = 0.0;
   return DELTA_OK;
@@ -183,6 +189,10 @@ delta_status_t delta_state_prefill_kernel_ms(delta_state_t* st, float* ms) {
 
 int32_t delta_state_position(const delta_state_t* st) { return st ? st->n : -1; }
 
+int32_t delta_state_sequence_position(const delta_state_t* st, int32_t b) {
+  return (st && b >= 0 && b < st->cfg.B) ? st->n_b[(size_t)b] : -1;
+}
+
 // Can prefill kernel `which` (1 or 2) serve this state?
 static bool tc_eligible(const delta_state* st, int which) {
   if (st->cfg.dtype != DELTA_BF16 || !tc_kernel_available(64)) return false;
@@ -229,21 +239,40 @@ static delta_status_t check_theta_window(float theta, int32_t window) {
   return DELTA_OK;
 }
 
-delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* k, const void* v,
-                                  void* out, int32_t T, int32_t H, int32_t H_kv, int32_t d,
-                                  float theta, int32_t window, void* stream) {
-  if (!st || !q || !k || !v || !out) return DELTA_ERR_INVALID_ARG;
-  if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return DELTA_ERR_INVALID_ARG;
+}  // extern "C"
+
+// The state's workspace and shape as one batch element sees them (every array is laid out batch
+// element by batch element; the counters are shared).
+static void view_of(const delta_state* st, int b, Shape* sh, Workspace* w) {
   const delta_config_t& c = st->cfg;
-  if (H != c.H || H_kv != c.H_kv || d != c.d) return DELTA_ERR_INVALID_ARG;
-  delta_status_t s = check_theta_window(theta, window);
-  if (s != DELTA_OK) return s;
-  if (T < 1) return DELTA_ERR_INVALID_ARG;
-  if (T > c.T_max) return DELTA_ERR_CAPACITY;
-  if (st->n != 0) return DELTA_ERR_STATE;
-  cudaStream_t cs = (cudaStream_t)stream;
+  *sh = st->shape;
+  sh->B = 1;
+  *w = st->ws;
+  const size_t Hs = (c.source == DELTA_SRC_KEY) ? c.H_kv : c.H;      // heads of the delta stream
+  const size_t nt = st->shape.n_tiles, nck = st->shape.n_ckpt(), g = c.H / c.H_kv;
+  const size_t ub = (size_t)b;
+  w->dq += ub * Hs * c.T_max * c.d;
+  w->mask += ub * Hs * c.T_max * (c.d / 32);
+  w->row_nnz += ub * Hs * c.T_max;
+  w->tile_nnz += ub * Hs * nt;
+  w->idx += ub * Hs * c.T_max * c.d;
+  w->qhat_tile += ub * Hs * nt * c.d;
+  w->ckpt += ub * Hs * nck * c.d;
+  w->qhat[0] += ub * Hs * c.d;
+  w->qhat[1] += ub * Hs * c.d;
+  w->R += ub * c.H * c.T_max;
+  w->dec_partial += ub * c.H_kv * kMaxDecodeSplits * g * (c.d + 2);
+  w->dec_ticket += ub * c.H_kv;
+  if (w->kt) w->kt += ub * c.H_kv * c.d * (((size_t)c.T_max + 3) / 4 * 4);
+  if (w->qhat_rows) w->qhat_rows += ub * Hs * c.T_max * c.d;
+}
+
+// The three kernels of a prefill over one view (the whole batch, or one batch element).
+static delta_status_t prefill_launch(delta_state* st, const Shape& shape, const Workspace& ws, const void* q,
+                                     const void* k, const void* v, void* out, int32_t T, float theta,
+                                     int32_t window, cudaStream_t cs, bool prof) {
+  const delta_config_t& c = st->cfg;
   cudaError_t e;
-  const bool prof = st->profiling;
 #define MARK(i) do { if (prof && (e = cudaEventRecord(st->ev[i], cs)) != cudaSuccess) return cuda_fail(e); } while (0)
   const int which = delta_state_prefill_kernel(st);
   const bool use_tc = which == 1;
@@ -259,30 +288,30 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   const bool chained = (which == 2) && !prof;
   MARK(0);
   // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
-  if ((e = launch_delta_chain(st->shape, st->ws, key ? k : q, T, theta, c.dtype, c.init, key, rev, cs)) != cudaSuccess)
+  if ((e = launch_delta_chain(shape, ws, key ? k : q, T, theta, c.dtype, c.init, key, rev, cs)) != cudaSuccess)
     return cuda_fail(e);
   auto attention = [&]() -> cudaError_t {
-    if (use_tc) return launch_hybrid_attn_tc(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, cs);
+    if (use_tc) return launch_hybrid_attn_tc(shape, ws, q, k, v, out, T, window, c.prefill_window, cs);
     if (which == 2)
-      return launch_hybrid_attn_tcq(st->shape, st->ws, q, k, v, out, T, theta, c.init, window, c.prefill_window, key,
+      return launch_hybrid_attn_tcq(shape, ws, q, k, v, out, T, theta, c.init, window, c.prefill_window, key,
                                     rev, cs);
-    return launch_hybrid_attn_generic(st->shape, st->ws, q, k, v, out, T, window, c.prefill_window, c.dtype, cs);
+    return launch_hybrid_attn_generic(shape, ws, q, k, v, out, T, window, c.prefill_window, c.dtype, cs);
   };
   if (chained && !key) {
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
-    if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
+    if ((e = launch_delta_finish(shape, ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
                                  use_tc, key, rev, true, cs)) != cudaSuccess)
       return cuda_fail(e);
   } else if (chained) {
     // key deltas: the finish kernel writes the reference-key rows the attention kernel streams,
     // so it comes first (both programmatically serialised behind the kernel in front)
-    if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
+    if ((e = launch_delta_finish(shape, ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
                                  use_tc, key, rev, true, cs)) != cudaSuccess)
       return cuda_fail(e);
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
   } else {
     MARK(1);
-    if ((e = launch_delta_finish(st->shape, st->ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
+    if ((e = launch_delta_finish(shape, ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
                                  use_tc, key, rev, false, cs)) != cudaSuccess)
       return cuda_fail(e);
     MARK(2);
@@ -291,11 +320,73 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
   MARK(3);
   MARK(4);
 #undef MARK
+  return DELTA_OK;
+}
+
+extern "C" {
+
+delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* k, const void* v,
+                                  void* out, int32_t T, int32_t H, int32_t H_kv, int32_t d,
+                                  float theta, int32_t window, void* stream) {
+  if (!st || !q || !k || !v || !out) return DELTA_ERR_INVALID_ARG;
+  if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return DELTA_ERR_INVALID_ARG;
+  const delta_config_t& c = st->cfg;
+  if (H != c.H || H_kv != c.H_kv || d != c.d) return DELTA_ERR_INVALID_ARG;
+  delta_status_t s = check_theta_window(theta, window);
+  if (s != DELTA_OK) return s;
+  if (T < 1) return DELTA_ERR_INVALID_ARG;
+  if (T > c.T_max) return DELTA_ERR_CAPACITY;
+  if (st->n != 0) return DELTA_ERR_STATE;
+  const bool prof = st->profiling;
+  s = prefill_launch(st, st->shape, st->ws, q, k, v, out, T, theta, window, (cudaStream_t)stream, prof);
+  if (s != DELTA_OK) return s;
   st->profiled = prof;
   st->n = T;
+  st->n_b.assign((size_t)c.B, T);
+  st->ragged = false;
   st->qhat_sel = 0;
-  st->win_sum[0] += (double)(window < T ? window : T);
-  st->len_sum[0] += (double)T;
+  st->win_sum[0] += (double)c.B * (double)(window < T ? window : T);
+  st->len_sum[0] += (double)c.B * (double)T;
+  return DELTA_OK;
+}
+
+delta_status_t delta_attn_prefill_varlen(delta_state_t* st, const void* q, const void* k, const void* v,
+                                         void* out, const int32_t* seq_lens, const int32_t* windows,
+                                         float theta, void* stream) {
+  if (!st || !q || !k || !v || !out || !seq_lens || !windows) return DELTA_ERR_INVALID_ARG;
+  if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return DELTA_ERR_INVALID_ARG;
+  const delta_config_t& c = st->cfg;
+  if (!(theta >= 0.0f) || !std::isfinite(theta)) return DELTA_ERR_INVALID_ARG;
+  for (int b = 0; b < c.B; ++b) {
+    if (seq_lens[b] < 1 || windows[b] < 0) return DELTA_ERR_INVALID_ARG;
+    if (seq_lens[b] > c.T_max) return DELTA_ERR_CAPACITY;
+  }
+  if (st->n != 0) return DELTA_ERR_STATE;
+  const size_t es = c.dtype == DELTA_F32 ? 4 : 2;
+  size_t q_off = 0;     // elements in front of sequence b in the packed query / output arrays
+  int t_longest = 0;
+  bool same = true;
+  for (int b = 0; b < c.B; ++b) {
+    Shape sh;
+    Workspace ws;
+    view_of(st, b, &sh, &ws);
+    const int T = seq_lens[b];
+    const size_t kv_off = (size_t)b * c.H_kv * c.T_max * c.d * es;
+    delta_status_t s = prefill_launch(st, sh, ws, (const char*)q + q_off * es, (const char*)k + kv_off,
+                                      (const char*)v + kv_off, (char*)out + q_off * es, T, theta, windows[b],
+                                      (cudaStream_t)stream, false);
+    if (s != DELTA_OK) return s;
+    q_off += (size_t)c.H * T * c.d;
+    st->n_b[(size_t)b] = T;
+    st->win_sum[0] += (double)(windows[b] < T ? windows[b] : T);
+    st->len_sum[0] += (double)T;
+    t_longest = T > t_longest ? T : t_longest;
+    same = same && T == seq_lens[0];
+  }
+  st->profiled = false;
+  st->n = t_longest;
+  st->ragged = !same;
+  st->qhat_sel = 0;
   return DELTA_OK;
 }
 
@@ -354,6 +445,29 @@ delta_status_t delta_attn_prefill_host(delta_state_t* st, const void* q_host, co
   return DELTA_OK;
 }
 
+}  // extern "C"
+
+// One decode-step launch over a view (the whole batch, or one batch element) at position n.
+static cudaError_t decode_launch(delta_state* st, const Shape& shape, const Workspace& ws, const void* q_new,
+                                 const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* out,
+                                 int n, float theta, int32_t window, DecodeTmapCache* tmap, DecodeTmapCache* tmap_h,
+                                 cudaStream_t cs) {
+  const bool tcs = decode_tc_possible(st) &&
+                   (st->forced_decode_kernel >= 0 ? st->forced_decode_kernel == 1
+                                                  : decode_tc_applies(shape, st->cfg.dtype, n));
+  if (st->cfg.source == DELTA_SRC_KEY)
+    return tcs ? launch_decode_step_key_tc(shape, ws, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window,
+                                           st->qhat_sel, tmap, tmap_h, cs)
+               : launch_decode_step_key(shape, ws, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window,
+                                        st->qhat_sel, cs);
+  return tcs ? launch_decode_step_tc(shape, ws, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window,
+                                     st->qhat_sel, tmap, cs)
+             : launch_decode_step(shape, ws, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window,
+                                  st->cfg.dtype, st->qhat_sel, cs);
+}
+
+extern "C" {
+
 delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, const void* k_new,
                                       const void* v_new, void* k_cache, void* v_cache, void* out,
                                       float theta, int32_t window, void* stream) {
@@ -364,26 +478,39 @@ delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, cons
     return DELTA_ERR_INVALID_ARG;
   delta_status_t s = check_theta_window(theta, window);
   if (s != DELTA_OK) return s;
-  if (st->cfg.source == DELTA_SRC_QUERY_BOTTOM_UP) return DELTA_ERR_UNSUPPORTED;   // strategy (2) has no decode
+  const delta_config_t& c = st->cfg;
+  if (c.source == DELTA_SRC_QUERY_BOTTOM_UP) return DELTA_ERR_UNSUPPORTED;   // strategy (2) has no decode
   if (st->n < 1) return DELTA_ERR_STATE;
-  if (st->n >= st->cfg.T_max) return DELTA_ERR_CAPACITY;
-  const bool tcs = delta_state_decode_kernel(st) == 1;
+  if (st->n >= c.T_max) return DELTA_ERR_CAPACITY;      // (the longest sequence decides)
   cudaStream_t cs = (cudaStream_t)stream;
-  cudaError_t e;
-  if (st->cfg.source == DELTA_SRC_KEY)
-    e = tcs ? launch_decode_step_key_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
-                                        window, st->qhat_sel, &st->dec_tmap, &st->dec_tmap_h, cs)
-            : launch_decode_step_key(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
-                                     window, st->qhat_sel, cs);
-  else
-    e = tcs ? launch_decode_step_tc(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
-                                    window, st->qhat_sel, &st->dec_tmap, cs)
-            : launch_decode_step(st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta,
-                                 window, st->cfg.dtype, st->qhat_sel, cs);
-  if (e != cudaSuccess) return cuda_fail(e);
-  const int L = st->n + 1;
-  st->win_sum[1] += (double)(window < L ? window : L);
-  st->len_sum[1] += (double)L;
+  cudaError_t e = cudaSuccess;
+  if (!st->ragged) {
+    e = decode_launch(st, st->shape, st->ws, q_new, k_new, v_new, k_cache, v_cache, out, st->n, theta, window,
+                      &st->dec_tmap, &st->dec_tmap_h, cs);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const int L = st->n + 1;
+    st->win_sum[1] += (double)c.B * (double)(window < L ? window : L);
+    st->len_sum[1] += (double)c.B * (double)L;
+  } else {
+    // the batch elements stand at different positions: one launch per element over its view
+    const size_t es = c.dtype == DELTA_F32 ? 4 : 2;
+    if (st->dec_tmap_b.size() != (size_t)c.B) { st->dec_tmap_b.resize((size_t)c.B); st->dec_tmap_h_b.resize((size_t)c.B); }
+    for (int b = 0; b < c.B; ++b) {
+      Shape sh;
+      Workspace ws;
+      view_of(st, b, &sh, &ws);
+      const size_t qo = (size_t)b * c.H * c.d * es, ko = (size_t)b * c.H_kv * c.d * es;
+      const size_t co = (size_t)b * c.H_kv * c.T_max * c.d * es;
+      e = decode_launch(st, sh, ws, (const char*)q_new + qo, (const char*)k_new + ko, (const char*)v_new + ko,
+                        (char*)k_cache + co, (char*)v_cache + co, (char*)out + qo, st->n_b[(size_t)b], theta, window,
+                        &st->dec_tmap_b[(size_t)b], &st->dec_tmap_h_b[(size_t)b], cs);
+      if (e != cudaSuccess) return cuda_fail(e);
+      const int L = st->n_b[(size_t)b] + 1;
+      st->win_sum[1] += (double)(window < L ? window : L);
+      st->len_sum[1] += (double)L;
+    }
+  }
+  for (auto& nb : st->n_b) nb += 1;
   st->qhat_sel ^= 1;
   st->n += 1;
   return DELTA_OK;

@@ -84,6 +84,8 @@ def test_null_and_misaligned_arguments_are_rejected_before_any_device_work():
         assert B.lib.delta_attn_decode_step_noalloc(*ptrs, ok, ok + 64, ok, 10, 1, 8, 2, 64, 128, B.DELTA_BF16,
                                                     0.1, 4, None) == B.DELTA_ERR_INVALID_ARG
     assert B.lib.delta_noalloc_device_status(None, None) == B.DELTA_ERR_INVALID_ARG
+    assert B.lib.delta_attn_prefill_varlen(None, 16, 16, 16, 16, None, None, 0.1, None) == B.DELTA_ERR_INVALID_ARG
+    assert B.lib.delta_state_sequence_position(None, 0) == -1
     assert B.lib.delta_state_position(None) == -1
 
 
