@@ -529,7 +529,8 @@ def run_sweep(args, B, torch, w, q, k, v, out, st, flush):
     return res
 
 
-def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_b1", "llama32_1b_decode_b16")):
+def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_b1", "llama32_1b_decode_b16"),
+               packed=False):
     """Decode leg: cache prefilled to 2048 tokens, then 256 steps; batch 1 and 16.
     source="key": the paper's adopted strategy (3) (key deltas; the carried state is the reference key)."""
     res = {}
@@ -541,6 +542,8 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
         cfg = B.make_config(w.B, w.H, w.H_kv, w.d, w.T_max, w.dtype, prefill_window=B.DELTA_WIN_SLIDING,
                             source=B.DELTA_SRC_KEY if key else B.DELTA_SRC_QUERY)
         st = B.delta_state_init(cfg)
+        if packed:
+            B.delta_state_set_key_cache(st, True)     # decode from the compressed key-delta cache
         q = to_dev(tens["q"], w.dtype, torch)
 
         def cache(x):
@@ -572,6 +575,10 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
             eager.append(e0.elapsed_time(e1) * 1e3 / w.n_decode)
         od_eager = od.clone()
         dstats = B.delta_sparsity_stats(st)
+        cache_bytes = None
+        if packed:
+            pb, db = B.delta_key_cache_bytes(st)
+            cache_bytes = {"packed": pb, "dense_reference_keys": db, "ratio": pb / db}
         # the same 256 launches replayed from a CUDA graph (removes the host launch path)
         graph_us, graph_ok = None, None
         try:
@@ -599,6 +606,8 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
         # (and read it, where the step runs on the FP32 pipes: the tensor-core form recomputes it)
         r_passes = 0 if key else (1 if B.delta_state_decode_kernel(st) == 1 else 2)
         bytes_step = w.B * (2 * w.H_kv * n_avg * w.d * es + r_passes * w.H * n_avg * 4)
+        if packed:      # values + V rows: the key side is the encoding, not dense rows
+            bytes_step = w.B * w.H_kv * n_avg * w.d * es * (1.0 + cache_bytes["ratio"])
         # the same steps with L2 flushed before each one (in a model every layer's cache passes
         # through L2 between two steps of the same layer, so a step finds its cache in HBM):
         # device time of each step alone, by events
@@ -637,7 +646,9 @@ def run_decode(args, B, torch, peaks, source="query", names=("llama32_1b_decode_
             "us_per_step_eager": statistics.median(eager), "us_per_step_graph": graph_us,
             "us_per_step_l2_flushed": flushed_us, "us_per_step_l2_flushed_by_read": flushed_read_us,
             "graph_matches_eager": graph_ok, "steps": w.n_decode,
-            "decode_kernel": "tensor-core scores" if B.delta_state_decode_kernel(st) == 1 else "FP32 pipes", "cache_tokens": w.T, "theta": theta,
+            "decode_kernel": ("FP32 pipes, compressed key-delta cache" if packed else
+                              "tensor-core scores" if B.delta_state_decode_kernel(st) == 1 else "FP32 pipes"),
+            "key_cache_bytes": cache_bytes, "cache_tokens": w.T, "theta": theta,
             "window": w.window, "algorithmic_bytes_per_step": bytes_step,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
                          "frac": gbs / float(peaks["hbm_gbs"]),
@@ -665,7 +676,9 @@ def run_key_deltas(args, B, torch, w, tens, theta, flush, peaks):
     return {"prefill": {"theta": theta, "ms_per_step": statistics.mean(ms),
                         "tokens_per_s": w.B * w.T / (statistics.mean(ms) * 1e-3), "S_m": stt["S_m"],
                         "S_c_exact": stt["S_c_exact"]},
-            "decode": run_decode(args, B, torch, peaks, source="key", names=("llama32_1b_decode_b16",))}
+            "decode": run_decode(args, B, torch, peaks, source="key", names=("llama32_1b_decode_b16",)),
+            "decode_packed_cache": run_decode(args, B, torch, peaks, source="key", names=("llama32_1b_decode_b16",),
+                                              packed=True)}
 
 
 

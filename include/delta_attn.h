@@ -271,10 +271,13 @@ DELTA_API int32_t delta_window_from_gamma(int32_t n, double gamma, int32_t w_max
  *   QHAT_TILE float    [B, H, ceil(T_max/64), d]  reference state before each tile's first row
  *   QHAT      float    [B, H, d]               current reference state
  *   R         float    [B, H, T_max]           current score row (un-scaled), entries 0..n-1
+ *   COUNTERS  uint64   [144]                   raw device counters; word 8 is the device status word
+ *                                              (0, or the DELTA_ERR_* a kernel recorded), which
+ *                                              delta_sparsity_stats reports and returns
  */
 typedef enum {
   DELTA_VIEW_DQ = 0, DELTA_VIEW_MASK = 1, DELTA_VIEW_ROW_NNZ = 2, DELTA_VIEW_TILE_NNZ = 3,
-  DELTA_VIEW_IDX = 4, DELTA_VIEW_QHAT_TILE = 5, DELTA_VIEW_QHAT = 6, DELTA_VIEW_R = 7
+  DELTA_VIEW_IDX = 4, DELTA_VIEW_QHAT_TILE = 5, DELTA_VIEW_QHAT = 6, DELTA_VIEW_R = 7, DELTA_VIEW_COUNTERS = 8
 } delta_view_t;
 DELTA_API delta_status_t delta_state_view(const delta_state_t* st, int32_t what, const void** dev_ptr,
                                 size_t* bytes);
@@ -306,6 +309,27 @@ DELTA_API int32_t delta_state_decode_kernel(const delta_state_t* st);
  * step (the default).  Host-side only. */
 DELTA_API delta_status_t delta_state_set_decode_kernel(delta_state_t* st, int32_t which);
 DELTA_API delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which);
+
+/* Key deltas (DELTA_SRC_KEY, bf16): which form of the thresholded key stream the decode steps
+ * read (Section III-A "Decoding Stage Considerations", Section III-C: the cache holds the key
+ * deltas instead of the keys, plus the last W_d original keys).
+ *   packed = 0 (default): dense rows of reference keys k_hat(j), streamed like a key cache;
+ *   packed = 1: the delta stream itself -- per key row a bit mask of the elements that fired and
+ *     the fired values packed behind one another, the reference key in front of every 32 rows
+ *     and the offsets of those 32-row segments; a decode step rebuilds the reference-key rows of
+ *     a tile in shared memory from that.  The keys inside the decode window are read from
+ *     k_cache.  Same results bit for bit; the bytes a step reads for the keys shrink with the
+ *     delta sparsity (delta_key_cache_bytes), the step itself runs on the FP32 pipes.
+ * Set it on a fresh or reset state (DELTA_ERR_STATE otherwise): the prefill builds the encoding.
+ * The workspace reserves the packed pool for the worst case (every element fires) beside the
+ * dense rows the prefill kernel streams, so the choice changes what decoding reads, not what
+ * delta_state_workspace_bytes asks for. */
+DELTA_API delta_status_t delta_state_set_key_cache(delta_state_t* st, int32_t packed);
+/* Bytes of the packed key-delta encoding in use (values, masks, counts, segment bases and
+ * offsets over all batch elements and KV heads) and of the dense reference-key rows of the
+ * same tokens.  Synchronises `stream`.  DELTA_ERR_UNSUPPORTED unless the packed cache is on. */
+DELTA_API delta_status_t delta_key_cache_bytes(const delta_state_t* st, uint64_t* packed_bytes,
+                                     uint64_t* dense_bytes, void* stream);
 
 /* Per-kernel timing of delta_attn_prefill.  With profiling enabled the call records a CUDA
  * event in front of and behind each of its kernels on the caller's stream (host-side event

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdelta_attn.so")
 SOURCES = ["api.cu", "k1_delta_construct.cu", "k2_hybrid_attn_generic.cu", "k2_hybrid_attn_tc.cu", "k2_hybrid_attn_tcq.cu",
-           "k3_decode_step.cu", "k3_decode_step_tc.cu", "k3_decode_step_key.cu", "decode_noalloc.cu"]
+           "k3_decode_step.cu", "k3_decode_step_tc.cu", "k3_decode_step_key.cu", "k3_decode_step_keypacked.cu", "decode_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
               "-DDELTA_BUILDING_LIB", "-lcuda"]

@@ -23,7 +23,7 @@ DELTA_SRC_QUERY, DELTA_SRC_KEY, DELTA_SRC_QUERY_BOTTOM_UP = 0, 1, 2
 DELTA_WIN_BLOCK, DELTA_WIN_SLIDING = 0, 1
 DELTA_INIT_BASIS_EXACT, DELTA_INIT_ZERO_STATE = 0, 1
 (DELTA_VIEW_DQ, DELTA_VIEW_MASK, DELTA_VIEW_ROW_NNZ, DELTA_VIEW_TILE_NNZ, DELTA_VIEW_IDX,
- DELTA_VIEW_QHAT_TILE, DELTA_VIEW_QHAT, DELTA_VIEW_R) = range(8)
+ DELTA_VIEW_QHAT_TILE, DELTA_VIEW_QHAT, DELTA_VIEW_R, DELTA_VIEW_COUNTERS) = range(9)
 
 EXPORTED = [
     "delta_state_workspace_bytes", "delta_state_init", "delta_state_reset", "delta_state_destroy",
@@ -32,7 +32,7 @@ EXPORTED = [
     "delta_attn_decode_step", "delta_sparsity_stats", "delta_window_from_gamma", "delta_state_view",
     "delta_state_position", "delta_state_prefill_kernel", "delta_state_decode_kernel",
     "delta_state_set_decode_kernel",
-    "delta_state_set_prefill_kernel",
+    "delta_state_set_prefill_kernel", "delta_state_set_key_cache", "delta_key_cache_bytes",
     "delta_launch_count", "delta_status_string", "delta_last_cuda_error",
     "delta_state_enable_profiling", "delta_state_prefill_kernel_ms",
     "delta_attn_decode_step_noalloc", "delta_noalloc_device_status",
@@ -96,6 +96,8 @@ def _load() -> C.CDLL:
         "delta_state_decode_kernel": (i32, [vp]),
         "delta_state_set_decode_kernel": (C.c_int, [vp, i32]),
         "delta_state_set_prefill_kernel": (C.c_int, [vp, i32]),
+        "delta_state_set_key_cache": (C.c_int, [vp, i32]),
+        "delta_key_cache_bytes": (C.c_int, [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), vp]),
         "delta_state_enable_profiling": (C.c_int, [vp, i32]),
         "delta_state_prefill_kernel_ms": (C.c_int, [vp, C.POINTER(C.c_float)]),
         "delta_attn_decode_step_noalloc": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32,
@@ -268,6 +270,17 @@ def delta_state_set_prefill_kernel(st: DeltaState, which: int):
     _check(lib.delta_state_set_prefill_kernel(st.handle, which), "delta_state_set_prefill_kernel")
 
 
+def delta_state_set_key_cache(st: DeltaState, packed: bool):
+    _check(lib.delta_state_set_key_cache(st.handle, int(packed)), "delta_state_set_key_cache")
+
+
+def delta_key_cache_bytes(st: DeltaState, stream=None):
+    """(bytes of the packed key-delta encoding in use, bytes of the dense reference-key rows)."""
+    a, b = C.c_uint64(0), C.c_uint64(0)
+    _check(lib.delta_key_cache_bytes(st.handle, C.byref(a), C.byref(b), _stream(stream)), "delta_key_cache_bytes")
+    return a.value, b.value
+
+
 def delta_state_enable_profiling(st: DeltaState, enable: bool):
     _check(lib.delta_state_enable_profiling(st.handle, int(enable)), "delta_state_enable_profiling")
 
@@ -284,7 +297,7 @@ def delta_launch_count() -> int:
 
 _VIEW_DTYPES = {DELTA_VIEW_DQ: "float32", DELTA_VIEW_MASK: "int32", DELTA_VIEW_ROW_NNZ: "int16",
                 DELTA_VIEW_TILE_NNZ: "int32", DELTA_VIEW_IDX: "uint8", DELTA_VIEW_QHAT_TILE: "float32",
-                DELTA_VIEW_QHAT: "float32", DELTA_VIEW_R: "float32"}
+                DELTA_VIEW_QHAT: "float32", DELTA_VIEW_R: "float32", DELTA_VIEW_COUNTERS: "int64"}
 
 
 def delta_state_view(st: DeltaState, what: int):
@@ -299,5 +312,6 @@ def delta_state_view(st: DeltaState, what: int):
     shapes = {DELTA_VIEW_DQ: (c.B, c.H, c.T_max, c.d), DELTA_VIEW_MASK: (c.B, c.H, c.T_max, c.d // 32),
               DELTA_VIEW_ROW_NNZ: (c.B, c.H, c.T_max), DELTA_VIEW_TILE_NNZ: (c.B, c.H, nt),
               DELTA_VIEW_IDX: (c.B, c.H, c.T_max, c.d), DELTA_VIEW_QHAT_TILE: (c.B, c.H, nt, c.d),
-              DELTA_VIEW_QHAT: (c.B, c.H, c.d), DELTA_VIEW_R: (c.B, c.H, c.T_max)}
+              DELTA_VIEW_QHAT: (c.B, c.H, c.d), DELTA_VIEW_R: (c.B, c.H, c.T_max),
+              DELTA_VIEW_COUNTERS: (n.value // 8,)}
     return raw.view(getattr(torch, _VIEW_DTYPES[what])).view(shapes[what])

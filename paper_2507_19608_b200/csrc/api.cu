@@ -6,6 +6,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "delta_internal.cuh"
 #include "k2_tc.cuh"
 
@@ -20,6 +22,14 @@ delta_status_t cuda_fail(cudaError_t e) {
 }  // namespace delta
 
 using namespace delta;
+
+// NVTX range over an entry point (shows up in a timeline profiler; free when none is attached).
+namespace {
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
+}  // namespace
 
 struct delta_state {
   delta_config_t cfg;
@@ -38,6 +48,7 @@ struct delta_state {
   DecodeTmapCache dec_tmap;   // tensor map of the key cache the decode steps read
   DecodeTmapCache dec_tmap_h; // and of the reference-key cache (key deltas)
   int forced_decode_kernel = -1;   // -1: chosen per step
+  bool key_cache_packed = false;   // key deltas: decode from the compressed key-delta cache
   // optional per-kernel timing of prefill (host-side event objects)
   bool profiling = false, profiled = false;
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -97,6 +108,19 @@ static void carve(const delta_config_t& c, char* base, Workspace* w) {
               ? (float*)take(BKV * c.d * (((size_t)c.T_max + 3) / 4 * 4) * 4) : nullptr;
   w->qhat_rows = (c.dtype == DELTA_BF16 && tcq_kernel_shape(c.d))
                      ? (__nv_bfloat16*)take(BH * c.T_max * c.d * 2) : nullptr;
+  if (c.source == DELTA_SRC_KEY && c.dtype == DELTA_BF16) {
+    // compressed key-delta cache: sized for the worst case (every element fires)
+    const size_t nseg = (size_t)keypack_segments(c.T_max);
+    w->kp_vals = (uint16_t*)take(BKV * keypack_capacity(c.T_max, c.d) * 2);
+    w->kp_segoff = (uint32_t*)take(BKV * (nseg + 1) * 4);
+    w->kp_base = (uint16_t*)take(BKV * nseg * c.d * 2);
+    w->kp_used = (uint32_t*)take(BKV * 4);
+    w->kp_mask = (uint32_t*)take(BKV * nseg * 32 * (c.d / 32) * 4);
+    w->kp_nnz = (uint16_t*)take(BKV * nseg * 32 * 2);
+  } else {
+    w->kp_vals = nullptr; w->kp_segoff = nullptr; w->kp_base = nullptr; w->kp_used = nullptr;
+    w->kp_mask = nullptr; w->kp_nnz = nullptr;
+  }
   w->total_bytes = off;
 }
 
@@ -225,6 +249,39 @@ delta_status_t delta_state_set_decode_kernel(delta_state_t* st, int32_t which) {
   return DELTA_OK;
 }
 
+delta_status_t delta_state_set_key_cache(delta_state_t* st, int32_t packed) {
+  if (!st || packed < 0 || packed > 1) return DELTA_ERR_INVALID_ARG;
+  if (st->cfg.source != DELTA_SRC_KEY || !st->ws.kp_vals) return DELTA_ERR_UNSUPPORTED;
+  if (st->n != 0) return DELTA_ERR_STATE;      // the encoding is built by the prefill
+  st->key_cache_packed = packed != 0;
+  return DELTA_OK;
+}
+
+delta_status_t delta_key_cache_bytes(const delta_state_t* st, uint64_t* packed_bytes, uint64_t* dense_bytes,
+                                     void* stream) {
+  if (!st || !packed_bytes || !dense_bytes) return DELTA_ERR_INVALID_ARG;
+  const delta_config_t& c = st->cfg;
+  if (c.source != DELTA_SRC_KEY || !st->ws.kp_vals || !st->key_cache_packed) return DELTA_ERR_UNSUPPORTED;
+  const size_t bkv = (size_t)c.B * c.H_kv;
+  std::vector<uint32_t> used(bkv);
+  cudaError_t e = cudaMemcpyAsync(used.data(), st->ws.kp_used, bkv * 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaStreamSynchronize((cudaStream_t)stream)) != cudaSuccess) return cuda_fail(e);
+  uint64_t packed = 0, dense = 0;
+  for (int b = 0; b < c.B; ++b) {
+    const uint64_t rows = (uint64_t)st->n_b[(size_t)b], segs = (rows + 31) / 32;
+    for (int h = 0; h < c.H_kv; ++h)
+      packed += 2ull * used[(size_t)b * c.H_kv + h]            // values (with the segments' padding)
+                + rows * (uint64_t)(c.d / 8)                    // mask words
+                + rows * 2                                      // fired counts
+                + segs * (uint64_t)c.d * 2 + (segs + 1) * 4;    // segment bases and offsets
+    dense += (uint64_t)c.H_kv * rows * (uint64_t)c.d * 2;
+  }
+  *packed_bytes = packed;
+  *dense_bytes = dense;
+  return DELTA_OK;
+}
+
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
   if (!st || which < -1 || which > 2) return DELTA_ERR_INVALID_ARG;
   if (which >= 1 && !tc_eligible(st, which)) return DELTA_ERR_UNSUPPORTED;
@@ -265,6 +322,15 @@ static void view_of(const delta_state* st, int b, Shape* sh, Workspace* w) {
   w->dec_ticket += ub * c.H_kv;
   if (w->kt) w->kt += ub * c.H_kv * c.d * (((size_t)c.T_max + 3) / 4 * 4);
   if (w->qhat_rows) w->qhat_rows += ub * Hs * c.T_max * c.d;
+  if (w->kp_vals) {
+    const size_t nseg = (size_t)keypack_segments(c.T_max);
+    w->kp_vals += ub * c.H_kv * keypack_capacity(c.T_max, c.d);
+    w->kp_segoff += ub * c.H_kv * (nseg + 1);
+    w->kp_base += ub * c.H_kv * nseg * c.d;
+    w->kp_used += ub * c.H_kv;
+    w->kp_mask += ub * c.H_kv * nseg * 32 * (c.d / 32);
+    w->kp_nnz += ub * c.H_kv * nseg * 32;
+  }
 }
 
 // The three kernels of a prefill over one view (the whole batch, or one batch element).
@@ -318,6 +384,8 @@ static delta_status_t prefill_launch(delta_state* st, const Shape& shape, const 
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
   }
   MARK(3);
+  // key deltas with the compressed cache: encode the key stream behind everything it is built from
+  if (key && st->key_cache_packed && (e = launch_pack_keys(shape, ws, k, T, cs)) != cudaSuccess) return cuda_fail(e);
   MARK(4);
 #undef MARK
   return DELTA_OK;
@@ -328,6 +396,7 @@ extern "C" {
 delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* k, const void* v,
                                   void* out, int32_t T, int32_t H, int32_t H_kv, int32_t d,
                                   float theta, int32_t window, void* stream) {
+  NvtxRange range("delta_attn_prefill");
   if (!st || !q || !k || !v || !out) return DELTA_ERR_INVALID_ARG;
   if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return DELTA_ERR_INVALID_ARG;
   const delta_config_t& c = st->cfg;
@@ -353,6 +422,7 @@ delta_status_t delta_attn_prefill(delta_state_t* st, const void* q, const void* 
 delta_status_t delta_attn_prefill_varlen(delta_state_t* st, const void* q, const void* k, const void* v,
                                          void* out, const int32_t* seq_lens, const int32_t* windows,
                                          float theta, void* stream) {
+  NvtxRange range("delta_attn_prefill_varlen");
   if (!st || !q || !k || !v || !out || !seq_lens || !windows) return DELTA_ERR_INVALID_ARG;
   if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15u) != 0) return DELTA_ERR_INVALID_ARG;
   const delta_config_t& c = st->cfg;
@@ -455,6 +525,9 @@ static cudaError_t decode_launch(delta_state* st, const Shape& shape, const Work
   const bool tcs = decode_tc_possible(st) &&
                    (st->forced_decode_kernel >= 0 ? st->forced_decode_kernel == 1
                                                   : decode_tc_applies(shape, st->cfg.dtype, n));
+  if (st->cfg.source == DELTA_SRC_KEY && st->key_cache_packed)
+    return launch_decode_step_keypacked(shape, ws, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window,
+                                        st->qhat_sel, cs);
   if (st->cfg.source == DELTA_SRC_KEY)
     return tcs ? launch_decode_step_key_tc(shape, ws, q_new, k_new, v_new, k_cache, v_cache, out, n, theta, window,
                                            st->qhat_sel, tmap, tmap_h, cs)
@@ -471,6 +544,7 @@ extern "C" {
 delta_status_t delta_attn_decode_step(delta_state_t* st, const void* q_new, const void* k_new,
                                       const void* v_new, void* k_cache, void* v_cache, void* out,
                                       float theta, int32_t window, void* stream) {
+  NvtxRange range("delta_attn_decode_step");
   if (!st || !q_new || !k_new || !v_new || !k_cache || !v_cache || !out) return DELTA_ERR_INVALID_ARG;
   // every decode kernel stages cache tiles with bulk copies and reads rows as 16-byte vectors
   if ((((uintptr_t)q_new | (uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache | (uintptr_t)v_cache |
@@ -524,6 +598,7 @@ static void finish_stage(delta_stage_stats_t* o, const unsigned long long* c, do
 }
 
 delta_status_t delta_sparsity_stats(const delta_state_t* st, delta_stats_t* host_out, void* stream) {
+  NvtxRange range("delta_sparsity_stats");
   if (!st || !host_out) return DELTA_ERR_INVALID_ARG;
   unsigned long long c[CNT_TOTAL];
   cudaError_t e = cudaMemcpyAsync(c, st->ws.counters, sizeof(c), cudaMemcpyDeviceToHost,
@@ -569,6 +644,7 @@ delta_status_t delta_state_view(const delta_state_t* st, int32_t what, const voi
     case DELTA_VIEW_QHAT_TILE: *dev_ptr = st->ws.qhat_tile; *bytes = BH * nt * c.d * 4; break;
     case DELTA_VIEW_QHAT: *dev_ptr = st->ws.qhat[st->qhat_sel]; *bytes = BH * c.d * 4; break;
     case DELTA_VIEW_R: *dev_ptr = st->ws.R; *bytes = BH * c.T_max * 4; break;
+    case DELTA_VIEW_COUNTERS: *dev_ptr = st->ws.counters; *bytes = (size_t)CNT_TOTAL * 8; break;
     default: return DELTA_ERR_INVALID_ARG;
   }
   return DELTA_OK;

@@ -40,6 +40,14 @@ struct Workspace {
   uint32_t* dec_ticket; // [B,H_kv]
   float* kt;            // [B,H_kv,d,round_up(T_max,4)] channel-major fp32 keys (tensor-core prefill only)
   __nv_bfloat16* qhat_rows;  // [B,H,T_max,d] reference state after every row (telescoped prefill only)
+  // compressed key-delta cache (key deltas, bf16): values, segment offsets, segment bases, pool
+  // fill per KV head, and its own 32-row-aligned copies of the mask words and fired counts
+  uint16_t* kp_vals;    // [B,H_kv,capacity]
+  uint32_t* kp_segoff;  // [B,H_kv,segments+1]
+  uint16_t* kp_base;    // [B,H_kv,segments,d]
+  uint32_t* kp_used;    // [B,H_kv]
+  uint32_t* kp_mask;    // [B,H_kv,segments*32,d/32]
+  uint16_t* kp_nnz;     // [B,H_kv,segments*32]
   size_t zero_bytes;    // leading span of the workspace that a reset clears (q_hat, counters, tickets)
   size_t total_bytes;
 };
@@ -96,6 +104,14 @@ cudaError_t launch_decode_step_key_tc(const Shape& s, const Workspace& w, const 
                                       const void* v_new, void* k_cache, void* v_cache, void* out, int n,
                                       float theta, int window, int qhat_sel, DecodeTmapCache* cache_k,
                                       DecodeTmapCache* cache_h, cudaStream_t st);
+// K3 (key deltas) from the compressed key-delta cache, the kernel that builds that cache behind a
+// prefill, and its geometry (values per KV head at most, 32-row segments).
+size_t keypack_capacity(int T_max, int d);
+int keypack_segments(int T_max);
+cudaError_t launch_pack_keys(const Shape& s, const Workspace& w, const void* k, int T, cudaStream_t st);
+cudaError_t launch_decode_step_keypacked(const Shape& s, const Workspace& w, const void* q_new, const void* k_new,
+                                         const void* v_new, void* k_cache, void* v_cache, void* out, int n,
+                                         float theta, int window, int qhat_sel, cudaStream_t st);
 cudaError_t launch_decode_step_key(const Shape& s, const Workspace& w, const void* q_new,
                                    const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                    void* out, int n, float theta, int window, int qhat_sel,

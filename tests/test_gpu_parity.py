@@ -308,6 +308,26 @@ def test_decode_steps_match_oracle(B, Bn, H, Hk, T, d, dtype, theta, W, steps, d
             assert stats[name][key] == pytest.approx(want[key], abs=1e-12), (name, key)
 
 
+# ------------------------------------------------------------------ device status word -> host
+def test_device_status_word_reaches_the_host(B):
+    """A kernel whose bounded wait runs out records DELTA_ERR_TIMEOUT in the device status word.
+    No wait is made to run out here: the word is written by the host, through the counters view,
+    and delta_sparsity_stats must report it (return value and device_status) until a reset."""
+    from tests.gpu_helpers import run_prefill
+    q, k, v = _inputs(1, 2, 1, 40, 64, "bf16", seed=2)
+    st, out, _, _ = run_prefill(B, q, k, v, 0.1, 8, "bf16")
+    assert B.delta_sparsity_stats(st)["device_status"] == 0
+    counters = B.delta_state_view(st, B.DELTA_VIEW_COUNTERS)
+    assert counters.numel() == 144
+    counters[8] = B.DELTA_ERR_TIMEOUT
+    torch.cuda.synchronize()
+    with pytest.raises(B.DeltaError) as e:
+        B.delta_sparsity_stats(st)
+    assert e.value.status == B.DELTA_ERR_TIMEOUT
+    B.delta_state_reset(st)
+    assert B.delta_sparsity_stats(st)["device_status"] == 0
+
+
 # ------------------------------------------------------------------ call-order and capacity errors
 def test_state_errors(B):
     from tests.gpu_helpers import run_prefill, to_dev
@@ -526,10 +546,12 @@ def test_key_delta_prefill_matches_oracle(B, case):
     (3, 4, 4, 1500, 64, 0.2, 300, 2),      # window over three tiles: key-cache tiles, one mixed tile
     (40, 4, 4, 1100, 64, 0.2, 64, 2),      # 160 KV heads: one slice of 9 tiles per head
 ])
-@pytest.mark.parametrize("decode_kernel", [0, 1], ids=["fp32_pipes", "tc_scores"])
+@pytest.mark.parametrize("decode_kernel", [0, 1, 2], ids=["fp32_pipes", "tc_scores", "packed_cache"])
 def test_key_delta_decode_steps_match_oracle(B, Bn, H, Hk, T, d, theta, W, steps, decode_kernel):
     """Strategy (3) carried into decoding: the reference key per KV head is the carried state,
-    old keys are scored through the reference-key rows, the W_d most recent ones exactly."""
+    old keys are scored through the reference-key rows, the W_d most recent ones exactly.
+    packed_cache: the reference-key rows are rebuilt from the compressed key-delta cache (mask,
+    packed fired values, segment bases), which the prefill builds and every step extends."""
     from tests.gpu_helpers import to_cache, to_dev, to_host_f64
     w = WL.Workload("t", Bn, H, Hk, T, d, "bf16", 0.95, 0.5, W, (), 500 + T, n_decode=steps)
     t = WL.make_qkv(w)
@@ -538,8 +560,12 @@ def test_key_delta_decode_steps_match_oracle(B, Bn, H, Hk, T, d, theta, W, steps
     st = B.delta_state_init(cfg)
     if decode_kernel == 1 and d != 64:
         pytest.skip("tensor-core decode scores: d = 64")
-    B.delta_state_set_decode_kernel(st, decode_kernel)
-    assert B.delta_state_decode_kernel(st) == decode_kernel
+    packed = decode_kernel == 2
+    if packed:
+        B.delta_state_set_key_cache(st, True)
+    else:
+        B.delta_state_set_decode_kernel(st, decode_kernel)
+        assert B.delta_state_decode_kernel(st) == decode_kernel
     dq_, kc, vc = to_dev(t["q"], "bf16"), to_cache(t["k"], T_max, "bf16"), to_cache(t["v"], T_max, "bf16")
     out = torch.full_like(dq_, float("nan"))
     B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, float(theta), int(W))
@@ -572,6 +598,23 @@ def test_key_delta_decode_steps_match_oracle(B, Bn, H, Hk, T, d, theta, W, steps
     assert sd["device_status"] == 0
     sd = sd["decode"]
     assert (sd["nnz"], sd["elements"], sd["macs_done"], sd["macs_dense"]) == (nnz, Bn * Hk * d * steps, done, dense)
+    if packed:
+        # bytes of the encoding in use: values (2 bytes per fired element, segments padded to 8
+        # values), mask words, counts, segment bases and offsets -- recounted from the oracle's masks
+        got_packed, got_dense = B.delta_key_cache_bytes(st)
+        n_tok = T + steps
+        want = 0
+        for key in states:
+            rn = row_nnz[key]
+            vals = 0
+            for s0 in range(0, n_tok, 32):
+                seg = int(sum(rn[s0:s0 + 32]))
+                vals = (vals + 7) // 8 * 8 if s0 else 0        # a segment starts on a multiple of 8 values
+                vals += seg
+            segs = (n_tok + 31) // 32
+            want += 2 * vals + n_tok * (d // 8) + n_tok * 2 + segs * d * 2 + (segs + 1) * 4
+        assert got_dense == Bn * Hk * n_tok * d * 2
+        assert got_packed == want
 
 
 # ------------------------------------------------------------------ strategy (2): bottom-up query deltas
@@ -727,7 +770,7 @@ def test_two_states_on_two_streams_match_the_default_stream(B):
 
 # ------------------------------------------------------------------ long decode runs
 @pytest.mark.parametrize("source", ["query", "key"])
-@pytest.mark.parametrize("decode_kernel", [0, 1], ids=["fp32_pipes", "tc_scores"])
+@pytest.mark.parametrize("decode_kernel", [0, 1, 2], ids=["fp32_pipes", "tc_scores", "packed_cache"])
 def test_long_decode_run_crosses_tile_and_slice_boundaries(B, source, decode_kernel):
     """300 decode steps from a 100-token prompt: the cache grows across three 128-key tile
     boundaries and the number of key slices per head changes on the way; every step's output is
@@ -741,7 +784,12 @@ def test_long_decode_run_crosses_tile_and_slice_boundaries(B, source, decode_ker
     cfg = B.make_config(Bn, H, Hk, d, T_max, dtype, prefill_window=B.DELTA_WIN_SLIDING,
                         source=B.DELTA_SRC_KEY if source == "key" else B.DELTA_SRC_QUERY)
     st = B.delta_state_init(cfg)
-    B.delta_state_set_decode_kernel(st, decode_kernel)
+    if decode_kernel == 2:
+        if source != "key":
+            pytest.skip("the compressed cache belongs to key deltas")
+        B.delta_state_set_key_cache(st, True)
+    else:
+        B.delta_state_set_decode_kernel(st, decode_kernel)
     dq_, kc, vc = to_dev(t["q"], dtype), to_cache(t["k"], T_max, dtype), to_cache(t["v"], T_max, dtype)
     out = torch.full_like(dq_, float("nan"))
     B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, theta, W)
