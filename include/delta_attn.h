@@ -52,7 +52,9 @@ typedef enum {
   DELTA_ERR_STATE = 5,        /* call order: prefill on a used state, decode before prefill    */
   DELTA_ERR_CUDA = 6,         /* a CUDA runtime call failed (delta_last_cuda_error has it)     */
   DELTA_ERR_TIMEOUT = 7,      /* a bounded device-side wait ran out (status word on device)    */
-  DELTA_ERR_SCRATCH_LIMIT = 8 /* problem larger than the built-in scratch of the no-alloc call */
+  DELTA_ERR_SCRATCH_LIMIT = 8, /* problem larger than the built-in scratch of the no-alloc call */
+  DELTA_ERR_BOUNDS = 9        /* bounds-checking build only: a kernel formed an index outside its
+                                 array; the access was skipped and the status word records it    */
 } delta_status_t;
 
 typedef enum { DELTA_F32 = 0, DELTA_BF16 = 1 } delta_dtype_t;
@@ -340,6 +342,13 @@ DELTA_API delta_status_t delta_key_cache_bytes(const delta_state_t* st, uint64_t
  * DELTA_ERR_STATE if profiling is off or no prefill was recorded. */
 DELTA_API delta_status_t delta_state_enable_profiling(delta_state_t* st, int32_t enable);
 DELTA_API delta_status_t delta_state_prefill_kernel_ms(delta_state_t* st, float* ms);
+
+/* 1 if this library was built with -DDELTA_DEBUG_BOUNDS: every global index the kernels compute
+ * by hand is range-checked against the extent of its array, an index out of range is not
+ * accessed and DELTA_ERR_BOUNDS goes to the device status word (delta_sparsity_stats reports it).
+ * 0 for the regular build, whose kernels carry no such checks.  (Tile copies by TMA are
+ * bounded by their tensor maps in both builds.) */
+DELTA_API int32_t delta_debug_bounds_build(void);
 
 /* Kernels launched by this library in the calling process since it was loaded. */
 DELTA_API uint64_t delta_launch_count(void);

@@ -17,7 +17,7 @@ DELTA_TILE_ROWS = 64
 # enums (values of include/delta_attn.h)
 DELTA_OK = 0
 DELTA_ERR_INVALID_ARG, DELTA_ERR_UNSUPPORTED, DELTA_ERR_WORKSPACE, DELTA_ERR_CAPACITY = 1, 2, 3, 4
-DELTA_ERR_STATE, DELTA_ERR_CUDA, DELTA_ERR_TIMEOUT, DELTA_ERR_SCRATCH_LIMIT = 5, 6, 7, 8
+DELTA_ERR_STATE, DELTA_ERR_CUDA, DELTA_ERR_TIMEOUT, DELTA_ERR_SCRATCH_LIMIT, DELTA_ERR_BOUNDS = 5, 6, 7, 8, 9
 DELTA_F32, DELTA_BF16 = 0, 1
 DELTA_SRC_QUERY, DELTA_SRC_KEY, DELTA_SRC_QUERY_BOTTOM_UP = 0, 1, 2
 DELTA_WIN_BLOCK, DELTA_WIN_SLIDING = 0, 1
@@ -33,7 +33,7 @@ EXPORTED = [
     "delta_state_position", "delta_state_prefill_kernel", "delta_state_decode_kernel",
     "delta_state_set_decode_kernel",
     "delta_state_set_prefill_kernel", "delta_state_set_key_cache", "delta_key_cache_bytes",
-    "delta_launch_count", "delta_status_string", "delta_last_cuda_error",
+    "delta_launch_count", "delta_status_string", "delta_last_cuda_error", "delta_debug_bounds_build",
     "delta_state_enable_profiling", "delta_state_prefill_kernel_ms",
     "delta_attn_decode_step_noalloc", "delta_noalloc_device_status",
 ]
@@ -73,7 +73,9 @@ class DeltaError(RuntimeError):
 
 
 def _load() -> C.CDLL:
-    path = _build.build()          # raises if nvcc or the sources are missing
+    # DELTA_ATTN_DEBUG_BOUNDS=1 selects the bounds-checking build of the library
+    debug = os.environ.get("DELTA_ATTN_DEBUG_BOUNDS", "") not in ("", "0")
+    path = _build.build(debug_bounds=debug)          # raises if nvcc or the sources are missing
     l = C.CDLL(path)
     vp, i32, f32, sz = C.c_void_p, C.c_int32, C.c_float, C.c_size_t
     cfgp = C.POINTER(delta_config_t)
@@ -104,6 +106,7 @@ def _load() -> C.CDLL:
                                                      i32, i32, C.c_int, f32, i32, vp]),
         "delta_noalloc_device_status": (C.c_int, [C.POINTER(C.c_uint32), vp]),
         "delta_launch_count": (C.c_uint64, []),
+        "delta_debug_bounds_build": (i32, []),
         "delta_status_string": (C.c_char_p, [C.c_int]),
         "delta_last_cuda_error": (C.c_char_p, []),
     }
@@ -115,7 +118,7 @@ def _load() -> C.CDLL:
 
 
 lib = _load()
-LIB_PATH = _build.LIB
+LIB_PATH = _build.LIB_DEBUG if lib.delta_debug_bounds_build() else _build.LIB
 
 
 def _check(status: int, where: str):

@@ -650,6 +650,14 @@ delta_status_t delta_state_view(const delta_state_t* st, int32_t what, const voi
   return DELTA_OK;
 }
 
+int32_t delta_debug_bounds_build(void) {
+#ifdef DELTA_DEBUG_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
+}
+
 uint64_t delta_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* delta_status_string(delta_status_t s) {
@@ -662,6 +670,7 @@ const char* delta_status_string(delta_status_t s) {
     case DELTA_ERR_STATE: return "call order: state not in the required condition";
     case DELTA_ERR_CUDA: return "CUDA runtime error";
     case DELTA_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case DELTA_ERR_BOUNDS: return "index out of range in a kernel (bounds-checking build)";
     case DELTA_ERR_SCRATCH_LIMIT:
       return "problem larger than the built-in scratch of delta_attn_decode_step_noalloc";
   }

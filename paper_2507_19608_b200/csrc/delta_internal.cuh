@@ -117,6 +117,22 @@ cudaError_t launch_decode_step_key(const Shape& s, const Workspace& w, const voi
                                    void* out, int n, float theta, int window, int qhat_sel,
                                    cudaStream_t st);
 
+// ---- bounds-checking build ------------------------------------------------------------
+// DELTA_IN(index, extent, counters) guards a global access whose index a kernel computed by
+// hand: true in the regular build (the guard compiles away); in a -DDELTA_DEBUG_BOUNDS build
+// false for an index outside [0, extent), with DELTA_ERR_BOUNDS recorded in the status word, so
+// the access is skipped instead of made (no trap, no assert: the context stays usable).
+#ifdef DELTA_DEBUG_BOUNDS
+__device__ __forceinline__ bool delta_in_bounds(size_t idx, size_t extent, unsigned long long* counters) {
+  if (idx < extent) return true;
+  atomicMax(&counters[CNT_STATUS], (unsigned long long)DELTA_ERR_BOUNDS);
+  return false;
+}
+#define DELTA_IN(idx, extent, counters) delta_in_bounds((size_t)(idx), (size_t)(extent), (counters))
+#else
+#define DELTA_IN(idx, extent, counters) true
+#endif
+
 // ---- small device helpers -------------------------------------------------------------
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }

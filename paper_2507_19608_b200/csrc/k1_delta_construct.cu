@@ -47,7 +47,7 @@ template <> __device__ __forceinline__ float lds_elem<__nv_bfloat16>(uint32_t ad
 // 8-row block (ckptp).  basis_row: the stage's first row is the un-thresholded basis.
 template <typename TIn, int D>
 __device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, bool basis_row, float& qh,
-                                            float theta, float* ckptp) {
+                                            float theta, float* ckptp, int n_ckpt, unsigned long long* counters) {
   if (nrows == RC && !basis_row) {
     // full stage, no basis row: nothing but loads, the dependent chain and the checkpoints
     float x[RC];
@@ -56,14 +56,16 @@ __device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, 
     for (int r = 0; r < RC; ++r) x[r] = lds_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
 #pragma unroll
     for (int r = 0; r < RC; ++r) {
-      if ((r % DELTA_CKPT_ROWS) == 0) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      if ((r % DELTA_CKPT_ROWS) == 0 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
+        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
       const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
       const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
       qh = fire ? x[r] : qh;
     }
   } else {
     for (int r = 0; r < nrows; ++r) {
-      if (((t0 + r) % DELTA_CKPT_ROWS) == 0) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      if (((t0 + r) % DELTA_CKPT_ROWS) == 0 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
+        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
       const float x = to_f32(rows[r * D]);
       const bool fire = (r == 0 && basis_row) || (fabsf(__fsub_rn(x, qh)) > theta);
       qh = fire ? x : qh;
@@ -76,7 +78,7 @@ __device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, 
 // basis_last: the stage's last row is row T-1, the un-thresholded basis of this order.
 template <typename TIn, int D>
 __device__ __forceinline__ void chain_stage_rev(const TIn* rows, int t0, int nrows, bool basis_last, float& qh,
-                                                float theta, float* ckptp) {
+                                                float theta, float* ckptp, int n_ckpt, unsigned long long* counters) {
   if (nrows == RC && !basis_last) {
     float x[RC];
     const uint32_t saddr = smem_u32(rows);
@@ -84,14 +86,16 @@ __device__ __forceinline__ void chain_stage_rev(const TIn* rows, int t0, int nro
     for (int r = 0; r < RC; ++r) x[r] = lds_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
 #pragma unroll
     for (int r = RC - 1; r >= 0; --r) {
-      if ((r % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1) ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      if ((r % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
+        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
       const float diff = __fsub_rn(x[r], qh);
       const bool fire = fabsf(diff) > theta;
       qh = fire ? x[r] : qh;
     }
   } else {
     for (int r = nrows - 1; r >= 0; --r) {
-      if (((t0 + r) % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 || r == nrows - 1)
+      if ((((t0 + r) % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 || r == nrows - 1) &&
+          DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
         ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
       const float x = to_f32(rows[r * D]);
       const bool fire = (r == nrows - 1 && basis_last) || (fabsf(__fsub_rn(x, qh)) > theta);
@@ -146,6 +150,8 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
         const int ci = reverse ? n_chunks - 1 - i : i;      // stage of the head in token order
         const int rows = min(RC, T - ci * RC);
         const uint32_t bytes = (uint32_t)rows * ROW_BYTES;
+        // (bounds-checking build: the stage's rows lie inside the head's rows of the stream)
+        if (!DELTA_IN((size_t)ci * RC + rows - 1, src_rows, counters)) { s_fail = 1; break; }
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full0 + 8 * s),
                      "r"(bytes)
                      : "memory");
@@ -165,15 +171,15 @@ __global__ void __launch_bounds__(D + 32) delta_chain_kernel(
     for (int i = 0; i < n_chunks; ++i) {
       const int s = i % NS;
       const int t0 = (reverse ? n_chunks - 1 - i : i) * RC;
-      if (qhat_tile && (t0 % DELTA_TILE_ROWS) == 0)
+      if (qhat_tile && (t0 % DELTA_TILE_ROWS) == 0 && DELTA_IN(t0 / DELTA_TILE_ROWS, n_tiles, counters))
         qhat_tile[((size_t)bh * n_tiles + t0 / DELTA_TILE_ROWS) * D + c] = qh;
       if (!mbar_wait(full0 + 8 * s, (i / NS) & 1)) { failed = true; break; }
       const TIn* rows = reinterpret_cast<const TIn*>(ring + (size_t)s * STAGE_BYTES) + c;
       const int nrows = min(RC, T - t0);
       if (reverse)
-        chain_stage_rev<TIn, D>(rows, t0, nrows, t0 + nrows == T && basis_exact, qh, theta, ckptp);
+        chain_stage_rev<TIn, D>(rows, t0, nrows, t0 + nrows == T && basis_exact, qh, theta, ckptp, n_ckpt, counters);
       else
-        chain_stage<TIn, D>(rows, t0, nrows, t0 == 0 && basis_exact, qh, theta, ckptp);
+        chain_stage<TIn, D>(rows, t0, nrows, t0 == 0 && basis_exact, qh, theta, ckptp, n_ckpt, counters);
       __syncwarp();
       if (lane == 0)
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * s) : "memory");
@@ -260,7 +266,8 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
       for (int w2 = 0; w2 < NW; ++w2) {
         const int c = w2 * 32 + lane;
         uint32_t word_mine = 0;
-        if (rbase < T) {
+        if (rbase < T && DELTA_IN(rbase / DELTA_CKPT_ROWS, n_ckpt, counters) && DELTA_IN(rbase + 7 < T ? rbase + 7 : T - 1, src_rows, counters) &&
+            DELTA_IN(T - 1, T_max, counters)) {
           float ref = ckpt[((size_t)bh * n_ckpt + rbase / DELTA_CKPT_ROWS) * D + c];
           float x[8];
 #pragma unroll
@@ -295,7 +302,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
       }
     }
     unsigned long long done = 0, dense = 0, tsum = 0;
-    if (lane < 8 && r_mine < rows) {
+    if (lane < 8 && r_mine < rows && DELTA_IN(t0 + r_mine, T_max, counters)) {
       int nnz = 0;
 #pragma unroll
       for (int w2 = 0; w2 < NW; ++w2) nnz += __popc(mw[w2]);
@@ -355,7 +362,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
     if (tid == 0) {
       unsigned long long a = 0, b2 = 0, c2 = 0;
       for (int w2 = 0; w2 < 8; ++w2) { a += s_red[0][w2]; b2 += s_red[1][w2]; c2 += s_red[2][w2]; }
-      tile_nnz[(size_t)bh * n_tiles + tile] = (uint32_t)a;
+      if (DELTA_IN(tile, n_tiles, counters)) tile_nnz[(size_t)bh * n_tiles + tile] = (uint32_t)a;
       unsigned long long* cs = counters + CNT_SHARD_BASE + 4 * (blockIdx.x % CNT_SHARDS);
       atomicAdd(&cs[0], a);
       atomicAdd(&cs[1], (unsigned long long)rows * D);
@@ -408,7 +415,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
       float acc = 0.0f;
 #pragma unroll 8
       for (int c = 0; c < D; ++c) acc = fmaf(qh[hh][c], tile[c][j], acc);
-      if (j0 + j < T) R[((size_t)b * H + kvh * g + hh) * T_max + j0 + j] = acc;
+      if (j0 + j < T && DELTA_IN(j0 + j, T_max, counters)) R[((size_t)b * H + kvh * g + hh) * T_max + j0 + j] = acc;
     }
   }
 }

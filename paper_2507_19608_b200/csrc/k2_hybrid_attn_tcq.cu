@@ -389,7 +389,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
       for (int bk = 0; bk < NBK; ++bk) {
         const int r0 = i0 + seg * SEG + bk * DELTA_CKPT_ROWS;
-        ref[bk] = (r0 < T) ? p.ckpt[((size_t)bh * p.n_ckpt + r0 / DELTA_CKPT_ROWS) * D + c] : 0.0f;
+        ref[bk] = (r0 < T && DELTA_IN(r0 / DELTA_CKPT_ROWS, p.n_ckpt, p.counters))
+                      ? p.ckpt[((size_t)bh * p.n_ckpt + r0 / DELTA_CKPT_ROWS) * D + c] : 0.0f;
       }
       mbar_wait(BAR(BAR_Q), 0, abort_flag);      // the query tile has landed
 #pragma unroll
@@ -646,7 +647,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const float a_me = ex2(m_used - m_all), a_o = ex2(m_o - m_all);     // ex2(-inf) = 0 for an empty group
     const float inv = 1.0f / (l_sum * a_me + l_o * a_o);
     const float f_me = a_me * inv, f_o = a_o * inv;
-    const bool store = (i < T) && !*abort_flag;
+    const bool store = (i < T) && !*abort_flag && DELTA_IN(i, T, p.counters);
 #pragma unroll
     for (int ch = 0; ch < HC / 32; ++ch) {
       uint32_t u[32];

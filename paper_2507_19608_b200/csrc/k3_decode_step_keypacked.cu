@@ -32,7 +32,8 @@ __global__ void __launch_bounds__(256) pack_keys_kernel(
     const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ khat_rows,
     const uint32_t* __restrict__ mask, const uint16_t* __restrict__ row_nnz, uint16_t* __restrict__ vals,
     uint32_t* __restrict__ seg_off, uint16_t* __restrict__ base, uint32_t* __restrict__ used,
-    uint32_t* __restrict__ kp_mask, uint16_t* __restrict__ kp_nnz, int T, int T_max, size_t cap, int nseg_max) {
+    uint32_t* __restrict__ kp_mask, uint16_t* __restrict__ kp_nnz, int T, int T_max, size_t cap, int nseg_max,
+    unsigned long long* __restrict__ counters) {
   constexpr int NW = D / 32;
   extern __shared__ uint32_t s_off[];          // [nseg + 1]
   const int bkv = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -81,7 +82,7 @@ __global__ void __launch_bounds__(256) pack_keys_kernel(
 #pragma unroll
       for (int w = 0; w < NW; ++w) {
         const uint32_t word = mk[(size_t)row * NW + w];
-        if ((word >> lane) & 1u)
+        if (((word >> lane) & 1u) && DELTA_IN(off + below + __popc(word & ((1u << lane) - 1u)), cap, counters))
           vp[off + below + __popc(word & ((1u << lane) - 1u))] =
               reinterpret_cast<const uint16_t*>(kp)[(size_t)row * D + w * 32 + lane];
         below += __popc(word);
@@ -184,14 +185,15 @@ __global__ void __launch_bounds__(DNT) decode_step_keypacked_kernel(
       if (fire) {
         uint32_t rank = __popc(s_words[tid >> 5] & ((1u << (tid & 31)) - 1u));
         for (int w = 0; w < (tid >> 5); ++w) rank += __popc(s_words[w]);
-        vals_g[pos + rank] = reinterpret_cast<const uint16_t*>(k_new)[(size_t)bkv * D + tid];
+        if (DELTA_IN(pos + rank, cap, counters))
+          vals_g[pos + rank] = reinterpret_cast<const uint16_t*>(k_new)[(size_t)bkv * D + tid];
       }
       if (tid < NW) {
         mask[((size_t)bkv * T_max + n) * NW + tid] = s_words[tid];
         kp_mask[((size_t)bkv * nseg_max * SEG + n) * NW + tid] = s_words[tid];
       }
     }
-    if (tid == 0) {
+    if (tid == 0 && DELTA_IN(seg_n + 1, nseg_max + 1, counters)) {
       if (opens) so_g[seg_n] = pos;
       so_g[seg_n + 1] = pos + (uint32_t)fired_total;
       used[bkv] = pos + (uint32_t)fired_total;
@@ -410,11 +412,12 @@ cudaError_t launch_pack_keys(const Shape& s, const Workspace& w, const void* k, 
   using TC = __nv_bfloat16;
   if (s.d == 64)
     pack_keys_kernel<64><<<bkv, 256, smem, st>>>((const TC*)k, w.qhat_rows, w.mask, w.row_nnz, w.kp_vals, w.kp_segoff,
-                                                 w.kp_base, w.kp_used, w.kp_mask, w.kp_nnz, T, s.T_max, cap, nseg_max);
+                                                 w.kp_base, w.kp_used, w.kp_mask, w.kp_nnz, T, s.T_max, cap, nseg_max,
+                                                 w.counters);
   else if (s.d == 128)
     pack_keys_kernel<128><<<bkv, 256, smem, st>>>((const TC*)k, w.qhat_rows, w.mask, w.row_nnz, w.kp_vals,
                                                   w.kp_segoff, w.kp_base, w.kp_used, w.kp_mask, w.kp_nnz, T, s.T_max, cap,
-                                                  nseg_max);
+                                                  nseg_max, w.counters);
   else return cudaErrorNotSupported;
   count_launch();
   return cudaGetLastError();

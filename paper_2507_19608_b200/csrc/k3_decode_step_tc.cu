@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
   float new_s[G];         // scaled hybrid score of the new key, per head (warp 0, all lanes)
 #pragma unroll
   for (int hh = 0; hh < G; ++hh) new_s[hh] = -INFINITY;
-  if (has_new) {
+  if (has_new && DELTA_IN(n, T_max, counters)) {
     for (int e = tid; e < D; e += DNT) {
       k_cache[((size_t)bkv * T_max + n) * D + e] = k_new[(size_t)bkv * D + e];
       v_cache[((size_t)bkv * T_max + n) * D + e] = v_new[(size_t)bkv * D + e];
@@ -380,7 +380,7 @@ __global__ void __launch_bounds__(DNT, 2) decode_step_tc_kernel(
           if constexpr (KEY) {
             s = v[hh] * scale_log2e;                          // the tile's rows already are the hybrid keys
           } else {
-            Rg[(size_t)hh * T_max + j] = v[hh];               // R[j] = q_hat . k_j
+            if (DELTA_IN(j, T_max, counters)) Rg[(size_t)hh * T_max + j] = v[hh];   // R[j] = q_hat . k_j
             s = ((n - j < W) ? v[G + hh] : v[hh]) * scale_log2e;
           }
           sv[u][hh] = s;
