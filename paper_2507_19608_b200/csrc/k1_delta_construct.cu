@@ -3,15 +3,16 @@
 //
 // delta_chain_kernel: the token-sequential part.  Eq. 3 makes every channel a chain along the
 // tokens (the reference is the last value that fired), so the only parallelism is across
-// channels: one thread per channel, one warp per 32 channels, one CTA per (batch, head) of the
-// stream (query heads, or KV heads for key deltas).  The chain itself is three dependent FP32
-// operations per token and a lone warp issues slowly, so everything else is kept off it: a
-// producer warp streams the head's rows into a ring of shared-memory stages with bulk
-// asynchronous copies (the rows do not depend on the carried state), and the chain warps store
-// nothing but the reference in front of every 8-row block (and every 64-row tile, and the final
-// one).  Given those checkpoints every 8-row block of Eq. 2-3 is independent of the others:
-// fire bits, delta values, mask words and reference rows are recomputed from them by
-// row-parallel code (the finish kernel below, the attention kernel for its own query tile).
+// channels: one thread per channel, one CTA per (batch, head, 32 channels) of the stream (query
+// heads, or KV heads for key deltas).  The chain itself is three dependent FP32 operations per
+// token and a lone warp issues slowly, so everything else is kept off it: a producer warp
+// streams the rows into a ring of shared-memory stages with TMA (the rows do not depend on the
+// carried state), helper warps precompute everything about a four-row sub-block that does not
+// involve the carried state (see the kernel), and the chain warp stores nothing but the
+// reference in front of every 8-row block (and every 64-row tile, and the final one).  Given
+// those checkpoints every 8-row block of Eq. 2-3 is independent of the others: fire bits,
+// delta values, mask words and reference rows are recomputed from them by row-parallel code
+// (the finish kernel below, the attention kernel for its own query tile).
 //
 // delta_finish_kernel: everything that is parallel over rows -- Eq. 2-3 over 8-row blocks
 // from the checkpoints: delta values, mask words and (key deltas) the reference-key rows;
@@ -20,197 +21,255 @@
 // hand-off row R(T-1)[j] = q_hat(T-1).k_j for decode and, for the tensor-core attention kernel
 // with the FP32 delta path, the channel-major fp32 copy of the keys.
 #include "delta_internal.cuh"
-#include "mbar.cuh"
+#include "tc_common.cuh"
 
 namespace delta {
 
 namespace {
 
 constexpr int RC = 64;       // rows per ring stage (= one 64-row tile)
-constexpr int NS = 4;        // ring stages
+constexpr int NS = 6;        // stages of staged rows
+constexpr int NZ = 2;        // stages of sub-block tables
+constexpr int CH = 32;       // channels per CTA: one chain warp, thread = channel
+constexpr int SBR = 4;       // rows per sub-block
+constexpr int NSB = RC / SBR;
+constexpr int NHELP = 3;     // warps that build the sub-block tables
+constexpr int Z_STAGE = NSB * 2 * CH;    // float4 per table stage: per (sub-block, channel) x0..x3 and z0..z2
+constexpr int CHAIN_THREADS = 32 * (1 + NHELP + 1);
 
-// One element of the staged rows by shared-memory address, widened to fp32.
-template <typename TIn> __device__ __forceinline__ float lds_elem(uint32_t addr);
-template <> __device__ __forceinline__ float lds_elem<float>(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-  return v;
-}
-template <> __device__ __forceinline__ float lds_elem<__nv_bfloat16>(uint32_t addr) {
-  uint32_t u;
-  asm volatile("ld.shared.u16 %0, [%1];" : "=r"(u) : "r"(addr));
-  return __uint_as_float(u << 16);
-}
-
-// One ring stage of the chain for one thread (= one channel): rows t0 .. t0+nrows-1, the
-// thread's values at rows[r * D]; updates the reference qh and leaves it in front of every
-// 8-row block (ckptp).  basis_row: the stage's first row is the un-thresholded basis.
-template <typename TIn, int D>
-__device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, bool basis_row, float& qh,
-                                            float theta, float* ckptp, int n_ckpt, unsigned long long* counters) {
-  if (nrows == RC && !basis_row) {
-    // full stage, no basis row: nothing but loads, the dependent chain and the checkpoints
-    float x[RC];
-    const uint32_t saddr = smem_u32(rows);
-#pragma unroll
-    for (int r = 0; r < RC; ++r) x[r] = lds_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
-#pragma unroll
-    for (int r = 0; r < RC; ++r) {
-      if ((r % DELTA_CKPT_ROWS) == 0 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
-        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
-      const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
-      const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
-      qh = fire ? x[r] : qh;
-    }
-  } else {
-    for (int r = 0; r < nrows; ++r) {
-      if (((t0 + r) % DELTA_CKPT_ROWS) == 0 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
-        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
-      const float x = to_f32(rows[r * D]);
-      const bool fire = (r == 0 && basis_row) || (fabsf(__fsub_rn(x, qh)) > theta);
-      qh = fire ? x : qh;
-    }
-  }
+template <typename TIn> __device__ __forceinline__ float lds_elem(const TIn* p);
+template <> __device__ __forceinline__ float lds_elem<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float lds_elem<__nv_bfloat16>(const __nv_bfloat16* p) {
+  return __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(p)) << 16);
 }
 
-// Strategy (2): the same stage of the query stream taken from its last row down to its first.
-// The checkpoint of an 8-row block is the reference before the block's highest row.
-// basis_last: the stage's last row is row T-1, the un-thresholded basis of this order.
-template <typename TIn, int D>
-__device__ __forceinline__ void chain_stage_rev(const TIn* rows, int t0, int nrows, bool basis_last, float& qh,
-                                                float theta, float* ckptp, int n_ckpt, unsigned long long* counters) {
-  if (nrows == RC && !basis_last) {
-    float x[RC];
-    const uint32_t saddr = smem_u32(rows);
-#pragma unroll
-    for (int r = 0; r < RC; ++r) x[r] = lds_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
-#pragma unroll
-    for (int r = RC - 1; r >= 0; --r) {
-      if ((r % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
-        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
-      const float diff = __fsub_rn(x[r], qh);
-      const bool fire = fabsf(diff) > theta;
-      qh = fire ? x[r] : qh;
-    }
-  } else {
-    for (int r = nrows - 1; r >= 0; --r) {
-      if ((((t0 + r) % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 || r == nrows - 1) &&
-          DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
-        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
-      const float x = to_f32(rows[r * D]);
-      const bool fire = (r == nrows - 1 && basis_last) || (fabsf(__fsub_rn(x, qh)) > theta);
-      qh = fire ? x : qh;
-    }
-  }
+// Does the reference x_ref fire on value x (Eq. 3: one IEEE subtraction, strict compare, NaN false)?
+__device__ __forceinline__ bool fires(float x, float x_ref, float theta) {
+  return fabsf(__fsub_rn(x, x_ref)) > theta;
+}
+
+// Tight bounded poll of an mbarrier phase (a suspended wait wakes up late, and the hand-overs
+// below are on the chain's path); false once the CTA has given up.
+__device__ __forceinline__ bool poll_ok(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_test_wait(bar, parity)) return true;
+  mbar_poll(bar, parity, abort_flag);
+  return *abort_flag == 0;
 }
 
 }  // namespace
 
+// The chain of Eq. 3 costs three dependent operations per row (subtract, compare, select), about
+// 17 clocks.  Most of that can be taken off the carried state.  Over a sub-block of four rows
+// x0..x3 (in processing order) the state r either survives, or the first row i that fires
+// against r replaces it -- and from there on the chain no longer depends on r: the state at the
+// end of the sub-block is z_i, the end state of the chain that starts with reference x_i at
+// row i.  z_3 = x3, z_2 = fires(x3, x2) ? x3 : x2, and in general z_i = z_j for the first j > i
+// that fires against x_i (x_i if none does): six pair tests per sub-block, none of which
+// involves r.  Helper warps compute the z tables a stage ahead; the chain warp then does, per
+// sub-block, four tests against r in parallel and a two-level select: the dependent path is
+// subtract, compare, three selects per FOUR rows.  Every test is the same subtraction and
+// comparison the sequential chain would make, so the result is bit-identical.
+//
+// One CTA per (head, 32 channels): warp 0 carries the chain (thread = channel), warps 1-3 build
+// the tables, warp 4 streams the rows in with TMA.  Stages that hold the un-thresholded basis
+// row or are cut short by the end of the sequence take the sequential form from the staged
+// values.
 template <typename TIn, int D>
-__global__ void __launch_bounds__(D + 32) delta_chain_kernel(
-    const TIn* __restrict__ q, float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
+__global__ void __launch_bounds__(CHAIN_THREADS) delta_chain_kernel(
+    const __grid_constant__ CUtensorMap tm_x, float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
     float* __restrict__ ckpt, unsigned long long* __restrict__ counters, int T, int n_tiles, int n_ckpt,
-    float theta, int basis_exact, int src_rows, int reverse) {
-  // q: the stream that becomes the delta matrix, [heads][src_rows][D] with rows 0..T-1 read
-  // (queries: src_rows = T; keys in the KV-cache layout: src_rows = T_max)
-  constexpr int NW = D / 32;                       // chain warps
-  constexpr uint32_t ROW_BYTES = D * sizeof(TIn);
-  constexpr uint32_t STAGE_BYTES = RC * ROW_BYTES;
-  extern __shared__ __align__(128) unsigned char ring[];   // [NS][RC][D] of TIn
-  __shared__ __align__(8) unsigned long long bars[2 * NS];   // full[NS], empty[NS]
-  __shared__ int s_fail;
+    float theta, int basis_exact, int reverse) {
+  // tm_x: the stream that becomes the delta matrix as [heads][rows 0..T-1][D]; box = [64 rows][32 channels]
+  constexpr int NSL = D / CH;                      // channel slices (CTAs) per head
+  constexpr uint32_t RAW_STAGE_BYTES = RC * CH * sizeof(TIn);
+  extern __shared__ __align__(128) unsigned char dyn[];
+  TIn* raw = reinterpret_cast<TIn*>(dyn);                                   // [NS][RC][CH]
+  float4* zb = reinterpret_cast<float4*>(dyn + NS * RAW_STAGE_BYTES);       // [NZ][NSB][x | z][CH]
+  __shared__ __align__(8) unsigned long long bars[2 * NS + 2 * NZ];
+  __shared__ uint32_t s_abort;
 
-  const int bh = blockIdx.x;
+  const int bh = blockIdx.x / NSL, sl = blockIdx.x - bh * NSL;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[NS]);
+  const uint32_t zfull0 = smem_u32(&bars[2 * NS]), zfree0 = smem_u32(&bars[2 * NS + NZ]);
+  volatile uint32_t* abort_flag = &s_abort;
   const int n_chunks = (T + RC - 1) / RC;
 
-  if (tid == 0) {
-    for (int s = 0; s < NS; ++s) {
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * s), "r"(1) : "memory");
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty0 + 8 * s), "r"(NW) : "memory");
-    }
-    s_fail = 0;
+  if (tid < 2 * NS + 2 * NZ) {      // one barrier per thread
+    const uint32_t cnt = (tid < NS) ? 1u : (tid < 2 * NS) ? (uint32_t)NHELP : (tid < 2 * NS + NZ) ? (uint32_t)NHELP : 1u;
+    tc::mbar_init(full0 + 8 * tid, cnt);
+    if (tid == 0) s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc::fence_proxy_async();
   }
+  if (tid == 32 * (1 + NHELP))
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_x) : "memory");
   __syncthreads();
   // a kernel launched behind this one with programmatic stream serialisation may become
   // resident and run its prologue now; it sees this kernel's results only after its own
   // grid-dependency wait
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  if (warp == NW) {
-    // ---- producer: keeps up to NS stages of query rows in flight
+  if (warp == 1 + NHELP) {
+    // ---- producer: keeps up to NS stages of rows in flight
     if (lane == 0) {
-      const unsigned char* src = reinterpret_cast<const unsigned char*>(q) + (size_t)bh * src_rows * ROW_BYTES;
-      const uint32_t ring0 = smem_u32(ring);
-      for (int i = 0; i < n_chunks; ++i) {
+      const uint32_t raw0 = smem_u32(raw);
+      for (int i = 0; i < n_chunks && !*abort_flag; ++i) {
         const int s = i % NS;
-        if (i >= NS && !mbar_wait(empty0 + 8 * s, ((i / NS) - 1) & 1)) { s_fail = 1; break; }
+        if (i >= NS) mbar_wait(empty0 + 8 * s, ((i / NS) - 1) & 1, abort_flag);
         const int ci = reverse ? n_chunks - 1 - i : i;      // stage of the head in token order
-        const int rows = min(RC, T - ci * RC);
-        const uint32_t bytes = (uint32_t)rows * ROW_BYTES;
-        // (bounds-checking build: the stage's rows lie inside the head's rows of the stream)
-        if (!DELTA_IN((size_t)ci * RC + rows - 1, src_rows, counters)) { s_fail = 1; break; }
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full0 + 8 * s),
-                     "r"(bytes)
-                     : "memory");
-        asm volatile(
-            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                ring0 + s * STAGE_BYTES),
-            "l"(src + (size_t)ci * STAGE_BYTES), "r"(bytes), "r"(full0 + 8 * s)
-            : "memory");
+        tc::mbar_expect_tx(full0 + 8 * s, RAW_STAGE_BYTES); // rows past T arrive as zeros
+        tc::tma_load_3d(raw0 + s * RAW_STAGE_BYTES, &tm_x, full0 + 8 * s, sl * CH, ci * RC, bh);
       }
     }
-  } else {
-    // ---- chain warps: thread c owns channel c
-    const int c = tid;
-    float* ckptp = ckpt + (size_t)bh * n_ckpt * D + c;
-    float qh = 0.0f;          // reference state, starts at zero (Eq. 3)
-    bool failed = false;
+  } else if (warp >= 1) {
+    // ---- helpers: helper hw takes sub-blocks hw, hw + 3, ... of every stage; rows in processing
+    // order (reverse: from the stage's last row down), tables in processing order of the sub-blocks
+    const int hw = warp - 1;
+    int s = 0, zs = 0;
+    uint32_t ph_full = 0, ph_zfree = 0;      // parity of the completion waited for next
     for (int i = 0; i < n_chunks; ++i) {
-      const int s = i % NS;
-      const int t0 = (reverse ? n_chunks - 1 - i : i) * RC;
-      if (qhat_tile && (t0 % DELTA_TILE_ROWS) == 0 && DELTA_IN(t0 / DELTA_TILE_ROWS, n_tiles, counters))
-        qhat_tile[((size_t)bh * n_tiles + t0 / DELTA_TILE_ROWS) * D + c] = qh;
-      if (!mbar_wait(full0 + 8 * s, (i / NS) & 1)) { failed = true; break; }
-      const TIn* rows = reinterpret_cast<const TIn*>(ring + (size_t)s * STAGE_BYTES) + c;
-      const int nrows = min(RC, T - t0);
-      if (reverse)
-        chain_stage_rev<TIn, D>(rows, t0, nrows, t0 + nrows == T && basis_exact, qh, theta, ckptp, n_ckpt, counters);
-      else
-        chain_stage<TIn, D>(rows, t0, nrows, t0 == 0 && basis_exact, qh, theta, ckptp, n_ckpt, counters);
+      if (!poll_ok(full0 + 8 * s, ph_full, abort_flag)) break;
+      const TIn* rows = raw + (size_t)s * RC * CH + lane;
+      constexpr int NJ = (NSB + NHELP - 1) / NHELP;
+      float y[NJ][SBR];        // every load in front of the first store (both are shared memory)
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) {
+        const int sb = min(hw + NHELP * j, NSB - 1);
+#pragma unroll
+        for (int k = 0; k < SBR; ++k) y[j][k] = lds_elem<TIn>(rows + (sb * SBR + (reverse ? SBR - 1 - k : k)) * CH);
+      }
+      if (i >= NZ && !poll_ok(zfree0 + 8 * zs, ph_zfree, abort_flag)) break;
+      float4* zp = zb + (size_t)zs * Z_STAGE + lane;
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) {
+        const int sb = hw + NHELP * j;
+        if (sb < NSB) {
+          const float z2 = fires(y[j][3], y[j][2], theta) ? y[j][3] : y[j][2];
+          float z1 = fires(y[j][3], y[j][1], theta) ? y[j][3] : y[j][1];
+          z1 = fires(y[j][2], y[j][1], theta) ? z2 : z1;
+          float z0 = fires(y[j][3], y[j][0], theta) ? y[j][3] : y[j][0];
+          z0 = fires(y[j][2], y[j][0], theta) ? z2 : z0;
+          z0 = fires(y[j][1], y[j][0], theta) ? z1 : z0;
+          float4* o = zp + (reverse ? NSB - 1 - sb : sb) * (2 * CH);
+          o[0] = make_float4(y[j][0], y[j][1], y[j][2], y[j][3]);
+          o[CH] = make_float4(z0, z1, z2, 0.0f);
+        }
+      }
       __syncwarp();
-      if (lane == 0)
-        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * s) : "memory");
+      if (lane == 0) {
+        tc::mbar_arrive(zfull0 + 8 * zs);
+        tc::mbar_arrive(empty0 + 8 * s);
+      }
+      if (++s == NS) { s = 0; ph_full ^= 1u; }
+      if (++zs == NZ) { zs = 0; if (i >= NZ) ph_zfree ^= 1u; }
     }
-    if (!failed && qhat_out) qhat_out[(size_t)bh * D + c] = qh;
-    if (failed) s_fail = 1;
+  } else {
+    // ---- chain warp: thread owns channel c
+    const int c = sl * CH + lane;
+    float r = 0.0f;           // reference state, starts at zero (Eq. 3)
+    int zs = 0;
+    uint32_t ph_zfull = 0;
+    static_assert(RC == DELTA_TILE_ROWS, "one tile reference per stage");
+    float* const ckpt_c = ckpt + (size_t)bh * n_ckpt * D + c;
+    float* const qtile = qhat_tile ? qhat_tile + (size_t)bh * n_tiles * D + c : nullptr;
+    const ptrdiff_t cstep = reverse ? -(ptrdiff_t)D : (ptrdiff_t)D;
+    int t0 = reverse ? (n_chunks - 1) * RC : 0;       // first row of the stage, stepped by dt
+    const int dt = reverse ? -RC : RC;
+    // checkpoint of the 8-row block the processing order enters next (full stages step it)
+    float* cp = ckpt_c + (size_t)((t0 + (reverse ? RC - SBR : 0)) / DELTA_CKPT_ROWS) * D;
+    bool ready = false;       // the stage's tables were seen complete during the stage before
+    for (int i = 0; i < n_chunks; ++i, t0 += dt) {
+      const int nrows = min(RC, T - t0);
+      if (qhat_tile && DELTA_IN(t0 / DELTA_TILE_ROWS, n_tiles, counters)) qtile[(size_t)(t0 / DELTA_TILE_ROWS) * D] = r;
+      if (!ready && !poll_ok(zfull0 + 8 * zs, ph_zfull, abort_flag)) break;
+      const int zs_next = (zs + 1 == NZ) ? 0 : zs + 1;
+      const uint32_t ph_next = (zs + 1 == NZ) ? ph_zfull ^ 1u : ph_zfull;
+      const float4* zp = zb + (size_t)zs * Z_STAGE + lane;
+      const bool has_basis = basis_exact && i == 0;      // row 0, or row T-1 in reverse
+      if (nrows == RC) {
+        float4 x = zp[0], z = zp[CH];
+#pragma unroll
+        for (int lsb = 0; lsb < NSB; ++lsb) {
+          // the next sub-block's tables while this one is worked on
+          const float4 xn = zp[(lsb + 1 < NSB ? lsb + 1 : lsb) * (2 * CH)];
+          const float4 zn = zp[(lsb + 1 < NSB ? lsb + 1 : lsb) * (2 * CH) + CH];
+          if ((lsb & 1) == 0) {
+            // the reference in front of an 8-row block (reverse: in front of its highest row)
+            if (DELTA_IN((size_t)(cp - ckpt_c) / D, n_ckpt, counters)) *cp = r;
+            cp += cstep;
+          }
+          // (a look at the next stage's barrier a few sub-blocks before the end: the answer is
+          // back by the time it is needed)
+          if (lsb == NSB - 4) ready = mbar_test_wait(zfull0 + 8 * zs_next, ph_next);
+          const bool p3 = fires(x.w, r, theta), p2 = fires(x.z, r, theta);
+          bool p0 = fires(x.x, r, theta);
+          if (lsb == 0) p0 = p0 || has_basis;      // the basis row is taken un-thresholded
+          const bool p1 = fires(x.y, r, theta);
+          float b = p3 ? x.w : r;
+          b = p2 ? z.z : b;
+          const float a = p0 ? z.x : z.y;          // the first of rows 0, 1 that fired, if one did
+          r = (p0 || p1) ? a : b;
+          x = xn; z = zn;
+        }
+      } else {
+        // a stage cut short by the end of the sequence: row by row from the staged values
+        ready = false;
+        for (int lsb = 0; lsb < NSB; ++lsb) {
+          const float4 x4 = zp[lsb * (2 * CH)];
+          const float xs[SBR] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+          for (int k = 0; k < SBR; ++k) {
+            const int l = lsb * SBR + k;
+            const int pr = reverse ? RC - 1 - l : l;     // row of the stage
+            if (pr < nrows) {
+              const int t = t0 + pr;
+              const bool at_ckpt = reverse ? ((t % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 || pr == nrows - 1)
+                                           : (t % DELTA_CKPT_ROWS) == 0;
+              if (at_ckpt && DELTA_IN(t / DELTA_CKPT_ROWS, n_ckpt, counters))
+                ckpt_c[(size_t)(t / DELTA_CKPT_ROWS) * D] = r;
+              const bool basis_here = has_basis && (reverse ? pr == nrows - 1 : pr == 0);
+              r = (basis_here || fires(xs[k], r, theta)) ? xs[k] : r;
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(zfree0 + 8 * zs);
+      if (nrows != RC) cp = ckpt_c + (size_t)((t0 + dt + (reverse ? RC - SBR : 0)) / DELTA_CKPT_ROWS) * D;
+      zs = zs_next; ph_zfull = ph_next;
+    }
+    if (!*abort_flag && qhat_out) qhat_out[(size_t)bh * D + c] = r;
   }
   __syncthreads();
-  if (tid == 0 && s_fail) atomicMax(&counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
+  if (tid == 0 && s_abort) atomicMax(&counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
 }
 
 
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
                                int init, bool key_stream, bool reverse, cudaStream_t st) {
   if (key_stream && reverse) return cudaErrorNotSupported;
-  const int grid = s.B * (key_stream ? s.H_kv : s.H);
+  const int heads = s.B * (key_stream ? s.H_kv : s.H);
   const int src_rows = key_stream ? s.T_max : T;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
+  const bool f32 = dtype == DELTA_F32;
+  const size_t esz = f32 ? sizeof(float) : sizeof(__nv_bfloat16);
+  CUtensorMap tm;
+  if (!tc::encode3(&tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, q, (uint64_t)s.d,
+                   (uint64_t)T, (uint64_t)heads, (uint64_t)s.d * esz, (uint64_t)src_rows * s.d * esz, CH, RC,
+                   CU_TENSOR_MAP_SWIZZLE_NONE))
+    return cudaErrorInvalidValue;
   cudaError_t err = cudaSuccess;
 #define LAUNCH(TIN, DD)                                                                          \
   do {                                                                                           \
     auto kern = delta_chain_kernel<TIN, DD>;                                                     \
-    const size_t smem = (size_t)NS * RC * DD * sizeof(TIN);                                      \
-    if (smem > 48 * 1024) {                                                                      \
-      err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-      if (err != cudaSuccess) return err;                                                        \
-    }                                                                                            \
-    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.qhat_tile, w.qhat[0], w.ckpt, w.counters, T, s.n_tiles, \
-                                      s.n_ckpt(), theta, basis, src_rows, reverse ? 1 : 0);      \
+    const size_t smem = (size_t)NS * RC * CH * sizeof(TIN) + (size_t)NZ * Z_STAGE * sizeof(float4); \
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
+    if (err != cudaSuccess) return err;                                                          \
+    kern<<<heads * (DD / CH), CHAIN_THREADS, smem, st>>>(tm, w.qhat_tile, w.qhat[0], w.ckpt, w.counters, T, \
+                                                         s.n_tiles, s.n_ckpt(), theta, basis, reverse ? 1 : 0); \
   } while (0)
-  if (dtype == DELTA_F32) {
+  if (f32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
   } else {
     if (s.d == 64) LAUNCH(__nv_bfloat16, 64); else LAUNCH(__nv_bfloat16, 128);
