@@ -220,7 +220,8 @@ int32_t delta_state_sequence_position(const delta_state_t* st, int32_t b) {
 // Can prefill kernel `which` (1 or 2) serve this state?
 static bool tc_eligible(const delta_state* st, int which) {
   if (st->cfg.dtype != DELTA_BF16 || !tc_kernel_available(64)) return false;
-  if (st->cfg.source != DELTA_SRC_QUERY && which != 2) return false;
+  if (st->cfg.source != DELTA_SRC_QUERY && which != 2 && which != 3 && which != 4) return false;
+  if (which == 4 && (st->cfg.source == DELTA_SRC_KEY || st->cfg.d != 64 || (st->shape.g() % 2) != 0)) return false;
   return which == 1 ? tc_kernel_shape(st->cfg.d) : tcq_kernel_shape(st->cfg.d);
 }
 
@@ -283,7 +284,7 @@ delta_status_t delta_key_cache_bytes(const delta_state_t* st, uint64_t* packed_b
 }
 
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
-  if (!st || which < -1 || which > 2) return DELTA_ERR_INVALID_ARG;
+  if (!st || which < -1 || which > 4) return DELTA_ERR_INVALID_ARG;
   if (which >= 1 && !tc_eligible(st, which)) return DELTA_ERR_UNSUPPORTED;
   if (which == 0 && st->cfg.source != DELTA_SRC_QUERY) return DELTA_ERR_UNSUPPORTED;
   st->forced_kernel = which;
@@ -344,23 +345,24 @@ static delta_status_t prefill_launch(delta_state* st, const Shape& shape, const 
   const bool use_tc = which == 1;
   const bool key = c.source == DELTA_SRC_KEY;
   const bool rev = c.source == DELTA_SRC_QUERY_BOTTOM_UP;
-  if ((key || rev) && which != 2) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
+  const bool tcq = which >= 2 && which <= 4;
+  if ((key || rev) && !tcq) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
   // The telescoped attention kernel reads nothing the finish kernel writes (delta values,
   // mask words, counts, indices, counters, hand-off row), so it runs directly behind the chain
   // kernel and the finish kernel comes last.  Both are launched with programmatic stream
   // serialisation: the attention CTAs are resident and set up by the time the chain ends, and
   // the finish kernel's launch overlaps the end of the attention kernel.  With per-kernel
   // timing on, the kernels run in their natural order with events between them.
-  const bool chained = (which == 2) && !prof;
+  const bool chained = tcq && !prof;
   MARK(0);
   // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
   if ((e = launch_delta_chain(shape, ws, key ? k : q, T, theta, c.dtype, c.init, key, rev, cs)) != cudaSuccess)
     return cuda_fail(e);
   auto attention = [&]() -> cudaError_t {
     if (use_tc) return launch_hybrid_attn_tc(shape, ws, q, k, v, out, T, window, c.prefill_window, cs);
-    if (which == 2)
+    if (tcq)
       return launch_hybrid_attn_tcq(shape, ws, q, k, v, out, T, theta, c.init, window, c.prefill_window, key,
-                                    rev, cs);
+                                    rev, /*form=*/which == 3 ? 1 : which == 4 ? 2 : 0, cs);
     return launch_hybrid_attn_generic(shape, ws, q, k, v, out, T, window, c.prefill_window, c.dtype, cs);
   };
   if (chained && !key) {

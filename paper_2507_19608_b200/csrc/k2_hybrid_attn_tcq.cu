@@ -64,24 +64,26 @@ constexpr float RESCALE_LOG2 = 8.0f;       // a row is rescaled when its maximum
 // the 128-byte-swizzle layout.  OFF_QH holds the reference-query tile (query deltas) or the
 // original keys of a window tile (key deltas).  When the key loop is over, the ring space
 // carries the exchange buffer of the final merge.
-template <int D> struct TqSmem {
+template <int D, bool PAIR> struct TqSmem {
   static constexpr uint32_t NKB = D / 64;                 // 64-element blocks per row
   static constexpr uint32_t SZ_TILE = NKB * SZ_BLK;       // one [128][D] operand tile
-  static constexpr uint32_t NKS = (D == 64) ? 4 : 3;      // key ring stages
-  static constexpr uint32_t NVS = (D == 64) ? 4 : 2;      // value ring stages
-  static constexpr uint32_t OFF_Q = 0;
-  static constexpr uint32_t OFF_QH = OFF_Q + SZ_TILE;
+  static constexpr uint32_t NQ = PAIR ? 2 : 1;            // query tiles (heads) per CTA
+  static constexpr uint32_t NKS = PAIR ? 3 : (D == 64) ? 4 : 3;      // key ring stages
+  static constexpr uint32_t NVS = PAIR ? 3 : (D == 64) ? 4 : 2;      // value ring stages
+  static constexpr uint32_t OFF_Q = 0;                    // [NQ] query tiles
+  static constexpr uint32_t OFF_QH = OFF_Q + NQ * SZ_TILE;   // [NQ] reference-query tiles
   // d = 64, query deltas: two operand tiles mixed by row halves, [Q rows 0-63; Q_hat rows
   // 64-127] and [Q_hat rows 0-63; Q rows 64-127] (mixed tiles of block windows whose edges
   // fall on multiples of 64)
-  static constexpr uint32_t OFF_QM = OFF_QH + SZ_TILE;
-  static constexpr uint32_t OFF_K = OFF_QM + ((D == 64) ? 2 * SZ_TILE : 0);
+  static constexpr uint32_t OFF_QM = OFF_QH + NQ * SZ_TILE;  // [NQ][2]
+  static constexpr uint32_t OFF_K = OFF_QM + ((D == 64) ? 2 * NQ * SZ_TILE : 0);
   static constexpr uint32_t OFF_V = OFF_K + NKS * SZ_TILE;
   static constexpr uint32_t OFF_BAR = OFF_V + NVS * SZ_TILE;
   static constexpr uint32_t OFF_MISC = OFF_BAR + 40 * 8;
   static constexpr uint32_t BYTES = OFF_MISC + 16 + 1024;
   static constexpr uint32_t XCH_FLOATS = 2 * 128 * (D / 2 + 2);   // merge exchange: [group][column][row]
-  static_assert(XCH_FLOATS * 4 <= (NKS + NVS) * SZ_TILE, "the exchange buffer fits the ring space");
+  static_assert(PAIR || XCH_FLOATS * 4 <= (NKS + NVS) * SZ_TILE, "the exchange buffer fits the ring space");
+  static_assert(!PAIR || D == 64, "head pairs: d = 64 only");
   static_assert(BYTES <= 227 * 1024, "shared memory budget");
 };
 
@@ -117,6 +119,76 @@ struct TqParams {
 // make the compiler reserve all sixteen hardware barriers).
 __device__ __forceinline__ void softmax_groups_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
+// Maximum of the 32-column chunk Q of a score row; MASKED: only the columns up to `lane`.
+template <int Q, bool MASKED>
+__device__ __forceinline__ float chunk_max(const uint32_t (&u)[128], int lane) {
+  float m0 = __uint_as_float(u[32 * Q]), m1 = -INFINITY;
+#pragma unroll
+  for (int c = 1; c < 32; c += 2) {
+    const float a0 = __uint_as_float(u[32 * Q + c]);
+    const float a1 = (c + 1 < 32) ? __uint_as_float(u[32 * Q + c + 1]) : -INFINITY;
+    if (!MASKED) {
+      m0 = fmax3(m0, a0, a1);
+    } else {
+      m0 = fmaxf(m0, c <= lane ? a0 : -INFINITY);
+      m1 = fmaxf(m1, c + 1 <= lane ? a1 : -INFINITY);
+    }
+  }
+  return fmaxf(m0, m1);
+}
+
+// Eq. 2-3 re-run over NBK 8-row blocks of two neighbouring channels of a query tile in shared
+// memory (128-byte swizzle, offs[rr] = offset of row rr of a block), from the references in
+// front of the blocks (ck[bk * ck_stride], `first` = the first block's, already loaded; the
+// next block's is fetched while a block is worked on; the block loop is not unrolled: this code
+// runs once per CTA and straight-line code costs more to fetch than it saves); writes the
+// reference rows into the operand tile at qh_dst and, with
+// `quarters`, the two row-mixed operand tiles at qm_dst ([Q rows 0-63; Q_hat rows 64-127] and
+// the reverse).  REV: strategy (2), rows from the top.  CHECK: the tile holds rows past the
+// end of the sequence (row0 + r >= T) or the un-thresholded basis row.
+template <bool REV, bool CHECK, int NBK>
+__device__ __forceinline__ void build_ref_rows(const unsigned char* q_src, unsigned char* qh_dst, unsigned char* qm_dst,
+                                               uint32_t sz_tile, const uint32_t (&offs)[DELTA_CKPT_ROWS],
+                                               const float* ck, int ck_stride, float2 first, float theta,
+                                               bool quarters, int seg_row0, int row0, int T, int basis_row) {
+  float2 nxt = first;
+#pragma unroll 1
+  for (int bk = 0; bk < NBK; ++bk) {
+    float cur0 = nxt.x, cur1 = nxt.y;
+    // (a block that starts inside the sequence has its reference: T <= T_max bounds the index)
+    if (bk + 1 < NBK)
+      nxt = (row0 + seg_row0 + (bk + 1) * DELTA_CKPT_ROWS < T)
+                ? *reinterpret_cast<const float2*>(ck + (size_t)(bk + 1) * ck_stride) : make_float2(0.0f, 0.0f);
+    const bool low = (seg_row0 + bk * DELTA_CKPT_ROWS) < 64;
+    unsigned char* const m_q = qm_dst + (low ? 0u : sz_tile);     // takes the query rows of this block
+    unsigned char* const m_h = qm_dst + (low ? sz_tile : 0u);     // takes the reference rows
+#pragma unroll
+    for (int rr = 0; rr < DELTA_CKPT_ROWS; ++rr) {
+      const int r8 = REV ? DELTA_CKPT_ROWS - 1 - rr : rr;
+      const uint32_t off = (uint32_t)bk * 1024u + offs[r8];
+      const uint32_t xw = *reinterpret_cast<const uint32_t*>(q_src + off);
+      const float x0 = __uint_as_float(xw << 16), x1 = __uint_as_float(xw & 0xffff0000u);
+      bool f0 = fabsf(__fsub_rn(x0, cur0)) > theta, f1 = fabsf(__fsub_rn(x1, cur1)) > theta;
+      if (CHECK) {
+        // rows past the end of the sequence carry no state (in reverse they come first)
+        const int gi = row0 + seg_row0 + bk * DELTA_CKPT_ROWS + r8;
+        const bool basis = gi == basis_row, valid = gi < T;
+        f0 = (f0 || basis) && valid;
+        f1 = (f1 || basis) && valid;
+      }
+      cur0 = f0 ? x0 : cur0;
+      cur1 = f1 ? x1 : cur1;
+      // exact: the reference is a copy of an input element (or the zero it starts from)
+      const uint32_t hw = __byte_perm(__float_as_uint(cur0), __float_as_uint(cur1), 0x7632);
+      *reinterpret_cast<uint32_t*>(qh_dst + off) = hw;
+      if (quarters) {
+        *reinterpret_cast<uint32_t*>(m_q + off) = xw;
+        *reinterpret_cast<uint32_t*>(m_h + off) = hw;
+      }
+    }
+  }
+}
+
 }  // namespace
 
 // KEY = false: query deltas (strategy 1, or 2 with p.reverse): telescoped scores Q_hat.K^T.  The
@@ -126,7 +198,7 @@ __device__ __forceinline__ void softmax_groups_sync() { asm volatile("bar.sync 1
 // recursion telescopes to S[i][j] = q_i.k_hat(j), so the telescoped scores are Q.K_hat^T; tm_qh
 // maps the reference-key rows (per KV head), which take the place of the key tiles in the ring,
 // and the original keys are fetched only for tiles that touch the window.
-template <int D, bool KEY>
+template <int D, bool KEY, bool PAIR>
 __global__ void __launch_bounds__(NTHR, 1)
 hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qh,
                        const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -135,7 +207,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* sm = smem_raw + (base - raw);
-  using SM = TqSmem<D>;
+  using SM = TqSmem<D, PAIR>;
+  static_assert(!(KEY && PAIR), "head pairs: query deltas only");
   constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKS = SM::NKS, NVS = SM::NVS;
   constexpr uint32_t OFF_Q = SM::OFF_Q, OFF_QH = SM::OFF_QH, OFF_K = SM::OFF_K, OFF_V = SM::OFF_V,
                      OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC, OFF_QM = SM::OFF_QM;
@@ -146,13 +219,20 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;  // heaviest query tiles of every head first
-  const int bh = blockIdx.x;
+  // PAIR: the CTA owns the same query tile of two neighbouring heads of one KV group, bh and
+  // bh + 1 (group X of the softmax warps takes head bh + X and every key tile)
+  const int bh = PAIR ? 2 * (int)blockIdx.x : (int)blockIdx.x;
   const int b = bh / p.H, h = bh - b * p.H;
   const int bkv = b * (p.H / p.g) + h / p.g;
   const int T = p.T, W = p.W, shape = p.shape;
   const int i0 = qt * BM;
   const int i1 = min(i0 + BM, T) - 1;
   const int n = qt + 1;                                 // key tiles up to the diagonal
+  // A unit is one (key tile, group) pair, issued and consumed in the order u = 0, 1, 2, ...;
+  // unit u belongs to group u & 1 and is that group's (u >> 1)-th.  Key-split form: unit u is
+  // key tile u; head-pair form: units 2t and 2t + 1 are key tile t for the two heads.
+  const int U = PAIR ? 2 * n : n;
+  auto tile_of = [&](int u) -> int { return PAIR ? (u >> 1) : u; };
   // d = 128 fills tensor memory with two score buffers and two output tiles: the probabilities
   // overwrite the scores they come from and a group's next score product has to follow its
   // P.V (one issuing thread does both).  d = 64 leaves room for the probabilities beside the
@@ -218,8 +298,9 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
         for (uint32_t kb = 0; kb < NKB; ++kb) tma_load_3d(dst + kb * SZ_BLK, tm, bar, 64 * kb, row0, outer);
       };
-      mbar_expect_tx(BAR(BAR_Q), SZ_TILE);
-      load_tile(base + OFF_Q, &tm_q, BAR(BAR_Q), i0, bh);
+      mbar_expect_tx(BAR(BAR_Q), SM::NQ * SZ_TILE);
+#pragma unroll
+      for (uint32_t x = 0; x < SM::NQ; ++x) load_tile(base + OFF_Q + x * SZ_TILE, &tm_q, BAR(BAR_Q), i0, bh + (int)x);
       // key deltas: the ring streams reference-key rows, which the finish kernel in front of
       // this one writes (programmatic stream serialisation): wait for them.  Queries, keys and
       // values themselves are inputs.
@@ -260,9 +341,12 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       };
       const uint32_t IDESC_QK64 = make_idesc(64, 0);
       int n_kx = 0, n_sx0 = 0, n_sx1 = 0;
-      // first scores of key tile t, for group t & 1: telescoped, or exact where the whole tile
+      // first scores of unit u, for group u & 1: telescoped, or exact where the whole tile
       // lies inside the window
-      auto first_scores = [&](int t) {
+      auto first_scores = [&](int u) {
+        const int t = tile_of(u);
+        const uint32_t X = (uint32_t)u & 1u;
+        const uint32_t qsel = PAIR ? X * SZ_TILE : 0u;       // the group's own query tiles
         mbar_poll(BAR(BAR_KFULL0 + (uint32_t)t % NKS), (t / NKS) & 1, abort_flag);
         tc_fence_after();
         // query deltas: Q for an exact tile, Q_hat otherwise, against the keys; key deltas: Q
@@ -272,13 +356,13 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (cls == 3) {
           // each half of 64 keys against the operand tile whose row halves are Q where the
           // quarter lies inside the window and Q_hat where it does not
-          const uint32_t X = (uint32_t)t & 1u;
           const int rb0 = i0 / W, rb1 = (i0 + 64) / W;
 #pragma unroll
           for (int hf = 0; hf < 2; ++hf) {
             const int jb = (t * BN + 64 * hf) / W;
             const bool in0 = rb0 == jb, in1 = rb1 == jb;
-            const uint32_t a = base + (in0 ? (in1 ? OFF_Q : OFF_QM) : (in1 ? OFF_QM + SZ_TILE : OFF_QH));
+            const uint32_t a = base + (in0 ? (in1 ? OFF_Q + qsel : OFF_QM + 2 * qsel)
+                                           : (in1 ? OFF_QM + 2 * qsel + SZ_TILE : OFF_QH + qsel));
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks)
               tc_mma(tmem + TMEM_S + 128u * X + 64u * hf, make_desc(a + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
@@ -289,21 +373,23 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           return;
         }
         const bool q_exact = KEY || cls == 2;
-        scores((uint32_t)t & 1u, base + (q_exact ? OFF_Q : OFF_QH), ring);
+        scores(X, base + (q_exact ? OFF_Q : OFF_QH) + qsel, ring);
       };
       mbar_poll(BAR(BAR_Q), 0, abort_flag);
       if (!KEY) mbar_poll(BAR(BAR_QH), 0, abort_flag);   // the softmax warps have built Q_hat
       tc_fence_after();
       first_scores(0);
-      if (n > 1) first_scores(1);
-      for (int t = 0; t < n; ++t) {
-        const uint32_t X = (uint32_t)t & 1u;
+      if (U > 1) first_scores(1);
+      for (int u = 0; u < U; ++u) {
+        const int t = tile_of(u);
+        const uint32_t X = (uint32_t)u & 1u;
         if (tile_class(t) == 1) {
           // mixed tile: Q.K^T over each half of 64 keys once the group has that half's
           // telescoped scores in registers
           if (KEY) mbar_poll(BAR(BAR_KXFULL), n_kx & 1, abort_flag);
           int& n_sx = X ? n_sx1 : n_sx0;
           const uint32_t kx = KEY ? base + OFF_QH : base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE;
+          const uint32_t qx = base + OFF_Q + (PAIR ? X * SZ_TILE : 0u);
 #pragma unroll
           for (int hf = 0; hf < 2; ++hf) {
             mbar_poll(BAR(BAR_SXREQ0 + X), n_sx & 1, abort_flag);
@@ -312,31 +398,32 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks)
               tc_mma(tmem + TMEM_S + 128u * X + 64u * hf,
-                     make_desc(base + OFF_Q + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
+                     make_desc(qx + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024),
                      make_desc(kx + 8192u * hf + (ks >> 2) * SZ_BLK + (ks & 3) * 32, 16, 1024), IDESC_QK64,
                      ks > 0 ? 1u : 0u);
             tc_commit(BAR(BAR_SFULL0 + X));
           }
           if (KEY) { tc_commit(BAR(BAR_KXFREE)); ++n_kx; }
         }
-        tc_commit(BAR(BAR_KFREE0 + (uint32_t)t % NKS));   // every product that reads this key stage is issued
+        // every product that reads this key stage is issued (head pairs: after the second head's)
+        if (!PAIR || X == 1u) tc_commit(BAR(BAR_KFREE0 + (uint32_t)t % NKS));
         if (ALIAS) {
           // P.V of this tile into the group's output tile, then the group's next scores at once
           mbar_poll(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
-          mbar_poll(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
+          mbar_poll(BAR(BAR_PRDY0 + X), (u >> 1) & 1, abort_flag);
           tc_fence_after();
           const uint32_t vb = base + OFF_V + ((uint32_t)t % NVS) * SZ_TILE;
 #pragma unroll
           for (int ks = 0; ks < BN / 16; ++ks)
             tc_mma_ts(tmem + TMEM_O + (uint32_t)D * X, tmem + TMEM_S + 128u * X + 8u * ks,
-                      make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (t >= 2 || ks > 0) ? 1u : 0u);
+                      make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (u >= 2 || ks > 0) ? 1u : 0u);
           tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
-          if (t + 2 >= n) tc_commit(BAR(BAR_ODONE0 + X));   // the group's last product
-          else first_scores(t + 2);
-        } else if (t + 2 < n) {
-          // the group's next scores as soon as it has read this tile's
-          mbar_poll(BAR(BAR_SCONS0 + X), (t >> 1) & 1, abort_flag);
-          first_scores(t + 2);
+          if (u + 2 >= U) tc_commit(BAR(BAR_ODONE0 + X));   // the group's last product
+          else first_scores(u + 2);
+        } else if (u + 2 < U) {
+          // the group's next scores as soon as it has read this unit's
+          mbar_poll(BAR(BAR_SCONS0 + X), (u >> 1) & 1, abort_flag);
+          first_scores(u + 2);
         }
       }
     }
@@ -345,26 +432,30 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // =========================== tensor-core issue: P.V (d = 64) ============================
     if (!ALIAS && lane == 0) {
       const uint32_t IDESC_PV = make_idesc(D, 1);
-      for (int t = 0; t < n; ++t) {
-        const uint32_t X = (uint32_t)t & 1u;
+      for (int u = 0; u < U; ++u) {
+        const int t = tile_of(u);
+        const uint32_t X = (uint32_t)u & 1u;
         mbar_poll(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
-        mbar_poll(BAR(BAR_PRDY0 + X), (t >> 1) & 1, abort_flag);
+        mbar_poll(BAR(BAR_PRDY0 + X), (u >> 1) & 1, abort_flag);
         tc_fence_after();
         const uint32_t vb = base + OFF_V + ((uint32_t)t % NVS) * SZ_TILE;
 #pragma unroll
         for (int ks = 0; ks < BN / 16; ++ks)
           tc_mma_ts(tmem + TMEM_O + (uint32_t)D * X, tmem + TMEM_P64 + 64u * X + 8u * ks,
-                    make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (t >= 2 || ks > 0) ? 1u : 0u);
-        tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
-        if (t + 2 >= n) tc_commit(BAR(BAR_ODONE0 + X));   // the group's last product
+                    make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (u >= 2 || ks > 0) ? 1u : 0u);
+        if (!PAIR || X == 1u) tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
+        if (u + 2 >= U) tc_commit(BAR(BAR_ODONE0 + X));   // the group's last product
         else tc_commit(BAR(BAR_PFREE0 + X));              // the group may write its next probabilities
       }
     }
     __syncwarp();
   } else {
     // =========================== softmax warps: one thread per score row ====================
-    const uint32_t X = (uint32_t)warp >> 2;        // group: key tiles t with t & 1 == X
-    const int row = 32 * (warp & 3) + lane;        // tensor-memory lane = row of the tile
+    const uint32_t X = (uint32_t)warp >> 2;        // group: units u with u & 1 == X
+    const int bh_x = bh + (PAIR ? (int)X : 0);     // the head whose rows this group holds
+    const uint32_t qsel = PAIR ? X * SZ_TILE : 0u; // its query tiles in shared memory
+    const int w4 = warp & 3;
+    const int row = 32 * w4 + lane;                // tensor-memory lane = row of the tile
     const int i = i0 + row;
     const uint32_t lane_sel = (uint32_t)(32 * (warp & 3)) << 16;
     const uint32_t t_s = tmem + TMEM_S + 128u * X + lane_sel;
@@ -374,47 +465,38 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     if (!KEY) {
       // ---- reference-query tile.  The chain kernel left the reference in front of every 8-row
-      // block; thread (channel c, row segment) re-runs Eq. 2-3 over its blocks from there (the
+      // block; thread (channel pair, row segment) re-runs Eq. 2-3 over its blocks from there (the
       // reference after row r is the last fired q[.][c] at or below r) and writes the rows of
-      // Q_hat straight into the operand layout.  Blocks are independent of one another.
-      constexpr int SEG = BM / ((NSW * 32) / D);     // rows per thread: 32 (d = 64), 64 (d = 128)
+      // Q_hat straight into the operand layout, two channels (one 32-bit word) at a time.
+      // Blocks are independent of one another.  (head pairs: each group builds its own head's tile)
+      constexpr int NBT = PAIR ? NSW * 16 : NSW * 32;   // threads per tile
+      constexpr int SEG = BM / (NBT / (D / 2));      // rows per thread: 16 or 32
       constexpr int NBK = SEG / DELTA_CKPT_ROWS;
-      const int c = tid % D, seg = tid / D;
-      auto elem_off = [&](int r) -> uint32_t {   // byte offset of (r, c) in a [128][D] tile, 128-byte swizzle
-        return (uint32_t)(c >> 6) * SZ_BLK + (uint32_t)r * 128u + ((((uint32_t)(c & 63) >> 3) ^ ((uint32_t)r & 7u)) << 4) +
-               ((uint32_t)c & 7u) * 2u;
-      };
-      float ref[NBK];
+      const int tb = PAIR ? (tid & (NBT - 1)) : tid;
+      const int c = 2 * (tb % (D / 2)), seg = tb / (D / 2);   // first channel of the pair, segment
+      // byte offset of (row rr of an 8-row block, channel c) in a [128][D] tile with 128-byte
+      // swizzle, less the block's own offset (8 rows = 1024 bytes, so r & 7 = rr)
+      uint32_t offs[DELTA_CKPT_ROWS];
+#pragma unroll
+      for (int rr = 0; rr < DELTA_CKPT_ROWS; ++rr)
+        offs[rr] = (uint32_t)rr * 128u + ((((uint32_t)(c & 63) >> 3) ^ (uint32_t)rr) << 4) + ((uint32_t)c & 7u) * 2u;
+      const uint32_t thr_off = (uint32_t)(c >> 6) * SZ_BLK + (uint32_t)(seg * SEG) * 128u;
       asm volatile("griddepcontrol.wait;" ::: "memory");    // the chain kernel's checkpoints
-#pragma unroll
-      for (int bk = 0; bk < NBK; ++bk) {
-        const int r0 = i0 + seg * SEG + bk * DELTA_CKPT_ROWS;
-        ref[bk] = (r0 < T && DELTA_IN(r0 / DELTA_CKPT_ROWS, p.n_ckpt, p.counters))
-                      ? p.ckpt[((size_t)bh * p.n_ckpt + r0 / DELTA_CKPT_ROWS) * D + c] : 0.0f;
-      }
+      const int r00 = i0 + seg * SEG;              // the thread's first row
+      const float* const ck = p.ckpt + ((size_t)bh_x * p.n_ckpt + r00 / DELTA_CKPT_ROWS) * D + c;
+      const float2 ref0 = (r00 < T && DELTA_IN((r00 + SEG - 1) / DELTA_CKPT_ROWS, p.n_ckpt, p.counters))
+                              ? *reinterpret_cast<const float2*>(ck) : make_float2(0.0f, 0.0f);
       mbar_wait(BAR(BAR_Q), 0, abort_flag);      // the query tile has landed
-#pragma unroll
-      for (int bk = 0; bk < NBK; ++bk) {
-        float cur = ref[bk];
-#pragma unroll
-        for (int rr = 0; rr < DELTA_CKPT_ROWS; ++rr) {
-          const int r8 = p.reverse ? DELTA_CKPT_ROWS - 1 - rr : rr;   // strategy (2): from the top
-          const int r = seg * SEG + bk * DELTA_CKPT_ROWS + r8;
-          const uint32_t off = elem_off(r);
-          const uint32_t xb = *reinterpret_cast<const uint16_t*>(sm + OFF_Q + off);
-          const float x = __uint_as_float(xb << 16);
-          // rows past the end of the sequence carry no state (in reverse they come first)
-          const bool fire = (i0 + r < T) && ((fabsf(__fsub_rn(x, cur)) > p.theta) || (i0 + r == p.basis_row));
-          cur = fire ? x : cur;
-          // exact: the reference is a copy of an input element (or the zero it starts from)
-          const uint16_t hb = (uint16_t)(__float_as_uint(cur) >> 16);
-          *reinterpret_cast<uint16_t*>(sm + OFF_QH + off) = hb;
-          if (quarters) {
-            *reinterpret_cast<uint16_t*>(sm + OFF_QM + off) = (r < 64) ? (uint16_t)xb : hb;
-            *reinterpret_cast<uint16_t*>(sm + OFF_QM + SZ_TILE + off) = (r < 64) ? hb : (uint16_t)xb;
-          }
-        }
-      }
+      const unsigned char* const q_src = sm + OFF_Q + qsel + thr_off;
+      unsigned char* const qh_dst = sm + OFF_QH + qsel + thr_off;
+      unsigned char* const qm_dst = sm + OFF_QM + 2 * qsel + thr_off;
+      const bool check = (i0 + BM > T) || (p.basis_row >= i0 && p.basis_row < i0 + BM);
+#define BUILD(REV, CHECK)                                                                              \
+  build_ref_rows<REV, CHECK, NBK>(q_src, qh_dst, qm_dst, SZ_TILE, offs, ck, D, ref0, p.theta, quarters, seg * SEG, \
+                                  i0, T, p.basis_row)
+      if (p.reverse) { if (check) BUILD(true, true); else BUILD(true, false); }
+      else { if (check) BUILD(false, true); else BUILD(false, false); }
+#undef BUILD
       fence_proxy_async();      // written through the generic proxy, read by the tensor cores
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(BAR_QH));
@@ -440,9 +522,9 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
     };
     bool pv_waited = false;
-    auto p_free = [&](int t) {
-      if (!ALIAS && t >= 2 && !pv_waited) {
-        mbar_wait(BAR(BAR_PFREE0 + X), ((t >> 1) - 1) & 1, abort_flag);
+    auto p_free = [&](int u) {
+      if (!ALIAS && u >= 2 && !pv_waited) {
+        mbar_wait(BAR(BAR_PFREE0 + X), ((u >> 1) - 1) & 1, abort_flag);
         tc_fence_after();
         pv_waited = true;
       }
@@ -454,7 +536,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // tensor-memory accesses are warp-wide).
     // has_o: the output tile holds earlier products of the group; has_p0: the first half of this
     // tile's probabilities is already stored (second half of a mixed tile)
-    auto settle_scale = [&](int t, float mx, bool has_o, bool has_p0) {
+    auto settle_scale = [&](int u, float mx, bool has_o, bool has_p0) {
       const float m_new = fmaxf(m_used, mx * scale);
       if (!has_o && !has_p0) { m_used = m_new; return; }     // nothing stored at the old scale yet
       const bool grow = (m_new - m_used) > RESCALE_LOG2;
@@ -462,7 +544,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const float al = grow ? ex2(m_used - m_new) : 1.0f;
         if (grow) { l_sum *= al; m_used = m_new; }
         if (has_o) {
-          p_free(t);
+          p_free(u);
 #pragma unroll
           for (int ch = 0; ch < D / 32; ++ch) {
             uint32_t u[32];
@@ -488,22 +570,32 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     };
     // 64 scores -> probabilities at the row's scale, bf16 pairs into tensor-memory columns
     // [32 hf, 32 hf + 32) of the probability buffer, row sum
-    auto exp_store = [&](const float (&v)[64], int hf, int t) {
+    // live: how many of the half's two 32-column chunks hold anything but masked scores (the
+    // same for every thread of the warp; the others' probabilities are zero without being computed)
+    auto exp_store = [&](const float (&v)[64], int hf, int u, int live) {
       const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-m_used, -m_used);
       float2 sum_a = make_float2(0.0f, 0.0f), sum_b = make_float2(0.0f, 0.0f);
       uint32_t w[32];
 #pragma unroll
-      for (int c = 0; c < 64; c += 4) {
-        const float2 e0 = ffma2(make_float2(v[c], v[c + 1]), sc2, nm2);
-        const float2 e1 = ffma2(make_float2(v[c + 2], v[c + 3]), sc2, nm2);
-        const float p0 = ex2(e0.x), p1 = ex2(e0.y), p2 = ex2(e1.x), p3 = ex2(e1.y);
-        sum_a = fadd2(sum_a, make_float2(p0, p1));
-        sum_b = fadd2(sum_b, make_float2(p2, p3));
-        const __nv_bfloat162 pk0 = __floats2bfloat162_rn(p0, p1), pk1 = __floats2bfloat162_rn(p2, p3);
-        w[c >> 1] = *reinterpret_cast<const uint32_t*>(&pk0);
-        w[(c >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&pk1);
+      for (int qq = 0; qq < 2; ++qq) {
+        if (qq < live) {
+#pragma unroll
+          for (int c = 32 * qq; c < 32 * qq + 32; c += 4) {
+            const float2 e0 = ffma2(make_float2(v[c], v[c + 1]), sc2, nm2);
+            const float2 e1 = ffma2(make_float2(v[c + 2], v[c + 3]), sc2, nm2);
+            const float p0 = ex2(e0.x), p1 = ex2(e0.y), p2 = ex2(e1.x), p3 = ex2(e1.y);
+            sum_a = fadd2(sum_a, make_float2(p0, p1));
+            sum_b = fadd2(sum_b, make_float2(p2, p3));
+            const __nv_bfloat162 pk0 = __floats2bfloat162_rn(p0, p1), pk1 = __floats2bfloat162_rn(p2, p3);
+            w[c >> 1] = *reinterpret_cast<const uint32_t*>(&pk0);
+            w[(c >> 1) + 1] = *reinterpret_cast<const uint32_t*>(&pk1);
+          }
+        } else {
+#pragma unroll
+          for (int c = 16 * qq; c < 16 * qq + 16; ++c) w[c] = 0u;
+        }
       }
-      p_free(t);      // the group's previous P.V has read the probabilities
+      p_free(u);      // the group's previous P.V has read the probabilities
       tc_st32(t_p + 32u * hf, w);
       l_sum += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
     };
@@ -519,7 +611,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
     };
 
-    for (int t = (int)X; t < n; t += 2) {
+    for (int u = (int)X; u < U; u += 2) {
+      const int t = tile_of(u);
       mbar_wait(BAR(BAR_SFULL0 + X), s_phase & 1u, abort_flag);
       ++s_phase;
       tc_fence_after();
@@ -533,27 +626,32 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         {
           uint32_t u[128];
           tc_ld128(t_s, u);
-          if (diag) {
+          if (!diag) {
+            float m0 = fmax3(__uint_as_float(u[0]), __uint_as_float(u[1]), __uint_as_float(u[2]));
+            float m1 = fmax3(__uint_as_float(u[3]), __uint_as_float(u[4]), __uint_as_float(u[5]));
+            float m2 = fmax3(__uint_as_float(u[6]), __uint_as_float(u[7]), __uint_as_float(u[8]));
+            float m3 = fmax3(__uint_as_float(u[9]), __uint_as_float(u[10]), __uint_as_float(u[11]));
 #pragma unroll
-            for (int c = 0; c < 128; ++c)
-              if (j0 + c > i) u[c] = 0xff800000u;     // causal mask on the diagonal tile (-inf)
+            for (int c = 12; c < 124; c += 8) {
+              m0 = fmax3(m0, __uint_as_float(u[c]), __uint_as_float(u[c + 1]));
+              m1 = fmax3(m1, __uint_as_float(u[c + 2]), __uint_as_float(u[c + 3]));
+              m2 = fmax3(m2, __uint_as_float(u[c + 4]), __uint_as_float(u[c + 5]));
+              m3 = fmax3(m3, __uint_as_float(u[c + 6]), __uint_as_float(u[c + 7]));
+            }
+            m0 = fmax3(m0, __uint_as_float(u[124]), __uint_as_float(u[125]));
+            m1 = fmax3(m1, __uint_as_float(u[126]), __uint_as_float(u[127]));
+            mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+          } else {
+            // causal mask on the diagonal tile.  The warp's rows are 32 w4 .. 32 w4 + 31 of the
+            // tile: the 32-column chunks in front of chunk w4 are unmasked for all of them, chunk
+            // w4 is masked behind each thread's own column, the chunks after it entirely
+            mx = (w4 == 0) ? chunk_max<0, true>(u, lane) : chunk_max<0, false>(u, lane);
+            if (w4 >= 1) mx = fmaxf(mx, (w4 == 1) ? chunk_max<1, true>(u, lane) : chunk_max<1, false>(u, lane));
+            if (w4 >= 2) mx = fmaxf(mx, (w4 == 2) ? chunk_max<2, true>(u, lane) : chunk_max<2, false>(u, lane));
+            if (w4 >= 3) mx = fmaxf(mx, chunk_max<3, true>(u, lane));
           }
-          float m0 = fmax3(__uint_as_float(u[0]), __uint_as_float(u[1]), __uint_as_float(u[2]));
-          float m1 = fmax3(__uint_as_float(u[3]), __uint_as_float(u[4]), __uint_as_float(u[5]));
-          float m2 = fmax3(__uint_as_float(u[6]), __uint_as_float(u[7]), __uint_as_float(u[8]));
-          float m3 = fmax3(__uint_as_float(u[9]), __uint_as_float(u[10]), __uint_as_float(u[11]));
-#pragma unroll
-          for (int c = 12; c < 124; c += 8) {
-            m0 = fmax3(m0, __uint_as_float(u[c]), __uint_as_float(u[c + 1]));
-            m1 = fmax3(m1, __uint_as_float(u[c + 2]), __uint_as_float(u[c + 3]));
-            m2 = fmax3(m2, __uint_as_float(u[c + 4]), __uint_as_float(u[c + 5]));
-            m3 = fmax3(m3, __uint_as_float(u[c + 6]), __uint_as_float(u[c + 7]));
-          }
-          m0 = fmax3(m0, __uint_as_float(u[124]), __uint_as_float(u[125]));
-          m1 = fmax3(m1, __uint_as_float(u[126]), __uint_as_float(u[127]));
-          mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         }
-        settle_scale(t, mx, t >= 2, false);
+        settle_scale(u, mx, u >= 2, false);
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
           float v[64];
@@ -564,12 +662,19 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int c = 0; c < 64; ++c) v[c] = __uint_as_float(u[c]);
           }
           if (hf == 1) s_consumed();
+          int live = 2;
           if (diag) {
+            live = min(max(w4 + 1 - 2 * hf, 0), 2);
+            // chunk w4 of the tile, if it lies in this half: masked behind the thread's own column
+            // (selects on every element of the half: no index may depend on w4)
 #pragma unroll
-            for (int c = 0; c < 64; ++c)
-              if (j0 + 64 * hf + c > i) v[c] = -INFINITY;
+            for (int qq = 0; qq < 2; ++qq) {
+              const bool part = w4 == 2 * hf + qq;
+#pragma unroll
+              for (int c = 1; c < 32; ++c) v[32 * qq + c] = (part && c > lane) ? -INFINITY : v[32 * qq + c];
+            }
           }
-          exp_store(v, hf, t);
+          exp_store(v, hf, u, live);
         }
       } else {
         // ---- a mixed tile (Section III-B hybrid select), one half of 64 keys at a time: the
@@ -606,8 +711,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int c = 0; c < 64; ++c)
               if (j0 + 64 * hf + c > i) v[c] = -INFINITY;
           }
-          settle_scale(t, max64(v), t >= 2, hf == 1);
-          exp_store(v, hf, t);
+          settle_scale(u, max64(v), u >= 2, hf == 1);
+          exp_store(v, hf, u, 2);
         }
       }
       tc_wait_st();
@@ -616,6 +721,30 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (lane == 0) mbar_arrive(BAR(BAR_PRDY0 + X));
     }
 
+    if (PAIR) {
+      // ---- head pairs: the group's output tile is the whole result of its head's rows
+      mbar_wait(BAR(BAR_ODONE0 + X), 0, abort_flag);
+      tc_fence_after();
+      const float inv = 1.0f / l_sum;
+      const bool store = (i < T) && !*abort_flag && DELTA_IN(i, T, p.counters);
+#pragma unroll
+      for (int ch = 0; ch < D / 32; ++ch) {
+        uint32_t u[32];
+        tc_ld32(t_o + 32u * ch, u);
+        if (store) {
+          uint32_t w[16];
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(u[c]) * inv, __uint_as_float(u[c + 1]) * inv);
+            w[c >> 1] = *reinterpret_cast<const uint32_t*>(&t2);
+          }
+          uint4* op = reinterpret_cast<uint4*>(p.out + ((size_t)bh_x * T + i) * D + 32 * ch);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) op[q4] = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
+        }
+      }
+      tc_fence_before();
+    } else {
     // ---- merge the two groups' partial results, normalise, store.  Each group reads its own
     // output row from tensor memory, keeps the half of the columns it will store (group 0 the
     // lower half) and hands the other half, with its maximum and row sum, to the other group
@@ -668,6 +797,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
     }
     tc_fence_before();
+    }
   }
 
   __syncthreads();
@@ -680,7 +810,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #undef BAR
 }
 
-template <int D, bool KEY>
+template <int D, bool KEY, bool PAIR>
 static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
                               void* out, int T, float theta, int init, int window, int shape, bool reverse,
                               cudaStream_t st) {
@@ -697,8 +827,8 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
       encode3(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, v, D, (uint64_t)T, BKV, D * 2, (uint64_t)s.T_max * D * 2, 64,
               128, CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) return cudaErrorInvalidValue;
-  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D, KEY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)TqSmem<D>::BYTES);
+  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D, KEY, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)TqSmem<D, PAIR>::BYTES);
   if (err != cudaSuccess) return err;
   TqParams p;
   p.out = (__nv_bfloat16*)out;
@@ -714,33 +844,56 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
   // delta chain kernel in front is still running; they wait for its results with
   // griddepcontrol.wait.
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)BH, (unsigned)((T + BM - 1) / BM));
+  cfg.gridDim = dim3((unsigned)(PAIR ? BH / 2 : BH), (unsigned)((T + BM - 1) / BM));
   cfg.blockDim = dim3(NTHR);
-  cfg.dynamicSmemBytes = TqSmem<D>::BYTES;
+  cfg.dynamicSmemBytes = TqSmem<D, PAIR>::BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  err = cudaLaunchKernelEx(&cfg, hybrid_attn_tcq_kernel<D, KEY>, tq, tqh, tk, tv, p);
+  err = cudaLaunchKernelEx(&cfg, hybrid_attn_tcq_kernel<D, KEY, PAIR>, tq, tqh, tk, tv, p);
   count_launch();
   return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
 
+// SMs of the current device (queried once per device).
+static int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (!cached[dev]) {
+    int n = 0;
+    cached[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+  }
+  return cached[dev];
+}
+
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
                                    const void* v, void* out, int T, float theta, int init, int window,
-                                   int shape, bool key_deltas, bool reverse, cudaStream_t st) {
+                                   int shape, bool key_deltas, bool reverse, int form, cudaStream_t st) {
   if (key_deltas && reverse) return cudaErrorNotSupported;
   if (!w.qhat_rows) return cudaErrorNotSupported;
-  if (s.d == 64)
-    return key_deltas ? launch_tcq<64, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st)
-                      : launch_tcq<64, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+  if (s.d == 64) {
+    if (key_deltas && form == 2) return cudaErrorNotSupported;
+    if (key_deltas) return launch_tcq<64, true, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+    // Two heads of a KV group per CTA share every key and value tile and need no merge, but a
+    // head's key tiles are then walked by one softmax group instead of two: that pays once
+    // there are at least two such CTAs per SM (stack layer 0.925 of the one-head form's
+    // time; a single layer of 1024 tokens 1.13).
+    const long ctas_pair = (long)s.B * s.H / 2 * ((T + BM - 1) / BM);
+    if (form == 2 && (s.g() % 2) != 0) return cudaErrorNotSupported;
+    if (form == 2 || (form == 0 && (s.g() % 2) == 0 && ctas_pair >= 2L * sm_count()))
+      return launch_tcq<64, false, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+    return launch_tcq<64, false, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+  }
+  if (form == 2) return cudaErrorNotSupported;
   if (s.d == 128)
-    return key_deltas ? launch_tcq<128, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st)
-                      : launch_tcq<128, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+    return key_deltas ? launch_tcq<128, true, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st)
+                      : launch_tcq<128, false, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
   return cudaErrorNotSupported;
 }
 
