@@ -367,20 +367,21 @@ static delta_status_t prefill_launch(delta_state* st, const Shape& shape, const 
   };
   if (chained && !key) {
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
+    // (released by the attention CTAs once the chain is complete: it runs beside their last wave)
     if ((e = launch_delta_finish(shape, ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
-                                 use_tc, key, rev, true, cs)) != cudaSuccess)
+                                 use_tc, key, rev, 2, cs)) != cudaSuccess)
       return cuda_fail(e);
   } else if (chained) {
     // key deltas: the finish kernel writes the reference-key rows the attention kernel streams,
     // so it comes first (both programmatically serialised behind the kernel in front)
     if ((e = launch_delta_finish(shape, ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
-                                 use_tc, key, rev, true, cs)) != cudaSuccess)
+                                 use_tc, key, rev, 1, cs)) != cudaSuccess)
       return cuda_fail(e);
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);
   } else {
     MARK(1);
     if ((e = launch_delta_finish(shape, ws, q, k, T, theta, window, c.prefill_window, c.dtype, c.init,
-                                 use_tc, key, rev, false, cs)) != cudaSuccess)
+                                 use_tc, key, rev, 0, cs)) != cudaSuccess)
       return cuda_fail(e);
     MARK(2);
     if ((e = attention()) != cudaSuccess) return cuda_fail(e);

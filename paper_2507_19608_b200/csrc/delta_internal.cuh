@@ -71,11 +71,13 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 // K1b: row-parallel finish: delta values, mask words and (key stream) reference rows from the
 // 8-row checkpoints; counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
-// programmatic: launched with programmatic stream serialisation (its launch overlaps the end
-// of the kernel in front; the kernel waits for that kernel's completion itself).
+// programmatic: 1 = launched with programmatic stream serialisation (its launch overlaps the end
+// of the kernel in front; the kernel waits for that kernel's completion itself); 2 = the same, but
+// the kernel does not wait: the kernel in front releases it once the chain kernel's results are
+// complete (query deltas behind the telescoped attention kernel); 0 = an ordinary launch.
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
                                 float theta, int window, int shape, int dtype, int init, bool want_kt,
-                                bool key_stream, bool reverse, bool programmatic, cudaStream_t st);
+                                bool key_stream, bool reverse, int programmatic, cudaStream_t st);
 // K2 (generic): fused hybrid attention on CUDA cores, any supported dtype.
 cudaError_t launch_hybrid_attn_generic(const Shape& s, const Workspace& w, const void* q,
                                        const void* k, const void* v, void* out, int T, int window,

@@ -296,14 +296,18 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
     int T_max, int n_tiles, int BH, int H, int g, int W, int shape, int n_idx_blocks, int kt_ld,
     int key_stream, const TIn* __restrict__ q, int src_rows, float* __restrict__ dq,
     __nv_bfloat16* __restrict__ ref_rows, const float* __restrict__ ckpt, int n_ckpt, float theta,
-    int basis_exact, int reverse) {
+    int basis_exact, int reverse, int wait_front) {
   // q: the stream the chain kernel ran over, [heads][src_rows][D]; ref_rows (key deltas): the
   // reference after every row, the cache of reference keys
   constexpr int NW = D / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // launched with programmatic stream serialisation behind the attention kernel: the results
-  // of everything in front are visible from here on (no effect in an ordinary launch)
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Launched with programmatic stream serialisation.  wait_front: the results of everything
+  // in front are visible from here on (no effect in an ordinary launch).  Without it (query
+  // deltas behind the telescoped attention kernel, of which this kernel needs nothing): every
+  // CTA of the attention kernel has released this kernel after its own wait for the chain
+  // kernel, so the chain's results are complete; they are read past the L1 cache (ld.global.cg),
+  // and the blocks run on the SMs the attention kernel's last wave leaves idle.
+  if (wait_front) asm volatile("griddepcontrol.wait;" ::: "memory");
   // key deltas: the attention kernel is serialised programmatically behind this one and may set
   // itself up meanwhile (it waits for this kernel's results itself)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -327,7 +331,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
         uint32_t word_mine = 0;
         if (rbase < T && DELTA_IN(rbase / DELTA_CKPT_ROWS, n_ckpt, counters) && DELTA_IN(rbase + 7 < T ? rbase + 7 : T - 1, src_rows, counters) &&
             DELTA_IN(T - 1, T_max, counters)) {
-          float ref = ckpt[((size_t)bh * n_ckpt + rbase / DELTA_CKPT_ROWS) * D + c];
+          float ref = __ldcg(&ckpt[((size_t)bh * n_ckpt + rbase / DELTA_CKPT_ROWS) * D + c]);
           float x[8];
 #pragma unroll
           for (int r = 0; r < 8; ++r)
@@ -458,7 +462,7 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
   }
   for (int e = tid; e < g * D; e += 256) {
     const int hh = e / D, c = e - hh * D;
-    qh[hh][c] = qhat[((size_t)b * H + kvh * g + hh) * D + c];
+    qh[hh][c] = __ldcg(&qhat[((size_t)b * H + kvh * g + hh) * D + c]);
   }
   __syncthreads();
   if (kt != nullptr) {
@@ -481,7 +485,9 @@ __global__ void __launch_bounds__(256, 5) delta_finish_kernel(
 
 cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* q, const void* k, int T,
                                 float theta, int window, int shape, int dtype, int init, bool want_kt,
-                                bool key_stream, bool reverse, bool programmatic, cudaStream_t st) {
+                                bool key_stream, bool reverse, int programmatic, cudaStream_t st) {
+  // programmatic: 0 = ordinary launch, 1 = programmatic serialisation, 2 = the same and the kernel
+  // does not wait for the kernel in front (see the kernel)
   // key deltas: the index/counter pass runs over the KV heads and there is no hand-off row
   const int BH = s.B * (key_stream ? s.H_kv : s.H);
   const int tiles_used = (T + DELTA_TILE_ROWS - 1) / DELTA_TILE_ROWS;
@@ -505,7 +511,7 @@ cudaError_t launch_delta_finish(const Shape& s, const Workspace& w, const void* 
       s.T_max, s.n_tiles, BH, s.H, s.g(), window, shape, n_idx_blocks, kt_ld, key_stream ? 1 : 0,   \
       key_stream ? (const TIN*)k : (const TIN*)q, key_stream ? s.T_max : T, w.dq,                 \
       key_stream ? w.qhat_rows : (__nv_bfloat16*)nullptr, (const float*)w.ckpt, s.n_ckpt(), theta, \
-      init == DELTA_INIT_BASIS_EXACT ? 1 : 0, reverse ? 1 : 0)
+      init == DELTA_INIT_BASIS_EXACT ? 1 : 0, reverse ? 1 : 0, programmatic == 2 ? 0 : 1)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
   } else {

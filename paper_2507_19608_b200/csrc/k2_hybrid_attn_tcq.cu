@@ -247,17 +247,32 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (tid >= 32 && tid < 32 + NUM_BARS) {       // one barrier per thread of warp 1 (and 2)
-    const int i = tid - 32;
-    uint32_t cnt = 1;
-    if (i == BAR_QH) cnt = NSW;
-    if (i == BAR_PRDY0 || i == BAR_PRDY1 || i == BAR_SXREQ0 || i == BAR_SXREQ1 || i == BAR_SCONS0 ||
-        i == BAR_SCONS1)
-      cnt = 4;
-    mbar_init(BAR(i), cnt);
-    if (i == 0) sMisc[1] = 0;
+  if (warp == WARP_TMA) {
+    // the loader warp sets the barriers up (a thread takes barrier `lane` and, for the few past
+    // 32, `lane + 32`) and has the query tile on its way before the CTA has even met: the
+    // query tile is what the prologue waits for
+    static_assert(NUM_BARS <= 64, "two barriers per thread at most");
+#pragma unroll
+    for (int i = lane; i < NUM_BARS; i += 32) {
+      uint32_t cnt = 1;
+      if (i == BAR_QH) cnt = NSW;
+      if (i == BAR_PRDY0 || i == BAR_PRDY1 || i == BAR_SXREQ0 || i == BAR_SXREQ1 || i == BAR_SCONS0 ||
+          i == BAR_SCONS1)
+        cnt = 4;
+      mbar_init(BAR(i), cnt);
+    }
+    if (lane == 0) sMisc[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      mbar_expect_tx(BAR(BAR_Q), SM::NQ * SZ_TILE);
+#pragma unroll
+      for (uint32_t x = 0; x < SM::NQ; ++x)
+#pragma unroll
+        for (uint32_t kb = 0; kb < NKB; ++kb)
+          tma_load_3d(base + OFF_Q + x * SZ_TILE + kb * SZ_BLK, &tm_q, BAR(BAR_Q), 64 * kb, i0, bh + (int)x);
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -298,9 +313,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
         for (uint32_t kb = 0; kb < NKB; ++kb) tma_load_3d(dst + kb * SZ_BLK, tm, bar, 64 * kb, row0, outer);
       };
-      mbar_expect_tx(BAR(BAR_Q), SM::NQ * SZ_TILE);
-#pragma unroll
-      for (uint32_t x = 0; x < SM::NQ; ++x) load_tile(base + OFF_Q + x * SZ_TILE, &tm_q, BAR(BAR_Q), i0, bh + (int)x);
+      // (the query tile is already on its way: see the set-up)
       // key deltas: the ring streams reference-key rows, which the finish kernel in front of
       // this one writes (programmatic stream serialisation): wait for them.  Queries, keys and
       // values themselves are inputs.
@@ -463,7 +476,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const uint32_t t_p = ALIAS ? t_s : tmem + TMEM_P64 + 64u * X + lane_sel;   // bf16 probabilities
     const float scale = p.scale_log2e;
 
-    if (!KEY) {
+    auto build_tile = [&]() {
       // ---- reference-query tile.  The chain kernel left the reference in front of every 8-row
       // block; thread (channel pair, row segment) re-runs Eq. 2-3 over its blocks from there (the
       // reference after row r is the last fired q[.][c] at or below r) and writes the rows of
@@ -482,9 +495,12 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         offs[rr] = (uint32_t)rr * 128u + ((((uint32_t)(c & 63) >> 3) ^ (uint32_t)rr) << 4) + ((uint32_t)c & 7u) * 2u;
       const uint32_t thr_off = (uint32_t)(c >> 6) * SZ_BLK + (uint32_t)(seg * SEG) * 128u;
       asm volatile("griddepcontrol.wait;" ::: "memory");    // the chain kernel's checkpoints
+      // the finish kernel behind needs the chain's results and nothing of this kernel's: once
+      // every CTA has come by here (the last wave included) it may run on the SMs left idle
+      if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
       const int r00 = i0 + seg * SEG;              // the thread's first row
       const float* const ck = p.ckpt + ((size_t)bh_x * p.n_ckpt + r00 / DELTA_CKPT_ROWS) * D + c;
-      const float2 ref0 = (r00 < T && DELTA_IN((r00 + SEG - 1) / DELTA_CKPT_ROWS, p.n_ckpt, p.counters))
+      const float2 ref0 = (r00 < T && DELTA_IN(min(r00 + SEG - 1, T - 1) / DELTA_CKPT_ROWS, p.n_ckpt, p.counters))
                               ? *reinterpret_cast<const float2*>(ck) : make_float2(0.0f, 0.0f);
       mbar_wait(BAR(BAR_Q), 0, abort_flag);      // the query tile has landed
       const unsigned char* const q_src = sm + OFF_Q + qsel + thr_off;
@@ -500,7 +516,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       fence_proxy_async();      // written through the generic proxy, read by the tensor cores
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(BAR_QH));
-    }
+    };
 
     int wlo = 0, whi = 0;       // exact keys of row i: wlo <= j < whi
     if (W > 0) {
@@ -611,6 +627,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
     };
 
+    if (!KEY) build_tile();
     for (int u = (int)X; u < U; u += 2) {
       const int t = tile_of(u);
       mbar_wait(BAR(BAR_SFULL0 + X), s_phase & 1u, abort_flag);
@@ -652,8 +669,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           }
         }
         settle_scale(u, mx, u >= 2, false);
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
+        // the exponentials, one half of 64 columns at a time
+        auto exp_half = [&](int hf) {
           float v[64];
           {
             uint32_t u[64];
@@ -675,13 +692,21 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
           }
           exp_store(v, hf, u, live);
+        };
+        if (D == 64) {
+          // (two copies of the code: 8 % faster in the steady state than a loop)
+          exp_half(0);
+          exp_half(1);
+        } else {
+          // (d = 128: the two-copy form spills)
+#pragma unroll 1
+          for (int hf = 0; hf < 2; ++hf) exp_half(hf);
         }
       } else {
         // ---- a mixed tile (Section III-B hybrid select), one half of 64 keys at a time: the
         // half's telescoped scores go to registers, its columns go back for the exact product,
         // the in-window elements are taken from that
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
+        auto mixed_half = [&](int hf) {
           float v[64];
           {
             uint32_t u[64];
@@ -713,6 +738,13 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           }
           settle_scale(u, max64(v), u >= 2, hf == 1);
           exp_store(v, hf, u, 2);
+        };
+        if (D == 64) {
+          mixed_half(0);
+          mixed_half(1);
+        } else {
+#pragma unroll 1
+          for (int hf = 0; hf < 2; ++hf) mixed_half(hf);
         }
       }
       tc_wait_st();
