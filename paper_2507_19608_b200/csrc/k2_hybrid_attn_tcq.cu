@@ -59,6 +59,11 @@ constexpr uint32_t TMEM_O = 256;           // output tile of group 0 at 256, of 
 constexpr uint32_t TMEM_P64 = 384;         // d = 64: probabilities of group 0 at 384, of group 1 at 448
 constexpr uint32_t SZ_BLK = 128 * 64 * 2;  // one [128 rows][64 elements] bf16 block, 16 KiB
 constexpr float RESCALE_LOG2 = 8.0f;       // a row is rescaled when its maximum grew by more than 2^8
+#ifndef DELTA_POLY_EVERY
+#define DELTA_POLY_EVERY 4
+#endif
+constexpr int POLY_EVERY = DELTA_POLY_EVERY; // every n-th pair of exponentials by polynomial (0: none)
+static_assert(POLY_EVERY == 0 || POLY_EVERY == 2 || POLY_EVERY == 4 || POLY_EVERY == 8 || POLY_EVERY == 16, "");
 
 // Shared-memory map for head dimension D.  Operand tiles are D/64 blocks of [128][64] bf16 in
 // the 128-byte-swizzle layout.  OFF_QH holds the reference-query tile (query deltas) or the
@@ -198,7 +203,10 @@ __device__ __forceinline__ void build_ref_rows(const unsigned char* q_src, unsig
 // recursion telescopes to S[i][j] = q_i.k_hat(j), so the telescoped scores are Q.K_hat^T; tm_qh
 // maps the reference-key rows (per KV head), which take the place of the key tiles in the ring,
 // and the original keys are fetched only for tiles that touch the window.
-template <int D, bool KEY, bool PAIR>
+// MIXED = false: no key tile of the launch is mixed (no window; or, query deltas at d = 64, a
+// block window whose edges fall on multiples of 64): the code of the mixed tiles is left out,
+// and with it every register spill of the kernel.
+template <int D, bool KEY, bool PAIR, bool MIXED>
 __global__ void __launch_bounds__(NTHR, 1)
 hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qh,
                        const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -327,7 +335,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         // (key deltas: a tile scored exactly throughout needs the original keys, not the reference keys)
         const int cls = tile_class(t);
         load_tile(base + OFF_K + ks * SZ_TILE, (KEY && cls == 2) ? &tm_k : tm_ring, BAR(BAR_KFULL0 + ks), t * BN, bkv);
-        if (KEY && cls == 1) {
+        if (MIXED && KEY && cls == 1) {
           if (n_kx > 0) mbar_wait(BAR(BAR_KXFREE), (n_kx - 1) & 1, abort_flag);
           mbar_expect_tx(BAR(BAR_KXFULL), SZ_TILE);
           load_tile(base + OFF_QH, &tm_k, BAR(BAR_KXFULL), t * BN, bkv);
@@ -396,7 +404,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       for (int u = 0; u < U; ++u) {
         const int t = tile_of(u);
         const uint32_t X = (uint32_t)u & 1u;
-        if (tile_class(t) == 1) {
+        if (MIXED && tile_class(t) == 1) {
           // mixed tile: Q.K^T over each half of 64 keys once the group has that half's
           // telescoped scores in registers
           if (KEY) mbar_poll(BAR(BAR_KXFULL), n_kx & 1, abort_flag);
@@ -599,7 +607,11 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           for (int c = 32 * qq; c < 32 * qq + 32; c += 4) {
             const float2 e0 = ffma2(make_float2(v[c], v[c + 1]), sc2, nm2);
             const float2 e1 = ffma2(make_float2(v[c + 2], v[c + 3]), sc2, nm2);
-            const float p0 = ex2(e0.x), p1 = ex2(e0.y), p2 = ex2(e1.x), p3 = ex2(e1.y);
+            // one pair in POLY_EVERY on the FMA pipe instead of the exponential unit
+            const bool poly = POLY_EVERY > 0 && (((c >> 1) + 1) % POLY_EVERY) == POLY_EVERY - 1;   // (POLY_EVERY: 2, 4, 8, 16)
+            const float p0 = ex2(e0.x), p1 = ex2(e0.y);
+            const float2 pp = poly ? ex2_poly2(e1) : make_float2(ex2(e1.x), ex2(e1.y));
+            const float p2 = pp.x, p3 = pp.y;
             sum_a = fadd2(sum_a, make_float2(p0, p1));
             sum_b = fadd2(sum_b, make_float2(p2, p3));
             const __nv_bfloat162 pk0 = __floats2bfloat162_rn(p0, p1), pk1 = __floats2bfloat162_rn(p2, p3);
@@ -636,7 +648,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const int j0 = t * BN;
       const bool diag = (t == qt);
       pv_waited = false;
-      if (tile_class(t) != 1) {
+      if (!MIXED || tile_class(t) != 1) {
         // ---- the common tile: two passes over the score buffer, the row maximum first, then the
         // exponentials in halves of 64 columns
         float mx;
@@ -842,8 +854,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #undef BAR
 }
 
-template <int D, bool KEY, bool PAIR>
-static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
+template <int D, bool KEY, bool PAIR, bool MIXED>
+static cudaError_t launch_tcq_m(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
                               void* out, int T, float theta, int init, int window, int shape, bool reverse,
                               cudaStream_t st) {
   const uint64_t BH = (uint64_t)s.B * s.H, BKV = (uint64_t)s.B * s.H_kv;
@@ -859,7 +871,7 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
       encode3(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, v, D, (uint64_t)T, BKV, D * 2, (uint64_t)s.T_max * D * 2, 64,
               128, CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) return cudaErrorInvalidValue;
-  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D, KEY, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D, KEY, PAIR, MIXED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)TqSmem<D, PAIR>::BYTES);
   if (err != cudaSuccess) return err;
   TqParams p;
@@ -885,9 +897,27 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  err = cudaLaunchKernelEx(&cfg, hybrid_attn_tcq_kernel<D, KEY, PAIR>, tq, tqh, tk, tv, p);
+  err = cudaLaunchKernelEx(&cfg, hybrid_attn_tcq_kernel<D, KEY, PAIR, MIXED>, tq, tqh, tk, tv, p);
   count_launch();
   return err != cudaSuccess ? err : cudaGetLastError();
+}
+
+// Can a key tile be mixed (partly inside the window with no quarter structure)?  Mirrors the
+// kernel's tile classes.
+template <int D, bool KEY>
+static bool mixed_tiles_possible(int window, int shape) {
+  if (window <= 0) return false;
+  const bool quarters = (D == 64) && !KEY && shape == 0 && (window % 64) == 0;
+  return !quarters;
+}
+
+template <int D, bool KEY, bool PAIR>
+static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
+                              void* out, int T, float theta, int init, int window, int shape, bool reverse,
+                              cudaStream_t st) {
+  return mixed_tiles_possible<D, KEY>(window, shape)
+             ? launch_tcq_m<D, KEY, PAIR, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st)
+             : launch_tcq_m<D, KEY, PAIR, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
 }
 
 bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
