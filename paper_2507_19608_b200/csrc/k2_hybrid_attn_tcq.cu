@@ -203,8 +203,9 @@ __device__ __forceinline__ void build_ref_rows(const unsigned char* q_src, unsig
 // recursion telescopes to S[i][j] = q_i.k_hat(j), so the telescoped scores are Q.K_hat^T; tm_qh
 // maps the reference-key rows (per KV head), which take the place of the key tiles in the ring,
 // and the original keys are fetched only for tiles that touch the window.
-// MIXED = false: no key tile of the launch is mixed (no window; or, query deltas at d = 64, a
-// block window whose edges fall on multiples of 64): the code of the mixed tiles is left out,
+// MIXED = false: no key tile of the launch is mixed (no window; a block window of whole
+// 128-key tiles; or, query deltas at d = 64, a block window whose edges fall on multiples of
+// 64): the code of the mixed tiles is left out,
 // and with it every register spill of the kernel.
 template <int D, bool KEY, bool PAIR, bool MIXED>
 __global__ void __launch_bounds__(NTHR, 1)
@@ -907,6 +908,8 @@ static cudaError_t launch_tcq_m(const Shape& s, const Workspace& w, const void* 
 template <int D, bool KEY>
 static bool mixed_tiles_possible(int window, int shape) {
   if (window <= 0) return false;
+  // a block window of whole tiles: every key tile lies inside one block or outside it
+  if (shape == 0 && (window % BN) == 0) return false;
   const bool quarters = (D == 64) && !KEY && shape == 0 && (window % 64) == 0;
   return !quarters;
 }
