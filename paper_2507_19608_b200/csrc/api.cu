@@ -220,8 +220,8 @@ int32_t delta_state_sequence_position(const delta_state_t* st, int32_t b) {
 // Can prefill kernel `which` (1 or 2) serve this state?
 static bool tc_eligible(const delta_state* st, int which) {
   if (st->cfg.dtype != DELTA_BF16 || !tc_kernel_available(64)) return false;
-  if (st->cfg.source != DELTA_SRC_QUERY && which != 2 && which != 3 && which != 4) return false;
-  if (which == 4 && (st->cfg.source == DELTA_SRC_KEY || st->cfg.d != 64 || (st->shape.g() % 2) != 0)) return false;
+  if (st->cfg.source != DELTA_SRC_QUERY && which != 2 && which != 3 && which != 4 && which != 5) return false;
+  if ((which == 4 || which == 5) && (st->cfg.source == DELTA_SRC_KEY || st->cfg.d != 64 || (st->shape.g() % 2) != 0)) return false;
   return which == 1 ? tc_kernel_shape(st->cfg.d) : tcq_kernel_shape(st->cfg.d);
 }
 
@@ -284,7 +284,7 @@ delta_status_t delta_key_cache_bytes(const delta_state_t* st, uint64_t* packed_b
 }
 
 delta_status_t delta_state_set_prefill_kernel(delta_state_t* st, int32_t which) {
-  if (!st || which < -1 || which > 4) return DELTA_ERR_INVALID_ARG;
+  if (!st || which < -1 || which > 5) return DELTA_ERR_INVALID_ARG;
   if (which >= 1 && !tc_eligible(st, which)) return DELTA_ERR_UNSUPPORTED;
   if (which == 0 && st->cfg.source != DELTA_SRC_QUERY) return DELTA_ERR_UNSUPPORTED;
   st->forced_kernel = which;
@@ -345,7 +345,7 @@ static delta_status_t prefill_launch(delta_state* st, const Shape& shape, const 
   const bool use_tc = which == 1;
   const bool key = c.source == DELTA_SRC_KEY;
   const bool rev = c.source == DELTA_SRC_QUERY_BOTTOM_UP;
-  const bool tcq = which >= 2 && which <= 4;
+  const bool tcq = which >= 2 && which <= 5;
   if ((key || rev) && !tcq) return DELTA_ERR_UNSUPPORTED;   // no tensor-core kernel on this device
   // The telescoped attention kernel reads nothing the finish kernel writes (delta values,
   // mask words, counts, indices, counters, hand-off row), so it runs directly behind the chain
@@ -362,7 +362,7 @@ static delta_status_t prefill_launch(delta_state* st, const Shape& shape, const 
     if (use_tc) return launch_hybrid_attn_tc(shape, ws, q, k, v, out, T, window, c.prefill_window, cs);
     if (tcq)
       return launch_hybrid_attn_tcq(shape, ws, q, k, v, out, T, theta, c.init, window, c.prefill_window, key,
-                                    rev, /*form=*/which == 3 ? 1 : which == 4 ? 2 : 0, cs);
+                                    rev, /*form=*/which == 3 ? 1 : which == 4 ? 2 : which == 5 ? 3 : 0, cs);
     return launch_hybrid_attn_generic(shape, ws, q, k, v, out, T, window, c.prefill_window, c.dtype, cs);
   };
   if (chained && !key) {

@@ -87,7 +87,7 @@ template <int D, bool PAIR> struct TqSmem {
   static constexpr uint32_t OFF_MISC = OFF_BAR + 40 * 8;
   static constexpr uint32_t BYTES = OFF_MISC + 16 + 1024;
   static constexpr uint32_t XCH_FLOATS = 2 * 128 * (D / 2 + 2);   // merge exchange: [group][column][row]
-  static_assert(PAIR || XCH_FLOATS * 4 <= (NKS + NVS) * SZ_TILE, "the exchange buffer fits the ring space");
+  static_assert(XCH_FLOATS * 4 <= (NKS + NVS) * SZ_TILE, "the exchange buffer fits the ring space");
   static_assert(!PAIR || D == 64, "head pairs: d = 64 only");
   static_assert(BYTES <= 227 * 1024, "shared memory budget");
 };
@@ -115,6 +115,8 @@ struct TqParams {
   unsigned long long* counters;
   const float* ckpt;           // [B,H,n_ckpt,D] reference in front of every 8-row block (query deltas only)
   int T, T_max, n_ckpt, H, g, W, shape;
+  int BH;            // heads in all (batch x query heads)
+  int n_one;         // two-head layout: the n_one heaviest query tiles of every head go one head per CTA
   int reverse;       // strategy (2): Eq. 2-3 runs from row T-1 down to row 0
   int basis_row;     // the un-thresholded basis row (0, or T-1 in reverse), -1 if there is none
   float scale_log2e, theta;
@@ -142,7 +144,7 @@ __device__ __forceinline__ float chunk_max(const uint32_t (&u)[128], int lane) {
   return fmaxf(m0, m1);
 }
 
-// Eq. 2-3 re-run over NBK 8-row blocks of two neighbouring channels of a query tile in shared
+// Eq. 2-3 re-run over nbk 8-row blocks of two neighbouring channels of a query tile in shared
 // memory (128-byte swizzle, offs[rr] = offset of row rr of a block), from the references in
 // front of the blocks (ck[bk * ck_stride], `first` = the first block's, already loaded; the
 // next block's is fetched while a block is worked on; the block loop is not unrolled: this code
@@ -151,17 +153,17 @@ __device__ __forceinline__ float chunk_max(const uint32_t (&u)[128], int lane) {
 // `quarters`, the two row-mixed operand tiles at qm_dst ([Q rows 0-63; Q_hat rows 64-127] and
 // the reverse).  REV: strategy (2), rows from the top.  CHECK: the tile holds rows past the
 // end of the sequence (row0 + r >= T) or the un-thresholded basis row.
-template <bool REV, bool CHECK, int NBK>
+template <bool REV, bool CHECK>
 __device__ __forceinline__ void build_ref_rows(const unsigned char* q_src, unsigned char* qh_dst, unsigned char* qm_dst,
                                                uint32_t sz_tile, const uint32_t (&offs)[DELTA_CKPT_ROWS],
-                                               const float* ck, int ck_stride, float2 first, float theta,
+                                               const float* ck, int ck_stride, float2 first, int nbk, float theta,
                                                bool quarters, int seg_row0, int row0, int T, int basis_row) {
   float2 nxt = first;
 #pragma unroll 1
-  for (int bk = 0; bk < NBK; ++bk) {
+  for (int bk = 0; bk < nbk; ++bk) {
     float cur0 = nxt.x, cur1 = nxt.y;
     // (a block that starts inside the sequence has its reference: T <= T_max bounds the index)
-    if (bk + 1 < NBK)
+    if (bk + 1 < nbk)
       nxt = (row0 + seg_row0 + (bk + 1) * DELTA_CKPT_ROWS < T)
                 ? *reinterpret_cast<const float2*>(ck + (size_t)(bk + 1) * ck_stride) : make_float2(0.0f, 0.0f);
     const bool low = (seg_row0 + bk * DELTA_CKPT_ROWS) < 64;
@@ -207,7 +209,9 @@ __device__ __forceinline__ void build_ref_rows(const unsigned char* q_src, unsig
 // 128-key tiles; or, query deltas at d = 64, a block window whose edges fall on multiples of
 // 64): the code of the mixed tiles is left out,
 // and with it every register spill of the kernel.
-template <int D, bool KEY, bool PAIR, bool MIXED>
+// FORM: 0 = every CTA one head; 1 = every CTA two heads; 2 = two-head layout, the form of a CTA
+// follows its place in the grid (see below).
+template <int D, bool KEY, int FORM, bool MIXED>
 __global__ void __launch_bounds__(NTHR, 1)
 hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_qh,
                        const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -216,6 +220,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* sm = smem_raw + (base - raw);
+  constexpr bool PAIR = FORM != 0;       // the layout holds two query tiles
   using SM = TqSmem<D, PAIR>;
   static_assert(!(KEY && PAIR), "head pairs: query deltas only");
   constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKS = SM::NKS, NVS = SM::NVS;
@@ -227,10 +232,29 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #define BAR(i) (bar0 + 8u * (uint32_t)(i))
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;  // heaviest query tiles of every head first
-  // PAIR: the CTA owns the same query tile of two neighbouring heads of one KV group, bh and
-  // bh + 1 (group X of the softmax warps takes head bh + X and every key tile)
-  const int bh = PAIR ? 2 * (int)blockIdx.x : (int)blockIdx.x;
+  // Heaviest query tiles of every head first.  PAIR (the layout holds two query tiles): a
+  // one-dimensional grid; its first BH * n_one CTAs take the n_one heaviest query tiles of every
+  // head in the one-head form (key tiles dealt to the two softmax groups, merge at the end), the
+  // others the same query tile of two neighbouring heads of one KV group, bh and bh + 1 (group
+  // X of the softmax warps takes head bh + X and every key tile).  pr: this CTA is of the
+  // second kind.
+  int qt, bh;
+  bool pr = false;
+  if (PAIR) {
+    const int nqt = (p.T + BM - 1) / BM, idx = (int)blockIdx.x, n1 = (FORM == 1) ? 0 : p.BH * p.n_one;
+    if (FORM == 2 && idx < n1) {
+      qt = nqt - 1 - idx / p.BH;
+      bh = idx % p.BH;
+    } else {
+      const int j = idx - n1, hp = p.BH / 2;
+      pr = true;
+      qt = nqt - ((FORM == 1) ? 0 : p.n_one) - 1 - j / hp;
+      bh = 2 * (j % hp);
+    }
+  } else {
+    qt = (int)gridDim.y - 1 - (int)blockIdx.y;
+    bh = (int)blockIdx.x;
+  }
   const int b = bh / p.H, h = bh - b * p.H;
   const int bkv = b * (p.H / p.g) + h / p.g;
   const int T = p.T, W = p.W, shape = p.shape;
@@ -240,8 +264,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   // A unit is one (key tile, group) pair, issued and consumed in the order u = 0, 1, 2, ...;
   // unit u belongs to group u & 1 and is that group's (u >> 1)-th.  Key-split form: unit u is
   // key tile u; head-pair form: units 2t and 2t + 1 are key tile t for the two heads.
-  const int U = PAIR ? 2 * n : n;
-  auto tile_of = [&](int u) -> int { return PAIR ? (u >> 1) : u; };
+  const int U = pr ? 2 * n : n;
+  auto tile_of = [&](int u) -> int { return pr ? (u >> 1) : u; };
   // d = 128 fills tensor memory with two score buffers and two output tiles: the probabilities
   // overwrite the scores they come from and a group's next score product has to follow its
   // P.V (one issuing thread does both).  d = 64 leaves room for the probabilities beside the
@@ -275,9 +299,9 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     fence_proxy_async();
     __syncwarp();
     if (lane == 0) {
-      mbar_expect_tx(BAR(BAR_Q), SM::NQ * SZ_TILE);
-#pragma unroll
-      for (uint32_t x = 0; x < SM::NQ; ++x)
+      const uint32_t nq = pr ? 2u : 1u;
+      mbar_expect_tx(BAR(BAR_Q), nq * SZ_TILE);
+      for (uint32_t x = 0; x < nq; ++x)
 #pragma unroll
         for (uint32_t kb = 0; kb < NKB; ++kb)
           tma_load_3d(base + OFF_Q + x * SZ_TILE + kb * SZ_BLK, &tm_q, BAR(BAR_Q), 64 * kb, i0, bh + (int)x);
@@ -368,7 +392,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       auto first_scores = [&](int u) {
         const int t = tile_of(u);
         const uint32_t X = (uint32_t)u & 1u;
-        const uint32_t qsel = PAIR ? X * SZ_TILE : 0u;       // the group's own query tiles
+        const uint32_t qsel = pr ? X * SZ_TILE : 0u;         // the group's own query tiles
         mbar_poll(BAR(BAR_KFULL0 + (uint32_t)t % NKS), (t / NKS) & 1, abort_flag);
         tc_fence_after();
         // query deltas: Q for an exact tile, Q_hat otherwise, against the keys; key deltas: Q
@@ -411,7 +435,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (KEY) mbar_poll(BAR(BAR_KXFULL), n_kx & 1, abort_flag);
           int& n_sx = X ? n_sx1 : n_sx0;
           const uint32_t kx = KEY ? base + OFF_QH : base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE;
-          const uint32_t qx = base + OFF_Q + (PAIR ? X * SZ_TILE : 0u);
+          const uint32_t qx = base + OFF_Q + (pr ? X * SZ_TILE : 0u);
 #pragma unroll
           for (int hf = 0; hf < 2; ++hf) {
             mbar_poll(BAR(BAR_SXREQ0 + X), n_sx & 1, abort_flag);
@@ -428,7 +452,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (KEY) { tc_commit(BAR(BAR_KXFREE)); ++n_kx; }
         }
         // every product that reads this key stage is issued (head pairs: after the second head's)
-        if (!PAIR || X == 1u) tc_commit(BAR(BAR_KFREE0 + (uint32_t)t % NKS));
+        if (!pr || X == 1u) tc_commit(BAR(BAR_KFREE0 + (uint32_t)t % NKS));
         if (ALIAS) {
           // P.V of this tile into the group's output tile, then the group's next scores at once
           mbar_poll(BAR(BAR_VFULL0 + (uint32_t)t % NVS), (t / NVS) & 1, abort_flag);
@@ -465,7 +489,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int ks = 0; ks < BN / 16; ++ks)
           tc_mma_ts(tmem + TMEM_O + (uint32_t)D * X, tmem + TMEM_P64 + 64u * X + 8u * ks,
                     make_desc(vb + ks * 2048, SZ_BLK, 1024), IDESC_PV, (u >= 2 || ks > 0) ? 1u : 0u);
-        if (!PAIR || X == 1u) tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
+        if (!pr || X == 1u) tc_commit(BAR(BAR_VFREE0 + (uint32_t)t % NVS));
         if (u + 2 >= U) tc_commit(BAR(BAR_ODONE0 + X));   // the group's last product
         else tc_commit(BAR(BAR_PFREE0 + X));              // the group may write its next probabilities
       }
@@ -474,8 +498,8 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   } else {
     // =========================== softmax warps: one thread per score row ====================
     const uint32_t X = (uint32_t)warp >> 2;        // group: units u with u & 1 == X
-    const int bh_x = bh + (PAIR ? (int)X : 0);     // the head whose rows this group holds
-    const uint32_t qsel = PAIR ? X * SZ_TILE : 0u; // its query tiles in shared memory
+    const int bh_x = bh + (pr ? (int)X : 0);       // the head whose rows this group holds
+    const uint32_t qsel = pr ? X * SZ_TILE : 0u;   // its query tiles in shared memory
     const int w4 = warp & 3;
     const int row = 32 * w4 + lane;                // tensor-memory lane = row of the tile
     const int i = i0 + row;
@@ -491,10 +515,10 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       // reference after row r is the last fired q[.][c] at or below r) and writes the rows of
       // Q_hat straight into the operand layout, two channels (one 32-bit word) at a time.
       // Blocks are independent of one another.  (head pairs: each group builds its own head's tile)
-      constexpr int NBT = PAIR ? NSW * 16 : NSW * 32;   // threads per tile
-      constexpr int SEG = BM / (NBT / (D / 2));      // rows per thread: 16 or 32
-      constexpr int NBK = SEG / DELTA_CKPT_ROWS;
-      const int tb = PAIR ? (tid & (NBT - 1)) : tid;
+      const int NBT = pr ? NSW * 16 : NSW * 32;      // threads per tile
+      const int SEG = BM / (NBT / (D / 2));          // rows per thread: 16, 32 or 64
+      const int nbk = SEG / DELTA_CKPT_ROWS;
+      const int tb = pr ? (tid & (NBT - 1)) : tid;
       const int c = 2 * (tb % (D / 2)), seg = tb / (D / 2);   // first channel of the pair, segment
       // byte offset of (row rr of an 8-row block, channel c) in a [128][D] tile with 128-byte
       // swizzle, less the block's own offset (8 rows = 1024 bytes, so r & 7 = rr)
@@ -517,7 +541,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       unsigned char* const qm_dst = sm + OFF_QM + 2 * qsel + thr_off;
       const bool check = (i0 + BM > T) || (p.basis_row >= i0 && p.basis_row < i0 + BM);
 #define BUILD(REV, CHECK)                                                                              \
-  build_ref_rows<REV, CHECK, NBK>(q_src, qh_dst, qm_dst, SZ_TILE, offs, ck, D, ref0, p.theta, quarters, seg * SEG, \
+  build_ref_rows<REV, CHECK>(q_src, qh_dst, qm_dst, SZ_TILE, offs, ck, D, ref0, nbk, p.theta, quarters, seg * SEG, \
                                   i0, T, p.basis_row)
       if (p.reverse) { if (check) BUILD(true, true); else BUILD(true, false); }
       else { if (check) BUILD(false, true); else BUILD(false, false); }
@@ -766,7 +790,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (lane == 0) mbar_arrive(BAR(BAR_PRDY0 + X));
     }
 
-    if (PAIR) {
+    if (pr) {
       // ---- head pairs: the group's output tile is the whole result of its head's rows
       mbar_wait(BAR(BAR_ODONE0 + X), 0, abort_flag);
       tc_fence_after();
@@ -855,10 +879,11 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #undef BAR
 }
 
-template <int D, bool KEY, bool PAIR, bool MIXED>
+template <int D, bool KEY, int FORM, bool MIXED>
 static cudaError_t launch_tcq_m(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
-                              void* out, int T, float theta, int init, int window, int shape, bool reverse,
-                              cudaStream_t st) {
+                                void* out, int T, float theta, int init, int window, int shape, bool reverse,
+                                int n_one, cudaStream_t st) {
+  constexpr bool PAIR = FORM != 0;
   const uint64_t BH = (uint64_t)s.B * s.H, BKV = (uint64_t)s.B * s.H_kv;
   const uint64_t ref_heads = KEY ? BKV : BH;   // the reference rows follow the delta stream
   CUtensorMap tq, tqh, tk, tv;
@@ -872,7 +897,7 @@ static cudaError_t launch_tcq_m(const Shape& s, const Workspace& w, const void* 
       encode3(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, v, D, (uint64_t)T, BKV, D * 2, (uint64_t)s.T_max * D * 2, 64,
               128, CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) return cudaErrorInvalidValue;
-  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D, KEY, PAIR, MIXED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t err = cudaFuncSetAttribute(hybrid_attn_tcq_kernel<D, KEY, FORM, MIXED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)TqSmem<D, PAIR>::BYTES);
   if (err != cudaSuccess) return err;
   TqParams p;
@@ -889,7 +914,10 @@ static cudaError_t launch_tcq_m(const Shape& s, const Workspace& w, const void* 
   // delta chain kernel in front is still running; they wait for its results with
   // griddepcontrol.wait.
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(PAIR ? BH / 2 : BH), (unsigned)((T + BM - 1) / BM));
+  const int nqt = (T + BM - 1) / BM;
+  p.BH = (int)BH;
+  p.n_one = (FORM == 2) ? (n_one < nqt ? n_one : nqt) : 0;
+  cfg.gridDim = PAIR ? dim3((unsigned)(BH * p.n_one + BH / 2 * (nqt - p.n_one))) : dim3((unsigned)BH, (unsigned)nqt);
   cfg.blockDim = dim3(NTHR);
   cfg.dynamicSmemBytes = TqSmem<D, PAIR>::BYTES;
   cfg.stream = st;
@@ -898,7 +926,7 @@ static cudaError_t launch_tcq_m(const Shape& s, const Workspace& w, const void* 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  err = cudaLaunchKernelEx(&cfg, hybrid_attn_tcq_kernel<D, KEY, PAIR, MIXED>, tq, tqh, tk, tv, p);
+  err = cudaLaunchKernelEx(&cfg, hybrid_attn_tcq_kernel<D, KEY, FORM, MIXED>, tq, tqh, tk, tv, p);
   count_launch();
   return err != cudaSuccess ? err : cudaGetLastError();
 }
@@ -914,13 +942,13 @@ static bool mixed_tiles_possible(int window, int shape) {
   return !quarters;
 }
 
-template <int D, bool KEY, bool PAIR>
+template <int D, bool KEY, int FORM>
 static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q, const void* k, const void* v,
                               void* out, int T, float theta, int init, int window, int shape, bool reverse,
-                              cudaStream_t st) {
+                              int n_one, cudaStream_t st) {
   return mixed_tiles_possible<D, KEY>(window, shape)
-             ? launch_tcq_m<D, KEY, PAIR, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st)
-             : launch_tcq_m<D, KEY, PAIR, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+             ? launch_tcq_m<D, KEY, FORM, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, n_one, st)
+             : launch_tcq_m<D, KEY, FORM, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, n_one, st);
 }
 
 bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
@@ -942,23 +970,35 @@ cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const voi
                                    int shape, bool key_deltas, bool reverse, int form, cudaStream_t st) {
   if (key_deltas && reverse) return cudaErrorNotSupported;
   if (!w.qhat_rows) return cudaErrorNotSupported;
+  const bool two_heads_ok = s.d == 64 && !key_deltas && (s.g() % 2) == 0;
+  if ((form == 2 || form == 3) && !two_heads_ok) return cudaErrorNotSupported;
   if (s.d == 64) {
-    if (key_deltas && form == 2) return cudaErrorNotSupported;
-    if (key_deltas) return launch_tcq<64, true, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+    if (key_deltas)
+      return launch_tcq<64, true, 0>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st);
     // Two heads of a KV group per CTA share every key and value tile and need no merge, but a
-    // head's key tiles are then walked by one softmax group instead of two: that pays once
-    // there are at least two such CTAs per SM (stack layer 0.925 of the one-head form's
-    // time; a single layer of 1024 tokens 1.13).
-    const long ctas_pair = (long)s.B * s.H / 2 * ((T + BM - 1) / BM);
-    if (form == 2 && (s.g() % 2) != 0) return cudaErrorNotSupported;
-    if (form == 2 || (form == 0 && (s.g() % 2) == 0 && ctas_pair >= 2L * sm_count()))
-      return launch_tcq<64, false, true>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
-    return launch_tcq<64, false, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+    // head's key tiles are then walked by one softmax group instead of two.  That pays once
+    // there are at least two such CTAs per SM (stack layer: 0.925 of the one-head form's time).
+    // On a smaller grid that the one-head form cannot place in one wave, the heaviest query
+    // tiles of every head go one head per CTA and the rest two heads per CTA, as many of the
+    // former as one wave of SMs allows.
+    const long BH = (long)s.B * s.H, nqt = (T + BM - 1) / BM, sms = sm_count();
+    int n_one = -1;                       // -1: the one-head kernel
+    if (form == 2) n_one = 0;
+    else if (form == 3) n_one = 1;
+    else if (form == 0 && two_heads_ok) {
+      if (BH / 2 * nqt >= 2 * sms) n_one = 0;
+      else if (BH * nqt > sms && BH / 2 * nqt <= sms) n_one = (int)((sms - BH / 2 * nqt) / (BH / 2));
+    }
+    if (n_one == 0)
+      return launch_tcq<64, false, 1>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st);
+    if (n_one > 0)
+      return launch_tcq<64, false, 2>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, n_one, st);
+    return launch_tcq<64, false, 0>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st);
   }
-  if (form == 2) return cudaErrorNotSupported;
   if (s.d == 128)
-    return key_deltas ? launch_tcq<128, true, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st)
-                      : launch_tcq<128, false, false>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, st);
+    return key_deltas
+               ? launch_tcq<128, true, 0>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st)
+               : launch_tcq<128, false, 0>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st);
   return cudaErrorNotSupported;
 }
 

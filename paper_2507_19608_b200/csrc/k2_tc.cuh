@@ -16,8 +16,8 @@ bool tcq_kernel_shape(int d);
 // on the tensor cores; w.qhat_rows holds the reference rows of the delta stream.
 // form: 1 = a CTA owns one head's query tile and splits its key tiles between two softmax
 // groups; 2 = a CTA owns the same query tile of two heads of a KV group (query deltas, d = 64,
-// an even number of query heads per KV head; cudaErrorNotSupported otherwise); 0 = form 2
-// where it applies and the grid is large enough for it to pay, else form 1.
+// an even number of query heads per KV head; cudaErrorNotSupported otherwise); 3 = form 2 with
+// the heaviest query tile of every head in form 1; 0 = chosen by the size of the grid.
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
                                    const void* v, void* out, int T, float theta, int init, int window,
                                    int shape, bool key_deltas, bool reverse, int form, cudaStream_t st);

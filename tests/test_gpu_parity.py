@@ -174,7 +174,7 @@ CASES = [
 
 
 @pytest.mark.parametrize("case", CASES, ids=[f"{c[5]}-T{c[3]}-d{c[4]}-W{c[7]}{c[8][0]}-th{c[6]}{'-zs' if len(c) > 9 else ''}" for c in CASES])
-@pytest.mark.parametrize("kernel", [0, 1, 2, 3, 4], ids=["generic", "tc_delta", "tc_telescoped", "tc_telescoped_one_head", "tc_telescoped_two_heads"])
+@pytest.mark.parametrize("kernel", [0, 1, 2, 3, 4, 5], ids=["generic", "tc_delta", "tc_telescoped", "tc_telescoped_one_head", "tc_telescoped_two_heads", "tc_telescoped_both_forms"])
 def test_prefill_output_matches_oracle(B, case, kernel):
     from tests.gpu_helpers import run_prefill, to_host_f64
     Bn, H, Hk, T, d, dtype, theta, W, shape = case[:9]

@@ -36,7 +36,7 @@ def _draw(rng, mode, large):
         shape=str(rng.choice(["block", "sliding"])), theta=float(rng.choice([0.0, 0.05, 0.2, 0.4, 1e9])),
         init=str(rng.choice(["basis_exact", "basis_exact", "zero_state"])) if mode != "key" else "basis_exact",
         steps=int(rng.integers(1, 4)), seed=int(rng.integers(1, 1 << 30)),
-        kernel=int(rng.choice([0, 1, 2, 3, 4])), decode_kernel=int(rng.choice([0, 1])),
+        kernel=int(rng.choice([0, 1, 2, 3, 4, 5])), decode_kernel=int(rng.choice([0, 1])),
         W_d=int(rng.choice([0, 2, 64, 200, 5000])))
 
 
