@@ -71,6 +71,8 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 // K1b: row-parallel finish: delta values, mask words and (key stream) reference rows from the
 // 8-row checkpoints; counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.
+// SMs of the current device (queried once per device).
+int device_sm_count();
 // programmatic: 1 = launched with programmatic stream serialisation (its launch overlaps the end
 // of the kernel in front; the kernel waits for that kernel's completion itself); 2 = the same, but
 // the kernel does not wait: the kernel in front releases it once the chain kernel's results are

@@ -48,11 +48,18 @@ __device__ __forceinline__ bool fires(float x, float x_ref, float theta) {
   return fabsf(__fsub_rn(x, x_ref)) > theta;
 }
 
-// Tight bounded poll of an mbarrier phase (a suspended wait wakes up late, and the hand-overs
-// below are on the chain's path); false once the CTA has given up.
+// Tight bounded poll of an mbarrier phase for the chain warp (a suspended wait wakes up late,
+// and the hand-over is on the chain's path); false once the CTA has given up.
 __device__ __forceinline__ bool poll_ok(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
   if (mbar_test_wait(bar, parity)) return true;
   mbar_poll(bar, parity, abort_flag);
+  return *abort_flag == 0;
+}
+// The helpers' waits: suspended (they run ahead of the chain warp, and where several CTAs share
+// an SM a spinning helper would take issue slots from another CTA's chain warp).
+__device__ __forceinline__ bool wait_ok(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_test_wait(bar, parity)) return true;
+  mbar_wait(bar, parity, abort_flag);
   return *abort_flag == 0;
 }
 
@@ -110,6 +117,9 @@ __global__ void __launch_bounds__(CHAIN_THREADS) delta_chain_kernel(
   // grid-dependency wait
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  // Which of the four compute warps carries the chain rotates with the CTA: where several CTAs
+  // share an SM their chain warps, the busiest, then sit on different schedulers.
+  const int cw = (int)blockIdx.x & 3;
   if (warp == 1 + NHELP) {
     // ---- producer: keeps up to NS stages of rows in flight
     if (lane == 0) {
@@ -122,14 +132,14 @@ __global__ void __launch_bounds__(CHAIN_THREADS) delta_chain_kernel(
         tc::tma_load_3d(raw0 + s * RAW_STAGE_BYTES, &tm_x, full0 + 8 * s, sl * CH, ci * RC, bh);
       }
     }
-  } else if (warp >= 1) {
+  } else if (warp != cw) {
     // ---- helpers: helper hw takes sub-blocks hw, hw + 3, ... of every stage; rows in processing
     // order (reverse: from the stage's last row down), tables in processing order of the sub-blocks
-    const int hw = warp - 1;
+    const int hw = (warp - cw - 1) & 3;      // 0, 1, 2
     int s = 0, zs = 0;
     uint32_t ph_full = 0, ph_zfree = 0;      // parity of the completion waited for next
     for (int i = 0; i < n_chunks; ++i) {
-      if (!poll_ok(full0 + 8 * s, ph_full, abort_flag)) break;
+      if (!wait_ok(full0 + 8 * s, ph_full, abort_flag)) break;
       const TIn* rows = raw + (size_t)s * RC * CH + lane;
       constexpr int NJ = (NSB + NHELP - 1) / NHELP;
       float y[NJ][SBR];        // every load in front of the first store (both are shared memory)
@@ -139,7 +149,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS) delta_chain_kernel(
 #pragma unroll
         for (int k = 0; k < SBR; ++k) y[j][k] = lds_elem<TIn>(rows + (sb * SBR + (reverse ? SBR - 1 - k : k)) * CH);
       }
-      if (i >= NZ && !poll_ok(zfree0 + 8 * zs, ph_zfree, abort_flag)) break;
+      if (i >= NZ && !wait_ok(zfree0 + 8 * zs, ph_zfree, abort_flag)) break;
       float4* zp = zb + (size_t)zs * Z_STAGE + lane;
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
@@ -246,9 +256,8 @@ __global__ void __launch_bounds__(CHAIN_THREADS) delta_chain_kernel(
 }
 
 
-cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
-                               int init, bool key_stream, bool reverse, cudaStream_t st) {
-  if (key_stream && reverse) return cudaErrorNotSupported;
+static cudaError_t launch_delta_chain_tables(const Shape& s, const Workspace& w, const void* q, int T, float theta,
+                                            int dtype, int init, bool key_stream, bool reverse, cudaStream_t st) {
   const int heads = s.B * (key_stream ? s.H_kv : s.H);
   const int src_rows = key_stream ? s.T_max : T;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
@@ -277,6 +286,234 @@ cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q
 #undef LAUNCH
   count_launch();
   return err != cudaSuccess ? err : cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// delta_chain_rows_kernel: the chain row by row, for streams of many heads.  One CTA per (batch,
+// head): D/32 chain warps (thread = channel) + one producer warp that streams the head's rows
+// into a ring of shared-memory stages with bulk copies.  Per row one shared-memory load, one
+// widening, the three dependent operations of Eq. 2-3 and a checkpoint store every 8 rows.  It
+// does 3 times fewer instructions and 10 times less shared-memory traffic per row than the
+// kernel above, whose tables (32 bytes written and read per element) saturate the shared-memory
+// bandwidth of an SM from about two CTAs per SM on: with every head of a large batch resident
+// at once this one is faster (stack layer: 59 us against 82), with few heads the other one
+// (a single Llama layer: 14.3 us against 18.4).
+namespace {
+
+constexpr int RROWS = 64;    // rows per ring stage
+constexpr int RSTAGES = 4;   // ring stages
+
+// One element of the staged rows by shared-memory address, widened to fp32.
+template <typename TIn> __device__ __forceinline__ float lds_row_elem(uint32_t addr);
+template <> __device__ __forceinline__ float lds_row_elem<float>(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+template <> __device__ __forceinline__ float lds_row_elem<__nv_bfloat16>(uint32_t addr) {
+  uint32_t u;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=r"(u) : "r"(addr));
+  return __uint_as_float(u << 16);
+}
+
+// One ring stage of the chain for one thread (= one channel): rows t0 .. t0+nrows-1, the
+// thread's values at rows[r * D]; updates the reference qh and leaves it in front of every
+// 8-row block (ckptp).  basis_row: the stage's first row is the un-thresholded basis.
+template <typename TIn, int D>
+__device__ __forceinline__ void chain_stage(const TIn* rows, int t0, int nrows, bool basis_row, float& qh,
+                                            float theta, float* ckptp, int n_ckpt, unsigned long long* counters) {
+  if (nrows == RROWS && !basis_row) {
+    // full stage, no basis row: nothing but loads, the dependent chain and the checkpoints
+    float x[RROWS];
+    const uint32_t saddr = smem_u32(rows);
+#pragma unroll
+    for (int r = 0; r < RROWS; ++r) x[r] = lds_row_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
+#pragma unroll
+    for (int r = 0; r < RROWS; ++r) {
+      if ((r % DELTA_CKPT_ROWS) == 0 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
+        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      const float diff = __fsub_rn(x[r], qh);      // one IEEE subtraction
+      const bool fire = fabsf(diff) > theta;       // strict; NaN compares false
+      qh = fire ? x[r] : qh;
+    }
+  } else {
+    for (int r = 0; r < nrows; ++r) {
+      if (((t0 + r) % DELTA_CKPT_ROWS) == 0 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
+        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      const float x = to_f32(rows[r * D]);
+      const bool fire = (r == 0 && basis_row) || (fabsf(__fsub_rn(x, qh)) > theta);
+      qh = fire ? x : qh;
+    }
+  }
+}
+
+// Strategy (2): the same stage of the query stream taken from its last row down to its first.
+// The checkpoint of an 8-row block is the reference before the block's highest row.
+// basis_last: the stage's last row is row T-1, the un-thresholded basis of this order.
+template <typename TIn, int D>
+__device__ __forceinline__ void chain_stage_rev(const TIn* rows, int t0, int nrows, bool basis_last, float& qh,
+                                                float theta, float* ckptp, int n_ckpt, unsigned long long* counters) {
+  if (nrows == RROWS && !basis_last) {
+    float x[RROWS];
+    const uint32_t saddr = smem_u32(rows);
+#pragma unroll
+    for (int r = 0; r < RROWS; ++r) x[r] = lds_row_elem<TIn>(saddr + (uint32_t)(r * D * sizeof(TIn)));
+#pragma unroll
+    for (int r = RROWS - 1; r >= 0; --r) {
+      if ((r % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 && DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
+        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      const float diff = __fsub_rn(x[r], qh);
+      const bool fire = fabsf(diff) > theta;
+      qh = fire ? x[r] : qh;
+    }
+  } else {
+    for (int r = nrows - 1; r >= 0; --r) {
+      if ((((t0 + r) % DELTA_CKPT_ROWS) == DELTA_CKPT_ROWS - 1 || r == nrows - 1) &&
+          DELTA_IN((t0 + r) / DELTA_CKPT_ROWS, n_ckpt, counters))
+        ckptp[(size_t)((t0 + r) / DELTA_CKPT_ROWS) * D] = qh;
+      const float x = to_f32(rows[r * D]);
+      const bool fire = (r == nrows - 1 && basis_last) || (fabsf(__fsub_rn(x, qh)) > theta);
+      qh = fire ? x : qh;
+    }
+  }
+}
+
+}  // namespace
+
+template <typename TIn, int D>
+__global__ void __launch_bounds__(D + 32) delta_chain_rows_kernel(
+    const TIn* __restrict__ q, float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
+    float* __restrict__ ckpt, unsigned long long* __restrict__ counters, int T, int n_tiles, int n_ckpt,
+    float theta, int basis_exact, int src_rows, int reverse) {
+  // q: the stream that becomes the delta matrix, [heads][src_rows][D] with rows 0..T-1 read
+  // (queries: src_rows = T; keys in the KV-cache layout: src_rows = T_max)
+  constexpr int NW = D / 32;                       // chain warps
+  constexpr uint32_t ROW_BYTES = D * sizeof(TIn);
+  constexpr uint32_t STAGE_BYTES = RROWS * ROW_BYTES;
+  extern __shared__ __align__(128) unsigned char ring[];   // [RSTAGES][RROWS][D] of TIn
+  __shared__ __align__(8) unsigned long long bars[2 * RSTAGES];   // full[RSTAGES], empty[RSTAGES]
+  __shared__ int s_fail;
+
+  const int bh = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[RSTAGES]);
+  const int n_chunks = (T + RROWS - 1) / RROWS;
+
+  if (tid == 0) {
+    for (int s = 0; s < RSTAGES; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * s), "r"(1) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty0 + 8 * s), "r"(NW) : "memory");
+    }
+    s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  // a kernel launched behind this one with programmatic stream serialisation may become
+  // resident and run its prologue now; it sees this kernel's results only after its own
+  // grid-dependency wait
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  if (warp == NW) {
+    // ---- producer: keeps up to RSTAGES stages of query rows in flight
+    if (lane == 0) {
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(q) + (size_t)bh * src_rows * ROW_BYTES;
+      const uint32_t ring0 = smem_u32(ring);
+      for (int i = 0; i < n_chunks; ++i) {
+        const int s = i % RSTAGES;
+        if (i >= RSTAGES && !mbar_wait(empty0 + 8 * s, ((i / RSTAGES) - 1) & 1)) { s_fail = 1; break; }
+        const int ci = reverse ? n_chunks - 1 - i : i;      // stage of the head in token order
+        const int rows = min(RROWS, T - ci * RROWS);
+        const uint32_t bytes = (uint32_t)rows * ROW_BYTES;
+        // (bounds-checking build: the stage's rows lie inside the head's rows of the stream)
+        if (!DELTA_IN((size_t)ci * RROWS + rows - 1, src_rows, counters)) { s_fail = 1; break; }
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full0 + 8 * s),
+                     "r"(bytes)
+                     : "memory");
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                ring0 + s * STAGE_BYTES),
+            "l"(src + (size_t)ci * STAGE_BYTES), "r"(bytes), "r"(full0 + 8 * s)
+            : "memory");
+      }
+    }
+  } else {
+    // ---- chain warps: thread c owns channel c
+    const int c = tid;
+    float* ckptp = ckpt + (size_t)bh * n_ckpt * D + c;
+    float qh = 0.0f;          // reference state, starts at zero (Eq. 3)
+    bool failed = false;
+    for (int i = 0; i < n_chunks; ++i) {
+      const int s = i % RSTAGES;
+      const int t0 = (reverse ? n_chunks - 1 - i : i) * RROWS;
+      if (qhat_tile && (t0 % DELTA_TILE_ROWS) == 0 && DELTA_IN(t0 / DELTA_TILE_ROWS, n_tiles, counters))
+        qhat_tile[((size_t)bh * n_tiles + t0 / DELTA_TILE_ROWS) * D + c] = qh;
+      if (!mbar_wait(full0 + 8 * s, (i / RSTAGES) & 1)) { failed = true; break; }
+      const TIn* rows = reinterpret_cast<const TIn*>(ring + (size_t)s * STAGE_BYTES) + c;
+      const int nrows = min(RROWS, T - t0);
+      if (reverse)
+        chain_stage_rev<TIn, D>(rows, t0, nrows, t0 + nrows == T && basis_exact, qh, theta, ckptp, n_ckpt, counters);
+      else
+        chain_stage<TIn, D>(rows, t0, nrows, t0 == 0 && basis_exact, qh, theta, ckptp, n_ckpt, counters);
+      __syncwarp();
+      if (lane == 0)
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * s) : "memory");
+    }
+    if (!failed && qhat_out) qhat_out[(size_t)bh * D + c] = qh;
+    if (failed) s_fail = 1;
+  }
+  __syncthreads();
+  if (tid == 0 && s_fail) atomicMax(&counters[CNT_STATUS], (unsigned long long)DELTA_ERR_TIMEOUT);
+}
+
+
+static cudaError_t launch_delta_chain_rows(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
+                               int init, bool key_stream, bool reverse, cudaStream_t st) {
+  if (key_stream && reverse) return cudaErrorNotSupported;
+  const int grid = s.B * (key_stream ? s.H_kv : s.H);
+  const int src_rows = key_stream ? s.T_max : T;
+  const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
+  cudaError_t err = cudaSuccess;
+#define LAUNCH(TIN, DD)                                                                          \
+  do {                                                                                           \
+    auto kern = delta_chain_rows_kernel<TIN, DD>;                                                     \
+    const size_t smem = (size_t)RSTAGES * RROWS * DD * sizeof(TIN);                                      \
+    if (smem > 48 * 1024) {                                                                      \
+      err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+      if (err != cudaSuccess) return err;                                                        \
+    }                                                                                            \
+    kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.qhat_tile, w.qhat[0], w.ckpt, w.counters, T, s.n_tiles, \
+                                      s.n_ckpt(), theta, basis, src_rows, reverse ? 1 : 0);      \
+  } while (0)
+  if (dtype == DELTA_F32) {
+    if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
+  } else {
+    if (s.d == 64) LAUNCH(__nv_bfloat16, 64); else LAUNCH(__nv_bfloat16, 128);
+  }
+#undef LAUNCH
+  count_launch();
+  return err != cudaSuccess ? err : cudaGetLastError();
+}
+
+// SMs of the current device (queried once per device).
+int device_sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (!cached[dev]) {
+    int n = 0;
+    cached[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+  }
+  return cached[dev];
+}
+
+cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
+                               int init, bool key_stream, bool reverse, cudaStream_t st) {
+  if (key_stream && reverse) return cudaErrorNotSupported;
+  // the table kernel while every one of its CTAs (head x 32 channels) has an SM of its own
+  const long ctas = (long)s.B * (key_stream ? s.H_kv : s.H) * (s.d / CH);
+  if (ctas <= device_sm_count())
+    return launch_delta_chain_tables(s, w, q, T, theta, dtype, init, key_stream, reverse, st);
+  return launch_delta_chain_rows(s, w, q, T, theta, dtype, init, key_stream, reverse, st);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -953,18 +953,6 @@ static cudaError_t launch_tcq(const Shape& s, const Workspace& w, const void* q,
 
 bool tcq_kernel_shape(int d) { return d == 64 || d == 128; }
 
-// SMs of the current device (queried once per device).
-static int sm_count() {
-  static int cached[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-  if (!cached[dev]) {
-    int n = 0;
-    cached[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
-  }
-  return cached[dev];
-}
-
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,
                                    const void* v, void* out, int T, float theta, int init, int window,
                                    int shape, bool key_deltas, bool reverse, int form, cudaStream_t st) {
@@ -981,7 +969,7 @@ cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const voi
     // On a smaller grid that the one-head form cannot place in one wave, the heaviest query
     // tiles of every head go one head per CTA and the rest two heads per CTA, as many of the
     // former as one wave of SMs allows.
-    const long BH = (long)s.B * s.H, nqt = (T + BM - 1) / BM, sms = sm_count();
+    const long BH = (long)s.B * s.H, nqt = (T + BM - 1) / BM, sms = device_sm_count();
     int n_one = -1;                       // -1: the one-head kernel
     if (form == 2) n_one = 0;
     else if (form == 3) n_one = 1;

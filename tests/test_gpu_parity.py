@@ -81,6 +81,8 @@ def _check_delta_arrays(B, st, q, theta, init, T):
     (1, 2, 65, 128, "f32", 0.0, "basis_exact"),
     (1, 4, 1000, 64, "bf16", 0.29, "zero_state"),
     (1, 2, 17, 64, "bf16", 1e9, "basis_exact"),
+    (2, 80, 70, 64, "bf16", 0.2, "basis_exact"),       # more heads than SMs: the row-by-row chain kernel
+    (1, 80, 130, 128, "f32", 0.1, "zero_state"),
 ])
 def test_delta_construction_bit_exact(B, Bn, H, T, d, dtype, theta, init):
     from tests.gpu_helpers import run_prefill
@@ -494,6 +496,7 @@ KEY_CASES = [
     (1, 8, 2, 384, 128, 0.25, 128, "block"),
     (1, 2, 1, 130, 64, 0.1, 1000, "block"),        # window covers everything
     (1, 2, 1, 1, 64, 0.1, 4, "block"),
+    (2, 80, 80, 150, 64, 0.2, 64, "block"),        # more KV heads than SMs: the row-by-row chain kernel
 ]
 
 
@@ -626,6 +629,7 @@ BOTTOM_UP_CASES = [
     (1, 8, 2, 384, 128, 0.25, 128, "block", "basis_exact"),
     (1, 2, 1, 1000, 64, 0.29, 64, "block", "zero_state"),
     (1, 2, 1, 1, 64, 0.1, 4, "block", "basis_exact"),
+    (1, 96, 96, 150, 64, 0.2, 64, "block", "basis_exact"),      # more heads than SMs: the row-by-row chain kernel
 ]
 
 
