@@ -296,7 +296,7 @@ DELTA_API int32_t delta_state_sequence_position(const delta_state_t* st, int32_t
  *   2 = tcgen05/TMA kernel, out-of-window scores by the telescoped form of Eq. 4,
  *       R(i)[j] = q_hat(i).k_j, as one more tensor-core product (bf16, d = 64 or 128).
  *       A CTA takes one head's query tile and splits its key tiles between two softmax
- *       groups, or (query deltas at d = 64 with an even number of query heads per KV head)
+ *       groups, or (d = 64 with an even number of query heads per KV head)
  *       the same query tile of two heads of a KV group, so that every key and value tile
  *       is fetched once for both; which CTAs take which form follows the size of the grid;
  *   3 = kernel 2 with every CTA in the one-head form, 4 = every CTA in the two-heads form,

@@ -221,7 +221,7 @@ int32_t delta_state_sequence_position(const delta_state_t* st, int32_t b) {
 static bool tc_eligible(const delta_state* st, int which) {
   if (st->cfg.dtype != DELTA_BF16 || !tc_kernel_available(64)) return false;
   if (st->cfg.source != DELTA_SRC_QUERY && which != 2 && which != 3 && which != 4 && which != 5) return false;
-  if ((which == 4 || which == 5) && (st->cfg.source == DELTA_SRC_KEY || st->cfg.d != 64 || (st->shape.g() % 2) != 0)) return false;
+  if ((which == 4 || which == 5) && (st->cfg.d != 64 || (st->shape.g() % 2) != 0)) return false;
   return which == 1 ? tc_kernel_shape(st->cfg.d) : tcq_kernel_shape(st->cfg.d);
 }
 

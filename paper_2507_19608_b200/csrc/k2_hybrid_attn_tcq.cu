@@ -222,7 +222,6 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   unsigned char* sm = smem_raw + (base - raw);
   constexpr bool PAIR = FORM != 0;       // the layout holds two query tiles
   using SM = TqSmem<D, PAIR>;
-  static_assert(!(KEY && PAIR), "head pairs: query deltas only");
   constexpr uint32_t NKB = SM::NKB, SZ_TILE = SM::SZ_TILE, NKS = SM::NKS, NVS = SM::NVS;
   constexpr uint32_t OFF_Q = SM::OFF_Q, OFF_QH = SM::OFF_QH, OFF_K = SM::OFF_K, OFF_V = SM::OFF_V,
                      OFF_BAR = SM::OFF_BAR, OFF_MISC = SM::OFF_MISC, OFF_QM = SM::OFF_QM;
@@ -432,7 +431,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (MIXED && tile_class(t) == 1) {
           // mixed tile: Q.K^T over each half of 64 keys once the group has that half's
           // telescoped scores in registers
-          if (KEY) mbar_poll(BAR(BAR_KXFULL), n_kx & 1, abort_flag);
+          if (KEY) mbar_poll(BAR(BAR_KXFULL), n_kx & 1, abort_flag);   // (head pairs: the same tile for both heads)
           int& n_sx = X ? n_sx1 : n_sx0;
           const uint32_t kx = KEY ? base + OFF_QH : base + OFF_K + ((uint32_t)t % NKS) * SZ_TILE;
           const uint32_t qx = base + OFF_Q + (pr ? X * SZ_TILE : 0u);
@@ -449,7 +448,7 @@ hybrid_attn_tcq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                      ks > 0 ? 1u : 0u);
             tc_commit(BAR(BAR_SFULL0 + X));
           }
-          if (KEY) { tc_commit(BAR(BAR_KXFREE)); ++n_kx; }
+          if (KEY && (!pr || X == 1u)) { tc_commit(BAR(BAR_KXFREE)); ++n_kx; }
         }
         // every product that reads this key stage is issued (head pairs: after the second head's)
         if (!pr || X == 1u) tc_commit(BAR(BAR_KFREE0 + (uint32_t)t % NKS));
@@ -958,11 +957,9 @@ cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const voi
                                    int shape, bool key_deltas, bool reverse, int form, cudaStream_t st) {
   if (key_deltas && reverse) return cudaErrorNotSupported;
   if (!w.qhat_rows) return cudaErrorNotSupported;
-  const bool two_heads_ok = s.d == 64 && !key_deltas && (s.g() % 2) == 0;
+  const bool two_heads_ok = s.d == 64 && (s.g() % 2) == 0;
   if ((form == 2 || form == 3) && !two_heads_ok) return cudaErrorNotSupported;
   if (s.d == 64) {
-    if (key_deltas)
-      return launch_tcq<64, true, 0>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st);
     // Two heads of a KV group per CTA share every key and value tile and need no merge, but a
     // head's key tiles are then walked by one softmax group instead of two.  That pays once
     // there are at least two such CTAs per SM (stack layer: 0.925 of the one-head form's time).
@@ -976,6 +973,13 @@ cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const voi
     else if (form == 0 && two_heads_ok) {
       if (BH / 2 * nqt >= 2 * sms) n_one = 0;
       else if (BH * nqt > sms && BH / 2 * nqt <= sms) n_one = (int)((sms - BH / 2 * nqt) / (BH / 2));
+    }
+    if (key_deltas) {
+      if (n_one == 0)
+        return launch_tcq<64, true, 1>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st);
+      if (n_one > 0)
+        return launch_tcq<64, true, 2>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, n_one, st);
+      return launch_tcq<64, true, 0>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st);
     }
     if (n_one == 0)
       return launch_tcq<64, false, 1>(s, w, q, k, v, out, T, theta, init, window, shape, reverse, 0, st);

@@ -15,7 +15,7 @@ bool tcq_kernel_shape(int d);
 // Telescoped variant: out-of-window scores as Q_hat.K^T (query deltas) or Q.K_hat^T (key deltas)
 // on the tensor cores; w.qhat_rows holds the reference rows of the delta stream.
 // form: 1 = a CTA owns one head's query tile and splits its key tiles between two softmax
-// groups; 2 = a CTA owns the same query tile of two heads of a KV group (query deltas, d = 64,
+// groups; 2 = a CTA owns the same query tile of two heads of a KV group (d = 64,
 // an even number of query heads per KV head; cudaErrorNotSupported otherwise); 3 = form 2 with
 // the heaviest query tile of every head in form 1; 0 = chosen by the size of the grid.
 cudaError_t launch_hybrid_attn_tcq(const Shape& s, const Workspace& w, const void* q, const void* k,

@@ -501,14 +501,21 @@ KEY_CASES = [
 
 
 @pytest.mark.parametrize("case", KEY_CASES, ids=[f"T{c[3]}-d{c[4]}-W{c[6]}{c[7][0]}" for c in KEY_CASES])
-def test_key_delta_prefill_matches_oracle(B, case):
-    """Strategy (3): the key stream of every KV head becomes the delta matrix."""
+@pytest.mark.parametrize("form", [2, 3, 4, 5], ids=["auto", "one_head", "two_heads", "both_forms"])
+def test_key_delta_prefill_matches_oracle(B, case, form):
+    """Strategy (3): the key stream of every KV head becomes the delta matrix (every form of the
+    attention kernel's grid that the configuration has)."""
     from tests.gpu_helpers import to_cache, to_dev, to_host_f64
     Bn, H, Hk, T, d, theta, W, shape = case
     q, k, v = _inputs(Bn, H, Hk, T, d, "bf16", seed=300 + T + d)
     cfg = B.make_config(Bn, H, Hk, d, T, "bf16", source=B.DELTA_SRC_KEY,
                         prefill_window=B.DELTA_WIN_BLOCK if shape == "block" else B.DELTA_WIN_SLIDING)
     st = B.delta_state_init(cfg)
+    try:
+        B.delta_state_set_prefill_kernel(st, form)
+    except B.DeltaError as e:
+        assert e.status == B.DELTA_ERR_UNSUPPORTED and form in (4, 5)
+        pytest.skip("no two-head form for this configuration")
     dq_, kc, vc = to_dev(q, "bf16"), to_cache(k, T, "bf16"), to_cache(v, T, "bf16")
     out = torch.full_like(dq_, float("nan"))
     B.delta_attn_prefill(st, dq_, kc, vc, out, T, H, Hk, d, float(theta), int(W))
