@@ -117,8 +117,10 @@ DELTA_API delta_status_t delta_state_workspace_bytes(const delta_config_t* cfg, 
 DELTA_API delta_status_t delta_state_init(const delta_config_t* cfg, void* workspace, size_t workspace_bytes,
                                 void* stream, delta_state_t** out);
 
-/* Back to the freshly initialised condition (position 0, reference 0, counters 0): the same
- * one small memset on `stream`. */
+/* Back to the freshly initialised condition (position 0, reference 0, counters 0).  Host-side
+ * only: the clearing of the device span is done by the first kernel of the next prefill on this
+ * state, on that call's stream (`stream` is unused); delta_sparsity_stats reports zeros in
+ * between, delta_state_view still shows the old contents until that prefill. */
 DELTA_API delta_status_t delta_state_reset(delta_state_t* st, void* stream);
 
 /* Frees the host object only. */

@@ -51,6 +51,9 @@ struct delta_state {
   bool key_cache_packed = false;   // key deltas: decode from the compressed key-delta cache
   // optional per-kernel timing of prefill (host-side event objects)
   bool profiling = false, profiled = false;
+  // a reset has been asked for and the chain kernel of the next prefill does the clearing (no
+  // launch of its own: a memset in front of the chain kernel costs 2 us of a 38 us step)
+  bool zero_pending = false;
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
 };
 
@@ -136,10 +139,16 @@ delta_status_t delta_state_workspace_bytes(const delta_config_t* cfg, size_t* by
   return DELTA_OK;
 }
 
-static delta_status_t zero_state(delta_state* st, cudaStream_t stream) {
-  // one memset: the span carve() put at the front of the workspace
-  cudaError_t e = cudaMemsetAsync(st->base, 0, st->ws.zero_bytes, stream);
-  if (e != cudaSuccess) return cuda_fail(e);
+// defer: leave the clearing of the device span to the next prefill (see zero_pending)
+static delta_status_t zero_state(delta_state* st, cudaStream_t stream, bool defer) {
+  if (defer) {
+    st->zero_pending = true;
+  } else {
+    // one memset: the span carve() put at the front of the workspace
+    cudaError_t e = cudaMemsetAsync(st->base, 0, st->ws.zero_bytes, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    st->zero_pending = false;
+  }
   st->n = 0;
   st->n_b.assign((size_t)st->cfg.B, 0);
   st->ragged = false;
@@ -168,7 +177,7 @@ delta_status_t delta_state_init(const delta_config_t* cfg, void* workspace, size
   st->base = workspace;
   st->bytes = workspace_bytes;
   st->forced_kernel = -1;
-  s = zero_state(st, (cudaStream_t)stream);
+  s = zero_state(st, (cudaStream_t)stream, /*defer=*/false);
   if (s != DELTA_OK) { delete st; return s; }
   *out = st;
   return DELTA_OK;
@@ -176,7 +185,7 @@ delta_status_t delta_state_init(const delta_config_t* cfg, void* workspace, size
 
 delta_status_t delta_state_reset(delta_state_t* st, void* stream) {
   if (!st) return DELTA_ERR_INVALID_ARG;
-  return zero_state(st, (cudaStream_t)stream);
+  return zero_state(st, (cudaStream_t)stream, /*defer=*/true);
 }
 
 delta_status_t delta_state_destroy(delta_state_t* st) {
@@ -340,6 +349,16 @@ static delta_status_t prefill_launch(delta_state* st, const Shape& shape, const 
                                      int32_t window, cudaStream_t cs, bool prof) {
   const delta_config_t& c = st->cfg;
   cudaError_t e;
+  // a pending reset: the chain kernel clears the span, less the front of qhat[0] that the chain
+  // kernels of this prefill fill themselves (one reference per head of the delta stream)
+  void* zero_ptr = nullptr;
+  size_t zero_bytes = 0;
+  if (st->zero_pending) {
+    const size_t skip = (size_t)c.B * (c.source == DELTA_SRC_KEY ? c.H_kv : c.H) * c.d * sizeof(float);
+    zero_ptr = (char*)st->base + skip;
+    zero_bytes = st->ws.zero_bytes - skip;
+    st->zero_pending = false;
+  }
 #define MARK(i) do { if (prof && (e = cudaEventRecord(st->ev[i], cs)) != cudaSuccess) return cuda_fail(e); } while (0)
   const int which = delta_state_prefill_kernel(st);
   const bool use_tc = which == 1;
@@ -356,7 +375,7 @@ static delta_status_t prefill_launch(delta_state* st, const Shape& shape, const 
   const bool chained = tcq && !prof;
   MARK(0);
   // the delta stream: the queries (strategy 1) or the keys, per KV head (strategy 3)
-  if ((e = launch_delta_chain(shape, ws, key ? k : q, T, theta, c.dtype, c.init, key, rev, cs)) != cudaSuccess)
+  if ((e = launch_delta_chain(shape, ws, key ? k : q, T, theta, c.dtype, c.init, key, rev, zero_ptr, zero_bytes, cs)) != cudaSuccess)
     return cuda_fail(e);
   auto attention = [&]() -> cudaError_t {
     if (use_tc) return launch_hybrid_attn_tc(shape, ws, q, k, v, out, T, window, c.prefill_window, cs);
@@ -603,11 +622,13 @@ static void finish_stage(delta_stage_stats_t* o, const unsigned long long* c, do
 delta_status_t delta_sparsity_stats(const delta_state_t* st, delta_stats_t* host_out, void* stream) {
   NvtxRange range("delta_sparsity_stats");
   if (!st || !host_out) return DELTA_ERR_INVALID_ARG;
-  unsigned long long c[CNT_TOTAL];
-  cudaError_t e = cudaMemcpyAsync(c, st->ws.counters, sizeof(c), cudaMemcpyDeviceToHost,
-                                  (cudaStream_t)stream);
-  if (e != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaStreamSynchronize((cudaStream_t)stream)) != cudaSuccess) return cuda_fail(e);
+  unsigned long long c[CNT_TOTAL] = {};
+  if (!st->zero_pending) {      // (after a reset the counters are zero, whatever the device still holds)
+    cudaError_t e = cudaMemcpyAsync(c, st->ws.counters, sizeof(c), cudaMemcpyDeviceToHost,
+                                    (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamSynchronize((cudaStream_t)stream)) != cudaSuccess) return cuda_fail(e);
+  }
   memset(host_out, 0, sizeof(*host_out));
   for (int sh = 0; sh < CNT_SHARDS; ++sh)          // prefill counters are sharded on the device
     for (int i = 0; i < 4; ++i) c[CNT_PREFILL_NNZ + i] += c[CNT_SHARD_BASE + 4 * sh + i];

@@ -66,8 +66,11 @@ delta_status_t cuda_fail(cudaError_t e);
 // every 64-row tile, and the final reference.
 // key_stream: the stream is K in the KV-cache layout, one chain set per KV head (strategy 3).
 // reverse: rows are taken from T-1 down to 0 (strategy 2; query stream only).
+// zero_ptr, zero_bytes: a span (16-byte aligned, a multiple of 16 bytes) that the kernel's first
+// CTA clears before anything else: the deferred clearing of a state reset (none if null).
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
-                               int init, bool key_stream, bool reverse, cudaStream_t st);
+                               int init, bool key_stream, bool reverse, void* zero_ptr, size_t zero_bytes,
+                               cudaStream_t st);
 // K1b: row-parallel finish: delta values, mask words and (key stream) reference rows from the
 // 8-row checkpoints; counts, compacted indices, Eq. 6 counters, the decode hand-off row
 // R(T-1)[j] = q_hat . k_j and (want_kt) the channel-major fp32 key copy.

@@ -85,7 +85,7 @@ template <typename TIn, int D>
 __global__ void __launch_bounds__(CHAIN_THREADS) delta_chain_kernel(
     const __grid_constant__ CUtensorMap tm_x, float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
     float* __restrict__ ckpt, unsigned long long* __restrict__ counters, int T, int n_tiles, int n_ckpt,
-    float theta, int basis_exact, int reverse) {
+    float theta, int basis_exact, int reverse, uint4* zero_ptr, unsigned zero_n16) {
   // tm_x: the stream that becomes the delta matrix as [heads][rows 0..T-1][D]; box = [64 rows][32 channels]
   constexpr int NSL = D / CH;                      // channel slices (CTAs) per head
   constexpr uint32_t RAW_STAGE_BYTES = RC * CH * sizeof(TIn);
@@ -101,6 +101,10 @@ __global__ void __launch_bounds__(CHAIN_THREADS) delta_chain_kernel(
   const uint32_t zfull0 = smem_u32(&bars[2 * NS]), zfree0 = smem_u32(&bars[2 * NS + NZ]);
   volatile uint32_t* abort_flag = &s_abort;
   const int n_chunks = (T + RC - 1) / RC;
+  // the deferred clearing of a state reset (counters, tickets, second reference buffer): nothing
+  // of this launch or of the kernels behind it touches that span before this kernel is complete
+  if (zero_ptr && blockIdx.x == 0)
+    for (unsigned i = tid; i < zero_n16; i += blockDim.x) zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
 
   if (tid < 2 * NS + 2 * NZ) {      // one barrier per thread
     const uint32_t cnt = (tid < NS) ? 1u : (tid < 2 * NS) ? (uint32_t)NHELP : (tid < 2 * NS + NZ) ? (uint32_t)NHELP : 1u;
@@ -257,7 +261,8 @@ __global__ void __launch_bounds__(CHAIN_THREADS) delta_chain_kernel(
 
 
 static cudaError_t launch_delta_chain_tables(const Shape& s, const Workspace& w, const void* q, int T, float theta,
-                                            int dtype, int init, bool key_stream, bool reverse, cudaStream_t st) {
+                                            int dtype, int init, bool key_stream, bool reverse, void* zero_ptr,
+                                            size_t zero_bytes, cudaStream_t st) {
   const int heads = s.B * (key_stream ? s.H_kv : s.H);
   const int src_rows = key_stream ? s.T_max : T;
   const int basis = (init == DELTA_INIT_BASIS_EXACT) ? 1 : 0;
@@ -276,7 +281,8 @@ static cudaError_t launch_delta_chain_tables(const Shape& s, const Workspace& w,
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
     if (err != cudaSuccess) return err;                                                          \
     kern<<<heads * (DD / CH), CHAIN_THREADS, smem, st>>>(tm, w.qhat_tile, w.qhat[0], w.ckpt, w.counters, T, \
-                                                         s.n_tiles, s.n_ckpt(), theta, basis, reverse ? 1 : 0); \
+                                                         s.n_tiles, s.n_ckpt(), theta, basis, reverse ? 1 : 0, \
+                                                         (uint4*)zero_ptr, (unsigned)(zero_bytes / 16)); \
   } while (0)
   if (f32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
@@ -384,7 +390,7 @@ template <typename TIn, int D>
 __global__ void __launch_bounds__(D + 32) delta_chain_rows_kernel(
     const TIn* __restrict__ q, float* __restrict__ qhat_tile, float* __restrict__ qhat_out,
     float* __restrict__ ckpt, unsigned long long* __restrict__ counters, int T, int n_tiles, int n_ckpt,
-    float theta, int basis_exact, int src_rows, int reverse) {
+    float theta, int basis_exact, int src_rows, int reverse, uint4* zero_ptr, unsigned zero_n16) {
   // q: the stream that becomes the delta matrix, [heads][src_rows][D] with rows 0..T-1 read
   // (queries: src_rows = T; keys in the KV-cache layout: src_rows = T_max)
   constexpr int NW = D / 32;                       // chain warps
@@ -398,6 +404,9 @@ __global__ void __launch_bounds__(D + 32) delta_chain_rows_kernel(
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[RSTAGES]);
   const int n_chunks = (T + RROWS - 1) / RROWS;
+  // the deferred clearing of a state reset (see the table kernel)
+  if (zero_ptr && blockIdx.x == 0)
+    for (unsigned i = tid; i < zero_n16; i += blockDim.x) zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
 
   if (tid == 0) {
     for (int s = 0; s < RSTAGES; ++s) {
@@ -466,8 +475,9 @@ __global__ void __launch_bounds__(D + 32) delta_chain_rows_kernel(
 }
 
 
-static cudaError_t launch_delta_chain_rows(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
-                               int init, bool key_stream, bool reverse, cudaStream_t st) {
+static cudaError_t launch_delta_chain_rows(const Shape& s, const Workspace& w, const void* q, int T, float theta,
+                                          int dtype, int init, bool key_stream, bool reverse, void* zero_ptr,
+                                          size_t zero_bytes, cudaStream_t st) {
   if (key_stream && reverse) return cudaErrorNotSupported;
   const int grid = s.B * (key_stream ? s.H_kv : s.H);
   const int src_rows = key_stream ? s.T_max : T;
@@ -482,7 +492,8 @@ static cudaError_t launch_delta_chain_rows(const Shape& s, const Workspace& w, c
       if (err != cudaSuccess) return err;                                                        \
     }                                                                                            \
     kern<<<grid, DD + 32, smem, st>>>((const TIN*)q, w.qhat_tile, w.qhat[0], w.ckpt, w.counters, T, s.n_tiles, \
-                                      s.n_ckpt(), theta, basis, src_rows, reverse ? 1 : 0);      \
+                                      s.n_ckpt(), theta, basis, src_rows, reverse ? 1 : 0,       \
+                                      (uint4*)zero_ptr, (unsigned)(zero_bytes / 16));            \
   } while (0)
   if (dtype == DELTA_F32) {
     if (s.d == 64) LAUNCH(float, 64); else LAUNCH(float, 128);
@@ -507,13 +518,15 @@ int device_sm_count() {
 }
 
 cudaError_t launch_delta_chain(const Shape& s, const Workspace& w, const void* q, int T, float theta, int dtype,
-                               int init, bool key_stream, bool reverse, cudaStream_t st) {
+                               int init, bool key_stream, bool reverse, void* zero_ptr, size_t zero_bytes,
+                               cudaStream_t st) {
   if (key_stream && reverse) return cudaErrorNotSupported;
+  if (((uintptr_t)zero_ptr | zero_bytes) & 15u) return cudaErrorInvalidValue;
   // the table kernel while every one of its CTAs (head x 32 channels) has an SM of its own
   const long ctas = (long)s.B * (key_stream ? s.H_kv : s.H) * (s.d / CH);
   if (ctas <= device_sm_count())
-    return launch_delta_chain_tables(s, w, q, T, theta, dtype, init, key_stream, reverse, st);
-  return launch_delta_chain_rows(s, w, q, T, theta, dtype, init, key_stream, reverse, st);
+    return launch_delta_chain_tables(s, w, q, T, theta, dtype, init, key_stream, reverse, zero_ptr, zero_bytes, st);
+  return launch_delta_chain_rows(s, w, q, T, theta, dtype, init, key_stream, reverse, zero_ptr, zero_bytes, st);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -328,6 +328,13 @@ def test_device_status_word_reaches_the_host(B):
     assert e.value.status == B.DELTA_ERR_TIMEOUT
     B.delta_state_reset(st)
     assert B.delta_sparsity_stats(st)["device_status"] == 0
+    # the word itself is cleared by the next prefill
+    from tests.gpu_helpers import to_cache, to_dev
+    o2 = torch.empty_like(out)
+    B.delta_attn_prefill(st, to_dev(q, "bf16"), to_cache(k, 40, "bf16"), to_cache(v, 40, "bf16"), o2, 40, 2, 1, 64, 0.1, 8)
+    torch.cuda.synchronize()
+    assert int(B.delta_state_view(st, B.DELTA_VIEW_COUNTERS)[8].item()) == 0
+    assert B.delta_sparsity_stats(st)["device_status"] == 0 and torch.equal(o2, out)
 
 
 # ------------------------------------------------------------------ call-order and capacity errors
@@ -335,6 +342,7 @@ def test_state_errors(B):
     from tests.gpu_helpers import run_prefill, to_dev
     q, k, v = _inputs(1, 2, 1, 32, 64, "bf16", seed=1)
     st, out, kc, vc = run_prefill(B, q, k, v, 0.1, 4, "bf16", T_max=33)
+    first = B.delta_sparsity_stats(st)["prefill"]
     with pytest.raises(B.DeltaError) as e:
         B.delta_attn_prefill(st, out, kc, vc, out, 32, 2, 1, 64, 0.1, 4)
     assert e.value.status == B.DELTA_ERR_STATE
@@ -362,6 +370,9 @@ def test_state_errors(B):
     B.delta_attn_prefill(st, td(q, "bf16"), kc, vc, out2, 32, 2, 1, 64, 0.1, 4)
     torch.cuda.synchronize()
     assert torch.equal(out2, out)
+    # ... with counters that started from zero again (the reset's clearing is done by the prefill)
+    again = B.delta_sparsity_stats(st)
+    assert again["prefill"] == first and again["decode"]["macs_dense"] == 0 and again["device_status"] == 0
     assert B.delta_launch_count() > 0
 
 
