@@ -860,7 +860,7 @@ def run_cpu_baseline(args, w, tens, theta):
 
 
 def run_config_leg(args, B, torch, name, thetas, flush, peaks, n_sm, iters=10):
-    """One BASELINE configuration that is not the headline: step time (reset + prefill, L2
+    """One of the named workloads besides the headline: step time (reset + prefill, L2
     flushed), tokens/s, per-kernel times and the hybrid-attention roofline, per theta."""
     w = WL.WORKLOADS[name]
     tens = WL.make_qkv(w, n_decode=0)
